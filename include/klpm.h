@@ -1,0 +1,143 @@
+/*
+ * klpm.h -- C ABI of the device-resident k-LPM scheduling path (sm_100a).
+ *
+ * The library keeps a flattened radix tree of cached prompts in device memory and runs, on the GPU,
+ * batched longest-prefix matching, the k-LPM / FCFS / LPM selection rule and the schedule replay
+ * under the paper's prefix-reuse cost model.
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise:
+ *   - `d_*` arguments are DEVICE pointers owned by the caller (4-byte aligned for int32 data,
+ *     8-byte aligned for int64 data).  The library never frees them and does not keep them after
+ *     the work enqueued by the call has completed.  A pointer documented "nullable" may be NULL.
+ *   - prompts are int32 token strings in CSR form: prompt i is tokens[offsets[i] .. offsets[i+1]);
+ *     offsets are int64, non-decreasing, offsets[0] may be non-zero.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is enqueued on it;
+ *     entry points return without waiting for the device, except where stated.
+ *   - the return value reports argument and launch errors found on the host.  Conditions found on the
+ *     device (capacity exhausted, budget too small, a bounded wait that ran out) are recorded in a
+ *     status word inside the tree and returned by rt_sync_status(); nothing traps or aborts.
+ *   - a tree may be used from one stream at a time; calls on one tree must not overlap on the GPU.
+ *   - all arithmetic is integer; there is no floating point on this path.
+ */
+#ifndef KLPM_H_
+#define KLPM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t rt_status;
+enum {
+    RT_OK = 0,
+    RT_ERR_INVALID = -1,   /* bad argument (null pointer, negative count, k < 1, ...) */
+    RT_ERR_CAPACITY = -2,  /* node, token-pool or clock capacity of the tree exhausted */
+    RT_ERR_BUDGET = -3,    /* the KV budget cannot hold a prompt even after evicting everything evictable */
+    RT_ERR_LIMIT = -4,     /* a bounded device-side wait or probe loop ran out */
+    RT_ERR_CUDA = -5       /* a CUDA runtime call failed */
+};
+
+enum { KLPM_POLICY_FCFS = 0, KLPM_POLICY_LPM = 1, KLPM_POLICY_KLPM = 2 };
+
+typedef struct rt_tree rt_tree; /* opaque; owned by the library from rt_build/rt_create until rt_destroy */
+
+typedef struct {
+    int32_t vocab;            /* informational: token ids are expected in [0, vocab) */
+    int64_t max_nodes;        /* capacity in tree nodes (every processed prompt adds at most 2) */
+    int64_t max_pool_tokens;  /* capacity of the append-only int32 token pool */
+    int64_t budget_tokens;    /* KV-cache budget in tokens with LRU eviction; 0 = unbounded */
+    int64_t max_clock;        /* capacity in processed prompts over the tree's life; 0 = max_nodes */
+} rt_config;
+
+typedef struct {
+    int32_t policy;      /* KLPM_POLICY_* ; LPM = every pick is a longest-match pick */
+    int32_t k;           /* Algorithm 1's k (>= 1); used by KLPM only */
+    int64_t c_num;       /* c_attn = c_num / c_den (Definition 2); times are in units of 1/c_den tick */
+    int64_t c_den;       /* >= 1 */
+    int64_t start_tick;  /* tick at which processing starts (R of the "previous" query for the first pick) */
+} klpm_params;
+
+/* ---- radix tree of cached prompts (RadixAttention, Section 1: "stores the KV cache of processed
+ *      queries ... by maintaining a radix tree", "least recently used (LRU) eviction") ---- */
+
+/* Create an empty tree.  Synchronous (allocates device memory). */
+rt_status rt_create(const rt_config* cfg, rt_tree** out);
+
+/* Create a tree and store n_prompts prompts in it, as if processed one after the other in index
+ * order (prompt i is stamped with logical clock i+1 for LRU).  Equivalent to rt_create + rt_insert. */
+rt_status rt_build(const int32_t* d_tokens, const int64_t* d_offsets, int32_t n_prompts,
+                   const rt_config* cfg, void* stream, rt_tree** out);
+
+/* Store n more prompts, one after the other in index order: each is matched against the tree as it
+ * stands, a node boundary is put at its match end, its uncached tail is appended as a new leaf, the
+ * logical clock advances by one, and (with a budget) least-recently-used leaves are evicted first to
+ * make room.  d_new_tokens (nullable, int32[n]) receives |x_i| - match length at its own insertion.
+ * If the device runs out of capacity the prompts before the failing one stay inserted and the tree
+ * stays valid; the condition is reported by rt_sync_status. */
+rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n,
+                    int32_t* d_new_tokens, void* stream);
+
+/* Batched longest-prefix match (Section 1.3: overlap(x, y); RadixAttention "matches them with new
+ * incoming prompts"): d_match_len[i] = max over cached prompts y of overlap(q_i, y) = the longest
+ * prefix of query i that lies on a root path of the tree, counted token by token (partial edges
+ * count).  Read-only on the tree.  d_term_node / d_term_off (nullable, int32[nq]) receive where the
+ * match ended: the node whose edge holds the last matched token (0 = root when nothing matched) and
+ * how many tokens of that edge matched. */
+rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
+                         int32_t nq, int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off,
+                         void* stream);
+
+/* Counters of the tree (synchronises the stream the tree was last used on).  Any pointer may be NULL.
+ * n_nodes: live nodes, root excluded; n_tokens: tokens held by live nodes; clock: prompts processed;
+ * evictions: leaves evicted so far; pool_used: tokens appended to the pool so far. */
+rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* clock,
+                   int64_t* evictions, int64_t* pool_used);
+
+/* Wait for `stream` and return the tree's device-side status word (RT_OK or the first error recorded). */
+rt_status rt_sync_status(rt_tree* tree, void* stream);
+
+/* Free the tree and everything it owns.  Synchronous. */
+rt_status rt_destroy(rt_tree* tree);
+
+/* ---- scheduling (Algorithm 1 "k-LPM"; FCFS and LPM of Section 1 as its k = 1 and k = infinity limits) ---- */
+
+/* One scheduling decision as a pure function of its inputs.  Among the queries with d_waiting[i] != 0:
+ *   - oldest-first pick (FCFS; or KLPM when pick_counter % k == 0): the query with the smallest
+ *     (arrival, index);
+ *   - longest-match pick (LPM; or KLPM otherwise): the query with the largest d_match_len, ties to the
+ *     smallest (arrival, index).
+ * d_pick (int32[1]) receives the index, or -1 if no query is waiting.  Uses library-owned scratch that
+ * is allocated on the first call on each device. */
+rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting,
+                      int32_t nq, int64_t pick_counter, const klpm_params* params, int32_t* d_pick,
+                      void* stream);
+
+/* Definition 2 along a given processing order: for j = d_order[0], d_order[1], ...:
+ *   m = longest prefix of x_j in the tree; uncached = |x_j| - m;
+ *   R_j = max(R_prev, t_j) + (c_den + c_num |x_j|) * uncached;  TTFT_j = R_j - t_j;
+ * then x_j is stored in the tree (as rt_insert does).  Outputs are indexed by query: d_uncached
+ * (int32[n_queries]), d_ttft (int64[n_queries]), d_completion (nullable, int64[n_queries]); entries of
+ * queries that are not in d_order are left untouched. */
+rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, const int32_t* d_q_tokens,
+                      const int64_t* d_q_offsets, const int64_t* d_arrival, int32_t n_queries,
+                      const klpm_params* params, int32_t* d_uncached, int64_t* d_ttft,
+                      int64_t* d_completion, void* stream);
+
+/* The whole scheduling loop on the device (Algorithm 1 with Definitions 1 and 2): until all n queries
+ * are processed -- wait for the next arrival if nobody is waiting; pick by the policy among the queries
+ * that have arrived (match lengths are those against the tree at that moment, which includes every
+ * query processed so far); charge the pick by Definition 2; store it in the tree (LRU eviction under
+ * the budget).  d_order[c] (int32[n]) = query processed at decision c; the other outputs are as in
+ * klpm_replay.  The pick counter of KLPM never resets. */
+rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
+                   const int64_t* d_arrival, int32_t n, const klpm_params* params, int32_t* d_order,
+                   int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
+
+/* Version of the ABI (bumped when a signature changes). */
+int32_t klpm_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KLPM_H_ */

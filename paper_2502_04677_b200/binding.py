@@ -1,0 +1,194 @@
+"""ctypes binding of libklpm.so: argument marshalling only.
+
+Same names as the C ABI (include/klpm.h).  Tensors must live on the CUDA device; every step of the
+path runs in the library's kernels.  There is no CPU fallback: importing this module fails if the
+library has not been built, and every call fails on a non-CUDA tensor.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libklpm.so")
+
+RT_OK, RT_ERR_INVALID, RT_ERR_CAPACITY, RT_ERR_BUDGET, RT_ERR_LIMIT, RT_ERR_CUDA = 0, -1, -2, -3, -4, -5
+POLICY_FCFS, POLICY_LPM, POLICY_KLPM = 0, 1, 2
+_ERR = {-1: "RT_ERR_INVALID", -2: "RT_ERR_CAPACITY", -3: "RT_ERR_BUDGET", -4: "RT_ERR_LIMIT", -5: "RT_ERR_CUDA"}
+
+
+class KlpmError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__("%s returned %s (%d)" % (where, _ERR.get(code, "?"), code))
+        self.code = code
+
+
+class rt_config(ctypes.Structure):
+    _fields_ = [("vocab", ctypes.c_int32), ("max_nodes", ctypes.c_int64), ("max_pool_tokens", ctypes.c_int64),
+                ("budget_tokens", ctypes.c_int64), ("max_clock", ctypes.c_int64)]
+
+
+class klpm_params(ctypes.Structure):
+    _fields_ = [("policy", ctypes.c_int32), ("k", ctypes.c_int32), ("c_num", ctypes.c_int64),
+                ("c_den", ctypes.c_int64), ("start_tick", ctypes.c_int64)]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError("libklpm.so is not built: run `python -m paper_2502_04677_b200.build` "
+                      "(there is no CPU fallback for this library)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+_vp, _i32, _i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+
+_lib.klpm_abi_version.restype = _i32
+_lib.rt_create.restype = _i32
+_lib.rt_create.argtypes = [ctypes.POINTER(rt_config), ctypes.POINTER(_vp)]
+_lib.rt_build.restype = _i32
+_lib.rt_build.argtypes = [_vp, _vp, _i32, ctypes.POINTER(rt_config), _vp, ctypes.POINTER(_vp)]
+_lib.rt_insert.restype = _i32
+_lib.rt_insert.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp]
+_lib.rt_match_batch.restype = _i32
+_lib.rt_match_batch.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
+_lib.rt_stats.restype = _i32
+_lib.rt_stats.argtypes = [_vp] + [ctypes.POINTER(_i64)] * 5
+_lib.rt_sync_status.restype = _i32
+_lib.rt_sync_status.argtypes = [_vp, _vp]
+_lib.rt_destroy.restype = _i32
+_lib.rt_destroy.argtypes = [_vp]
+_lib.klpm_select.restype = _i32
+_lib.klpm_select.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
+_lib.klpm_replay.restype = _i32
+_lib.klpm_replay.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp]
+_lib.klpm_run.restype = _i32
+_lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
+
+EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
+           "rt_sync_status", "rt_destroy", "klpm_select", "klpm_replay", "klpm_run"]
+
+
+def lib() -> ctypes.CDLL:
+    return _lib
+
+
+def _dev(t: Optional[torch.Tensor], dtype, name: str, nullable: bool = False):
+    if t is None:
+        if nullable:
+            return None
+        raise ValueError("%s must not be None" % name)
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (this library has no CPU path)" % name)
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous %s tensor" % (name, dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, where: str) -> None:
+    if code != RT_OK:
+        raise KlpmError(code, where)
+
+
+def make_params(policy: int, k: int = 1, c_num: int = 0, c_den: int = 1, start_tick: int = 0) -> klpm_params:
+    return klpm_params(int(policy), int(k), int(c_num), int(c_den), int(start_tick))
+
+
+class Tree:
+    """Handle of a device radix tree (rt_tree*)."""
+
+    def __init__(self, handle: ctypes.c_void_p):
+        self._h = handle
+
+    @property
+    def handle(self) -> ctypes.c_void_p:
+        if not self._h:
+            raise ValueError("tree was destroyed")
+        return self._h
+
+    def destroy(self) -> None:
+        if self._h:
+            _check(_lib.rt_destroy(self._h), "rt_destroy")
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def rt_create(max_nodes: int, max_pool_tokens: int, budget_tokens: int = 0, vocab: int = 0, max_clock: int = 0) -> Tree:
+    cfg = rt_config(int(vocab), int(max_nodes), int(max_pool_tokens), int(budget_tokens), int(max_clock))
+    h = ctypes.c_void_p()
+    _check(_lib.rt_create(ctypes.byref(cfg), ctypes.byref(h)), "rt_create")
+    return Tree(h)
+
+
+def rt_build(tokens: torch.Tensor, offsets: torch.Tensor, max_nodes: int, max_pool_tokens: int,
+             budget_tokens: int = 0, vocab: int = 0, max_clock: int = 0) -> Tree:
+    cfg = rt_config(int(vocab), int(max_nodes), int(max_pool_tokens), int(budget_tokens), int(max_clock))
+    h = ctypes.c_void_p()
+    n = offsets.numel() - 1
+    _check(_lib.rt_build(_dev(tokens, torch.int32, "tokens", n == 0), _dev(offsets, torch.int64, "offsets"), n,
+                         ctypes.byref(cfg), _stream(), ctypes.byref(h)), "rt_build")
+    return Tree(h)
+
+
+def rt_insert(tree: Tree, tokens: torch.Tensor, offsets: torch.Tensor, new_tokens: Optional[torch.Tensor] = None) -> None:
+    n = offsets.numel() - 1
+    _check(_lib.rt_insert(tree.handle, _dev(tokens, torch.int32, "tokens"), _dev(offsets, torch.int64, "offsets"), n,
+                          _dev(new_tokens, torch.int32, "new_tokens", True), _stream()), "rt_insert")
+
+
+def rt_match_batch(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, match_len: torch.Tensor,
+                   term_node: Optional[torch.Tensor] = None, term_off: Optional[torch.Tensor] = None) -> None:
+    nq = q_offsets.numel() - 1
+    _check(_lib.rt_match_batch(tree.handle, _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
+                               nq, _dev(match_len, torch.int32, "match_len"), _dev(term_node, torch.int32, "term_node", True),
+                               _dev(term_off, torch.int32, "term_off", True), _stream()), "rt_match_batch")
+
+
+def rt_stats(tree: Tree) -> dict:
+    v = [ctypes.c_int64() for _ in range(5)]
+    _check(_lib.rt_stats(tree.handle, *[ctypes.byref(x) for x in v]), "rt_stats")
+    return dict(n_nodes=v[0].value, tokens=v[1].value, clock=v[2].value, evictions=v[3].value, pool_used=v[4].value)
+
+
+def rt_sync_status(tree: Tree) -> int:
+    return int(_lib.rt_sync_status(tree.handle, _stream()))
+
+
+def rt_destroy(tree: Tree) -> None:
+    tree.destroy()
+
+
+def klpm_select(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, pick_counter: int,
+                params: klpm_params, pick: torch.Tensor) -> None:
+    _check(_lib.klpm_select(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
+                            _dev(waiting, torch.uint8, "waiting"), match_len.numel(), int(pick_counter),
+                            ctypes.byref(params), _dev(pick, torch.int32, "pick"), _stream()), "klpm_select")
+
+
+def klpm_replay(tree: Tree, order: torch.Tensor, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arrival: torch.Tensor,
+                params: klpm_params, uncached: torch.Tensor, ttft: torch.Tensor,
+                completion: Optional[torch.Tensor] = None) -> None:
+    _check(_lib.klpm_replay(tree.handle, _dev(order, torch.int32, "order"), order.numel(),
+                            _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
+                            _dev(arrival, torch.int64, "arrival"), arrival.numel(), ctypes.byref(params),
+                            _dev(uncached, torch.int32, "uncached"), _dev(ttft, torch.int64, "ttft"),
+                            _dev(completion, torch.int64, "completion", True), _stream()), "klpm_replay")
+
+
+def klpm_run(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arrival: torch.Tensor, params: klpm_params,
+             order: torch.Tensor, uncached: torch.Tensor, ttft: torch.Tensor,
+             completion: Optional[torch.Tensor] = None) -> None:
+    n = arrival.numel()
+    _check(_lib.klpm_run(tree.handle, _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
+                         _dev(arrival, torch.int64, "arrival"), n, ctypes.byref(params), _dev(order, torch.int32, "order"),
+                         _dev(uncached, torch.int32, "uncached"), _dev(ttft, torch.int64, "ttft"),
+                         _dev(completion, torch.int64, "completion", True), _stream()), "klpm_run")

@@ -1,0 +1,970 @@
+// Device-resident k-LPM scheduling path for sm_100a: flattened radix tree, batched longest-prefix
+// match, k-LPM selection, schedule replay with LRU eviction.  See include/klpm.h for the ABI.
+//
+// Layout in HBM
+//   nodes   : structure of arrays indexed by node id (0 = root): parent, depth_start, span_len, nchild
+//             (int32), span_off, last_access (int64), dead (uint8).  Ids are never reused.
+//   pool    : append-only int32 token pool; node v's edge label is pool[span_off[v] .. +span_len[v]).
+//             A split never moves tokens, so "pool index of the last matched token" identifies a
+//             position in the tree for as long as the tree lives.
+//   children: one open-addressing hash table for the whole tree keyed by (parent id, first token of the
+//             child's edge).  An entry is one 32-byte sector and carries what a walk needs for the hop
+//             (child id, edge length, edge offset), so a hop costs one dependent sector read.
+//   LRU     : last_access holds logical clocks.  Only the node where a processed prompt's cached part
+//             ends and its new leaf are stamped; when a leaf is evicted its stamp is handed to its
+//             parent if newer.  For every leaf this equals the clock of the last processed prompt
+//             whose path covers it, which is all eviction looks at.  clock_owner[c] names the node
+//             holding stamp c, so the least recently used leaf is found by a cursor that only moves
+//             forward over clock values.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+#include <new>
+
+#include "klpm.h"
+
+#define FULL_MASK 0xffffffffu
+#define KLPM_ABI_VERSION 1
+
+namespace {
+
+struct alignas(32) Entry {
+    unsigned long long key;   // ((parent + 1) << 32) | first token ; 0 = empty slot
+    int32_t child;            // node id, or -1 if the child was evicted (slot is reused on re-insert)
+    int32_t span_len;
+    int64_t span_off;
+    int64_t pad;
+};
+
+struct TreeState {
+    long long n_nodes;      // next free node id
+    long long pool_used;
+    long long tokens_live;
+    long long live_nodes;   // root excluded
+    long long clock;
+    long long lru_cursor;
+    long long evictions;
+    int status;
+    int pad;
+};
+
+struct TreeDev {
+    int32_t* parent;
+    int32_t* depth_start;
+    int32_t* span_len;
+    int32_t* nchild;
+    int64_t* span_off;
+    int64_t* last_access;
+    uint8_t* dead;
+    int32_t* clock_owner;
+    Entry* table;
+    unsigned long long table_mask;
+    int32_t* pool;
+    TreeState* st;
+    long long max_nodes, max_pool, max_clock, budget;
+};
+
+// ------------------------------------------------------------------------------------------------
+// loads: RO = the kernel never writes what it reads (read-only path), otherwise L2-coherent loads
+// ------------------------------------------------------------------------------------------------
+template <bool RO> __device__ __forceinline__ int32_t ld32(const int32_t* p) { return RO ? __ldg(p) : __ldcg(p); }
+template <bool RO> __device__ __forceinline__ Entry ld_entry(const Entry* e) {
+    const int4* p = reinterpret_cast<const int4*>(e);
+    int4 a = RO ? __ldg(p) : __ldcg(p);
+    int4 b = RO ? __ldg(p + 1) : __ldcg(p + 1);
+    Entry r;
+    r.key = ((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x;
+    r.child = a.z;
+    r.span_len = a.w;
+    r.span_off = (int64_t)(((unsigned long long)(unsigned)b.y << 32) | (unsigned)b.x);
+    r.pad = 0;
+    return r;
+}
+
+__device__ __forceinline__ unsigned long long make_key(int32_t parent, int32_t tok) {
+    return ((unsigned long long)(unsigned)(parent + 1) << 32) | (unsigned)tok;
+}
+// 64-bit finaliser of MurmurHash3 (public domain, A. Appleby)
+__device__ __forceinline__ unsigned long long hash64(unsigned long long k) {
+    k ^= k >> 33; k *= 0xff51afd7ed558ccdULL; k ^= k >> 33; k *= 0xc4ceb9fe1a85ec53ULL; k ^= k >> 33;
+    return k;
+}
+
+__device__ __forceinline__ void set_status(TreeState* st, int code) { atomicCAS(&st->status, 0, code); }
+
+// First index in [0, n) where a and b differ, or n.  Warp-cooperative: every lane gets the result.
+// Lane l reads elements l, l+32, l+64, l+96 of each 128-token chunk: each load instruction of the warp
+// is one contiguous 128-byte request, whatever the 4-byte phase of the two streams.
+template <bool RO>
+__device__ __forceinline__ int32_t first_mismatch(const int32_t* __restrict__ a, const int32_t* __restrict__ b, int32_t n) {
+    const int lane = threadIdx.x & 31;
+    for (int32_t base = 0; base < n; base += 128) {
+        int32_t x[4], y[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int32_t idx = base + j * 32 + lane;
+            bool in = idx < n;
+            x[j] = in ? ld32<RO>(a + idx) : 0;
+            y[j] = in ? ld32<RO>(b + idx) : 0;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            unsigned bad = __ballot_sync(FULL_MASK, x[j] != y[j]);
+            if (bad) return base + j * 32 + (__ffs(bad) - 1);
+        }
+    }
+    return n;
+}
+
+struct Term {
+    int32_t m;      // matched tokens
+    int32_t node;   // node whose edge holds the last matched token (0 = root)
+    int32_t off;    // tokens of that edge matched
+    int64_t pos;    // pool index of the last matched token, -1 at the root
+};
+
+// Longest prefix of q on a root path.  Warp-cooperative and warp-uniform.
+template <bool RO>
+__device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t len) {
+    Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1;
+    if (len <= 0) return t;
+    unsigned long long key = make_key(0, ld32<RO>(q));
+    unsigned long long slot = hash64(key) & T.table_mask;
+    Entry c = ld_entry<RO>(T.table + slot);
+    for (;;) {
+        unsigned probes = 0;
+        while (c.key != key) {
+            if (c.key == 0ULL || ++probes > 4096u) return t;
+            slot = (slot + 1) & T.table_mask;
+            c = ld_entry<RO>(T.table + slot);
+        }
+        if (c.child < 0) return t;
+        const int32_t rem = len - t.m;
+        const int32_t n = c.span_len < rem ? c.span_len : rem;
+        const bool has_next = c.span_len < rem;
+        // issue the probe of the next hop before comparing this edge: it depends only on this entry
+        unsigned long long key2 = 0, slot2 = 0;
+        Entry nx; nx.key = 0; nx.child = -1; nx.span_len = 0; nx.span_off = 0;
+        if (has_next) {
+            key2 = make_key(c.child, ld32<RO>(q + t.m + c.span_len));
+            slot2 = hash64(key2) & T.table_mask;
+            nx = ld_entry<RO>(T.table + slot2);
+        }
+        const int32_t i = first_mismatch<RO>(q + t.m, T.pool + c.span_off, n);
+        t.m += i;
+        t.node = c.child;
+        t.off = i;
+        t.pos = c.span_off + i - 1;     // i >= 1: the first token is the key
+        if (i < c.span_len || !has_next) return t;
+        key = key2; slot = slot2; c = nx;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// single-thread tree updates (callers serialise them)
+// ------------------------------------------------------------------------------------------------
+__device__ long long table_find(const TreeDev& T, int32_t parent, int32_t tok) {
+    unsigned long long key = make_key(parent, tok);
+    unsigned long long slot = hash64(key) & T.table_mask;
+    for (unsigned long long probes = 0; probes <= T.table_mask; ++probes) {
+        unsigned long long k = __ldcg(&T.table[slot].key);
+        if (k == key) return (long long)slot;
+        if (k == 0ULL) return -1;
+        slot = (slot + 1) & T.table_mask;
+    }
+    return -1;
+}
+
+__device__ bool table_put(const TreeDev& T, int32_t parent, int32_t tok, int32_t child, int32_t span_len, int64_t span_off) {
+    unsigned long long key = make_key(parent, tok);
+    unsigned long long slot = hash64(key) & T.table_mask;
+    for (unsigned long long probes = 0; probes <= T.table_mask; ++probes) {
+        unsigned long long k = __ldcg(&T.table[slot].key);
+        if (k == key || k == 0ULL) {
+            Entry* e = T.table + slot;
+            e->child = child; e->span_len = span_len; e->span_off = span_off; e->pad = 0;
+            e->key = key;
+            return true;
+        }
+        slot = (slot + 1) & T.table_mask;
+    }
+    return false;
+}
+
+// Node boundary `o` tokens into v's edge (0 < o < span_len[v]): a new node takes the upper part and v's
+// place under v's parent; v keeps the lower part, its children and its id.
+__device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o) {
+    TreeState* S = T.st;
+    int32_t u = (int32_t)S->n_nodes++;
+    S->live_nodes++;
+    int32_t par = T.parent[v], ds = T.depth_start[v], len = T.span_len[v];
+    int64_t off = T.span_off[v];
+    T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = off; T.span_len[u] = o;
+    T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = T.last_access[v];
+    long long slot = table_find(T, par, __ldcg(T.pool + off));
+    if (slot >= 0) { T.table[slot].child = u; T.table[slot].span_len = o; }
+    else set_status(S, RT_ERR_LIMIT);
+    T.span_off[v] = off + o; T.span_len[v] = len - o; T.depth_start[v] = ds + o; T.parent[v] = u;
+    if (!table_put(T, u, __ldcg(T.pool + off + o), v, len - o, off + o)) set_status(S, RT_ERR_CAPACITY);
+    return u;
+}
+
+__device__ void evict_leaf(const TreeDev& T, int32_t v) {
+    TreeState* S = T.st;
+    int32_t P = T.parent[v];
+    T.dead[v] = 1;
+    long long slot = table_find(T, P, __ldcg(T.pool + T.span_off[v]));
+    if (slot >= 0) T.table[slot].child = -1;
+    T.nchild[P]--;
+    S->tokens_live -= T.span_len[v];
+    S->live_nodes--;
+    S->evictions++;
+    if (P != 0 && T.last_access[v] >= T.last_access[P]) {
+        T.last_access[P] = T.last_access[v];
+        T.clock_owner[T.last_access[v]] = P;
+    }
+}
+
+struct InsertOut {
+    int32_t leaf;      // id of the new leaf, -1 if the prompt was fully cached
+    int32_t unc;       // tokens to copy into the pool
+    int64_t leaf_off;  // pool offset of the new leaf's edge
+    int32_t evicted;   // 1 if any leaf was evicted
+    int32_t ok;        // 0 if the prompt could not be stored (status word says why)
+};
+
+// Store prompt x (|x| = len) whose cached part is m tokens long and ends in `hint` or an ancestor of it.
+// Everything except copying the new leaf's tokens into the pool.  One thread.
+__device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, int32_t m, int32_t hint, InsertOut* out) {
+    TreeState* S = T.st;
+    out->leaf = -1; out->unc = 0; out->leaf_off = 0; out->evicted = 0; out->ok = 0;
+    if (S->clock + 1 >= T.max_clock || S->n_nodes + 2 > T.max_nodes) { set_status(S, RT_ERR_CAPACITY); return; }
+    const long long clock = ++S->clock;
+    int32_t a = hint;
+    while (a != 0 && m <= T.depth_start[a]) a = T.parent[a];
+    const int32_t o = a == 0 ? 0 : m - T.depth_start[a];
+    int32_t end = a;
+    if (a != 0 && o < T.span_len[a]) end = split_node(T, a, o);
+    if (end != 0) { T.last_access[end] = clock; T.clock_owner[clock] = end; }
+    const int32_t unc = len - m;
+    if (T.budget > 0) {
+        while (S->tokens_live + unc > T.budget) {
+            long long cur = S->lru_cursor;
+            int32_t victim = -1;
+            while (cur < clock) {
+                int32_t v = T.clock_owner[cur];
+                if (v > 0 && !T.dead[v] && T.last_access[v] == cur && T.nchild[v] == 0) { victim = v; break; }
+                ++cur;
+            }
+            S->lru_cursor = cur;
+            if (victim < 0) { set_status(S, RT_ERR_BUDGET); return; }
+            evict_leaf(T, victim);
+            out->evicted = 1;
+        }
+    }
+    if (unc > 0) {
+        if (S->pool_used + unc > T.max_pool) { set_status(S, RT_ERR_CAPACITY); return; }
+        int32_t leaf = (int32_t)S->n_nodes++;
+        int64_t off = S->pool_used;
+        S->pool_used += unc;
+        T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = off; T.span_len[leaf] = unc;
+        T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = clock;
+        T.clock_owner[clock] = leaf;
+        T.nchild[end]++;
+        if (!table_put(T, end, __ldcg(x + m), leaf, unc, off)) { set_status(S, RT_ERR_CAPACITY); return; }
+        S->tokens_live += unc;
+        S->live_nodes++;
+        out->leaf = leaf; out->unc = unc; out->leaf_off = off;
+    }
+    out->ok = 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// rt_match_batch
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
+                   int32_t* __restrict__ mlen, int32_t* __restrict__ tnode, int32_t* __restrict__ toff,
+                   unsigned long long* counter) {
+    const int lane = threadIdx.x & 31;
+    for (;;) {
+        unsigned long long i = 0;
+        if (lane == 0) i = atomicAdd(counter, 1ULL);
+        i = __shfl_sync(FULL_MASK, i, 0);
+        if (i >= (unsigned long long)nq) return;
+        const int64_t lo = __ldg(qoff + i), hi = __ldg(qoff + i + 1);
+        int64_t len = hi - lo;
+        if (len < 0 || len > 0x7fffffffLL) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
+        Term t = walk<true>(T, qtok + lo, (int32_t)len);
+        if (lane == 0) {
+            mlen[i] = t.m;
+            if (tnode) tnode[i] = t.node;
+            if (toff) toff[i] = t.off;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// sequential processing of prompts by one CTA: rt_insert and klpm_replay
+// ------------------------------------------------------------------------------------------------
+struct SeqArgs {
+    const int32_t* tok; const int64_t* off; const int64_t* arrival; const int32_t* order;
+    int32_t n;                       // prompts to process
+    long long c_num, c_den, start_tick;
+    int32_t* new_tokens;             // rt_insert: indexed by position
+    int32_t* uncached; int64_t* ttft; int64_t* completion;   // replay: indexed by query
+};
+
+__global__ void __launch_bounds__(1024)
+sequential_kernel(TreeDev T, SeqArgs A) {
+    __shared__ Term s_term;
+    __shared__ InsertOut s_out;
+    long long now = A.start_tick;
+    for (int32_t k = 0; k < A.n; ++k) {
+        const int32_t j = A.order ? __ldg(A.order + k) : k;
+        const int64_t lo = __ldg(A.off + j), hi = __ldg(A.off + j + 1);
+        const int32_t len = (int32_t)(hi - lo);
+        const int32_t* x = A.tok + lo;
+        if (threadIdx.x < 32) {
+            Term t = walk<false>(T, x, len);
+            if (threadIdx.x == 0) {
+                s_term = t;
+                insert_serial(T, x, len, t.m, t.node, &s_out);
+                if (s_out.ok) {
+                    int32_t unc = len - t.m;
+                    if (A.new_tokens) A.new_tokens[k] = unc;
+                    if (A.uncached) {
+                        long long tj = __ldg(A.arrival + j);
+                        long long begin = now > tj ? now : tj;
+                        long long R = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
+                        A.uncached[j] = unc; A.ttft[j] = R - tj;
+                        if (A.completion) A.completion[j] = R;
+                        now = R;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (!s_out.ok) return;
+        const int32_t unc = s_out.unc, m = s_term.m;
+        int32_t* dst = T.pool + s_out.leaf_off;
+        for (int32_t i = threadIdx.x; i < unc; i += blockDim.x) dst[i] = __ldg(x + m + i);
+        __threadfence();
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// klpm_select: one decision as a pure function
+// ------------------------------------------------------------------------------------------------
+struct Cand { int32_t m; int32_t idx; long long t; };   // idx < 0 = none
+
+__device__ __forceinline__ bool better_lpm(const Cand& a, const Cand& b) {      // a beats b
+    if (b.idx < 0) return a.idx >= 0;
+    if (a.idx < 0) return false;
+    if (a.m != b.m) return a.m > b.m;
+    if (a.t != b.t) return a.t < b.t;
+    return a.idx < b.idx;
+}
+__device__ __forceinline__ bool better_fcfs(const Cand& a, const Cand& b) {
+    if (b.idx < 0) return a.idx >= 0;
+    if (a.idx < 0) return false;
+    if (a.t != b.t) return a.t < b.t;
+    return a.idx < b.idx;
+}
+template <bool LPM> __device__ __forceinline__ Cand cand_best(Cand a, Cand b) {
+    return (LPM ? better_lpm(b, a) : better_fcfs(b, a)) ? b : a;
+}
+template <bool LPM> __device__ __forceinline__ Cand warp_best(Cand c) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        Cand o;
+        o.m = __shfl_xor_sync(FULL_MASK, c.m, d);
+        o.idx = __shfl_xor_sync(FULL_MASK, c.idx, d);
+        o.t = __shfl_xor_sync(FULL_MASK, c.t, d);
+        c = cand_best<LPM>(c, o);
+    }
+    return c;
+}
+template <bool LPM> __device__ Cand block_best(Cand c, Cand* smem /*32*/) {
+    c = warp_best<LPM>(c);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    if (lane == 0) smem[w] = c;
+    __syncthreads();
+    Cand r; r.m = 0; r.idx = -1; r.t = 0;
+    if (w == 0) {
+        if (lane < nw) r = smem[lane];
+        r = warp_best<LPM>(r);
+    }
+    return r;   // valid in warp 0
+}
+
+struct SelectScratch { Cand partial[1024]; unsigned int ticket; };
+
+template <bool LPM>
+__global__ void __launch_bounds__(512)
+select_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict__ arrival, const uint8_t* __restrict__ waiting,
+              int32_t nq, int32_t* pick, SelectScratch* sc) {
+    __shared__ Cand s_c[32];
+    __shared__ bool s_last;
+    Cand best; best.m = 0; best.idx = -1; best.t = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nq; i += (int64_t)gridDim.x * blockDim.x) {
+        if (__ldg(waiting + i)) {
+            Cand c; c.m = LPM ? __ldg(mlen + i) : 0; c.idx = (int32_t)i; c.t = __ldg(arrival + i);
+            best = cand_best<LPM>(best, c);
+        }
+    }
+    best = block_best<LPM>(best, s_c);
+    if (threadIdx.x == 0) {
+        sc->partial[blockIdx.x] = best;
+        __threadfence();
+        unsigned t = atomicAdd(&sc->ticket, 1u);
+        s_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    Cand c; c.m = 0; c.idx = -1; c.t = 0;
+    for (int b = threadIdx.x; b < (int)gridDim.x; b += blockDim.x) {
+        Cand o;
+        o.m = __ldcg(&sc->partial[b].m); o.idx = __ldcg(&sc->partial[b].idx); o.t = __ldcg(&sc->partial[b].t);
+        c = cand_best<LPM>(c, o);
+    }
+    __syncthreads();
+    c = block_best<LPM>(c, s_c);
+    if (threadIdx.x == 0) { *pick = c.idx; sc->ticket = 0; }
+}
+
+// ------------------------------------------------------------------------------------------------
+// klpm_run: the whole loop as one cooperative kernel
+// ------------------------------------------------------------------------------------------------
+struct GridBarrier { unsigned int count; unsigned int gen; };
+
+struct RunState {
+    long long now;
+    long long c;          // decisions taken
+    long long head;       // first slot not yet processed (slots are queries in arrival order)
+    long long admitted;   // slots < admitted have a match state
+    int abort;
+    int evicted;          // the previous decision evicted something
+    // the previously processed prompt, for the refresh of the queries tied with it
+    int last_valid;       // it appended a leaf
+    int32_t last_q;       // query index
+    int32_t last_m;       // its match length before it was stored
+    int32_t last_len;
+    int32_t last_leaf;
+    long long last_pos;   // its position (pool index of its last matched token) before it was stored
+    long long last_leaf_off;
+    GridBarrier bar;
+};
+
+struct RunArgs {
+    const int32_t* tok; const int64_t* off; const int64_t* arrival;
+    int32_t n;
+    int32_t policy, k;
+    long long c_num, c_den, start_tick;
+    int32_t* order; int32_t* uncached; int64_t* ttft; int64_t* completion;
+    // scratch (library-owned)
+    int32_t* ord;          // slot -> query index, by (arrival, index)
+    long long* sorted_t;   // slot -> arrival
+    int32_t* m;            // slot -> current match length
+    int32_t* hint;         // slot -> node at or below the node where the match ends
+    long long* pos;        // slot -> pool index of the last matched token (-1 = root)
+    uint8_t* done;         // slot processed
+    unsigned long long* partial;   // per CTA best key
+    RunState* rs;
+};
+
+// All CTAs of a cooperative launch meet here.  The wait is bounded: if it runs out, the status word is set
+// and every CTA leaves the kernel at its next check of rs->abort.
+__device__ bool grid_sync(RunState* rs, TreeState* st, unsigned nblocks) {
+    __shared__ int s_ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        if (nblocks > 1) {
+            volatile unsigned* gen = &rs->bar.gen;
+            unsigned my = *gen;
+            __threadfence();
+            unsigned t = atomicAdd(&rs->bar.count, 1u);
+            if (t == nblocks - 1) {
+                rs->bar.count = 0;
+                __threadfence();
+                atomicAdd(&rs->bar.gen, 1u);
+            } else {
+                unsigned long long spins = 0;
+                while (*gen == my) {
+                    __nanosleep(32);
+                    if (++spins > (1ULL << 26)) { set_status(st, RT_ERR_LIMIT); *(volatile int*)&rs->abort = 1; ok = 0; break; }
+                }
+            }
+            __threadfence();
+        }
+        if (*(volatile int*)&rs->abort) ok = 0;
+        s_ok = ok;
+    }
+    __syncthreads();
+    return s_ok != 0;
+}
+
+__global__ void __launch_bounds__(512)
+run_kernel(TreeDev T, RunArgs A) {
+    __shared__ unsigned long long s_red[16];
+    __shared__ long long s_bound[2];      // admitted_new, now
+    __shared__ InsertOut s_out;
+    __shared__ int32_t s_j[4];            // slot, m, len
+    __shared__ const int32_t* s_x;
+    RunState* rs = A.rs;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long TT = (long long)gridDim.x * blockDim.x;
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+
+    for (long long c = 0; c < A.n; ++c) {
+        // ---------------- phase A: bring the waiting queue's match state up to date, reduce the keys
+        const long long head = *(volatile long long*)&rs->head;
+        const long long admitted = *(volatile long long*)&rs->admitted;
+        if (threadIdx.x == 0) {
+            long long now = *(volatile long long*)&rs->now;
+            long long th = __ldg(A.sorted_t + head);
+            if (th > now) now = th;                    // nobody waiting: idle until the next arrival
+            long long lo = head, hi = A.n;             // first slot with arrival > now
+            while (lo < hi) { long long mid = (lo + hi) >> 1; if (__ldg(A.sorted_t + mid) <= now) lo = mid + 1; else hi = mid; }
+            s_bound[0] = lo; s_bound[1] = now;
+        }
+        __syncthreads();
+        const long long adm_new = s_bound[0];
+        const int evicted = __ldcg(&rs->evicted);
+        const int last_valid = __ldcg(&rs->last_valid);
+        const int32_t last_m = __ldcg(&rs->last_m), last_len = __ldcg(&rs->last_len), last_leaf = __ldcg(&rs->last_leaf);
+        const long long last_pos = __ldcg(&rs->last_pos), last_leaf_off = __ldcg(&rs->last_leaf_off);
+        const int32_t* last_x = last_valid ? A.tok + __ldg(A.off + __ldcg(&rs->last_q)) : nullptr;
+
+        unsigned long long best = 0;
+        for (long long base = (head / TT) * TT; base < adm_new; base += TT) {
+            const long long r = base + gtid;
+            const bool active = r >= head && r < adm_new && !__ldcg(A.done + r);
+            int32_t qi = 0, qlen = 0, m = 0, hint = 0;
+            long long pos = -1;
+            const int32_t* q = nullptr;
+            if (active) {
+                qi = __ldg(A.ord + r);
+                const int64_t lo = __ldg(A.off + qi);
+                qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
+                q = A.tok + lo;
+            }
+            const bool fresh = active && r >= admitted;
+            unsigned wm = __ballot_sync(FULL_MASK, fresh);
+            while (wm) {                                  // newly arrived queries: full walk, one warp each
+                const int src = __ffs(wm) - 1; wm &= wm - 1;
+                const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+                const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
+                Term t = walk<false>(T, qq, ql);
+                if (lane == src) { m = t.m; hint = t.node; pos = t.pos; }
+            }
+            bool dirty = fresh;
+            bool cmp = false;
+            if (active && !fresh) {
+                m = __ldcg(A.m + r); pos = __ldcg(A.pos + r);
+                if (evicted) {                            // drop out of evicted leaves
+                    hint = __ldcg(A.hint + r);
+                    int32_t a = hint, m0 = m;
+                    while (a != 0) {
+                        const bool dead = __ldcg(T.dead + a) != 0;
+                        const int32_t ds = __ldcg(T.depth_start + a);
+                        if (dead) { if (ds < m) m = ds; }
+                        else if (m > ds) break;
+                        a = __ldcg(T.parent + a);
+                    }
+                    if (a != hint || m != m0) {
+                        hint = a;
+                        pos = a == 0 ? -1 : __ldcg(T.span_off + a) + (m - __ldcg(T.depth_start + a)) - 1;
+                        dirty = true;
+                    }
+                }
+                // tied with the prompt processed last: it may now match into that prompt's new leaf
+                if (last_valid && pos == last_pos && m == last_m && m < qlen)
+                    cmp = __ldg(q + m) == __ldg(last_x + m);
+            }
+            unsigned cm = __ballot_sync(FULL_MASK, cmp);
+            while (cm) {
+                const int src = __ffs(cm) - 1; cm &= cm - 1;
+                const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+                const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
+                const int32_t lim = (ql < last_len ? ql : last_len) - last_m;
+                const int32_t e = first_mismatch<true>(qq + last_m, last_x + last_m, lim);
+                if (lane == src) { m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1; dirty = true; }
+            }
+            if (active) {
+                if (dirty) { A.m[r] = m; A.pos[r] = pos; A.hint[r] = hint; }
+                const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
+                if (key > best) best = key;
+            }
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            unsigned long long o = __shfl_xor_sync(FULL_MASK, best, d);
+            if (o > best) best = o;
+        }
+        if (lane == 0) s_red[warp] = best;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long b = 0;
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) if (s_red[w] > b) b = s_red[w];
+            A.partial[blockIdx.x] = b;
+        }
+        if (!grid_sync(rs, T.st, gridDim.x)) return;
+
+        // ---------------- phase B: CTA 0 picks, charges (Definition 2) and stores the prompt
+        if (blockIdx.x == 0) {
+            if (threadIdx.x == 0) {
+                const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
+                long long slot;
+                if (fcfs_turn) slot = head;
+                else {
+                    unsigned long long b = 0;
+                    for (unsigned g = 0; g < gridDim.x; ++g) { unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
+                    slot = (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
+                }
+                const int32_t qi = __ldg(A.ord + slot);
+                const int64_t lo = __ldg(A.off + qi);
+                const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
+                const int32_t* x = A.tok + lo;
+                const int32_t m = __ldcg(A.m + slot);
+                const int32_t hint = __ldcg(A.hint + slot);
+                const long long pos = __ldcg(A.pos + slot);
+                insert_serial(T, x, len, m, hint, &s_out);
+                s_j[0] = (int32_t)slot; s_j[1] = m; s_j[2] = len; s_x = x;
+                if (s_out.ok) {
+                    const long long tj = __ldg(A.arrival + qi);
+                    const long long now = s_bound[1];
+                    const long long begin = now > tj ? now : tj;
+                    const long long unc = len - m;
+                    const long long R = begin + (A.c_den + A.c_num * (long long)len) * unc;
+                    A.order[c] = qi; A.uncached[qi] = (int32_t)unc; A.ttft[qi] = R - tj;
+                    if (A.completion) A.completion[qi] = R;
+                    A.done[slot] = 1;
+                    long long h = head;
+                    while (h < A.n && (h == slot || __ldcg(A.done + h))) ++h;
+                    rs->head = h; rs->now = R; rs->admitted = adm_new; rs->c = c + 1;
+                    rs->evicted = s_out.evicted;
+                    rs->last_valid = s_out.unc > 0; rs->last_q = qi; rs->last_m = m; rs->last_len = len;
+                    rs->last_leaf = s_out.leaf; rs->last_pos = pos; rs->last_leaf_off = s_out.leaf_off;
+                } else {
+                    rs->abort = 1;
+                }
+            }
+            __syncthreads();
+            if (s_out.ok) {
+                const int32_t unc = s_out.unc, m = s_j[1];
+                const int32_t* x = s_x;
+                int32_t* dst = T.pool + s_out.leaf_off;
+                for (int32_t i = threadIdx.x; i < unc; i += blockDim.x) dst[i] = __ldg(x + m + i);
+            }
+            __threadfence();
+        }
+        if (!grid_sync(rs, T.st, gridDim.x)) return;
+    }
+}
+
+// slot order: bitonic sort of (arrival, index) pairs, padded to a power of two
+__global__ void rank_init_kernel(const int64_t* __restrict__ arrival, int32_t n, long long np2, long long* key, int32_t* idx) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= np2) return;
+    key[i] = i < n ? arrival[i] : 0x7fffffffffffffffLL;
+    idx[i] = i < n ? (int32_t)i : 0x7fffffff;
+}
+__global__ void bitonic_step_kernel(long long* key, int32_t* idx, long long np2, long long k, long long j) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= np2) return;
+    long long l = i ^ j;
+    if (l > i) {
+        long long ki = key[i], kl = key[l];
+        int32_t ii = idx[i], il = idx[l];
+        bool gt = ki > kl || (ki == kl && ii > il);
+        bool up = (i & k) == 0;
+        if (gt == up) { key[i] = kl; key[l] = ki; idx[i] = il; idx[l] = ii; }
+    }
+}
+
+}  // namespace
+
+// ====================================================================================================
+// host side
+// ====================================================================================================
+struct rt_tree {
+    rt_config cfg;
+    TreeDev dev;
+    int device;
+    cudaStream_t last_stream;
+    unsigned long long* match_counter;
+    // klpm_run scratch
+    long long run_cap;      // slots allocated (power of two)
+    long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos; uint8_t* run_done;
+    unsigned long long* run_partial; RunState* run_rs;
+    int num_sms;
+};
+
+namespace {
+
+#define CK(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { \
+    fprintf(stderr, "klpm: %s failed at %s:%d: %s\n", #call, __FILE__, __LINE__, cudaGetErrorString(e_)); return RT_ERR_CUDA; } } while (0)
+
+template <typename P> rt_status dalloc(P** p, size_t count) {
+    void* v = nullptr;
+    CK(cudaMalloc(&v, count * sizeof(P) + 256));
+    *p = (P*)v;
+    return RT_OK;
+}
+
+void free_tree(rt_tree* t) {
+    TreeDev& d = t->dev;
+    cudaFree(d.parent); cudaFree(d.depth_start); cudaFree(d.span_len); cudaFree(d.nchild);
+    cudaFree(d.span_off); cudaFree(d.last_access); cudaFree(d.dead); cudaFree(d.clock_owner);
+    cudaFree(d.table); cudaFree(d.pool); cudaFree(d.st); cudaFree(t->match_counter);
+    cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
+    cudaFree(t->run_pos); cudaFree(t->run_done); cudaFree(t->run_partial); cudaFree(t->run_rs);
+    delete t;
+}
+
+rt_status ensure_run_scratch(rt_tree* t, long long n) {
+    long long np2 = 1;
+    while (np2 < n) np2 <<= 1;
+    if (np2 <= t->run_cap) return RT_OK;
+    cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
+    cudaFree(t->run_pos); cudaFree(t->run_done);
+    t->run_key = nullptr; t->run_ord = nullptr; t->run_m = nullptr; t->run_hint = nullptr; t->run_pos = nullptr; t->run_done = nullptr;
+    t->run_cap = 0;
+    rt_status s;
+    if ((s = dalloc(&t->run_key, np2))) return s;
+    if ((s = dalloc(&t->run_ord, np2))) return s;
+    if ((s = dalloc(&t->run_m, np2))) return s;
+    if ((s = dalloc(&t->run_hint, np2))) return s;
+    if ((s = dalloc(&t->run_pos, np2))) return s;
+    if ((s = dalloc(&t->run_done, np2))) return s;
+    t->run_cap = np2;
+    return RT_OK;
+}
+
+bool params_ok(const klpm_params* p) {
+    return p && p->policy >= KLPM_POLICY_FCFS && p->policy <= KLPM_POLICY_KLPM && p->k >= 1 && p->c_den >= 1 && p->c_num >= 0;
+}
+
+SelectScratch* g_select_scratch[64] = {nullptr};
+
+}  // namespace
+
+extern "C" {
+
+int32_t klpm_abi_version(void) { return KLPM_ABI_VERSION; }
+
+rt_status rt_create(const rt_config* cfg, rt_tree** out) {
+    if (!cfg || !out || cfg->max_nodes < 2 || cfg->max_pool_tokens < 1 || cfg->budget_tokens < 0 ||
+        cfg->max_nodes > 0x7ffffff0LL || cfg->max_clock < 0) return RT_ERR_INVALID;
+    rt_tree* t = new (std::nothrow) rt_tree();
+    if (!t) return RT_ERR_CUDA;
+    memset(t, 0, sizeof(*t));
+    t->cfg = *cfg;
+    CK(cudaGetDevice(&t->device));
+    CK(cudaDeviceGetAttribute(&t->num_sms, cudaDevAttrMultiProcessorCount, t->device));
+    TreeDev& d = t->dev;
+    d.max_nodes = cfg->max_nodes;
+    d.max_pool = cfg->max_pool_tokens;
+    d.max_clock = (cfg->max_clock > 0 ? cfg->max_clock : cfg->max_nodes) + 2;
+    d.budget = cfg->budget_tokens;
+    unsigned long long cap = 1024;
+    while (cap < 2ULL * (unsigned long long)cfg->max_nodes) cap <<= 1;
+    d.table_mask = cap - 1;
+    rt_status s = RT_OK;
+    if ((s = dalloc(&d.parent, d.max_nodes)) || (s = dalloc(&d.depth_start, d.max_nodes)) ||
+        (s = dalloc(&d.span_len, d.max_nodes)) || (s = dalloc(&d.nchild, d.max_nodes)) ||
+        (s = dalloc(&d.span_off, d.max_nodes)) || (s = dalloc(&d.last_access, d.max_nodes)) ||
+        (s = dalloc(&d.dead, d.max_nodes)) || (s = dalloc(&d.clock_owner, d.max_clock)) ||
+        (s = dalloc(&d.table, cap)) || (s = dalloc(&d.pool, d.max_pool)) || (s = dalloc(&d.st, 1)) ||
+        (s = dalloc(&t->match_counter, 1)) || (s = dalloc(&t->run_partial, 1024)) || (s = dalloc(&t->run_rs, 1))) {
+        free_tree(t);
+        return s;
+    }
+    // root: node 0, empty edge
+    cudaError_t e = cudaMemset(d.table, 0, cap * sizeof(Entry));
+    if (e == cudaSuccess) e = cudaMemset(d.clock_owner, 0, d.max_clock * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(d.parent, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(d.depth_start, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(d.span_len, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(d.nchild, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(d.span_off, 0, sizeof(int64_t));
+    if (e == cudaSuccess) e = cudaMemset(d.last_access, 0, sizeof(int64_t));
+    if (e == cudaSuccess) e = cudaMemset(d.dead, 0, 1);
+    TreeState st0;
+    memset(&st0, 0, sizeof(st0));
+    st0.n_nodes = 1;
+    st0.lru_cursor = 1;
+    if (e == cudaSuccess) e = cudaMemcpy(d.st, &st0, sizeof(st0), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        fprintf(stderr, "klpm: tree initialisation failed: %s\n", cudaGetErrorString(e));
+        free_tree(t);
+        return RT_ERR_CUDA;
+    }
+    *out = t;
+    return RT_OK;
+}
+
+rt_status rt_destroy(rt_tree* tree) {
+    if (!tree) return RT_ERR_INVALID;
+    cudaDeviceSynchronize();
+    free_tree(tree);
+    return RT_OK;
+}
+
+rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n,
+                    int32_t* d_new_tokens, void* stream) {
+    if (!tree || n < 0 || (n > 0 && (!d_tokens || !d_offsets))) return RT_ERR_INVALID;
+    if (n == 0) return RT_OK;
+    SeqArgs a;
+    memset(&a, 0, sizeof(a));
+    a.tok = d_tokens; a.off = d_offsets; a.n = n; a.new_tokens = d_new_tokens; a.c_den = 1;
+    tree->last_stream = (cudaStream_t)stream;
+    sequential_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(tree->dev, a);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status rt_build(const int32_t* d_tokens, const int64_t* d_offsets, int32_t n_prompts, const rt_config* cfg,
+                   void* stream, rt_tree** out) {
+    if (!out || n_prompts < 0) return RT_ERR_INVALID;
+    rt_tree* t = nullptr;
+    rt_status s = rt_create(cfg, &t);
+    if (s) return s;
+    s = rt_insert(t, d_tokens, d_offsets, n_prompts, nullptr, stream);
+    if (s) { rt_destroy(t); return s; }
+    *out = t;
+    return RT_OK;
+}
+
+rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, int32_t nq,
+                         int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off, void* stream) {
+    if (!tree || nq < 0 || (nq > 0 && (!d_q_tokens || !d_q_offsets || !d_match_len))) return RT_ERR_INVALID;
+    if (nq == 0) return RT_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    const_cast<rt_tree*>(tree)->last_stream = s;
+    CK(cudaMemsetAsync(tree->match_counter, 0, sizeof(unsigned long long), s));
+    const int threads = 256, warps_per_block = threads / 32;
+    long long blocks = ((long long)nq + warps_per_block - 1) / warps_per_block;
+    long long max_blocks = (long long)tree->num_sms * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    match_batch_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
+                                                           d_term_node, d_term_off, tree->match_counter);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* clock, int64_t* evictions, int64_t* pool_used) {
+    if (!tree) return RT_ERR_INVALID;
+    CK(cudaStreamSynchronize(tree->last_stream));
+    TreeState st;
+    CK(cudaMemcpy(&st, tree->dev.st, sizeof(st), cudaMemcpyDeviceToHost));
+    if (n_nodes) *n_nodes = st.live_nodes;
+    if (n_tokens) *n_tokens = st.tokens_live;
+    if (clock) *clock = st.clock;
+    if (evictions) *evictions = st.evictions;
+    if (pool_used) *pool_used = st.pool_used;
+    return RT_OK;
+}
+
+rt_status rt_sync_status(rt_tree* tree, void* stream) {
+    if (!tree) return RT_ERR_INVALID;
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    TreeState st;
+    CK(cudaMemcpy(&st, tree->dev.st, sizeof(st), cudaMemcpyDeviceToHost));
+    return (rt_status)st.status;
+}
+
+rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting, int32_t nq,
+                      int64_t pick_counter, const klpm_params* params, int32_t* d_pick, void* stream) {
+    if (!params_ok(params) || nq < 0 || !d_pick || pick_counter < 0 ||
+        (nq > 0 && (!d_match_len || !d_arrival || !d_waiting))) return RT_ERR_INVALID;
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return RT_ERR_INVALID;
+    if (!g_select_scratch[dev]) {
+        SelectScratch* p = nullptr;
+        CK(cudaMalloc((void**)&p, sizeof(SelectScratch)));
+        CK(cudaMemset(p, 0, sizeof(SelectScratch)));
+        g_select_scratch[dev] = p;
+    }
+    const bool fcfs_turn = params->policy == KLPM_POLICY_FCFS ||
+                           (params->policy == KLPM_POLICY_KLPM && pick_counter % params->k == 0);
+    long long blocks = ((long long)nq + 2047) / 2048;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 1024) blocks = 1024;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (fcfs_turn) select_kernel<false><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, g_select_scratch[dev]);
+    else select_kernel<true><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, g_select_scratch[dev]);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, const int32_t* d_q_tokens,
+                      const int64_t* d_q_offsets, const int64_t* d_arrival, int32_t n_queries, const klpm_params* params,
+                      int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream) {
+    if (!tree || !params_ok(params) || n_order < 0 || n_queries < 0 ||
+        (n_order > 0 && (!d_order || !d_q_tokens || !d_q_offsets || !d_arrival || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
+    if (n_order == 0) return RT_OK;
+    SeqArgs a;
+    memset(&a, 0, sizeof(a));
+    a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.order = d_order; a.n = n_order;
+    a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
+    a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
+    tree->last_stream = (cudaStream_t)stream;
+    sequential_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(tree->dev, a);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
+                   int32_t n, const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                   int64_t* d_completion, void* stream) {
+    if (!tree || !params_ok(params) || n < 0 ||
+        (n > 0 && (!d_q_tokens || !d_q_offsets || !d_arrival || !d_order || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
+    if (n == 0) return RT_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    tree->last_stream = s;
+    rt_status st = ensure_run_scratch(tree, n);
+    if (st) return st;
+    long long np2 = 1;
+    while (np2 < n) np2 <<= 1;
+    // slots = queries ordered by (arrival, index)
+    {
+        unsigned blocks = (unsigned)((np2 + 255) / 256);
+        rank_init_kernel<<<blocks, 256, 0, s>>>(d_arrival, n, np2, tree->run_key, tree->run_ord);
+        for (long long k = 2; k <= np2; k <<= 1)
+            for (long long j = k >> 1; j > 0; j >>= 1)
+                bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_key, tree->run_ord, np2, k, j);
+        CK(cudaGetLastError());
+    }
+    CK(cudaMemsetAsync(tree->run_done, 0, (size_t)n, s));
+    RunState rs0;
+    memset(&rs0, 0, sizeof(rs0));
+    rs0.now = params->start_tick;
+    CK(cudaMemcpyAsync(tree->run_rs, &rs0, sizeof(rs0), cudaMemcpyHostToDevice, s));
+    RunArgs a;
+    memset(&a, 0, sizeof(a));
+    a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.n = n;
+    a.policy = params->policy; a.k = params->k; a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
+    a.order = d_order; a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
+    a.ord = tree->run_ord; a.sorted_t = tree->run_key; a.m = tree->run_m; a.hint = tree->run_hint; a.pos = tree->run_pos;
+    a.done = tree->run_done; a.partial = tree->run_partial; a.rs = tree->run_rs;
+    const int threads = 512;
+    int per_sm = 0;
+    CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, run_kernel, threads, 0));
+    if (per_sm < 1) return RT_ERR_CUDA;
+    long long blocks = ((long long)n + threads * 4 - 1) / (threads * 4);
+    if (blocks < 1) blocks = 1;
+    if (blocks > tree->num_sms) blocks = tree->num_sms;
+    void* kargs[] = {(void*)&tree->dev, (void*)&a};
+    CK(cudaLaunchCooperativeKernel((void*)run_kernel, dim3((unsigned)blocks), dim3(threads), kargs, 0, s));
+    return RT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,321 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI.  Integer work: the bar is bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import definition as D
+from paper_2502_04677_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def K():
+    from paper_2502_04677_b200 import binding
+    return binding
+
+
+def dev(t):
+    return t.cuda() if isinstance(t, torch.Tensor) else torch.as_tensor(t).cuda()
+
+
+def csr(prompts):
+    return W.to_csr(prompts)
+
+
+def caps(*token_counts, n_prompts=0):
+    total = int(sum(token_counts))
+    return dict(max_nodes=2 * n_prompts + 16, max_pool_tokens=total + 16, max_clock=n_prompts + 16)
+
+
+def gpu_tree(K, tokens, offsets, extra_prompts=0, extra_tokens=0, budget=0):
+    n = offsets.numel() - 1
+    c = caps(tokens.numel(), extra_tokens, n_prompts=n + extra_prompts)
+    if n == 0:
+        return K.rt_create(budget_tokens=budget, **c)
+    return K.rt_build(dev(tokens), dev(offsets), budget_tokens=budget, **c)
+
+
+def gpu_match(K, tree, qt, qo):
+    nq = qo.numel() - 1
+    m = torch.full((nq,), -7, dtype=torch.int32, device="cuda")
+    node = torch.full((nq,), -7, dtype=torch.int32, device="cuda")
+    off = torch.full((nq,), -7, dtype=torch.int32, device="cuda")
+    K.rt_match_batch(tree, dev(qt), dev(qo), m, node, off)
+    assert K.rt_sync_status(tree) == 0
+    return m.cpu().numpy(), node.cpu().numpy(), off.cpu().numpy()
+
+
+def oracle_tree(tokens, offsets, budget=0):
+    t = oracle.OracleTree(budget)
+    if offsets.numel() > 1:
+        t.insert(tokens.numpy(), offsets.numpy())
+    return t
+
+
+# ------------------------------------------------------------------ batched match
+
+def check_match(K, pt, po, qt, qo):
+    tree = gpu_tree(K, pt, po)
+    m, node, off = gpu_match(K, tree, qt, qo)
+    ot = oracle_tree(pt, po)
+    want = ot.match(qt.numpy(), qo.numpy())
+    assert np.array_equal(m, want)
+    assert np.array_equal(node == 0, m == 0) and np.all(off >= 0) and np.all(off <= m)
+    st, ost = K.rt_stats(tree), ot.stats()
+    assert (st["n_nodes"], st["tokens"], st["clock"]) == (ost["n_nodes"], ost["tokens"], ost["clock"])
+    K.rt_destroy(tree)
+    return m
+
+
+def test_match_tiny_config(K):
+    w = W.tiny()
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    m = check_match(K, pt, po, qt, qo)
+    assert m.min() >= 512          # every query shares one of the 8 cached prefixes
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_match_small_alphabet_ragged_and_empty(K, seed):
+    """Frequent overlaps, empty prompts and queries, lengths that straddle the 128-token compare chunk."""
+    cached, _ = W.random_small_queue(seed, 300, vocab=2, max_len=400)
+    queries, _ = W.random_small_queue(seed + 50, 257, vocab=2, max_len=420)
+    long_a = [1] * 1000 + [0]
+    cached += [long_a, [1] * 127, [1] * 128 + [0], [0] * 129, []]
+    queries += [[1] * 1000, [1] * 1001, long_a + [1], [1] * 128, [0] * 130, [], [1] * 127 + [0]]
+    check_match(K, *csr(cached), *csr(queries))
+    # brute force against every cached prompt as well (definition of the match length)
+    tree = gpu_tree(K, *csr(cached))
+    m, _, _ = gpu_match(K, tree, *csr(queries))
+    ct, co = csr(cached)
+    qt, qo = csr(queries)
+    assert np.array_equal(m, oracle.match_bruteforce(qt.numpy(), qo.numpy(), ct.numpy(), co.numpy()))
+
+
+def test_match_empty_tree_and_no_queries(K):
+    tree = K.rt_create(max_nodes=16, max_pool_tokens=16)
+    qt, qo = csr([[1, 2, 3], []])
+    m, node, off = gpu_match(K, tree, qt, qo)
+    assert m.tolist() == [0, 0] and node.tolist() == [0, 0]
+    K.rt_match_batch(tree, dev(qt), dev(torch.zeros(1, dtype=torch.int64)), torch.empty(0, dtype=torch.int32, device="cuda"))
+    assert K.rt_sync_status(tree) == 0
+
+
+@pytest.mark.parametrize("name,scale", [("medium", 1 / 64), ("hierarchical", 1 / 512), ("adversarial", 1 / 1024)])
+def test_match_scaled_configs(K, name, scale):
+    w = W.WORKLOADS[name](scale=scale)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    check_match(K, pt, po, qt, qo)
+
+
+# ------------------------------------------------------------------ insert
+
+@pytest.mark.parametrize("budget", [0, 60])
+def test_insert_new_tokens_and_stats(K, budget):
+    prompts, _ = W.random_small_queue(9, 200, vocab=2, max_len=16, min_len=0)
+    pt, po = csr(prompts)
+    tree = K.rt_create(budget_tokens=budget, **caps(pt.numel(), n_prompts=len(prompts)))
+    new = torch.zeros(len(prompts), dtype=torch.int32, device="cuda")
+    half = len(prompts) // 2
+    K.rt_insert(tree, dev(pt), dev(po[:half + 1]), new[:half])
+    K.rt_insert(tree, dev(pt), dev(po[half:]), new[half:])
+    assert K.rt_sync_status(tree) == 0
+    ot = oracle.OracleTree(budget)
+    want = ot.insert(pt.numpy(), po.numpy())
+    assert np.array_equal(new.cpu().numpy(), want)
+    st, ost = K.rt_stats(tree), ot.stats()
+    for key in ("n_nodes", "tokens", "clock", "evictions"):
+        assert st[key] == ost[key], key
+    if budget:
+        assert ost["evictions"] > 0 and st["tokens"] <= budget
+    qs, _ = W.random_small_queue(10, 100, vocab=2, max_len=18)
+    m, _, _ = gpu_match(K, tree, *csr(qs))
+    qt, qo = csr(qs)
+    assert np.array_equal(m, ot.match(qt.numpy(), qo.numpy()))
+
+
+def test_capacity_and_budget_errors_are_reported_not_fatal(K):
+    pt, po = csr([[1, 2, 3, 4, 5, 6, 7, 8], [9, 9, 9]])
+    tree = K.rt_create(max_nodes=64, max_pool_tokens=4)
+    K.rt_insert(tree, dev(pt), dev(po))
+    assert K.rt_sync_status(tree) == K.RT_ERR_CAPACITY
+    tree2 = K.rt_create(max_nodes=64, max_pool_tokens=64, budget_tokens=5)
+    K.rt_insert(tree2, dev(pt), dev(po))
+    assert K.rt_sync_status(tree2) == K.RT_ERR_BUDGET
+    # the device is still usable
+    tree3 = K.rt_build(dev(pt), dev(po), max_nodes=64, max_pool_tokens=64)
+    m, _, _ = gpu_match(K, tree3, *csr([[1, 2, 3, 9]]))
+    assert m.tolist() == [3]
+
+
+def test_invalid_arguments(K):
+    with pytest.raises(K.KlpmError) as e:
+        K.rt_create(max_nodes=0, max_pool_tokens=10)
+    assert e.value.code == K.RT_ERR_INVALID
+    tree = K.rt_create(max_nodes=16, max_pool_tokens=16)
+    z = torch.zeros(4, dtype=torch.int32, device="cuda")
+    a = torch.zeros(4, dtype=torch.int64, device="cuda")
+    wmask = torch.ones(4, dtype=torch.uint8, device="cuda")
+    pick = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(K.KlpmError):
+        K.klpm_select(z, a, wmask, 0, K.make_params(K.POLICY_KLPM, k=0), pick)
+    with pytest.raises(K.KlpmError):
+        K.klpm_select(z, a, wmask, -1, K.make_params(K.POLICY_KLPM, k=2), pick)
+    with pytest.raises(ValueError):
+        K.rt_match_batch(tree, torch.zeros(4, dtype=torch.int32), a, z)     # CPU tensor: no CPU path
+
+
+# ------------------------------------------------------------------ selection (one decision)
+
+def select_by_definition(m, t, waiting, c, policy, k):
+    idx = [i for i in range(len(m)) if waiting[i]]
+    if not idx:
+        return -1
+    if policy == 0 or (policy == 2 and c % k == 0):
+        return min(idx, key=lambda i: (t[i], i))
+    return min(idx, key=lambda i: (-m[i], t[i], i))
+
+
+@pytest.mark.parametrize("n", [1, 33, 1000, 70001])
+def test_select_single_decision(K, n):
+    g = torch.Generator().manual_seed(n)
+    m = torch.randint(0, 6, (n,), generator=g, dtype=torch.int32)
+    t = torch.randint(0, 50, (n,), generator=g, dtype=torch.int64) * (1 << 33)
+    waiting = (torch.rand(n, generator=g) < 0.7).to(torch.uint8)
+    pick = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for policy, k, c in [(0, 1, 0), (1, 1, 5), (2, 3, 0), (2, 3, 1), (2, 3, 2), (2, 3, 3), (2, 1, 7)]:
+        K.klpm_select(dev(m), dev(t), dev(waiting), c, K.make_params(policy, k), pick)
+        assert int(pick.item()) == select_by_definition(m.tolist(), t.tolist(), waiting.tolist(), c, policy, k)
+    K.klpm_select(dev(m), dev(t), dev(torch.zeros(n, dtype=torch.uint8)), 1, K.make_params(1), pick)
+    assert int(pick.item()) == -1
+
+
+# ------------------------------------------------------------------ replay along a fixed order
+
+@pytest.mark.parametrize("budget", [0, 50])
+def test_replay_fixed_order(K, budget):
+    prompts, arr = W.random_small_queue(21, 150, vocab=2, max_len=16, min_len=1, max_gap=9)
+    prefill, _ = W.random_small_queue(22, 20, vocab=2, max_len=12, min_len=1)
+    qt, qo = csr(prompts)
+    pt, po = csr(prefill)
+    order = torch.randperm(len(prompts), generator=torch.Generator().manual_seed(1)).to(torch.int32)
+    tree = gpu_tree(K, pt, po, extra_prompts=len(prompts), extra_tokens=qt.numel(), budget=budget)
+    n = len(prompts)
+    unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    p = K.make_params(K.POLICY_FCFS, 1, c_num=1, c_den=3, start_tick=5)
+    K.klpm_replay(tree, dev(order), dev(qt), dev(qo), dev(torch.tensor(arr)), p, unc, ttft, comp)
+    assert K.rt_sync_status(tree) == 0
+    ot = oracle_tree(pt, po, budget)
+    ou, ottft, ocomp = oracle.replay(order.numpy(), qt.numpy(), qo.numpy(), arr, 1, 3, 5, oracle.CACHE_TREE, ot)
+    assert np.array_equal(unc.cpu().numpy(), ou)
+    assert np.array_equal(ttft.cpu().numpy(), ottft)
+    assert np.array_equal(comp.cpu().numpy(), ocomp)
+    assert K.rt_stats(tree)["evictions"] == ot.stats()["evictions"]
+
+
+# ------------------------------------------------------------------ the whole loop
+
+def run_gpu(K, pt, po, qt, qo, arr, policy, k, budget=0, start=0, c_num=0, c_den=1):
+    n = qo.numel() - 1
+    tree = gpu_tree(K, pt, po, extra_prompts=n, extra_tokens=qt.numel(), budget=budget)
+    order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    K.klpm_run(tree, dev(qt), dev(qo), dev(torch.as_tensor(arr, dtype=torch.int64)),
+               K.make_params(policy, k, c_num, c_den, start), order, unc, ttft, comp)
+    assert K.rt_sync_status(tree) == 0
+    st = K.rt_stats(tree)
+    K.rt_destroy(tree)
+    return order.cpu().numpy(), unc.cpu().numpy(), ttft.cpu().numpy(), comp.cpu().numpy(), st
+
+
+def run_oracle(pt, po, qt, qo, arr, policy, k, budget=0, start=0, c_num=0, c_den=1, tier=oracle.TIER_UPDATE):
+    ot = oracle_tree(pt, po, budget)
+    out = oracle.schedule(qt.numpy(), qo.numpy(), np.asarray(arr, dtype=np.int64), policy, k, c_num, c_den, start,
+                          oracle.CACHE_TREE, tier, ot)
+    return out + (ot.stats(),)
+
+
+def assert_same_schedule(got, want):
+    for g, w, name in zip(got[:4], want[:4], ("order", "uncached", "ttft", "completion")):
+        assert np.array_equal(g, w), name
+    for key in ("n_nodes", "tokens", "clock", "evictions"):
+        assert got[4][key] == want[4][key], key
+
+
+def test_run_toy_example_on_device(K):
+    """Section 4.2's toy example with the whole tree cached: LPM / 2-LPM order x1,x3,x2,x4, TTFT 10,15,25,30."""
+    prompts, arr = W.regular_arrival_shuffled_queue(4, 2, 5, 5, 0, [1, 2, 3, 4])
+    qt, qo = csr(prompts)
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    for policy, k in ((K.POLICY_LPM, 1), (K.POLICY_KLPM, 2)):
+        order, unc, ttft, comp, _ = run_gpu(K, *e, qt, qo, arr, policy, k)
+        assert order.tolist() == [0, 2, 1, 3] and ttft.tolist() == [10, 25, 15, 30]
+    order, unc, ttft, comp, _ = run_gpu(K, *e, qt, qo, arr, K.POLICY_FCFS, 1)
+    assert order.tolist() == [0, 1, 2, 3] and ttft.tolist() == [10, 20, 25, 30]
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("budget", [0, 48])
+def test_run_fuzz_small_alphabet(K, seed, budget):
+    """Tiny alphabet: ties, identical prompts, prompts that are prefixes of others, idle periods, eviction."""
+    prompts, arr = W.random_small_queue(seed + 700, 120, vocab=2, max_len=14, min_len=0, max_gap=5)
+    prefill, _ = W.random_small_queue(seed + 800, 12, vocab=2, max_len=10, min_len=1)
+    qt, qo = csr(prompts)
+    pt, po = csr(prefill)
+    for policy, k in ((0, 1), (1, 1), (2, 1), (2, 2), (2, 3), (2, 200)):
+        got = run_gpu(K, pt, po, qt, qo, arr, policy, k, budget=budget, c_num=1, c_den=2)
+        want = run_oracle(pt, po, qt, qo, arr, policy, k, budget=budget, c_num=1, c_den=2, tier=oracle.TIER_REMATCH)
+        assert_same_schedule(got, want)
+        ref = D.schedule(prompts, arr, policy, k, 1, 2, 0, D.TREE, prefill, budget)
+        assert got[0].tolist() == ref[0] and got[2].tolist() == ref[2]
+
+
+def test_run_tiny_config_full(K):
+    """Configuration 'tiny' as stated: 1,000 waiting queries, tree of 2,000 prompts, k = 2; oracle re-matches every pick."""
+    w = W.tiny()
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    got = run_gpu(K, pt, po, qt, qo, w.arrivals, K.POLICY_KLPM, 2, start=w.start_tick)
+    want = run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_KLPM, 2, start=w.start_tick, tier=oracle.TIER_REMATCH)
+    assert_same_schedule(got, want)
+    # unbounded tree cache: total uncached tokens = growth of the tree
+    assert int(got[1].sum()) == got[4]["tokens"] - int(oracle_tree(pt, po).stats()["tokens"])
+
+
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_run_medium_scaled(K, k):
+    w = W.medium(scale=1 / 32)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    got = run_gpu(K, pt, po, qt, qo, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick)
+    want = run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_KLPM, k, start=w.start_tick)
+    assert_same_schedule(got, want)
+
+
+@pytest.mark.parametrize("policy,k", [(0, 1), (1, 1), (2, 4)])
+def test_run_streaming_scaled_with_lru(K, policy, k):
+    """Poisson arrivals from an empty tree under a KV budget with LRU eviction; per-query integer TTFT."""
+    w = W.streaming(scale=1 / 100)
+    qt, qo = w.queries.materialize()
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    got = run_gpu(K, *e, qt, qo, w.arrivals, policy, k, budget=w.budget_tokens)
+    want = run_oracle(*e, qt, qo, w.arrivals, policy, k, budget=w.budget_tokens)
+    assert_same_schedule(got, want)
+    assert want[4]["evictions"] > 0
+
+
+@pytest.mark.parametrize("name,scale,k", [("hierarchical", 1 / 256, 4), ("adversarial", 1 / 512, 4)])
+def test_run_scaled_configs(K, name, scale, k):
+    w = W.WORKLOADS[name](scale=scale)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    got = run_gpu(K, pt, po, qt, qo, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick)
+    want = run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_KLPM, k, start=w.start_tick)
+    assert_same_schedule(got, want)
