@@ -58,8 +58,9 @@ typedef struct {
     int64_t start_tick;  /* tick at which processing starts (R of the "previous" query for the first pick) */
 } klpm_params;
 
-/* ---- radix tree of cached prompts (RadixAttention, Section 1: "stores the KV cache of processed
- *      queries ... by maintaining a radix tree", "least recently used (LRU) eviction") ---- */
+/* ---- radix tree of cached prompts (RadixAttention as Section 1 describes it: processed prompts are
+ *      kept in a radix tree so that later prompts reuse their shared prefixes; under a fixed memory
+ *      budget the least recently used entries are evicted) ---- */
 
 /* Create an empty tree.  Synchronous (allocates device memory). */
 rt_status rt_create(const rt_config* cfg, rt_tree** out);
@@ -74,12 +75,15 @@ rt_status rt_build(const int32_t* d_tokens, const int64_t* d_offsets, int32_t n_
  * logical clock advances by one, and (with a budget) least-recently-used leaves are evicted first to
  * make room.  d_new_tokens (nullable, int32[n]) receives |x_i| - match length at its own insertion.
  * If the device runs out of capacity the prompts before the failing one stay inserted and the tree
- * stays valid; the condition is reported by rt_sync_status. */
+ * stays valid; the condition is reported by rt_sync_status.
+ * When d_new_tokens is NULL, the tree has no budget and n >= 64, the prompts are inserted concurrently
+ * in rounds instead (same resulting set of cached prefixes and node boundaries; node numbering may
+ * differ from run to run); this form waits for `stream` between rounds. */
 rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n,
                     int32_t* d_new_tokens, void* stream);
 
-/* Batched longest-prefix match (Section 1.3: overlap(x, y); RadixAttention "matches them with new
- * incoming prompts"): d_match_len[i] = max over cached prompts y of overlap(q_i, y) = the longest
+/* Batched longest-prefix match (Section 1.3 defines overlap(x, y); Section 1 has the tree matched
+ * against each incoming prompt): d_match_len[i] = max over cached prompts y of overlap(q_i, y) = the longest
  * prefix of query i that lies on a root path of the tree, counted token by token (partial edges
  * count).  Read-only on the tree.  d_term_node / d_term_off (nullable, int32[nq]) receive where the
  * match ended: the node whose edge holds the last matched token (0 = root when nothing matched) and
@@ -93,6 +97,14 @@ rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const i
  * evictions: leaves evicted so far; pool_used: tokens appended to the pool so far. */
 rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* clock,
                    int64_t* evictions, int64_t* pool_used);
+
+/* Remember the tree as it is now (device-to-device copies of the node arrays, the child table and the
+ * counters; the token pool is append-only and is not copied).  One checkpoint per tree; a later call replaces it. */
+rt_status rt_checkpoint(rt_tree* tree, void* stream);
+
+/* Put the tree back to its last checkpoint, undoing every insertion and eviction since.
+ * RT_ERR_INVALID if there is no checkpoint. */
+rt_status rt_rollback(rt_tree* tree, void* stream);
 
 /* Wait for `stream` and return the tree's device-side status word (RT_OK or the first error recorded). */
 rt_status rt_sync_status(rt_tree* tree, void* stream);

@@ -54,6 +54,10 @@ _lib.rt_match_batch.restype = _i32
 _lib.rt_match_batch.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.rt_stats.restype = _i32
 _lib.rt_stats.argtypes = [_vp] + [ctypes.POINTER(_i64)] * 5
+_lib.rt_checkpoint.restype = _i32
+_lib.rt_checkpoint.argtypes = [_vp, _vp]
+_lib.rt_rollback.restype = _i32
+_lib.rt_rollback.argtypes = [_vp, _vp]
 _lib.rt_sync_status.restype = _i32
 _lib.rt_sync_status.argtypes = [_vp, _vp]
 _lib.rt_destroy.restype = _i32
@@ -66,7 +70,7 @@ _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_destroy", "klpm_select", "klpm_replay", "klpm_run"]
+           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_replay", "klpm_run"]
 
 
 def lib() -> ctypes.CDLL:
@@ -157,6 +161,14 @@ def rt_stats(tree: Tree) -> dict:
     v = [ctypes.c_int64() for _ in range(5)]
     _check(_lib.rt_stats(tree.handle, *[ctypes.byref(x) for x in v]), "rt_stats")
     return dict(n_nodes=v[0].value, tokens=v[1].value, clock=v[2].value, evictions=v[3].value, pool_used=v[4].value)
+
+
+def rt_checkpoint(tree: Tree) -> None:
+    _check(_lib.rt_checkpoint(tree.handle, _stream()), "rt_checkpoint")
+
+
+def rt_rollback(tree: Tree) -> None:
+    _check(_lib.rt_rollback(tree.handle, _stream()), "rt_rollback")
 
 
 def rt_sync_status(tree: Tree) -> int:

@@ -122,12 +122,13 @@ struct Term {
     int32_t node;   // node whose edge holds the last matched token (0 = root)
     int32_t off;    // tokens of that edge matched
     int64_t pos;    // pool index of the last matched token, -1 at the root
+    int32_t full;   // 1 if the match ends exactly at the end of that node's edge (or at the root)
 };
 
 // Longest prefix of q on a root path.  Warp-cooperative and warp-uniform.
 template <bool RO>
 __device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t len) {
-    Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1;
+    Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1; t.full = 1;
     if (len <= 0) return t;
     unsigned long long key = make_key(0, ld32<RO>(q));
     unsigned long long slot = hash64(key) & T.table_mask;
@@ -156,6 +157,7 @@ __device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t le
         t.node = c.child;
         t.off = i;
         t.pos = c.span_off + i - 1;     // i >= 1: the first token is the key
+        t.full = i == c.span_len;
         if (i < c.span_len || !has_next) return t;
         key = key2; slot = slot2; c = nx;
     }
@@ -667,6 +669,130 @@ run_kernel(TreeDev T, RunArgs A) {
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// bulk insertion of many prompts into a tree without a budget.  The set of node boundaries a radix tree
+// ends up with does not depend on the order in which prompts are stored, so prompts are inserted in
+// rounds: every pending prompt is walked from the root (read-only), then at most one prompt per edge
+// cuts that edge, and prompts that end at a node boundary add their leaves concurrently (the hash
+// table's compare-and-swap on the key decides between prompts that want the same child).
+// ------------------------------------------------------------------------------------------------
+struct BulkArgs {
+    const int32_t* tok; const int64_t* off;
+    const int32_t* pend_in; int32_t* pend_out; unsigned int* n_out;
+    int32_t* claim;                    // per node: lowest prompt index that wants to cut its edge
+    int32_t* pm; int32_t* pnode; int32_t* poff;   // per prompt: where its walk ended
+};
+
+__global__ void __launch_bounds__(256)
+bulk_walk_kernel(TreeDev T, BulkArgs A, unsigned n_pending) {
+    const int lane = threadIdx.x & 31;
+    const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
+        const int32_t i = __ldg(A.pend_in + p);
+        const int64_t lo = __ldg(A.off + i);
+        const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
+        Term t = walk<true>(T, A.tok + lo, len);
+        if (lane == 0 && !(t.m == len && t.full)) {
+            A.pm[i] = t.m; A.pnode[i] = t.node; A.poff[i] = t.full ? -1 : t.off;
+            if (!t.full) atomicMin(&A.claim[t.node], i);
+            A.pend_out[atomicAdd(A.n_out, 1u)] = i;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+bulk_apply_kernel(TreeDev T, BulkArgs A) {
+    const unsigned n_pending = *A.n_out;
+    const int lane = threadIdx.x & 31;
+    const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
+    TreeState* S = T.st;
+    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
+        const int32_t i = A.pend_out[p];
+        const int64_t lo = __ldg(A.off + i);
+        const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
+        const int32_t* x = A.tok + lo;
+        const int32_t m = A.pm[i], node = A.pnode[i], off = A.poff[i];
+        const int32_t unc = len - m;
+        int64_t dst = -1;
+        if (lane == 0) {
+            bool go = true;
+            int32_t end = node;
+            if (off >= 0) {                                 // the match ends inside node's edge: cut it
+                if (A.claim[node] != i) go = false;
+                else {
+                    A.claim[node] = 0x7fffffff;
+                    const long long u = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
+                    if (u >= T.max_nodes) { set_status(S, RT_ERR_CAPACITY); go = false; }
+                    else {
+                        atomicAdd((unsigned long long*)&S->live_nodes, 1ULL);
+                        const int32_t par = T.parent[node], ds = T.depth_start[node], sl = T.span_len[node];
+                        const int64_t so = T.span_off[node];
+                        T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
+                        T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
+                        long long slot = table_find(T, par, T.pool[so]);
+                        if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; }
+                        else set_status(S, RT_ERR_LIMIT);
+                        T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
+                        T.parent[node] = (int32_t)u;
+                        end = (int32_t)u;
+                        // (u, first token of the lower part) -> node : nobody else can want this key
+                        unsigned long long key = make_key(end, T.pool[so + off]);
+                        unsigned long long sl2 = hash64(key) & T.table_mask;
+                        for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+                            if (atomicCAS(&T.table[sl2].key, 0ULL, key) == 0ULL) {
+                                T.table[sl2].child = node; T.table[sl2].span_len = sl - off; T.table[sl2].span_off = so + off;
+                                break;
+                            }
+                            sl2 = (sl2 + 1) & T.table_mask;
+                        }
+                    }
+                }
+            }
+            if (go && unc > 0) {
+                unsigned long long key = make_key(end, __ldg(x + m));
+                unsigned long long sl2 = hash64(key) & T.table_mask;
+                long long won = -1;
+                for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+                    unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
+                    if (old == 0ULL) { won = (long long)sl2; break; }
+                    if (old == key) break;                  // another prompt of this round added that child
+                    sl2 = (sl2 + 1) & T.table_mask;
+                }
+                if (won >= 0) {
+                    const long long leaf = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
+                    const long long po = (long long)atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)unc);
+                    if (leaf >= T.max_nodes || po + unc > T.max_pool) {
+                        set_status(S, RT_ERR_CAPACITY);
+                        T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0;
+                    } else {
+                        T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
+                        T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
+                        T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
+                        atomicAdd(&T.nchild[end], 1);
+                        atomicAdd((unsigned long long*)&S->tokens_live, (unsigned long long)unc);
+                        atomicAdd((unsigned long long*)&S->live_nodes, 1ULL);
+                        dst = po;
+                    }
+                }
+            }
+        }
+        dst = __shfl_sync(FULL_MASK, dst, 0);
+        if (dst >= 0)
+            for (int32_t t = lane; t < unc; t += 32) T.pool[dst + t] = __ldg(x + m + t);
+    }
+}
+
+__global__ void bulk_iota_kernel(int32_t* p, int32_t n) {
+    int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = i;
+}
+__global__ void bulk_fill_kernel(int32_t* p, long long n, int32_t v) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+__global__ void bulk_finish_kernel(TreeState* S, long long n) { S->clock += n; }
+
 // slot order: bitonic sort of (arrival, index) pairs, padded to a power of two
 __global__ void rank_init_kernel(const int64_t* __restrict__ arrival, int32_t n, long long np2, long long* key, int32_t* idx) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -703,6 +829,14 @@ struct rt_tree {
     long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos; uint8_t* run_done;
     unsigned long long* run_partial; RunState* run_rs;
     int num_sms;
+    int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
+    // checkpoint (rt_checkpoint / rt_rollback): copies of everything a later call can modify
+    bool ck_valid;
+    int32_t *ck_parent, *ck_depth_start, *ck_span_len, *ck_nchild, *ck_clock_owner;
+    int64_t *ck_span_off, *ck_last_access;
+    uint8_t* ck_dead;
+    Entry* ck_table;
+    TreeState* ck_st;
 };
 
 namespace {
@@ -724,6 +858,10 @@ void free_tree(rt_tree* t) {
     cudaFree(d.table); cudaFree(d.pool); cudaFree(d.st); cudaFree(t->match_counter);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
     cudaFree(t->run_pos); cudaFree(t->run_done); cudaFree(t->run_partial); cudaFree(t->run_rs);
+    cudaFree(t->claim);
+    cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
+    cudaFree(t->ck_clock_owner); cudaFree(t->ck_span_off); cudaFree(t->ck_last_access); cudaFree(t->ck_dead);
+    cudaFree(t->ck_table); cudaFree(t->ck_st);
     delete t;
 }
 
@@ -751,6 +889,52 @@ bool params_ok(const klpm_params* p) {
 }
 
 SelectScratch* g_select_scratch[64] = {nullptr};
+
+// Many prompts at once into a tree without a budget (see the bulk kernels).  Waits for the stream once per round.
+rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s) {
+    int32_t *pend_a = nullptr, *pend_b = nullptr, *pm = nullptr, *pnode = nullptr, *poff = nullptr;
+    unsigned int* n_out = nullptr;
+    rt_status st = RT_OK;
+    if ((st = dalloc(&pend_a, n)) || (st = dalloc(&pend_b, n)) || (st = dalloc(&pm, n)) || (st = dalloc(&pnode, n)) ||
+        (st = dalloc(&poff, n)) || (st = dalloc(&n_out, 1))) {
+        cudaFree(pend_a); cudaFree(pend_b); cudaFree(pm); cudaFree(pnode); cudaFree(poff); cudaFree(n_out);
+        return st;
+    }
+    bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(pend_a, n);
+    unsigned count = (unsigned)n;
+    cudaError_t e = cudaGetLastError();
+    int rounds = 0;
+    while (e == cudaSuccess && count > 0) {
+        if (++rounds > 1000000) { st = RT_ERR_LIMIT; break; }
+        BulkArgs a;
+        a.tok = d_tokens; a.off = d_offsets; a.pend_in = pend_a; a.pend_out = pend_b; a.n_out = n_out;
+        a.claim = t->claim; a.pm = pm; a.pnode = pnode; a.poff = poff;
+        long long blocks = ((long long)count + 7) / 8;
+        if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
+        e = cudaMemsetAsync(n_out, 0, sizeof(unsigned), s);
+        if (e != cudaSuccess) break;
+        bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
+        bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) break;
+        e = cudaMemcpyAsync(&count, n_out, sizeof(unsigned), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        int32_t* tmp = pend_a; pend_a = pend_b; pend_b = tmp;
+        if (e == cudaSuccess && count > 0) {
+            TreeState h;
+            e = cudaMemcpy(&h, t->dev.st, sizeof(h), cudaMemcpyDeviceToHost);
+            if (e == cudaSuccess && h.status != 0) break;      // capacity ran out: stop, the status word says why
+        }
+    }
+    if (e == cudaSuccess && st == RT_OK) {
+        bulk_finish_kernel<<<1, 1, 0, s>>>(t->dev.st, (long long)n);
+        e = cudaGetLastError();
+    }
+    cudaStreamSynchronize(s);
+    cudaFree(pend_a); cudaFree(pend_b); cudaFree(pm); cudaFree(pnode); cudaFree(poff); cudaFree(n_out);
+    if (e != cudaSuccess) { fprintf(stderr, "klpm: bulk insert failed: %s\n", cudaGetErrorString(e)); return RT_ERR_CUDA; }
+    return st;
+}
 
 }  // namespace
 
@@ -781,7 +965,8 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
         (s = dalloc(&d.span_off, d.max_nodes)) || (s = dalloc(&d.last_access, d.max_nodes)) ||
         (s = dalloc(&d.dead, d.max_nodes)) || (s = dalloc(&d.clock_owner, d.max_clock)) ||
         (s = dalloc(&d.table, cap)) || (s = dalloc(&d.pool, d.max_pool)) || (s = dalloc(&d.st, 1)) ||
-        (s = dalloc(&t->match_counter, 1)) || (s = dalloc(&t->run_partial, 1024)) || (s = dalloc(&t->run_rs, 1))) {
+        (s = dalloc(&t->match_counter, 1)) || (s = dalloc(&t->run_partial, 1024)) || (s = dalloc(&t->run_rs, 1)) ||
+        (s = dalloc(&t->claim, d.max_nodes))) {
         free_tree(t);
         return s;
     }
@@ -795,6 +980,10 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
     if (e == cudaSuccess) e = cudaMemset(d.span_off, 0, sizeof(int64_t));
     if (e == cudaSuccess) e = cudaMemset(d.last_access, 0, sizeof(int64_t));
     if (e == cudaSuccess) e = cudaMemset(d.dead, 0, 1);
+    if (e == cudaSuccess) {
+        bulk_fill_kernel<<<(unsigned)((d.max_nodes + 255) / 256), 256>>>(t->claim, d.max_nodes, 0x7fffffff);
+        e = cudaGetLastError();
+    }
     TreeState st0;
     memset(&st0, 0, sizeof(st0));
     st0.n_nodes = 1;
@@ -821,6 +1010,10 @@ rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_off
                     int32_t* d_new_tokens, void* stream) {
     if (!tree || n < 0 || (n > 0 && (!d_tokens || !d_offsets))) return RT_ERR_INVALID;
     if (n == 0) return RT_OK;
+    if (!d_new_tokens && tree->cfg.budget_tokens == 0 && n >= 64) {
+        tree->last_stream = (cudaStream_t)stream;
+        return bulk_insert(tree, d_tokens, d_offsets, n, (cudaStream_t)stream);
+    }
     SeqArgs a;
     memset(&a, 0, sizeof(a));
     a.tok = d_tokens; a.off = d_offsets; a.n = n; a.new_tokens = d_new_tokens; a.c_den = 1;
@@ -869,6 +1062,55 @@ rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* 
     if (clock) *clock = st.clock;
     if (evictions) *evictions = st.evictions;
     if (pool_used) *pool_used = st.pool_used;
+    return RT_OK;
+}
+
+rt_status rt_checkpoint(rt_tree* tree, void* stream) {
+    if (!tree) return RT_ERR_INVALID;
+    TreeDev& d = tree->dev;
+    const unsigned long long cap = d.table_mask + 1;
+    rt_status s = RT_OK;
+    if (!tree->ck_parent) {
+        if ((s = dalloc(&tree->ck_parent, d.max_nodes)) || (s = dalloc(&tree->ck_depth_start, d.max_nodes)) ||
+            (s = dalloc(&tree->ck_span_len, d.max_nodes)) || (s = dalloc(&tree->ck_nchild, d.max_nodes)) ||
+            (s = dalloc(&tree->ck_span_off, d.max_nodes)) || (s = dalloc(&tree->ck_last_access, d.max_nodes)) ||
+            (s = dalloc(&tree->ck_dead, d.max_nodes)) || (s = dalloc(&tree->ck_clock_owner, d.max_clock)) ||
+            (s = dalloc(&tree->ck_table, cap)) || (s = dalloc(&tree->ck_st, 1))) return s;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    tree->last_stream = st;
+    const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
+    CK(cudaMemcpyAsync(tree->ck_parent, d.parent, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_depth_start, d.depth_start, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_span_len, d.span_len, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_nchild, d.nchild, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_span_off, d.span_off, d.max_nodes * sizeof(int64_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_last_access, d.last_access, d.max_nodes * sizeof(int64_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_dead, d.dead, d.max_nodes, k, st));
+    CK(cudaMemcpyAsync(tree->ck_clock_owner, d.clock_owner, d.max_clock * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_table, d.table, cap * sizeof(Entry), k, st));
+    CK(cudaMemcpyAsync(tree->ck_st, d.st, sizeof(TreeState), k, st));
+    tree->ck_valid = true;
+    return RT_OK;
+}
+
+rt_status rt_rollback(rt_tree* tree, void* stream) {
+    if (!tree || !tree->ck_valid) return RT_ERR_INVALID;
+    TreeDev& d = tree->dev;
+    const unsigned long long cap = d.table_mask + 1;
+    cudaStream_t st = (cudaStream_t)stream;
+    tree->last_stream = st;
+    const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
+    CK(cudaMemcpyAsync(d.parent, tree->ck_parent, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(d.depth_start, tree->ck_depth_start, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(d.span_len, tree->ck_span_len, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(d.nchild, tree->ck_nchild, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(d.span_off, tree->ck_span_off, d.max_nodes * sizeof(int64_t), k, st));
+    CK(cudaMemcpyAsync(d.last_access, tree->ck_last_access, d.max_nodes * sizeof(int64_t), k, st));
+    CK(cudaMemcpyAsync(d.dead, tree->ck_dead, d.max_nodes, k, st));
+    CK(cudaMemcpyAsync(d.clock_owner, tree->ck_clock_owner, d.max_clock * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(d.table, tree->ck_table, cap * sizeof(Entry), k, st));
+    CK(cudaMemcpyAsync(d.st, tree->ck_st, sizeof(TreeState), k, st));
     return RT_OK;
 }
 

@@ -319,3 +319,66 @@ def test_run_scaled_configs(K, name, scale, k):
     got = run_gpu(K, pt, po, qt, qo, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick)
     want = run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_KLPM, k, start=w.start_tick)
     assert_same_schedule(got, want)
+
+
+# ------------------------------------------------------------------ bulk insertion, checkpoint / rollback
+
+@pytest.mark.parametrize("seed", range(3))
+def test_bulk_insert_equals_sequential_insert(K, seed):
+    """Concurrent insertion in rounds gives the same cached prefixes and node boundaries as one-by-one."""
+    prompts, _ = W.random_small_queue(seed + 900, 700, vocab=2, max_len=40, min_len=0)
+    prompts += [[1] * 300, [1] * 300, [1] * 150, [1] * 299 + [0], []]
+    pt, po = csr(prompts)
+    c = caps(pt.numel(), n_prompts=len(prompts))
+    bulk = K.rt_build(dev(pt), dev(po), **c)                       # n >= 64, no budget: rounds
+    seq = K.rt_create(**c)
+    new = torch.zeros(len(prompts), dtype=torch.int32, device="cuda")
+    K.rt_insert(seq, dev(pt), dev(po), new)                        # asks for new_tokens: one by one
+    assert K.rt_sync_status(bulk) == 0 and K.rt_sync_status(seq) == 0
+    a, b = K.rt_stats(bulk), K.rt_stats(seq)
+    ost = oracle_tree(pt, po).stats()
+    for key in ("n_nodes", "tokens", "clock"):
+        assert a[key] == b[key] == ost[key], key
+    qs, _ = W.random_small_queue(seed + 950, 300, vocab=2, max_len=45)
+    qt, qo = csr(qs)
+    ma, _, _ = gpu_match(K, bulk, qt, qo)
+    mb, _, _ = gpu_match(K, seq, qt, qo)
+    assert np.array_equal(ma, mb)
+    # a second bulk batch on top of the first
+    more, _ = W.random_small_queue(seed + 960, 200, vocab=2, max_len=40, min_len=1)
+    mt, mo = csr(more)
+    big = K.rt_build(dev(pt), dev(po), **caps(pt.numel(), mt.numel(), n_prompts=len(prompts) + len(more)))
+    K.rt_insert(big, dev(mt), dev(mo))
+    ot = oracle_tree(pt, po)
+    ot.insert(mt.numpy(), mo.numpy())
+    st = K.rt_stats(big)
+    assert (st["n_nodes"], st["tokens"], st["clock"]) == (ot.stats()["n_nodes"], ot.stats()["tokens"], ot.stats()["clock"])
+    m, _, _ = gpu_match(K, big, qt, qo)
+    assert np.array_equal(m, ot.match(qt.numpy(), qo.numpy()))
+
+
+def test_checkpoint_and_rollback(K):
+    w = W.medium(scale=1 / 128)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    n = qo.numel() - 1
+    tree = gpu_tree(K, pt, po, extra_prompts=2 * n, extra_tokens=2 * qt.numel())
+    K.rt_checkpoint(tree)
+    before = K.rt_stats(tree)
+    outs = []
+    for _ in range(2):
+        order = torch.zeros(n, dtype=torch.int32, device="cuda")
+        unc = torch.zeros(n, dtype=torch.int32, device="cuda")
+        ttft = torch.zeros(n, dtype=torch.int64, device="cuda")
+        K.klpm_run(tree, dev(qt), dev(qo), dev(w.arrivals), K.make_params(K.POLICY_KLPM, 4, start_tick=w.start_tick),
+                   order, unc, ttft)
+        assert K.rt_sync_status(tree) == 0
+        assert K.rt_stats(tree)["tokens"] > before["tokens"]
+        outs.append((order.cpu(), unc.cpu(), ttft.cpu()))
+        K.rt_rollback(tree)
+        after = K.rt_stats(tree)
+        assert {k: after[k] for k in ("n_nodes", "tokens", "clock")} == {k: before[k] for k in ("n_nodes", "tokens", "clock")}
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    m, _, _ = gpu_match(K, tree, qt, qo)
+    assert np.array_equal(m, oracle_tree(pt, po).match(qt.numpy(), qo.numpy()))
