@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the device-resident k-LPM scheduling path.
+
+One step = one pass of the whole path over one synthetic batch: batched longest-prefix match of every
+query of the stream against the cached radix tree (rt_match_batch), then the k-LPM scheduling loop until
+the queue drains (klpm_run: select, charge, insert, LRU, refresh).  The tree is put back to its
+checkpoint between steps (untimed).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--scale S] [--impl reference]
+
+Prints ONE JSON line.  `--impl reference` times the CPU oracle (as it stands) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2502_04677_b200 import workloads as W  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+DEFAULT_WORKLOAD = "adversarial"
+
+# dram bytes (read + write) per launch of the match kernel from an ncu capture, keyed by (workload, scale);
+# filled in from profiles/ once captured, None while the kernel has changed since
+TRAFFIC = {}
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                for name, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def _distinct_bound(sp: W.SegmentedPrompts) -> int:
+    """Upper bound on distinct tokens a set of segmented prompts can put in a tree: every stream window once."""
+    total = 0
+    prev_end = None
+    for key, end in zip(sp.seg_key, sp.seg_end):
+        length = end if prev_end is None else end - prev_end
+        if key.numel() == 0:
+            return 0
+        order = torch.argsort(key)
+        ks, ls = key[order], length[order]
+        uniq, inv = torch.unique_consecutive(ks, return_inverse=True)
+        mx = torch.zeros(uniq.numel(), dtype=torch.int64).scatter_reduce_(0, inv, ls, "amax", include_self=True)
+        total += int(mx.sum())
+        prev_end = end
+    return total
+
+
+def device_workload(w: W.Workload, device, build_chunk_tokens: int = 1 << 30):
+    """Materialise the workload on the device: tree (built by the library), queries, arrivals."""
+    from paper_2502_04677_b200 import binding as K
+    nq = w.queries.n
+    q_total = w.queries.total_tokens()
+    pre_total = w.prefill.total_tokens()
+    pre_n = w.prefill.n
+    max_nodes = 2 * (pre_n + nq) + 64           # every processed prompt adds at most two nodes
+    if w.budget_tokens > 0:                     # evicted prefixes are appended again when they come back
+        max_pool = pre_total + q_total + 1024
+    else:                                       # the pool only receives uncached tails
+        max_pool = min(pre_total, _distinct_bound(w.prefill)) + min(q_total, _distinct_bound(w.queries)) + 1024
+    tree = K.rt_create(max_nodes=max_nodes, max_pool_tokens=max_pool, budget_tokens=w.budget_tokens, vocab=w.vocab,
+                       max_clock=pre_n + nq + 64)
+    a = 0
+    off_all = w.prefill.offsets()
+    while a < pre_n:
+        limit = int(off_all[a]) + build_chunk_tokens
+        b = int(torch.searchsorted(off_all, torch.tensor(limit), right=True)) - 1
+        b = max(a + 1, min(b, pre_n))
+        tok, off = w.prefill.materialize(device, a, b)
+        K.rt_insert(tree, tok, off.to(device))
+        st = K.rt_sync_status(tree)
+        if st != 0:
+            raise RuntimeError("tree build failed with status %d" % st)
+        del tok
+        a = b
+    q_tok = torch.empty(q_total, dtype=torch.int32, device=device)
+    w.queries.materialize_into(q_tok, 0, nq)
+    q_off = w.queries.offsets().to(device)
+    arr = w.arrivals.to(device)
+    K.rt_checkpoint(tree)
+    torch.cuda.synchronize()
+    return tree, q_tok, q_off, arr
+
+
+def pick_k(name: str, w: W.Workload, k_arg: int) -> int:
+    if k_arg > 0:
+        return k_arg
+    return 4 if name == "medium" else w.ks[0]
+
+
+def run_ours(args):
+    rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
+    multi = world > 1
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if multi:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2502_04677_b200 import binding as K
+
+    name = args.workload
+    maker = W.WORKLOADS[name]
+    kw = {} if name == "tiny" else {"scale": args.scale}
+    # weak scaling: every rank schedules its own stream (same recipe, its own seed) against its own tree
+    seed = maker(**kw).recipe["seed"] + 1000 * rank
+    w = maker(seed=seed, **kw)
+    k = pick_k(name, w, args.k)
+    nq = w.queries.n
+    t_setup = time.perf_counter()
+    tree, q_tok, q_off, arr = device_workload(w, device)
+    t_setup = time.perf_counter() - t_setup
+    stats0 = K.rt_stats(tree)
+    params = K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick)
+
+    match_len = torch.zeros(nq, dtype=torch.int32, device=device)
+    order = torch.zeros(nq, dtype=torch.int32, device=device)
+    unc = torch.zeros(nq, dtype=torch.int32, device=device)
+    ttft = torch.zeros(nq, dtype=torch.int64, device=device)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        K.rt_rollback(tree)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(stream)
+        K.rt_match_batch(tree, q_tok, q_off, match_len)
+        ev[1].record(stream)
+        K.klpm_run(tree, q_tok, q_off, arr, params, order, unc, ttft)
+        ev[2].record(stream)
+        return ev
+
+    def barrier():
+        if multi:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    events = [step() for _ in range(args.steps)]
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    status = K.rt_sync_status(tree)
+    if status != 0:
+        raise RuntimeError("device status %d" % status)
+    t_match = sum(e[0].elapsed_time(e[1]) for e in events) / 1e3
+    t_run = sum(e[1].elapsed_time(e[2]) for e in events) / 1e3
+    t_total = t_match + t_run
+
+    # algorithmic bytes of the match kernel: both streams read once up to and including the first mismatch
+    qlen = q_off[1:] - q_off[:-1]
+    cmp_tokens = int(torch.minimum(match_len.to(torch.int64) + 1, qlen).sum().item())
+    alg_bytes = 8 * cmp_tokens
+
+    # ---- end to end through the C ABI with host buffers: H2D of the step's inputs, D2H of its results
+    h_tok, h_off, h_arr = q_tok.cpu().pin_memory(), q_off.cpu().pin_memory(), arr.cpu().pin_memory()
+    h_match = torch.empty(nq, dtype=torch.int32).pin_memory()
+    h_order = torch.empty(nq, dtype=torch.int32).pin_memory()
+    h_unc = torch.empty(nq, dtype=torch.int32).pin_memory()
+    h_ttft = torch.empty(nq, dtype=torch.int64).pin_memory()
+    d_tok, d_off, d_arr = torch.empty_like(q_tok), torch.empty_like(q_off), torch.empty_like(arr)
+    e2e_t = []
+    for it in range(max(1, min(args.steps, 3)) + 1):
+        K.rt_rollback(tree)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        d_tok.copy_(h_tok, non_blocking=True)
+        d_off.copy_(h_off, non_blocking=True)
+        d_arr.copy_(h_arr, non_blocking=True)
+        K.rt_match_batch(tree, d_tok, d_off, match_len)
+        K.klpm_run(tree, d_tok, d_off, d_arr, params, order, unc, ttft)
+        h_match.copy_(match_len, non_blocking=True)
+        h_order.copy_(order, non_blocking=True)
+        h_unc.copy_(unc, non_blocking=True)
+        h_ttft.copy_(ttft, non_blocking=True)
+        b.record(stream)
+        barrier()
+        if it > 0:
+            e2e_t.append(a.elapsed_time(b) / 1e3)
+    e2e_s = sum(e2e_t) / len(e2e_t)
+    h2d = h_tok.numel() * 4 + h_off.numel() * 8 + h_arr.numel() * 8
+    d2h = nq * (4 + 4 + 4 + 8)
+
+    times = torch.tensor([t_total, t_match, t_run, e2e_s], dtype=torch.float64, device=device)
+    if multi:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)          # slowest rank decides
+    t_total, t_match, t_run, e2e_s = times.tolist()
+    stats1 = K.rt_stats(tree)
+    if rank != 0:
+        if multi:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    achieved = alg_bytes / (t_match / args.steps) / 1e9
+    np2 = 1
+    while np2 < nq:
+        np2 <<= 1
+    lg = np2.bit_length() - 1
+    launches_per_step = 1 + 1 + lg * (lg + 1) // 2 + 1      # match, slot keys, bitonic steps, scheduling loop
+    ttft_cpu = ttft.cpu()
+    out = {
+        "metric": "prefix_match_queries_per_sec",
+        "value": world * nq * args.steps / t_match,
+        "unit": "queries/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * t_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "decisions_per_sec": world * nq * args.steps / t_run,
+        "phases_ms_per_step": {"rt_match_batch": 1e3 * t_match / args.steps, "klpm_run": 1e3 * t_run / args.steps},
+        "config": {"workload": name, "scale": args.scale if name != "tiny" else 1.0, "k": k, "policy": "k-LPM",
+                   "queries": nq, "query_tokens": int(q_tok.numel()), "tree_nodes": stats0["n_nodes"],
+                   "tree_tokens": stats0["tokens"], "budget_tokens": w.budget_tokens,
+                   "l2": "inputs larger than L2" if q_tok.numel() * 4 > 2 * 126e6 else "inputs smaller than L2",
+                   "seed": seed, "recipe": w.recipe, "setup_s": t_setup},
+        "roofline": {"bound": "hbm", "kernel": "match_batch_kernel", "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_of_nominal_8000": achieved / 8000.0,
+                     "algorithmic_bytes_per_launch": alg_bytes, "traffic": TRAFFIC.get((name, args.scale))},
+        "e2e": {"value": world * nq / e2e_s, "unit": "queries/s (whole step, copies included)",
+                "ms_per_step": 1e3 * e2e_s, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks,
+        "result": {"total_uncached_tokens": int(unc.sum().item()),
+                   "ttft_p50": int(ttft_cpu.kthvalue(max(1, nq // 2)).values), "ttft_max": int(ttft_cpu.max()),
+                   "tree_tokens_after": stats1["tokens"]},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(name, args.scale, k, budget_s=args.cpu_seconds)
+    print(json.dumps(out), flush=True)
+    if multi:
+        dist.destroy_process_group()
+
+
+def cpu_sample(name: str, scale: float, max_tokens: float = 3.0e8):
+    """A bounded sample of the workload for the CPU oracle: the same recipe at a reduced scale."""
+    maker = W.WORKLOADS[name]
+    if name == "tiny":
+        return maker(), 1.0
+    s = scale
+    while True:
+        w = maker(scale=s)
+        if w.prefill.total_tokens() + w.queries.total_tokens() <= max_tokens or s < 1e-4:
+            return w, s
+        s /= 2
+
+
+def cpu_baseline(name: str, scale: float, k: int, budget_s: float = 20.0):
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
+    import oracle
+    cores = os.cpu_count() or 1
+    w, s = cpu_sample(name, scale)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    tree = oracle.OracleTree(w.budget_tokens)
+    if w.prefill.n:
+        tree.insert(pt.numpy(), po.numpy())
+    qtn, qon = qt.numpy(), qo.numpy()
+    nq = w.queries.n
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        tree.match(qtn, qon, threads=cores)
+        reps += 1
+        if time.perf_counter() - t0 > budget_s / 4 or reps >= 50:
+            break
+    t_match = (time.perf_counter() - t0) / reps
+    t0 = time.perf_counter()
+    tree.match(qtn, qon, threads=1)
+    t_match_1 = time.perf_counter() - t0
+    # decisions/s of the scheduling loop (single thread: every pick depends on the previous one)
+    n_sched = min(nq, 4096)
+    sub = w.queries.select(torch.arange(n_sched))
+    st, so = sub.materialize()
+    arr = w.arrivals[:n_sched]
+    t0 = time.perf_counter()
+    oracle.schedule(st.numpy(), so.numpy(), arr.numpy(), oracle.POLICY_KLPM, k, 0, 1,
+                    int(arr.max()) if w.start_tick else 0, oracle.CACHE_TREE, oracle.TIER_UPDATE, tree)
+    t_sched = time.perf_counter() - t0
+    return {"value": nq / t_match, "unit": "queries/s", "cores": cores, "kind": "oracle",
+            "sample": "%s at scale %.6g: %d queries (%d tokens) against a tree of %d prompts; match on %d threads"
+                      % (name, s, nq, qt.numel(), w.prefill.n, cores),
+            "single_thread_queries_per_sec": nq / t_match_1,
+            "decisions_per_sec": n_sched / t_sched, "decisions_sample": n_sched}
+
+
+def run_reference(args):
+    """The CPU oracle through its own API on a bounded sample: each step = match + schedule of the sample."""
+    if env_int("RANK", 0) != 0:
+        return
+    import oracle
+    cores = os.cpu_count() or 1
+    name = args.workload
+    w, s = cpu_sample(name, args.scale, max_tokens=1.0e8)
+    k = pick_k(name, w, args.k)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    nq = w.queries.n
+    qtn, qon = qt.numpy(), qo.numpy()
+    n_sched = min(nq, 2048)
+    st, so = w.queries.select(torch.arange(n_sched)).materialize()
+    arr = w.arrivals[:n_sched]
+    t_match = t_total = 0.0
+    for it in range(args.warmup + args.steps):
+        tree = oracle.OracleTree(w.budget_tokens)
+        if w.prefill.n:
+            tree.insert(pt.numpy(), po.numpy())
+        t0 = time.perf_counter()
+        tree.match(qtn, qon, threads=cores)
+        t1 = time.perf_counter()
+        oracle.schedule(st.numpy(), so.numpy(), arr.numpy(), oracle.POLICY_KLPM, k, 0, 1,
+                        int(arr.max()) if w.start_tick else 0, oracle.CACHE_TREE, oracle.TIER_UPDATE, tree)
+        t2 = time.perf_counter()
+        if it >= args.warmup:
+            t_match += t1 - t0
+            t_total += t2 - t0
+        tree.close()
+    sample = ("%s at scale %.6g: %d queries matched on %d threads, %d of them scheduled (single thread)"
+              % (name, s, nq, cores, n_sched))
+    val = nq * args.steps / t_match
+    out = {"impl": "reference", "metric": "prefix_match_queries_per_sec", "value": val, "unit": "queries/s",
+           "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+           "config": {"workload": name, "scale": args.scale if name != "tiny" else 1.0, "k": k, "policy": "k-LPM"},
+           "decisions_per_sec": n_sched * args.steps / max(t_total - t_match, 1e-9),
+           "cpu_baseline": {"value": val, "unit": "queries/s", "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": val, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--k", type=int, default=0, help="k of k-LPM (0 = the configuration's own)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
