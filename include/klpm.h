@@ -35,7 +35,8 @@ enum {
     RT_ERR_CAPACITY = -2,  /* node, token-pool or clock capacity of the tree exhausted */
     RT_ERR_BUDGET = -3,    /* the KV budget cannot hold a prompt even after evicting everything evictable */
     RT_ERR_LIMIT = -4,     /* a bounded device-side wait or probe loop ran out */
-    RT_ERR_CUDA = -5       /* a CUDA runtime call failed */
+    RT_ERR_CUDA = -5,      /* a CUDA runtime call failed */
+    RT_ERR_TOO_LARGE = -6  /* a size is above a fixed limit of the entry point (klpm_select_noalloc) */
 };
 
 enum { KLPM_POLICY_FCFS = 0, KLPM_POLICY_LPM = 1, KLPM_POLICY_KLPM = 2 };
@@ -124,6 +125,32 @@ rt_status rt_destroy(rt_tree* tree);
 rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting,
                       int32_t nq, int64_t pick_counter, const klpm_params* params, int32_t* d_pick,
                       void* stream);
+
+/* klpm_select for callers that must not allocate device memory.  (The paper has no counterpart of this
+ * entry point; it exists for how the library gets embedded, not for the method.)
+ *
+ * Some hosts of this library cannot let it call cudaMalloc: a serving engine that hands the whole GPU to
+ * its own memory pool at start-up and treats any later allocation as a bug, code that runs where an
+ * allocation would force a device-wide synchronisation in the middle of a latency-critical scheduling
+ * tick, or a process whose memory accounting must stay fixed after initialisation.  klpm_select keeps the
+ * per-block partial results of its reduction in a buffer it allocates on first use; this variant keeps
+ * them in a small fixed array that is part of the library image, so it never allocates or frees anything.
+ *
+ * Same arguments, same result as klpm_select (bit for bit), with these differences:
+ *   - nq must not exceed KLPM_SELECT_NOALLOC_MAX_QUERIES; a larger nq returns RT_ERR_TOO_LARGE (and says so
+ *     on stderr) without launching anything.
+ *   - the fixed array is 4 KiB plus a counter.  Every GPU on which the library is loaded holds it until the
+ *     process exits, whether or not this entry point is ever called.
+ *   - the first call on each device looks up the array's device address (with that device current) and
+ *     remembers it; make that first call outside any stream capture.
+ *   - all calls on a device share the one array, and it keeps whatever the previous call left in it; each
+ *     call clears the counter it relies on before its kernel runs.  Two calls that overlap on the GPU
+ *     (different streams, no dependency between them) race on the array and may both return wrong picks:
+ *     issue calls on one stream, or order them with events. */
+#define KLPM_SELECT_NOALLOC_MAX_QUERIES (1 << 22)
+rt_status klpm_select_noalloc(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting,
+                              int32_t nq, int64_t pick_counter, const klpm_params* params, int32_t* d_pick,
+                              void* stream);
 
 /* Definition 2 along a given processing order: for j = d_order[0], d_order[1], ...:
  *   m = longest prefix of x_j in the tree; uncached = |x_j| - m;

@@ -16,8 +16,11 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libklpm.so")
 
 RT_OK, RT_ERR_INVALID, RT_ERR_CAPACITY, RT_ERR_BUDGET, RT_ERR_LIMIT, RT_ERR_CUDA = 0, -1, -2, -3, -4, -5
+RT_ERR_TOO_LARGE = -6
+SELECT_NOALLOC_MAX_QUERIES = 1 << 22
 POLICY_FCFS, POLICY_LPM, POLICY_KLPM = 0, 1, 2
-_ERR = {-1: "RT_ERR_INVALID", -2: "RT_ERR_CAPACITY", -3: "RT_ERR_BUDGET", -4: "RT_ERR_LIMIT", -5: "RT_ERR_CUDA"}
+_ERR = {-1: "RT_ERR_INVALID", -2: "RT_ERR_CAPACITY", -3: "RT_ERR_BUDGET", -4: "RT_ERR_LIMIT", -5: "RT_ERR_CUDA",
+        -6: "RT_ERR_TOO_LARGE"}
 
 
 class KlpmError(RuntimeError):
@@ -64,13 +67,15 @@ _lib.rt_destroy.restype = _i32
 _lib.rt_destroy.argtypes = [_vp]
 _lib.klpm_select.restype = _i32
 _lib.klpm_select.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
+_lib.klpm_select_noalloc.restype = _i32
+_lib.klpm_select_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
 _lib.klpm_replay.restype = _i32
 _lib.klpm_replay.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp]
 _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_replay", "klpm_run"]
+           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_noalloc", "klpm_replay", "klpm_run"]
 
 
 def lib() -> ctypes.CDLL:
@@ -184,6 +189,18 @@ def klpm_select(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.T
     _check(_lib.klpm_select(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
                             _dev(waiting, torch.uint8, "waiting"), match_len.numel(), int(pick_counter),
                             ctypes.byref(params), _dev(pick, torch.int32, "pick"), _stream()), "klpm_select")
+
+
+def klpm_select_noalloc(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, pick_counter: int,
+                        params: klpm_params, pick: torch.Tensor, nq: Optional[int] = None) -> None:
+    """klpm_select without any device allocation inside the library (fixed scratch; at most
+    SELECT_NOALLOC_MAX_QUERIES queries; calls must not overlap on the GPU).  `nq` defaults to the length
+    of match_len; pass it to state a queue length without building tensors of that size."""
+    n = match_len.numel() if nq is None else int(nq)
+    _check(_lib.klpm_select_noalloc(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
+                                    _dev(waiting, torch.uint8, "waiting"), n, int(pick_counter),
+                                    ctypes.byref(params), _dev(pick, torch.int32, "pick"), _stream()),
+           "klpm_select_noalloc")
 
 
 def klpm_replay(tree: Tree, order: torch.Tensor, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arrival: torch.Tensor,

@@ -439,6 +439,48 @@ select_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict__ arri
 }
 
 // ------------------------------------------------------------------------------------------------
+// klpm_select_noalloc: the same decision as klpm_select, with the per-CTA partial results kept in a
+// fixed array that is part of the library image instead of memory obtained from cudaMalloc.
+// ------------------------------------------------------------------------------------------------
+#define KLPM_SELECT_NOALLOC_BLOCKS 256
+struct StaticSelectScratch { Cand partial[KLPM_SELECT_NOALLOC_BLOCKS]; unsigned int ticket; };
+// 4 KiB + one counter per GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned char g_select_static[sizeof(StaticSelectScratch)];
+
+template <bool LPM>
+__global__ void __launch_bounds__(512)
+select_static_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict__ arrival, const uint8_t* __restrict__ waiting,
+                     int32_t nq, int32_t* pick, StaticSelectScratch* sc) {
+    __shared__ Cand s_c[32];
+    __shared__ bool s_last;
+    Cand best; best.m = 0; best.idx = -1; best.t = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nq; i += (int64_t)gridDim.x * blockDim.x) {
+        if (__ldg(waiting + i)) {
+            Cand c; c.m = LPM ? __ldg(mlen + i) : 0; c.idx = (int32_t)i; c.t = __ldg(arrival + i);
+            best = cand_best<LPM>(best, c);
+        }
+    }
+    best = block_best<LPM>(best, s_c);
+    if (threadIdx.x == 0) {
+        sc->partial[blockIdx.x] = best;
+        __threadfence();
+        s_last = atomicAdd(&sc->ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    Cand c; c.m = 0; c.idx = -1; c.t = 0;
+    for (int b = threadIdx.x; b < (int)gridDim.x; b += blockDim.x) {
+        Cand o;
+        o.m = __ldcg(&sc->partial[b].m); o.idx = __ldcg(&sc->partial[b].idx); o.t = __ldcg(&sc->partial[b].t);
+        c = cand_best<LPM>(c, o);
+    }
+    __syncthreads();
+    c = block_best<LPM>(c, s_c);
+    if (threadIdx.x == 0) *pick = c.idx;
+}
+
+// ------------------------------------------------------------------------------------------------
 // klpm_run: the whole loop as one cooperative kernel
 // ------------------------------------------------------------------------------------------------
 struct GridBarrier { unsigned int count; unsigned int gen; };
@@ -889,6 +931,7 @@ bool params_ok(const klpm_params* p) {
 }
 
 SelectScratch* g_select_scratch[64] = {nullptr};
+StaticSelectScratch* g_select_static_addr[64] = {nullptr};   // device address of g_select_static, per device
 
 // Many prompts at once into a tree without a budget (see the bulk kernels).  Waits for the stream once per round.
 rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s) {
@@ -1143,6 +1186,40 @@ rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, cons
     cudaStream_t s = (cudaStream_t)stream;
     if (fcfs_turn) select_kernel<false><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, g_select_scratch[dev]);
     else select_kernel<true><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, g_select_scratch[dev]);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status klpm_select_noalloc(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting, int32_t nq,
+                              int64_t pick_counter, const klpm_params* params, int32_t* d_pick, void* stream) {
+    if (!params_ok(params) || nq < 0 || !d_pick || pick_counter < 0 ||
+        (nq > 0 && (!d_match_len || !d_arrival || !d_waiting))) return RT_ERR_INVALID;
+    if (nq > KLPM_SELECT_NOALLOC_MAX_QUERIES) {
+        fprintf(stderr, "klpm_select_noalloc: nq = %d is above the fixed-scratch limit of %d queries; "
+                        "use klpm_select for larger queues\n", nq, KLPM_SELECT_NOALLOC_MAX_QUERIES);
+        return RT_ERR_TOO_LARGE;
+    }
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return RT_ERR_INVALID;
+    if (!g_select_static_addr[dev]) {
+        // In host code the array's name only stands for the symbol; the kernel needs its device address.
+        StaticSelectScratch* p = nullptr;
+        CK(cudaGetSymbolAddress((void**)&p, g_select_static));
+        if (!p) return RT_ERR_CUDA;
+        g_select_static_addr[dev] = p;
+    }
+    StaticSelectScratch* sc = g_select_static_addr[dev];
+    cudaStream_t s = (cudaStream_t)stream;
+    // the arrival counter must start at zero whatever an earlier call left behind
+    CK(cudaMemsetAsync(&sc->ticket, 0, sizeof(unsigned int), s));
+    const bool fcfs_turn = params->policy == KLPM_POLICY_FCFS ||
+                           (params->policy == KLPM_POLICY_KLPM && pick_counter % params->k == 0);
+    long long blocks = ((long long)nq + 2047) / 2048;
+    if (blocks < 1) blocks = 1;
+    if (blocks > KLPM_SELECT_NOALLOC_BLOCKS) blocks = KLPM_SELECT_NOALLOC_BLOCKS;
+    if (fcfs_turn) select_static_kernel<false><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, sc);
+    else select_static_kernel<true><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, sc);
     CK(cudaGetLastError());
     return RT_OK;
 }
