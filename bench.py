@@ -127,9 +127,10 @@ def device_workload(w: W.Workload, device, build_chunk_tokens: int = 1 << 30):
     pre_n = w.prefill.n
     max_nodes = 2 * (pre_n + nq) + 64           # every processed prompt adds at most two nodes
     if w.budget_tokens > 0:                     # evicted prefixes are appended again when they come back
-        max_pool = pre_total + q_total + 1024
+        max_pool = pre_total + q_total + 8 * (pre_n + nq) + 1024
     else:                                       # the pool only receives uncached tails
-        max_pool = min(pre_total, _distinct_bound(w.prefill)) + min(q_total, _distinct_bound(w.queries)) + 1024
+        max_pool = (min(pre_total, _distinct_bound(w.prefill)) + min(q_total, _distinct_bound(w.queries))
+                    + 8 * (pre_n + nq) + 1024)
     tree = K.rt_create(max_nodes=max_nodes, max_pool_tokens=max_pool, budget_tokens=w.budget_tokens, vocab=w.vocab,
                        max_clock=pre_n + nq + 64)
     a = 0

@@ -46,7 +46,8 @@ typedef struct rt_tree rt_tree; /* opaque; owned by the library from rt_build/rt
 typedef struct {
     int32_t vocab;            /* informational: token ids are expected in [0, vocab) */
     int64_t max_nodes;        /* capacity in tree nodes (every processed prompt adds at most 2) */
-    int64_t max_pool_tokens;  /* capacity of the append-only int32 token pool */
+    int64_t max_pool_tokens;  /* capacity of the append-only int32 token pool: the uncached tokens of every
+                                 stored prompt plus up to 8 tokens of alignment padding per prompt */
     int64_t budget_tokens;    /* KV-cache budget in tokens with LRU eviction; 0 = unbounded */
     int64_t max_clock;        /* capacity in processed prompts over the tree's life; 0 = max_nodes */
 } rt_config;

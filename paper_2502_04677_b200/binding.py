@@ -13,7 +13,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libklpm.so")
+LIB_PATH = os.environ.get("KLPM_LIB") or os.path.join(_HERE, "libklpm.so")
 
 RT_OK, RT_ERR_INVALID, RT_ERR_CAPACITY, RT_ERR_BUDGET, RT_ERR_LIMIT, RT_ERR_CUDA = 0, -1, -2, -3, -4, -5
 RT_ERR_TOO_LARGE = -6

@@ -34,7 +34,7 @@ struct alignas(32) Entry {
     int32_t child;            // node id, or -1 if the child was evicted (slot is reused on re-insert)
     int32_t span_len;
     int64_t span_off;
-    int64_t pad;
+    int64_t chain_end;        // pool index one past the contiguous pool run this edge is part of (see walk_chain)
 };
 
 struct TreeState {
@@ -61,6 +61,7 @@ struct TreeDev {
     Entry* table;
     unsigned long long table_mask;
     int32_t* pool;
+    int32_t* end_node;        // per pool index: id of the node whose edge ends with that token, else -1
     TreeState* st;
     long long max_nodes, max_pool, max_clock, budget;
 };
@@ -78,17 +79,19 @@ template <bool RO> __device__ __forceinline__ Entry ld_entry(const Entry* e) {
     r.child = a.z;
     r.span_len = a.w;
     r.span_off = (int64_t)(((unsigned long long)(unsigned)b.y << 32) | (unsigned)b.x);
-    r.pad = 0;
+    r.chain_end = (int64_t)(((unsigned long long)(unsigned)b.w << 32) | (unsigned)b.z);
     return r;
 }
 
 __device__ __forceinline__ unsigned long long make_key(int32_t parent, int32_t tok) {
     return ((unsigned long long)(unsigned)(parent + 1) << 32) | (unsigned)tok;
 }
-// 64-bit finaliser of MurmurHash3 (public domain, A. Appleby)
-__device__ __forceinline__ unsigned long long hash64(unsigned long long k) {
-    k ^= k >> 33; k *= 0xff51afd7ed558ccdULL; k ^= k >> 33; k *= 0xc4ceb9fe1a85ec53ULL; k ^= k >> 33;
-    return k;
+// Table hash: the two key halves are combined with the golden-ratio multiplier and run through the
+// 32-bit finaliser of MurmurHash3 (public domain, A. Appleby).  32-bit arithmetic keeps a hop cheap.
+__device__ __forceinline__ unsigned long long hash_key(unsigned long long k) {
+    unsigned h = (unsigned)(k >> 32) * 0x9E3779B1u + (unsigned)k;
+    h ^= h >> 16; h *= 0x85ebca6bu; h ^= h >> 13; h *= 0xc2b2ae35u; h ^= h >> 16;
+    return (unsigned long long)h;
 }
 
 __device__ __forceinline__ void set_status(TreeState* st, int code) { atomicCAS(&st->status, 0, code); }
@@ -131,7 +134,7 @@ __device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t le
     Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1; t.full = 1;
     if (len <= 0) return t;
     unsigned long long key = make_key(0, ld32<RO>(q));
-    unsigned long long slot = hash64(key) & T.table_mask;
+    unsigned long long slot = hash_key(key) & T.table_mask;
     Entry c = ld_entry<RO>(T.table + slot);
     for (;;) {
         unsigned probes = 0;
@@ -146,10 +149,10 @@ __device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t le
         const bool has_next = c.span_len < rem;
         // issue the probe of the next hop before comparing this edge: it depends only on this entry
         unsigned long long key2 = 0, slot2 = 0;
-        Entry nx; nx.key = 0; nx.child = -1; nx.span_len = 0; nx.span_off = 0;
+        Entry nx; nx.key = 0; nx.child = -1; nx.span_len = 0; nx.span_off = 0; nx.chain_end = 0;
         if (has_next) {
             key2 = make_key(c.child, ld32<RO>(q + t.m + c.span_len));
-            slot2 = hash64(key2) & T.table_mask;
+            slot2 = hash_key(key2) & T.table_mask;
             nx = ld_entry<RO>(T.table + slot2);
         }
         const int32_t i = first_mismatch<RO>(q + t.m, T.pool + c.span_off, n);
@@ -163,12 +166,147 @@ __device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t le
     }
 }
 
+// The walk of the read-only batched kernel on a tree that never evicts (no budget).
+//
+// A leaf's edge is written to the pool as one contiguous run, and later cuts only put node boundaries
+// inside that run: the pieces stay adjacent, each the one child of the previous for the token that
+// follows.  So a query that enters such a run at the start of a node matches exactly as far as it agrees
+// with the contiguous pool tokens, whatever the number of boundaries it crosses; no child lookup is needed
+// inside the run.  Every table entry carries chain_end, the pool index where its run ends, and
+// end_node[] tells whether a pool token is the last one of a node: a lookup is only made where the
+// comparison stops on a node boundary (another child may continue there) or the run is exhausted.
+// The comparison itself is a stream: 128-bit loads of both sides, two 128-token chunks in flight.
+//
+// Coordinates are depths (token positions in the query).  Every edge is placed so that
+// span_off = depth_start (mod 4), hence the pool tokens of depths 4i..4i+3 are one aligned 128-bit load.
+// The query side is read with aligned 128-bit loads too and shifted across lanes when the query does not
+// start on a 16-byte boundary.  The 16-byte units that hold the query's first and last token are read
+// whole: the token buffer must be 16-byte aligned (as cudaMalloc'd memory is).
+struct QWin {
+    const int32_t* qa;   // q rounded down to 16 bytes
+    int32_t s;           // tokens q is past that boundary (0..3)
+    int32_t len;
+};
+
+// tokens of depths cb + 4 lane .. + 3 (cb a multiple of 4); zeros where nothing needs to be read
+__device__ __forceinline__ int4 qwin_load(const QWin& Q, int32_t cb, int lane) {
+    const int4 z = make_int4(0, 0, 0, 0);
+    const int32_t p0 = cb + 4 * lane;
+    int4 v = (p0 - Q.s < Q.len) ? __ldg(reinterpret_cast<const int4*>(Q.qa + p0)) : z;
+    if (Q.s == 0) return v;                                            // warp-uniform
+    int4 e = (cb + 128 - Q.s < Q.len) ? __ldg(reinterpret_cast<const int4*>(Q.qa + cb + 128)) : z;
+    int4 n;
+    n.x = __shfl_down_sync(FULL_MASK, v.x, 1); n.y = __shfl_down_sync(FULL_MASK, v.y, 1); n.z = __shfl_down_sync(FULL_MASK, v.z, 1);
+    if (lane == 31) { n.x = e.x; n.y = e.y; n.z = e.z; }
+    if (Q.s == 1) return make_int4(v.y, v.z, v.w, n.x);
+    if (Q.s == 2) return make_int4(v.z, v.w, n.x, n.y);
+    return make_int4(v.w, n.x, n.y, n.z);
+}
+
+// First depth >= lo of this 128-token chunk (lane l: depths p0 .. p0+3) where A and P differ, or -1.
+__device__ __forceinline__ int32_t chunk_mismatch(const int4& A, const int4& P, int32_t p0, int32_t lo) {
+    int32_t dx = P.x ^ A.x, dy = P.y ^ A.y, dz = P.z ^ A.z, dw = P.w ^ A.w;
+    const int32_t hm = lo - p0;                     // leading tokens of this lane that are before lo
+    if (hm > 0) dx = 0;
+    if (hm > 1) dy = 0;
+    if (hm > 2) dz = 0;
+    const int32_t fc = dx ? 0 : dy ? 1 : dz ? 2 : dw ? 3 : 4;
+    const unsigned bad = __ballot_sync(FULL_MASK, fc < 4);
+    if (!bad) return -1;
+    const int L = __ffs(bad) - 1;
+    return __shfl_sync(FULL_MASK, p0 + fc, L);
+}
+
+// First depth in [lo, hi) where the query differs from pool_d[depth], or hi.  pool_d is the pool pointer
+// shifted so that pool_d[p] pairs with depth p; it is 16-byte aligned.
+__device__ __forceinline__ int32_t compare_run(const QWin& Q, const int32_t* __restrict__ pool_d, int32_t lo, int32_t hi, int lane) {
+    const int4* __restrict__ pool4 = reinterpret_cast<const int4*>(pool_d);
+    for (int32_t cb = lo & ~127; cb < hi; cb += 256) {
+        const int32_t p0 = cb + 4 * lane, p1 = p0 + 128;
+        const bool two = cb + 128 < hi;                                 // warp-uniform
+        int4 A0 = qwin_load(Q, cb, lane);
+        int4 A1 = A0;
+        if (two) A1 = qwin_load(Q, cb + 128, lane);
+        int4 P0 = A0, P1 = A1;
+        if (p0 + 4 > lo && p0 < hi) P0 = __ldg(pool4 + (p0 >> 2));
+        if (two && p1 < hi) P1 = __ldg(pool4 + (p1 >> 2));
+        int32_t r = chunk_mismatch(A0, P0, p0, lo);
+        if (r >= 0) return r < hi ? r : hi;
+        if (two) {
+            r = chunk_mismatch(A1, P1, p1, lo);
+            if (r >= 0) return r < hi ? r : hi;
+        }
+    }
+    return hi;
+}
+
+// id of the live node whose edge ends with pool token `pos`, or -1.  Entries of end_node[] can be stale
+// after a rollback, so a candidate is checked against the node arrays.
+__device__ __forceinline__ int32_t node_ending_at(const TreeDev& T, int64_t pos, long long n_nodes) {
+    const int32_t e = __ldg(T.end_node + pos);
+    if (e <= 0 || e >= n_nodes) return -1;
+    if (__ldg(T.span_off + e) + __ldg(T.span_len + e) - 1 != pos || __ldg(T.dead + e)) return -1;
+    return e;
+}
+
+__device__ Term walk_chain(const TreeDev& T, const int32_t* __restrict__ q, int32_t len, bool want_node) {
+    const int lane = threadIdx.x & 31;
+    Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1; t.full = 1;
+    if (len <= 0) return t;
+    QWin Q;
+    Q.s = (int32_t)((reinterpret_cast<uintptr_t>(q) >> 2) & 3);
+    Q.qa = q - Q.s;
+    Q.len = len;
+    const long long n_nodes = *reinterpret_cast<const volatile long long*>(&T.st->n_nodes);
+    int32_t cur = 0;
+    int32_t tok = __ldg(q);
+    for (;;) {
+        const unsigned long long key = make_key(cur, tok);
+        unsigned long long slot = hash_key(key) & T.table_mask;
+        Entry c = ld_entry<true>(T.table + slot);
+        unsigned probes = 0;
+        while (c.key != key) {
+            if (c.key == 0ULL || ++probes > 4096u) return t;
+            slot = (slot + 1) & T.table_mask;
+            c = ld_entry<true>(T.table + slot);
+        }
+        if (c.child < 0) return t;
+        int64_t run = c.chain_end - c.span_off;
+        if (run > (int64_t)(len - t.m)) run = len - t.m;
+        const int32_t x = compare_run(Q, T.pool + (c.span_off - (int64_t)t.m), t.m, t.m + (int32_t)run, lane);
+        const int64_t pos = c.span_off + (x - t.m) - 1;        // x > t.m: the first token is the key
+        t.m = x;
+        t.pos = pos;
+        const int32_t e = node_ending_at(T, pos, n_nodes);
+        if (e < 0) {                                           // stopped inside an edge
+            t.full = 0;
+            t.node = c.child;
+            if (want_node) {                                   // the node whose end comes next in this run
+                int32_t found = -1;
+                for (int64_t p = pos + 1; found < 0 && p < c.chain_end; p += 32) {
+                    const int32_t cand = (p + lane < c.chain_end) ? node_ending_at(T, p + lane, n_nodes) : -1;
+                    const unsigned hit = __ballot_sync(FULL_MASK, cand >= 0);
+                    if (hit) found = __shfl_sync(FULL_MASK, cand, __ffs(hit) - 1);
+                }
+                if (found >= 0) { t.node = found; t.off = t.m - __ldg(T.depth_start + found); }
+            }
+            return t;
+        }
+        t.full = 1;
+        t.node = e;
+        if (want_node) t.off = __ldg(T.span_len + e);
+        if (t.m >= len) return t;
+        cur = e;
+        tok = __ldg(q + t.m);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // single-thread tree updates (callers serialise them)
 // ------------------------------------------------------------------------------------------------
 __device__ long long table_find(const TreeDev& T, int32_t parent, int32_t tok) {
     unsigned long long key = make_key(parent, tok);
-    unsigned long long slot = hash64(key) & T.table_mask;
+    unsigned long long slot = hash_key(key) & T.table_mask;
     for (unsigned long long probes = 0; probes <= T.table_mask; ++probes) {
         unsigned long long k = __ldcg(&T.table[slot].key);
         if (k == key) return (long long)slot;
@@ -178,14 +316,15 @@ __device__ long long table_find(const TreeDev& T, int32_t parent, int32_t tok) {
     return -1;
 }
 
-__device__ bool table_put(const TreeDev& T, int32_t parent, int32_t tok, int32_t child, int32_t span_len, int64_t span_off) {
+__device__ bool table_put(const TreeDev& T, int32_t parent, int32_t tok, int32_t child, int32_t span_len, int64_t span_off,
+                          int64_t chain_end) {
     unsigned long long key = make_key(parent, tok);
-    unsigned long long slot = hash64(key) & T.table_mask;
+    unsigned long long slot = hash_key(key) & T.table_mask;
     for (unsigned long long probes = 0; probes <= T.table_mask; ++probes) {
         unsigned long long k = __ldcg(&T.table[slot].key);
         if (k == key || k == 0ULL) {
             Entry* e = T.table + slot;
-            e->child = child; e->span_len = span_len; e->span_off = span_off; e->pad = 0;
+            e->child = child; e->span_len = span_len; e->span_off = span_off; e->chain_end = chain_end;
             e->key = key;
             return true;
         }
@@ -205,10 +344,12 @@ __device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o) {
     T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = off; T.span_len[u] = o;
     T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = T.last_access[v];
     long long slot = table_find(T, par, __ldcg(T.pool + off));
-    if (slot >= 0) { T.table[slot].child = u; T.table[slot].span_len = o; }
+    int64_t chain_end = off + len;
+    if (slot >= 0) { T.table[slot].child = u; T.table[slot].span_len = o; chain_end = T.table[slot].chain_end; }
     else set_status(S, RT_ERR_LIMIT);
     T.span_off[v] = off + o; T.span_len[v] = len - o; T.depth_start[v] = ds + o; T.parent[v] = u;
-    if (!table_put(T, u, __ldcg(T.pool + off + o), v, len - o, off + o)) set_status(S, RT_ERR_CAPACITY);
+    if (!table_put(T, u, __ldcg(T.pool + off + o), v, len - o, off + o, chain_end)) set_status(S, RT_ERR_CAPACITY);
+    T.end_node[off + o - 1] = u;
     return u;
 }
 
@@ -266,15 +407,16 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
         }
     }
     if (unc > 0) {
-        if (S->pool_used + unc > T.max_pool) { set_status(S, RT_ERR_CAPACITY); return; }
+        if (S->pool_used + unc + 6 > T.max_pool) { set_status(S, RT_ERR_CAPACITY); return; }
         int32_t leaf = (int32_t)S->n_nodes++;
-        int64_t off = S->pool_used;
-        S->pool_used += unc;
+        const int64_t off = ((S->pool_used + 3) & ~3LL) + (m & 3);    // span_off = depth_start (mod 4)
+        S->pool_used = off + unc;
         T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = off; T.span_len[leaf] = unc;
         T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = clock;
         T.clock_owner[clock] = leaf;
         T.nchild[end]++;
-        if (!table_put(T, end, __ldcg(x + m), leaf, unc, off)) { set_status(S, RT_ERR_CAPACITY); return; }
+        if (!table_put(T, end, __ldcg(x + m), leaf, unc, off, off + unc)) { set_status(S, RT_ERR_CAPACITY); return; }
+        T.end_node[off + unc - 1] = leaf;
         S->tokens_live += unc;
         S->live_nodes++;
         out->leaf = leaf; out->unc = unc; out->leaf_off = off;
@@ -285,10 +427,13 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
 // ------------------------------------------------------------------------------------------------
 // rt_match_batch
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+#ifndef KLPM_MATCH_MIN_BLOCKS
+#define KLPM_MATCH_MIN_BLOCKS 4
+#endif
+__global__ void __launch_bounds__(256, KLPM_MATCH_MIN_BLOCKS)
 match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
                    int32_t* __restrict__ mlen, int32_t* __restrict__ tnode, int32_t* __restrict__ toff,
-                   unsigned long long* counter) {
+                   unsigned long long* counter, int chain) {
     const int lane = threadIdx.x & 31;
     for (;;) {
         unsigned long long i = 0;
@@ -298,7 +443,8 @@ match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* _
         const int64_t lo = __ldg(qoff + i), hi = __ldg(qoff + i + 1);
         int64_t len = hi - lo;
         if (len < 0 || len > 0x7fffffffLL) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
-        Term t = walk<true>(T, qtok + lo, (int32_t)len);
+        Term t = chain ? walk_chain(T, qtok + lo, (int32_t)len, tnode != nullptr || toff != nullptr)
+                       : walk<true>(T, qtok + lo, (int32_t)len);
         if (lane == 0) {
             mlen[i] = t.m;
             if (tnode) tnode[i] = t.node;
@@ -773,17 +919,20 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                         T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
                         T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
                         long long slot = table_find(T, par, T.pool[so]);
-                        if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; }
+                        int64_t chain_end = so + sl;
+                        if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = T.table[slot].chain_end; }
                         else set_status(S, RT_ERR_LIMIT);
+                        T.end_node[so + off - 1] = (int32_t)u;
                         T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
                         T.parent[node] = (int32_t)u;
                         end = (int32_t)u;
                         // (u, first token of the lower part) -> node : nobody else can want this key
                         unsigned long long key = make_key(end, T.pool[so + off]);
-                        unsigned long long sl2 = hash64(key) & T.table_mask;
+                        unsigned long long sl2 = hash_key(key) & T.table_mask;
                         for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
                             if (atomicCAS(&T.table[sl2].key, 0ULL, key) == 0ULL) {
                                 T.table[sl2].child = node; T.table[sl2].span_len = sl - off; T.table[sl2].span_off = so + off;
+                                T.table[sl2].chain_end = chain_end;
                                 break;
                             }
                             sl2 = (sl2 + 1) & T.table_mask;
@@ -793,7 +942,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
             }
             if (go && unc > 0) {
                 unsigned long long key = make_key(end, __ldg(x + m));
-                unsigned long long sl2 = hash64(key) & T.table_mask;
+                unsigned long long sl2 = hash_key(key) & T.table_mask;
                 long long won = -1;
                 for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
                     unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
@@ -803,14 +952,17 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                 }
                 if (won >= 0) {
                     const long long leaf = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
-                    const long long po = (long long)atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)unc);
-                    if (leaf >= T.max_nodes || po + unc > T.max_pool) {
+                    const long long raw = (long long)atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)(unc + 6));
+                    const long long po = ((raw + 3) & ~3LL) + (m & 3);                  // span_off = depth_start (mod 4)
+                    if (leaf >= T.max_nodes || raw + unc + 6 > T.max_pool) {
                         set_status(S, RT_ERR_CAPACITY);
-                        T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0;
+                        T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0; T.table[won].chain_end = 0;
                     } else {
                         T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
                         T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
                         T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
+                        T.table[won].chain_end = po + unc;
+                        T.end_node[po + unc - 1] = (int32_t)leaf;
                         atomicAdd(&T.nchild[end], 1);
                         atomicAdd((unsigned long long*)&S->tokens_live, (unsigned long long)unc);
                         atomicAdd((unsigned long long*)&S->live_nodes, 1ULL);
@@ -897,7 +1049,7 @@ void free_tree(rt_tree* t) {
     TreeDev& d = t->dev;
     cudaFree(d.parent); cudaFree(d.depth_start); cudaFree(d.span_len); cudaFree(d.nchild);
     cudaFree(d.span_off); cudaFree(d.last_access); cudaFree(d.dead); cudaFree(d.clock_owner);
-    cudaFree(d.table); cudaFree(d.pool); cudaFree(d.st); cudaFree(t->match_counter);
+    cudaFree(d.table); cudaFree(d.pool); cudaFree(d.end_node); cudaFree(d.st); cudaFree(t->match_counter);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
     cudaFree(t->run_pos); cudaFree(t->run_done); cudaFree(t->run_partial); cudaFree(t->run_rs);
     cudaFree(t->claim);
@@ -1008,6 +1160,7 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
         (s = dalloc(&d.span_off, d.max_nodes)) || (s = dalloc(&d.last_access, d.max_nodes)) ||
         (s = dalloc(&d.dead, d.max_nodes)) || (s = dalloc(&d.clock_owner, d.max_clock)) ||
         (s = dalloc(&d.table, cap)) || (s = dalloc(&d.pool, d.max_pool)) || (s = dalloc(&d.st, 1)) ||
+        (s = dalloc(&d.end_node, d.max_pool)) ||
         (s = dalloc(&t->match_counter, 1)) || (s = dalloc(&t->run_partial, 1024)) || (s = dalloc(&t->run_rs, 1)) ||
         (s = dalloc(&t->claim, d.max_nodes))) {
         free_tree(t);
@@ -1015,6 +1168,7 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
     }
     // root: node 0, empty edge
     cudaError_t e = cudaMemset(d.table, 0, cap * sizeof(Entry));
+    if (e == cudaSuccess) e = cudaMemset(d.end_node, 0xff, d.max_pool * sizeof(int32_t) + 256);
     if (e == cudaSuccess) e = cudaMemset(d.clock_owner, 0, d.max_clock * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(d.parent, 0, sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(d.depth_start, 0, sizeof(int32_t));
@@ -1090,7 +1244,8 @@ rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const i
     long long max_blocks = (long long)tree->num_sms * 8;
     if (blocks > max_blocks) blocks = max_blocks;
     match_batch_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
-                                                           d_term_node, d_term_off, tree->match_counter);
+                                                           d_term_node, d_term_off, tree->match_counter,
+                                                           tree->cfg.budget_tokens == 0 ? 1 : 0);
     CK(cudaGetLastError());
     return RT_OK;
 }

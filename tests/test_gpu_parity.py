@@ -26,7 +26,7 @@ def csr(prompts):
 
 def caps(*token_counts, n_prompts=0):
     total = int(sum(token_counts))
-    return dict(max_nodes=2 * n_prompts + 16, max_pool_tokens=total + 16, max_clock=n_prompts + 16)
+    return dict(max_nodes=2 * n_prompts + 16, max_pool_tokens=total + 8 * n_prompts + 16, max_clock=n_prompts + 16)
 
 
 def gpu_tree(K, tokens, offsets, extra_prompts=0, extra_tokens=0, budget=0):
