@@ -218,23 +218,30 @@ __device__ __forceinline__ int32_t chunk_mismatch(const int4& A, const int4& P, 
 }
 
 // First depth in [lo, hi) where the query differs from pool_d[depth], or hi.  pool_d is the pool pointer
-// shifted so that pool_d[p] pairs with depth p; it is 16-byte aligned.
+// shifted so that pool_d[p] pairs with depth p; it is 16-byte aligned.  KLPM_MATCH_UNROLL chunks of 128
+// tokens are loaded from both sides before the first of them is examined.
+#ifndef KLPM_MATCH_UNROLL
+#define KLPM_MATCH_UNROLL 1
+#endif
 __device__ __forceinline__ int32_t compare_run(const QWin& Q, const int32_t* __restrict__ pool_d, int32_t lo, int32_t hi, int lane) {
+    constexpr int U = KLPM_MATCH_UNROLL;
     const int4* __restrict__ pool4 = reinterpret_cast<const int4*>(pool_d);
-    for (int32_t cb = lo & ~127; cb < hi; cb += 256) {
-        const int32_t p0 = cb + 4 * lane, p1 = p0 + 128;
-        const bool two = cb + 128 < hi;                                 // warp-uniform
-        int4 A0 = qwin_load(Q, cb, lane);
-        int4 A1 = A0;
-        if (two) A1 = qwin_load(Q, cb + 128, lane);
-        int4 P0 = A0, P1 = A1;
-        if (p0 + 4 > lo && p0 < hi) P0 = __ldg(pool4 + (p0 >> 2));
-        if (two && p1 < hi) P1 = __ldg(pool4 + (p1 >> 2));
-        int32_t r = chunk_mismatch(A0, P0, p0, lo);
-        if (r >= 0) return r < hi ? r : hi;
-        if (two) {
-            r = chunk_mismatch(A1, P1, p1, lo);
-            if (r >= 0) return r < hi ? r : hi;
+    for (int32_t cb = lo & ~127; cb < hi; cb += 128 * U) {
+        int4 A[U], P[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int32_t p = cb + 128 * u + 4 * lane;
+            A[u] = make_int4(0, 0, 0, 0);
+            if (cb + 128 * u < hi) A[u] = qwin_load(Q, cb + 128 * u, lane);      // warp-uniform condition
+            P[u] = A[u];
+            if (p + 4 > lo && p < hi) P[u] = __ldg(pool4 + (p >> 2));
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (cb + 128 * u < hi) {
+                const int32_t r = chunk_mismatch(A[u], P[u], cb + 128 * u + 4 * lane, lo);
+                if (r >= 0) return r < hi ? r : hi;
+            }
         }
     }
     return hi;
@@ -242,62 +249,71 @@ __device__ __forceinline__ int32_t compare_run(const QWin& Q, const int32_t* __r
 
 // id of the live node whose edge ends with pool token `pos`, or -1.  Entries of end_node[] can be stale
 // after a rollback, so a candidate is checked against the node arrays.
-__device__ __forceinline__ int32_t node_ending_at(const TreeDev& T, int64_t pos, long long n_nodes) {
-    const int32_t e = __ldg(T.end_node + pos);
+struct EndIndex {             // what is needed to resolve end_node[] entries, passed by value
+    const int32_t* end_node; const int64_t* span_off; const int32_t* span_len; const uint8_t* dead;
+    const TreeState* st;
+};
+__device__ __forceinline__ EndIndex end_index(const TreeDev& T) {
+    EndIndex X; X.end_node = T.end_node; X.span_off = T.span_off; X.span_len = T.span_len; X.dead = T.dead; X.st = T.st;
+    return X;
+}
+__device__ __forceinline__ int32_t node_ending_at(const EndIndex X, int64_t pos, long long n_nodes) {
+    const int32_t e = __ldg(X.end_node + pos);
     if (e <= 0 || e >= n_nodes) return -1;
-    if (__ldg(T.span_off + e) + __ldg(T.span_len + e) - 1 != pos || __ldg(T.dead + e)) return -1;
+    if (__ldg(X.span_off + e) + __ldg(X.span_len + e) - 1 != pos || __ldg(X.dead + e)) return -1;
     return e;
 }
 
-__device__ Term walk_chain(const TreeDev& T, const int32_t* __restrict__ q, int32_t len, bool want_node) {
+// The node of this run whose edge ends first after pool token `pos` (the match stopped inside its edge).
+__device__ __noinline__ int32_t node_after(const EndIndex X, int64_t pos, int64_t chain_end) {
     const int lane = threadIdx.x & 31;
-    Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1; t.full = 1;
-    if (len <= 0) return t;
+    const long long n_nodes = *reinterpret_cast<const volatile long long*>(&X.st->n_nodes);
+    for (int64_t p = pos + 1; p < chain_end; p += 32) {
+        const int32_t cand = (p + lane < chain_end) ? node_ending_at(X, p + lane, n_nodes) : -1;
+        const unsigned hit = __ballot_sync(FULL_MASK, cand >= 0);
+        if (hit) return __shfl_sync(FULL_MASK, cand, __ffs(hit) - 1);
+    }
+    return -1;
+}
+
+// Returns the match length; *node / *off (where the match ended) are filled when want_node is set.
+__device__ __forceinline__ int32_t walk_chain(const TreeDev& T, const int32_t* __restrict__ q, int32_t len, bool want_node,
+                              int32_t* node, int32_t* off) {
+    const int lane = threadIdx.x & 31;
+    *node = 0; *off = 0;
+    if (len <= 0) return 0;
     QWin Q;
     Q.s = (int32_t)((reinterpret_cast<uintptr_t>(q) >> 2) & 3);
     Q.qa = q - Q.s;
     Q.len = len;
-    const long long n_nodes = *reinterpret_cast<const volatile long long*>(&T.st->n_nodes);
-    int32_t cur = 0;
-    int32_t tok = __ldg(q);
+    int32_t m = 0, cur = 0;
     for (;;) {
-        const unsigned long long key = make_key(cur, tok);
+        const unsigned long long key = make_key(cur, __ldg(q + m));
         unsigned long long slot = hash_key(key) & T.table_mask;
         Entry c = ld_entry<true>(T.table + slot);
         unsigned probes = 0;
         while (c.key != key) {
-            if (c.key == 0ULL || ++probes > 4096u) return t;
+            if (c.key == 0ULL || ++probes > 4096u) return m;
             slot = (slot + 1) & T.table_mask;
             c = ld_entry<true>(T.table + slot);
         }
-        if (c.child < 0) return t;
+        if (c.child < 0) return m;
         int64_t run = c.chain_end - c.span_off;
-        if (run > (int64_t)(len - t.m)) run = len - t.m;
-        const int32_t x = compare_run(Q, T.pool + (c.span_off - (int64_t)t.m), t.m, t.m + (int32_t)run, lane);
-        const int64_t pos = c.span_off + (x - t.m) - 1;        // x > t.m: the first token is the key
-        t.m = x;
-        t.pos = pos;
-        const int32_t e = node_ending_at(T, pos, n_nodes);
+        if (run > (int64_t)(len - m)) run = len - m;
+        const int32_t x = compare_run(Q, T.pool + (c.span_off - (int64_t)m), m, m + (int32_t)run, lane);
+        const int64_t pos = c.span_off + (x - m) - 1;          // x > m: the first token is the key
+        m = x;
+        const int32_t e = node_ending_at(end_index(T), pos, *reinterpret_cast<const volatile long long*>(&T.st->n_nodes));
         if (e < 0) {                                           // stopped inside an edge
-            t.full = 0;
-            t.node = c.child;
-            if (want_node) {                                   // the node whose end comes next in this run
-                int32_t found = -1;
-                for (int64_t p = pos + 1; found < 0 && p < c.chain_end; p += 32) {
-                    const int32_t cand = (p + lane < c.chain_end) ? node_ending_at(T, p + lane, n_nodes) : -1;
-                    const unsigned hit = __ballot_sync(FULL_MASK, cand >= 0);
-                    if (hit) found = __shfl_sync(FULL_MASK, cand, __ffs(hit) - 1);
-                }
-                if (found >= 0) { t.node = found; t.off = t.m - __ldg(T.depth_start + found); }
+            if (want_node) {
+                const int32_t f = node_after(end_index(T), pos, c.chain_end);
+                if (f >= 0) { *node = f; *off = m - __ldg(T.depth_start + f); }
             }
-            return t;
+            return m;
         }
-        t.full = 1;
-        t.node = e;
-        if (want_node) t.off = __ldg(T.span_len + e);
-        if (t.m >= len) return t;
+        if (want_node) { *node = e; *off = __ldg(T.span_len + e); }
+        if (m >= len) return m;
         cur = e;
-        tok = __ldg(q + t.m);
     }
 }
 
@@ -428,12 +444,39 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
 // rt_match_batch
 // ------------------------------------------------------------------------------------------------
 #ifndef KLPM_MATCH_MIN_BLOCKS
-#define KLPM_MATCH_MIN_BLOCKS 4
+#define KLPM_MATCH_MIN_BLOCKS 8
 #endif
+// One warp per query, queries handed out by an atomic counter (persistent grid).
+// Trees without a budget: stream along contiguous pool runs.
 __global__ void __launch_bounds__(256, KLPM_MATCH_MIN_BLOCKS)
+match_chain_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
+                   int32_t* __restrict__ mlen, int32_t* __restrict__ tnode, int32_t* __restrict__ toff,
+                   unsigned long long* counter) {
+    const int lane = threadIdx.x & 31;
+    const bool want_node = tnode != nullptr || toff != nullptr;
+    for (;;) {
+        unsigned long long i = 0;
+        if (lane == 0) i = atomicAdd(counter, 1ULL);
+        i = __shfl_sync(FULL_MASK, i, 0);
+        if (i >= (unsigned long long)nq) return;
+        const int64_t lo = __ldg(qoff + i);
+        int64_t len = __ldg(qoff + i + 1) - lo;
+        if (len < 0 || len > 0x7fffffffLL) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
+        int32_t node, off;
+        const int32_t m = walk_chain(T, qtok + lo, (int32_t)len, want_node, &node, &off);
+        if (lane == 0) {
+            mlen[i] = m;
+            if (tnode) tnode[i] = node;
+            if (toff) toff[i] = off;
+        }
+    }
+}
+
+// Trees with a budget (evicted children break the runs): hop by hop.
+__global__ void __launch_bounds__(256)
 match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
                    int32_t* __restrict__ mlen, int32_t* __restrict__ tnode, int32_t* __restrict__ toff,
-                   unsigned long long* counter, int chain) {
+                   unsigned long long* counter) {
     const int lane = threadIdx.x & 31;
     for (;;) {
         unsigned long long i = 0;
@@ -443,8 +486,7 @@ match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* _
         const int64_t lo = __ldg(qoff + i), hi = __ldg(qoff + i + 1);
         int64_t len = hi - lo;
         if (len < 0 || len > 0x7fffffffLL) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
-        Term t = chain ? walk_chain(T, qtok + lo, (int32_t)len, tnode != nullptr || toff != nullptr)
-                       : walk<true>(T, qtok + lo, (int32_t)len);
+        Term t = walk<true>(T, qtok + lo, (int32_t)len);
         if (lane == 0) {
             mlen[i] = t.m;
             if (tnode) tnode[i] = t.node;
@@ -1243,9 +1285,12 @@ rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const i
     long long blocks = ((long long)nq + warps_per_block - 1) / warps_per_block;
     long long max_blocks = (long long)tree->num_sms * 8;
     if (blocks > max_blocks) blocks = max_blocks;
-    match_batch_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
-                                                           d_term_node, d_term_off, tree->match_counter,
-                                                           tree->cfg.budget_tokens == 0 ? 1 : 0);
+    if (tree->cfg.budget_tokens == 0)
+        match_chain_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
+                                                               d_term_node, d_term_off, tree->match_counter);
+    else
+        match_batch_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
+                                                               d_term_node, d_term_off, tree->match_counter);
     CK(cudaGetLastError());
     return RT_OK;
 }
