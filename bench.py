@@ -161,6 +161,23 @@ def pick_k(name: str, w: W.Workload, k_arg: int) -> int:
     return 4 if name == "medium" else w.ks[0]
 
 
+def rank_workload(name: str, scale: float, rank: int) -> W.Workload:
+    """Weak scaling: every rank schedules its own stream (same recipe, its own seed) against its own tree."""
+    maker = W.WORKLOADS[name]
+    kw = {} if name == "tiny" else {"scale": scale}
+    seed = maker(**kw).recipe["seed"] + 1000 * rank
+    return maker(seed=seed, **kw)
+
+
+def reduce_max(values, device, multi: bool):
+    """Per-rank timings -> the slowest rank's (what the job waits for)."""
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if multi:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 def run_ours(args):
     rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
     multi = world > 1
@@ -172,11 +189,8 @@ def run_ours(args):
     from paper_2502_04677_b200 import binding as K
 
     name = args.workload
-    maker = W.WORKLOADS[name]
-    kw = {} if name == "tiny" else {"scale": args.scale}
-    # weak scaling: every rank schedules its own stream (same recipe, its own seed) against its own tree
-    seed = maker(**kw).recipe["seed"] + 1000 * rank
-    w = maker(seed=seed, **kw)
+    w = rank_workload(name, args.scale, rank)
+    seed = w.recipe["seed"]
     k = pick_k(name, w, args.k)
     nq = w.queries.n
     t_setup = time.perf_counter()
@@ -258,10 +272,7 @@ def run_ours(args):
     h2d = h_tok.numel() * 4 + h_off.numel() * 8 + h_arr.numel() * 8
     d2h = nq * (4 + 4 + 4 + 8)
 
-    times = torch.tensor([t_total, t_match, t_run, e2e_s], dtype=torch.float64, device=device)
-    if multi:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)          # slowest rank decides
-    t_total, t_match, t_run, e2e_s = times.tolist()
+    t_total, t_match, t_run, e2e_s = reduce_max([t_total, t_match, t_run, e2e_s], device, multi)
     stats1 = K.rt_stats(tree)
     if rank != 0:
         if multi:

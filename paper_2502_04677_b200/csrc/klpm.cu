@@ -670,26 +670,30 @@ select_static_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict
 
 // ------------------------------------------------------------------------------------------------
 // klpm_run: the whole loop as one cooperative kernel
+//
+// Slots are the queries ordered by (arrival, index).  Per decision c:
+//   phase A (every CTA): bring the match state of the waiting slots up to date -- walk newly arrived
+//     queries, drop queries out of evicted leaves, extend the queries that were tied with the prompt
+//     processed last into its new leaf -- and reduce the keys (match << 32 | ~slot) to one per CTA;
+//   phase B (CTA 0): pick (oldest waiting slot or largest key), charge by Definition 2, store the prompt.
+// The two phases hand over through two monotone counters in global memory (`arrive`: CTAs that finished
+// phase A; `seq`: decisions completed), and what phase A needs to know about the last decision travels
+// in one broadcast record.  While the kernel runs only CTA 0 mutates the tree; it keeps the tree's
+// counters in shared memory and writes them back at the end.
 // ------------------------------------------------------------------------------------------------
-struct GridBarrier { unsigned int count; unsigned int gen; };
-
-struct RunState {
-    long long now;
-    long long c;          // decisions taken
-    long long head;       // first slot not yet processed (slots are queries in arrival order)
-    long long admitted;   // slots < admitted have a match state
-    int abort;
-    int evicted;          // the previous decision evicted something
-    // the previously processed prompt, for the refresh of the queries tied with it
-    int last_valid;       // it appended a leaf
-    int32_t last_q;       // query index
-    int32_t last_m;       // its match length before it was stored
-    int32_t last_len;
-    int32_t last_leaf;
-    long long last_pos;   // its position (pool index of its last matched token) before it was stored
-    long long last_leaf_off;
-    GridBarrier bar;
+struct RunBcast {
+    long long now;            // completion time of the last processed query
+    long long head;           // first slot not yet processed
+    long long admitted;       // slots < admitted have a match state
+    long long last_pos;       // position (pool index of last matched token) of the last processed prompt, before it was stored
+    long long last_leaf_off;  // pool offset of the leaf it appended
+    int32_t evicted;          // the last decision evicted something
+    int32_t last_valid;       // the last decision appended a leaf
+    int32_t last_q, last_m, last_len, last_leaf;
+    int32_t abort;
+    int32_t pad;
 };
+struct RunSync { unsigned long long arrive; unsigned long long seq; };
 
 struct RunArgs {
     const int32_t* tok; const int64_t* off; const int64_t* arrival;
@@ -700,107 +704,135 @@ struct RunArgs {
     // scratch (library-owned)
     int32_t* ord;          // slot -> query index, by (arrival, index)
     long long* sorted_t;   // slot -> arrival
-    int32_t* m;            // slot -> current match length
+    int32_t* m;            // slot -> current match length; -1 once processed
     int32_t* hint;         // slot -> node at or below the node where the match ends
     long long* pos;        // slot -> pool index of the last matched token (-1 = root)
-    uint8_t* done;         // slot processed
     unsigned long long* partial;   // per CTA best key
-    RunState* rs;
+    RunBcast* bc;
+    RunSync* sy;
 };
 
-// All CTAs of a cooperative launch meet here.  The wait is bounded: if it runs out, the status word is set
-// and every CTA leaves the kernel at its next check of rs->abort.
-__device__ bool grid_sync(RunState* rs, TreeState* st, unsigned nblocks) {
-    __shared__ int s_ok;
-    __syncthreads();
+#define KLPM_RUN_THREADS 512
+#define KLPM_RUN_SLOTS 4          // slots per thread whose state is loaded together
+#define KLPM_WAIT_LIMIT (1ULL << 25)
+
+// Thread 0 of the CTA polls *p until it reaches target (bounded), then the CTA learns whether to go on.
+__device__ bool run_wait(volatile unsigned long long* p, unsigned long long target, RunBcast* bc, TreeState* st) {
+    __shared__ int s_go;
     if (threadIdx.x == 0) {
-        int ok = 1;
-        if (nblocks > 1) {
-            volatile unsigned* gen = &rs->bar.gen;
-            unsigned my = *gen;
-            __threadfence();
-            unsigned t = atomicAdd(&rs->bar.count, 1u);
-            if (t == nblocks - 1) {
-                rs->bar.count = 0;
-                __threadfence();
-                atomicAdd(&rs->bar.gen, 1u);
-            } else {
-                unsigned long long spins = 0;
-                while (*gen == my) {
-                    __nanosleep(32);
-                    if (++spins > (1ULL << 26)) { set_status(st, RT_ERR_LIMIT); *(volatile int*)&rs->abort = 1; ok = 0; break; }
-                }
-            }
-            __threadfence();
+        int go = 1;
+        unsigned long long spins = 0;
+        while (*p < target) {
+            if (++spins > KLPM_WAIT_LIMIT) { set_status(st, RT_ERR_LIMIT); *(volatile int32_t*)&bc->abort = 1; go = 0; break; }
         }
-        if (*(volatile int*)&rs->abort) ok = 0;
-        s_ok = ok;
+        __threadfence();
+        if (*(volatile int32_t*)&bc->abort) go = 0;
+        s_go = go;
     }
     __syncthreads();
-    return s_ok != 0;
+    const bool go = s_go != 0;
+    __syncthreads();
+    return go;
 }
 
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(KLPM_RUN_THREADS)
 run_kernel(TreeDev T, RunArgs A) {
-    __shared__ unsigned long long s_red[16];
-    __shared__ long long s_bound[2];      // admitted_new, now
+    __shared__ unsigned long long s_red[KLPM_RUN_THREADS / 32];
+    __shared__ long long s_bound[2];      // slots admitted in this decision, time at which the pick is made
     __shared__ InsertOut s_out;
-    __shared__ int32_t s_j[4];            // slot, m, len
+    __shared__ int32_t s_j[2];            // match length and length of the picked prompt
     __shared__ const int32_t* s_x;
-    RunState* rs = A.rs;
+    __shared__ TreeState s_st;            // CTA 0: the tree's counters while the kernel runs
+    __shared__ RunBcast s_bc;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long TT = (long long)gridDim.x * blockDim.x;
+    const unsigned G = gridDim.x;
+    const long long TT = (long long)G * blockDim.x;
     const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    TreeState* const gst = T.st;
+    TreeDev T0 = T;                        // CTA 0's view: counters in shared memory
+    if (blockIdx.x == 0) {
+        if (threadIdx.x == 0) s_st = *gst;
+        T0.st = &s_st;
+    }
+    __syncthreads();
 
     for (long long c = 0; c < A.n; ++c) {
-        // ---------------- phase A: bring the waiting queue's match state up to date, reduce the keys
-        const long long head = *(volatile long long*)&rs->head;
-        const long long admitted = *(volatile long long*)&rs->admitted;
+        // ---------------- wait for decision c-1, fetch what it left
+        if (blockIdx.x != 0) {
+            if (!run_wait(&A.sy->seq, (unsigned long long)c, A.bc, gst)) return;
+        }
         if (threadIdx.x == 0) {
-            long long now = *(volatile long long*)&rs->now;
-            long long th = __ldg(A.sorted_t + head);
-            if (th > now) now = th;                    // nobody waiting: idle until the next arrival
-            long long lo = head, hi = A.n;             // first slot with arrival > now
-            while (lo < hi) { long long mid = (lo + hi) >> 1; if (__ldg(A.sorted_t + mid) <= now) lo = mid + 1; else hi = mid; }
+            RunBcast b;
+            const long long* src = reinterpret_cast<const long long*>(A.bc);
+            long long* dst = reinterpret_cast<long long*>(&b);
+#pragma unroll
+            for (int i = 0; i < (int)(sizeof(RunBcast) / 8); ++i) dst[i] = __ldcg(src + i);
+            s_bc = b;
+            long long now = b.now;
+            if (b.head >= b.admitted) {                // nobody waiting: idle until the next arrival
+                const long long th = __ldg(A.sorted_t + b.head);
+                if (th > now) now = th;
+            }
+            // first slot with arrival > now; everything below `admitted` has arrived, so gallop from there
+            long long lo = b.admitted > b.head ? b.admitted : b.head, hi = A.n;
+            if (lo < hi && __ldg(A.sorted_t + lo) <= now) {
+                long long step = 1;
+                ++lo;
+                while (lo + step <= hi && __ldg(A.sorted_t + lo + step - 1) <= now) { lo += step; step <<= 1; }
+                if (lo + step < hi) hi = lo + step;
+                while (lo < hi) { const long long mid = (lo + hi) >> 1; if (__ldg(A.sorted_t + mid) <= now) lo = mid + 1; else hi = mid; }
+            }
             s_bound[0] = lo; s_bound[1] = now;
         }
         __syncthreads();
-        const long long adm_new = s_bound[0];
-        const int evicted = __ldcg(&rs->evicted);
-        const int last_valid = __ldcg(&rs->last_valid);
-        const int32_t last_m = __ldcg(&rs->last_m), last_len = __ldcg(&rs->last_len), last_leaf = __ldcg(&rs->last_leaf);
-        const long long last_pos = __ldcg(&rs->last_pos), last_leaf_off = __ldcg(&rs->last_leaf_off);
-        const int32_t* last_x = last_valid ? A.tok + __ldg(A.off + __ldcg(&rs->last_q)) : nullptr;
+        const long long head = s_bc.head, admitted = s_bc.admitted, adm_new = s_bound[0];
+        const int evicted = s_bc.evicted, last_valid = s_bc.last_valid;
+        const int32_t last_m = s_bc.last_m, last_len = s_bc.last_len, last_leaf = s_bc.last_leaf;
+        const long long last_pos = s_bc.last_pos, last_leaf_off = s_bc.last_leaf_off;
+        const int32_t* last_x = last_valid ? A.tok + __ldg(A.off + s_bc.last_q) : nullptr;
 
+        // ---------------- phase A
         unsigned long long best = 0;
-        for (long long base = (head / TT) * TT; base < adm_new; base += TT) {
-            const long long r = base + gtid;
-            const bool active = r >= head && r < adm_new && !__ldcg(A.done + r);
-            int32_t qi = 0, qlen = 0, m = 0, hint = 0;
-            long long pos = -1;
-            const int32_t* q = nullptr;
-            if (active) {
-                qi = __ldg(A.ord + r);
-                const int64_t lo = __ldg(A.off + qi);
-                qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
-                q = A.tok + lo;
+        for (long long base = (head / TT) * TT; base < adm_new; base += TT * KLPM_RUN_SLOTS) {
+            int32_t mm[KLPM_RUN_SLOTS];
+            long long pp[KLPM_RUN_SLOTS];
+#pragma unroll
+            for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
+                const long long r = base + u * TT + gtid;
+                const bool have = r >= head && r < admitted && r < adm_new;
+                mm[u] = have ? __ldcg(A.m + r) : -1;
+                pp[u] = have ? __ldcg(A.pos + r) : -1;
             }
-            const bool fresh = active && r >= admitted;
-            unsigned wm = __ballot_sync(FULL_MASK, fresh);
-            while (wm) {                                  // newly arrived queries: full walk, one warp each
-                const int src = __ffs(wm) - 1; wm &= wm - 1;
-                const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
-                const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
-                Term t = walk<false>(T, qq, ql);
-                if (lane == src) { m = t.m; hint = t.node; pos = t.pos; }
-            }
-            bool dirty = fresh;
-            bool cmp = false;
-            if (active && !fresh) {
-                m = __ldcg(A.m + r); pos = __ldcg(A.pos + r);
-                if (evicted) {                            // drop out of evicted leaves
+#pragma unroll
+            for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
+                if (base + u * TT >= adm_new) break;                               // warp-uniform
+                const long long r = base + u * TT + gtid;
+                const bool fresh = r >= head && r >= admitted && r < adm_new;
+                int32_t m = mm[u], hint = 0;
+                long long pos = pp[u];
+                bool dirty = false;
+                unsigned wm = __ballot_sync(FULL_MASK, fresh);
+                if (wm) {                                  // newly arrived queries: full walk, one warp each
+                    const int32_t* q = nullptr; int32_t qlen = 0;
+                    if (fresh) {
+                        const int32_t qi = __ldg(A.ord + r);
+                        const int64_t lo = __ldg(A.off + qi);
+                        qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
+                        q = A.tok + lo;
+                    }
+                    while (wm) {
+                        const int src = __ffs(wm) - 1; wm &= wm - 1;
+                        const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+                        const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
+                        Term t = walk<false>(T, qq, ql);
+                        if (lane == src) { m = t.m; hint = t.node; pos = t.pos; dirty = true; }
+                    }
+                }
+                const bool waiting = fresh || m >= 0;
+                if (waiting && !fresh && evicted) {        // drop out of evicted leaves
                     hint = __ldcg(A.hint + r);
-                    int32_t a = hint, m0 = m;
+                    int32_t a = hint;
+                    const int32_t m0 = m;
                     while (a != 0) {
                         const bool dead = __ldcg(T.dead + a) != 0;
                         const int32_t ds = __ldcg(T.depth_start + a);
@@ -812,30 +844,39 @@ run_kernel(TreeDev T, RunArgs A) {
                         hint = a;
                         pos = a == 0 ? -1 : __ldcg(T.span_off + a) + (m - __ldcg(T.depth_start + a)) - 1;
                         dirty = true;
+                    } else {
+                        hint = -1;                          // unchanged: do not rewrite
                     }
                 }
                 // tied with the prompt processed last: it may now match into that prompt's new leaf
-                if (last_valid && pos == last_pos && m == last_m && m < qlen)
-                    cmp = __ldg(q + m) == __ldg(last_x + m);
-            }
-            unsigned cm = __ballot_sync(FULL_MASK, cmp);
-            while (cm) {
-                const int src = __ffs(cm) - 1; cm &= cm - 1;
-                const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
-                const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
-                const int32_t lim = (ql < last_len ? ql : last_len) - last_m;
-                const int32_t e = first_mismatch<true>(qq + last_m, last_x + last_m, lim);
-                if (lane == src) { m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1; dirty = true; }
-            }
-            if (active) {
-                if (dirty) { A.m[r] = m; A.pos[r] = pos; A.hint[r] = hint; }
-                const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
-                if (key > best) best = key;
+                bool cmp = false;
+                const int32_t* q = nullptr; int32_t qlen = 0;
+                if (waiting && !fresh && last_valid && pos == last_pos && m == last_m) {
+                    const int32_t qi = __ldg(A.ord + r);
+                    const int64_t lo = __ldg(A.off + qi);
+                    qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
+                    q = A.tok + lo;
+                    cmp = m < qlen && __ldg(q + m) == __ldg(last_x + m);
+                }
+                unsigned cm = __ballot_sync(FULL_MASK, cmp);
+                while (cm) {
+                    const int src = __ffs(cm) - 1; cm &= cm - 1;
+                    const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+                    const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
+                    const int32_t lim = (ql < last_len ? ql : last_len) - last_m;
+                    const int32_t e = first_mismatch<true>(qq + last_m, last_x + last_m, lim);
+                    if (lane == src) { m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1; dirty = true; }
+                }
+                if (waiting) {
+                    if (dirty) { A.m[r] = m; A.pos[r] = pos; if (hint >= 0) A.hint[r] = hint; }
+                    const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
+                    if (key > best) best = key;
+                }
             }
         }
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
-            unsigned long long o = __shfl_xor_sync(FULL_MASK, best, d);
+            const unsigned long long o = __shfl_xor_sync(FULL_MASK, best, d);
             if (o > best) best = o;
         }
         if (lane == 0) s_red[warp] = best;
@@ -844,61 +885,121 @@ run_kernel(TreeDev T, RunArgs A) {
             unsigned long long b = 0;
             for (int w = 0; w < (int)(blockDim.x >> 5); ++w) if (s_red[w] > b) b = s_red[w];
             A.partial[blockIdx.x] = b;
+            __threadfence();
+            atomicAdd(&A.sy->arrive, 1ULL);
         }
-        if (!grid_sync(rs, T.st, gridDim.x)) return;
+        if (blockIdx.x != 0) continue;
 
         // ---------------- phase B: CTA 0 picks, charges (Definition 2) and stores the prompt
-        if (blockIdx.x == 0) {
-            if (threadIdx.x == 0) {
-                const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
-                long long slot;
-                if (fcfs_turn) slot = head;
-                else {
-                    unsigned long long b = 0;
-                    for (unsigned g = 0; g < gridDim.x; ++g) { unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
-                    slot = (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
+        if (!run_wait(&A.sy->arrive, (unsigned long long)(c + 1) * G, A.bc, gst)) break;
+        if (warp == 0) {
+            unsigned long long b = 0;
+            for (unsigned g = lane; g < G; g += 32) { const unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const unsigned long long o = __shfl_xor_sync(FULL_MASK, b, d);
+                if (o > b) b = o;
+            }
+            const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
+            const long long slot = fcfs_turn ? head : (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
+            const int32_t qi = __ldg(A.ord + slot);
+            const int32_t m = __ldcg(A.m + slot);
+            const int32_t hint = __ldcg(A.hint + slot);
+            const long long pos = __ldcg(A.pos + slot);
+            const int64_t lo = __ldg(A.off + qi);
+            const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
+            const long long tj = __ldg(A.arrival + qi);
+            const int32_t* x = A.tok + lo;
+            if (lane == 0) { s_j[0] = m; s_j[1] = len; s_x = x; }
+            // Warm the lines the serial insertion is about to read one after the other: the first uncached
+            // token, the tokens around the cut, and the three child-table slots it will probe.
+            {
+                int32_t a = hint;
+                while (a != 0 && m <= T.depth_start[a]) a = T.parent[a];
+                const int32_t o = a == 0 ? 0 : m - T.depth_start[a];
+                const bool mid = a != 0 && o < T.span_len[a];
+                const int64_t so = a == 0 ? 0 : T.span_off[a];
+                int32_t v = 0;
+                if (lane == 0 && m < len) v = __ldcg(x + m);
+                if (lane == 1 && mid) v = __ldcg(T.pool + so + o);
+                if (lane == 2 && mid) v = __ldcg(T.pool + so);
+                const int32_t xm = __shfl_sync(FULL_MASK, v, 0), pt = __shfl_sync(FULL_MASK, v, 1), ft = __shfl_sync(FULL_MASK, v, 2);
+                const int32_t end = mid ? (int32_t)s_st.n_nodes : a;
+                unsigned long long key = 0;
+                bool want = false;
+                if (lane == 0) { key = make_key(end, xm); want = m < len; }
+                if (lane == 1) { key = make_key(end, pt); want = mid; }
+                if (lane == 2) { key = make_key(T.parent[a], ft); want = mid; }
+                if (want) {
+                    const Entry* e = T.table + (hash_key(key) & T.table_mask);
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(e));
                 }
-                const int32_t qi = __ldg(A.ord + slot);
-                const int64_t lo = __ldg(A.off + qi);
-                const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
-                const int32_t* x = A.tok + lo;
-                const int32_t m = __ldcg(A.m + slot);
-                const int32_t hint = __ldcg(A.hint + slot);
-                const long long pos = __ldcg(A.pos + slot);
-                insert_serial(T, x, len, m, hint, &s_out);
-                s_j[0] = (int32_t)slot; s_j[1] = m; s_j[2] = len; s_x = x;
+            }
+            if (lane == 0) {
+                insert_serial(T0, x, len, m, hint, &s_out);
+                RunBcast nb = s_bc;
                 if (s_out.ok) {
-                    const long long tj = __ldg(A.arrival + qi);
                     const long long now = s_bound[1];
                     const long long begin = now > tj ? now : tj;
                     const long long unc = len - m;
                     const long long R = begin + (A.c_den + A.c_num * (long long)len) * unc;
                     A.order[c] = qi; A.uncached[qi] = (int32_t)unc; A.ttft[qi] = R - tj;
                     if (A.completion) A.completion[qi] = R;
-                    A.done[slot] = 1;
+                    A.m[slot] = -1;
                     long long h = head;
-                    while (h < A.n && (h == slot || __ldcg(A.done + h))) ++h;
-                    rs->head = h; rs->now = R; rs->admitted = adm_new; rs->c = c + 1;
-                    rs->evicted = s_out.evicted;
-                    rs->last_valid = s_out.unc > 0; rs->last_q = qi; rs->last_m = m; rs->last_len = len;
-                    rs->last_leaf = s_out.leaf; rs->last_pos = pos; rs->last_leaf_off = s_out.leaf_off;
+                    while (h < A.n && (h == slot || (h < adm_new && __ldcg(A.m + h) < 0))) ++h;
+                    nb.head = h; nb.now = R; nb.admitted = adm_new;
+                    nb.evicted = s_out.evicted;
+                    nb.last_valid = s_out.unc > 0; nb.last_q = qi; nb.last_m = m; nb.last_len = len;
+                    nb.last_leaf = s_out.leaf; nb.last_pos = pos; nb.last_leaf_off = s_out.leaf_off;
                 } else {
-                    rs->abort = 1;
+                    nb.abort = 1;
                 }
+                *A.bc = nb;
             }
-            __syncthreads();
-            if (s_out.ok) {
-                const int32_t unc = s_out.unc, m = s_j[1];
-                const int32_t* x = s_x;
-                int32_t* dst = T.pool + s_out.leaf_off;
-                for (int32_t i = threadIdx.x; i < unc; i += blockDim.x) dst[i] = __ldg(x + m + i);
+        } else if (warp == 1) {
+            // meanwhile: bring the tokens that will be copied into the pool close (the pick is warp 0's;
+            // this warp repeats the cheap part of it to learn which prompt it is)
+            unsigned long long b = 0;
+            for (unsigned g = lane; g < G; g += 32) { const unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const unsigned long long o = __shfl_xor_sync(FULL_MASK, b, d);
+                if (o > b) b = o;
             }
-            __threadfence();
+            const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
+            const long long slot = fcfs_turn ? head : (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
+            const int32_t qi = __ldg(A.ord + slot);
+            const int32_t m = __ldcg(A.m + slot);
+            const int64_t lo = __ldg(A.off + qi);
+            const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
+            const int32_t* x = A.tok + lo + m;
+            for (int32_t i = lane * 32; i < len - m; i += 32 * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + i));
         }
-        if (!grid_sync(rs, T.st, gridDim.x)) return;
+        __syncthreads();
+        if (!s_out.ok) break;
+        {
+            const int32_t unc = s_out.unc, m = s_j[0];
+            const int32_t* x = s_x;
+            int32_t* dst = T.pool + s_out.leaf_off;
+            for (int32_t i = threadIdx.x; i < unc; i += blockDim.x) dst[i] = __ldg(x + m + i);
+        }
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) { atomicExch(&A.sy->seq, (unsigned long long)(c + 1)); }
+    }
+    if (blockIdx.x == 0) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int st_global = *(volatile int*)&gst->status;
+            TreeState out = s_st;
+            if (out.status == 0) out.status = st_global;
+            *gst = out;
+            __threadfence();
+            atomicExch(&A.sy->seq, (unsigned long long)A.n + 1);      // releases anybody still waiting
+        }
     }
 }
-
 
 // ------------------------------------------------------------------------------------------------
 // bulk insertion of many prompts into a tree without a budget.  The set of node boundaries a radix tree
@@ -1062,8 +1163,8 @@ struct rt_tree {
     unsigned long long* match_counter;
     // klpm_run scratch
     long long run_cap;      // slots allocated (power of two)
-    long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos; uint8_t* run_done;
-    unsigned long long* run_partial; RunState* run_rs;
+    long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos;
+    unsigned long long* run_partial; RunBcast* run_bc; RunSync* run_sy;
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
     // checkpoint (rt_checkpoint / rt_rollback): copies of everything a later call can modify
@@ -1093,7 +1194,7 @@ void free_tree(rt_tree* t) {
     cudaFree(d.span_off); cudaFree(d.last_access); cudaFree(d.dead); cudaFree(d.clock_owner);
     cudaFree(d.table); cudaFree(d.pool); cudaFree(d.end_node); cudaFree(d.st); cudaFree(t->match_counter);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
-    cudaFree(t->run_pos); cudaFree(t->run_done); cudaFree(t->run_partial); cudaFree(t->run_rs);
+    cudaFree(t->run_pos); cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
     cudaFree(t->claim);
     cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
     cudaFree(t->ck_clock_owner); cudaFree(t->ck_span_off); cudaFree(t->ck_last_access); cudaFree(t->ck_dead);
@@ -1106,8 +1207,8 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     while (np2 < n) np2 <<= 1;
     if (np2 <= t->run_cap) return RT_OK;
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
-    cudaFree(t->run_pos); cudaFree(t->run_done);
-    t->run_key = nullptr; t->run_ord = nullptr; t->run_m = nullptr; t->run_hint = nullptr; t->run_pos = nullptr; t->run_done = nullptr;
+    cudaFree(t->run_pos);
+    t->run_key = nullptr; t->run_ord = nullptr; t->run_m = nullptr; t->run_hint = nullptr; t->run_pos = nullptr;
     t->run_cap = 0;
     rt_status s;
     if ((s = dalloc(&t->run_key, np2))) return s;
@@ -1115,7 +1216,6 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->run_m, np2))) return s;
     if ((s = dalloc(&t->run_hint, np2))) return s;
     if ((s = dalloc(&t->run_pos, np2))) return s;
-    if ((s = dalloc(&t->run_done, np2))) return s;
     t->run_cap = np2;
     return RT_OK;
 }
@@ -1203,7 +1303,7 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
         (s = dalloc(&d.dead, d.max_nodes)) || (s = dalloc(&d.clock_owner, d.max_clock)) ||
         (s = dalloc(&d.table, cap)) || (s = dalloc(&d.pool, d.max_pool)) || (s = dalloc(&d.st, 1)) ||
         (s = dalloc(&d.end_node, d.max_pool)) ||
-        (s = dalloc(&t->match_counter, 1)) || (s = dalloc(&t->run_partial, 1024)) || (s = dalloc(&t->run_rs, 1)) ||
+        (s = dalloc(&t->match_counter, 1)) || (s = dalloc(&t->run_partial, 1024)) || (s = dalloc(&t->run_bc, 1)) || (s = dalloc(&t->run_sy, 1)) ||
         (s = dalloc(&t->claim, d.max_nodes))) {
         free_tree(t);
         return s;
@@ -1462,19 +1562,19 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
                 bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_key, tree->run_ord, np2, k, j);
         CK(cudaGetLastError());
     }
-    CK(cudaMemsetAsync(tree->run_done, 0, (size_t)n, s));
-    RunState rs0;
-    memset(&rs0, 0, sizeof(rs0));
-    rs0.now = params->start_tick;
-    CK(cudaMemcpyAsync(tree->run_rs, &rs0, sizeof(rs0), cudaMemcpyHostToDevice, s));
+    RunBcast bc0;
+    memset(&bc0, 0, sizeof(bc0));
+    bc0.now = params->start_tick;
+    CK(cudaMemcpyAsync(tree->run_bc, &bc0, sizeof(bc0), cudaMemcpyHostToDevice, s));
+    CK(cudaMemsetAsync(tree->run_sy, 0, sizeof(RunSync), s));
     RunArgs a;
     memset(&a, 0, sizeof(a));
     a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.n = n;
     a.policy = params->policy; a.k = params->k; a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
     a.order = d_order; a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
     a.ord = tree->run_ord; a.sorted_t = tree->run_key; a.m = tree->run_m; a.hint = tree->run_hint; a.pos = tree->run_pos;
-    a.done = tree->run_done; a.partial = tree->run_partial; a.rs = tree->run_rs;
-    const int threads = 512;
+    a.partial = tree->run_partial; a.bc = tree->run_bc; a.sy = tree->run_sy;
+    const int threads = KLPM_RUN_THREADS;
     int per_sm = 0;
     CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, run_kernel, threads, 0));
     if (per_sm < 1) return RT_ERR_CUDA;
