@@ -735,171 +735,211 @@ __device__ bool run_wait(volatile unsigned long long* p, unsigned long long targ
     return go;
 }
 
+// Time at which the next pick is made and the number of slots that have arrived by then (one thread).
+// Everything below `admitted` has arrived already, so the search gallops from there.
+__device__ void run_bound(const RunArgs& A, const RunBcast& b, long long* adm_new, long long* now_out) {
+    long long now = b.now;
+    if (b.head >= b.admitted && b.head < A.n) {   // nobody waiting: idle until the next arrival
+        const long long th = __ldg(A.sorted_t + b.head);
+        if (th > now) now = th;
+    }
+    long long lo = b.admitted > b.head ? b.admitted : b.head, hi = A.n;
+    if (lo < hi && __ldg(A.sorted_t + lo) <= now) {
+        long long step = 1;
+        ++lo;
+        while (lo + step <= hi && __ldg(A.sorted_t + lo + step - 1) <= now) { lo += step; step <<= 1; }
+        if (lo + step < hi) hi = lo + step;
+        while (lo < hi) { const long long mid = (lo + hi) >> 1; if (__ldg(A.sorted_t + mid) <= now) lo = mid + 1; else hi = mid; }
+    }
+    *adm_new = lo; *now_out = now;
+}
+
+// Phase A for one CTA of the `nscan` scanning CTAs: returns (in warp lanes) this thread's best key.
+__device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const RunBcast& bc, long long adm_new,
+                                       unsigned scan_id, unsigned nscan) {
+    const int lane = threadIdx.x & 31;
+    const long long TT = (long long)nscan * blockDim.x;
+    const long long gtid = (long long)scan_id * blockDim.x + threadIdx.x;
+    const long long head = bc.head, admitted = bc.admitted;
+    const int evicted = bc.evicted, last_valid = bc.last_valid;
+    const int32_t last_m = bc.last_m, last_len = bc.last_len, last_leaf = bc.last_leaf;
+    const long long last_pos = bc.last_pos, last_leaf_off = bc.last_leaf_off;
+    const int32_t* last_x = last_valid ? A.tok + __ldg(A.off + bc.last_q) : nullptr;
+    unsigned long long best = 0;
+    for (long long base = (head / TT) * TT; base < adm_new; base += TT * KLPM_RUN_SLOTS) {
+        int32_t mm[KLPM_RUN_SLOTS];
+        long long pp[KLPM_RUN_SLOTS];
+#pragma unroll
+        for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
+            const long long r = base + u * TT + gtid;
+            const bool have = r >= head && r < admitted && r < adm_new;
+            mm[u] = have ? __ldcg(A.m + r) : -1;
+            pp[u] = have ? __ldcg(A.pos + r) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
+            if (base + u * TT >= adm_new) break;                               // warp-uniform
+            const long long r = base + u * TT + gtid;
+            const bool fresh = r >= head && r >= admitted && r < adm_new;
+            int32_t m = mm[u], hint = 0;
+            long long pos = pp[u];
+            bool dirty = false;
+            unsigned wm = __ballot_sync(FULL_MASK, fresh);
+            if (wm) {                                  // newly arrived queries: full walk, one warp each
+                const int32_t* q = nullptr; int32_t qlen = 0;
+                if (fresh) {
+                    const int32_t qi = __ldg(A.ord + r);
+                    const int64_t lo = __ldg(A.off + qi);
+                    qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
+                    q = A.tok + lo;
+                }
+                while (wm) {
+                    const int src = __ffs(wm) - 1; wm &= wm - 1;
+                    const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+                    const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
+                    Term t = walk<false>(T, qq, ql);
+                    if (lane == src) { m = t.m; hint = t.node; pos = t.pos; dirty = true; }
+                }
+            }
+            const bool waiting = fresh || m >= 0;
+            if (waiting && !fresh && evicted) {        // drop out of evicted leaves
+                hint = __ldcg(A.hint + r);
+                int32_t a = hint;
+                const int32_t m0 = m;
+                while (a != 0) {
+                    const bool dead = __ldcg(T.dead + a) != 0;
+                    const int32_t ds = __ldcg(T.depth_start + a);
+                    if (dead) { if (ds < m) m = ds; }
+                    else if (m > ds) break;
+                    a = __ldcg(T.parent + a);
+                }
+                if (a != hint || m != m0) {
+                    hint = a;
+                    pos = a == 0 ? -1 : __ldcg(T.span_off + a) + (m - __ldcg(T.depth_start + a)) - 1;
+                    dirty = true;
+                } else {
+                    hint = -1;                          // unchanged: do not rewrite
+                }
+            }
+            // tied with the prompt processed last: it may now match into that prompt's new leaf
+            bool cmp = false;
+            const int32_t* q = nullptr; int32_t qlen = 0;
+            if (waiting && !fresh && last_valid && pos == last_pos && m == last_m) {
+                const int32_t qi = __ldg(A.ord + r);
+                const int64_t lo = __ldg(A.off + qi);
+                qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
+                q = A.tok + lo;
+                cmp = m < qlen && __ldg(q + m) == __ldg(last_x + m);
+            }
+            unsigned cm = __ballot_sync(FULL_MASK, cmp);
+            while (cm) {
+                const int src = __ffs(cm) - 1; cm &= cm - 1;
+                const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+                const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
+                const int32_t lim = (ql < last_len ? ql : last_len) - last_m;
+                const int32_t e = first_mismatch<true>(qq + last_m, last_x + last_m, lim);
+                if (lane == src) { m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1; dirty = true; }
+            }
+            if (waiting) {
+                if (dirty) { A.m[r] = m; A.pos[r] = pos; if (hint >= 0) A.hint[r] = hint; }
+                const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
+                if (key > best) best = key;
+            }
+        }
+    }
+    return best;
+}
+
+__device__ __forceinline__ unsigned long long warp_max64(unsigned long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(FULL_MASK, v, d);
+        if (o > v) v = o;
+    }
+    return v;
+}
+
+// CTA 0 is the sequencer (picks, charges, mutates the tree); CTAs 1..G-1 scan.  With a single CTA it does both.
+// Without a budget, and when the next decision admits no new arrivals, the sequencer publishes its pick --
+// including the id and pool offset its new leaf is going to get, which follow from the tree's counters --
+// before it performs the insertion, so the scanners refresh the waiting queue for the next decision while
+// the tree is being updated (they only read query tokens and their own slots' state then).
 __global__ void __launch_bounds__(KLPM_RUN_THREADS)
 run_kernel(TreeDev T, RunArgs A) {
     __shared__ unsigned long long s_red[KLPM_RUN_THREADS / 32];
-    __shared__ long long s_bound[2];      // slots admitted in this decision, time at which the pick is made
+    __shared__ long long s_bound[2];      // slots admitted by this decision, time at which the pick is made
     __shared__ InsertOut s_out;
     __shared__ int32_t s_j[2];            // match length and length of the picked prompt
     __shared__ const int32_t* s_x;
     __shared__ TreeState s_st;            // CTA 0: the tree's counters while the kernel runs
     __shared__ RunBcast s_bc;
+    __shared__ int s_flag[2];             // CTA 0: publish-before-insert, predicted leaf
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned G = gridDim.x;
-    const long long TT = (long long)G * blockDim.x;
-    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned nscan = G > 1 ? G - 1 : 1;
     TreeState* const gst = T.st;
-    TreeDev T0 = T;                        // CTA 0's view: counters in shared memory
-    if (blockIdx.x == 0) {
-        if (threadIdx.x == 0) s_st = *gst;
-        T0.st = &s_st;
+
+    if (blockIdx.x != 0) {
+        // ------------------------------------------------------------ scanners
+        for (long long c = 0; c < A.n; ++c) {
+            if (!run_wait(&A.sy->seq, (unsigned long long)c, A.bc, gst)) return;
+            if (threadIdx.x == 0) {
+                RunBcast b;
+                const long long* src = reinterpret_cast<const long long*>(A.bc);
+                long long* dst = reinterpret_cast<long long*>(&b);
+#pragma unroll
+                for (int i = 0; i < (int)(sizeof(RunBcast) / 8); ++i) dst[i] = __ldcg(src + i);
+                s_bc = b;
+                run_bound(A, b, &s_bound[0], &s_bound[1]);
+            }
+            __syncthreads();
+            unsigned long long best = warp_max64(run_scan(T, A, s_bc, s_bound[0], blockIdx.x - 1, nscan));
+            if (lane == 0) s_red[warp] = best;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                unsigned long long b = 0;
+                for (int w = 0; w < (int)(blockDim.x >> 5); ++w) if (s_red[w] > b) b = s_red[w];
+                A.partial[blockIdx.x - 1] = b;
+                __threadfence();
+                atomicAdd(&A.sy->arrive, 1ULL);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------- sequencer (CTA 0)
+    TreeDev T0 = T;                        // its view of the tree: counters in shared memory
+    T0.st = &s_st;
+    if (threadIdx.x == 0) {
+        s_st = *gst;
+        RunBcast b;
+        const long long* src = reinterpret_cast<const long long*>(A.bc);
+        long long* dst = reinterpret_cast<long long*>(&b);
+#pragma unroll
+        for (int i = 0; i < (int)(sizeof(RunBcast) / 8); ++i) dst[i] = __ldcg(src + i);
+        s_bc = b;
     }
     __syncthreads();
-
-    for (long long c = 0; c < A.n; ++c) {
-        // ---------------- wait for decision c-1, fetch what it left
-        if (blockIdx.x != 0) {
-            if (!run_wait(&A.sy->seq, (unsigned long long)c, A.bc, gst)) return;
-        }
-        if (threadIdx.x == 0) {
-            RunBcast b;
-            const long long* src = reinterpret_cast<const long long*>(A.bc);
-            long long* dst = reinterpret_cast<long long*>(&b);
-#pragma unroll
-            for (int i = 0; i < (int)(sizeof(RunBcast) / 8); ++i) dst[i] = __ldcg(src + i);
-            s_bc = b;
-            long long now = b.now;
-            if (b.head >= b.admitted) {                // nobody waiting: idle until the next arrival
-                const long long th = __ldg(A.sorted_t + b.head);
-                if (th > now) now = th;
-            }
-            // first slot with arrival > now; everything below `admitted` has arrived, so gallop from there
-            long long lo = b.admitted > b.head ? b.admitted : b.head, hi = A.n;
-            if (lo < hi && __ldg(A.sorted_t + lo) <= now) {
-                long long step = 1;
-                ++lo;
-                while (lo + step <= hi && __ldg(A.sorted_t + lo + step - 1) <= now) { lo += step; step <<= 1; }
-                if (lo + step < hi) hi = lo + step;
-                while (lo < hi) { const long long mid = (lo + hi) >> 1; if (__ldg(A.sorted_t + mid) <= now) lo = mid + 1; else hi = mid; }
-            }
-            s_bound[0] = lo; s_bound[1] = now;
-        }
+    bool ok = true;
+    for (long long c = 0; c < A.n && ok; ++c) {
+        if (threadIdx.x == 0) run_bound(A, s_bc, &s_bound[0], &s_bound[1]);
         __syncthreads();
-        const long long head = s_bc.head, admitted = s_bc.admitted, adm_new = s_bound[0];
-        const int evicted = s_bc.evicted, last_valid = s_bc.last_valid;
-        const int32_t last_m = s_bc.last_m, last_len = s_bc.last_len, last_leaf = s_bc.last_leaf;
-        const long long last_pos = s_bc.last_pos, last_leaf_off = s_bc.last_leaf_off;
-        const int32_t* last_x = last_valid ? A.tok + __ldg(A.off + s_bc.last_q) : nullptr;
-
-        // ---------------- phase A
-        unsigned long long best = 0;
-        for (long long base = (head / TT) * TT; base < adm_new; base += TT * KLPM_RUN_SLOTS) {
-            int32_t mm[KLPM_RUN_SLOTS];
-            long long pp[KLPM_RUN_SLOTS];
-#pragma unroll
-            for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
-                const long long r = base + u * TT + gtid;
-                const bool have = r >= head && r < admitted && r < adm_new;
-                mm[u] = have ? __ldcg(A.m + r) : -1;
-                pp[u] = have ? __ldcg(A.pos + r) : -1;
-            }
-#pragma unroll
-            for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
-                if (base + u * TT >= adm_new) break;                               // warp-uniform
-                const long long r = base + u * TT + gtid;
-                const bool fresh = r >= head && r >= admitted && r < adm_new;
-                int32_t m = mm[u], hint = 0;
-                long long pos = pp[u];
-                bool dirty = false;
-                unsigned wm = __ballot_sync(FULL_MASK, fresh);
-                if (wm) {                                  // newly arrived queries: full walk, one warp each
-                    const int32_t* q = nullptr; int32_t qlen = 0;
-                    if (fresh) {
-                        const int32_t qi = __ldg(A.ord + r);
-                        const int64_t lo = __ldg(A.off + qi);
-                        qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
-                        q = A.tok + lo;
-                    }
-                    while (wm) {
-                        const int src = __ffs(wm) - 1; wm &= wm - 1;
-                        const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
-                        const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
-                        Term t = walk<false>(T, qq, ql);
-                        if (lane == src) { m = t.m; hint = t.node; pos = t.pos; dirty = true; }
-                    }
-                }
-                const bool waiting = fresh || m >= 0;
-                if (waiting && !fresh && evicted) {        // drop out of evicted leaves
-                    hint = __ldcg(A.hint + r);
-                    int32_t a = hint;
-                    const int32_t m0 = m;
-                    while (a != 0) {
-                        const bool dead = __ldcg(T.dead + a) != 0;
-                        const int32_t ds = __ldcg(T.depth_start + a);
-                        if (dead) { if (ds < m) m = ds; }
-                        else if (m > ds) break;
-                        a = __ldcg(T.parent + a);
-                    }
-                    if (a != hint || m != m0) {
-                        hint = a;
-                        pos = a == 0 ? -1 : __ldcg(T.span_off + a) + (m - __ldcg(T.depth_start + a)) - 1;
-                        dirty = true;
-                    } else {
-                        hint = -1;                          // unchanged: do not rewrite
-                    }
-                }
-                // tied with the prompt processed last: it may now match into that prompt's new leaf
-                bool cmp = false;
-                const int32_t* q = nullptr; int32_t qlen = 0;
-                if (waiting && !fresh && last_valid && pos == last_pos && m == last_m) {
-                    const int32_t qi = __ldg(A.ord + r);
-                    const int64_t lo = __ldg(A.off + qi);
-                    qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
-                    q = A.tok + lo;
-                    cmp = m < qlen && __ldg(q + m) == __ldg(last_x + m);
-                }
-                unsigned cm = __ballot_sync(FULL_MASK, cmp);
-                while (cm) {
-                    const int src = __ffs(cm) - 1; cm &= cm - 1;
-                    const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
-                    const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
-                    const int32_t lim = (ql < last_len ? ql : last_len) - last_m;
-                    const int32_t e = first_mismatch<true>(qq + last_m, last_x + last_m, lim);
-                    if (lane == src) { m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1; dirty = true; }
-                }
-                if (waiting) {
-                    if (dirty) { A.m[r] = m; A.pos[r] = pos; if (hint >= 0) A.hint[r] = hint; }
-                    const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
-                    if (key > best) best = key;
-                }
+        const long long head = s_bc.head, adm_new = s_bound[0];
+        unsigned long long b = 0;
+        if (G == 1) {
+            unsigned long long best = warp_max64(run_scan(T, A, s_bc, adm_new, 0, 1));
+            if (lane == 0) s_red[warp] = best;
+            __syncthreads();
+            if (warp == 0) b = warp_max64(lane < (int)(blockDim.x >> 5) ? s_red[lane] : 0ULL);
+        } else {
+            if (!run_wait(&A.sy->arrive, (unsigned long long)(c + 1) * nscan, A.bc, gst)) { ok = false; break; }
+            if (warp == 0) {
+                for (unsigned g = lane; g < nscan; g += 32) { const unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
+                b = warp_max64(b);
             }
         }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(FULL_MASK, best, d);
-            if (o > best) best = o;
-        }
-        if (lane == 0) s_red[warp] = best;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned long long b = 0;
-            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) if (s_red[w] > b) b = s_red[w];
-            A.partial[blockIdx.x] = b;
-            __threadfence();
-            atomicAdd(&A.sy->arrive, 1ULL);
-        }
-        if (blockIdx.x != 0) continue;
-
-        // ---------------- phase B: CTA 0 picks, charges (Definition 2) and stores the prompt
-        if (!run_wait(&A.sy->arrive, (unsigned long long)(c + 1) * G, A.bc, gst)) break;
+        // ---- pick (warp 0; lane 0 decides), charge by Definition 2
         if (warp == 0) {
-            unsigned long long b = 0;
-            for (unsigned g = lane; g < G; g += 32) { const unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const unsigned long long o = __shfl_xor_sync(FULL_MASK, b, d);
-                if (o > b) b = o;
-            }
             const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
             const long long slot = fcfs_turn ? head : (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
             const int32_t qi = __ldg(A.ord + slot);
@@ -910,15 +950,17 @@ run_kernel(TreeDev T, RunArgs A) {
             const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
             const long long tj = __ldg(A.arrival + qi);
             const int32_t* x = A.tok + lo;
-            if (lane == 0) { s_j[0] = m; s_j[1] = len; s_x = x; }
-            // Warm the lines the serial insertion is about to read one after the other: the first uncached
-            // token, the tokens around the cut, and the three child-table slots it will probe.
+            // where the cached part ends, and what the insertion is going to allocate
+            int32_t a = hint;
+            while (a != 0 && m <= T.depth_start[a]) a = T.parent[a];
+            const int32_t o = a == 0 ? 0 : m - T.depth_start[a];
+            const bool mid = a != 0 && o < T.span_len[a];
+            const int64_t so = a == 0 ? 0 : T.span_off[a];
+            const int32_t unc = len - m;
+            const int32_t leaf_pred = unc > 0 ? (int32_t)s_st.n_nodes + (mid ? 1 : 0) : -1;
+            const long long leaf_off_pred = unc > 0 ? ((s_st.pool_used + 3) & ~3LL) + (m & 3) : 0;
+            // warm the lines the serial insertion reads one after the other
             {
-                int32_t a = hint;
-                while (a != 0 && m <= T.depth_start[a]) a = T.parent[a];
-                const int32_t o = a == 0 ? 0 : m - T.depth_start[a];
-                const bool mid = a != 0 && o < T.span_len[a];
-                const int64_t so = a == 0 ? 0 : T.span_off[a];
                 int32_t v = 0;
                 if (lane == 0 && m < len) v = __ldcg(x + m);
                 if (lane == 1 && mid) v = __ldcg(T.pool + so + o);
@@ -934,50 +976,43 @@ run_kernel(TreeDev T, RunArgs A) {
                     const Entry* e = T.table + (hash_key(key) & T.table_mask);
                     asm volatile("prefetch.global.L2 [%0];" ::"l"(e));
                 }
+                for (int32_t i = lane * 32; i < unc; i += 32 * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + m + i));
             }
             if (lane == 0) {
-                insert_serial(T0, x, len, m, hint, &s_out);
+                s_j[0] = m; s_j[1] = len; s_x = x;
+                const long long now = s_bound[1];
+                const long long begin = now > tj ? now : tj;
+                const long long R = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
+                A.order[c] = qi; A.uncached[qi] = unc; A.ttft[qi] = R - tj;
+                if (A.completion) A.completion[qi] = R;
+                A.m[slot] = -1;
+                long long h = head;
+                while (h < A.n && (h == slot || (h < adm_new && __ldcg(A.m + h) < 0))) ++h;
                 RunBcast nb = s_bc;
-                if (s_out.ok) {
-                    const long long now = s_bound[1];
-                    const long long begin = now > tj ? now : tj;
-                    const long long unc = len - m;
-                    const long long R = begin + (A.c_den + A.c_num * (long long)len) * unc;
-                    A.order[c] = qi; A.uncached[qi] = (int32_t)unc; A.ttft[qi] = R - tj;
-                    if (A.completion) A.completion[qi] = R;
-                    A.m[slot] = -1;
-                    long long h = head;
-                    while (h < A.n && (h == slot || (h < adm_new && __ldcg(A.m + h) < 0))) ++h;
-                    nb.head = h; nb.now = R; nb.admitted = adm_new;
-                    nb.evicted = s_out.evicted;
-                    nb.last_valid = s_out.unc > 0; nb.last_q = qi; nb.last_m = m; nb.last_len = len;
-                    nb.last_leaf = s_out.leaf; nb.last_pos = pos; nb.last_leaf_off = s_out.leaf_off;
-                } else {
-                    nb.abort = 1;
+                nb.head = h; nb.now = R; nb.admitted = adm_new;
+                nb.evicted = 0;
+                nb.last_valid = unc > 0; nb.last_q = qi; nb.last_m = m; nb.last_len = len;
+                nb.last_leaf = leaf_pred; nb.last_pos = pos; nb.last_leaf_off = leaf_off_pred;
+                s_bc = nb;
+                // may the scanners start on the next decision while the tree is being updated?
+                long long adm_next, now_next;
+                run_bound(A, nb, &adm_next, &now_next);
+                const int early = (G > 1 && T.budget == 0 && adm_next == adm_new && c + 1 < A.n) ? 1 : 0;
+                s_flag[0] = early; s_flag[1] = leaf_pred;
+                if (early) {
+                    *A.bc = nb;
+                    __threadfence();
+                    atomicExch(&A.sy->seq, (unsigned long long)(c + 1));
                 }
-                *A.bc = nb;
+                insert_serial(T0, x, len, m, hint, &s_out);
+                if (s_out.ok && (s_out.leaf != leaf_pred || (unc > 0 && s_out.leaf_off != leaf_off_pred))) {
+                    set_status(&s_st, RT_ERR_LIMIT);           // cannot happen: the prediction repeats the allocation rule
+                    s_out.ok = 0;
+                }
             }
-        } else if (warp == 1) {
-            // meanwhile: bring the tokens that will be copied into the pool close (the pick is warp 0's;
-            // this warp repeats the cheap part of it to learn which prompt it is)
-            unsigned long long b = 0;
-            for (unsigned g = lane; g < G; g += 32) { const unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const unsigned long long o = __shfl_xor_sync(FULL_MASK, b, d);
-                if (o > b) b = o;
-            }
-            const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
-            const long long slot = fcfs_turn ? head : (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
-            const int32_t qi = __ldg(A.ord + slot);
-            const int32_t m = __ldcg(A.m + slot);
-            const int64_t lo = __ldg(A.off + qi);
-            const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
-            const int32_t* x = A.tok + lo + m;
-            for (int32_t i = lane * 32; i < len - m; i += 32 * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + i));
         }
         __syncthreads();
-        if (!s_out.ok) break;
+        if (!s_out.ok) { ok = false; break; }
         {
             const int32_t unc = s_out.unc, m = s_j[0];
             const int32_t* x = s_x;
@@ -986,18 +1021,25 @@ run_kernel(TreeDev T, RunArgs A) {
         }
         __threadfence();
         __syncthreads();
-        if (threadIdx.x == 0) { atomicExch(&A.sy->seq, (unsigned long long)(c + 1)); }
-    }
-    if (blockIdx.x == 0) {
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const int st_global = *(volatile int*)&gst->status;
-            TreeState out = s_st;
-            if (out.status == 0) out.status = st_global;
-            *gst = out;
-            __threadfence();
-            atomicExch(&A.sy->seq, (unsigned long long)A.n + 1);      // releases anybody still waiting
+        if (threadIdx.x == 0 && !s_flag[0]) {
+            s_bc.evicted = s_out.evicted;
+            if (G > 1 && c + 1 < A.n) {
+                *A.bc = s_bc;
+                __threadfence();
+                atomicExch(&A.sy->seq, (unsigned long long)(c + 1));
+            }
         }
+        __syncthreads();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int st_global = *(volatile int*)&gst->status;
+        TreeState out = s_st;
+        if (out.status == 0) out.status = st_global;
+        *gst = out;
+        if (!ok) *(volatile int32_t*)&A.bc->abort = 1;
+        __threadfence();
+        atomicExch(&A.sy->seq, (unsigned long long)A.n + 1);      // releases anybody still waiting
     }
 }
 
@@ -1578,8 +1620,9 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
     int per_sm = 0;
     CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, run_kernel, threads, 0));
     if (per_sm < 1) return RT_ERR_CUDA;
-    long long blocks = ((long long)n + threads * 4 - 1) / (threads * 4);
-    if (blocks < 1) blocks = 1;
+    // one sequencer CTA plus scanners; small queues are handled by the sequencer alone
+    long long blocks = 1;
+    if (n > threads * 8) blocks = 1 + ((long long)n + threads * KLPM_RUN_SLOTS - 1) / (threads * KLPM_RUN_SLOTS);
     if (blocks > tree->num_sms) blocks = tree->num_sms;
     void* kargs[] = {(void*)&tree->dev, (void*)&a};
     CK(cudaLaunchCooperativeKernel((void*)run_kernel, dim3((unsigned)blocks), dim3(threads), kargs, 0, s));
