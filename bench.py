@@ -32,7 +32,7 @@ DEFAULT_WORKLOAD = "adversarial"
 
 # dram bytes (read + write) per launch of the match kernel from an ncu capture, keyed by (workload, scale);
 # filled in from profiles/ once captured, None while the kernel has changed since
-TRAFFIC = {}
+TRAFFIC = {("adversarial", 1.0): 17.05e9}    # profiles/match_chain_kernel_adversarial.md
 
 
 def env_int(name, default):
