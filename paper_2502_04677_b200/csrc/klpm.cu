@@ -349,9 +349,43 @@ __device__ bool table_put(const TreeDev& T, int32_t parent, int32_t tok, int32_t
     return false;
 }
 
+// What a caller has already read for an insertion, so that the serial part need not wait for memory again:
+// the tokens that key the table operations and the keys seen in the slots those operations probe first.
+struct InsertPre {
+    int32_t xm, pt, ft;                       // x[m]; pool token just below the cut; first token of the cut edge
+    unsigned long long k_leaf, k_low, k_par;  // keys seen in the first slots of (end, xm), (upper, pt), (parent, ft)
+};
+
+__device__ long long table_find_seen(const TreeDev& T, int32_t parent, int32_t tok, unsigned long long seen) {
+    const unsigned long long key = make_key(parent, tok);
+    if (seen == key) return (long long)(hash_key(key) & T.table_mask);
+    return table_find(T, parent, tok);
+}
+
+// table_put that trusts `seen` for the first slot unless that slot is `taken` (written since it was read).
+__device__ long long table_put_seen(const TreeDev& T, int32_t parent, int32_t tok, int32_t child, int32_t span_len, int64_t span_off,
+                                   int64_t chain_end, unsigned long long seen, long long taken) {
+    const unsigned long long key = make_key(parent, tok);
+    unsigned long long slot = hash_key(key) & T.table_mask;
+    bool first = (long long)slot != taken;
+    for (unsigned long long probes = 0; probes <= T.table_mask; ++probes) {
+        const unsigned long long k = first ? seen : __ldcg(&T.table[slot].key);
+        first = false;
+        if (k == key || k == 0ULL) {
+            Entry* e = T.table + slot;
+            e->child = child; e->span_len = span_len; e->span_off = span_off; e->chain_end = chain_end;
+            e->key = key;
+            return (long long)slot;
+        }
+        slot = (slot + 1) & T.table_mask;
+    }
+    return -1;
+}
+
 // Node boundary `o` tokens into v's edge (0 < o < span_len[v]): a new node takes the upper part and v's
-// place under v's parent; v keeps the lower part, its children and its id.
-__device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o) {
+// place under v's parent; v keeps the lower part, its children and its id.  Returns the new node;
+// *low_slot receives the table slot that now holds (new node, first token of the lower part).
+__device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o, const InsertPre* pre, long long* low_slot) {
     TreeState* S = T.st;
     int32_t u = (int32_t)S->n_nodes++;
     S->live_nodes++;
@@ -359,12 +393,15 @@ __device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o) {
     int64_t off = T.span_off[v];
     T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = off; T.span_len[u] = o;
     T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = T.last_access[v];
-    long long slot = table_find(T, par, __ldcg(T.pool + off));
+    const long long slot = pre ? table_find_seen(T, par, pre->ft, pre->k_par) : table_find(T, par, __ldcg(T.pool + off));
     int64_t chain_end = off + len;
     if (slot >= 0) { T.table[slot].child = u; T.table[slot].span_len = o; chain_end = T.table[slot].chain_end; }
     else set_status(S, RT_ERR_LIMIT);
     T.span_off[v] = off + o; T.span_len[v] = len - o; T.depth_start[v] = ds + o; T.parent[v] = u;
-    if (!table_put(T, u, __ldcg(T.pool + off + o), v, len - o, off + o, chain_end)) set_status(S, RT_ERR_CAPACITY);
+    const long long ls = pre ? table_put_seen(T, u, pre->pt, v, len - o, off + o, chain_end, pre->k_low, -1)
+                             : table_put_seen(T, u, __ldcg(T.pool + off + o), v, len - o, off + o, chain_end, 0ULL, (long long)(hash_key(make_key(u, __ldcg(T.pool + off + o))) & T.table_mask));
+    if (ls < 0) set_status(S, RT_ERR_CAPACITY);
+    *low_slot = ls;
     T.end_node[off + o - 1] = u;
     return u;
 }
@@ -395,7 +432,8 @@ struct InsertOut {
 
 // Store prompt x (|x| = len) whose cached part is m tokens long and ends in `hint` or an ancestor of it.
 // Everything except copying the new leaf's tokens into the pool.  One thread.
-__device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, int32_t m, int32_t hint, InsertOut* out) {
+__device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, int32_t m, int32_t hint, InsertOut* out,
+                              const InsertPre* pre = nullptr) {
     TreeState* S = T.st;
     out->leaf = -1; out->unc = 0; out->leaf_off = 0; out->evicted = 0; out->ok = 0;
     if (S->clock + 1 >= T.max_clock || S->n_nodes + 2 > T.max_nodes) { set_status(S, RT_ERR_CAPACITY); return; }
@@ -404,7 +442,8 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
     while (a != 0 && m <= T.depth_start[a]) a = T.parent[a];
     const int32_t o = a == 0 ? 0 : m - T.depth_start[a];
     int32_t end = a;
-    if (a != 0 && o < T.span_len[a]) end = split_node(T, a, o);
+    long long low_slot = -1;
+    if (a != 0 && o < T.span_len[a]) end = split_node(T, a, o, pre, &low_slot);
     if (end != 0) { T.last_access[end] = clock; T.clock_owner[clock] = end; }
     const int32_t unc = len - m;
     if (T.budget > 0) {
@@ -431,7 +470,9 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
         T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = clock;
         T.clock_owner[clock] = leaf;
         T.nchild[end]++;
-        if (!table_put(T, end, __ldcg(x + m), leaf, unc, off, off + unc)) { set_status(S, RT_ERR_CAPACITY); return; }
+        const long long put = pre ? table_put_seen(T, end, pre->xm, leaf, unc, off, off + unc, pre->k_leaf, low_slot)
+                                  : (table_put(T, end, __ldcg(x + m), leaf, unc, off, off + unc) ? 0 : -1);
+        if (put < 0) { set_status(S, RT_ERR_CAPACITY); return; }
         T.end_node[off + unc - 1] = leaf;
         S->tokens_live += unc;
         S->live_nodes++;
@@ -691,7 +732,7 @@ struct RunBcast {
     int32_t last_valid;       // the last decision appended a leaf
     int32_t last_q, last_m, last_len, last_leaf;
     int32_t abort;
-    int32_t pad;
+    int32_t last_xm;          // first uncached token of the last processed prompt
 };
 struct RunSync { unsigned long long arrive; unsigned long long seq; };
 
@@ -704,9 +745,12 @@ struct RunArgs {
     // scratch (library-owned)
     int32_t* ord;          // slot -> query index, by (arrival, index)
     long long* sorted_t;   // slot -> arrival
+    long long* soff;       // slot -> offset of the query's first token
+    int32_t* slen;         // slot -> query length
     int32_t* m;            // slot -> current match length; -1 once processed
     int32_t* hint;         // slot -> node at or below the node where the match ends
     long long* pos;        // slot -> pool index of the last matched token (-1 = root)
+    int32_t* ntok;         // slot -> the query token right after its match (meaningful while m < length)
     unsigned long long* partial;   // per CTA best key
     RunBcast* bc;
     RunSync* sy;
@@ -764,10 +808,11 @@ __device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const
     const int evicted = bc.evicted, last_valid = bc.last_valid;
     const int32_t last_m = bc.last_m, last_len = bc.last_len, last_leaf = bc.last_leaf;
     const long long last_pos = bc.last_pos, last_leaf_off = bc.last_leaf_off;
+    const int32_t last_xm = bc.last_xm;
     const int32_t* last_x = last_valid ? A.tok + __ldg(A.off + bc.last_q) : nullptr;
     unsigned long long best = 0;
     for (long long base = (head / TT) * TT; base < adm_new; base += TT * KLPM_RUN_SLOTS) {
-        int32_t mm[KLPM_RUN_SLOTS];
+        int32_t mm[KLPM_RUN_SLOTS], nn[KLPM_RUN_SLOTS];
         long long pp[KLPM_RUN_SLOTS];
 #pragma unroll
         for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
@@ -775,30 +820,26 @@ __device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const
             const bool have = r >= head && r < admitted && r < adm_new;
             mm[u] = have ? __ldcg(A.m + r) : -1;
             pp[u] = have ? __ldcg(A.pos + r) : -1;
+            nn[u] = have ? __ldcg(A.ntok + r) : 0;
         }
 #pragma unroll
         for (int u = 0; u < KLPM_RUN_SLOTS; ++u) {
             if (base + u * TT >= adm_new) break;                               // warp-uniform
             const long long r = base + u * TT + gtid;
             const bool fresh = r >= head && r >= admitted && r < adm_new;
-            int32_t m = mm[u], hint = 0;
+            int32_t m = mm[u], hint = 0, ntok = nn[u];
             long long pos = pp[u];
             bool dirty = false;
             unsigned wm = __ballot_sync(FULL_MASK, fresh);
             if (wm) {                                  // newly arrived queries: full walk, one warp each
                 const int32_t* q = nullptr; int32_t qlen = 0;
-                if (fresh) {
-                    const int32_t qi = __ldg(A.ord + r);
-                    const int64_t lo = __ldg(A.off + qi);
-                    qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
-                    q = A.tok + lo;
-                }
+                if (fresh) { qlen = __ldg(A.slen + r); q = A.tok + __ldg(A.soff + r); }
                 while (wm) {
                     const int src = __ffs(wm) - 1; wm &= wm - 1;
                     const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
                     const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
                     Term t = walk<false>(T, qq, ql);
-                    if (lane == src) { m = t.m; hint = t.node; pos = t.pos; dirty = true; }
+                    if (lane == src) { m = t.m; hint = t.node; pos = t.pos; ntok = t.m < ql ? __ldg(qq + t.m) : 0; dirty = true; }
                 }
             }
             const bool waiting = fresh || m >= 0;
@@ -816,6 +857,7 @@ __device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const
                 if (a != hint || m != m0) {
                     hint = a;
                     pos = a == 0 ? -1 : __ldcg(T.span_off + a) + (m - __ldcg(T.depth_start + a)) - 1;
+                    if (m != m0) ntok = m < __ldg(A.slen + r) ? __ldg(A.tok + __ldg(A.soff + r) + m) : 0;
                     dirty = true;
                 } else {
                     hint = -1;                          // unchanged: do not rewrite
@@ -824,12 +866,10 @@ __device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const
             // tied with the prompt processed last: it may now match into that prompt's new leaf
             bool cmp = false;
             const int32_t* q = nullptr; int32_t qlen = 0;
-            if (waiting && !fresh && last_valid && pos == last_pos && m == last_m) {
-                const int32_t qi = __ldg(A.ord + r);
-                const int64_t lo = __ldg(A.off + qi);
-                qlen = (int32_t)(__ldg(A.off + qi + 1) - lo);
-                q = A.tok + lo;
-                cmp = m < qlen && __ldg(q + m) == __ldg(last_x + m);
+            if (waiting && !fresh && last_valid && pos == last_pos && m == last_m && ntok == last_xm) {
+                qlen = __ldg(A.slen + r);
+                q = A.tok + __ldg(A.soff + r);
+                cmp = m < qlen;
             }
             unsigned cm = __ballot_sync(FULL_MASK, cmp);
             while (cm) {
@@ -838,10 +878,14 @@ __device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const
                 const int32_t ql = __shfl_sync(FULL_MASK, qlen, src);
                 const int32_t lim = (ql < last_len ? ql : last_len) - last_m;
                 const int32_t e = first_mismatch<true>(qq + last_m, last_x + last_m, lim);
-                if (lane == src) { m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1; dirty = true; }
+                if (lane == src) {
+                    m = last_m + e; hint = last_leaf; pos = last_leaf_off + e - 1;
+                    ntok = m < ql ? __ldg(qq + m) : 0;
+                    dirty = true;
+                }
             }
             if (waiting) {
-                if (dirty) { A.m[r] = m; A.pos[r] = pos; if (hint >= 0) A.hint[r] = hint; }
+                if (dirty) { A.m[r] = m; A.pos[r] = pos; A.ntok[r] = ntok; if (hint >= 0) A.hint[r] = hint; }
                 const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
                 if (key > best) best = key;
             }
@@ -946,37 +990,42 @@ run_kernel(TreeDev T, RunArgs A) {
             const int32_t m = __ldcg(A.m + slot);
             const int32_t hint = __ldcg(A.hint + slot);
             const long long pos = __ldcg(A.pos + slot);
-            const int64_t lo = __ldg(A.off + qi);
-            const int32_t len = (int32_t)(__ldg(A.off + qi + 1) - lo);
-            const long long tj = __ldg(A.arrival + qi);
-            const int32_t* x = A.tok + lo;
+            const int32_t ntok = __ldcg(A.ntok + slot);
+            const int32_t len = __ldg(A.slen + slot);
+            const long long tj = __ldg(A.sorted_t + slot);
+            const int32_t* x = A.tok + __ldg(A.soff + slot);
             // where the cached part ends, and what the insertion is going to allocate
             int32_t a = hint;
-            while (a != 0 && m <= T.depth_start[a]) a = T.parent[a];
-            const int32_t o = a == 0 ? 0 : m - T.depth_start[a];
-            const bool mid = a != 0 && o < T.span_len[a];
-            const int64_t so = a == 0 ? 0 : T.span_off[a];
+            int32_t a_ds = T.depth_start[a], a_sl = T.span_len[a], a_par = T.parent[a];   // read side by side
+            int64_t a_so = T.span_off[a];
+            while (a != 0 && m <= a_ds) {
+                a = a_par;
+                a_ds = T.depth_start[a]; a_sl = T.span_len[a]; a_par = T.parent[a]; a_so = T.span_off[a];
+            }
+            const int32_t o = a == 0 ? 0 : m - a_ds;
+            const bool mid = a != 0 && o < a_sl;
+            const int64_t so = a == 0 ? 0 : a_so;
             const int32_t unc = len - m;
             const int32_t leaf_pred = unc > 0 ? (int32_t)s_st.n_nodes + (mid ? 1 : 0) : -1;
             const long long leaf_off_pred = unc > 0 ? ((s_st.pool_used + 3) & ~3LL) + (m & 3) : 0;
-            // warm the lines the serial insertion reads one after the other
+            // Three lanes read, side by side, what the serial insertion would otherwise wait for one after
+            // the other: the tokens that key its table operations, then the first slot each will probe.
+            InsertPre pre;
             {
                 int32_t v = 0;
-                if (lane == 0 && m < len) v = __ldcg(x + m);
+                if (lane == 0 && unc > 0) v = ntok;
                 if (lane == 1 && mid) v = __ldcg(T.pool + so + o);
                 if (lane == 2 && mid) v = __ldcg(T.pool + so);
-                const int32_t xm = __shfl_sync(FULL_MASK, v, 0), pt = __shfl_sync(FULL_MASK, v, 1), ft = __shfl_sync(FULL_MASK, v, 2);
                 const int32_t end = mid ? (int32_t)s_st.n_nodes : a;
-                unsigned long long key = 0;
+                unsigned long long key = 0, seen = 0;
                 bool want = false;
-                if (lane == 0) { key = make_key(end, xm); want = m < len; }
-                if (lane == 1) { key = make_key(end, pt); want = mid; }
-                if (lane == 2) { key = make_key(T.parent[a], ft); want = mid; }
-                if (want) {
-                    const Entry* e = T.table + (hash_key(key) & T.table_mask);
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(e));
-                }
+                if (lane == 0) { key = make_key(end, v); want = unc > 0; }
+                if (lane == 1) { key = make_key(end, v); want = mid; }
+                if (lane == 2) { key = make_key(a_par, v); want = mid; }
+                if (want) seen = __ldcg(&T.table[hash_key(key) & T.table_mask].key);
                 for (int32_t i = lane * 32; i < unc; i += 32 * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + m + i));
+                pre.xm = __shfl_sync(FULL_MASK, v, 0); pre.pt = __shfl_sync(FULL_MASK, v, 1); pre.ft = __shfl_sync(FULL_MASK, v, 2);
+                pre.k_leaf = __shfl_sync(FULL_MASK, seen, 0); pre.k_low = __shfl_sync(FULL_MASK, seen, 1); pre.k_par = __shfl_sync(FULL_MASK, seen, 2);
             }
             if (lane == 0) {
                 s_j[0] = m; s_j[1] = len; s_x = x;
@@ -987,12 +1036,12 @@ run_kernel(TreeDev T, RunArgs A) {
                 if (A.completion) A.completion[qi] = R;
                 A.m[slot] = -1;
                 long long h = head;
-                while (h < A.n && (h == slot || (h < adm_new && __ldcg(A.m + h) < 0))) ++h;
+                if (slot == head) while (h < A.n && (h == slot || (h < adm_new && __ldcg(A.m + h) < 0))) ++h;
                 RunBcast nb = s_bc;
                 nb.head = h; nb.now = R; nb.admitted = adm_new;
                 nb.evicted = 0;
                 nb.last_valid = unc > 0; nb.last_q = qi; nb.last_m = m; nb.last_len = len;
-                nb.last_leaf = leaf_pred; nb.last_pos = pos; nb.last_leaf_off = leaf_off_pred;
+                nb.last_leaf = leaf_pred; nb.last_pos = pos; nb.last_leaf_off = leaf_off_pred; nb.last_xm = pre.xm;
                 s_bc = nb;
                 // may the scanners start on the next decision while the tree is being updated?
                 long long adm_next, now_next;
@@ -1004,7 +1053,7 @@ run_kernel(TreeDev T, RunArgs A) {
                     __threadfence();
                     atomicExch(&A.sy->seq, (unsigned long long)(c + 1));
                 }
-                insert_serial(T0, x, len, m, hint, &s_out);
+                insert_serial(T0, x, len, m, hint, &s_out, &pre);
                 if (s_out.ok && (s_out.leaf != leaf_pred || (unc > 0 && s_out.leaf_off != leaf_off_pred))) {
                     set_status(&s_st, RT_ERR_LIMIT);           // cannot happen: the prediction repeats the allocation rule
                     s_out.ok = 0;
@@ -1019,7 +1068,7 @@ run_kernel(TreeDev T, RunArgs A) {
             int32_t* dst = T.pool + s_out.leaf_off;
             for (int32_t i = threadIdx.x; i < unc; i += blockDim.x) dst[i] = __ldg(x + m + i);
         }
-        __threadfence();
+        if (!s_flag[0]) __threadfence();       // published next: others may walk the tree (the early mode's readers never touch it)
         __syncthreads();
         if (threadIdx.x == 0 && !s_flag[0]) {
             s_bc.evicted = s_out.evicted;
@@ -1179,6 +1228,14 @@ __global__ void rank_init_kernel(const int64_t* __restrict__ arrival, int32_t n,
     key[i] = i < n ? arrival[i] : 0x7fffffffffffffffLL;
     idx[i] = i < n ? (int32_t)i : 0x7fffffff;
 }
+__global__ void slot_arrays_kernel(const int32_t* __restrict__ ord, const int64_t* __restrict__ off, int32_t n, long long* soff, int32_t* slen) {
+    int32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    const int32_t qi = ord[r];
+    const int64_t lo = off[qi];
+    soff[r] = lo;
+    slen[r] = (int32_t)(off[qi + 1] - lo);
+}
 __global__ void bitonic_step_kernel(long long* key, int32_t* idx, long long np2, long long k, long long j) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= np2) return;
@@ -1206,6 +1263,7 @@ struct rt_tree {
     // klpm_run scratch
     long long run_cap;      // slots allocated (power of two)
     long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos;
+    long long* run_soff; int32_t* run_slen; int32_t* run_ntok;
     unsigned long long* run_partial; RunBcast* run_bc; RunSync* run_sy;
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -1236,7 +1294,8 @@ void free_tree(rt_tree* t) {
     cudaFree(d.span_off); cudaFree(d.last_access); cudaFree(d.dead); cudaFree(d.clock_owner);
     cudaFree(d.table); cudaFree(d.pool); cudaFree(d.end_node); cudaFree(d.st); cudaFree(t->match_counter);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
-    cudaFree(t->run_pos); cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
+    cudaFree(t->run_pos); cudaFree(t->run_soff); cudaFree(t->run_slen); cudaFree(t->run_ntok);
+    cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
     cudaFree(t->claim);
     cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
     cudaFree(t->ck_clock_owner); cudaFree(t->ck_span_off); cudaFree(t->ck_last_access); cudaFree(t->ck_dead);
@@ -1249,8 +1308,10 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     while (np2 < n) np2 <<= 1;
     if (np2 <= t->run_cap) return RT_OK;
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
-    cudaFree(t->run_pos);
+    cudaFree(t->run_pos); cudaFree(t->run_soff); cudaFree(t->run_slen); cudaFree(t->run_ntok);
+    t->run_ntok = nullptr;
     t->run_key = nullptr; t->run_ord = nullptr; t->run_m = nullptr; t->run_hint = nullptr; t->run_pos = nullptr;
+    t->run_soff = nullptr; t->run_slen = nullptr;
     t->run_cap = 0;
     rt_status s;
     if ((s = dalloc(&t->run_key, np2))) return s;
@@ -1258,6 +1319,9 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->run_m, np2))) return s;
     if ((s = dalloc(&t->run_hint, np2))) return s;
     if ((s = dalloc(&t->run_pos, np2))) return s;
+    if ((s = dalloc(&t->run_soff, np2))) return s;
+    if ((s = dalloc(&t->run_slen, np2))) return s;
+    if ((s = dalloc(&t->run_ntok, np2))) return s;
     t->run_cap = np2;
     return RT_OK;
 }
@@ -1602,6 +1666,7 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
         for (long long k = 2; k <= np2; k <<= 1)
             for (long long j = k >> 1; j > 0; j >>= 1)
                 bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_key, tree->run_ord, np2, k, j);
+        slot_arrays_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, d_q_offsets, n, tree->run_soff, tree->run_slen);
         CK(cudaGetLastError());
     }
     RunBcast bc0;
@@ -1614,6 +1679,7 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
     a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.n = n;
     a.policy = params->policy; a.k = params->k; a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
     a.order = d_order; a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
+    a.soff = tree->run_soff; a.slen = tree->run_slen; a.ntok = tree->run_ntok;
     a.ord = tree->run_ord; a.sorted_t = tree->run_key; a.m = tree->run_m; a.hint = tree->run_hint; a.pos = tree->run_pos;
     a.partial = tree->run_partial; a.bc = tree->run_bc; a.sy = tree->run_sy;
     const int threads = KLPM_RUN_THREADS;
