@@ -302,10 +302,12 @@ def run_ours(args):
                    "tree_tokens": stats0["tokens"], "budget_tokens": w.budget_tokens,
                    "l2": "inputs larger than L2" if q_tok.numel() * 4 > 2 * 126e6 else "inputs smaller than L2",
                    "seed": seed, "recipe": w.recipe, "setup_s": t_setup},
-        "roofline": {"bound": "hbm", "kernel": "match_batch_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "match_chain_kernel" if w.budget_tokens == 0 else "match_batch_kernel", "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": alg_bytes, "traffic": TRAFFIC.get((name, args.scale))},
+        "decision_loop": {"kernel": "run_kernel", "bound": "latency", "us_per_decision": 1e6 * t_run / (nq * args.steps),
+                          "note": "sequential chain: every pick depends on the tree after the previous one"},
         "e2e": {"value": world * nq / e2e_s, "unit": "queries/s (whole step, copies included)",
                 "ms_per_step": 1e3 * e2e_s, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps,
