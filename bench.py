@@ -197,7 +197,8 @@ def run_ours(args):
     tree, q_tok, q_off, arr = device_workload(w, device)
     t_setup = time.perf_counter() - t_setup
     stats0 = K.rt_stats(tree)
-    params = K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick)
+    policy = {"klpm": K.POLICY_KLPM, "fcfs": K.POLICY_FCFS, "lpm": K.POLICY_LPM}[args.policy]
+    params = K.make_params(policy, k, 0, 1, w.start_tick)
 
     match_len = torch.zeros(nq, dtype=torch.int32, device=device)
     order = torch.zeros(nq, dtype=torch.int32, device=device)
@@ -297,7 +298,7 @@ def run_ours(args):
         "dtype": "int32", "data": "synthetic",
         "decisions_per_sec": world * nq * args.steps / t_run,
         "phases_ms_per_step": {"rt_match_batch": 1e3 * t_match / args.steps, "klpm_run": 1e3 * t_run / args.steps},
-        "config": {"workload": name, "scale": args.scale if name != "tiny" else 1.0, "k": k, "policy": "k-LPM",
+        "config": {"workload": name, "scale": args.scale if name != "tiny" else 1.0, "k": k, "policy": args.policy,
                    "queries": nq, "query_tokens": int(q_tok.numel()), "tree_nodes": stats0["n_nodes"],
                    "tree_tokens": stats0["tokens"], "budget_tokens": w.budget_tokens,
                    "l2": "inputs larger than L2" if q_tok.numel() * 4 > 2 * 126e6 else "inputs smaller than L2",
@@ -313,7 +314,11 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
         "result": {"total_uncached_tokens": int(unc.sum().item()),
-                   "ttft_p50": int(ttft_cpu.kthvalue(max(1, nq // 2)).values), "ttft_max": int(ttft_cpu.max()),
+                   "ttft_p50": int(ttft_cpu.kthvalue(max(1, nq // 2)).values),
+                   "ttft_p90": int(ttft_cpu.kthvalue(max(1, (nq * 90) // 100)).values),
+                   "ttft_p95": int(ttft_cpu.kthvalue(max(1, (nq * 95) // 100)).values),
+                   "ttft_p99": int(ttft_cpu.kthvalue(max(1, (nq * 99) // 100)).values),
+                   "ttft_max": int(ttft_cpu.max()), "ticks_per_sec": w.ticks_per_sec,
                    "tree_tokens_after": stats1["tokens"]},
     }
     if not args.no_cpu_baseline and world == 1:
@@ -428,6 +433,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--k", type=int, default=0, help="k of k-LPM (0 = the configuration's own)")
+    ap.add_argument("--policy", default="klpm", choices=["klpm", "fcfs", "lpm"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     args = ap.parse_args()

@@ -97,22 +97,26 @@ __device__ __forceinline__ unsigned long long hash_key(unsigned long long k) {
 __device__ __forceinline__ void set_status(TreeState* st, int code) { atomicCAS(&st->status, 0, code); }
 
 // First index in [0, n) where a and b differ, or n.  Warp-cooperative: every lane gets the result.
-// Lane l reads elements l, l+32, l+64, l+96 of each 128-token chunk: each load instruction of the warp
-// is one contiguous 128-byte request, whatever the 4-byte phase of the two streams.
-template <bool RO>
+// Lane l reads elements l, l+32, l+64, ... of each chunk: each load instruction of the warp is one
+// contiguous 128-byte request, whatever the 4-byte phase of the two streams.  U * 128 tokens of both
+// streams are requested before the first of them is examined, so a long common prefix costs one memory
+// latency per U * 128 tokens.
+template <bool RO, int U = 4>
 __device__ __forceinline__ int32_t first_mismatch(const int32_t* __restrict__ a, const int32_t* __restrict__ b, int32_t n) {
     const int lane = threadIdx.x & 31;
-    for (int32_t base = 0; base < n; base += 128) {
-        int32_t x[4], y[4];
+    constexpr int R = 4 * U;
+    for (int32_t base = 0; base < n; base += 32 * R) {
+        int32_t x[R], y[R];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < R; ++j) {
             int32_t idx = base + j * 32 + lane;
             bool in = idx < n;
             x[j] = in ? ld32<RO>(a + idx) : 0;
             y[j] = in ? ld32<RO>(b + idx) : 0;
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < R; ++j) {
+            if (base + j * 32 >= n) break;                  // warp-uniform
             unsigned bad = __ballot_sync(FULL_MASK, x[j] != y[j]);
             if (bad) return base + j * 32 + (__ffs(bad) - 1);
         }

@@ -336,8 +336,38 @@ def adversarial(seed: int = 4, scale: float = 1.0) -> Workload:
                                 cut="U[1,16384]", tail="U[36,164]"))
 
 
+def prefix_ratio(u: int, d: int, seed: int = 5, n: int = 2000, rep: int = 4, scale: float = 1.0) -> Workload:
+    """The prefix-to-prompt ratio experiment of Appendix C.2 under the cost model: a regular-arrival-style
+    queue (Definition 3) of n random-string prompts (user)(doc), each user substring of length u shared by
+    `rep` prompts, each doc substring of length d unique, shuffled, arriving as a Poisson stream of 80
+    queries per second; empty cache; policies k = 1, 4 and LPM.  One tick = one prefilled token at a rate
+    of 300,000 tokens per second (offered load about 1 for u = d = 3000 with perfect reuse)."""
+    vocab = 128_256
+    n = max(rep, int(n * scale) // rep * rep)
+    tps = 300_000
+    user = torch.arange(n) // rep
+    order = torch.argsort(uniform_u53(seed, _K_PICK_Q, n))          # random shuffle of the queue
+    user = user[order]
+    ukeys = stream_key(seed, _K_PREFIX, torch.arange(n // rep))
+    dkeys = stream_key(seed, _K_SUFFIX_Q, torch.arange(n))
+    e0 = torch.full((n,), u, dtype=torch.int64)
+    q = SegmentedPrompts(vocab, [ukeys[user], dkeys], [e0, e0 + d])
+    empty = SegmentedPrompts(vocab, [torch.zeros(0, dtype=torch.int64)] * 2, [torch.zeros(0, dtype=torch.int64)] * 2)
+    arr = poisson_arrivals(seed, _K_ARRIVAL, n, 80.0, tps)
+    return Workload("ratio_%d_%d" % (u, d), vocab, empty, q, arr, tps, (4,), 0,
+                    recipe=dict(seed=seed, scale=scale, u=u, d=d, n=n, rep=rep, rate=80))
+
+
+def _ratio(u, d):
+    def make(seed: int = 5, scale: float = 1.0) -> Workload:
+        return prefix_ratio(u, d, seed=seed, scale=scale)
+    return make
+
+
 WORKLOADS = {"tiny": tiny, "medium": medium, "hierarchical": hierarchical,
-             "streaming": streaming, "adversarial": adversarial}
+             "streaming": streaming, "adversarial": adversarial,
+             "ratio_1000_5000": _ratio(1000, 5000), "ratio_3000_3000": _ratio(3000, 3000),
+             "ratio_5000_1000": _ratio(5000, 1000)}
 
 
 # ---------------------------------------------------------------------------

@@ -382,3 +382,19 @@ def test_checkpoint_and_rollback(K):
         assert torch.equal(a, b)
     m, _, _ = gpu_match(K, tree, qt, qo)
     assert np.array_equal(m, oracle_tree(pt, po).match(qt.numpy(), qo.numpy()))
+
+
+# ------------------------------------------------------------------ prefix-to-prompt ratio experiment (Appendix C.2)
+
+@pytest.mark.parametrize("u,d", [(1000, 5000), (3000, 3000), (5000, 1000)])
+def test_run_prefix_ratio_experiment(K, u, d):
+    """n = 2000 random-string prompts, 4 replicas per prefix, Poisson 80/s, policies k = 1, 4 and LPM."""
+    w = W.prefix_ratio(u, d)
+    qt, qo = w.queries.materialize()
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    for policy, k in ((K.POLICY_KLPM, 1), (K.POLICY_KLPM, 4), (K.POLICY_LPM, 1)):
+        got = run_gpu(K, *e, qt, qo, w.arrivals, policy, k)
+        want = run_oracle(*e, qt, qo, w.arrivals, policy, k)
+        assert_same_schedule(got, want)
+    # every prefix is prefilled once, every doc once: total uncached tokens under an unbounded tree cache
+    assert int(got[1].sum()) == (w.queries.n // 4) * u + w.queries.n * d
