@@ -398,3 +398,34 @@ def test_run_prefix_ratio_experiment(K, u, d):
         assert_same_schedule(got, want)
     # every prefix is prefilled once, every doc once: total uncached tokens under an unbounded tree cache
     assert int(got[1].sum()) == (w.queries.n // 4) * u + w.queries.n * d
+
+
+# ------------------------------------------------------------------ long edges, every alignment, degenerate streams
+
+def test_match_long_edges_all_alignments(K):
+    """One 70,001-token cached prompt plus prefixes of it; queries that agree with it for every length in a
+    ragged set (around the 128-token chunks and the 16-byte units), starting at every 4-byte phase."""
+    g = torch.Generator().manual_seed(7)
+    base = torch.randint(0, 50000, (70001,), generator=g, dtype=torch.int32).tolist()
+    cached = [base, base[:4097], base[:130] + [7, 7, 7], base[:1]]
+    lens = [0, 1, 2, 3, 4, 5, 127, 128, 129, 255, 256, 257, 511, 4096, 4097, 4098, 65535, 70000, 70001]
+    queries = []
+    for i, n in enumerate(lens):
+        queries.append(base[:n] + [60000 + i])            # diverges right after n tokens
+        queries.append(base[:n])                          # ends there
+        queries.append([1] * (i % 4))                     # filler that shifts the alignment of what follows
+    check_match(K, *csr(cached), *csr(queries))
+
+
+def test_run_degenerate_streams(K):
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    # one query; identical prompts arriving together; empty prompts; everything at the same tick
+    for prompts, arr in [([[5, 6, 7]], [3]),
+                         ([[1, 2, 3]] * 9, [0] * 9),
+                         ([[], [], [4], []], [0, 0, 0, 0]),
+                         ([[9] * 300, [9] * 299 + [1], [9] * 300 + [2], [9] * 150], [5, 5, 5, 5])]:
+        qt, qo = csr(prompts)
+        for policy, k in ((0, 1), (1, 1), (2, 2)):
+            got = run_gpu(K, *e, qt, qo, arr, policy, k)
+            want = run_oracle(*e, qt, qo, arr, policy, k, tier=oracle.TIER_REMATCH)
+            assert_same_schedule(got, want)
