@@ -127,6 +127,14 @@ rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, cons
                       int32_t nq, int64_t pick_counter, const klpm_params* params, int32_t* d_pick,
                       void* stream);
 
+/* The kk best longest-match candidates of one snapshot of the queue, best first: d_out[j] (int32[kk]) is the
+ * waiting query that ranks j-th by (largest d_match_len, then smallest arrival, then smallest index), or -1
+ * when fewer than kk queries are waiting.  1 <= kk <= 64.  These are the k-1 picks that follow an oldest-first
+ * pick in Algorithm 1 *if match lengths did not move*; they do move when a processed prompt extends the cache
+ * (klpm_run accounts for that, this call does not).  Uses library-owned scratch allocated on first use. */
+rt_status klpm_select_topk(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting,
+                           int32_t nq, int32_t kk, int32_t* d_out, void* stream);
+
 /* klpm_select for callers that must not allocate device memory.  (The paper has no counterpart of this
  * entry point; it exists for how the library gets embedded, not for the method.)
  *

@@ -67,6 +67,8 @@ _lib.rt_destroy.restype = _i32
 _lib.rt_destroy.argtypes = [_vp]
 _lib.klpm_select.restype = _i32
 _lib.klpm_select.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
+_lib.klpm_select_topk.restype = _i32
+_lib.klpm_select_topk.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp]
 _lib.klpm_select_noalloc.restype = _i32
 _lib.klpm_select_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
 _lib.klpm_replay.restype = _i32
@@ -75,7 +77,7 @@ _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_noalloc", "klpm_replay", "klpm_run"]
+           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run"]
 
 
 def lib() -> ctypes.CDLL:
@@ -189,6 +191,13 @@ def klpm_select(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.T
     _check(_lib.klpm_select(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
                             _dev(waiting, torch.uint8, "waiting"), match_len.numel(), int(pick_counter),
                             ctypes.byref(params), _dev(pick, torch.int32, "pick"), _stream()), "klpm_select")
+
+
+def klpm_select_topk(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, out: torch.Tensor) -> None:
+    """out (int32[kk]) receives the kk best longest-match candidates of this snapshot, best first."""
+    _check(_lib.klpm_select_topk(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
+                                 _dev(waiting, torch.uint8, "waiting"), match_len.numel(), out.numel(),
+                                 _dev(out, torch.int32, "out"), _stream()), "klpm_select_topk")
 
 
 def klpm_select_noalloc(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, pick_counter: int,

@@ -672,6 +672,69 @@ select_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict__ arri
 }
 
 // ------------------------------------------------------------------------------------------------
+// klpm_select_topk: the kk best longest-match candidates of one queue snapshot, best first.
+// The j-th best is the best element strictly worse than the (j-1)-th in the total order
+// (match desc, arrival asc, index asc), so no element is ever marked as taken: each CTA extracts its own
+// kk best by kk passes over its slice, and the last CTA to finish merges the per-CTA lists the same way.
+// ------------------------------------------------------------------------------------------------
+#define KLPM_TOPK_MAX 64
+#define KLPM_TOPK_BLOCKS 128
+struct TopkScratch { Cand cand[KLPM_TOPK_BLOCKS * KLPM_TOPK_MAX]; unsigned int ticket; };
+
+__global__ void __launch_bounds__(512)
+select_topk_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict__ arrival, const uint8_t* __restrict__ waiting,
+                   int32_t nq, int32_t kk, int32_t* out, TopkScratch* sc) {
+    __shared__ Cand s_c[32];
+    __shared__ Cand s_prev;
+    __shared__ bool s_last;
+    Cand prev; prev.m = 0; prev.idx = -1; prev.t = 0;          // idx < 0: no bound yet
+    for (int j = 0; j < kk; ++j) {
+        Cand best; best.m = 0; best.idx = -1; best.t = 0;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nq; i += (int64_t)gridDim.x * blockDim.x) {
+            if (__ldg(waiting + i)) {
+                Cand c; c.m = __ldg(mlen + i); c.idx = (int32_t)i; c.t = __ldg(arrival + i);
+                if (prev.idx < 0 || better_lpm(prev, c)) best = cand_best<true>(best, c);
+            }
+        }
+        best = block_best<true>(best, s_c);
+        if (threadIdx.x == 0) { s_prev = best; sc->cand[blockIdx.x * KLPM_TOPK_MAX + j] = best; }
+        __syncthreads();
+        prev = s_prev;
+        __syncthreads();
+        if (prev.idx < 0) {                                     // slice exhausted: pad the rest
+            if (threadIdx.x == 0) for (int r = j + 1; r < kk; ++r) sc->cand[blockIdx.x * KLPM_TOPK_MAX + r] = prev;
+            break;
+        }
+    }
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&sc->ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    prev.m = 0; prev.idx = -1; prev.t = 0;
+    bool done = false;
+    for (int j = 0; j < kk; ++j) {
+        Cand best; best.m = 0; best.idx = -1; best.t = 0;
+        if (!done) {
+            for (int e = threadIdx.x; e < (int)gridDim.x * kk; e += blockDim.x) {
+                const Cand* src = &sc->cand[(e / kk) * KLPM_TOPK_MAX + (e % kk)];
+                Cand c; c.m = __ldcg(&src->m); c.idx = __ldcg(&src->idx); c.t = __ldcg(&src->t);
+                if (c.idx >= 0 && (prev.idx < 0 || better_lpm(prev, c))) best = cand_best<true>(best, c);
+            }
+        }
+        __syncthreads();
+        best = block_best<true>(best, s_c);
+        if (threadIdx.x == 0) { s_prev = best; out[j] = best.idx; }
+        __syncthreads();
+        if (s_prev.idx < 0) done = true; else prev = s_prev;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) sc->ticket = 0;
+}
+
+// ------------------------------------------------------------------------------------------------
 // klpm_select_noalloc: the same decision as klpm_select, with the per-CTA partial results kept in a
 // fixed array that is part of the library image instead of memory obtained from cudaMalloc.
 // ------------------------------------------------------------------------------------------------
@@ -1335,6 +1398,7 @@ bool params_ok(const klpm_params* p) {
 }
 
 SelectScratch* g_select_scratch[64] = {nullptr};
+TopkScratch* g_topk_scratch[64] = {nullptr};
 StaticSelectScratch* g_select_static_addr[64] = {nullptr};   // device address of g_select_static, per device
 
 // Many prompts at once into a tree without a budget (see the bulk kernels).  Waits for the stream once per round.
@@ -1596,6 +1660,27 @@ rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, cons
     cudaStream_t s = (cudaStream_t)stream;
     if (fcfs_turn) select_kernel<false><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, g_select_scratch[dev]);
     else select_kernel<true><<<(unsigned)blocks, 512, 0, s>>>(d_match_len, d_arrival, d_waiting, nq, d_pick, g_select_scratch[dev]);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status klpm_select_topk(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting, int32_t nq,
+                           int32_t kk, int32_t* d_out, void* stream) {
+    if (nq < 0 || kk < 1 || kk > KLPM_TOPK_MAX || !d_out || (nq > 0 && (!d_match_len || !d_arrival || !d_waiting))) return RT_ERR_INVALID;
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return RT_ERR_INVALID;
+    if (!g_topk_scratch[dev]) {
+        TopkScratch* p = nullptr;
+        CK(cudaMalloc((void**)&p, sizeof(TopkScratch)));
+        CK(cudaMemset(p, 0, sizeof(TopkScratch)));
+        g_topk_scratch[dev] = p;
+    }
+    long long blocks = ((long long)nq + 4095) / 4096;
+    if (blocks < 1) blocks = 1;
+    if (blocks > KLPM_TOPK_BLOCKS) blocks = KLPM_TOPK_BLOCKS;
+    select_topk_kernel<<<(unsigned)blocks, 512, 0, (cudaStream_t)stream>>>(d_match_len, d_arrival, d_waiting, nq, kk, d_out,
+                                                                            g_topk_scratch[dev]);
     CK(cudaGetLastError());
     return RT_OK;
 }

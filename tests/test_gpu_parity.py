@@ -429,3 +429,22 @@ def test_run_degenerate_streams(K):
             got = run_gpu(K, *e, qt, qo, arr, policy, k)
             want = run_oracle(*e, qt, qo, arr, policy, k, tier=oracle.TIER_REMATCH)
             assert_same_schedule(got, want)
+
+
+@pytest.mark.parametrize("n,kk", [(1, 3), (50, 7), (5000, 1), (5000, 16), (300001, 64)])
+def test_select_topk_snapshot(K, n, kk):
+    g = torch.Generator().manual_seed(n + kk)
+    m = torch.randint(0, 4, (n,), generator=g, dtype=torch.int32)
+    t = torch.randint(0, 30, (n,), generator=g, dtype=torch.int64) * (1 << 35)
+    waiting = (torch.rand(n, generator=g) < 0.5).to(torch.uint8)
+    out = torch.full((kk,), -9, dtype=torch.int32, device="cuda")
+    for _ in range(2):                                   # the scratch is reused
+        K.klpm_select_topk(dev(m), dev(t), dev(waiting), out)
+        idx = [i for i in range(n) if waiting[i]]
+        idx.sort(key=lambda i: (-int(m[i]), int(t[i]), i))
+        want = (idx + [-1] * kk)[:kk]
+        assert out.tolist() == want
+    # its first entry is klpm_select's longest-match pick
+    pick = torch.zeros(1, dtype=torch.int32, device="cuda")
+    K.klpm_select(dev(m), dev(t), dev(waiting), 1, K.make_params(K.POLICY_LPM), pick)
+    assert int(pick.item()) == want[0]
