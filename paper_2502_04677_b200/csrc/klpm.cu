@@ -54,6 +54,7 @@ struct TreeDev {
     int32_t* depth_start;
     int32_t* span_len;
     int32_t* nchild;
+    int32_t* first_tok;       // first token of the node's edge (= pool[span_off])
     int64_t* span_off;
     int64_t* last_access;
     uint8_t* dead;
@@ -397,13 +398,16 @@ __device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o, const Inse
     int64_t off = T.span_off[v];
     T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = off; T.span_len[u] = o;
     T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = T.last_access[v];
-    const long long slot = pre ? table_find_seen(T, par, pre->ft, pre->k_par) : table_find(T, par, __ldcg(T.pool + off));
+    const int32_t ft = pre ? pre->ft : __ldcg(T.pool + off);
+    const int32_t pt = pre ? pre->pt : __ldcg(T.pool + off + o);
+    T.first_tok[u] = ft; T.first_tok[v] = pt;
+    const long long slot = pre ? table_find_seen(T, par, ft, pre->k_par) : table_find(T, par, ft);
     int64_t chain_end = off + len;
     if (slot >= 0) { T.table[slot].child = u; T.table[slot].span_len = o; chain_end = T.table[slot].chain_end; }
     else set_status(S, RT_ERR_LIMIT);
     T.span_off[v] = off + o; T.span_len[v] = len - o; T.depth_start[v] = ds + o; T.parent[v] = u;
-    const long long ls = pre ? table_put_seen(T, u, pre->pt, v, len - o, off + o, chain_end, pre->k_low, -1)
-                             : table_put_seen(T, u, __ldcg(T.pool + off + o), v, len - o, off + o, chain_end, 0ULL, (long long)(hash_key(make_key(u, __ldcg(T.pool + off + o))) & T.table_mask));
+    const long long ls = pre ? table_put_seen(T, u, pt, v, len - o, off + o, chain_end, pre->k_low, -1)
+                             : table_put_seen(T, u, pt, v, len - o, off + o, chain_end, 0ULL, (long long)(hash_key(make_key(u, pt)) & T.table_mask));
     if (ls < 0) set_status(S, RT_ERR_CAPACITY);
     *low_slot = ls;
     T.end_node[off + o - 1] = u;
@@ -474,8 +478,10 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
         T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = clock;
         T.clock_owner[clock] = leaf;
         T.nchild[end]++;
-        const long long put = pre ? table_put_seen(T, end, pre->xm, leaf, unc, off, off + unc, pre->k_leaf, low_slot)
-                                  : (table_put(T, end, __ldcg(x + m), leaf, unc, off, off + unc) ? 0 : -1);
+        const int32_t xm = pre ? pre->xm : __ldcg(x + m);
+        T.first_tok[leaf] = xm;
+        const long long put = pre ? table_put_seen(T, end, xm, leaf, unc, off, off + unc, pre->k_leaf, low_slot)
+                                  : (table_put(T, end, xm, leaf, unc, off, off + unc) ? 0 : -1);
         if (put < 0) { set_status(S, RT_ERR_CAPACITY); return; }
         T.end_node[off + unc - 1] = leaf;
         S->tokens_live += unc;
@@ -1063,15 +1069,14 @@ run_kernel(TreeDev T, RunArgs A) {
             const int32_t* x = A.tok + __ldg(A.soff + slot);
             // where the cached part ends, and what the insertion is going to allocate
             int32_t a = hint;
-            int32_t a_ds = T.depth_start[a], a_sl = T.span_len[a], a_par = T.parent[a];   // read side by side
-            int64_t a_so = T.span_off[a];
+            int32_t a_ds = T.depth_start[a], a_sl = T.span_len[a], a_par = T.parent[a], a_ft = T.first_tok[a];   // side by side
+            const int32_t below = __ldcg(T.pool + (pos + 1));       // the pool token under the cut, if there is a cut
             while (a != 0 && m <= a_ds) {
                 a = a_par;
-                a_ds = T.depth_start[a]; a_sl = T.span_len[a]; a_par = T.parent[a]; a_so = T.span_off[a];
+                a_ds = T.depth_start[a]; a_sl = T.span_len[a]; a_par = T.parent[a]; a_ft = T.first_tok[a];
             }
             const int32_t o = a == 0 ? 0 : m - a_ds;
             const bool mid = a != 0 && o < a_sl;
-            const int64_t so = a == 0 ? 0 : a_so;
             const int32_t unc = len - m;
             const int32_t leaf_pred = unc > 0 ? (int32_t)s_st.n_nodes + (mid ? 1 : 0) : -1;
             const long long leaf_off_pred = unc > 0 ? ((s_st.pool_used + 3) & ~3LL) + (m & 3) : 0;
@@ -1081,8 +1086,8 @@ run_kernel(TreeDev T, RunArgs A) {
             {
                 int32_t v = 0;
                 if (lane == 0 && unc > 0) v = ntok;
-                if (lane == 1 && mid) v = __ldcg(T.pool + so + o);
-                if (lane == 2 && mid) v = __ldcg(T.pool + so);
+                if (lane == 1 && mid) v = below;
+                if (lane == 2 && mid) v = a_ft;
                 const int32_t end = mid ? (int32_t)s_st.n_nodes : a;
                 unsigned long long key = 0, seen = 0;
                 bool want = false;
@@ -1219,6 +1224,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                         const int64_t so = T.span_off[node];
                         T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
                         T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
+                        T.first_tok[u] = T.pool[so]; T.first_tok[node] = T.pool[so + off];
                         long long slot = table_find(T, par, T.pool[so]);
                         int64_t chain_end = so + sl;
                         if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = T.table[slot].chain_end; }
@@ -1261,6 +1267,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                     } else {
                         T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
                         T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
+                        T.first_tok[leaf] = __ldg(x + m);
                         T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
                         T.table[won].chain_end = po + unc;
                         T.end_node[po + unc - 1] = (int32_t)leaf;
@@ -1336,7 +1343,7 @@ struct rt_tree {
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
     // checkpoint (rt_checkpoint / rt_rollback): copies of everything a later call can modify
     bool ck_valid;
-    int32_t *ck_parent, *ck_depth_start, *ck_span_len, *ck_nchild, *ck_clock_owner;
+    int32_t *ck_parent, *ck_depth_start, *ck_span_len, *ck_nchild, *ck_clock_owner, *ck_first_tok;
     int64_t *ck_span_off, *ck_last_access;
     uint8_t* ck_dead;
     Entry* ck_table;
@@ -1357,7 +1364,8 @@ template <typename P> rt_status dalloc(P** p, size_t count) {
 
 void free_tree(rt_tree* t) {
     TreeDev& d = t->dev;
-    cudaFree(d.parent); cudaFree(d.depth_start); cudaFree(d.span_len); cudaFree(d.nchild);
+    cudaFree(d.parent); cudaFree(d.depth_start); cudaFree(d.span_len); cudaFree(d.nchild); cudaFree(d.first_tok);
+    cudaFree(t->ck_first_tok);
     cudaFree(d.span_off); cudaFree(d.last_access); cudaFree(d.dead); cudaFree(d.clock_owner);
     cudaFree(d.table); cudaFree(d.pool); cudaFree(d.end_node); cudaFree(d.st); cudaFree(t->match_counter);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
@@ -1472,7 +1480,7 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
     d.table_mask = cap - 1;
     rt_status s = RT_OK;
     if ((s = dalloc(&d.parent, d.max_nodes)) || (s = dalloc(&d.depth_start, d.max_nodes)) ||
-        (s = dalloc(&d.span_len, d.max_nodes)) || (s = dalloc(&d.nchild, d.max_nodes)) ||
+        (s = dalloc(&d.span_len, d.max_nodes)) || (s = dalloc(&d.nchild, d.max_nodes)) || (s = dalloc(&d.first_tok, d.max_nodes)) ||
         (s = dalloc(&d.span_off, d.max_nodes)) || (s = dalloc(&d.last_access, d.max_nodes)) ||
         (s = dalloc(&d.dead, d.max_nodes)) || (s = dalloc(&d.clock_owner, d.max_clock)) ||
         (s = dalloc(&d.table, cap)) || (s = dalloc(&d.pool, d.max_pool)) || (s = dalloc(&d.st, 1)) ||
@@ -1490,6 +1498,7 @@ rt_status rt_create(const rt_config* cfg, rt_tree** out) {
     if (e == cudaSuccess) e = cudaMemset(d.depth_start, 0, sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(d.span_len, 0, sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(d.nchild, 0, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(d.first_tok, 0, sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(d.span_off, 0, sizeof(int64_t));
     if (e == cudaSuccess) e = cudaMemset(d.last_access, 0, sizeof(int64_t));
     if (e == cudaSuccess) e = cudaMemset(d.dead, 0, 1);
@@ -1590,6 +1599,7 @@ rt_status rt_checkpoint(rt_tree* tree, void* stream) {
     if (!tree->ck_parent) {
         if ((s = dalloc(&tree->ck_parent, d.max_nodes)) || (s = dalloc(&tree->ck_depth_start, d.max_nodes)) ||
             (s = dalloc(&tree->ck_span_len, d.max_nodes)) || (s = dalloc(&tree->ck_nchild, d.max_nodes)) ||
+            (s = dalloc(&tree->ck_first_tok, d.max_nodes)) ||
             (s = dalloc(&tree->ck_span_off, d.max_nodes)) || (s = dalloc(&tree->ck_last_access, d.max_nodes)) ||
             (s = dalloc(&tree->ck_dead, d.max_nodes)) || (s = dalloc(&tree->ck_clock_owner, d.max_clock)) ||
             (s = dalloc(&tree->ck_table, cap)) || (s = dalloc(&tree->ck_st, 1))) return s;
@@ -1601,6 +1611,7 @@ rt_status rt_checkpoint(rt_tree* tree, void* stream) {
     CK(cudaMemcpyAsync(tree->ck_depth_start, d.depth_start, d.max_nodes * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(tree->ck_span_len, d.span_len, d.max_nodes * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(tree->ck_nchild, d.nchild, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(tree->ck_first_tok, d.first_tok, d.max_nodes * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(tree->ck_span_off, d.span_off, d.max_nodes * sizeof(int64_t), k, st));
     CK(cudaMemcpyAsync(tree->ck_last_access, d.last_access, d.max_nodes * sizeof(int64_t), k, st));
     CK(cudaMemcpyAsync(tree->ck_dead, d.dead, d.max_nodes, k, st));
@@ -1622,6 +1633,7 @@ rt_status rt_rollback(rt_tree* tree, void* stream) {
     CK(cudaMemcpyAsync(d.depth_start, tree->ck_depth_start, d.max_nodes * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(d.span_len, tree->ck_span_len, d.max_nodes * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(d.nchild, tree->ck_nchild, d.max_nodes * sizeof(int32_t), k, st));
+    CK(cudaMemcpyAsync(d.first_tok, tree->ck_first_tok, d.max_nodes * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(d.span_off, tree->ck_span_off, d.max_nodes * sizeof(int64_t), k, st));
     CK(cudaMemcpyAsync(d.last_access, tree->ck_last_access, d.max_nodes * sizeof(int64_t), k, st));
     CK(cudaMemcpyAsync(d.dead, tree->ck_dead, d.max_nodes, k, st));
