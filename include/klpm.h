@@ -182,6 +182,15 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
                    const int64_t* d_arrival, int32_t n, const klpm_params* params, int32_t* d_order,
                    int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
 
+/* Batch size B (Section 2.1: the order is cut into consecutive bins of B queries, and a query is finished when
+ * the last query of its bin is).  d_order (int32[n_order]) is a processing order and d_completion (int64, indexed
+ * by query) its batch-size-one completion times, as klpm_run / klpm_replay produce them; d_completion_b and
+ * d_ttft_b (int64, indexed by query; entries of queries not in d_order are left untouched) receive the
+ * completion time of the query's bin and that minus its arrival.  batch_size >= 1; must not alias the inputs. */
+rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_t* d_arrival,
+                           const int64_t* d_completion, int32_t batch_size, int64_t* d_ttft_b,
+                           int64_t* d_completion_b, void* stream);
+
 /* Version of the ABI (bumped when a signature changes). */
 int32_t klpm_abi_version(void);
 

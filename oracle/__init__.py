@@ -58,6 +58,8 @@ def lib():
         L.oc_tree_match.argtypes = [vp, vp, vp, i32, vp, i32]
         L.oc_replay.restype = i32
         L.oc_replay.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, i64, i64, i32, vp, vp, vp]
+        L.oc_batch_times.restype = None
+        L.oc_batch_times.argtypes = [vp, i32, vp, vp, i32, vp, vp]
         L.oc_schedule.restype = i32
         L.oc_schedule.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i64, i32, i32, vp, vp, vp, vp]
         _lib = L
@@ -160,3 +162,13 @@ def replay(order, tokens, offsets, arrivals, c_num: int = 0, c_den: int = 1, sta
     if rc:
         raise RuntimeError("oracle: replay failed (%d)" % rc)
     return unc, ttft, comp
+
+
+def batch_times(order, arrivals, completion, B: int):
+    """Section 2.1: with batch size B a query finishes with the last query of its bin of the order.
+    Returns ttft_b, completion_b (indexed by query)."""
+    od, a, c = _i32(order), _i64(arrivals), _i64(completion)
+    ttft = np.zeros(len(a), dtype=np.int64)
+    comp = np.zeros(len(a), dtype=np.int64)
+    lib().oc_batch_times(_p(od), len(od), _p(a), _p(c), int(B), _p(ttft), _p(comp))
+    return ttft, comp

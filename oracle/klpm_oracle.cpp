@@ -283,6 +283,19 @@ int32_t oc_replay(void* tp, const int32_t* order, int32_t n_order, const tok_t* 
     return 0;
 }
 
+// Batch size B (Section 2.1): the processing order is cut into consecutive bins of B queries; a query is
+// finished when the last query of its bin is.  completion_b / ttft_b are indexed by query.
+void oc_batch_times(const int32_t* order, int32_t n_order, const int64_t* arrival, const int64_t* completion,
+                    int32_t B, int64_t* ttft_b, int64_t* completion_b) {
+    for (int32_t i = 0; i < n_order; ++i) {
+        int32_t last = (i / B + 1) * B - 1;
+        if (last > n_order - 1) last = n_order - 1;
+        const int64_t R = completion[order[last]];
+        completion_b[order[i]] = R;
+        ttft_b[order[i]] = R - arrival[order[i]];
+    }
+}
+
 // Algorithm 1 (k-LPM) with its FCFS and LPM limits, run over the whole stream.
 // order[c] = index processed at decision c; uncached/ttft/completion are indexed by query.
 int32_t oc_schedule(void* tp, const tok_t* tok, const int64_t* off, const int64_t* arrival, int32_t n,

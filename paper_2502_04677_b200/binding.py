@@ -73,11 +73,13 @@ _lib.klpm_select_noalloc.restype = _i32
 _lib.klpm_select_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
 _lib.klpm_replay.restype = _i32
 _lib.klpm_replay.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp]
+_lib.klpm_batch_times.restype = _i32
+_lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp]
 _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run"]
+           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_batch_times"]
 
 
 def lib() -> ctypes.CDLL:
@@ -230,3 +232,11 @@ def klpm_run(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arriva
                          _dev(arrival, torch.int64, "arrival"), n, ctypes.byref(params), _dev(order, torch.int32, "order"),
                          _dev(uncached, torch.int32, "uncached"), _dev(ttft, torch.int64, "ttft"),
                          _dev(completion, torch.int64, "completion", True), _stream()), "klpm_run")
+
+
+def klpm_batch_times(order: torch.Tensor, arrival: torch.Tensor, completion: torch.Tensor, batch_size: int,
+                     ttft_b: torch.Tensor, completion_b: torch.Tensor) -> None:
+    _check(_lib.klpm_batch_times(_dev(order, torch.int32, "order"), order.numel(), _dev(arrival, torch.int64, "arrival"),
+                                 _dev(completion, torch.int64, "completion"), int(batch_size),
+                                 _dev(ttft_b, torch.int64, "ttft_b"), _dev(completion_b, torch.int64, "completion_b"),
+                                 _stream()), "klpm_batch_times")

@@ -1295,6 +1295,19 @@ __global__ void bulk_fill_kernel(int32_t* p, long long n, int32_t v) {
 }
 __global__ void bulk_finish_kernel(TreeState* S, long long n) { S->clock += n; }
 
+// batch size B: a query is finished when the last query of its bin of the processing order is
+__global__ void batch_times_kernel(const int32_t* __restrict__ order, int32_t n, const int64_t* __restrict__ arrival,
+                                   const int64_t* __restrict__ completion, int32_t B, int64_t* ttft_b, int64_t* completion_b) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    int64_t last = (i / B + 1) * (int64_t)B - 1;
+    if (last > n - 1) last = n - 1;
+    const int64_t R = __ldg(completion + __ldg(order + last));
+    const int32_t j = __ldg(order + i);
+    completion_b[j] = R;
+    ttft_b[j] = R - __ldg(arrival + j);
+}
+
 // slot order: bitonic sort of (arrival, index) pairs, padded to a power of two
 __global__ void rank_init_kernel(const int64_t* __restrict__ arrival, int32_t n, long long np2, long long* key, int32_t* idx) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -1744,6 +1757,17 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
     a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
     tree->last_stream = (cudaStream_t)stream;
     sequential_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(tree->dev, a);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
+rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_t* d_arrival, const int64_t* d_completion,
+                           int32_t batch_size, int64_t* d_ttft_b, int64_t* d_completion_b, void* stream) {
+    if (n_order < 0 || batch_size < 1 || (n_order > 0 && (!d_order || !d_arrival || !d_completion || !d_ttft_b || !d_completion_b)))
+        return RT_ERR_INVALID;
+    if (n_order == 0) return RT_OK;
+    batch_times_kernel<<<(unsigned)((n_order + 255) / 256), 256, 0, (cudaStream_t)stream>>>(d_order, n_order, d_arrival, d_completion,
+                                                                                           batch_size, d_ttft_b, d_completion_b);
     CK(cudaGetLastError());
     return RT_OK;
 }

@@ -448,3 +448,17 @@ def test_select_topk_snapshot(K, n, kk):
     pick = torch.zeros(1, dtype=torch.int32, device="cuda")
     K.klpm_select(dev(m), dev(t), dev(waiting), 1, K.make_params(K.POLICY_LPM), pick)
     assert int(pick.item()) == want[0]
+
+
+@pytest.mark.parametrize("B", [1, 2, 7, 64, 100000])
+def test_batch_times(K, B):
+    w = W.medium(scale=1 / 64)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    order, unc, ttft, comp, _ = run_gpu(K, pt, po, qt, qo, w.arrivals, K.POLICY_KLPM, 4, start=w.start_tick)
+    n = len(order)
+    tb = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    cb = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    K.klpm_batch_times(dev(torch.from_numpy(order)), dev(w.arrivals), dev(torch.from_numpy(comp)), B, tb, cb)
+    ot, oc = oracle.batch_times(order, w.arrivals.numpy(), comp, B)
+    assert np.array_equal(tb.cpu().numpy(), ot) and np.array_equal(cb.cpu().numpy(), oc)

@@ -320,3 +320,18 @@ def test_lru_evicts_least_recently_used_leaf_by_hand():
     assert t.match(*csr([[1, 1, 1], [2, 2, 2], [3, 3, 3], [4, 4, 4]])).tolist() == [0, 3, 0, 3]
     with pytest.raises(RuntimeError):
         oracle.OracleTree(2).insert(*csr([[1, 2, 3]]))
+
+
+# ---------------------------------------------------------------- batch size B (Section 2.1)
+
+def test_batch_times_by_hand_and_limits():
+    """Toy example under LPM: order x1,x3,x2,x4 completes at 10,15,25,30; with B = 2 the bins finish at 15 and 30."""
+    order = [0, 2, 1, 3]
+    comp = np.array([10, 25, 15, 30], dtype=np.int64)          # indexed by query
+    arr = [0, 0, 0, 0]
+    ttft, cb = oracle.batch_times(order, arr, comp, 2)
+    assert cb.tolist() == [15, 30, 15, 30] and ttft.tolist() == [15, 30, 15, 30]
+    assert oracle.batch_times(order, arr, comp, 1)[1].tolist() == comp.tolist()       # B = 1 changes nothing
+    assert oracle.batch_times(order, arr, comp, 9)[1].tolist() == [30] * 4            # one bin: everyone waits for the last
+    ttft, cb = oracle.batch_times(order, [0, 5, 1, 2], comp, 3)                       # ragged last bin, arrivals subtracted
+    assert cb.tolist() == [25, 25, 25, 30] and ttft.tolist() == [25, 20, 24, 28]
