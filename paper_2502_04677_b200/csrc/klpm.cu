@@ -831,6 +831,9 @@ struct RunArgs {
 
 #define KLPM_RUN_THREADS 512
 #define KLPM_RUN_SLOTS 4          // slots per thread whose state is loaded together
+#ifndef KLPM_RUN_SPT
+#define KLPM_RUN_SPT 2            // slots per scanner thread the grid is sized for
+#endif
 #define KLPM_WAIT_LIMIT (1ULL << 25)
 
 // Thread 0 of the CTA polls *p until it reaches target (bounded), then the CTA learns whether to go on.
@@ -1813,7 +1816,7 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
     if (per_sm < 1) return RT_ERR_CUDA;
     // one sequencer CTA plus scanners; small queues are handled by the sequencer alone
     long long blocks = 1;
-    if (n > threads * 8) blocks = 1 + ((long long)n + threads * KLPM_RUN_SLOTS - 1) / (threads * KLPM_RUN_SLOTS);
+    if (n > threads * 8) blocks = 1 + ((long long)n + threads * KLPM_RUN_SPT - 1) / (threads * KLPM_RUN_SPT);
     if (blocks > tree->num_sms) blocks = tree->num_sms;
     void* kargs[] = {(void*)&tree->dev, (void*)&a};
     CK(cudaLaunchCooperativeKernel((void*)run_kernel, dim3((unsigned)blocks), dim3(threads), kargs, 0, s));
