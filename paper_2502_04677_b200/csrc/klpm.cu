@@ -1085,30 +1085,27 @@ run_kernel(TreeDev T, RunArgs A) {
             const long long leaf_off_pred = unc > 0 ? ((s_st.pool_used + 3) & ~3LL) + (m & 3) : 0;
             // Three lanes read, side by side, what the serial insertion would otherwise wait for one after
             // the other: the tokens that key its table operations, then the first slot each will probe.
-            InsertPre pre;
+            // The reads are issued here and collected after the pick has been published.
+            int32_t v = 0;
+            if (lane == 0 && unc > 0) v = ntok;
+            if (lane == 1 && mid) v = below;
+            if (lane == 2 && mid) v = a_ft;
+            unsigned long long seen = 0;
             {
-                int32_t v = 0;
-                if (lane == 0 && unc > 0) v = ntok;
-                if (lane == 1 && mid) v = below;
-                if (lane == 2 && mid) v = a_ft;
                 const int32_t end = mid ? (int32_t)s_st.n_nodes : a;
-                unsigned long long key = 0, seen = 0;
+                unsigned long long key = 0;
                 bool want = false;
                 if (lane == 0) { key = make_key(end, v); want = unc > 0; }
                 if (lane == 1) { key = make_key(end, v); want = mid; }
                 if (lane == 2) { key = make_key(a_par, v); want = mid; }
                 if (want) seen = __ldcg(&T.table[hash_key(key) & T.table_mask].key);
                 for (int32_t i = lane * 32; i < unc; i += 32 * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(x + m + i));
-                pre.xm = __shfl_sync(FULL_MASK, v, 0); pre.pt = __shfl_sync(FULL_MASK, v, 1); pre.ft = __shfl_sync(FULL_MASK, v, 2);
-                pre.k_leaf = __shfl_sync(FULL_MASK, seen, 0); pre.k_low = __shfl_sync(FULL_MASK, seen, 1); pre.k_par = __shfl_sync(FULL_MASK, seen, 2);
             }
             if (lane == 0) {
                 s_j[0] = m; s_j[1] = len; s_x = x;
                 const long long now = s_bound[1];
                 const long long begin = now > tj ? now : tj;
                 const long long R = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
-                A.order[c] = qi; A.uncached[qi] = unc; A.ttft[qi] = R - tj;
-                if (A.completion) A.completion[qi] = R;
                 A.m[slot] = -1;
                 long long h = head;
                 if (slot == head) while (h < A.n && (h == slot || (h < adm_new && __ldcg(A.m + h) < 0))) ++h;
@@ -1116,7 +1113,7 @@ run_kernel(TreeDev T, RunArgs A) {
                 nb.head = h; nb.now = R; nb.admitted = adm_new;
                 nb.evicted = 0;
                 nb.last_valid = unc > 0; nb.last_q = qi; nb.last_m = m; nb.last_len = len;
-                nb.last_leaf = leaf_pred; nb.last_pos = pos; nb.last_leaf_off = leaf_off_pred; nb.last_xm = pre.xm;
+                nb.last_leaf = leaf_pred; nb.last_pos = pos; nb.last_leaf_off = leaf_off_pred; nb.last_xm = ntok;
                 s_bc = nb;
                 // may the scanners start on the next decision while the tree is being updated?
                 long long adm_next, now_next;
@@ -1128,6 +1125,13 @@ run_kernel(TreeDev T, RunArgs A) {
                     __threadfence();
                     atomicExch(&A.sy->seq, (unsigned long long)(c + 1));
                 }
+                A.order[c] = qi; A.uncached[qi] = unc; A.ttft[qi] = R - tj;
+                if (A.completion) A.completion[qi] = R;
+            }
+            InsertPre pre;
+            pre.xm = __shfl_sync(FULL_MASK, v, 0); pre.pt = __shfl_sync(FULL_MASK, v, 1); pre.ft = __shfl_sync(FULL_MASK, v, 2);
+            pre.k_leaf = __shfl_sync(FULL_MASK, seen, 0); pre.k_low = __shfl_sync(FULL_MASK, seen, 1); pre.k_par = __shfl_sync(FULL_MASK, seen, 2);
+            if (lane == 0) {
                 insert_serial(T0, x, len, m, hint, &s_out, &pre);
                 if (s_out.ok && (s_out.leaf != leaf_pred || (unc > 0 && s_out.leaf_off != leaf_off_pred))) {
                     set_status(&s_st, RT_ERR_LIMIT);           // cannot happen: the prediction repeats the allocation rule
