@@ -111,6 +111,11 @@ rt_status rt_rollback(rt_tree* tree, void* stream);
 /* Wait for `stream` and return the tree's device-side status word (RT_OK or the first error recorded). */
 rt_status rt_sync_status(rt_tree* tree, void* stream);
 
+/* A number that says which device-side check recorded the status word (0 if none did): 101/104 a child entry
+ * that should exist was not found, 102 a bounded wait of the scheduling loop ran out, 103 an internal
+ * prediction did not hold.  A debugging aid; synchronises like rt_stats. */
+rt_status rt_status_detail(rt_tree* tree, int32_t* detail);
+
 /* Free the tree and everything it owns.  Synchronous. */
 rt_status rt_destroy(rt_tree* tree);
 

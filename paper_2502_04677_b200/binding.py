@@ -61,6 +61,8 @@ _lib.rt_checkpoint.restype = _i32
 _lib.rt_checkpoint.argtypes = [_vp, _vp]
 _lib.rt_rollback.restype = _i32
 _lib.rt_rollback.argtypes = [_vp, _vp]
+_lib.rt_status_detail.restype = _i32
+_lib.rt_status_detail.argtypes = [_vp, ctypes.POINTER(_i32)]
 _lib.rt_sync_status.restype = _i32
 _lib.rt_sync_status.argtypes = [_vp, _vp]
 _lib.rt_destroy.restype = _i32
@@ -79,7 +81,7 @@ _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_batch_times"]
+           "rt_sync_status", "rt_status_detail", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_batch_times"]
 
 
 def lib() -> ctypes.CDLL:
@@ -178,6 +180,12 @@ def rt_checkpoint(tree: Tree) -> None:
 
 def rt_rollback(tree: Tree) -> None:
     _check(_lib.rt_rollback(tree.handle, _stream()), "rt_rollback")
+
+
+def rt_status_detail(tree: Tree) -> int:
+    d = ctypes.c_int32()
+    _check(_lib.rt_status_detail(tree.handle, ctypes.byref(d)), "rt_status_detail")
+    return int(d.value)
 
 
 def rt_sync_status(tree: Tree) -> int:

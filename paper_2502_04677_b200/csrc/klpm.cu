@@ -46,7 +46,7 @@ struct TreeState {
     long long lru_cursor;
     long long evictions;
     int status;
-    int pad;
+    int detail;             // which check recorded the status (a debugging aid, see rt_status_detail)
 };
 
 struct TreeDev {
@@ -95,7 +95,9 @@ __device__ __forceinline__ unsigned long long hash_key(unsigned long long k) {
     return (unsigned long long)h;
 }
 
-__device__ __forceinline__ void set_status(TreeState* st, int code) { atomicCAS(&st->status, 0, code); }
+__device__ __forceinline__ void set_status(TreeState* st, int code, int detail = 0) {
+    if (atomicCAS(&st->status, 0, code) == 0) st->detail = detail;
+}
 
 // First index in [0, n) where a and b differ, or n.  Warp-cooperative: every lane gets the result.
 // Lane l reads elements l, l+32, l+64, ... of each chunk: each load instruction of the warp is one
@@ -404,7 +406,7 @@ __device__ int32_t split_node(const TreeDev& T, int32_t v, int32_t o, const Inse
     const long long slot = pre ? table_find_seen(T, par, ft, pre->k_par) : table_find(T, par, ft);
     int64_t chain_end = off + len;
     if (slot >= 0) { T.table[slot].child = u; T.table[slot].span_len = o; chain_end = T.table[slot].chain_end; }
-    else set_status(S, RT_ERR_LIMIT);
+    else set_status(S, RT_ERR_LIMIT, 101);
     T.span_off[v] = off + o; T.span_len[v] = len - o; T.depth_start[v] = ds + o; T.parent[v] = u;
     const long long ls = pre ? table_put_seen(T, u, pt, v, len - o, off + o, chain_end, pre->k_low, -1)
                              : table_put_seen(T, u, pt, v, len - o, off + o, chain_end, 0ULL, (long long)(hash_key(make_key(u, pt)) & T.table_mask));
@@ -843,7 +845,7 @@ __device__ bool run_wait(volatile unsigned long long* p, unsigned long long targ
         int go = 1;
         unsigned long long spins = 0;
         while (*p < target) {
-            if (++spins > KLPM_WAIT_LIMIT) { set_status(st, RT_ERR_LIMIT); *(volatile int32_t*)&bc->abort = 1; go = 0; break; }
+            if (++spins > KLPM_WAIT_LIMIT) { set_status(st, RT_ERR_LIMIT, 102); *(volatile int32_t*)&bc->abort = 1; go = 0; break; }
         }
         __threadfence();
         if (*(volatile int32_t*)&bc->abort) go = 0;
@@ -1134,7 +1136,7 @@ run_kernel(TreeDev T, RunArgs A) {
             if (lane == 0) {
                 insert_serial(T0, x, len, m, hint, &s_out, &pre);
                 if (s_out.ok && (s_out.leaf != leaf_pred || (unc > 0 && s_out.leaf_off != leaf_off_pred))) {
-                    set_status(&s_st, RT_ERR_LIMIT);           // cannot happen: the prediction repeats the allocation rule
+                    set_status(&s_st, RT_ERR_LIMIT, 103);           // cannot happen: the prediction repeats the allocation rule
                     s_out.ok = 0;
                 }
             }
@@ -1235,7 +1237,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                         long long slot = table_find(T, par, T.pool[so]);
                         int64_t chain_end = so + sl;
                         if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = T.table[slot].chain_end; }
-                        else set_status(S, RT_ERR_LIMIT);
+                        else set_status(S, RT_ERR_LIMIT, 104);
                         T.end_node[so + off - 1] = (int32_t)u;
                         T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
                         T.parent[node] = (int32_t)u;
@@ -1660,6 +1662,15 @@ rt_status rt_rollback(rt_tree* tree, void* stream) {
     CK(cudaMemcpyAsync(d.clock_owner, tree->ck_clock_owner, d.max_clock * sizeof(int32_t), k, st));
     CK(cudaMemcpyAsync(d.table, tree->ck_table, cap * sizeof(Entry), k, st));
     CK(cudaMemcpyAsync(d.st, tree->ck_st, sizeof(TreeState), k, st));
+    return RT_OK;
+}
+
+rt_status rt_status_detail(rt_tree* tree, int32_t* detail) {
+    if (!tree || !detail) return RT_ERR_INVALID;
+    CK(cudaStreamSynchronize(tree->last_stream));
+    TreeState st;
+    CK(cudaMemcpy(&st, tree->dev.st, sizeof(st), cudaMemcpyDeviceToHost));
+    *detail = st.detail;
     return RT_OK;
 }
 

@@ -462,3 +462,40 @@ def test_batch_times(K, B):
     K.klpm_batch_times(dev(torch.from_numpy(order)), dev(w.arrivals), dev(torch.from_numpy(comp)), B, tb, cb)
     ot, oc = oracle.batch_times(order, w.arrivals.numpy(), comp, B)
     assert np.array_equal(tb.cpu().numpy(), ot) and np.array_equal(cb.cpu().numpy(), oc)
+
+
+# ------------------------------------------------------------------ queues large enough for the multi-CTA loop
+# (above 4,096 queries klpm_run uses a sequencer CTA plus scanner CTAs and publishes picks early)
+
+@pytest.mark.parametrize("k", [1, 3])
+def test_run_multi_cta_all_waiting(K, k):
+    w = W.medium(scale=1 / 4)
+    assert w.queries.n > 4096
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    got = run_gpu(K, pt, po, qt, qo, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick)
+    want = run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_KLPM, k, start=w.start_tick)
+    assert_same_schedule(got, want)
+
+
+@pytest.mark.parametrize("policy,k", [(2, 4), (1, 1)])
+def test_run_multi_cta_streaming_with_lru(K, policy, k):
+    w = W.streaming(scale=1 / 20)
+    assert w.queries.n > 4096
+    qt, qo = w.queries.materialize()
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    got = run_gpu(K, *e, qt, qo, w.arrivals, policy, k, budget=w.budget_tokens)
+    want = run_oracle(*e, qt, qo, w.arrivals, policy, k, budget=w.budget_tokens)
+    assert_same_schedule(got, want)
+    assert want[4]["evictions"] > 0
+
+
+def test_run_multi_cta_ratio_experiment(K):
+    w = W.prefix_ratio(3000, 3000, scale=2.5)          # 5,000 queries arriving over time, empty tree
+    assert w.queries.n > 4096
+    qt, qo = w.queries.materialize()
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    for policy, k in ((K.POLICY_KLPM, 4), (K.POLICY_LPM, 1)):
+        got = run_gpu(K, *e, qt, qo, w.arrivals, policy, k)
+        want = run_oracle(*e, qt, qo, w.arrivals, policy, k)
+        assert_same_schedule(got, want)
