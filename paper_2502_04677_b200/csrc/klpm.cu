@@ -5,11 +5,15 @@
 //   nodes   : structure of arrays indexed by node id (0 = root): parent, depth_start, span_len, nchild
 //             (int32), span_off, last_access (int64), dead (uint8).  Ids are never reused.
 //   pool    : append-only int32 token pool; node v's edge label is pool[span_off[v] .. +span_len[v]).
-//             A split never moves tokens, so "pool index of the last matched token" identifies a
-//             position in the tree for as long as the tree lives.
+//             Edges are placed so that span_off = depth_start (mod 4): the pool tokens that pair with
+//             query positions 4i..4i+3 are one aligned 128-bit load.  A split never moves tokens, so
+//             "pool index of the last matched token" identifies a position in the tree for as long as
+//             the tree lives, and the pieces of a leaf that was cut stay one contiguous run
+//             (chain_end in the child table, end_node[] per pool token: see walk_chain).
 //   children: one open-addressing hash table for the whole tree keyed by (parent id, first token of the
 //             child's edge).  An entry is one 32-byte sector and carries what a walk needs for the hop
-//             (child id, edge length, edge offset), so a hop costs one dependent sector read.
+//             (child id, edge length, edge offset, end of its contiguous run), so a hop costs one
+//             dependent sector read.
 //   LRU     : last_access holds logical clocks.  Only the node where a processed prompt's cached part
 //             ends and its new leaf are stamped; when a leaf is evicted its stamp is handed to its
 //             parent if newer.  For every leaf this equals the clock of the last processed prompt
@@ -25,7 +29,7 @@
 #include "klpm.h"
 
 #define FULL_MASK 0xffffffffu
-#define KLPM_ABI_VERSION 1
+#define KLPM_ABI_VERSION 2
 
 namespace {
 
@@ -1441,6 +1445,8 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         cudaFree(pend_a); cudaFree(pend_b); cudaFree(pm); cudaFree(pnode); cudaFree(poff); cudaFree(n_out);
         return st;
     }
+    // claim words start idle (an earlier call that ran out of capacity may have left some set)
+    bulk_fill_kernel<<<(unsigned)((t->dev.max_nodes + 255) / 256), 256, 0, s>>>(t->claim, t->dev.max_nodes, 0x7fffffff);
     bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(pend_a, n);
     unsigned count = (unsigned)n;
     cudaError_t e = cudaGetLastError();
