@@ -61,3 +61,17 @@ def test_configs_have_documented_sizes():
     a = W.adversarial()
     assert a.queries.n == 262144 and a.prefill.n == 2_000_000
     assert 2.0e9 < a.queries.total_tokens() < 2.4e9
+
+
+def test_prefix_ratio_queue_shape():
+    w = W.prefix_ratio(1000, 5000)
+    assert w.queries.n == 2000 and w.prefill.n == 0 and w.budget_tokens == 0
+    tok, off = w.queries.materialize()
+    assert bool(((off[1:] - off[:-1]) == 6000).all())
+    heads = {}
+    for i, o in enumerate(off[:-1].tolist()):
+        heads.setdefault(tuple(tok[o:o + 8].tolist()), []).append(i)
+    assert len(heads) == 500 and all(len(v) == 4 for v in heads.values())     # every user prefix exactly 4 times
+    # shuffled: the four replicas of a prefix are not adjacent in general
+    assert any(max(v) - min(v) > 3 for v in heads.values())
+    assert bool((w.arrivals[1:] >= w.arrivals[:-1]).all())
