@@ -840,16 +840,23 @@ struct RunArgs {
 #ifndef KLPM_RUN_SPT
 #define KLPM_RUN_SPT 2            // slots per scanner thread the grid is sized for
 #endif
-#define KLPM_WAIT_LIMIT (1ULL << 25)
+#define KLPM_WAIT_LIMIT_NS 30000000000ULL
 
 // Thread 0 of the CTA polls *p until it reaches target (bounded), then the CTA learns whether to go on.
 __device__ bool run_wait(volatile unsigned long long* p, unsigned long long target, RunBcast* bc, TreeState* st) {
     __shared__ int s_go;
     if (threadIdx.x == 0) {
         int go = 1;
-        unsigned long long spins = 0;
+        unsigned long long spins = 0, t0 = 0;
         while (*p < target) {
-            if (++spins > KLPM_WAIT_LIMIT) { set_status(st, RT_ERR_LIMIT, 102); *(volatile int32_t*)&bc->abort = 1; go = 0; break; }
+            if ((++spins & 4095ULL) == 0) {            // the wait is bounded in time: 30 s on the device's nanosecond timer
+                unsigned long long now;
+                asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+                if (t0 == 0) t0 = now;
+                if (now - t0 > KLPM_WAIT_LIMIT_NS || spins > (1ULL << 40)) {
+                    set_status(st, RT_ERR_LIMIT, 102); *(volatile int32_t*)&bc->abort = 1; go = 0; break;
+                }
+            }
         }
         __threadfence();
         if (*(volatile int32_t*)&bc->abort) go = 0;
