@@ -499,3 +499,31 @@ def test_run_multi_cta_ratio_experiment(K):
         got = run_gpu(K, *e, qt, qo, w.arrivals, policy, k)
         want = run_oracle(*e, qt, qo, w.arrivals, policy, k)
         assert_same_schedule(got, want)
+
+
+def test_match_after_the_loop_has_grown_the_tree(K):
+    """The scheduling loop cuts edges and appends leaves; the batched match (which streams along contiguous
+    pool runs) must see the grown tree exactly as the oracle's tree after the same schedule."""
+    w = W.adversarial(scale=1 / 32)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    n = w.queries.n
+    tree = gpu_tree(K, pt, po, extra_prompts=n, extra_tokens=qt.numel())
+    order = torch.zeros(n, dtype=torch.int32, device="cuda")
+    unc = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ttft = torch.zeros(n, dtype=torch.int64, device="cuda")
+    half = 3 * n // 4                               # schedule the first part of the stream only
+    assert half > 4096                              # large enough for the multi-CTA loop
+    K.klpm_run(tree, dev(qt), dev(qo[:half + 1]), dev(w.arrivals[:half]), K.make_params(K.POLICY_KLPM, 4, 0, 1, w.start_tick),
+               order[:half], unc[:half], ttft[:half])
+    assert K.rt_sync_status(tree) == 0
+    m, node, off = gpu_match(K, tree, qt, qo)
+    ot = oracle_tree(pt, po)
+    oracle.schedule(qt.numpy(), qo[:half + 1].numpy(), w.arrivals[:half].numpy(), oracle.POLICY_KLPM, 4, 0, 1, w.start_tick,
+                    oracle.CACHE_TREE, oracle.TIER_UPDATE, ot)
+    want = ot.match(qt.numpy(), qo.numpy())
+    assert np.array_equal(m, want)
+    lens = (qo[1:] - qo[:-1]).numpy()
+    assert np.array_equal(m[:half], lens[:half])    # what was processed is fully cached
+    st, ost = K.rt_stats(tree), ot.stats()
+    assert (st["n_nodes"], st["tokens"], st["clock"]) == (ost["n_nodes"], ost["tokens"], ost["clock"])
