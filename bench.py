@@ -327,11 +327,47 @@ def run_ours(args):
                    "ttft_max": int(ttft_cpu.max()), "ticks_per_sec": w.ticks_per_sec,
                    "tree_tokens_after": stats1["tokens"]},
     }
+    if args.sweep:
+        out["k_sweep"] = k_sweep(K, tree, q_tok, q_off, arr, w, [int(x) for x in args.sweep.split(",")], device)
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(name, args.scale, k, budget_s=args.cpu_seconds)
     print(json.dumps(out), flush=True)
     if multi:
         dist.destroy_process_group()
+
+
+def k_sweep(K, tree, q_tok, q_off, arr, w, ks, device):
+    """Back-testing k: the same stream scheduled for several k at once, each on a clone of the tree and its own
+    CUDA stream (the loop is latency-bound and leaves most SMs idle, so independent loops overlap)."""
+    nq = w.queries.n
+    K.rt_rollback(tree)
+    res = {}
+    for mode in ("one_after_the_other", "concurrent"):
+        trees = [K.rt_clone(tree) for _ in ks]
+        streams = [torch.cuda.Stream(device=device) for _ in ks]
+        outs = [(torch.zeros(nq, dtype=torch.int32, device=device), torch.zeros(nq, dtype=torch.int32, device=device),
+                 torch.zeros(nq, dtype=torch.int64, device=device)) for _ in ks]
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        main = torch.cuda.current_stream()
+        a.record(main)
+        for k, t, st, o in zip(ks, trees, streams, outs):
+            if mode == "concurrent":
+                st.wait_stream(main)
+                with torch.cuda.stream(st):
+                    K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
+                main.wait_stream(st)
+            else:
+                K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
+        b.record(main)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b)
+        bad = [K.rt_sync_status(t) for t in trees]
+        for t in trees:
+            K.rt_destroy(t)
+        res[mode] = {"ms": ms, "decisions_per_sec": len(ks) * nq / (ms / 1e3), "status": bad}
+    res["ks"] = ks
+    return res
 
 
 def cpu_sample(name: str, scale: float, max_tokens: float = 3.0e8):
@@ -440,6 +476,8 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--k", type=int, default=0, help="k of k-LPM (0 = the configuration's own)")
     ap.add_argument("--policy", default="klpm", choices=["klpm", "fcfs", "lpm"])
+    ap.add_argument("--sweep", default="", help="comma-separated k values scheduled concurrently on clones of the tree "
+                                                "(adds a k_sweep object to the line)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     args = ap.parse_args()

@@ -100,6 +100,12 @@ rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const i
 rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* clock,
                    int64_t* evictions, int64_t* pool_used);
 
+/* A second, independent tree with the same capacity and the same content (device-to-device copies enqueued on
+ * `stream`; the allocation itself is synchronous).  Several clones can be scheduled at the same time on
+ * different streams, e.g. to try several values of k on one stream of queries (the back-testing the paper
+ * suggests for choosing k, Section 4.2). */
+rt_status rt_clone(rt_tree* tree, void* stream, rt_tree** out);
+
 /* Remember the tree as it is now (device-to-device copies of the node arrays, the child table and the
  * counters; the token pool is append-only and is not copied).  One checkpoint per tree; a later call replaces it. */
 rt_status rt_checkpoint(rt_tree* tree, void* stream);

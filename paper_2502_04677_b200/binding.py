@@ -57,6 +57,8 @@ _lib.rt_match_batch.restype = _i32
 _lib.rt_match_batch.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.rt_stats.restype = _i32
 _lib.rt_stats.argtypes = [_vp] + [ctypes.POINTER(_i64)] * 5
+_lib.rt_clone.restype = _i32
+_lib.rt_clone.argtypes = [_vp, _vp, ctypes.POINTER(_vp)]
 _lib.rt_checkpoint.restype = _i32
 _lib.rt_checkpoint.argtypes = [_vp, _vp]
 _lib.rt_rollback.restype = _i32
@@ -81,7 +83,7 @@ _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_status_detail", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_batch_times"]
+           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_batch_times"]
 
 
 def lib() -> ctypes.CDLL:
@@ -172,6 +174,12 @@ def rt_stats(tree: Tree) -> dict:
     v = [ctypes.c_int64() for _ in range(5)]
     _check(_lib.rt_stats(tree.handle, *[ctypes.byref(x) for x in v]), "rt_stats")
     return dict(n_nodes=v[0].value, tokens=v[1].value, clock=v[2].value, evictions=v[3].value, pool_used=v[4].value)
+
+
+def rt_clone(tree: Tree) -> Tree:
+    h = ctypes.c_void_p()
+    _check(_lib.rt_clone(tree.handle, _stream(), ctypes.byref(h)), "rt_clone")
+    return Tree(h)
 
 
 def rt_checkpoint(tree: Tree) -> None:

@@ -1626,6 +1626,41 @@ rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* 
     return RT_OK;
 }
 
+rt_status rt_clone(rt_tree* tree, void* stream, rt_tree** out) {
+    if (!tree || !out) return RT_ERR_INVALID;
+    rt_tree* c = nullptr;
+    rt_status s = rt_create(&tree->cfg, &c);
+    if (s) return s;
+    const TreeDev& a = tree->dev;
+    TreeDev& b = c->dev;
+    const unsigned long long cap = a.table_mask + 1;
+    cudaStream_t st = (cudaStream_t)stream;
+    tree->last_stream = st;
+    c->last_stream = st;
+    const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
+    cudaError_t e = cudaMemcpyAsync(b.parent, a.parent, a.max_nodes * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.depth_start, a.depth_start, a.max_nodes * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.span_len, a.span_len, a.max_nodes * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.nchild, a.nchild, a.max_nodes * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.first_tok, a.first_tok, a.max_nodes * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.span_off, a.span_off, a.max_nodes * sizeof(int64_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.last_access, a.last_access, a.max_nodes * sizeof(int64_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.dead, a.dead, a.max_nodes, k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.clock_owner, a.clock_owner, a.max_clock * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.table, a.table, cap * sizeof(Entry), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.pool, a.pool, a.max_pool * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.end_node, a.end_node, a.max_pool * sizeof(int32_t), k, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.st, a.st, sizeof(TreeState), k, st);
+    if (e != cudaSuccess) {
+        fprintf(stderr, "klpm: rt_clone failed: %s\n", cudaGetErrorString(e));
+        cudaStreamSynchronize(st);
+        free_tree(c);
+        return RT_ERR_CUDA;
+    }
+    *out = c;
+    return RT_OK;
+}
+
 rt_status rt_checkpoint(rt_tree* tree, void* stream) {
     if (!tree) return RT_ERR_INVALID;
     TreeDev& d = tree->dev;

@@ -527,3 +527,36 @@ def test_match_after_the_loop_has_grown_the_tree(K):
     assert np.array_equal(m[:half], lens[:half])    # what was processed is fully cached
     st, ost = K.rt_stats(tree), ot.stats()
     assert (st["n_nodes"], st["tokens"], st["clock"]) == (ost["n_nodes"], ost["tokens"], ost["clock"])
+
+
+def test_concurrent_k_sweep_on_clones(K):
+    """Back-testing k: one stream of queries scheduled with k = 1, 2, 4, 8 at the same time, each on its own
+    clone of the tree and its own CUDA stream.  Every run must equal the oracle's run for that k."""
+    w = W.medium(scale=1 / 4)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    n = w.queries.n
+    base = gpu_tree(K, pt, po, extra_prompts=n, extra_tokens=qt.numel())
+    d_qt, d_qo, d_arr = dev(qt), dev(qo), dev(w.arrivals)
+    ks = [1, 2, 4, 8]
+    trees = [K.rt_clone(base) for _ in ks]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in ks]
+    outs = []
+    for k, tree, st in zip(ks, trees, streams):
+        with torch.cuda.stream(st):
+            order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+            unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+            ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+            comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+            K.klpm_run(tree, d_qt, d_qo, d_arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), order, unc, ttft, comp)
+            outs.append((order, unc, ttft, comp))
+    torch.cuda.synchronize()
+    for k, tree, (order, unc, ttft, comp) in zip(ks, trees, outs):
+        assert K.rt_sync_status(tree) == 0
+        got = (order.cpu().numpy(), unc.cpu().numpy(), ttft.cpu().numpy(), comp.cpu().numpy(), K.rt_stats(tree))
+        want = run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_KLPM, k, start=w.start_tick)
+        assert_same_schedule(got, want)
+    # the tree the clones were taken from is untouched
+    m, _, _ = gpu_match(K, base, qt, qo)
+    assert np.array_equal(m, oracle_tree(pt, po).match(qt.numpy(), qo.numpy()))
