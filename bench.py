@@ -356,9 +356,11 @@ def k_sweep(K, tree, q_tok, q_off, arr, w, ks, device):
                 st.wait_stream(main)
                 with torch.cuda.stream(st):
                     K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
-                main.wait_stream(st)
             else:
                 K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
+        if mode == "concurrent":
+            for st in streams:
+                main.wait_stream(st)
         b.record(main)
         torch.cuda.synchronize()
         ms = a.elapsed_time(b)
