@@ -60,6 +60,8 @@ def lib():
         L.oc_replay.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, i64, i64, i32, vp, vp, vp]
         L.oc_batch_times.restype = None
         L.oc_batch_times.argtypes = [vp, i32, vp, vp, i32, vp, vp]
+        L.oc_schedule_ex.restype = i32
+        L.oc_schedule_ex.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i64, i32, i32, vp, i32, vp, vp, vp, vp]
         L.oc_schedule.restype = i32
         L.oc_schedule.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i64, i32, i32, vp, vp, vp, vp]
         _lib = L
@@ -130,8 +132,11 @@ class OracleTree:
 
 def schedule(tokens, offsets, arrivals, policy: int, k: int = 1, c_num: int = 0, c_den: int = 1,
              start_tick: int = 0, cache_mode: int = CACHE_TREE, tier: int = TIER_UPDATE,
-             tree: Optional[OracleTree] = None) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
-    """Run FCFS / LPM / k-LPM over the stream.  Returns order, uncached, ttft, completion."""
+             tree: Optional[OracleTree] = None, tie_priority=None, score_mode: int = 0
+             ) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Run FCFS / LPM / k-LPM over the stream.  Returns order, uncached, ttft, completion.
+    tie_priority (optional int64 per query): smaller wins among equal scores of a longest-match pick.
+    score_mode 1: the score is the hit rate floor(match * 2^31 / length) instead of the match length."""
     t, o, a = _i32(tokens), _i64(offsets), _i64(arrivals)
     n = len(o) - 1
     if cache_mode == CACHE_TREE and tree is None:
@@ -140,8 +145,10 @@ def schedule(tokens, offsets, arrivals, policy: int, k: int = 1, c_num: int = 0,
     unc = np.zeros(n, dtype=np.int32)
     ttft = np.zeros(n, dtype=np.int64)
     comp = np.zeros(n, dtype=np.int64)
-    rc = lib().oc_schedule(tree._h if tree is not None else None, _p(t), _p(o), _p(a), n, policy, max(1, int(k)),
-                           c_num, c_den, start_tick, cache_mode, tier, _p(order), _p(unc), _p(ttft), _p(comp))
+    pr = None if tie_priority is None else _i64(tie_priority)
+    rc = lib().oc_schedule_ex(tree._h if tree is not None else None, _p(t), _p(o), _p(a), n, policy, max(1, int(k)),
+                              c_num, c_den, start_tick, cache_mode, tier, _p(pr), int(score_mode),
+                              _p(order), _p(unc), _p(ttft), _p(comp))
     if rc:
         raise RuntimeError("oracle: schedule failed (%d)" % rc)
     return order, unc, ttft, comp

@@ -91,7 +91,8 @@ class StringSetCache:
 def schedule(prompts: Sequence[Sequence[int]], arrivals: Sequence[int], policy: int, k: int = 1,
              c_num: int = 0, c_den: int = 1, start_tick: int = 0, cache_mode: int = TREE,
              prefill: Sequence[Sequence[int]] = (), budget: int = 0,
-             cache: Optional[StringSetCache] = None):
+             cache: Optional[StringSetCache] = None, tie_priority: Optional[Sequence[int]] = None,
+             score_mode: int = 0):
     """Algorithm 1 / FCFS / LPM with the cost model of Definition 2.
     Returns (order, uncached, ttft, completion); the last three are indexed by query."""
     n = len(prompts)
@@ -120,7 +121,12 @@ def schedule(prompts: Sequence[Sequence[int]], arrivals: Sequence[int], policy: 
         if policy == FCFS or (policy == KLPM and c % k == 0):
             j = min(waiting, key=lambda i: (arrivals[i], i))
         else:
-            j = min(waiting, key=lambda i: (-match(prompts[i]), arrivals[i], i))
+            def score(i):
+                mi = match(prompts[i])
+                if score_mode == 1:
+                    return (mi << 31) // len(prompts[i]) if len(prompts[i]) else 0
+                return mi
+            j = min(waiting, key=lambda i: (-score(i), tie_priority[i] if tie_priority is not None else 0, arrivals[i], i))
         x = prompts[j]
         if cache_mode == LAST_ONLY:
             u = len(x) - match(x)

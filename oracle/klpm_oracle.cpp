@@ -298,10 +298,16 @@ void oc_batch_times(const int32_t* order, int32_t n_order, const int64_t* arriva
 
 // Algorithm 1 (k-LPM) with its FCFS and LPM limits, run over the whole stream.
 // order[c] = index processed at decision c; uncached/ttft/completion are indexed by query.
-int32_t oc_schedule(void* tp, const tok_t* tok, const int64_t* off, const int64_t* arrival, int32_t n,
-                    int32_t policy, int32_t k, int64_t c_num, int64_t c_den, int64_t start_tick,
-                    int32_t cache_mode, int32_t tier,
-                    int32_t* order, int32_t* uncached, int64_t* ttft, int64_t* completion) {
+// Variants of the longest-match pick (both leave the oldest-first picks alone):
+//   tie_priority (nullable): among queries with the same score the one with the smallest priority wins, before
+//     arrival and index decide.  With priorities drawn at random this is the uniform tie-breaking the paper
+//     assumes for LPM (footnote to Theorem 2); the numbers are an input, nothing is drawn here.
+//   score_mode 0: score = match length (tokens).  score_mode 1: score = hit rate of the prompt, quantised to
+//     floor(match * 2^31 / |x|) (0 for an empty prompt) -- the other reading of "prefix cache hit rate".
+int32_t oc_schedule_ex(void* tp, const tok_t* tok, const int64_t* off, const int64_t* arrival, int32_t n,
+                       int32_t policy, int32_t k, int64_t c_num, int64_t c_den, int64_t start_tick,
+                       int32_t cache_mode, int32_t tier, const int64_t* tie_priority, int32_t score_mode,
+                       int32_t* order, int32_t* uncached, int64_t* ttft, int64_t* completion) {
     Stream s{tok, off, arrival, n};
     Tree* t = (Tree*)tp;
     std::vector<char> processed(n, 0), waiting(n, 0);
@@ -337,12 +343,19 @@ int32_t oc_schedule(void* tp, const tok_t* tok, const int64_t* off, const int64_
             for (int32_t i = 0; i < n; ++i)
                 if (waiting[i] && (j < 0 || earlier(s, i, j))) j = i;
         } else {
-            int32_t best = -1;
+            int64_t best = -1;
             for (int32_t i = 0; i < n; ++i) {
                 if (!waiting[i]) continue;
                 int32_t mi = tier == TIER_UPDATE ? m[i] : match_now(i);
                 if (tier != TIER_UPDATE) m[i] = mi;
-                if (j < 0 || mi > best || (mi == best && earlier(s, i, j))) { j = i; best = mi; }
+                int64_t score = mi;
+                if (score_mode == 1) score = s.len(i) > 0 ? ((int64_t)mi << 31) / s.len(i) : 0;
+                bool wins = j < 0 || score > best;
+                if (!wins && score == best) {
+                    if (tie_priority && tie_priority[i] != tie_priority[j]) wins = tie_priority[i] < tie_priority[j];
+                    else wins = earlier(s, i, j);
+                }
+                if (wins) { j = i; best = score; }
             }
         }
 
@@ -382,6 +395,15 @@ int32_t oc_schedule(void* tp, const tok_t* tok, const int64_t* off, const int64_
         }
     }
     return 0;
+}
+
+// Algorithm 1 as printed: match length as the score, ties to the earliest arrival.
+int32_t oc_schedule(void* tp, const tok_t* tok, const int64_t* off, const int64_t* arrival, int32_t n,
+                    int32_t policy, int32_t k, int64_t c_num, int64_t c_den, int64_t start_tick,
+                    int32_t cache_mode, int32_t tier,
+                    int32_t* order, int32_t* uncached, int64_t* ttft, int64_t* completion) {
+    return oc_schedule_ex(tp, tok, off, arrival, n, policy, k, c_num, c_den, start_tick, cache_mode, tier, nullptr, 0,
+                          order, uncached, ttft, completion);
 }
 
 }  // extern "C"

@@ -335,3 +335,72 @@ def test_batch_times_by_hand_and_limits():
     assert oracle.batch_times(order, arr, comp, 9)[1].tolist() == [30] * 4            # one bin: everyone waits for the last
     ttft, cb = oracle.batch_times(order, [0, 5, 1, 2], comp, 3)                       # ragged last bin, arrivals subtracted
     assert cb.tolist() == [25, 25, 25, 30] and ttft.tolist() == [25, 20, 24, 28]
+
+
+# ---------------------------------------------------------------- tie priorities and the hit-rate score
+
+def run_ex(prompts, arrivals, policy, k=1, prio=None, score_mode=0, tier=oracle.TIER_UPDATE, start=0, budget=0):
+    t, o = csr(prompts)
+    tree = oracle.OracleTree(budget)
+    out = oracle.schedule(t, o, arrivals, policy, k, 0, 1, start, oracle.CACHE_TREE, tier, tree, prio, score_mode)
+    return [v.tolist() for v in out]
+
+
+def test_tie_priorities_by_hand_on_the_toy_queue():
+    """Toy queue, burst: every first pick is a tie.  With priorities that favour x3, then x4: LPM processes
+    x3, x1 (same user as x3), x4, x2 and the completions are 10, 15, 25, 30 in that order."""
+    prompts, arr = W.regular_arrival_shuffled_queue(4, 2, 5, 5, 0, [1, 2, 3, 4])
+    order, unc, ttft, comp = run_ex(prompts, arr, oracle.POLICY_LPM, prio=[3, 2, 0, 1])
+    assert order == [2, 0, 3, 1] and ttft == [15, 30, 10, 25] and unc == [5, 5, 10, 10]
+    # priorities that repeat the arrival order change nothing
+    base = run_ex(prompts, arr, oracle.POLICY_LPM)
+    assert run_ex(prompts, arr, oracle.POLICY_LPM, prio=[0, 1, 2, 3]) == base
+    # k-LPM: the oldest-first picks ignore the priorities
+    order, _, _, _ = run_ex(prompts, arr, oracle.POLICY_KLPM, k=2, prio=[3, 2, 0, 1])
+    assert order == [0, 2, 1, 3]
+
+
+@pytest.mark.parametrize("n,rep,u,d,s", [(12, 4, 6, 1, 2), (8, 2, 3, 3, 1)])
+def test_lpm_closed_form_holds_for_random_ties(n, rep, u, d, s):
+    """The j-th completion under LPM is T + ceil(j/rep) u + j d whatever breaks the ties (proof of Theorem 2)."""
+    rng = np.random.RandomState(n)
+    for _ in range(6):
+        sigma = (rng.permutation(n) + 1).tolist()
+        prompts, arr = W.regular_arrival_shuffled_queue(n, rep, u, d, s, sigma)
+        prio = rng.permutation(n).tolist()
+        T = s * n
+        order, unc, ttft, comp = run_ex(prompts, arr, oracle.POLICY_LPM, prio=prio, start=T)
+        for pos, j in enumerate(order, start=1):
+            assert comp[j] == T + math.ceil(pos / rep) * u + d * pos
+        # first pick of every group of `rep` is the waiting query with the smallest priority among the ties
+        assert order[0] == min(range(n), key=lambda i: prio[i])
+
+
+def test_hit_rate_score_by_hand_and_on_constant_lengths():
+    """Cache holds "ab".  By match length "abX" and "abYZWQ" tie at 2 and beat "a"; by hit rate "a" is fully
+    cached (1), then "abX" (2/3), then "abYZWQ" (1/3)."""
+    cached = [[1, 2]]
+    qs = [[1, 2, 7, 8, 9, 10], [1, 2, 5], [1]]
+    t, o = csr(qs)
+    for mode, want in ((0, [0, 1, 2]), (1, [2, 1, 0])):
+        tree = oracle.OracleTree()
+        tree.insert(*csr(cached))
+        order = oracle.schedule(t, o, [0, 0, 0], oracle.POLICY_LPM, 1, 0, 1, 0, oracle.CACHE_TREE, oracle.TIER_REMATCH, tree,
+                                None, mode)[0].tolist()
+        assert order == want
+    # all prompts of a regular arrival queue have the same length: both scores order them alike
+    prompts, arr = W.regular_arrival_shuffled_queue(12, 3, 5, 2, 1, [5, 1, 9, 3, 12, 7, 2, 11, 4, 8, 6, 10])
+    assert run_ex(prompts, arr, oracle.POLICY_KLPM, k=3, score_mode=1) == run_ex(prompts, arr, oracle.POLICY_KLPM, k=3)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_variants_agree_with_the_definition_level_model(seed):
+    prompts, arr = W.random_small_queue(seed + 900, 26, vocab=2, max_len=11, min_len=0, max_gap=3)
+    prio = W.uniform_int(seed, 77, len(prompts), 0, 5).tolist()          # few distinct values: ties among priorities too
+    for policy, k in ((oracle.POLICY_LPM, 1), (oracle.POLICY_KLPM, 3)):
+        for mode in (0, 1):
+            for budget in (0, 40):
+                ref = D.schedule(prompts, arr, policy, k, budget=budget, tie_priority=prio, score_mode=mode)
+                for tier in (oracle.TIER_REMATCH, oracle.TIER_UPDATE):
+                    got = run_ex(prompts, arr, policy, k, prio, mode, tier, budget=budget)
+                    assert got == [list(v) for v in ref]
