@@ -193,6 +193,19 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
                    const int64_t* d_arrival, int32_t n, const klpm_params* params, int32_t* d_order,
                    int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
 
+/* klpm_run with two variants of the longest-match pick (the oldest-first picks are not affected):
+ *   d_tie_priority (nullable, int64[n]): among waiting queries with the same score the one with the smallest
+ *     priority wins; arrival and index decide only among equal priorities.  With priorities drawn uniformly at
+ *     random by the caller this is the tie-breaking the paper assumes for LPM (footnote in Section 4.2).
+ *   score_mode 0: the score is the match length in tokens (Algorithm 1 as klpm_run reads it).
+ *   score_mode 1: the score is the prompt's hit rate, quantised to floor(match * 2^31 / length) (0 for an empty
+ *     prompt) -- the other reading of "maximizes the prefix cache hit rate".
+ * klpm_run(...) is klpm_run_ex(..., NULL, 0, ...). */
+rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
+                      const int64_t* d_arrival, int32_t n, const klpm_params* params,
+                      const int64_t* d_tie_priority, int32_t score_mode, int32_t* d_order,
+                      int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
+
 /* Batch size B (Section 2.1: the order is cut into consecutive bins of B queries, and a query is finished when
  * the last query of its bin is).  d_order (int32[n_order]) is a processing order and d_completion (int64, indexed
  * by query) its batch-size-one completion times, as klpm_run / klpm_replay produce them; d_completion_b and

@@ -77,13 +77,15 @@ _lib.klpm_select_noalloc.restype = _i32
 _lib.klpm_select_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(klpm_params), _vp, _vp]
 _lib.klpm_replay.restype = _i32
 _lib.klpm_replay.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp]
+_lib.klpm_run_ex.restype = _i32
+_lib.klpm_run_ex.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.klpm_batch_times.restype = _i32
 _lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp]
 _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_batch_times"]
+           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_batch_times"]
 
 
 def lib() -> ctypes.CDLL:
@@ -256,3 +258,15 @@ def klpm_batch_times(order: torch.Tensor, arrival: torch.Tensor, completion: tor
                                  _dev(completion, torch.int64, "completion"), int(batch_size),
                                  _dev(ttft_b, torch.int64, "ttft_b"), _dev(completion_b, torch.int64, "completion_b"),
                                  _stream()), "klpm_batch_times")
+
+
+def klpm_run_ex(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arrival: torch.Tensor, params: klpm_params,
+                tie_priority: Optional[torch.Tensor], score_mode: int, order: torch.Tensor, uncached: torch.Tensor,
+                ttft: torch.Tensor, completion: Optional[torch.Tensor] = None) -> None:
+    n = arrival.numel()
+    _check(_lib.klpm_run_ex(tree.handle, _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
+                            _dev(arrival, torch.int64, "arrival"), n, ctypes.byref(params),
+                            _dev(tie_priority, torch.int64, "tie_priority", True), int(score_mode),
+                            _dev(order, torch.int32, "order"), _dev(uncached, torch.int32, "uncached"),
+                            _dev(ttft, torch.int64, "ttft"), _dev(completion, torch.int64, "completion", True), _stream()),
+           "klpm_run_ex")

@@ -830,6 +830,9 @@ struct RunArgs {
     int32_t* hint;         // slot -> node at or below the node where the match ends
     long long* pos;        // slot -> pool index of the last matched token (-1 = root)
     int32_t* ntok;         // slot -> the query token right after its match (meaningful while m < length)
+    const int32_t* prank;  // slot -> rank of the slot by (tie priority, slot); null = ties go to the lower slot
+    const int32_t* pinv;   // that rank -> slot
+    int32_t score_mode;    // 0: score = match length; 1: score = floor(match * 2^31 / length)
     unsigned long long* partial;   // per CTA best key
     RunBcast* bc;
     RunSync* sy;
@@ -975,7 +978,13 @@ __device__ unsigned long long run_scan(const TreeDev& T, const RunArgs& A, const
             }
             if (waiting) {
                 if (dirty) { A.m[r] = m; A.pos[r] = pos; A.ntok[r] = ntok; if (hint >= 0) A.hint[r] = hint; }
-                const unsigned long long key = ((unsigned long long)(unsigned)m << 32) | (unsigned)(0xffffffffu - (unsigned)r);
+                unsigned hi = (unsigned)m;
+                if (A.score_mode == 1) {
+                    const int32_t ql = __ldg(A.slen + r);
+                    hi = ql > 0 ? (unsigned)(((unsigned long long)(unsigned)m << 31) / (unsigned)ql) : 0u;
+                }
+                const unsigned lo = A.prank ? (unsigned)__ldg(A.prank + r) : (unsigned)r;
+                const unsigned long long key = ((unsigned long long)hi << 32) | (0xffffffffu - lo);
                 if (key > best) best = key;
             }
         }
@@ -1074,7 +1083,11 @@ run_kernel(TreeDev T, RunArgs A) {
         // ---- pick (warp 0; lane 0 decides), charge by Definition 2
         if (warp == 0) {
             const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
-            const long long slot = fcfs_turn ? head : (long long)(0xffffffffu - (unsigned)(b & 0xffffffffu));
+            long long slot = head;
+            if (!fcfs_turn) {
+                const unsigned rk = 0xffffffffu - (unsigned)(b & 0xffffffffu);
+                slot = A.pinv ? (long long)__ldg(A.pinv + rk) : (long long)rk;
+            }
             const int32_t qi = __ldg(A.ord + slot);
             const int32_t m = __ldcg(A.m + slot);
             const int32_t hint = __ldcg(A.hint + slot);
@@ -1343,6 +1356,17 @@ __global__ void slot_arrays_kernel(const int32_t* __restrict__ ord, const int64_
     soff[r] = lo;
     slen[r] = (int32_t)(off[qi + 1] - lo);
 }
+__global__ void prio_init_kernel(const int64_t* __restrict__ prio, const int32_t* __restrict__ ord, int32_t n, long long np2,
+                                 long long* key, int32_t* idx) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= np2) return;
+    key[i] = i < n ? prio[ord[i]] : 0x7fffffffffffffffLL;      // slot i holds query ord[i]
+    idx[i] = i < n ? (int32_t)i : 0x7fffffff;
+}
+__global__ void prio_rank_kernel(const int32_t* __restrict__ pinv, int32_t n, int32_t* prank) {
+    int32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < n) prank[pinv[r]] = r;
+}
 __global__ void bitonic_step_kernel(long long* key, int32_t* idx, long long np2, long long k, long long j) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= np2) return;
@@ -1371,6 +1395,7 @@ struct rt_tree {
     long long run_cap;      // slots allocated (power of two)
     long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos;
     long long* run_soff; int32_t* run_slen; int32_t* run_ntok;
+    long long* run_pkey; int32_t* run_pinv; int32_t* run_prank;
     unsigned long long* run_partial; RunBcast* run_bc; RunSync* run_sy;
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -1403,6 +1428,7 @@ void free_tree(rt_tree* t) {
     cudaFree(d.table); cudaFree(d.pool); cudaFree(d.end_node); cudaFree(d.st); cudaFree(t->match_counter);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
     cudaFree(t->run_pos); cudaFree(t->run_soff); cudaFree(t->run_slen); cudaFree(t->run_ntok);
+    cudaFree(t->run_pkey); cudaFree(t->run_pinv); cudaFree(t->run_prank);
     cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
     cudaFree(t->claim);
     cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
@@ -1417,7 +1443,8 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     if (np2 <= t->run_cap) return RT_OK;
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
     cudaFree(t->run_pos); cudaFree(t->run_soff); cudaFree(t->run_slen); cudaFree(t->run_ntok);
-    t->run_ntok = nullptr;
+    cudaFree(t->run_pkey); cudaFree(t->run_pinv); cudaFree(t->run_prank);
+    t->run_ntok = nullptr; t->run_pkey = nullptr; t->run_pinv = nullptr; t->run_prank = nullptr;
     t->run_key = nullptr; t->run_ord = nullptr; t->run_m = nullptr; t->run_hint = nullptr; t->run_pos = nullptr;
     t->run_soff = nullptr; t->run_slen = nullptr;
     t->run_cap = 0;
@@ -1430,6 +1457,9 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->run_soff, np2))) return s;
     if ((s = dalloc(&t->run_slen, np2))) return s;
     if ((s = dalloc(&t->run_ntok, np2))) return s;
+    if ((s = dalloc(&t->run_pkey, np2))) return s;
+    if ((s = dalloc(&t->run_pinv, np2))) return s;
+    if ((s = dalloc(&t->run_prank, np2))) return s;
     t->run_cap = np2;
     return RT_OK;
 }
@@ -1838,10 +1868,10 @@ rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_
     return RT_OK;
 }
 
-rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
-                   int32_t n, const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
-                   int64_t* d_completion, void* stream) {
-    if (!tree || !params_ok(params) || n < 0 ||
+rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
+                      int32_t n, const klpm_params* params, const int64_t* d_tie_priority, int32_t score_mode,
+                      int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream) {
+    if (!tree || !params_ok(params) || n < 0 || score_mode < 0 || score_mode > 1 ||
         (n > 0 && (!d_q_tokens || !d_q_offsets || !d_arrival || !d_order || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
     if (n == 0) return RT_OK;
     cudaStream_t s = (cudaStream_t)stream;
@@ -1858,6 +1888,13 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
             for (long long j = k >> 1; j > 0; j >>= 1)
                 bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_key, tree->run_ord, np2, k, j);
         slot_arrays_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, d_q_offsets, n, tree->run_soff, tree->run_slen);
+        if (d_tie_priority) {        // rank of every slot by (priority, slot)
+            prio_init_kernel<<<blocks, 256, 0, s>>>(d_tie_priority, tree->run_ord, n, np2, tree->run_pkey, tree->run_pinv);
+            for (long long k = 2; k <= np2; k <<= 1)
+                for (long long j = k >> 1; j > 0; j >>= 1)
+                    bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_pkey, tree->run_pinv, np2, k, j);
+            prio_rank_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_pinv, n, tree->run_prank);
+        }
         CK(cudaGetLastError());
     }
     RunBcast bc0;
@@ -1871,6 +1908,8 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
     a.policy = params->policy; a.k = params->k; a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
     a.order = d_order; a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
     a.soff = tree->run_soff; a.slen = tree->run_slen; a.ntok = tree->run_ntok;
+    a.prank = d_tie_priority ? tree->run_prank : nullptr; a.pinv = d_tie_priority ? tree->run_pinv : nullptr;
+    a.score_mode = score_mode;
     a.ord = tree->run_ord; a.sorted_t = tree->run_key; a.m = tree->run_m; a.hint = tree->run_hint; a.pos = tree->run_pos;
     a.partial = tree->run_partial; a.bc = tree->run_bc; a.sy = tree->run_sy;
     const int threads = KLPM_RUN_THREADS;
@@ -1884,6 +1923,13 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
     void* kargs[] = {(void*)&tree->dev, (void*)&a};
     CK(cudaLaunchCooperativeKernel((void*)run_kernel, dim3((unsigned)blocks), dim3(threads), kargs, 0, s));
     return RT_OK;
+}
+
+rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
+                   int32_t n, const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                   int64_t* d_completion, void* stream) {
+    return klpm_run_ex(tree, d_q_tokens, d_q_offsets, d_arrival, n, params, nullptr, 0, d_order, d_uncached, d_ttft,
+                       d_completion, stream);
 }
 
 }  // extern "C"

@@ -560,3 +560,65 @@ def test_concurrent_k_sweep_on_clones(K):
     # the tree the clones were taken from is untouched
     m, _, _ = gpu_match(K, base, qt, qo)
     assert np.array_equal(m, oracle_tree(pt, po).match(qt.numpy(), qo.numpy()))
+
+
+# ------------------------------------------------------------------ tie priorities and the hit-rate score
+
+def run_gpu_ex(K, pt, po, qt, qo, arr, policy, k, prio, score_mode, budget=0, start=0):
+    n = qo.numel() - 1
+    tree = gpu_tree(K, pt, po, extra_prompts=n, extra_tokens=qt.numel(), budget=budget)
+    order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    d_prio = None if prio is None else dev(torch.as_tensor(prio, dtype=torch.int64))
+    K.klpm_run_ex(tree, dev(qt), dev(qo), dev(torch.as_tensor(arr, dtype=torch.int64)), K.make_params(policy, k, 0, 1, start),
+                  d_prio, score_mode, order, unc, ttft, comp)
+    assert K.rt_sync_status(tree) == 0
+    st = K.rt_stats(tree)
+    K.rt_destroy(tree)
+    return order.cpu().numpy(), unc.cpu().numpy(), ttft.cpu().numpy(), comp.cpu().numpy(), st
+
+
+def run_oracle_ex(pt, po, qt, qo, arr, policy, k, prio, score_mode, budget=0, start=0, tier=oracle.TIER_UPDATE):
+    ot = oracle_tree(pt, po, budget)
+    out = oracle.schedule(qt.numpy(), qo.numpy(), np.asarray(arr, dtype=np.int64), policy, k, 0, 1, start,
+                          oracle.CACHE_TREE, tier, ot, prio, score_mode)
+    return out + (ot.stats(),)
+
+
+def test_run_ex_toy_queue_with_priorities(K):
+    prompts, arr = W.regular_arrival_shuffled_queue(4, 2, 5, 5, 0, [1, 2, 3, 4])
+    qt, qo = csr(prompts)
+    e = torch.zeros(0, dtype=torch.int32), torch.zeros(1, dtype=torch.int64)
+    order, unc, ttft, comp, _ = run_gpu_ex(K, *e, qt, qo, arr, K.POLICY_LPM, 1, [3, 2, 0, 1], 0)
+    assert order.tolist() == [2, 0, 3, 1] and ttft.tolist() == [15, 30, 10, 25]
+
+
+@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("score_mode", [0, 1])
+def test_run_ex_fuzz(K, seed, score_mode):
+    prompts, arr = W.random_small_queue(seed + 1200, 150, vocab=2, max_len=14, min_len=0, max_gap=4)
+    prefill, _ = W.random_small_queue(seed + 1300, 10, vocab=2, max_len=10, min_len=1)
+    prio = W.uniform_int(seed, 78, len(prompts), 0, 9).tolist()
+    qt, qo = csr(prompts)
+    pt, po = csr(prefill)
+    for policy, k in ((1, 1), (2, 3)):
+        for budget in (0, 48):
+            for p in (prio, None):
+                got = run_gpu_ex(K, pt, po, qt, qo, arr, policy, k, p, score_mode, budget=budget)
+                want = run_oracle_ex(pt, po, qt, qo, arr, policy, k, p, score_mode, budget=budget, tier=oracle.TIER_REMATCH)
+                assert_same_schedule(got, want)
+
+
+@pytest.mark.parametrize("score_mode", [0, 1])
+def test_run_ex_multi_cta_random_ties(K, score_mode):
+    """Uniformly random tie priorities (the paper's assumption for LPM) on a queue large enough for the multi-CTA loop."""
+    w = W.medium(scale=1 / 4)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    prio = W.uniform_u53(11, 79, w.queries.n).tolist()
+    got = run_gpu_ex(K, pt, po, qt, qo, w.arrivals, K.POLICY_LPM, 1, prio, score_mode, start=w.start_tick)
+    want = run_oracle_ex(pt, po, qt, qo, w.arrivals, oracle.POLICY_LPM, 1, prio, score_mode, start=w.start_tick)
+    assert_same_schedule(got, want)
+    assert not np.array_equal(got[0], run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_LPM, 1, start=w.start_tick)[0])
