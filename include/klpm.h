@@ -188,10 +188,20 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
  * that have arrived (match lengths are those against the tree at that moment, which includes every
  * query processed so far); charge the pick by Definition 2; store it in the tree (LRU eviction under
  * the budget).  d_order[c] (int32[n]) = query processed at decision c; the other outputs are as in
- * klpm_replay.  The pick counter of KLPM never resets. */
+ * klpm_replay.  The pick counter of KLPM never resets.
+ * On a tree without a budget nothing is ever evicted, so a query's match length changes only when a prompt is
+ * processed whose own match ended at the same place and goes on with the same token; the loop then keeps every
+ * query's match state itself and stores all processed prompts in the tree at the end, concurrently (as rt_insert
+ * does for large batches) -- same outputs, same cached prefixes and node boundaries.  In that case the call waits
+ * for `stream` (the concurrent insertion does between its rounds). */
 rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
                    const int64_t* d_arrival, int32_t n, const klpm_params* params, int32_t* d_order,
                    int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
+
+/* Which loop the last klpm_run / klpm_run_ex on this tree took: 0 = none yet, 1 = one decision at a time on the
+ * tree itself (trees with a budget; also a tree without one whose capacity might not hold the whole queue),
+ * 2 = the grouped loop (trees without a budget; see klpm_run).  Both give the same outputs. */
+int32_t klpm_run_path(const rt_tree* tree);
 
 /* klpm_run with two variants of the longest-match pick (the oldest-first picks are not affected):
  *   d_tie_priority (nullable, int64[n]): among waiting queries with the same score the one with the smallest

@@ -81,11 +81,13 @@ _lib.klpm_run_ex.restype = _i32
 _lib.klpm_run_ex.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.klpm_batch_times.restype = _i32
 _lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp]
+_lib.klpm_run_path.restype = _i32
+_lib.klpm_run_path.argtypes = [_vp]
 _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_batch_times"]
+           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times"]
 
 
 def lib() -> ctypes.CDLL:
@@ -250,6 +252,14 @@ def klpm_run(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arriva
                          _dev(arrival, torch.int64, "arrival"), n, ctypes.byref(params), _dev(order, torch.int32, "order"),
                          _dev(uncached, torch.int32, "uncached"), _dev(ttft, torch.int64, "ttft"),
                          _dev(completion, torch.int64, "completion", True), _stream()), "klpm_run")
+
+
+RUN_PATH_NONE, RUN_PATH_ONE_BY_ONE, RUN_PATH_GROUPED = 0, 1, 2
+
+
+def klpm_run_path(tree: Tree) -> int:
+    """Which loop the last klpm_run / klpm_run_ex on this tree took (RUN_PATH_*)."""
+    return int(_lib.klpm_run_path(tree.handle))
 
 
 def klpm_batch_times(order: torch.Tensor, arrival: torch.Tensor, completion: torch.Tensor, batch_size: int,

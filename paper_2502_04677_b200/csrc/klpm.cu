@@ -23,6 +23,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 #include <new>
 
@@ -288,10 +289,13 @@ __device__ __noinline__ int32_t node_after(const EndIndex X, int64_t pos, int64_
 }
 
 // Returns the match length; *node / *off (where the match ended) are filled when want_node is set.
+// With WANT_POS, *last_pos receives the pool index of the last matched token (-1 if nothing matched).
+template <bool WANT_POS = false>
 __device__ __forceinline__ int32_t walk_chain(const TreeDev& T, const int32_t* __restrict__ q, int32_t len, bool want_node,
-                              int32_t* node, int32_t* off) {
+                              int32_t* node, int32_t* off, int64_t* last_pos = nullptr) {
     const int lane = threadIdx.x & 31;
     *node = 0; *off = 0;
+    if (WANT_POS) *last_pos = -1;
     if (len <= 0) return 0;
     QWin Q;
     Q.s = (int32_t)((reinterpret_cast<uintptr_t>(q) >> 2) & 3);
@@ -314,6 +318,7 @@ __device__ __forceinline__ int32_t walk_chain(const TreeDev& T, const int32_t* _
         const int32_t x = compare_run(Q, T.pool + (c.span_off - (int64_t)m), m, m + (int32_t)run, lane);
         const int64_t pos = c.span_off + (x - m) - 1;          // x > m: the first token is the key
         m = x;
+        if (WANT_POS) *last_pos = pos;
         const int32_t e = node_ending_at(end_index(T), pos, *reinterpret_cast<const volatile long long*>(&T.st->n_nodes));
         if (e < 0) {                                           // stopped inside an edge
             if (want_node) {
@@ -1198,6 +1203,507 @@ run_kernel(TreeDev T, RunArgs A) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// klpm_run on a tree without a budget: the grouped loop.
+//
+// Without eviction the match length of a query only ever grows, and it grows exactly when a prompt is
+// processed whose own match ended at the same tree position and continues with the same token
+// (otherwise the processed prompt shares no more with the query than the tree already did).  So the loop
+// needs no tree at all:
+//   * every query -- arrived or not -- is matched once against the tree as it stands (one warp per query,
+//     streaming along contiguous pool runs), which gives its match length m, the position `pos` where the
+//     match ends (pool index of the last matched token) and the query token `ntok` that follows;
+//   * queries with the same (pos, ntok) form a group, held as a contiguous run of a member array
+//     (a bitonic sort by a 62-bit hash of the pair puts equal pairs side by side; a hash collision only
+//     puts two groups into one run, and members are checked against (pos, ntok) before they are touched);
+//   * when a prompt is processed its group is dissolved: every member is compared with the prompt's
+//     uncached tokens, gets its new m, a position inside the prompt's new leaf and its next token, and the
+//     members are regrouped by their new pairs inside the run they already occupy (they never need more
+//     room: the processed query leaves).  A query in a group of one costs nothing.  Leaves created by the
+//     loop get positions from a counter that starts above every real pool index;
+//   * the longest-match pick is the root of a tournament over the keys (score << 32 | ~rank) of the
+//     arrived queries: 32-ary, leaves in global memory, every level above in shared memory;
+//   * the oldest-first pick is a cursor over a bitmap of processed slots.
+// One CTA runs the whole loop: warp 0 is the sequencer, the other warps wait at a named barrier and join
+// for work that is worth sharing (a large group, a large batch of arrivals).  There is no wait on another
+// CTA anywhere.  The processed prompts are stored in the tree afterwards, all at once, by the concurrent
+// bulk insertion: the set of node boundaries does not depend on the order of insertion.
+// ------------------------------------------------------------------------------------------------
+struct alignas(32) FDyn {     // what the loop changes, one 32-byte sector per slot
+    long long pos;            // pool index (real or virtual) of the last matched token, -1 at the root
+    int32_t m;                // match length; -1 once processed
+    int32_t ntok;             // query token right after the match (meaningful while m < length)
+    int32_t gstart, gcount;   // the slot's group: run [gstart, gstart + gcount) of the member array
+    long long pad;
+};
+struct alignas(32) FStat {    // constant during the loop
+    long long soff;           // offset of the query's first token
+    long long t;              // arrival
+    int32_t len;
+    int32_t ord;              // query index
+    int32_t rank;             // low key bits: rank by (tie priority, slot), or the slot itself
+    int32_t pad;
+};
+
+struct FastArgs {
+    const int32_t* tok;
+    int32_t n;
+    int32_t policy, k, score_mode;
+    long long c_num, c_den, start_tick;
+    int32_t* order; int32_t* uncached; int64_t* ttft; int64_t* completion;
+    FDyn* dyn; FStat* stat;
+    unsigned long long* key;      // slot -> key it has (or will have once arrived); 0 once processed
+    int32_t* mem;                 // member array
+    const int32_t* pinv;          // rank -> slot, or null
+    long long* gh; int32_t* gidx; // group hashes and slots (sorted before the loop; scratch for large groups inside it)
+    unsigned int* done;           // bitmap of processed slots (used when it does not fit in shared memory)
+    long long vbase;              // first virtual pool index
+    int32_t lb_shift;             // log2 of the number of slots per tournament leaf block
+    int32_t nb;                   // number of leaf blocks
+    int32_t done_in_smem;
+    unsigned long long* counter;  // [0] work counter of the initial walk, [1] sum of the tokens it found uncached
+    TreeState* st;
+};
+
+#define KLPM_FAST_THREADS 512
+#define KLPM_FAST_SORT_CAP 4096          // largest group that is regrouped exactly (sorted in shared memory)
+#define KLPM_FAST_NOGROUP 0xffffffffffffffffULL
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {      // SplitMix64's finaliser
+    z ^= z >> 30; z *= 0xbf58476d1ce4e5b9ULL; z ^= z >> 27; z *= 0x94d049bb133111ebULL; z ^= z >> 31;
+    return z;
+}
+__device__ __forceinline__ unsigned long long group_hash(long long pos, int32_t ntok) {
+    return mix64((unsigned long long)(pos + 2) * 0x9E3779B97F4A7C15ULL + (unsigned)ntok) >> 2;
+}
+__device__ __forceinline__ unsigned long long single_hash(int32_t slot) {       // a query that is fully cached never regroups
+    return mix64(0xD1B54A32D192ED03ULL ^ (unsigned long long)(unsigned)slot) >> 2;
+}
+__device__ __forceinline__ unsigned long long fast_key(int32_t m, int32_t len, int32_t rank, int32_t score_mode) {
+    unsigned hi = (unsigned)m;
+    if (score_mode == 1) hi = len > 0 ? (unsigned)(((unsigned long long)(unsigned)m << 31) / (unsigned)len) : 0u;
+    return ((unsigned long long)hi << 32) | (0xffffffffu - (unsigned)rank);
+}
+__device__ __forceinline__ FDyn ld_dyn(const FDyn* p) {
+    const int4* q = reinterpret_cast<const int4*>(p);
+    const int4 a = __ldcg(q), b = __ldcg(q + 1);
+    FDyn d;
+    d.pos = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+    d.m = a.z; d.ntok = a.w; d.gstart = b.x; d.gcount = b.y; d.pad = 0;
+    return d;
+}
+__device__ __forceinline__ void st_dyn_state(FDyn* p, long long pos, int32_t m, int32_t ntok) {
+    __stcg(reinterpret_cast<int4*>(p), make_int4((int)(unsigned)(unsigned long long)pos, (int)(unsigned)((unsigned long long)pos >> 32), m, ntok));
+}
+__device__ __forceinline__ void st_dyn_group(FDyn* p, int32_t gstart, int32_t gcount) {
+    __stcg(reinterpret_cast<int2*>(p) + 2, make_int2(gstart, gcount));
+}
+__device__ __forceinline__ FStat ld_stat(const FStat* p) {
+    const int4* q = reinterpret_cast<const int4*>(p);
+    const int4 a = __ldg(q), b = __ldg(q + 1);
+    FStat s;
+    s.soff = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+    s.t = (long long)(((unsigned long long)(unsigned)a.w << 32) | (unsigned)a.z);
+    s.len = b.x; s.ord = b.y; s.rank = b.z; s.pad = 0;
+    return s;
+}
+__device__ __forceinline__ void named_bar(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// slot -> constant record (after the slots have been ordered by arrival)
+__global__ void fast_stat_kernel(const int32_t* __restrict__ ord, const long long* __restrict__ sorted_t,
+                                 const int64_t* __restrict__ off, const int32_t* __restrict__ prank, int32_t n, FStat* stat) {
+    const int32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    const int32_t qi = ord[r];
+    const int64_t lo = off[qi];
+    FStat s;
+    s.soff = lo; s.t = sorted_t[r]; s.len = (int32_t)(off[qi + 1] - lo); s.ord = qi; s.rank = prank ? prank[r] : r; s.pad = 0;
+    stat[r] = s;
+}
+
+// The one match of every query against the tree: one warp per slot, slots handed out by a counter.
+__global__ void __launch_bounds__(256)
+fast_walk_kernel(TreeDev T, FastArgs A, long long np2) {
+    const int lane = threadIdx.x & 31;
+    for (;;) {
+        unsigned long long i = 0;
+        if (lane == 0) i = atomicAdd(A.counter, 1ULL);
+        i = __shfl_sync(FULL_MASK, i, 0);
+        if (i >= (unsigned long long)np2) return;
+        const int32_t r = (int32_t)i;
+        if (r >= A.n) {                                   // padding of the sort
+            if (lane == 0) { A.gh[r] = 0x7fffffffffffffffLL; A.gidx[r] = 0x7fffffff; }
+            continue;
+        }
+        const FStat s = ld_stat(A.stat + r);
+        int32_t len = s.len;
+        if (len < 0) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
+        const int32_t* q = A.tok + s.soff;
+        int32_t node, off;
+        int64_t pos;
+        const int32_t m = walk_chain<true>(T, q, len, false, &node, &off, &pos);
+        if (lane == 0) {
+            const int32_t ntok = m < len ? __ldg(q + m) : 0;
+            atomicAdd(A.counter + 1, (unsigned long long)(len - m));      // an upper bound of what the queue will append
+            st_dyn_state(A.dyn + r, pos, m, ntok);
+            A.key[r] = fast_key(m, len, s.rank, A.score_mode);
+            A.gh[r] = (long long)(m < len ? group_hash(pos, ntok) : single_hash(r));
+            A.gidx[r] = r;
+        }
+    }
+}
+
+// after the sort by hash: runs of equal hashes are the groups
+__global__ void fast_group_kernel(FastArgs A) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= A.n) return;
+    const long long h = A.gh[i];
+    int32_t lo = 0, hi = i;                    // first index with gh >= h
+    while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (A.gh[mid] < h) lo = mid + 1; else hi = mid; }
+    const int32_t first = lo;
+    lo = i + 1; hi = A.n;                      // first index with gh > h
+    while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (A.gh[mid] <= h) lo = mid + 1; else hi = mid; }
+    const int32_t r = A.gidx[i];
+    A.mem[i] = r;
+    st_dyn_group(A.dyn + r, first, lo - first);
+}
+
+// ---- the tournament above the leaf blocks (shared memory) ----
+struct FastTour {
+    unsigned long long* t1;   // per leaf block (padded with zeros to a multiple of 32)
+    unsigned long long* t2;   // per 32 leaf blocks (padded likewise)
+    unsigned long long* t3;   // 32 entries
+    int32_t n2;               // entries of t2 in use
+    int32_t n3;               // entries of t3 in use
+};
+// Recompute the ancestors of leaf block b; returns the root.  One warp.
+__device__ __forceinline__ unsigned long long tour_update(const FastTour& R, int32_t b, int lane) {
+    const int32_t i2 = b >> 5;
+    unsigned long long v = warp_max64(R.t1[(i2 << 5) + lane]);
+    if (lane == 0) R.t2[i2] = v;
+    __syncwarp();
+    const int32_t i3 = i2 >> 5;
+    v = warp_max64(R.t2[(i3 << 5) + lane]);
+    if (lane == 0) R.t3[i3] = v;
+    __syncwarp();
+    return warp_max64(R.t3[lane]);
+}
+// Recompute t3 and the root from t2.  One warp.
+__device__ __forceinline__ unsigned long long tour_top(const FastTour& R, int lane) {
+    for (int32_t i3 = 0; i3 < R.n3; ++i3) {
+        const unsigned long long v = warp_max64(R.t2[(i3 << 5) + lane]);
+        if (lane == 0) R.t3[i3] = v;
+    }
+    __syncwarp();
+    return warp_max64(R.t3[lane]);
+}
+// Recompute t2 from t1.  Every warp of the CTA; the caller synchronises.
+__device__ __forceinline__ void tour_mid(const FastTour& R, int warp, int nwarps, int lane) {
+    for (int32_t i2 = warp; i2 < R.n2; i2 += nwarps) {
+        const unsigned long long v = warp_max64(R.t1[(i2 << 5) + lane]);
+        if (lane == 0) R.t2[i2] = v;
+    }
+}
+
+struct FastPick {             // the prompt being processed, as its group's members need it
+    int32_t slot, m, len, ntok;
+    const int32_t* x;         // its tokens
+    long long pos;
+    long long vleaf;          // virtual pool index of the first token of its new leaf
+    long long admitted;       // slots below this have arrived
+    int32_t gstart, gcount;
+};
+struct FastJob { int32_t type; int32_t a0, a1; FastPick pick; };
+enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2 };
+
+// One member of the dissolving group per lane (r < 0: none).  Members tied with the processed prompt are
+// compared with its uncached tokens and get their new state and key; every live member gets the hash of the
+// group it belongs to from now on (KLPM_FAST_NOGROUP: it leaves the run).  *touched: its key grew and it
+// has arrived, so its leaf block's ancestors need recomputing.  Warp-cooperative.
+__device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, const FastPick& P, const FastTour& R, int32_t r, int lane,
+                                                          bool* touched) {
+    const bool act = r >= 0 && r != P.slot;
+    FDyn d; d.pos = 0; d.m = -1; d.ntok = 0; d.gstart = 0; d.gcount = 0;
+    FStat s; s.soff = 0; s.t = 0; s.len = 0; s.ord = 0; s.rank = 0;
+    if (act) { d = ld_dyn(A.dyn + r); s = ld_stat(A.stat + r); }
+    const bool live = act && d.m >= 0;
+    const bool tied = live && d.pos == P.pos && d.ntok == P.ntok && d.m == P.m && d.m < s.len;
+    const int32_t* q = A.tok + s.soff;
+    int32_t e = 0;
+    unsigned cm = __ballot_sync(FULL_MASK, tied);
+    while (cm) {
+        const int src = __ffs(cm) - 1; cm &= cm - 1;
+        const int32_t* qq = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)q, src);
+        const int32_t ql = __shfl_sync(FULL_MASK, s.len, src);
+        const int32_t lim = (ql < P.len ? ql : P.len) - P.m;
+        const int32_t ee = first_mismatch<true>(qq + P.m, P.x + P.m, lim);
+        if (lane == src) e = ee;
+    }
+    *touched = false;
+    if (tied) {
+        d.m = P.m + e; d.pos = P.vleaf + e - 1; d.ntok = d.m < s.len ? __ldg(q + d.m) : 0;
+        st_dyn_state(A.dyn + r, d.pos, d.m, d.ntok);
+        const unsigned long long key = fast_key(d.m, s.len, s.rank, A.score_mode);
+        __stcg(A.key + r, key);
+        if ((long long)r < P.admitted) { atomicMax(R.t1 + (r >> A.lb_shift), key); *touched = true; }
+    }
+    if (!live) return KLPM_FAST_NOGROUP;
+    return d.m < s.len ? group_hash(d.pos, d.ntok) : single_hash(r);
+}
+
+// Work the whole CTA shares; every thread calls it with the same job.  Ends with t2 recomputed from t1.
+__device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J, unsigned long long* sh, int32_t* sr, int* s_cnt) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    if (J.type == FAST_JOB_ADMIT) {
+        // slots [a0, a1) have arrived: fold their keys into their leaf blocks
+        const int32_t b0 = J.a0 >> A.lb_shift, b1 = (J.a1 - 1) >> A.lb_shift;
+        const int32_t LB = 1 << A.lb_shift;
+        for (int32_t b = b0 + warp; b <= b1; b += nwarps) {
+            unsigned long long v = 0;
+            for (int32_t u = lane; u < LB; u += 32) {
+                const long long r = ((long long)b << A.lb_shift) + u;
+                if (r >= J.a0 && r < J.a1) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
+            }
+            v = warp_max64(v);
+            if (lane == 0 && v > R.t1[b]) R.t1[b] = v;
+        }
+    } else {
+        // dissolve a group of more than 32 members
+        const FastPick& P = J.pick;
+        const int32_t gs = P.gstart, gc = P.gcount;
+        const bool exact = gc <= KLPM_FAST_SORT_CAP;
+        int32_t p2 = 1;
+        while (p2 < gc) p2 <<= 1;
+        for (int32_t base = warp * 32; base < gc; base += nwarps * 32) {
+            const int32_t i = base + lane;
+            const int32_t r = i < gc ? __ldcg(A.mem + gs + i) : -1;
+            bool touched;
+            const unsigned long long h = fast_member(A, P, R, r, lane, &touched);
+            if (i < gc) {
+                if (exact) { sh[i] = h; sr[i] = r; }
+                else { __stcg(A.gh + i, (long long)h); __stcg(A.gidx + i, r); }
+            }
+        }
+        if (exact) for (int32_t i = gc + tid; i < p2; i += nthr) { sh[i] = KLPM_FAST_NOGROUP; sr[i] = -1; }
+        if (tid == 0) *s_cnt = 0;
+        __syncthreads();
+        if (exact) {
+            // regroup exactly: sort the members by the hash of their new group inside the run
+            for (int32_t k = 2; k <= p2; k <<= 1)
+                for (int32_t j = k >> 1; j > 0; j >>= 1) {
+                    for (int32_t i = tid; i < p2; i += nthr) {
+                        const int32_t l = i ^ j;
+                        if (l > i) {
+                            const unsigned long long a = sh[i], b = sh[l];
+                            if ((a > b) == ((i & k) == 0)) { sh[i] = b; sh[l] = a; const int32_t t = sr[i]; sr[i] = sr[l]; sr[l] = t; }
+                        }
+                    }
+                    __syncthreads();
+                }
+            for (int32_t i = tid; i < gc; i += nthr) {
+                const unsigned long long h = sh[i];
+                if (h == KLPM_FAST_NOGROUP) continue;
+                int32_t lo = 0, hi = i;
+                while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sh[mid] < h) lo = mid + 1; else hi = mid; }
+                const int32_t first = lo;
+                lo = i + 1; hi = gc;
+                while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sh[mid] <= h) lo = mid + 1; else hi = mid; }
+                const int32_t r = sr[i];
+                __stcg(A.mem + gs + i, r);
+                st_dyn_group(A.dyn + r, gs + first, lo - first);
+            }
+        } else {
+            // too large to sort here: the live members stay together as one run (a superset of every group in it)
+            for (int32_t i = tid; i < gc; i += nthr)
+                if ((unsigned long long)__ldcg(A.gh + i) != KLPM_FAST_NOGROUP) {
+                    const int32_t p = atomicAdd(s_cnt, 1);
+                    __stcg(A.mem + gs + p, __ldcg(A.gidx + i));
+                }
+            __syncthreads();
+            const int32_t cnt = *s_cnt;
+            for (int32_t i = tid; i < gc; i += nthr)
+                if ((unsigned long long)__ldcg(A.gh + i) != KLPM_FAST_NOGROUP) st_dyn_group(A.dyn + __ldcg(A.gidx + i), gs, cnt);
+        }
+    }
+    __syncthreads();
+    tour_mid(R, warp, nwarps, lane);
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(KLPM_FAST_THREADS, 1)
+fast_run_kernel(FastArgs A) {
+    extern __shared__ __align__(16) unsigned char fast_smem[];
+    __shared__ FastJob s_job;
+    __shared__ int s_cnt;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t n = A.n;
+    const int32_t nb1p = (A.nb + 31) & ~31, n2 = nb1p >> 5, n2p = (n2 + 31) & ~31, n3 = n2p >> 5;
+    const int32_t nwords = (n + 31) >> 5;
+    FastTour R;
+    R.t1 = reinterpret_cast<unsigned long long*>(fast_smem);
+    R.t2 = R.t1 + nb1p;
+    R.t3 = R.t2 + n2p;
+    R.n2 = n2; R.n3 = n3;
+    unsigned long long* sh = R.t3 + 32;
+    int32_t* sr = reinterpret_cast<int32_t*>(sh + KLPM_FAST_SORT_CAP);
+    unsigned int* s_done = reinterpret_cast<unsigned int*>(sr + KLPM_FAST_SORT_CAP);
+    for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
+    if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
+    __syncthreads();
+
+    if (warp != 0) {
+        for (;;) {
+            named_bar(1, KLPM_FAST_THREADS);
+            const FastJob J = s_job;
+            if (J.type == FAST_JOB_EXIT) return;
+            fast_job(A, R, J, sh, sr, &s_cnt);
+        }
+    }
+
+    // ---------------------------------------------------------------- the sequencer (warp 0)
+    const long long INF = 0x7fffffffffffffffLL;
+    long long now = A.start_tick, vnext = A.vbase;
+    int32_t head = 0, admitted = 0;
+    long long next_t = __ldg(&A.stat[0].t);
+    unsigned long long root = 0;
+    for (int32_t c = 0; c < n; ++c) {
+        // ---- time and arrivals: idle until somebody has arrived, then admit everybody who has
+        if (head == admitted && next_t > now) now = next_t;
+        if (next_t <= now) {
+            int32_t a1 = admitted;
+            {
+                const long long r = (long long)a1 + lane;
+                const bool in = r < n && __ldg(&A.stat[r].t) <= now;
+                const unsigned bal = __ballot_sync(FULL_MASK, in);
+                const int cnt = bal == FULL_MASK ? 32 : __ffs(~bal) - 1;
+                a1 += cnt;
+                if (cnt == 32 && a1 < n) {                 // a full window: gallop, then bisect (lane 0)
+                    long long lo = a1, hi = n;
+                    if (lane == 0 && __ldg(&A.stat[lo].t) <= now) {
+                        long long step = 1;
+                        ++lo;
+                        while (lo + step <= hi && __ldg(&A.stat[lo + step - 1].t) <= now) { lo += step; step <<= 1; }
+                        if (lo + step < hi) hi = lo + step;
+                        while (lo < hi) { const long long mid = (lo + hi) >> 1; if (__ldg(&A.stat[mid].t) <= now) lo = mid + 1; else hi = mid; }
+                    }
+                    a1 = (int32_t)__shfl_sync(FULL_MASK, lo, 0);
+                }
+            }
+            if (a1 - admitted <= 32) {
+                const int32_t r = admitted + lane;
+                if (r < a1) atomicMax(R.t1 + (r >> A.lb_shift), __ldcg(A.key + r));
+                __syncwarp();
+                root = tour_update(R, admitted >> A.lb_shift, lane);
+                if (((a1 - 1) >> A.lb_shift) != (admitted >> A.lb_shift)) root = tour_update(R, (a1 - 1) >> A.lb_shift, lane);
+            } else {
+                if (lane == 0) { s_job.type = FAST_JOB_ADMIT; s_job.a0 = admitted; s_job.a1 = a1; }
+                __syncwarp();
+                named_bar(1, KLPM_FAST_THREADS);
+                const FastJob J = s_job;
+                fast_job(A, R, J, sh, sr, &s_cnt);
+                root = tour_top(R, lane);
+            }
+            admitted = a1;
+            next_t = admitted < n ? __ldg(&A.stat[admitted].t) : INF;
+        }
+        // ---- pick
+        const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
+        int32_t slot = head;
+        if (!fcfs_turn) {
+            const unsigned rk = 0xffffffffu - (unsigned)(root & 0xffffffffULL);
+            slot = A.pinv ? __ldg(A.pinv + rk) : (int32_t)rk;
+        }
+        if (slot < 0 || slot >= admitted) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 105); break; }   // cannot happen
+        const FDyn d = ld_dyn(A.dyn + slot);
+        const FStat s = ld_stat(A.stat + slot);
+        const int32_t b = slot >> A.lb_shift;
+        unsigned long long bm = 0;                          // the pick's leaf block without the pick
+        for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
+            const long long r = ((long long)b << A.lb_shift) + u;
+            if (r < admitted && r != slot) { const unsigned long long kk = __ldcg(A.key + r); if (kk > bm) bm = kk; }
+        }
+        bm = warp_max64(bm);
+        // ---- charge (Definition 2)
+        const int32_t m = d.m, len = s.len, unc = len - m;
+        if (m < 0) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 106); break; }                           // cannot happen
+        const long long begin = now > s.t ? now : s.t;
+        const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
+        now = Rj;
+        if (lane == 0) {
+            A.order[c] = s.ord; A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
+            if (A.completion) A.completion[s.ord] = Rj;
+            st_dyn_state(A.dyn + slot, d.pos, -1, d.ntok);
+            __stcg(A.key + slot, 0ULL);
+            if (A.done_in_smem) s_done[slot >> 5] |= 1u << (slot & 31);
+            else __stcg(A.done + (slot >> 5), __ldcg(A.done + (slot >> 5)) | (1u << (slot & 31)));
+            R.t1[b] = bm;
+        }
+        __syncwarp();
+        const long long vleaf = vnext;
+        vnext += unc;
+        // ---- the queries tied with the pick now match into its new leaf
+        bool full = false;
+        if (unc > 0 && d.gcount > 1) {
+            FastPick P;
+            P.slot = slot; P.m = m; P.len = len; P.ntok = d.ntok; P.x = A.tok + s.soff; P.pos = d.pos; P.vleaf = vleaf;
+            P.admitted = admitted; P.gstart = d.gstart; P.gcount = d.gcount;
+            if (d.gcount <= 32) {
+                const int32_t r = lane < d.gcount ? __ldcg(A.mem + d.gstart + lane) : -1;
+                bool touched;
+                const unsigned long long h = fast_member(A, P, R, r, lane, &touched);
+                int32_t rank = 0, start = 0, cnt = 0;       // regroup inside the run
+                for (int k2 = 0; k2 < 32; ++k2) {
+                    const unsigned long long hk = __shfl_sync(FULL_MASK, h, k2);
+                    const bool lt = hk < h, eq = hk == h;
+                    start += lt; cnt += eq; rank += (lt || (eq && k2 < lane));
+                }
+                if (h != KLPM_FAST_NOGROUP) { __stcg(A.mem + d.gstart + rank, r); st_dyn_group(A.dyn + r, d.gstart + start, cnt); }
+                __syncwarp();
+                unsigned tm = __ballot_sync(FULL_MASK, touched);
+                while (tm) {
+                    const int src = __ffs(tm) - 1; tm &= tm - 1;
+                    const int32_t bb = __shfl_sync(FULL_MASK, r >> A.lb_shift, src);
+                    if (bb != b) root = tour_update(R, bb, lane);
+                }
+            } else {
+                if (lane == 0) { s_job.type = FAST_JOB_DISSOLVE; s_job.pick = P; }
+                __syncwarp();
+                named_bar(1, KLPM_FAST_THREADS);
+                const FastJob J = s_job;
+                fast_job(A, R, J, sh, sr, &s_cnt);
+                full = true;
+            }
+        }
+        root = full ? tour_top(R, lane) : tour_update(R, b, lane);
+        // ---- the oldest unprocessed slot
+        if (slot == head) {
+            int32_t w0 = head >> 5;
+            for (;;) {
+                const int32_t wi = w0 + lane;
+                unsigned w = 0u;                              // past the end: "unprocessed", so the search stops
+                if (wi < nwords) w = A.done_in_smem ? s_done[wi] : __ldcg(A.done + wi);
+                if (wi == (head >> 5)) w |= (1u << (head & 31)) - 1u;
+                const unsigned bal = __ballot_sync(FULL_MASK, w != 0xffffffffu);
+                if (bal) {
+                    const int src = __ffs(bal) - 1;
+                    const unsigned fw = ~__shfl_sync(FULL_MASK, w, src);
+                    head = (w0 + src) * 32 + __ffs(fw) - 1;
+                    break;
+                }
+                w0 += 32;
+            }
+            if (head > n) head = n;
+        }
+        __syncwarp();
+    }
+    if (lane == 0) s_job.type = FAST_JOB_EXIT;
+    __syncwarp();
+    named_bar(1, KLPM_FAST_THREADS);
+}
+
+// ------------------------------------------------------------------------------------------------
 // bulk insertion of many prompts into a tree without a budget.  The set of node boundaries a radix tree
 // ends up with does not depend on the order in which prompts are stored, so prompts are inserted in
 // rounds: every pending prompt is walked from the root (read-only), then at most one prompt per edge
@@ -1397,6 +1903,11 @@ struct rt_tree {
     long long* run_soff; int32_t* run_slen; int32_t* run_ntok;
     long long* run_pkey; int32_t* run_pinv; int32_t* run_prank;
     unsigned long long* run_partial; RunBcast* run_bc; RunSync* run_sy;
+    // scratch of the grouped loop (trees without a budget)
+    long long fast_cap;     // slots allocated (power of two)
+    FDyn* fast_dyn; FStat* fast_stat; unsigned long long* fast_key_arr; int32_t* fast_mem;
+    long long* fast_gh; int32_t* fast_gidx; unsigned int* fast_done; unsigned long long* fast_counter;
+    int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
     // checkpoint (rt_checkpoint / rt_rollback): copies of everything a later call can modify
@@ -1430,6 +1941,8 @@ void free_tree(rt_tree* t) {
     cudaFree(t->run_pos); cudaFree(t->run_soff); cudaFree(t->run_slen); cudaFree(t->run_ntok);
     cudaFree(t->run_pkey); cudaFree(t->run_pinv); cudaFree(t->run_prank);
     cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
+    cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
+    cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
     cudaFree(t->claim);
     cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
     cudaFree(t->ck_clock_owner); cudaFree(t->ck_span_off); cudaFree(t->ck_last_access); cudaFree(t->ck_dead);
@@ -1461,6 +1974,28 @@ rt_status ensure_run_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->run_pinv, np2))) return s;
     if ((s = dalloc(&t->run_prank, np2))) return s;
     t->run_cap = np2;
+    return RT_OK;
+}
+
+rt_status ensure_fast_scratch(rt_tree* t, long long n) {
+    long long np2 = 1;
+    while (np2 < n) np2 <<= 1;
+    if (np2 <= t->fast_cap) return RT_OK;
+    cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
+    cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
+    t->fast_dyn = nullptr; t->fast_stat = nullptr; t->fast_key_arr = nullptr; t->fast_mem = nullptr;
+    t->fast_gh = nullptr; t->fast_gidx = nullptr; t->fast_done = nullptr; t->fast_counter = nullptr;
+    t->fast_cap = 0;
+    rt_status s;
+    if ((s = dalloc(&t->fast_dyn, np2))) return s;
+    if ((s = dalloc(&t->fast_stat, np2))) return s;
+    if ((s = dalloc(&t->fast_key_arr, np2))) return s;
+    if ((s = dalloc(&t->fast_mem, np2))) return s;
+    if ((s = dalloc(&t->fast_gh, np2))) return s;
+    if ((s = dalloc(&t->fast_gidx, np2))) return s;
+    if ((s = dalloc(&t->fast_done, np2 / 32 + 64))) return s;
+    if ((s = dalloc(&t->fast_counter, 2))) return s;
+    t->fast_cap = np2;
     return RT_OK;
 }
 
@@ -1880,6 +2415,13 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     if (st) return st;
     long long np2 = 1;
     while (np2 < n) np2 <<= 1;
+    // A tree without a budget takes the grouped loop, provided the whole queue is certain to fit (otherwise the
+    // one-by-one loop below stores what fits and reports the rest).  KLPM_RUN_LEGACY=1 forces the older loop.
+    bool grouped = false;
+    if (tree->cfg.budget_tokens == 0) {
+        const char* legacy = getenv("KLPM_RUN_LEGACY");
+        grouped = !(legacy && legacy[0] == '1');
+    }
     // slots = queries ordered by (arrival, index)
     {
         unsigned blocks = (unsigned)((np2 + 255) / 256);
@@ -1896,6 +2438,62 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
             prio_rank_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_pinv, n, tree->run_prank);
         }
         CK(cudaGetLastError());
+    }
+    FastArgs f;
+    memset(&f, 0, sizeof(f));
+    if (grouped) {
+        st = ensure_fast_scratch(tree, n);
+        if (st) return st;
+        f.tok = d_q_tokens; f.n = n; f.policy = params->policy; f.k = params->k; f.score_mode = score_mode;
+        f.c_num = params->c_num; f.c_den = params->c_den; f.start_tick = params->start_tick;
+        f.order = d_order; f.uncached = d_uncached; f.ttft = d_ttft; f.completion = d_completion;
+        f.dyn = tree->fast_dyn; f.stat = tree->fast_stat; f.key = tree->fast_key_arr; f.mem = tree->fast_mem;
+        f.pinv = d_tie_priority ? tree->run_pinv : nullptr;
+        f.gh = tree->fast_gh; f.gidx = tree->fast_gidx; f.done = tree->fast_done; f.counter = tree->fast_counter;
+        f.vbase = tree->dev.max_pool + 16;
+        f.st = tree->dev.st;
+        // every query is matched once against the tree as it stands
+        fast_stat_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, tree->run_key, d_q_offsets,
+                                                                     d_tie_priority ? tree->run_prank : nullptr, n, f.stat);
+        CK(cudaMemsetAsync(f.counter, 0, 2 * sizeof(unsigned long long), s));
+        long long wblocks = (np2 + 7) / 8;
+        if (wblocks > (long long)tree->num_sms * 8) wblocks = (long long)tree->num_sms * 8;
+        fast_walk_kernel<<<(unsigned)wblocks, 256, 0, s>>>(tree->dev, f, np2);
+        CK(cudaGetLastError());
+        // does everything the queue can append fit?  (an upper bound: what the tree does not hold now)
+        TreeState h;
+        unsigned long long unc_bound = 0;
+        CK(cudaMemcpyAsync(&h, tree->dev.st, sizeof(h), cudaMemcpyDeviceToHost, s));
+        CK(cudaMemcpyAsync(&unc_bound, f.counter + 1, sizeof(unc_bound), cudaMemcpyDeviceToHost, s));
+        CK(cudaStreamSynchronize(s));
+        grouped = h.status == 0 && h.n_nodes + 2LL * n <= tree->dev.max_nodes &&
+                  h.pool_used + (long long)unc_bound + 6LL * n <= tree->dev.max_pool &&
+                  h.clock + (long long)n + 1 < tree->dev.max_clock;
+    }
+    if (grouped) {
+        int lbs = 5;
+        while ((((long long)n + (1LL << lbs) - 1) >> lbs) > 8192) ++lbs;
+        f.lb_shift = lbs;
+        f.nb = (int32_t)(((long long)n + (1LL << lbs) - 1) >> lbs);
+        const long long nb1p = (f.nb + 31) & ~31, n2p = ((nb1p >> 5) + 31) & ~31;
+        const long long nwords = ((long long)n + 31) >> 5;
+        size_t smem = (size_t)(nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
+        f.done_in_smem = smem + (size_t)nwords * 4 <= 200 * 1024 ? 1 : 0;
+        if (f.done_in_smem) smem += (size_t)nwords * 4;
+        const unsigned nblk = (unsigned)((n + 255) / 256), pblk = (unsigned)((np2 + 255) / 256);
+        CK(cudaMemsetAsync(f.done, 0, (size_t)(np2 / 32 + 64) * sizeof(unsigned int), s));
+        // groups: queries whose match ends at the same position and continues with the same token
+        for (long long k = 2; k <= np2; k <<= 1)
+            for (long long j = k >> 1; j > 0; j >>= 1)
+                bitonic_step_kernel<<<pblk, 256, 0, s>>>(f.gh, f.gidx, np2, k, j);
+        fast_group_kernel<<<nblk, 256, 0, s>>>(f);
+        CK(cudaGetLastError());
+        CK(cudaFuncSetAttribute(fast_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        fast_run_kernel<<<1, KLPM_FAST_THREADS, smem, s>>>(f);
+        CK(cudaGetLastError());
+        tree->run_path = 2;
+        // the processed prompts enter the tree together (the logical clock advances by n)
+        return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s);
     }
     RunBcast bc0;
     memset(&bc0, 0, sizeof(bc0));
@@ -1922,8 +2520,11 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     if (blocks > tree->num_sms) blocks = tree->num_sms;
     void* kargs[] = {(void*)&tree->dev, (void*)&a};
     CK(cudaLaunchCooperativeKernel((void*)run_kernel, dim3((unsigned)blocks), dim3(threads), kargs, 0, s));
+    tree->run_path = 1;
     return RT_OK;
 }
+
+int32_t klpm_run_path(const rt_tree* tree) { return tree ? tree->run_path : 0; }
 
 rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
                    int32_t n, const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,

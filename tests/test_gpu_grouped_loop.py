@@ -1,0 +1,169 @@
+"""The grouped scheduling loop (trees without a budget) against the oracle and against the one-by-one loop.
+
+klpm_run on a tree without a budget keeps every query's match state itself: queries whose match ends at the
+same tree position and continues with the same token form a group, and processing a prompt re-matches its
+group only.  These cases aim at the group machinery: groups of 2..32 (one warp), groups up to 4,096 (sorted in
+shared memory), larger groups (kept together), queries that have not arrived when their group changes,
+identical prompts, prompts that are prefixes of others, and the tie-priority / hit-rate variants."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2502_04677_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def K():
+    from paper_2502_04677_b200 import binding
+    return binding
+
+
+def dev(t):
+    return t.cuda() if isinstance(t, torch.Tensor) else torch.as_tensor(t).cuda()
+
+
+def run_gpu(K, prefill, prompts, arr, policy, k, prio=None, score_mode=0, start=0, c_num=0, c_den=1, legacy=False):
+    pt, po = W.to_csr(prefill)
+    qt, qo = W.to_csr(prompts)
+    n, npre = len(prompts), len(prefill)
+    cap = dict(max_nodes=2 * (n + npre) + 16, max_pool_tokens=pt.numel() + qt.numel() + 8 * (n + npre) + 16,
+               max_clock=n + npre + 16)
+    tree = K.rt_build(dev(pt), dev(po), **cap) if npre else K.rt_create(**cap)
+    order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    d_prio = None if prio is None else dev(torch.as_tensor(prio, dtype=torch.int64))
+    old = os.environ.pop("KLPM_RUN_LEGACY", None)
+    if legacy:
+        os.environ["KLPM_RUN_LEGACY"] = "1"
+    try:
+        K.klpm_run_ex(tree, dev(qt), dev(qo), dev(torch.as_tensor(arr, dtype=torch.int64)),
+                      K.make_params(policy, k, c_num, c_den, start), d_prio, score_mode, order, unc, ttft, comp)
+    finally:
+        os.environ.pop("KLPM_RUN_LEGACY", None)
+        if old is not None:
+            os.environ["KLPM_RUN_LEGACY"] = old
+    assert K.rt_sync_status(tree) == 0
+    assert K.klpm_run_path(tree) == (K.RUN_PATH_ONE_BY_ONE if legacy else K.RUN_PATH_GROUPED)
+    st = K.rt_stats(tree)
+    # the grown tree answers matches like the oracle's: every processed prompt is fully cached
+    m = torch.zeros(n, dtype=torch.int32, device="cuda")
+    K.rt_match_batch(tree, dev(qt), dev(qo), m)
+    assert K.rt_sync_status(tree) == 0
+    assert np.array_equal(m.cpu().numpy(), (qo[1:] - qo[:-1]).numpy())
+    K.rt_destroy(tree)
+    return order.cpu().numpy(), unc.cpu().numpy(), ttft.cpu().numpy(), comp.cpu().numpy(), st
+
+
+def run_oracle(prefill, prompts, arr, policy, k, prio=None, score_mode=0, start=0, c_num=0, c_den=1,
+               tier=oracle.TIER_UPDATE):
+    pt, po = W.to_csr(prefill)
+    qt, qo = W.to_csr(prompts)
+    ot = oracle.OracleTree(0)
+    if len(prefill):
+        ot.insert(pt.numpy(), po.numpy())
+    out = oracle.schedule(qt.numpy(), qo.numpy(), np.asarray(arr, dtype=np.int64), policy, k, c_num, c_den, start,
+                          oracle.CACHE_TREE, tier, ot, prio, score_mode)
+    return out + (ot.stats(),)
+
+
+def same(got, want):
+    for g, w, name in zip(got[:4], want[:4], ("order", "uncached", "ttft", "completion")):
+        assert np.array_equal(g, w), name
+    for key in ("n_nodes", "tokens", "clock"):
+        assert got[4][key] == want[4][key], key
+
+
+def shared_prefix_queue(seed, n, levels, tail, vocab, max_gap):
+    """Prompts = one block per level (each level has a few alternatives, so many prompts tie at every depth)
+    + a short random tail over a small alphabet; arrival gaps in [0, max_gap]."""
+    rng = np.random.RandomState(seed)
+    blocks = [[rng.randint(0, vocab, size=ln).tolist() for _ in range(alts)] for ln, alts in levels]
+    prompts, arr, t = [], [], 0
+    for _ in range(n):
+        p = []
+        for alts in blocks:
+            p += alts[rng.randint(len(alts))]
+        p += rng.randint(0, vocab, size=rng.randint(0, tail + 1)).tolist()
+        prompts.append(p)
+        t += int(rng.randint(0, max_gap + 1))
+        arr.append(t)
+    return prompts, arr
+
+
+@pytest.mark.parametrize("seed", range(3))
+@pytest.mark.parametrize("max_gap", [0, 40])
+def test_groups_of_every_size_small_queue(K, seed, max_gap):
+    """300 prompts over 3 levels of shared blocks and a binary tail: groups from 2 to ~150 members, identical
+    prompts, prompts that are prefixes of others; with gaps, members join their groups before they arrive."""
+    prompts, arr = shared_prefix_queue(seed, 300, [(6, 2), (5, 3), (4, 2)], tail=6, vocab=2, max_gap=max_gap)
+    prefill, _ = shared_prefix_queue(seed + 77, 10, [(6, 2), (5, 3)], tail=3, vocab=2, max_gap=0)
+    for policy, k in ((0, 1), (1, 1), (2, 2), (2, 5)):
+        got = run_gpu(K, prefill, prompts, arr, policy, k, c_num=1, c_den=3)
+        want = run_oracle(prefill, prompts, arr, policy, k, c_num=1, c_den=3, tier=oracle.TIER_REMATCH)
+        same(got, want)
+
+
+@pytest.mark.parametrize("max_gap", [0, 3])
+def test_groups_sorted_in_shared_memory(K, max_gap):
+    """3,000 prompts, empty tree: the first pick dissolves a group of ~1,500 (sorted inside the CTA), which
+    splits into groups of hundreds, and so on down to single queries."""
+    prompts, arr = shared_prefix_queue(5, 3000, [(12, 2), (9, 4), (7, 5)], tail=8, vocab=3, max_gap=max_gap)
+    for policy, k in ((1, 1), (2, 3)):
+        got = run_gpu(K, [], prompts, arr, policy, k)
+        want = run_oracle([], prompts, arr, policy, k)
+        same(got, want)
+
+
+@pytest.mark.parametrize("max_gap", [0, 2])
+def test_groups_too_large_to_sort(K, max_gap):
+    """6,000 prompts that all start with the same block: the first group has ~6,000 members (more than the CTA
+    sorts), so it stays one run whose members are checked one by one until it has shrunk."""
+    prompts, arr = shared_prefix_queue(9, 6000, [(10, 1), (8, 3), (6, 4)], tail=5, vocab=4, max_gap=max_gap)
+    got = run_gpu(K, [], prompts, arr, K.POLICY_KLPM, 4)
+    want = run_oracle([], prompts, arr, oracle.POLICY_KLPM, 4)
+    same(got, want)
+
+
+@pytest.mark.parametrize("score_mode", [0, 1])
+def test_grouped_loop_with_priorities_and_hit_rate(K, score_mode):
+    prompts, arr = shared_prefix_queue(21, 500, [(5, 2), (4, 3)], tail=7, vocab=2, max_gap=6)
+    prio = np.random.RandomState(3).randint(0, 50, size=len(prompts)).tolist()
+    for policy, k in ((1, 1), (2, 3)):
+        got = run_gpu(K, [], prompts, arr, policy, k, prio=prio, score_mode=score_mode)
+        want = run_oracle([], prompts, arr, policy, k, prio=prio, score_mode=score_mode, tier=oracle.TIER_REMATCH)
+        same(got, want)
+
+
+@pytest.mark.parametrize("name,scale,k", [("medium", 1 / 16, 4), ("adversarial", 1 / 256, 4), ("tiny", 1, 2)])
+def test_both_loops_agree(K, name, scale, k):
+    """The grouped loop and the one-by-one loop (forced by KLPM_RUN_LEGACY=1) give identical schedules."""
+    w = W.tiny() if name == "tiny" else W.WORKLOADS[name](scale=scale)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    prefill = [pt[po[i]:po[i + 1]].tolist() for i in range(po.numel() - 1)]
+    prompts = [qt[qo[i]:qo[i + 1]].tolist() for i in range(qo.numel() - 1)]
+    a = run_gpu(K, prefill, prompts, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick)
+    b = run_gpu(K, prefill, prompts, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick, legacy=True)
+    same(a, b)
+
+
+def test_capacity_too_small_falls_back_and_reports(K):
+    """A tree that cannot hold the whole queue takes the one-by-one loop, which reports the capacity error."""
+    prompts = [[1, 2, 3, 4, 5, 6, 7, 8, 9, 10], [1, 2, 3, 9, 9, 9, 9, 9, 9, 9], [5] * 12]
+    qt, qo = W.to_csr(prompts)
+    tree = K.rt_create(max_nodes=64, max_pool_tokens=20, max_clock=64)
+    n = len(prompts)
+    order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+    K.klpm_run(tree, dev(qt), dev(qo), dev(torch.zeros(n, dtype=torch.int64)), K.make_params(K.POLICY_LPM, 1), order, unc, ttft)
+    assert K.rt_sync_status(tree) == K.RT_ERR_CAPACITY
+    assert K.klpm_run_path(tree) == K.RUN_PATH_ONE_BY_ONE
+    K.rt_destroy(tree)
