@@ -289,7 +289,20 @@ def run_ours(args):
     while np2 < nq:
         np2 <<= 1
     lg = np2.bit_length() - 1
-    launches_per_step = 1 + 1 + lg * (lg + 1) // 2 + 1      # match, slot keys, bitonic steps, scheduling loop
+    run_path = K.klpm_run_path(tree)
+    sort_launches = lg * (lg + 1) // 2
+    if run_path == K.RUN_PATH_GROUPED:
+        # match; slot keys, arrival sort, slot arrays; slot records, walk of every query, group sort, groups, the loop;
+        # bulk insertion of the processed prompts: claim words, pending list, at least one round of two kernels, clock
+        launches_per_step = 1 + (1 + sort_launches + 1) + (1 + 1 + sort_launches + 1 + 1) + (1 + 1 + 2 + 1)
+        loop_kernel = "fast_run_kernel"
+        loop_note = ("sequential chain of picks in one CTA: per pick one dependent L2 round trip (the pick's state and its "
+                     "block of keys) plus a shared-memory tournament update; includes the walk of every query, two sorts "
+                     "and the bulk insertion of the processed prompts")
+    else:
+        launches_per_step = 1 + 1 + sort_launches + 1 + 1      # match, slot keys, bitonic steps, slot arrays, scheduling loop
+        loop_kernel = "run_kernel"
+        loop_note = "sequential chain: every pick depends on the tree after the previous one"
     ttft_cpu = ttft.cpu()
     out = {
         "metric": "prefix_match_queries_per_sec",
@@ -310,14 +323,15 @@ def run_ours(args):
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": alg_bytes, "traffic": TRAFFIC.get((name, args.scale))},
-        "decision_loop": {"kernel": "run_kernel", "bound": "latency", "us_per_decision": 1e6 * t_run / (nq * args.steps),
-                          "note": "sequential chain: every pick depends on the tree after the previous one"},
+        "decision_loop": {"kernel": loop_kernel, "bound": "latency", "us_per_decision": 1e6 * t_run / (nq * args.steps),
+                          "note": loop_note},
         "e2e": {"value": world * nq / e2e_match_s, "unit": "queries/s",
                 "what": "host query buffers in (pinned), rt_match_batch, match lengths out",
                 "ms_match_with_copies": 1e3 * e2e_match_s, "ms_per_step": 1e3 * e2e_s,
                 "decisions_per_sec_whole_step": world * nq / e2e_s,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * args.steps,
+        "gpu_launches_note": "lower bound: the bulk insertion at the end of klpm_run takes a data-dependent number of rounds",
         "clocks": clocks,
         "result": {"total_uncached_tokens": int(unc.sum().item()),
                    "ttft_p50": int(ttft_cpu.kthvalue(max(1, nq // 2)).values),
@@ -351,16 +365,24 @@ def k_sweep(K, tree, q_tok, q_off, arr, w, ks, device):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         main = torch.cuda.current_stream()
         a.record(main)
-        for k, t, st, o in zip(ks, trees, streams, outs):
-            if mode == "concurrent":
-                st.wait_stream(main)
+        if mode == "concurrent":
+            # klpm_run waits for its stream on trees without a budget, so every run gets a host thread of its own
+            def one(k, t, st, o):
+                torch.cuda.set_device(device)
                 with torch.cuda.stream(st):
                     K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
-            else:
-                K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
-        if mode == "concurrent":
+            for st in streams:
+                st.wait_stream(main)
+            threads = [threading.Thread(target=one, args=(k, t, st, o)) for k, t, st, o in zip(ks, trees, streams, outs)]
+            for th in threads:
+                th.start()
+            for th in threads:
+                th.join()
             for st in streams:
                 main.wait_stream(st)
+        else:
+            for k, t, st, o in zip(ks, trees, streams, outs):
+                K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
         b.record(main)
         torch.cuda.synchronize()
         ms = a.elapsed_time(b)

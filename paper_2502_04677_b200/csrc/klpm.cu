@@ -1369,6 +1369,15 @@ __global__ void fast_group_kernel(FastArgs A) {
     st_dyn_group(A.dyn + r, first, lo - first);
 }
 
+// Largest of the warp's 64-bit values with two hardware reductions: the high halves, then the low halves of
+// the lanes that hold the largest high half.
+__device__ __forceinline__ unsigned long long warp_max64r(unsigned long long v) {
+    const unsigned hi = (unsigned)(v >> 32);
+    const unsigned mh = __reduce_max_sync(FULL_MASK, hi);
+    const unsigned ml = __reduce_max_sync(FULL_MASK, hi == mh ? (unsigned)v : 0u);
+    return ((unsigned long long)mh << 32) | ml;
+}
+
 // ---- the tournament above the leaf blocks (shared memory) ----
 struct FastTour {
     unsigned long long* t1;   // per leaf block (padded with zeros to a multiple of 32)
@@ -1380,28 +1389,28 @@ struct FastTour {
 // Recompute the ancestors of leaf block b; returns the root.  One warp.
 __device__ __forceinline__ unsigned long long tour_update(const FastTour& R, int32_t b, int lane) {
     const int32_t i2 = b >> 5;
-    unsigned long long v = warp_max64(R.t1[(i2 << 5) + lane]);
+    unsigned long long v = warp_max64r(R.t1[(i2 << 5) + lane]);
     if (lane == 0) R.t2[i2] = v;
     __syncwarp();
     const int32_t i3 = i2 >> 5;
-    v = warp_max64(R.t2[(i3 << 5) + lane]);
+    v = warp_max64r(R.t2[(i3 << 5) + lane]);
     if (lane == 0) R.t3[i3] = v;
     __syncwarp();
-    return warp_max64(R.t3[lane]);
+    return warp_max64r(R.t3[lane]);
 }
 // Recompute t3 and the root from t2.  One warp.
 __device__ __forceinline__ unsigned long long tour_top(const FastTour& R, int lane) {
     for (int32_t i3 = 0; i3 < R.n3; ++i3) {
-        const unsigned long long v = warp_max64(R.t2[(i3 << 5) + lane]);
+        const unsigned long long v = warp_max64r(R.t2[(i3 << 5) + lane]);
         if (lane == 0) R.t3[i3] = v;
     }
     __syncwarp();
-    return warp_max64(R.t3[lane]);
+    return warp_max64r(R.t3[lane]);
 }
 // Recompute t2 from t1.  Every warp of the CTA; the caller synchronises.
 __device__ __forceinline__ void tour_mid(const FastTour& R, int warp, int nwarps, int lane) {
     for (int32_t i2 = warp; i2 < R.n2; i2 += nwarps) {
-        const unsigned long long v = warp_max64(R.t1[(i2 << 5) + lane]);
+        const unsigned long long v = warp_max64r(R.t1[(i2 << 5) + lane]);
         if (lane == 0) R.t2[i2] = v;
     }
 }
@@ -1568,6 +1577,7 @@ fast_run_kernel(FastArgs A) {
     int32_t head = 0, admitted = 0;
     long long next_t = __ldg(&A.stat[0].t);
     unsigned long long root = 0;
+    int32_t cyc = 0;                                        // c mod k
     for (int32_t c = 0; c < n; ++c) {
         // ---- time and arrivals: idle until somebody has arrived, then admit everybody who has
         if (head == admitted && next_t > now) now = next_t;
@@ -1609,7 +1619,8 @@ fast_run_kernel(FastArgs A) {
             next_t = admitted < n ? __ldg(&A.stat[admitted].t) : INF;
         }
         // ---- pick
-        const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
+        const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
+        if (++cyc == A.k) cyc = 0;
         int32_t slot = head;
         if (!fcfs_turn) {
             const unsigned rk = 0xffffffffu - (unsigned)(root & 0xffffffffULL);
@@ -1624,7 +1635,14 @@ fast_run_kernel(FastArgs A) {
             const long long r = ((long long)b << A.lb_shift) + u;
             if (r < admitted && r != slot) { const unsigned long long kk = __ldcg(A.key + r); if (kk > bm) bm = kk; }
         }
-        bm = warp_max64(bm);
+        // while those loads are in flight: the tournament without the pick's own ancestors
+        const int32_t i2 = b >> 5, i3 = i2 >> 5;
+        const unsigned long long o1 = warp_max64r(lane == (b & 31) ? 0ULL : R.t1[(i2 << 5) + lane]);
+        const unsigned long long o2 = warp_max64r(lane == (i2 & 31) ? 0ULL : R.t2[(i3 << 5) + lane]);
+        const unsigned long long o3 = warp_max64r(lane == i3 ? 0ULL : R.t3[lane]);
+        bm = warp_max64r(bm);
+        const unsigned long long v2 = bm > o1 ? bm : o1, v3 = v2 > o2 ? v2 : o2;
+        root = v3 > o3 ? v3 : o3;
         // ---- charge (Definition 2)
         const int32_t m = d.m, len = s.len, unc = len - m;
         if (m < 0) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 106); break; }                           // cannot happen
@@ -1638,7 +1656,7 @@ fast_run_kernel(FastArgs A) {
             __stcg(A.key + slot, 0ULL);
             if (A.done_in_smem) s_done[slot >> 5] |= 1u << (slot & 31);
             else __stcg(A.done + (slot >> 5), __ldcg(A.done + (slot >> 5)) | (1u << (slot & 31)));
-            R.t1[b] = bm;
+            R.t1[b] = bm; R.t2[i2] = v2; R.t3[i3] = v3;
         }
         __syncwarp();
         const long long vleaf = vnext;
@@ -1665,7 +1683,7 @@ fast_run_kernel(FastArgs A) {
                 while (tm) {
                     const int src = __ffs(tm) - 1; tm &= tm - 1;
                     const int32_t bb = __shfl_sync(FULL_MASK, r >> A.lb_shift, src);
-                    if (bb != b) root = tour_update(R, bb, lane);
+                    root = tour_update(R, bb, lane);
                 }
             } else {
                 if (lane == 0) { s_job.type = FAST_JOB_DISSOLVE; s_job.pick = P; }
@@ -1676,7 +1694,7 @@ fast_run_kernel(FastArgs A) {
                 full = true;
             }
         }
-        root = full ? tour_top(R, lane) : tour_update(R, b, lane);
+        if (full) root = tour_top(R, lane);
         // ---- the oldest unprocessed slot
         if (slot == head) {
             int32_t w0 = head >> 5;
