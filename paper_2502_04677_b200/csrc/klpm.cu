@@ -1235,11 +1235,11 @@ struct alignas(32) FDyn {     // what the loop changes, one 32-byte sector per s
     int32_t gstart, gcount;   // the slot's group: run [gstart, gstart + gcount) of the member array
     long long pad;
 };
-struct alignas(32) FStat {    // constant during the loop
-    long long soff;           // offset of the query's first token
+struct alignas(32) FStat {    // constant during the loop; the first 16 bytes are all that charging a pick needs
     long long t;              // arrival
     int32_t len;
     int32_t ord;              // query index
+    long long soff;           // offset of the query's first token
     int32_t rank;             // low key bits: rank by (tie priority, slot), or the slot itself
     int32_t pad;
 };
@@ -1260,12 +1260,14 @@ struct FastArgs {
     int32_t lb_shift;             // log2 of the number of slots per tournament leaf block
     int32_t nb;                   // number of leaf blocks
     int32_t done_in_smem;
+    int32_t run_ahead;            // the run-ahead mode of the loop can be used (32-slot leaf blocks, keys end in ~slot)
+    unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts
     unsigned long long* counter;  // [0] work counter of the initial walk, [1] sum of the tokens it found uncached
     TreeState* st;
 };
 
-#define KLPM_FAST_THREADS 512
-#define KLPM_FAST_SORT_CAP 4096          // largest group that is regrouped exactly (sorted in shared memory)
+#define KLPM_FAST_THREADS 256
+#define KLPM_FAST_SORT_CAP 2048          // largest group that is regrouped exactly (sorted in shared memory)
 #define KLPM_FAST_NOGROUP 0xffffffffffffffffULL
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {      // SplitMix64's finaliser
@@ -1301,9 +1303,10 @@ __device__ __forceinline__ FStat ld_stat(const FStat* p) {
     const int4* q = reinterpret_cast<const int4*>(p);
     const int4 a = __ldg(q), b = __ldg(q + 1);
     FStat s;
-    s.soff = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
-    s.t = (long long)(((unsigned long long)(unsigned)a.w << 32) | (unsigned)a.z);
-    s.len = b.x; s.ord = b.y; s.rank = b.z; s.pad = 0;
+    s.t = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+    s.len = a.z; s.ord = a.w;
+    s.soff = (long long)(((unsigned long long)(unsigned)b.y << 32) | (unsigned)b.x);
+    s.rank = b.z; s.pad = 0;
     return s;
 }
 __device__ __forceinline__ void named_bar(int id, int nthreads) {
@@ -1367,6 +1370,7 @@ __global__ void fast_group_kernel(FastArgs A) {
     const int32_t r = A.gidx[i];
     A.mem[i] = r;
     st_dyn_group(A.dyn + r, first, lo - first);
+    if (lo - first > 1) atomicOr(A.gbits + (r >> 5), 1u << (r & 31));
 }
 
 // Largest of the warp's 64-bit values with two hardware reductions: the high halves, then the low halves of
@@ -1379,10 +1383,16 @@ __device__ __forceinline__ unsigned long long warp_max64r(unsigned long long v) 
 }
 
 // ---- the tournament above the leaf blocks (shared memory) ----
+// t1[b] is the largest key of leaf block b among arrived, unprocessed slots; t1s[b] is the second largest, or
+// KLPM_FAST_PENDING when it is not known (whoever needs it then reads the block's keys).
+#define KLPM_FAST_PENDING 0xffffffffffffffffULL
 struct FastTour {
     unsigned long long* t1;   // per leaf block (padded with zeros to a multiple of 32)
+    unsigned long long* t1s;  // second largest key per leaf block, or KLPM_FAST_PENDING
     unsigned long long* t2;   // per 32 leaf blocks (padded likewise)
     unsigned long long* t3;   // 32 entries
+    unsigned int* done;       // bitmap of processed slots (shared memory), or null
+    unsigned int* gb;         // bitmap of slots whose group has more than one member (shared memory), or null
     int32_t n2;               // entries of t2 in use
     int32_t n3;               // entries of t3 in use
 };
@@ -1397,6 +1407,17 @@ __device__ __forceinline__ unsigned long long tour_update(const FastTour& R, int
     if (lane == 0) R.t3[i3] = v;
     __syncwarp();
     return warp_max64r(R.t3[lane]);
+}
+// Leaf block b's largest key becomes v: write it and its ancestors; returns the root.  One warp; every lane
+// performs the same stores, so each lane sees them in its own program order without a barrier.
+__device__ __forceinline__ unsigned long long tour_set(const FastTour& R, int32_t b, unsigned long long v, int lane) {
+    const int32_t i2 = b >> 5, i3 = i2 >> 5;
+    const unsigned long long o1 = warp_max64r(lane == (b & 31) ? 0ULL : R.t1[(i2 << 5) + lane]);
+    const unsigned long long o2 = warp_max64r(lane == (i2 & 31) ? 0ULL : R.t2[(i3 << 5) + lane]);
+    const unsigned long long o3 = warp_max64r(lane == i3 ? 0ULL : R.t3[lane]);
+    const unsigned long long v2 = v > o1 ? v : o1, v3 = v2 > o2 ? v2 : o2;
+    R.t1[b] = v; R.t2[i2] = v2; R.t3[i3] = v3;
+    return v3 > o3 ? v3 : o3;
 }
 // Recompute t3 and the root from t2.  One warp.
 __device__ __forceinline__ unsigned long long tour_top(const FastTour& R, int lane) {
@@ -1413,6 +1434,22 @@ __device__ __forceinline__ void tour_mid(const FastTour& R, int warp, int nwarps
         const unsigned long long v = warp_max64r(R.t1[(i2 << 5) + lane]);
         if (lane == 0) R.t2[i2] = v;
     }
+}
+// The two largest of the warp's keys (keys are distinct unless zero).
+__device__ __forceinline__ void warp_top2(unsigned long long k, unsigned long long* top1, unsigned long long* top2) {
+    const unsigned long long a = warp_max64r(k);
+    *top1 = a;
+    *top2 = warp_max64r(k == a ? 0ULL : k);
+}
+// has slot r been processed?  (the bitmap lives in shared memory when it fits)
+__device__ __forceinline__ bool slot_done(const FastTour& R, const FastArgs& A, long long r) {
+    const unsigned w = R.done ? R.done[r >> 5] : __ldcg(A.done + (r >> 5));
+    return (w >> (r & 31)) & 1u;
+}
+__device__ __forceinline__ void set_grouped(const FastTour& R, int32_t r, bool grouped) {
+    if (!R.gb) return;
+    if (grouped) atomicOr(R.gb + (r >> 5), 1u << (r & 31));
+    else atomicAnd(R.gb + (r >> 5), ~(1u << (r & 31)));
 }
 
 struct FastPick {             // the prompt being processed, as its group's members need it
@@ -1436,7 +1473,7 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
     FDyn d; d.pos = 0; d.m = -1; d.ntok = 0; d.gstart = 0; d.gcount = 0;
     FStat s; s.soff = 0; s.t = 0; s.len = 0; s.ord = 0; s.rank = 0;
     if (act) { d = ld_dyn(A.dyn + r); s = ld_stat(A.stat + r); }
-    const bool live = act && d.m >= 0;
+    const bool live = act && !slot_done(R, A, r);
     const bool tied = live && d.pos == P.pos && d.ntok == P.ntok && d.m == P.m && d.m < s.len;
     const int32_t* q = A.tok + s.soff;
     int32_t e = 0;
@@ -1455,7 +1492,11 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
         st_dyn_state(A.dyn + r, d.pos, d.m, d.ntok);
         const unsigned long long key = fast_key(d.m, s.len, s.rank, A.score_mode);
         __stcg(A.key + r, key);
-        if ((long long)r < P.admitted) { atomicMax(R.t1 + (r >> A.lb_shift), key); *touched = true; }
+        if ((long long)r < P.admitted) {
+            atomicMax(R.t1 + (r >> A.lb_shift), key);
+            R.t1s[r >> A.lb_shift] = KLPM_FAST_PENDING;
+            *touched = true;
+        }
     }
     if (!live) return KLPM_FAST_NOGROUP;
     return d.m < s.len ? group_hash(d.pos, d.ntok) : single_hash(r);
@@ -1466,17 +1507,21 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int tid = threadIdx.x, nthr = blockDim.x;
     if (J.type == FAST_JOB_ADMIT) {
-        // slots [a0, a1) have arrived: fold their keys into their leaf blocks
+        // slots [a0, a1) have arrived: the two largest keys of every leaf block they fall into
         const int32_t b0 = J.a0 >> A.lb_shift, b1 = (J.a1 - 1) >> A.lb_shift;
         const int32_t LB = 1 << A.lb_shift;
         for (int32_t b = b0 + warp; b <= b1; b += nwarps) {
-            unsigned long long v = 0;
+            unsigned long long v1 = 0, v2 = 0;              // this lane's two largest
             for (int32_t u = lane; u < LB; u += 32) {
                 const long long r = ((long long)b << A.lb_shift) + u;
-                if (r >= J.a0 && r < J.a1) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
+                if (r < J.a1 && !slot_done(R, A, r)) {
+                    const unsigned long long kk = __ldcg(A.key + r);
+                    if (kk > v1) { v2 = v1; v1 = kk; } else if (kk > v2) v2 = kk;
+                }
             }
-            v = warp_max64(v);
-            if (lane == 0 && v > R.t1[b]) R.t1[b] = v;
+            const unsigned long long top1 = warp_max64r(v1);
+            const unsigned long long top2 = warp_max64r(v1 == top1 ? v2 : v1);
+            if (lane == 0) { R.t1[b] = top1; R.t1s[b] = top2; }
         }
     } else {
         // dissolve a group of more than 32 members
@@ -1522,6 +1567,7 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
                 const int32_t r = sr[i];
                 __stcg(A.mem + gs + i, r);
                 st_dyn_group(A.dyn + r, gs + first, lo - first);
+                set_grouped(R, r, lo - first > 1);
             }
         } else {
             // too large to sort here: the live members stay together as one run (a superset of every group in it)
@@ -1533,13 +1579,22 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
             __syncthreads();
             const int32_t cnt = *s_cnt;
             for (int32_t i = tid; i < gc; i += nthr)
-                if ((unsigned long long)__ldcg(A.gh + i) != KLPM_FAST_NOGROUP) st_dyn_group(A.dyn + __ldcg(A.gidx + i), gs, cnt);
+                if ((unsigned long long)__ldcg(A.gh + i) != KLPM_FAST_NOGROUP) {
+                    const int32_t r = __ldcg(A.gidx + i);
+                    st_dyn_group(A.dyn + r, gs, cnt);
+                    set_grouped(R, r, cnt > 1);
+                }
         }
     }
     __syncthreads();
     tour_mid(R, warp, nwarps, lane);
     __syncthreads();
 }
+
+// Run-ahead mode of the sequencer: a pick whose state has not been read yet, and a leaf block whose keys have
+// been requested to find its second largest again.
+struct FastFlight { int32_t c; int32_t m; int4 s0; bool valid; };     // s0 = arrival, length, query index
+struct FastRefresh { int32_t b; unsigned long long k; bool valid; };
 
 __global__ void __launch_bounds__(KLPM_FAST_THREADS, 1)
 fast_run_kernel(FastArgs A) {
@@ -1552,14 +1607,18 @@ fast_run_kernel(FastArgs A) {
     const int32_t nwords = (n + 31) >> 5;
     FastTour R;
     R.t1 = reinterpret_cast<unsigned long long*>(fast_smem);
-    R.t2 = R.t1 + nb1p;
+    R.t1s = R.t1 + nb1p;
+    R.t2 = R.t1s + nb1p;
     R.t3 = R.t2 + n2p;
     R.n2 = n2; R.n3 = n3;
     unsigned long long* sh = R.t3 + 32;
     int32_t* sr = reinterpret_cast<int32_t*>(sh + KLPM_FAST_SORT_CAP);
     unsigned int* s_done = reinterpret_cast<unsigned int*>(sr + KLPM_FAST_SORT_CAP);
-    for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
+    R.done = A.done_in_smem ? s_done : nullptr;
+    R.gb = A.run_ahead ? s_done + nwords : nullptr;
+    for (int32_t i = threadIdx.x; i < 2 * nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
     if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
+    if (A.run_ahead) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) R.gb[i] = __ldcg(A.gbits + i);
     __syncthreads();
 
     if (warp != 0) {
@@ -1578,7 +1637,120 @@ fast_run_kernel(FastArgs A) {
     long long next_t = __ldg(&A.stat[0].t);
     unsigned long long root = 0;
     int32_t cyc = 0;                                        // c mod k
-    for (int32_t c = 0; c < n; ++c) {
+    int32_t c = 0;
+
+    // first unprocessed slot at or after `head` (which is processed)
+    auto advance_head = [&]() {
+        int32_t w0 = head >> 5;
+        for (;;) {
+            const int32_t wi = w0 + lane;
+            unsigned w = 0u;                                  // past the end: "unprocessed", so the search stops
+            if (wi < nwords) w = A.done_in_smem ? s_done[wi] : __ldcg(A.done + wi);
+            if (wi == (head >> 5)) w |= (1u << (head & 31)) - 1u;
+            const unsigned bal = __ballot_sync(FULL_MASK, w != 0xffffffffu);
+            if (bal) {
+                const int src = __ffs(bal) - 1;
+                const unsigned fw = ~__shfl_sync(FULL_MASK, w, src);
+                head = (w0 + src) * 32 + __ffs(fw) - 1;
+                break;
+            }
+            w0 += 32;
+        }
+        if (head > n) head = n;
+    };
+    // Definition 2 for one pick whose state has arrived; the outputs.  Every lane performs the same stores.
+    auto retire = [&](const FastFlight& F) {
+        const int32_t len = F.s0.z, ord = F.s0.w, unc = len - F.m;
+        const long long t = (long long)(((unsigned long long)(unsigned)F.s0.y << 32) | (unsigned)F.s0.x);
+        const long long begin = now > t ? now : t;
+        const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
+        now = Rj;
+        vnext += unc;
+        A.order[F.c] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - t;
+        if (A.completion) A.completion[ord] = Rj;
+    };
+    // The keys of leaf block G.b have arrived: its two largest among the unprocessed slots, as of now.
+    auto refresh_done = [&](const FastRefresh& G) {
+        const unsigned dw = s_done[G.b];
+        unsigned long long top1, top2;
+        warp_top2(((dw >> lane) & 1u) ? 0ULL : G.k, &top1, &top2);
+        R.t1s[G.b] = top2;
+        if (R.t1[G.b] != top1) root = tour_set(R, G.b, top1, lane);
+    };
+
+    while (c < n) {
+        // ================================================================ run-ahead
+        // Everybody has arrived, so the time of a pick no longer decides who can be picked: picks are made from
+        // shared memory alone (the block's second largest key takes over when its largest is picked), each
+        // pick's state is requested at once and used four picks later, and so are the keys of blocks whose
+        // second largest has to be found again.  A pick whose group has other members ends the burst: the
+        // picks in flight are finished in order and the careful step below takes that pick.
+        if (A.run_ahead && admitted == n) {
+            FastFlight F[4];
+            FastRefresh G[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { F[u].valid = false; G[u].valid = false; }
+            bool stop = false, draining = false;
+            for (;;) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (F[u].valid) { retire(F[u]); F[u].valid = false; }
+                    if (G[u].valid) { refresh_done(G[u]); G[u].valid = false; }
+                    if (stop) continue;
+                    if (c >= n) { stop = true; continue; }
+                    const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
+                    const int32_t j = fcfs_turn ? head : (int32_t)(0xffffffffu - (unsigned)(root & 0xffffffffULL));
+                    if (j < 0 || j >= n) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 107); stop = true; c = n; continue; }   // cannot happen
+                    if ((R.gb[j >> 5] >> (j & 31)) & 1u) { stop = true; continue; }
+                    // the pick is made
+                    if (++cyc == A.k) cyc = 0;
+                    F[u].c = c; F[u].valid = true;
+                    F[u].m = __ldcg(&A.dyn[j].m);
+                    F[u].s0 = __ldg(reinterpret_cast<const int4*>(A.stat + j));
+                    ++c;
+                    const int32_t b = j >> 5;
+                    s_done[b] |= 1u << (j & 31);
+                    const unsigned want = 0xffffffffu - (unsigned)j;          // low half of j's key
+                    const unsigned long long best = R.t1[b], sec = R.t1s[b];
+                    bool ask = false;
+                    if ((unsigned)best == want) {                              // j was its block's largest
+                        if (sec != KLPM_FAST_PENDING) {
+                            root = tour_set(R, b, sec, lane);
+                            R.t1s[b] = KLPM_FAST_PENDING;
+                            ask = true;
+                        } else {
+                            // the second largest is not known: take what is in flight, then read the block if need be
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) if (G[v].valid) { refresh_done(G[v]); G[v].valid = false; }
+                            if ((unsigned)R.t1[b] == want) {
+                                FastRefresh Q;
+                                Q.b = b; Q.valid = true;
+                                const long long r = ((long long)b << 5) + lane;
+                                Q.k = r < n ? __ldcg(A.key + r) : 0ULL;
+                                refresh_done(Q);
+                            }
+                        }
+                    } else if (sec != KLPM_FAST_PENDING && (unsigned)sec == want) {
+                        R.t1s[b] = KLPM_FAST_PENDING;
+                        ask = true;
+                    }
+                    if (ask) {
+                        const long long r = ((long long)b << 5) + lane;
+                        G[u].b = b; G[u].valid = true;
+                        G[u].k = r < n ? __ldcg(A.key + r) : 0ULL;
+                    }
+                    if (j == head) advance_head();
+                }
+                if (stop) {
+                    if (draining) break;
+                    draining = true;
+                }
+            }
+            __syncwarp();
+            if (c >= n) break;
+        }
+
+        // ================================================================ one careful step
         // ---- time and arrivals: idle until somebody has arrived, then admit everybody who has
         if (head == admitted && next_t > now) now = next_t;
         if (next_t <= now) {
@@ -1603,7 +1775,7 @@ fast_run_kernel(FastArgs A) {
             }
             if (a1 - admitted <= 32) {
                 const int32_t r = admitted + lane;
-                if (r < a1) atomicMax(R.t1 + (r >> A.lb_shift), __ldcg(A.key + r));
+                if (r < a1) { atomicMax(R.t1 + (r >> A.lb_shift), __ldcg(A.key + r)); R.t1s[r >> A.lb_shift] = KLPM_FAST_PENDING; }
                 __syncwarp();
                 root = tour_update(R, admitted >> A.lb_shift, lane);
                 if (((a1 - 1) >> A.lb_shift) != (admitted >> A.lb_shift)) root = tour_update(R, (a1 - 1) >> A.lb_shift, lane);
@@ -1630,37 +1802,40 @@ fast_run_kernel(FastArgs A) {
         const FDyn d = ld_dyn(A.dyn + slot);
         const FStat s = ld_stat(A.stat + slot);
         const int32_t b = slot >> A.lb_shift;
-        unsigned long long bm = 0;                          // the pick's leaf block without the pick
+        unsigned long long k1 = 0, k2 = 0;                  // this lane's two largest keys of the pick's leaf block, the pick left out
         for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
             const long long r = ((long long)b << A.lb_shift) + u;
-            if (r < admitted && r != slot) { const unsigned long long kk = __ldcg(A.key + r); if (kk > bm) bm = kk; }
+            if (r < admitted && r != slot && !slot_done(R, A, r)) {
+                const unsigned long long kk = __ldcg(A.key + r);
+                if (kk > k1) { k2 = k1; k1 = kk; } else if (kk > k2) k2 = kk;
+            }
         }
         // while those loads are in flight: the tournament without the pick's own ancestors
         const int32_t i2 = b >> 5, i3 = i2 >> 5;
         const unsigned long long o1 = warp_max64r(lane == (b & 31) ? 0ULL : R.t1[(i2 << 5) + lane]);
         const unsigned long long o2 = warp_max64r(lane == (i2 & 31) ? 0ULL : R.t2[(i3 << 5) + lane]);
         const unsigned long long o3 = warp_max64r(lane == i3 ? 0ULL : R.t3[lane]);
-        bm = warp_max64r(bm);
+        const unsigned long long bm = warp_max64r(k1);
+        const unsigned long long bs = warp_max64r(k1 == bm ? k2 : k1);
         const unsigned long long v2 = bm > o1 ? bm : o1, v3 = v2 > o2 ? v2 : o2;
         root = v3 > o3 ? v3 : o3;
         // ---- charge (Definition 2)
         const int32_t m = d.m, len = s.len, unc = len - m;
-        if (m < 0) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 106); break; }                           // cannot happen
+        if (slot_done(R, A, slot)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 106); break; }          // cannot happen
         const long long begin = now > s.t ? now : s.t;
         const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
         now = Rj;
         if (lane == 0) {
             A.order[c] = s.ord; A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
             if (A.completion) A.completion[s.ord] = Rj;
-            st_dyn_state(A.dyn + slot, d.pos, -1, d.ntok);
-            __stcg(A.key + slot, 0ULL);
             if (A.done_in_smem) s_done[slot >> 5] |= 1u << (slot & 31);
             else __stcg(A.done + (slot >> 5), __ldcg(A.done + (slot >> 5)) | (1u << (slot & 31)));
-            R.t1[b] = bm; R.t2[i2] = v2; R.t3[i3] = v3;
+            R.t1[b] = bm; R.t1s[b] = bs; R.t2[i2] = v2; R.t3[i3] = v3;
         }
         __syncwarp();
         const long long vleaf = vnext;
         vnext += unc;
+        ++c;
         // ---- the queries tied with the pick now match into its new leaf
         bool full = false;
         if (unc > 0 && d.gcount > 1) {
@@ -1672,12 +1847,16 @@ fast_run_kernel(FastArgs A) {
                 bool touched;
                 const unsigned long long h = fast_member(A, P, R, r, lane, &touched);
                 int32_t rank = 0, start = 0, cnt = 0;       // regroup inside the run
-                for (int k2 = 0; k2 < 32; ++k2) {
-                    const unsigned long long hk = __shfl_sync(FULL_MASK, h, k2);
+                for (int k2i = 0; k2i < 32; ++k2i) {
+                    const unsigned long long hk = __shfl_sync(FULL_MASK, h, k2i);
                     const bool lt = hk < h, eq = hk == h;
-                    start += lt; cnt += eq; rank += (lt || (eq && k2 < lane));
+                    start += lt; cnt += eq; rank += (lt || (eq && k2i < lane));
                 }
-                if (h != KLPM_FAST_NOGROUP) { __stcg(A.mem + d.gstart + rank, r); st_dyn_group(A.dyn + r, d.gstart + start, cnt); }
+                if (h != KLPM_FAST_NOGROUP) {
+                    __stcg(A.mem + d.gstart + rank, r);
+                    st_dyn_group(A.dyn + r, d.gstart + start, cnt);
+                    set_grouped(R, r, cnt > 1);
+                }
                 __syncwarp();
                 unsigned tm = __ballot_sync(FULL_MASK, touched);
                 while (tm) {
@@ -1696,24 +1875,7 @@ fast_run_kernel(FastArgs A) {
         }
         if (full) root = tour_top(R, lane);
         // ---- the oldest unprocessed slot
-        if (slot == head) {
-            int32_t w0 = head >> 5;
-            for (;;) {
-                const int32_t wi = w0 + lane;
-                unsigned w = 0u;                              // past the end: "unprocessed", so the search stops
-                if (wi < nwords) w = A.done_in_smem ? s_done[wi] : __ldcg(A.done + wi);
-                if (wi == (head >> 5)) w |= (1u << (head & 31)) - 1u;
-                const unsigned bal = __ballot_sync(FULL_MASK, w != 0xffffffffu);
-                if (bal) {
-                    const int src = __ffs(bal) - 1;
-                    const unsigned fw = ~__shfl_sync(FULL_MASK, w, src);
-                    head = (w0 + src) * 32 + __ffs(fw) - 1;
-                    break;
-                }
-                w0 += 32;
-            }
-            if (head > n) head = n;
-        }
+        if (slot == head) advance_head();
         __syncwarp();
     }
     if (lane == 0) s_job.type = FAST_JOB_EXIT;
@@ -2011,7 +2173,7 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_mem, np2))) return s;
     if ((s = dalloc(&t->fast_gh, np2))) return s;
     if ((s = dalloc(&t->fast_gidx, np2))) return s;
-    if ((s = dalloc(&t->fast_done, np2 / 32 + 64))) return s;
+    if ((s = dalloc(&t->fast_done, 2 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap
     if ((s = dalloc(&t->fast_counter, 2))) return s;
     t->fast_cap = np2;
     return RT_OK;
@@ -2495,11 +2657,16 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.nb = (int32_t)(((long long)n + (1LL << lbs) - 1) >> lbs);
         const long long nb1p = (f.nb + 31) & ~31, n2p = ((nb1p >> 5) + 31) & ~31;
         const long long nwords = ((long long)n + 31) >> 5;
-        size_t smem = (size_t)(nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
-        f.done_in_smem = smem + (size_t)nwords * 4 <= 200 * 1024 ? 1 : 0;
+        size_t smem = (size_t)(2 * nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
+        const size_t smem_max = 226 * 1024;
+        f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
+        // run-ahead needs both bitmaps in shared memory, 32-slot leaf blocks and keys whose low half names the slot
+        f.run_ahead = (f.done_in_smem && lbs == 5 && !d_tie_priority && smem + (size_t)nwords * 4 <= smem_max) ? 1 : 0;
+        if (f.run_ahead) smem += (size_t)nwords * 4;
+        f.gbits = tree->fast_done + (np2 / 32 + 32);
         const unsigned nblk = (unsigned)((n + 255) / 256), pblk = (unsigned)((np2 + 255) / 256);
-        CK(cudaMemsetAsync(f.done, 0, (size_t)(np2 / 32 + 64) * sizeof(unsigned int), s));
+        CK(cudaMemsetAsync(f.done, 0, (size_t)(2 * (np2 / 32 + 32)) * sizeof(unsigned int), s));
         // groups: queries whose match ends at the same position and continues with the same token
         for (long long k = 2; k <= np2; k <<= 1)
             for (long long j = k >> 1; j > 0; j >>= 1)
