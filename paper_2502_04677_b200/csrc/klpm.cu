@@ -1905,10 +1905,13 @@ bulk_walk_kernel(TreeDev T, BulkArgs A, unsigned n_pending) {
         const int32_t i = __ldg(A.pend_in + p);
         const int64_t lo = __ldg(A.off + i);
         const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
-        Term t = walk<true>(T, A.tok + lo, len);
-        if (lane == 0 && !(t.m == len && t.full)) {
-            A.pm[i] = t.m; A.pnode[i] = t.node; A.poff[i] = t.full ? -1 : t.off;
-            if (!t.full) atomicMin(&A.claim[t.node], i);
+        // the tree has no budget, so the walk streams along contiguous pool runs (as the batched match does)
+        int32_t node, off;
+        const int32_t m = walk_chain(T, A.tok + lo, len, true, &node, &off);
+        const bool full = node == 0 || off == __ldg(T.span_len + node);     // ends on a node boundary (or at the root)
+        if (lane == 0 && !(m == len && full)) {
+            A.pm[i] = m; A.pnode[i] = node; A.poff[i] = full ? -1 : off;
+            if (!full) atomicMin(&A.claim[node], i);
             A.pend_out[atomicAdd(A.n_out, 1u)] = i;
         }
     }
@@ -2090,6 +2093,9 @@ struct rt_tree {
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
+    long long bulk_cap;     // bulk insertion: prompts its per-prompt scratch holds
+    int32_t *bulk_pend_a, *bulk_pend_b, *bulk_pm, *bulk_pnode, *bulk_poff;
+    unsigned int* bulk_n_out;
     // checkpoint (rt_checkpoint / rt_rollback): copies of everything a later call can modify
     bool ck_valid;
     int32_t *ck_parent, *ck_depth_start, *ck_span_len, *ck_nchild, *ck_clock_owner, *ck_first_tok;
@@ -2124,6 +2130,8 @@ void free_tree(rt_tree* t) {
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
     cudaFree(t->claim);
+    cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
+    cudaFree(t->bulk_n_out);
     cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
     cudaFree(t->ck_clock_owner); cudaFree(t->ck_span_off); cudaFree(t->ck_last_access); cudaFree(t->ck_dead);
     cudaFree(t->ck_table); cudaFree(t->ck_st);
@@ -2189,14 +2197,18 @@ StaticSelectScratch* g_select_static_addr[64] = {nullptr};   // device address o
 
 // Many prompts at once into a tree without a budget (see the bulk kernels).  Waits for the stream once per round.
 rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s) {
-    int32_t *pend_a = nullptr, *pend_b = nullptr, *pm = nullptr, *pnode = nullptr, *poff = nullptr;
-    unsigned int* n_out = nullptr;
     rt_status st = RT_OK;
-    if ((st = dalloc(&pend_a, n)) || (st = dalloc(&pend_b, n)) || (st = dalloc(&pm, n)) || (st = dalloc(&pnode, n)) ||
-        (st = dalloc(&poff, n)) || (st = dalloc(&n_out, 1))) {
-        cudaFree(pend_a); cudaFree(pend_b); cudaFree(pm); cudaFree(pnode); cudaFree(poff); cudaFree(n_out);
-        return st;
+    if (n > t->bulk_cap) {                     // per-prompt scratch, kept for later calls
+        cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
+        t->bulk_pend_a = t->bulk_pend_b = t->bulk_pm = t->bulk_pnode = t->bulk_poff = nullptr;
+        t->bulk_cap = 0;
+        if ((st = dalloc(&t->bulk_pend_a, n)) || (st = dalloc(&t->bulk_pend_b, n)) || (st = dalloc(&t->bulk_pm, n)) ||
+            (st = dalloc(&t->bulk_pnode, n)) || (st = dalloc(&t->bulk_poff, n))) return st;
+        t->bulk_cap = n;
     }
+    if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 1))) return st;
+    int32_t *pend_a = t->bulk_pend_a, *pend_b = t->bulk_pend_b, *pm = t->bulk_pm, *pnode = t->bulk_pnode, *poff = t->bulk_poff;
+    unsigned int* n_out = t->bulk_n_out;
     // claim words start idle (an earlier call that ran out of capacity may have left some set)
     bulk_fill_kernel<<<(unsigned)((t->dev.max_nodes + 255) / 256), 256, 0, s>>>(t->claim, t->dev.max_nodes, 0x7fffffff);
     bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(pend_a, n);
@@ -2230,7 +2242,6 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         e = cudaGetLastError();
     }
     cudaStreamSynchronize(s);
-    cudaFree(pend_a); cudaFree(pend_b); cudaFree(pm); cudaFree(pnode); cudaFree(poff); cudaFree(n_out);
     if (e != cudaSuccess) { fprintf(stderr, "klpm: bulk insert failed: %s\n", cudaGetErrorString(e)); return RT_ERR_CUDA; }
     return st;
 }
@@ -2651,14 +2662,20 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
                   h.clock + (long long)n + 1 < tree->dev.max_clock;
     }
     if (grouped) {
+        // Leaf blocks of 32 slots while at most 8,192 of them are needed, larger ones beyond (queues above 262,144).
+        // Two environment variables shrink the limits so that small queues can exercise the large-queue layout:
+        // KLPM_FAST_MAX_BLOCKS (leaf blocks) and KLPM_FAST_SMEM_KB (shared memory the loop may use).
+        long long max_blocks = 8192;
+        size_t smem_max = 226 * 1024;
+        if (const char* e = getenv("KLPM_FAST_MAX_BLOCKS")) { const long long v = atoll(e); if (v >= 1 && v < max_blocks) max_blocks = v; }
+        if (const char* e = getenv("KLPM_FAST_SMEM_KB")) { const long long v = atoll(e); if (v >= 1 && (size_t)v * 1024 < smem_max) smem_max = (size_t)v * 1024; }
         int lbs = 5;
-        while ((((long long)n + (1LL << lbs) - 1) >> lbs) > 8192) ++lbs;
+        while ((((long long)n + (1LL << lbs) - 1) >> lbs) > max_blocks) ++lbs;
         f.lb_shift = lbs;
         f.nb = (int32_t)(((long long)n + (1LL << lbs) - 1) >> lbs);
         const long long nb1p = (f.nb + 31) & ~31, n2p = ((nb1p >> 5) + 31) & ~31;
         const long long nwords = ((long long)n + 31) >> 5;
         size_t smem = (size_t)(2 * nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
-        const size_t smem_max = 226 * 1024;
         f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
         // run-ahead needs both bitmaps in shared memory, 32-slot leaf blocks and keys whose low half names the slot

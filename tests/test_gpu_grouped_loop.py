@@ -2,7 +2,7 @@
 
 klpm_run on a tree without a budget keeps every query's match state itself: queries whose match ends at the
 same tree position and continues with the same token form a group, and processing a prompt re-matches its
-group only.  These cases aim at the group machinery: groups of 2..32 (one warp), groups up to 4,096 (sorted in
+group only.  These cases aim at the group machinery: groups of 2..32 (one warp), groups up to 2,048 (sorted in
 shared memory), larger groups (kept together), queries that have not arrived when their group changes,
 identical prompts, prompts that are prefixes of others, and the tie-priority / hit-rate variants."""
 import os
@@ -152,6 +152,35 @@ def test_both_loops_agree(K, name, scale, k):
     a = run_gpu(K, prefill, prompts, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick)
     b = run_gpu(K, prefill, prompts, w.arrivals, K.POLICY_KLPM, k, start=w.start_tick, legacy=True)
     same(a, b)
+
+
+@pytest.mark.parametrize("max_blocks,smem_kb", [(16, 0), (4, 60), (1, 0)])
+def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb, monkeypatch):
+    """Queues above 262,144 use larger tournament leaf blocks, and far larger ones keep the processed bitmap in
+    global memory; neither uses run-ahead.  Shrinking the limits makes a 3,000-query stream take those paths."""
+    monkeypatch.setenv("KLPM_FAST_MAX_BLOCKS", str(max_blocks))
+    if smem_kb:
+        monkeypatch.setenv("KLPM_FAST_SMEM_KB", str(smem_kb))
+    prompts, arr = shared_prefix_queue(31, 3000, [(12, 3), (9, 4)], tail=9, vocab=5, max_gap=2)
+    prefill, _ = shared_prefix_queue(32, 200, [(12, 3), (9, 4)], tail=4, vocab=5, max_gap=0)
+    for policy, k in ((2, 4), (0, 1)):
+        got = run_gpu(K, prefill, prompts, arr, policy, k)
+        want = run_oracle(prefill, prompts, arr, policy, k)
+        same(got, want)
+
+
+def test_run_ahead_bursts_all_arrived(K):
+    """Everybody waiting from the start and mostly distinct continuations: the loop runs ahead in long bursts,
+    broken by the few grouped queries (medium at 1/8: 4,096 queries, 64 prefixes)."""
+    w = W.medium(scale=1 / 8)
+    pt, po = w.prefill.materialize()
+    qt, qo = w.queries.materialize()
+    prefill = [pt[po[i]:po[i + 1]].tolist() for i in range(po.numel() - 1)]
+    prompts = [qt[qo[i]:qo[i + 1]].tolist() for i in range(qo.numel() - 1)]
+    for policy, k in ((K.POLICY_LPM, 1), (K.POLICY_KLPM, 3), (K.POLICY_FCFS, 1)):
+        got = run_gpu(K, prefill, prompts, w.arrivals, policy, k, start=w.start_tick)
+        want = run_oracle(prefill, prompts, w.arrivals, policy, k, start=w.start_tick)
+        same(got, want)
 
 
 def test_capacity_too_small_falls_back_and_reports(K):
