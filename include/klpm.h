@@ -193,14 +193,16 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
  * processed whose own match ended at the same place and goes on with the same token; the loop then keeps every
  * query's match state itself and stores all processed prompts in the tree at the end, concurrently (as rt_insert
  * does for large batches) -- same outputs, same cached prefixes and node boundaries.  In that case the call waits
- * for `stream` (the concurrent insertion does between its rounds). */
+ * for `stream` (the concurrent insertion does between its rounds), and a tree too small for the queue still gets
+ * every output (they do not depend on the tree's capacity) while the status word reports RT_ERR_CAPACITY and the
+ * tree, still valid, holds only part of the queue. */
 rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
                    const int64_t* d_arrival, int32_t n, const klpm_params* params, int32_t* d_order,
                    int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
 
 /* Which loop the last klpm_run / klpm_run_ex on this tree took: 0 = none yet, 1 = one decision at a time on the
- * tree itself (trees with a budget; also a tree without one whose capacity might not hold the whole queue),
- * 2 = the grouped loop (trees without a budget; see klpm_run).  Both give the same outputs. */
+ * tree itself (trees with a budget), 2 = the grouped loop (trees without a budget; see klpm_run).  Both give the
+ * same outputs.  Setting the environment variable KLPM_RUN_LEGACY=1 makes trees without a budget take loop 1 too. */
 int32_t klpm_run_path(const rt_tree* tree);
 
 /* klpm_run with two variants of the longest-match pick (the oldest-first picks are not affected):

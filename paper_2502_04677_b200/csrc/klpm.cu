@@ -1262,7 +1262,7 @@ struct FastArgs {
     int32_t done_in_smem;
     int32_t run_ahead;            // the run-ahead mode of the loop can be used (32-slot leaf blocks, keys end in ~slot)
     unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts
-    unsigned long long* counter;  // [0] work counter of the initial walk, [1] sum of the tokens it found uncached
+    unsigned long long* counter;  // work counter of the initial walk
     TreeState* st;
 };
 
@@ -1348,7 +1348,6 @@ fast_walk_kernel(TreeDev T, FastArgs A, long long np2) {
         const int32_t m = walk_chain<true>(T, q, len, false, &node, &off, &pos);
         if (lane == 0) {
             const int32_t ntok = m < len ? __ldg(q + m) : 0;
-            atomicAdd(A.counter + 1, (unsigned long long)(len - m));      // an upper bound of what the queue will append
             st_dyn_state(A.dyn + r, pos, m, ntok);
             A.key[r] = fast_key(m, len, s.rank, A.score_mode);
             A.gh[r] = (long long)(m < len ? group_hash(pos, ntok) : single_hash(r));
@@ -2015,7 +2014,10 @@ __global__ void bulk_fill_kernel(int32_t* p, long long n, int32_t v) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) p[i] = v;
 }
-__global__ void bulk_finish_kernel(TreeState* S, long long n) { S->clock += n; }
+__global__ void bulk_finish_kernel(TreeState* S, long long n, long long max_clock) {
+    if (S->clock + n + 1 >= max_clock) set_status(S, RT_ERR_CAPACITY);
+    else S->clock += n;
+}
 
 // batch size B: a query is finished when the last query of its bin of the processing order is
 __global__ void batch_times_kernel(const int32_t* __restrict__ order, int32_t n, const int64_t* __restrict__ arrival,
@@ -2182,7 +2184,7 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_gh, np2))) return s;
     if ((s = dalloc(&t->fast_gidx, np2))) return s;
     if ((s = dalloc(&t->fast_done, 2 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap
-    if ((s = dalloc(&t->fast_counter, 2))) return s;
+    if ((s = dalloc(&t->fast_counter, 1))) return s;
     t->fast_cap = np2;
     return RT_OK;
 }
@@ -2238,7 +2240,7 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         }
     }
     if (e == cudaSuccess && st == RT_OK) {
-        bulk_finish_kernel<<<1, 1, 0, s>>>(t->dev.st, (long long)n);
+        bulk_finish_kernel<<<1, 1, 0, s>>>(t->dev.st, (long long)n, t->dev.max_clock);
         e = cudaGetLastError();
     }
     cudaStreamSynchronize(s);
@@ -2606,8 +2608,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     if (st) return st;
     long long np2 = 1;
     while (np2 < n) np2 <<= 1;
-    // A tree without a budget takes the grouped loop, provided the whole queue is certain to fit (otherwise the
-    // one-by-one loop below stores what fits and reports the rest).  KLPM_RUN_LEGACY=1 forces the older loop.
+    // A tree without a budget takes the grouped loop.  KLPM_RUN_LEGACY=1 forces the one-by-one loop.
     bool grouped = false;
     if (tree->cfg.budget_tokens == 0) {
         const char* legacy = getenv("KLPM_RUN_LEGACY");
@@ -2630,9 +2631,9 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         }
         CK(cudaGetLastError());
     }
-    FastArgs f;
-    memset(&f, 0, sizeof(f));
     if (grouped) {
+        FastArgs f;
+        memset(&f, 0, sizeof(f));
         st = ensure_fast_scratch(tree, n);
         if (st) return st;
         f.tok = d_q_tokens; f.n = n; f.policy = params->policy; f.k = params->k; f.score_mode = score_mode;
@@ -2646,22 +2647,11 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         // every query is matched once against the tree as it stands
         fast_stat_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, tree->run_key, d_q_offsets,
                                                                      d_tie_priority ? tree->run_prank : nullptr, n, f.stat);
-        CK(cudaMemsetAsync(f.counter, 0, 2 * sizeof(unsigned long long), s));
+        CK(cudaMemsetAsync(f.counter, 0, sizeof(unsigned long long), s));
         long long wblocks = (np2 + 7) / 8;
         if (wblocks > (long long)tree->num_sms * 8) wblocks = (long long)tree->num_sms * 8;
         fast_walk_kernel<<<(unsigned)wblocks, 256, 0, s>>>(tree->dev, f, np2);
         CK(cudaGetLastError());
-        // does everything the queue can append fit?  (an upper bound: what the tree does not hold now)
-        TreeState h;
-        unsigned long long unc_bound = 0;
-        CK(cudaMemcpyAsync(&h, tree->dev.st, sizeof(h), cudaMemcpyDeviceToHost, s));
-        CK(cudaMemcpyAsync(&unc_bound, f.counter + 1, sizeof(unc_bound), cudaMemcpyDeviceToHost, s));
-        CK(cudaStreamSynchronize(s));
-        grouped = h.status == 0 && h.n_nodes + 2LL * n <= tree->dev.max_nodes &&
-                  h.pool_used + (long long)unc_bound + 6LL * n <= tree->dev.max_pool &&
-                  h.clock + (long long)n + 1 < tree->dev.max_clock;
-    }
-    if (grouped) {
         // Leaf blocks of 32 slots while at most 8,192 of them are needed, larger ones beyond (queues above 262,144).
         // Two environment variables shrink the limits so that small queues can exercise the large-queue layout:
         // KLPM_FAST_MAX_BLOCKS (leaf blocks) and KLPM_FAST_SMEM_KB (shared memory the loop may use).
@@ -2694,7 +2684,8 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         fast_run_kernel<<<1, KLPM_FAST_THREADS, smem, s>>>(f);
         CK(cudaGetLastError());
         tree->run_path = 2;
-        // the processed prompts enter the tree together (the logical clock advances by n)
+        // The processed prompts enter the tree together (the logical clock advances by n).  The loop itself needs
+        // no room in the tree; if the tree cannot hold the queue the insertion says so through the status word.
         return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s);
     }
     RunBcast bc0;

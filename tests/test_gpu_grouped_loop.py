@@ -183,16 +183,24 @@ def test_run_ahead_bursts_all_arrived(K):
         same(got, want)
 
 
-def test_capacity_too_small_falls_back_and_reports(K):
-    """A tree that cannot hold the whole queue takes the one-by-one loop, which reports the capacity error."""
-    prompts = [[1, 2, 3, 4, 5, 6, 7, 8, 9, 10], [1, 2, 3, 9, 9, 9, 9, 9, 9, 9], [5] * 12]
+def test_tree_too_small_for_the_queue(K):
+    """The grouped loop needs no room in the tree: every output is still produced, the insertion at the end
+    reports the capacity error, and the tree stays usable."""
+    prompts = [[1, 2, 3, 4, 5, 6, 7, 8, 9, 10], [1, 2, 3, 9, 9, 9, 9, 9, 9, 9], [5] * 12] * 30
+    arr = list(range(len(prompts)))
     qt, qo = W.to_csr(prompts)
-    tree = K.rt_create(max_nodes=64, max_pool_tokens=20, max_clock=64)
+    tree = K.rt_create(max_nodes=256, max_pool_tokens=20, max_clock=256)
     n = len(prompts)
     order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
     unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
     ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
-    K.klpm_run(tree, dev(qt), dev(qo), dev(torch.zeros(n, dtype=torch.int64)), K.make_params(K.POLICY_LPM, 1), order, unc, ttft)
+    K.klpm_run(tree, dev(qt), dev(qo), dev(torch.tensor(arr, dtype=torch.int64)), K.make_params(K.POLICY_LPM, 1), order, unc, ttft)
     assert K.rt_sync_status(tree) == K.RT_ERR_CAPACITY
-    assert K.klpm_run_path(tree) == K.RUN_PATH_ONE_BY_ONE
+    assert K.klpm_run_path(tree) == K.RUN_PATH_GROUPED
+    want = run_oracle([], prompts, arr, oracle.POLICY_LPM, 1)
+    assert np.array_equal(order.cpu().numpy(), want[0]) and np.array_equal(unc.cpu().numpy(), want[1])
+    assert np.array_equal(ttft.cpu().numpy(), want[2])
+    m = torch.zeros(n, dtype=torch.int32, device="cuda")
+    K.rt_match_batch(tree, dev(qt), dev(qo), m)           # the partly filled tree still answers
+    assert int(m.max()) <= 12
     K.rt_destroy(tree)
