@@ -1891,7 +1891,8 @@ fast_run_kernel(FastArgs A) {
 // ------------------------------------------------------------------------------------------------
 struct BulkArgs {
     const int32_t* tok; const int64_t* off;
-    const int32_t* pend_in; int32_t* pend_out; unsigned int* n_out;
+    const int32_t* pend_in; int32_t* pend_out; unsigned int* n_out;   // walk: prompts to walk -> prompts not fully stored yet
+    int32_t* pend_next; unsigned int* n_next;                          // apply: prompts that have to try again next round
     int32_t* claim;                    // per node: lowest prompt index that wants to cut its edge
     int32_t* pm; int32_t* pnode; int32_t* poff;   // per prompt: where its walk ended
 };
@@ -1931,10 +1932,10 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
         const int32_t unc = len - m;
         int64_t dst = -1;
         if (lane == 0) {
-            bool go = true;
+            bool go = true, retry = false;
             int32_t end = node;
             if (off >= 0) {                                 // the match ends inside node's edge: cut it
-                if (A.claim[node] != i) go = false;
+                if (A.claim[node] != i) { go = false; retry = true; }     // another prompt cuts this edge in this round
                 else {
                     A.claim[node] = 0x7fffffff;
                     const long long u = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
@@ -1975,7 +1976,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                 for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
                     unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
                     if (old == 0ULL) { won = (long long)sl2; break; }
-                    if (old == key) break;                  // another prompt of this round added that child
+                    if (old == key) { retry = true; break; }   // another prompt of this round added that child
                     sl2 = (sl2 + 1) & T.table_mask;
                 }
                 if (won >= 0) {
@@ -1999,6 +2000,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                     }
                 }
             }
+            if (retry) A.pend_next[atomicAdd(A.n_next, 1u)] = i;
         }
         dst = __shfl_sync(FULL_MASK, dst, 0);
         if (dst >= 0)
@@ -2208,7 +2210,7 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
             (st = dalloc(&t->bulk_pnode, n)) || (st = dalloc(&t->bulk_poff, n))) return st;
         t->bulk_cap = n;
     }
-    if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 1))) return st;
+    if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 2))) return st;      // walk's and apply's list lengths
     int32_t *pend_a = t->bulk_pend_a, *pend_b = t->bulk_pend_b, *pm = t->bulk_pm, *pnode = t->bulk_pnode, *poff = t->bulk_poff;
     unsigned int* n_out = t->bulk_n_out;
     // claim words start idle (an earlier call that ran out of capacity may have left some set)
@@ -2221,18 +2223,18 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         if (++rounds > 1000000) { st = RT_ERR_LIMIT; break; }
         BulkArgs a;
         a.tok = d_tokens; a.off = d_offsets; a.pend_in = pend_a; a.pend_out = pend_b; a.n_out = n_out;
+        a.pend_next = pend_a; a.n_next = n_out + 1;          // the walk has consumed pend_a by the time apply refills it
         a.claim = t->claim; a.pm = pm; a.pnode = pnode; a.poff = poff;
         long long blocks = ((long long)count + 7) / 8;
         if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
-        e = cudaMemsetAsync(n_out, 0, sizeof(unsigned), s);
+        e = cudaMemsetAsync(n_out, 0, 2 * sizeof(unsigned), s);
         if (e != cudaSuccess) break;
         bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
         bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
         e = cudaGetLastError();
         if (e != cudaSuccess) break;
-        e = cudaMemcpyAsync(&count, n_out, sizeof(unsigned), cudaMemcpyDeviceToHost, s);
+        e = cudaMemcpyAsync(&count, n_out + 1, sizeof(unsigned), cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-        int32_t* tmp = pend_a; pend_a = pend_b; pend_b = tmp;
         if (e == cudaSuccess && count > 0) {
             TreeState h;
             e = cudaMemcpy(&h, t->dev.st, sizeof(h), cudaMemcpyDeviceToHost);
