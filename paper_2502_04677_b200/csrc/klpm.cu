@@ -794,7 +794,9 @@ select_static_kernel(const int32_t* __restrict__ mlen, const int64_t* __restrict
 }
 
 // ------------------------------------------------------------------------------------------------
-// klpm_run: the whole loop as one cooperative kernel
+// klpm_run, one decision at a time on the tree itself: the whole loop as one cooperative kernel.
+// Trees with a budget take this loop (eviction can shorten matches, so match lengths are kept against
+// the tree as it changes); trees without one take the grouped loop further down.
 //
 // Slots are the queries ordered by (arrival, index).  Per decision c:
 //   phase A (every CTA): bring the match state of the waiting slots up to date -- walk newly arrived
