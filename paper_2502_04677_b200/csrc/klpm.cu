@@ -1592,9 +1592,7 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
     __syncthreads();
 }
 
-// Run-ahead mode of the sequencer: a pick whose state has not been read yet, and a leaf block whose keys have
-// been requested to find its second largest again.
-struct FastFlight { int32_t c; int32_t m; int4 s0; bool valid; };     // s0 = arrival, length, query index
+// Run-ahead mode of the sequencer: a leaf block whose keys have been requested to find its second largest again.
 struct FastRefresh { int32_t b; unsigned long long k; bool valid; };
 
 __global__ void __launch_bounds__(KLPM_FAST_THREADS, 1)
@@ -1659,24 +1657,21 @@ fast_run_kernel(FastArgs A) {
         }
         if (head > n) head = n;
     };
-    // Definition 2 for one pick whose state has arrived; the outputs.  Every lane performs the same stores.
-    auto retire = [&](const FastFlight& F) {
-        const int32_t len = F.s0.z, ord = F.s0.w, unc = len - F.m;
-        const long long t = (long long)(((unsigned long long)(unsigned)F.s0.y << 32) | (unsigned)F.s0.x);
-        const long long begin = now > t ? now : t;
-        const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
-        now = Rj;
-        vnext += unc;
-        A.order[F.c] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - t;
-        if (A.completion) A.completion[ord] = Rj;
-    };
     // The keys of leaf block G.b have arrived: its two largest among the unprocessed slots, as of now.
-    auto refresh_done = [&](const FastRefresh& G) {
+    auto refresh_full = [&](const FastRefresh& G) {
         const unsigned dw = s_done[G.b];
         unsigned long long top1, top2;
         warp_top2(((dw >> lane) & 1u) ? 0ULL : G.k, &top1, &top2);
         R.t1s[G.b] = top2;
         if (R.t1[G.b] != top1) root = tour_set(R, G.b, top1, lane);
+    };
+    // The same when the block's largest key is known to be right: only the second largest is computed.
+    auto refresh_second = [&](const FastRefresh& G) {
+        const unsigned dw = s_done[G.b];
+        const unsigned long long best = R.t1[G.b];
+        const int bl = (int)((0xffffffffu - (unsigned)best) & 31u);       // lane of the slot that holds `best`
+        const bool out = ((dw >> lane) & 1u) || (best != 0ULL && lane == bl);
+        R.t1s[G.b] = warp_max64r(out ? 0ULL : G.k);
     };
 
     while (c < n) {
@@ -1687,16 +1682,43 @@ fast_run_kernel(FastArgs A) {
         // second largest has to be found again.  A pick whose group has other members ends the burst: the
         // picks in flight are finished in order and the careful step below takes that pick.
         if (A.run_ahead && admitted == n) {
-            FastFlight F[4];
+            // Picks are charged 32 at a time.  Everybody has arrived, so a pick never waits for its query:
+            // completion times are a running sum of the picks' costs (Definition 2 with R_prev >= t_j).  Pick
+            // number p of the burst belongs to lane p mod 32, which requests the pick's state at once, into
+            // register set p mod 4 (a set is written again only four picks later, when its load has landed).
             FastRefresh G[4];
+            int4 fs[4];                                     // arrival, length, query index of this lane's pick
+            int32_t fm[4];                                  // its match length
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { F[u].valid = false; G[u].valid = false; }
+            for (int u = 0; u < 4; ++u) { G[u].valid = false; fs[u] = make_int4(0, 0, 0, 0); fm[u] = 0; }
+            int32_t p = 0;
+            auto retire_batch = [&](int32_t cnt) {          // lanes below cnt hold picks c - cnt + lane
+                const int set = lane & 3;
+                const int4 s = set == 0 ? fs[0] : set == 1 ? fs[1] : set == 2 ? fs[2] : fs[3];
+                const int32_t m = set == 0 ? fm[0] : set == 1 ? fm[1] : set == 2 ? fm[2] : fm[3];
+                const bool v = lane < cnt;
+                const int32_t len = s.z, ord = s.w, unc = v ? len - m : 0;
+                const long long tj = (long long)(((unsigned long long)(unsigned)s.y << 32) | (unsigned)s.x);
+                long long x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
+                long long y = unc;
+#pragma unroll
+                for (int dlt = 1; dlt < 32; dlt <<= 1) {
+                    const long long xo = __shfl_up_sync(FULL_MASK, x, dlt), yo = __shfl_up_sync(FULL_MASK, y, dlt);
+                    if (lane >= dlt) { x += xo; y += yo; }
+                }
+                const long long Rj = now + x;
+                if (v) {
+                    A.order[c - cnt + lane] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - tj;
+                    if (A.completion) A.completion[ord] = Rj;
+                }
+                now += __shfl_sync(FULL_MASK, x, 31);
+                vnext += __shfl_sync(FULL_MASK, y, 31);
+            };
             bool stop = false, draining = false;
             for (;;) {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    if (F[u].valid) { retire(F[u]); F[u].valid = false; }
-                    if (G[u].valid) { refresh_done(G[u]); G[u].valid = false; }
+                    if (G[u].valid) { refresh_second(G[u]); G[u].valid = false; }
                     if (stop) continue;
                     if (c >= n) { stop = true; continue; }
                     const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
@@ -1705,10 +1727,11 @@ fast_run_kernel(FastArgs A) {
                     if ((R.gb[j >> 5] >> (j & 31)) & 1u) { stop = true; continue; }
                     // the pick is made
                     if (++cyc == A.k) cyc = 0;
-                    F[u].c = c; F[u].valid = true;
-                    F[u].m = __ldcg(&A.dyn[j].m);
-                    F[u].s0 = __ldg(reinterpret_cast<const int4*>(A.stat + j));
-                    ++c;
+                    if (lane == (p & 31)) {
+                        fs[u] = __ldg(reinterpret_cast<const int4*>(A.stat + j));
+                        fm[u] = __ldcg(&A.dyn[j].m);
+                    }
+                    ++p; ++c;
                     const int32_t b = j >> 5;
                     s_done[b] |= 1u << (j & 31);
                     const unsigned want = 0xffffffffu - (unsigned)j;          // low half of j's key
@@ -1722,13 +1745,13 @@ fast_run_kernel(FastArgs A) {
                         } else {
                             // the second largest is not known: take what is in flight, then read the block if need be
 #pragma unroll
-                            for (int v = 0; v < 4; ++v) if (G[v].valid) { refresh_done(G[v]); G[v].valid = false; }
+                            for (int v = 0; v < 4; ++v) if (G[v].valid) { refresh_full(G[v]); G[v].valid = false; }
                             if ((unsigned)R.t1[b] == want) {
                                 FastRefresh Q;
                                 Q.b = b; Q.valid = true;
                                 const long long r = ((long long)b << 5) + lane;
                                 Q.k = r < n ? __ldcg(A.key + r) : 0ULL;
-                                refresh_done(Q);
+                                refresh_full(Q);
                             }
                         }
                     } else if (sec != KLPM_FAST_PENDING && (unsigned)sec == want) {
@@ -1741,12 +1764,14 @@ fast_run_kernel(FastArgs A) {
                         G[u].k = r < n ? __ldcg(A.key + r) : 0ULL;
                     }
                     if (j == head) advance_head();
+                    if ((p & 31) == 0) retire_batch(32);
                 }
                 if (stop) {
                     if (draining) break;
                     draining = true;
                 }
             }
+            if (p & 31) retire_batch(p & 31);
             __syncwarp();
             if (c >= n) break;
         }
