@@ -1262,14 +1262,16 @@ struct FastArgs {
     int32_t lb_shift;             // log2 of the number of slots per tournament leaf block
     int32_t nb;                   // number of leaf blocks
     int32_t done_in_smem;
-    int32_t run_ahead;            // the run-ahead mode of the loop can be used (32-slot leaf blocks, keys end in ~slot)
+    int32_t run_ahead;            // the list mode of the loop can be used (32-slot leaf blocks, all bitmaps in shared memory)
     unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts
+    const long long* lk;          // list mode: every slot's key, largest first, stored as ~key with the top bit flipped
+    const int32_t* ls;            //            and the slot it belongs to
     unsigned long long* counter;  // work counter of the initial walk
     TreeState* st;
 };
 
 #define KLPM_FAST_THREADS 256
-#define KLPM_FAST_SORT_CAP 2048          // largest group that is regrouped exactly (sorted in shared memory)
+#define KLPM_FAST_SORT_CAP 4096          // largest group that is regrouped exactly (sorted in shared memory)
 #define KLPM_FAST_NOGROUP 0xffffffffffffffffULL
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {      // SplitMix64's finaliser
@@ -1374,6 +1376,14 @@ __global__ void fast_group_kernel(FastArgs A) {
     if (lo - first > 1) atomicOr(A.gbits + (r >> 5), 1u << (r & 31));
 }
 
+// list mode: every slot's key in a form that sorts largest first (padding last)
+__global__ void fast_list_kernel(const unsigned long long* __restrict__ key, int32_t n, long long np2, long long* lk, int32_t* ls) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= np2) return;
+    lk[i] = i < n ? (long long)(~key[i] ^ 0x8000000000000000ULL) : 0x7fffffffffffffffLL;
+    ls[i] = i < n ? (int32_t)i : 0x7fffffff;
+}
+
 // Largest of the warp's 64-bit values with two hardware reductions: the high halves, then the low halves of
 // the lanes that hold the largest high half.
 __device__ __forceinline__ unsigned long long warp_max64r(unsigned long long v) {
@@ -1384,15 +1394,15 @@ __device__ __forceinline__ unsigned long long warp_max64r(unsigned long long v) 
 }
 
 // ---- the tournament above the leaf blocks (shared memory) ----
-// t1[b] is the largest key of leaf block b among arrived, unprocessed slots; t1s[b] is the second largest, or
-// KLPM_FAST_PENDING when it is not known (whoever needs it then reads the block's keys).
-#define KLPM_FAST_PENDING 0xffffffffffffffffULL
+// t1[b] is the largest key of leaf block b among the slots the tournament holds: the arrived, unprocessed slots
+// while arrivals are pending; in list mode (everybody has arrived) only those of them whose key has changed since
+// the keys were sorted -- the others are picked from the sorted list.
 struct FastTour {
     unsigned long long* t1;   // per leaf block (padded with zeros to a multiple of 32)
-    unsigned long long* t1s;  // second largest key per leaf block, or KLPM_FAST_PENDING
     unsigned long long* t2;   // per 32 leaf blocks (padded likewise)
     unsigned long long* t3;   // 32 entries
     unsigned int* done;       // bitmap of processed slots (shared memory), or null
+    unsigned int* skip;       // bitmap of slots the sorted list must pass over: processed, or key changed (shared memory), or null
     unsigned int* gb;         // bitmap of slots whose group has more than one member (shared memory), or null
     int32_t n2;               // entries of t2 in use
     int32_t n3;               // entries of t3 in use
@@ -1436,12 +1446,6 @@ __device__ __forceinline__ void tour_mid(const FastTour& R, int warp, int nwarps
         if (lane == 0) R.t2[i2] = v;
     }
 }
-// The two largest of the warp's keys (keys are distinct unless zero).
-__device__ __forceinline__ void warp_top2(unsigned long long k, unsigned long long* top1, unsigned long long* top2) {
-    const unsigned long long a = warp_max64r(k);
-    *top1 = a;
-    *top2 = warp_max64r(k == a ? 0ULL : k);
-}
 // has slot r been processed?  (the bitmap lives in shared memory when it fits)
 __device__ __forceinline__ bool slot_done(const FastTour& R, const FastArgs& A, long long r) {
     const unsigned w = R.done ? R.done[r >> 5] : __ldcg(A.done + (r >> 5));
@@ -1462,7 +1466,7 @@ struct FastPick {             // the prompt being processed, as its group's memb
     int32_t gstart, gcount;
 };
 struct FastJob { int32_t type; int32_t a0, a1; FastPick pick; };
-enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2 };
+enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2, FAST_JOB_REBUILD = 3 };
 
 // One member of the dissolving group per lane (r < 0: none).  Members tied with the processed prompt are
 // compared with its uncached tokens and get their new state and key; every live member gets the hash of the
@@ -1493,11 +1497,8 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
         st_dyn_state(A.dyn + r, d.pos, d.m, d.ntok);
         const unsigned long long key = fast_key(d.m, s.len, s.rank, A.score_mode);
         __stcg(A.key + r, key);
-        if ((long long)r < P.admitted) {
-            atomicMax(R.t1 + (r >> A.lb_shift), key);
-            R.t1s[r >> A.lb_shift] = KLPM_FAST_PENDING;
-            *touched = true;
-        }
+        if (R.skip) atomicOr(R.skip + (r >> 5), 1u << (r & 31));          // its entry of the sorted list is stale now
+        if ((long long)r < P.admitted) { atomicMax(R.t1 + (r >> A.lb_shift), key); *touched = true; }
     }
     if (!live) return KLPM_FAST_NOGROUP;
     return d.m < s.len ? group_hash(d.pos, d.ntok) : single_hash(r);
@@ -1508,21 +1509,25 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int tid = threadIdx.x, nthr = blockDim.x;
     if (J.type == FAST_JOB_ADMIT) {
-        // slots [a0, a1) have arrived: the two largest keys of every leaf block they fall into
+        // slots [a0, a1) have arrived: the largest key of every leaf block they fall into
         const int32_t b0 = J.a0 >> A.lb_shift, b1 = (J.a1 - 1) >> A.lb_shift;
         const int32_t LB = 1 << A.lb_shift;
         for (int32_t b = b0 + warp; b <= b1; b += nwarps) {
-            unsigned long long v1 = 0, v2 = 0;              // this lane's two largest
+            unsigned long long v = 0;
             for (int32_t u = lane; u < LB; u += 32) {
                 const long long r = ((long long)b << A.lb_shift) + u;
-                if (r < J.a1 && !slot_done(R, A, r)) {
-                    const unsigned long long kk = __ldcg(A.key + r);
-                    if (kk > v1) { v2 = v1; v1 = kk; } else if (kk > v2) v2 = kk;
-                }
+                if (r < J.a1 && !slot_done(R, A, r)) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
             }
-            const unsigned long long top1 = warp_max64r(v1);
-            const unsigned long long top2 = warp_max64r(v1 == top1 ? v2 : v1);
-            if (lane == 0) { R.t1[b] = top1; R.t1s[b] = top2; }
+            v = warp_max64r(v);
+            if (lane == 0) R.t1[b] = v;
+        }
+    } else if (J.type == FAST_JOB_REBUILD) {
+        // entering list mode (32-slot leaf blocks): the tournament keeps only the unprocessed slots whose key has changed
+        for (int32_t b = warp; b < A.nb; b += nwarps) {
+            const unsigned w = R.skip[b] & ~R.done[b];
+            unsigned long long v = 0;
+            if (w) v = warp_max64r(((w >> lane) & 1u) ? __ldcg(A.key + ((long long)b << 5) + lane) : 0ULL);
+            if (lane == 0) R.t1[b] = v;
         }
     } else {
         // dissolve a group of more than 32 members
@@ -1592,32 +1597,37 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
     __syncthreads();
 }
 
-// Run-ahead mode of the sequencer: a leaf block whose keys have been requested to find its second largest again.
-struct FastRefresh { int32_t b; unsigned long long k; bool valid; };
-
+// The loop.  While arrivals are pending every decision is one careful step: admit who has arrived, pick from the
+// tournament over all arrived slots (or the oldest slot), take the pick out of its leaf block, charge it and
+// dissolve its group.  Once everybody has arrived the time of a pick no longer decides who can be picked, and the
+// loop changes to list mode: all keys were sorted before the loop, so the longest-match pick is the next entry of
+// that list that is still unprocessed and whose key has not changed since; the tournament is cut down to the slots
+// whose key has changed (members of dissolved groups) and the pick is the larger of the two candidates.  A pick
+// from the list touches no tournament at all.  Picks whose group has no other member are charged 32 at a time.
 __global__ void __launch_bounds__(KLPM_FAST_THREADS, 1)
 fast_run_kernel(FastArgs A) {
     extern __shared__ __align__(16) unsigned char fast_smem[];
     __shared__ FastJob s_job;
     __shared__ int s_cnt;
+    __shared__ int32_t s_H[32], s_E[32];      // a batch's oldest-first and longest-match picks, by rank
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t n = A.n;
     const int32_t nb1p = (A.nb + 31) & ~31, n2 = nb1p >> 5, n2p = (n2 + 31) & ~31, n3 = n2p >> 5;
     const int32_t nwords = (n + 31) >> 5;
     FastTour R;
     R.t1 = reinterpret_cast<unsigned long long*>(fast_smem);
-    R.t1s = R.t1 + nb1p;
-    R.t2 = R.t1s + nb1p;
+    R.t2 = R.t1 + nb1p;
     R.t3 = R.t2 + n2p;
     R.n2 = n2; R.n3 = n3;
     unsigned long long* sh = R.t3 + 32;
     int32_t* sr = reinterpret_cast<int32_t*>(sh + KLPM_FAST_SORT_CAP);
     unsigned int* s_done = reinterpret_cast<unsigned int*>(sr + KLPM_FAST_SORT_CAP);
     R.done = A.done_in_smem ? s_done : nullptr;
-    R.gb = A.run_ahead ? s_done + nwords : nullptr;
-    for (int32_t i = threadIdx.x; i < 2 * nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
+    R.skip = A.run_ahead ? s_done + nwords : nullptr;
+    R.gb = A.run_ahead ? s_done + 2 * nwords : nullptr;
+    for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
     if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
-    if (A.run_ahead) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) R.gb[i] = __ldcg(A.gbits + i);
+    if (A.run_ahead) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
     __syncthreads();
 
     if (warp != 0) {
@@ -1637,9 +1647,11 @@ fast_run_kernel(FastArgs A) {
     unsigned long long root = 0;
     int32_t cyc = 0;                                        // c mod k
     int32_t c = 0;
+    bool failed = false;
 
     // first unprocessed slot at or after `head` (which is processed)
     auto advance_head = [&]() {
+        if (A.done_in_smem && head + 1 < n && !((s_done[(head + 1) >> 5] >> ((head + 1) & 31)) & 1u)) { ++head; return; }   // the usual case
         int32_t w0 = head >> 5;
         for (;;) {
             const int32_t wi = w0 + lane;
@@ -1657,213 +1669,29 @@ fast_run_kernel(FastArgs A) {
         }
         if (head > n) head = n;
     };
-    // The keys of leaf block G.b have arrived: its two largest among the unprocessed slots, as of now.
-    auto refresh_full = [&](const FastRefresh& G) {
-        const unsigned dw = s_done[G.b];
-        unsigned long long top1, top2;
-        warp_top2(((dw >> lane) & 1u) ? 0ULL : G.k, &top1, &top2);
-        R.t1s[G.b] = top2;
-        if (R.t1[G.b] != top1) root = tour_set(R, G.b, top1, lane);
+    // slot j is processed from now on (every lane performs the same shared-memory stores)
+    auto mark_done = [&](int32_t j) {
+        if (A.done_in_smem) s_done[j >> 5] |= 1u << (j & 31);
+        else if (lane == 0) __stcg(A.done + (j >> 5), __ldcg(A.done + (j >> 5)) | (1u << (j & 31)));
+        if (R.skip) R.skip[j >> 5] |= 1u << (j & 31);
+        __syncwarp();
     };
-    // The same when the block's largest key is known to be right: only the second largest is computed.
-    auto refresh_second = [&](const FastRefresh& G) {
-        const unsigned dw = s_done[G.b];
-        const unsigned long long best = R.t1[G.b];
-        const int bl = (int)((0xffffffffu - (unsigned)best) & 31u);       // lane of the slot that holds `best`
-        const bool out = ((dw >> lane) & 1u) || (best != 0ULL && lane == bl);
-        R.t1s[G.b] = warp_max64r(out ? 0ULL : G.k);
-    };
-
-    while (c < n) {
-        // ================================================================ run-ahead
-        // Everybody has arrived, so the time of a pick no longer decides who can be picked: picks are made from
-        // shared memory alone (the block's second largest key takes over when its largest is picked), each
-        // pick's state is requested at once and used four picks later, and so are the keys of blocks whose
-        // second largest has to be found again.  A pick whose group has other members ends the burst: the
-        // picks in flight are finished in order and the careful step below takes that pick.
-        if (A.run_ahead && admitted == n) {
-            // Picks are charged 32 at a time.  Everybody has arrived, so a pick never waits for its query:
-            // completion times are a running sum of the picks' costs (Definition 2 with R_prev >= t_j).  Pick
-            // number p of the burst belongs to lane p mod 32, which requests the pick's state at once, into
-            // register set p mod 4 (a set is written again only four picks later, when its load has landed).
-            FastRefresh G[4];
-            int4 fs[4];                                     // arrival, length, query index of this lane's pick
-            int32_t fm[4];                                  // its match length
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { G[u].valid = false; fs[u] = make_int4(0, 0, 0, 0); fm[u] = 0; }
-            int32_t p = 0;
-            auto retire_batch = [&](int32_t cnt) {          // lanes below cnt hold picks c - cnt + lane
-                const int set = lane & 3;
-                const int4 s = set == 0 ? fs[0] : set == 1 ? fs[1] : set == 2 ? fs[2] : fs[3];
-                const int32_t m = set == 0 ? fm[0] : set == 1 ? fm[1] : set == 2 ? fm[2] : fm[3];
-                const bool v = lane < cnt;
-                const int32_t len = s.z, ord = s.w, unc = v ? len - m : 0;
-                const long long tj = (long long)(((unsigned long long)(unsigned)s.y << 32) | (unsigned)s.x);
-                long long x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
-                long long y = unc;
-#pragma unroll
-                for (int dlt = 1; dlt < 32; dlt <<= 1) {
-                    const long long xo = __shfl_up_sync(FULL_MASK, x, dlt), yo = __shfl_up_sync(FULL_MASK, y, dlt);
-                    if (lane >= dlt) { x += xo; y += yo; }
-                }
-                const long long Rj = now + x;
-                if (v) {
-                    A.order[c - cnt + lane] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - tj;
-                    if (A.completion) A.completion[ord] = Rj;
-                }
-                now += __shfl_sync(FULL_MASK, x, 31);
-                vnext += __shfl_sync(FULL_MASK, y, 31);
-            };
-            bool stop = false, draining = false;
-            for (;;) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (G[u].valid) { refresh_second(G[u]); G[u].valid = false; }
-                    if (stop) continue;
-                    if (c >= n) { stop = true; continue; }
-                    const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
-                    const int32_t j = fcfs_turn ? head : (int32_t)(0xffffffffu - (unsigned)(root & 0xffffffffULL));
-                    if (j < 0 || j >= n) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 107); stop = true; c = n; continue; }   // cannot happen
-                    if ((R.gb[j >> 5] >> (j & 31)) & 1u) { stop = true; continue; }
-                    // the pick is made
-                    if (++cyc == A.k) cyc = 0;
-                    if (lane == (p & 31)) {
-                        fs[u] = __ldg(reinterpret_cast<const int4*>(A.stat + j));
-                        fm[u] = __ldcg(&A.dyn[j].m);
-                    }
-                    ++p; ++c;
-                    const int32_t b = j >> 5;
-                    s_done[b] |= 1u << (j & 31);
-                    const unsigned want = 0xffffffffu - (unsigned)j;          // low half of j's key
-                    const unsigned long long best = R.t1[b], sec = R.t1s[b];
-                    bool ask = false;
-                    if ((unsigned)best == want) {                              // j was its block's largest
-                        if (sec != KLPM_FAST_PENDING) {
-                            root = tour_set(R, b, sec, lane);
-                            R.t1s[b] = KLPM_FAST_PENDING;
-                            ask = true;
-                        } else {
-                            // the second largest is not known: take what is in flight, then read the block if need be
-#pragma unroll
-                            for (int v = 0; v < 4; ++v) if (G[v].valid) { refresh_full(G[v]); G[v].valid = false; }
-                            if ((unsigned)R.t1[b] == want) {
-                                FastRefresh Q;
-                                Q.b = b; Q.valid = true;
-                                const long long r = ((long long)b << 5) + lane;
-                                Q.k = r < n ? __ldcg(A.key + r) : 0ULL;
-                                refresh_full(Q);
-                            }
-                        }
-                    } else if (sec != KLPM_FAST_PENDING && (unsigned)sec == want) {
-                        R.t1s[b] = KLPM_FAST_PENDING;
-                        ask = true;
-                    }
-                    if (ask) {
-                        const long long r = ((long long)b << 5) + lane;
-                        G[u].b = b; G[u].valid = true;
-                        G[u].k = r < n ? __ldcg(A.key + r) : 0ULL;
-                    }
-                    if (j == head) advance_head();
-                    if ((p & 31) == 0) retire_batch(32);
-                }
-                if (stop) {
-                    if (draining) break;
-                    draining = true;
-                }
-            }
-            if (p & 31) retire_batch(p & 31);
-            __syncwarp();
-            if (c >= n) break;
-        }
-
-        // ================================================================ one careful step
-        // ---- time and arrivals: idle until somebody has arrived, then admit everybody who has
-        if (head == admitted && next_t > now) now = next_t;
-        if (next_t <= now) {
-            int32_t a1 = admitted;
-            {
-                const long long r = (long long)a1 + lane;
-                const bool in = r < n && __ldg(&A.stat[r].t) <= now;
-                const unsigned bal = __ballot_sync(FULL_MASK, in);
-                const int cnt = bal == FULL_MASK ? 32 : __ffs(~bal) - 1;
-                a1 += cnt;
-                if (cnt == 32 && a1 < n) {                 // a full window: gallop, then bisect (lane 0)
-                    long long lo = a1, hi = n;
-                    if (lane == 0 && __ldg(&A.stat[lo].t) <= now) {
-                        long long step = 1;
-                        ++lo;
-                        while (lo + step <= hi && __ldg(&A.stat[lo + step - 1].t) <= now) { lo += step; step <<= 1; }
-                        if (lo + step < hi) hi = lo + step;
-                        while (lo < hi) { const long long mid = (lo + hi) >> 1; if (__ldg(&A.stat[mid].t) <= now) lo = mid + 1; else hi = mid; }
-                    }
-                    a1 = (int32_t)__shfl_sync(FULL_MASK, lo, 0);
-                }
-            }
-            if (a1 - admitted <= 32) {
-                const int32_t r = admitted + lane;
-                if (r < a1) { atomicMax(R.t1 + (r >> A.lb_shift), __ldcg(A.key + r)); R.t1s[r >> A.lb_shift] = KLPM_FAST_PENDING; }
-                __syncwarp();
-                root = tour_update(R, admitted >> A.lb_shift, lane);
-                if (((a1 - 1) >> A.lb_shift) != (admitted >> A.lb_shift)) root = tour_update(R, (a1 - 1) >> A.lb_shift, lane);
-            } else {
-                if (lane == 0) { s_job.type = FAST_JOB_ADMIT; s_job.a0 = admitted; s_job.a1 = a1; }
-                __syncwarp();
-                named_bar(1, KLPM_FAST_THREADS);
-                const FastJob J = s_job;
-                fast_job(A, R, J, sh, sr, &s_cnt);
-                root = tour_top(R, lane);
-            }
-            admitted = a1;
-            next_t = admitted < n ? __ldg(&A.stat[admitted].t) : INF;
-        }
-        // ---- pick
-        const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
-        if (++cyc == A.k) cyc = 0;
-        int32_t slot = head;
-        if (!fcfs_turn) {
-            const unsigned rk = 0xffffffffu - (unsigned)(root & 0xffffffffULL);
-            slot = A.pinv ? __ldg(A.pinv + rk) : (int32_t)rk;
-        }
-        if (slot < 0 || slot >= admitted) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 105); break; }   // cannot happen
+    // Charge pick `slot` (Definition 2), write its outputs, and let the queries tied with it match into its new
+    // leaf.  The caller has taken the slot out of the tournament or the list and marked it processed.
+    auto careful = [&](int32_t slot) {
         const FDyn d = ld_dyn(A.dyn + slot);
         const FStat s = ld_stat(A.stat + slot);
-        const int32_t b = slot >> A.lb_shift;
-        unsigned long long k1 = 0, k2 = 0;                  // this lane's two largest keys of the pick's leaf block, the pick left out
-        for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
-            const long long r = ((long long)b << A.lb_shift) + u;
-            if (r < admitted && r != slot && !slot_done(R, A, r)) {
-                const unsigned long long kk = __ldcg(A.key + r);
-                if (kk > k1) { k2 = k1; k1 = kk; } else if (kk > k2) k2 = kk;
-            }
-        }
-        // while those loads are in flight: the tournament without the pick's own ancestors
-        const int32_t i2 = b >> 5, i3 = i2 >> 5;
-        const unsigned long long o1 = warp_max64r(lane == (b & 31) ? 0ULL : R.t1[(i2 << 5) + lane]);
-        const unsigned long long o2 = warp_max64r(lane == (i2 & 31) ? 0ULL : R.t2[(i3 << 5) + lane]);
-        const unsigned long long o3 = warp_max64r(lane == i3 ? 0ULL : R.t3[lane]);
-        const unsigned long long bm = warp_max64r(k1);
-        const unsigned long long bs = warp_max64r(k1 == bm ? k2 : k1);
-        const unsigned long long v2 = bm > o1 ? bm : o1, v3 = v2 > o2 ? v2 : o2;
-        root = v3 > o3 ? v3 : o3;
-        // ---- charge (Definition 2)
         const int32_t m = d.m, len = s.len, unc = len - m;
-        if (slot_done(R, A, slot)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 106); break; }          // cannot happen
         const long long begin = now > s.t ? now : s.t;
         const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
         now = Rj;
         if (lane == 0) {
             A.order[c] = s.ord; A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
             if (A.completion) A.completion[s.ord] = Rj;
-            if (A.done_in_smem) s_done[slot >> 5] |= 1u << (slot & 31);
-            else __stcg(A.done + (slot >> 5), __ldcg(A.done + (slot >> 5)) | (1u << (slot & 31)));
-            R.t1[b] = bm; R.t1s[b] = bs; R.t2[i2] = v2; R.t3[i3] = v3;
         }
-        __syncwarp();
         const long long vleaf = vnext;
         vnext += unc;
         ++c;
-        // ---- the queries tied with the pick now match into its new leaf
-        bool full = false;
         if (unc > 0 && d.gcount > 1) {
             FastPick P;
             P.slot = slot; P.m = m; P.len = len; P.ntok = d.ntok; P.x = A.tok + s.soff; P.pos = d.pos; P.vleaf = vleaf;
@@ -1896,14 +1724,267 @@ fast_run_kernel(FastArgs A) {
                 named_bar(1, KLPM_FAST_THREADS);
                 const FastJob J = s_job;
                 fast_job(A, R, J, sh, sr, &s_cnt);
-                full = true;
+                root = tour_top(R, lane);
             }
         }
-        if (full) root = tour_top(R, lane);
-        // ---- the oldest unprocessed slot
+    };
+
+    // everybody is waiting as the loop starts: no arrival will ever have to be admitted
+    if (A.run_ahead && __ldg(&A.stat[n - 1].t) <= now) { admitted = n; next_t = INF; }
+
+    // ================================================================ arrivals pending: one careful step per decision
+    while (c < n && !failed && !(A.run_ahead && admitted == n)) {
+        // ---- time and arrivals: idle until somebody has arrived, then admit everybody who has
+        if (head == admitted && next_t > now) now = next_t;
+        if (next_t <= now) {
+            int32_t a1 = admitted;
+            {
+                const long long r = (long long)a1 + lane;
+                const bool in = r < n && __ldg(&A.stat[r].t) <= now;
+                const unsigned bal = __ballot_sync(FULL_MASK, in);
+                const int cnt = bal == FULL_MASK ? 32 : __ffs(~bal) - 1;
+                a1 += cnt;
+                if (cnt == 32 && a1 < n) {                 // a full window: gallop, then bisect (lane 0)
+                    long long lo = a1, hi = n;
+                    if (lane == 0 && __ldg(&A.stat[lo].t) <= now) {
+                        long long step = 1;
+                        ++lo;
+                        while (lo + step <= hi && __ldg(&A.stat[lo + step - 1].t) <= now) { lo += step; step <<= 1; }
+                        if (lo + step < hi) hi = lo + step;
+                        while (lo < hi) { const long long mid = (lo + hi) >> 1; if (__ldg(&A.stat[mid].t) <= now) lo = mid + 1; else hi = mid; }
+                    }
+                    a1 = (int32_t)__shfl_sync(FULL_MASK, lo, 0);
+                }
+            }
+            if (a1 - admitted <= 32) {
+                const int32_t r = admitted + lane;
+                if (r < a1) atomicMax(R.t1 + (r >> A.lb_shift), __ldcg(A.key + r));
+                __syncwarp();
+                root = tour_update(R, admitted >> A.lb_shift, lane);
+                if (((a1 - 1) >> A.lb_shift) != (admitted >> A.lb_shift)) root = tour_update(R, (a1 - 1) >> A.lb_shift, lane);
+            } else {
+                if (lane == 0) { s_job.type = FAST_JOB_ADMIT; s_job.a0 = admitted; s_job.a1 = a1; }
+                __syncwarp();
+                named_bar(1, KLPM_FAST_THREADS);
+                const FastJob J = s_job;
+                fast_job(A, R, J, sh, sr, &s_cnt);
+                root = tour_top(R, lane);
+            }
+            admitted = a1;
+            next_t = admitted < n ? __ldg(&A.stat[admitted].t) : INF;
+        }
+        // ---- pick
+        const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
+        if (++cyc == A.k) cyc = 0;
+        int32_t slot = head;
+        if (!fcfs_turn) {
+            const unsigned rk = 0xffffffffu - (unsigned)(root & 0xffffffffULL);
+            slot = A.pinv ? __ldg(A.pinv + rk) : (int32_t)rk;
+        }
+        if (slot < 0 || slot >= admitted || slot_done(R, A, slot)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 105); failed = true; break; }   // cannot happen
+        // ---- the pick leaves its leaf block
+        const int32_t b = slot >> A.lb_shift;
+        unsigned long long bm = 0;
+        for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
+            const long long r = ((long long)b << A.lb_shift) + u;
+            if (r < admitted && r != slot && !slot_done(R, A, r)) { const unsigned long long kk = __ldcg(A.key + r); if (kk > bm) bm = kk; }
+        }
+        root = tour_set(R, b, warp_max64r(bm), lane);
+        mark_done(slot);
+        careful(slot);
         if (slot == head) advance_head();
         __syncwarp();
     }
+
+    // ================================================================ list mode
+    if (c < n && !failed) {
+        if (lane == 0) s_job.type = FAST_JOB_REBUILD;
+        __syncwarp();
+        named_bar(1, KLPM_FAST_THREADS);
+        {
+            const FastJob J = s_job;
+            fast_job(A, R, J, sh, sr, &s_cnt);
+        }
+        root = tour_top(R, lane);
+        // the sorted list, 32 entries at a time: lane l holds entry (cur & ~31) + l, the next 32 are on their way
+        int32_t cur = 0;
+        auto window = [&](int32_t base, long long* wk_, int32_t* ws_) {
+            const long long i = (long long)base + lane;
+            *wk_ = i < n ? __ldg(A.lk + i) : INF;
+            *ws_ = i < n ? __ldg(A.ls + i) : -1;
+        };
+        long long wk, nk; int32_t ws, ns;
+        window(0, &wk, &ws);
+        window(32, &nk, &ns);
+        auto advance_cur = [&]() {
+            ++cur;
+            if ((cur & 31) == 0) { wk = nk; ws = ns; window(cur + 32, &nk, &ns); }
+        };
+        // Picks whose group has no other member are charged 32 at a time.  Nobody waits for an arrival any more, so
+        // completion times are a running sum of the picks' costs (Definition 2 with R_prev >= t_j).  The p-th pick
+        // of a batch is remembered by lane p; when the batch is full every lane reads its own pick's state, the
+        // warp takes a prefix sum of the costs and writes the outputs -- one memory latency per 32 picks.
+        int32_t p = 0, myj = 0;
+        auto retire_batch = [&]() {                         // lanes below p hold picks c - p + lane
+            const bool v = lane < p;
+            int4 s = make_int4(0, 0, 0, 0);
+            int32_t m = 0;
+            if (v) { s = __ldg(reinterpret_cast<const int4*>(A.stat + myj)); m = __ldcg(&A.dyn[myj].m); }
+            const int32_t len = s.z, ord = s.w, unc = len - m;
+            const long long tj = (long long)(((unsigned long long)(unsigned)s.y << 32) | (unsigned)s.x);
+            long long x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
+            long long y = unc;
+#pragma unroll
+            for (int dlt = 1; dlt < 32; dlt <<= 1) {
+                const long long xo = __shfl_up_sync(FULL_MASK, x, dlt), yo = __shfl_up_sync(FULL_MASK, y, dlt);
+                if (lane >= dlt) { x += xo; y += yo; }
+            }
+            const long long Rj = now + x;
+            if (v) {
+                A.order[c - p + lane] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - tj;
+                if (A.completion) A.completion[ord] = Rj;
+            }
+            now += __shfl_sync(FULL_MASK, x, 31);
+            vnext += __shfl_sync(FULL_MASK, y, 31);
+            p = 0;
+        };
+        // Up to 32 decisions at once.  As long as nothing interferes, the coming longest-match picks are the next
+        // entries of the list that still count and the coming oldest-first picks are the next unprocessed slots,
+        // interleaved as the policy says.  The warp gathers both sets side by side and checks that they cannot
+        // have influenced each other: no slot in both (a list entry inside the range of slots the oldest-first
+        // picks consume), none whose group has other members, none whose key sits in the tournament, and the
+        // tournament's root below the smallest key taken from the list.  Then lane i makes decision c + i.
+        // If any check fails nothing has been changed and the decisions are made one at a time below.
+        auto try_batch = [&]() -> bool {
+            const int32_t B = n - c < 32 ? n - c : 32;
+            auto f_before = [&](int32_t x) -> int32_t {     // oldest-first turns among the next x decisions
+                if (A.policy == KLPM_POLICY_FCFS) return x;
+                if (A.policy == KLPM_POLICY_LPM) return 0;
+                return (cyc + x + A.k - 1) / A.k - (cyc + A.k - 1) / A.k;
+            };
+            const int32_t nF = f_before(B), nL = B - nF;
+            bool bad = false;
+            int32_t hmax = -1;
+            if (nF > 0) {                                   // the next nF unprocessed slots
+                const int32_t w0 = head >> 5, wi = w0 + lane;
+                unsigned w = wi < nwords ? s_done[wi] : 0xffffffffu;
+                if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
+                if (wi == w0) w |= (1u << (head & 31)) - 1u;
+                const unsigned fr = ~w;
+                const int32_t cnt = __popc(fr);
+                int32_t inc = cnt;
+#pragma unroll
+                for (int dlt = 1; dlt < 32; dlt <<= 1) { const int32_t o = __shfl_up_sync(FULL_MASK, inc, dlt); if (lane >= dlt) inc += o; }
+                if (__shfl_sync(FULL_MASK, inc, 31) < nF) return false;
+                const int32_t pre = inc - cnt;
+                for (int32_t qk = pre; qk < pre + cnt && qk < nF; ++qk) s_H[qk] = wi * 32 + (int32_t)__fns(fr, 0, qk - pre + 1);
+                __syncwarp();
+                hmax = s_H[nF - 1];
+                if (lane < nF) {
+                    const int32_t hs = s_H[lane];
+                    if (((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u) bad = true;      // key in the tournament, or grouped
+                }
+            }
+            int32_t consumed = 0;
+            if (nL > 0) {                                   // the next nL list entries that still count
+                const int32_t off = (cur & 31) + lane;      // lane l looks at entry cur + l: in this window or the next
+                const long long k0 = __shfl_sync(FULL_MASK, wk, off & 31), k1 = __shfl_sync(FULL_MASK, nk, off & 31);
+                const int32_t s0 = __shfl_sync(FULL_MASK, ws, off & 31), s1 = __shfl_sync(FULL_MASK, ns, off & 31);
+                const long long kk = off < 32 ? k0 : k1;
+                const int32_t es = off < 32 ? s0 : s1;
+                const bool valid = (long long)cur + lane < n;
+                const bool ok = valid && !((R.skip[es >> 5] >> (es & 31)) & 1u);
+                const unsigned mask = __ballot_sync(FULL_MASK, ok);
+                if (__popc(mask) < nL) return false;
+                const int32_t rank = __popc(mask & ((1u << lane) - 1u));
+                const bool chosen = ok && rank < nL;
+                const int lastlane = (int)__fns(mask, 0, nL);
+                consumed = lastlane + 1;
+                if (chosen && (((R.gb[es >> 5] >> (es & 31)) & 1u) || (es >= head && es <= hmax))) bad = true;
+                const unsigned long long ek_last = ~((unsigned long long)__shfl_sync(FULL_MASK, kk, lastlane) ^ 0x8000000000000000ULL);
+                if (root > ek_last) bad = true;
+                if (chosen) s_E[rank] = es;
+            }
+            if (__ballot_sync(FULL_MASK, bad)) return false;
+            __syncwarp();
+            // commit: lane i makes decision c + i
+            if (lane < B) {
+                const int32_t f0 = f_before(lane);
+                myj = f_before(lane + 1) > f0 ? s_H[f0] : s_E[lane - f0];
+                atomicOr(s_done + (myj >> 5), 1u << (myj & 31));
+                atomicOr(R.skip + (myj >> 5), 1u << (myj & 31));
+            }
+            __syncwarp();
+            c += B; p = B;
+            if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + B) % A.k;
+            if (consumed) {
+                const int32_t ncur = cur + consumed;
+                if ((ncur >> 5) != (cur >> 5)) { wk = nk; ws = ns; window((ncur & ~31) + 32, &nk, &ns); }
+                cur = ncur;
+            }
+            if (nF > 0) { head = hmax; advance_head(); }
+            else if (head < n && ((s_done[head >> 5] >> (head & 31)) & 1u)) advance_head();
+            retire_batch();
+            return true;
+        };
+        int32_t vb_wait = 0, vb_back = 1;                   // decisions until the next attempt; doubles while attempts fail
+        while (c < n && !failed) {
+            if (vb_wait <= 0) {
+                if (p) retire_batch();
+                if (try_batch()) { vb_back = 1; continue; }
+                vb_wait = vb_back;
+                vb_back = vb_back < 64 ? vb_back * 2 : 64;
+            }
+            --vb_wait;
+            const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
+            if (++cyc == A.k) cyc = 0;
+            int32_t j;
+            bool in_tour;                                   // the pick's key is in the tournament (it changed after the sort)
+            if (fcfs_turn) {
+                j = head;
+                in_tour = (R.skip[j >> 5] >> (j & 31)) & 1u;
+            } else {
+                unsigned long long ek = 0;                  // next entry of the list that still counts
+                int32_t es = -1;
+                while (cur < n) {
+                    const int src = cur & 31;
+                    const long long kk = __shfl_sync(FULL_MASK, wk, src);
+                    es = __shfl_sync(FULL_MASK, ws, src);
+                    if (!((R.skip[es >> 5] >> (es & 31)) & 1u)) { ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL); break; }
+                    es = -1;
+                    advance_cur();
+                }
+                if (root > ek) {
+                    const unsigned rk = 0xffffffffu - (unsigned)(root & 0xffffffffULL);
+                    j = A.pinv ? __ldg(A.pinv + rk) : (int32_t)rk;
+                    in_tour = true;
+                } else {
+                    j = es;
+                    in_tour = false;
+                    advance_cur();
+                }
+            }
+            if (j < 0 || j >= n || ((s_done[j >> 5] >> (j & 31)) & 1u)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 107); failed = true; break; }   // cannot happen
+            mark_done(j);
+            if (in_tour) {                                  // its leaf block's largest changed key, without it
+                const int32_t b = j >> 5;
+                const unsigned w = R.skip[b] & ~s_done[b];
+                const unsigned long long kk = ((w >> lane) & 1u) ? __ldcg(A.key + ((long long)b << 5) + lane) : 0ULL;
+                root = tour_set(R, b, warp_max64r(kk), lane);
+            }
+            if (j == head) advance_head();
+            if ((R.gb[j >> 5] >> (j & 31)) & 1u) {
+                if (p) retire_batch();
+                careful(j);
+            } else {
+                if (lane == p) myj = j;
+                ++p; ++c;
+                if (p == 32) retire_batch();
+            }
+        }
+        if (p) retire_batch();
+    }
+    __syncwarp();
     if (lane == 0) s_job.type = FAST_JOB_EXIT;
     __syncwarp();
     named_bar(1, KLPM_FAST_THREADS);
@@ -2121,6 +2202,7 @@ struct rt_tree {
     long long fast_cap;     // slots allocated (power of two)
     FDyn* fast_dyn; FStat* fast_stat; unsigned long long* fast_key_arr; int32_t* fast_mem;
     long long* fast_gh; int32_t* fast_gidx; unsigned int* fast_done; unsigned long long* fast_counter;
+    long long* fast_lk; int32_t* fast_ls;
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -2160,6 +2242,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
+    cudaFree(t->fast_lk); cudaFree(t->fast_ls);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
     cudaFree(t->bulk_n_out);
@@ -2202,6 +2285,8 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if (np2 <= t->fast_cap) return RT_OK;
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
+    cudaFree(t->fast_lk); cudaFree(t->fast_ls);
+    t->fast_lk = nullptr; t->fast_ls = nullptr;
     t->fast_dyn = nullptr; t->fast_stat = nullptr; t->fast_key_arr = nullptr; t->fast_mem = nullptr;
     t->fast_gh = nullptr; t->fast_gidx = nullptr; t->fast_done = nullptr; t->fast_counter = nullptr;
     t->fast_cap = 0;
@@ -2214,6 +2299,8 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_gidx, np2))) return s;
     if ((s = dalloc(&t->fast_done, 2 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap
     if ((s = dalloc(&t->fast_counter, 1))) return s;
+    if ((s = dalloc(&t->fast_lk, np2))) return s;
+    if ((s = dalloc(&t->fast_ls, np2))) return s;
     t->fast_cap = np2;
     return RT_OK;
 }
@@ -2685,7 +2772,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         // Two environment variables shrink the limits so that small queues can exercise the large-queue layout:
         // KLPM_FAST_MAX_BLOCKS (leaf blocks) and KLPM_FAST_SMEM_KB (shared memory the loop may use).
         long long max_blocks = 8192;
-        size_t smem_max = 226 * 1024;
+        size_t smem_max = 224 * 1024;
         if (const char* e = getenv("KLPM_FAST_MAX_BLOCKS")) { const long long v = atoll(e); if (v >= 1 && v < max_blocks) max_blocks = v; }
         if (const char* e = getenv("KLPM_FAST_SMEM_KB")) { const long long v = atoll(e); if (v >= 1 && (size_t)v * 1024 < smem_max) smem_max = (size_t)v * 1024; }
         int lbs = 5;
@@ -2694,12 +2781,12 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.nb = (int32_t)(((long long)n + (1LL << lbs) - 1) >> lbs);
         const long long nb1p = (f.nb + 31) & ~31, n2p = ((nb1p >> 5) + 31) & ~31;
         const long long nwords = ((long long)n + 31) >> 5;
-        size_t smem = (size_t)(2 * nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
+        size_t smem = (size_t)(nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
         f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
-        // run-ahead needs both bitmaps in shared memory, 32-slot leaf blocks and keys whose low half names the slot
-        f.run_ahead = (f.done_in_smem && lbs == 5 && !d_tie_priority && smem + (size_t)nwords * 4 <= smem_max) ? 1 : 0;
-        if (f.run_ahead) smem += (size_t)nwords * 4;
+        // list mode needs two more bitmaps in shared memory and 32-slot leaf blocks
+        f.run_ahead = (f.done_in_smem && lbs == 5 && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
+        if (f.run_ahead) smem += (size_t)nwords * 8;
         f.gbits = tree->fast_done + (np2 / 32 + 32);
         const unsigned nblk = (unsigned)((n + 255) / 256), pblk = (unsigned)((np2 + 255) / 256);
         CK(cudaMemsetAsync(f.done, 0, (size_t)(2 * (np2 / 32 + 32)) * sizeof(unsigned int), s));
@@ -2708,6 +2795,13 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
             for (long long j = k >> 1; j > 0; j >>= 1)
                 bitonic_step_kernel<<<pblk, 256, 0, s>>>(f.gh, f.gidx, np2, k, j);
         fast_group_kernel<<<nblk, 256, 0, s>>>(f);
+        if (f.run_ahead) {           // all keys, largest first
+            f.lk = tree->fast_lk; f.ls = tree->fast_ls;
+            fast_list_kernel<<<pblk, 256, 0, s>>>(f.key, n, np2, tree->fast_lk, tree->fast_ls);
+            for (long long k = 2; k <= np2; k <<= 1)
+                for (long long j = k >> 1; j > 0; j >>= 1)
+                    bitonic_step_kernel<<<pblk, 256, 0, s>>>(tree->fast_lk, tree->fast_ls, np2, k, j);
+        }
         CK(cudaGetLastError());
         CK(cudaFuncSetAttribute(fast_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         fast_run_kernel<<<1, KLPM_FAST_THREADS, smem, s>>>(f);
