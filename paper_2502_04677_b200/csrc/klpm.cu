@@ -1451,6 +1451,16 @@ __device__ __forceinline__ bool slot_done(const FastTour& R, const FastArgs& A, 
     const unsigned w = R.done ? R.done[r >> 5] : __ldcg(A.done + (r >> 5));
     return (w >> (r & 31)) & 1u;
 }
+// position of the k-th set bit of w (k >= 1, at most the number of set bits)
+__device__ __forceinline__ int kth_set_bit(unsigned w, int k) {
+    int pos = 0;
+    int cnt = __popc(w & 0xffffu); if (k > cnt) { k -= cnt; pos += 16; w >>= 16; }
+    cnt = __popc(w & 0xffu);       if (k > cnt) { k -= cnt; pos += 8; w >>= 8; }
+    cnt = __popc(w & 0xfu);        if (k > cnt) { k -= cnt; pos += 4; w >>= 4; }
+    cnt = __popc(w & 0x3u);        if (k > cnt) { k -= cnt; pos += 2; w >>= 2; }
+    if (k > (int)(w & 1u)) pos += 1;
+    return pos;
+}
 __device__ __forceinline__ void set_grouped(const FastTour& R, int32_t r, bool grouped) {
     if (!R.gb) return;
     if (grouped) atomicOr(R.gb + (r >> 5), 1u << (r & 31));
@@ -1824,14 +1834,16 @@ fast_run_kernel(FastArgs A) {
         // completion times are a running sum of the picks' costs (Definition 2 with R_prev >= t_j).  The p-th pick
         // of a batch is remembered by lane p; when the batch is full every lane reads its own pick's state, the
         // warp takes a prefix sum of the costs and writes the outputs -- one memory latency per 32 picks.
+        // The state is requested when a batch closes and used when the next one closes (or when exact times are needed),
+        // so its latency hides behind the picks in between.
         int32_t p = 0, myj = 0;
-        auto retire_batch = [&]() {                         // lanes below p hold picks c - p + lane
-            const bool v = lane < p;
-            int4 s = make_int4(0, 0, 0, 0);
-            int32_t m = 0;
-            if (v) { s = __ldg(reinterpret_cast<const int4*>(A.stat + myj)); m = __ldcg(&A.dyn[myj].m); }
-            const int32_t len = s.z, ord = s.w, unc = len - m;
-            const long long tj = (long long)(((unsigned long long)(unsigned)s.y << 32) | (unsigned)s.x);
+        int4 ps = make_int4(0, 0, 0, 0);                    // the closed batch: this lane's pick's arrival, length, query index
+        int32_t pm = 0, pend_p = 0, pend_c0 = 0;            // its match length; picks in the closed batch; its first decision
+        auto finish = [&]() {                               // charge the closed batch
+            if (!pend_p) return;
+            const bool v = lane < pend_p;
+            const int32_t len = ps.z, ord = ps.w, unc = len - pm;
+            const long long tj = (long long)(((unsigned long long)(unsigned)ps.y << 32) | (unsigned)ps.x);
             long long x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
             long long y = unc;
 #pragma unroll
@@ -1841,11 +1853,20 @@ fast_run_kernel(FastArgs A) {
             }
             const long long Rj = now + x;
             if (v) {
-                A.order[c - p + lane] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - tj;
+                A.order[pend_c0 + lane] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - tj;
                 if (A.completion) A.completion[ord] = Rj;
             }
             now += __shfl_sync(FULL_MASK, x, 31);
             vnext += __shfl_sync(FULL_MASK, y, 31);
+            pend_p = 0;
+        };
+        auto retire_batch = [&]() {                         // close the open batch: lanes below p hold picks c - p + lane
+            finish();
+            const bool v = lane < p;
+            ps = make_int4(0, 0, 0, 0);
+            pm = 0;
+            if (v) { ps = __ldg(reinterpret_cast<const int4*>(A.stat + myj)); pm = __ldcg(&A.dyn[myj].m); }
+            pend_p = p; pend_c0 = c - p;
             p = 0;
         };
         // Up to 32 decisions at once.  As long as nothing interferes, the coming longest-match picks are the next
@@ -1856,12 +1877,26 @@ fast_run_kernel(FastArgs A) {
         // tournament's root below the smallest key taken from the list.  Then lane i makes decision c + i.
         // If any check fails nothing has been changed and the decisions are made one at a time below.
         auto try_batch = [&]() -> bool {
-            const int32_t B = n - c < 32 ? n - c : 32;
             auto f_before = [&](int32_t x) -> int32_t {     // oldest-first turns among the next x decisions
                 if (A.policy == KLPM_POLICY_FCFS) return x;
                 if (A.policy == KLPM_POLICY_LPM) return 0;
                 return (cyc + x + A.k - 1) / A.k - (cyc + A.k - 1) / A.k;
             };
+            // the list entries cur .. cur + 31 (in this window or the next) that still count
+            long long kk; int32_t es; unsigned mask;
+            {
+                const int32_t off = (cur & 31) + lane;
+                const long long k0 = __shfl_sync(FULL_MASK, wk, off & 31), k1 = __shfl_sync(FULL_MASK, nk, off & 31);
+                const int32_t s0 = __shfl_sync(FULL_MASK, ws, off & 31), s1 = __shfl_sync(FULL_MASK, ns, off & 31);
+                kk = off < 32 ? k0 : k1;
+                es = off < 32 ? s0 : s1;
+                const bool valid = (long long)cur + lane < n;
+                mask = __ballot_sync(FULL_MASK, valid && !((R.skip[es >> 5] >> (es & 31)) & 1u));
+            }
+            // as many decisions as those entries allow: lane x asks whether x + 1 decisions need no more of them
+            const int32_t avail = __popc(mask);
+            const int32_t B = __popc(__ballot_sync(FULL_MASK, c + lane < n && (lane + 1) - f_before(lane + 1) <= avail));
+            if (B < 4) return false;
             const int32_t nF = f_before(B), nL = B - nF;
             bool bad = false;
             int32_t hmax = -1;
@@ -1876,29 +1911,24 @@ fast_run_kernel(FastArgs A) {
 #pragma unroll
                 for (int dlt = 1; dlt < 32; dlt <<= 1) { const int32_t o = __shfl_up_sync(FULL_MASK, inc, dlt); if (lane >= dlt) inc += o; }
                 if (__shfl_sync(FULL_MASK, inc, 31) < nF) return false;
-                const int32_t pre = inc - cnt;
-                for (int32_t qk = pre; qk < pre + cnt && qk < nF; ++qk) s_H[qk] = wi * 32 + (int32_t)__fns(fr, 0, qk - pre + 1);
-                __syncwarp();
-                hmax = s_H[nF - 1];
-                if (lane < nF) {
-                    const int32_t hs = s_H[lane];
-                    if (((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u) bad = true;      // key in the tournament, or grouped
-                }
+                // lane q finds the q-th of them: the first word whose running count exceeds q, then the bit inside it
+                const int32_t qk = lane < nF ? lane : nF - 1;
+                int L = 0;
+#pragma unroll
+                for (int step = 16; step > 0; step >>= 1) if (__shfl_sync(FULL_MASK, inc, L + step - 1) <= qk) L += step;
+                const unsigned frL = __shfl_sync(FULL_MASK, fr, L);
+                const int32_t preL = __shfl_sync(FULL_MASK, inc - cnt, L);
+                const int32_t hs = (w0 + L) * 32 + kth_set_bit(frL, qk - preL + 1);
+                if (lane < nF) s_H[lane] = hs;
+                hmax = __shfl_sync(FULL_MASK, hs, nF - 1);
+                if (lane < nF && ((((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u))) bad = true;   // key in the tournament, or grouped
             }
             int32_t consumed = 0;
-            if (nL > 0) {                                   // the next nL list entries that still count
-                const int32_t off = (cur & 31) + lane;      // lane l looks at entry cur + l: in this window or the next
-                const long long k0 = __shfl_sync(FULL_MASK, wk, off & 31), k1 = __shfl_sync(FULL_MASK, nk, off & 31);
-                const int32_t s0 = __shfl_sync(FULL_MASK, ws, off & 31), s1 = __shfl_sync(FULL_MASK, ns, off & 31);
-                const long long kk = off < 32 ? k0 : k1;
-                const int32_t es = off < 32 ? s0 : s1;
-                const bool valid = (long long)cur + lane < n;
-                const bool ok = valid && !((R.skip[es >> 5] >> (es & 31)) & 1u);
-                const unsigned mask = __ballot_sync(FULL_MASK, ok);
-                if (__popc(mask) < nL) return false;
+            if (nL > 0) {
+                const bool ok = (mask >> lane) & 1u;
                 const int32_t rank = __popc(mask & ((1u << lane) - 1u));
                 const bool chosen = ok && rank < nL;
-                const int lastlane = (int)__fns(mask, 0, nL);
+                const int lastlane = kth_set_bit(mask, nL);
                 consumed = lastlane + 1;
                 if (chosen && (((R.gb[es >> 5] >> (es & 31)) & 1u) || (es >= head && es <= hmax))) bad = true;
                 const unsigned long long ek_last = ~((unsigned long long)__shfl_sync(FULL_MASK, kk, lastlane) ^ 0x8000000000000000ULL);
@@ -1975,6 +2005,7 @@ fast_run_kernel(FastArgs A) {
             if (j == head) advance_head();
             if ((R.gb[j >> 5] >> (j & 31)) & 1u) {
                 if (p) retire_batch();
+                finish();
                 careful(j);
             } else {
                 if (lane == p) myj = j;
@@ -1983,6 +2014,7 @@ fast_run_kernel(FastArgs A) {
             }
         }
         if (p) retire_batch();
+        finish();
     }
     __syncwarp();
     if (lane == 0) s_job.type = FAST_JOB_EXIT;
