@@ -1895,12 +1895,12 @@ fast_run_kernel(FastArgs A) {
             }
             // as many decisions as those entries allow: lane x asks whether x + 1 decisions need no more of them
             const int32_t avail = __popc(mask);
-            const int32_t B = __popc(__ballot_sync(FULL_MASK, c + lane < n && (lane + 1) - f_before(lane + 1) <= avail));
-            if (B < 4) return false;
-            const int32_t nF = f_before(B), nL = B - nF;
-            bool bad = false;
-            int32_t hmax = -1;
-            if (nF > 0) {                                   // the next nF unprocessed slots
+            const int32_t B0 = __popc(__ballot_sync(FULL_MASK, c + lane < n && (lane + 1) - f_before(lane + 1) <= avail));
+            if (B0 < 4) return false;
+            const int32_t nF0 = f_before(B0), nL0 = B0 - nF0;
+            // the next nF0 unprocessed slots; limF = how many of them can be taken before one needs the careful step
+            int32_t hs = -1, hmax0 = -1, limF = nF0;
+            if (nF0 > 0) {
                 const int32_t w0 = head >> 5, wi = w0 + lane;
                 unsigned w = wi < nwords ? s_done[wi] : 0xffffffffu;
                 if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
@@ -1910,32 +1910,42 @@ fast_run_kernel(FastArgs A) {
                 int32_t inc = cnt;
 #pragma unroll
                 for (int dlt = 1; dlt < 32; dlt <<= 1) { const int32_t o = __shfl_up_sync(FULL_MASK, inc, dlt); if (lane >= dlt) inc += o; }
-                if (__shfl_sync(FULL_MASK, inc, 31) < nF) return false;
+                if (__shfl_sync(FULL_MASK, inc, 31) < nF0) return false;
                 // lane q finds the q-th of them: the first word whose running count exceeds q, then the bit inside it
-                const int32_t qk = lane < nF ? lane : nF - 1;
+                const int32_t qk = lane < nF0 ? lane : nF0 - 1;
                 int L = 0;
 #pragma unroll
                 for (int step = 16; step > 0; step >>= 1) if (__shfl_sync(FULL_MASK, inc, L + step - 1) <= qk) L += step;
                 const unsigned frL = __shfl_sync(FULL_MASK, fr, L);
                 const int32_t preL = __shfl_sync(FULL_MASK, inc - cnt, L);
-                const int32_t hs = (w0 + L) * 32 + kth_set_bit(frL, qk - preL + 1);
-                if (lane < nF) s_H[lane] = hs;
-                hmax = __shfl_sync(FULL_MASK, hs, nF - 1);
-                if (lane < nF && ((((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u))) bad = true;   // key in the tournament, or grouped
+                hs = (w0 + L) * 32 + kth_set_bit(frL, qk - preL + 1);
+                hmax0 = __shfl_sync(FULL_MASK, hs, nF0 - 1);
+                // its key sits in the tournament, or its group has other members
+                const unsigned badH = __ballot_sync(FULL_MASK, lane < nF0 && ((((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u)));
+                if (badH) limF = __ffs(badH) - 1;
             }
+            // limL = how many list entries can be taken before one is grouped, could also be an oldest-first pick of
+            // this batch, or has a key below the tournament's root
+            const bool ok = (mask >> lane) & 1u;
+            const int32_t rank = __popc(mask & ((1u << lane) - 1u));
+            int32_t limL = nL0;
+            {
+                const unsigned long long ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL);
+                const unsigned badE = __ballot_sync(FULL_MASK, ok && rank < nL0 &&
+                                                    ((((R.gb[es >> 5] >> (es & 31)) & 1u)) || (es >= head && es <= hmax0) || root > ek));
+                if (badE) limL = __popc(mask & ((1u << (__ffs(badE) - 1)) - 1u));
+            }
+            const int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_before(lane + 1) <= limF &&
+                                                   (lane + 1) - f_before(lane + 1) <= limL));
+            if (B < 4) return false;
+            const int32_t nF = f_before(B), nL = B - nF;
+            const int32_t hmax = nF > 0 ? __shfl_sync(FULL_MASK, hs, nF - 1) : -1;
+            if (lane < nF) s_H[lane] = hs;
             int32_t consumed = 0;
             if (nL > 0) {
-                const bool ok = (mask >> lane) & 1u;
-                const int32_t rank = __popc(mask & ((1u << lane) - 1u));
-                const bool chosen = ok && rank < nL;
-                const int lastlane = kth_set_bit(mask, nL);
-                consumed = lastlane + 1;
-                if (chosen && (((R.gb[es >> 5] >> (es & 31)) & 1u) || (es >= head && es <= hmax))) bad = true;
-                const unsigned long long ek_last = ~((unsigned long long)__shfl_sync(FULL_MASK, kk, lastlane) ^ 0x8000000000000000ULL);
-                if (root > ek_last) bad = true;
-                if (chosen) s_E[rank] = es;
+                consumed = kth_set_bit(mask, nL) + 1;
+                if (ok && rank < nL) s_E[rank] = es;
             }
-            if (__ballot_sync(FULL_MASK, bad)) return false;
             __syncwarp();
             // commit: lane i makes decision c + i
             if (lane < B) {
