@@ -1222,8 +1222,10 @@ run_kernel(TreeDev T, RunArgs A) {
 //     members are regrouped by their new pairs inside the run they already occupy (they never need more
 //     room: the processed query leaves).  A query in a group of one costs nothing.  Leaves created by the
 //     loop get positions from a counter that starts above every real pool index;
-//   * the longest-match pick is the root of a tournament over the keys (score << 32 | ~rank) of the
-//     arrived queries: 32-ary, leaves in global memory, every level above in shared memory;
+//   * while arrivals are pending, the longest-match pick is the root of a tournament over the keys
+//     (score << 32 | ~rank) of the arrived queries: 32-ary, leaves in global memory, every level above in shared
+//     memory; once everybody has arrived it is the next entry of a list of all keys sorted before the loop, and the
+//     tournament only holds the queries whose key has changed since (see fast_run_kernel);
 //   * the oldest-first pick is a cursor over a bitmap of processed slots.
 // One CTA runs the whole loop: warp 0 is the sequencer, the other warps wait at a named barrier and join
 // for work that is worth sharing (a large group, a large batch of arrivals).  There is no wait on another

@@ -141,6 +141,22 @@ def test_grouped_loop_with_priorities_and_hit_rate(K, score_mode):
         same(got, want)
 
 
+@pytest.mark.parametrize("score_mode", [0, 1])
+def test_list_mode_with_priorities_all_waiting(K, score_mode):
+    """Everybody waiting from the start, mostly distinct continuations, random tie priorities: the loop works from
+    the presorted key list in warp-wide steps, with key ranks that are not the slots."""
+    rng = np.random.RandomState(11)
+    prefixes = [rng.randint(0, 50, size=ln).tolist() for ln in (20, 35, 35, 50, 64)]
+    prompts = [prefixes[rng.randint(5)] + rng.randint(0, 5000, size=rng.randint(1, 30)).tolist() for _ in range(4000)]
+    prefill = [p + [7] for p in prefixes[:4]]
+    arr = [0] * len(prompts)
+    prio = rng.randint(0, 1000, size=len(prompts)).tolist()
+    for policy, k in ((1, 1), (2, 3), (2, 7)):
+        got = run_gpu(K, prefill, prompts, arr, policy, k, prio=prio, score_mode=score_mode)
+        want = run_oracle(prefill, prompts, arr, policy, k, prio=prio, score_mode=score_mode)
+        same(got, want)
+
+
 @pytest.mark.parametrize("name,scale,k", [("medium", 1 / 16, 4), ("adversarial", 1 / 256, 4), ("tiny", 1, 2)])
 def test_both_loops_agree(K, name, scale, k):
     """The grouped loop and the one-by-one loop (forced by KLPM_RUN_LEGACY=1) give identical schedules."""
