@@ -1542,24 +1542,62 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
             if (lane == 0) R.t1[b] = v;
         }
     } else {
-        // dissolve a group of more than 32 members
+        // dissolve a group of more than 32 members, or a smaller one whose members have long compares ahead
         const FastPick& P = J.pick;
         const int32_t gs = P.gstart, gc = P.gcount;
         const bool exact = gc <= KLPM_FAST_SORT_CAP;
         int32_t p2 = 1;
         while (p2 < gc) p2 <<= 1;
-        for (int32_t base = warp * 32; base < gc; base += nwarps * 32) {
-            const int32_t i = base + lane;
-            const int32_t r = i < gc ? __ldcg(A.mem + gs + i) : -1;
-            bool touched;
-            const unsigned long long h = fast_member(A, P, R, r, lane, &touched);
-            if (i < gc) {
-                if (exact) { sh[i] = h; sr[i] = r; }
-                else { __stcg(A.gh + i, (long long)h); __stcg(A.gidx + i, r); }
+        if (exact) {
+            // classify the members; the tied ones go on a list (A.gidx is free while the run is sorted in shared memory)
+            if (tid == 0) *s_cnt = 0;
+            __syncthreads();
+            for (int32_t base = warp * 32; base < gc; base += nwarps * 32) {
+                const int32_t i = base + lane;
+                const int32_t r = i < gc ? __ldcg(A.mem + gs + i) : -1;
+                const bool act = r >= 0 && r != P.slot;
+                unsigned long long h = KLPM_FAST_NOGROUP;
+                if (act && !slot_done(R, A, r)) {
+                    const FDyn d = ld_dyn(A.dyn + r);
+                    const FStat s = ld_stat(A.stat + r);
+                    if (d.pos == P.pos && d.ntok == P.ntok && d.m == P.m && d.m < s.len) __stcg(A.gidx + atomicAdd(s_cnt, 1), i);
+                    else h = d.m < s.len ? group_hash(d.pos, d.ntok) : single_hash(r);
+                }
+                if (i < gc) { sh[i] = h; sr[i] = r; }
             }
+            for (int32_t i = gc + tid; i < p2; i += nthr) { sh[i] = KLPM_FAST_NOGROUP; sr[i] = -1; }
+            __syncthreads();
+            // one tied member per warp at a time: compare it with the processed prompt's uncached tokens
+            const int32_t nt = *s_cnt;
+            for (int32_t k = warp; k < nt; k += nwarps) {
+                const int32_t i = __ldcg(A.gidx + k);
+                const int32_t r = sr[i];
+                const FStat s = ld_stat(A.stat + r);
+                const int32_t* qq = A.tok + s.soff;
+                const int32_t lim = (s.len < P.len ? s.len : P.len) - P.m;
+                const int32_t e = first_mismatch<true, 8>(qq + P.m, P.x + P.m, lim);
+                if (lane == 0) {
+                    const int32_t m2 = P.m + e;
+                    const long long pos2 = P.vleaf + e - 1;
+                    const int32_t ntok2 = m2 < s.len ? __ldg(qq + m2) : 0;
+                    st_dyn_state(A.dyn + r, pos2, m2, ntok2);
+                    const unsigned long long key = fast_key(m2, s.len, s.rank, A.score_mode);
+                    __stcg(A.key + r, key);
+                    if (R.skip) atomicOr(R.skip + (r >> 5), 1u << (r & 31));
+                    if ((long long)r < P.admitted) atomicMax(R.t1 + (r >> A.lb_shift), key);
+                    sh[i] = m2 < s.len ? group_hash(pos2, ntok2) : single_hash(r);
+                }
+            }
+        } else {
+            for (int32_t base = warp * 32; base < gc; base += nwarps * 32) {
+                const int32_t i = base + lane;
+                const int32_t r = i < gc ? __ldcg(A.mem + gs + i) : -1;
+                bool touched;
+                const unsigned long long h = fast_member(A, P, R, r, lane, &touched);
+                if (i < gc) { __stcg(A.gh + i, (long long)h); __stcg(A.gidx + i, r); }
+            }
+            if (tid == 0) *s_cnt = 0;
         }
-        if (exact) for (int32_t i = gc + tid; i < p2; i += nthr) { sh[i] = KLPM_FAST_NOGROUP; sr[i] = -1; }
-        if (tid == 0) *s_cnt = 0;
         __syncthreads();
         if (exact) {
             // regroup exactly: sort the members by the hash of their new group inside the run
@@ -1708,7 +1746,8 @@ fast_run_kernel(FastArgs A) {
             FastPick P;
             P.slot = slot; P.m = m; P.len = len; P.ntok = d.ntok; P.x = A.tok + s.soff; P.pos = d.pos; P.vleaf = vleaf;
             P.admitted = admitted; P.gstart = d.gstart; P.gcount = d.gcount;
-            if (d.gcount <= 32) {
+            // small groups are handled by this warp alone, unless several long compares are better spread over the CTA
+            if (d.gcount <= 32 && !(d.gcount > 2 && unc > 512)) {
                 const int32_t r = lane < d.gcount ? __ldcg(A.mem + d.gstart + lane) : -1;
                 bool touched;
                 const unsigned long long h = fast_member(A, P, R, r, lane, &touched);
