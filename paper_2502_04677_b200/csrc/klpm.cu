@@ -1887,10 +1887,16 @@ fast_run_kernel(FastArgs A) {
             const long long tj = (long long)(((unsigned long long)(unsigned)ps.y << 32) | (unsigned)ps.x);
             long long x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
             long long y = unc;
+            if (A.c_num == 0) {                             // cost = c_den tokens' worth each: one running sum serves both
 #pragma unroll
-            for (int dlt = 1; dlt < 32; dlt <<= 1) {
-                const long long xo = __shfl_up_sync(FULL_MASK, x, dlt), yo = __shfl_up_sync(FULL_MASK, y, dlt);
-                if (lane >= dlt) { x += xo; y += yo; }
+                for (int dlt = 1; dlt < 32; dlt <<= 1) { const long long yo = __shfl_up_sync(FULL_MASK, y, dlt); if (lane >= dlt) y += yo; }
+                x = A.c_den * y;
+            } else {
+#pragma unroll
+                for (int dlt = 1; dlt < 32; dlt <<= 1) {
+                    const long long xo = __shfl_up_sync(FULL_MASK, x, dlt), yo = __shfl_up_sync(FULL_MASK, y, dlt);
+                    if (lane >= dlt) { x += xo; y += yo; }
+                }
             }
             const long long Rj = now + x;
             if (v) {
@@ -1917,12 +1923,21 @@ fast_run_kernel(FastArgs A) {
         // picks consume), none whose group has other members, none whose key sits in the tournament, and the
         // tournament's root below the smallest key taken from the list.  Then lane i makes decision c + i.
         // If any check fails nothing has been changed and the decisions are made one at a time below.
+        const int32_t lane_div_k = lane / A.k;              // y / k for y = 0..31, looked up by shuffle
         auto try_batch = [&]() -> bool {
-            auto f_before = [&](int32_t x) -> int32_t {     // oldest-first turns among the next x decisions
-                if (A.policy == KLPM_POLICY_FCFS) return x;
-                if (A.policy == KLPM_POLICY_LPM) return 0;
-                return (cyc + x + A.k - 1) / A.k - (cyc + A.k - 1) / A.k;
-            };
+            // oldest-first turns among the next x decisions, for x = lane (f_lo) and x = lane + 1 (f_hi): under k-LPM
+            // the first such turn is decision i0 = (k - cyc) mod k, then every k-th
+            int32_t f_lo, f_hi;
+            if (A.policy == KLPM_POLICY_FCFS) { f_lo = lane; f_hi = lane + 1; }
+            else if (A.policy == KLPM_POLICY_LPM) { f_lo = 0; f_hi = 0; }
+            else {
+                const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;
+                const int32_t y_lo = lane - i0 - 1, y_hi = lane - i0;
+                const int32_t q_lo = __shfl_sync(FULL_MASK, lane_div_k, y_lo > 0 ? y_lo : 0);
+                const int32_t q_hi = __shfl_sync(FULL_MASK, lane_div_k, y_hi > 0 ? y_hi : 0);
+                f_lo = y_lo >= 0 ? q_lo + 1 : 0;
+                f_hi = y_hi >= 0 ? q_hi + 1 : 0;
+            }
             // the list entries cur .. cur + 31 (in this window or the next) that still count
             long long kk; int32_t es; unsigned mask;
             {
@@ -1936,9 +1951,9 @@ fast_run_kernel(FastArgs A) {
             }
             // as many decisions as those entries allow: lane x asks whether x + 1 decisions need no more of them
             const int32_t avail = __popc(mask);
-            const int32_t B0 = __popc(__ballot_sync(FULL_MASK, c + lane < n && (lane + 1) - f_before(lane + 1) <= avail));
+            const int32_t B0 = __popc(__ballot_sync(FULL_MASK, c + lane < n && (lane + 1) - f_hi <= avail));
             if (B0 < 4) return false;
-            const int32_t nF0 = f_before(B0), nL0 = B0 - nF0;
+            const int32_t nF0 = __shfl_sync(FULL_MASK, f_hi, B0 - 1), nL0 = B0 - nF0;
             // the next nF0 unprocessed slots; limF = how many of them can be taken before one needs the careful step
             int32_t hs = -1, hmax0 = -1, limF = nF0;
             if (nF0 > 0) {
@@ -1976,10 +1991,9 @@ fast_run_kernel(FastArgs A) {
                                                     ((((R.gb[es >> 5] >> (es & 31)) & 1u)) || (es >= head && es <= hmax0) || root > ek));
                 if (badE) limL = __popc(mask & ((1u << (__ffs(badE) - 1)) - 1u));
             }
-            const int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_before(lane + 1) <= limF &&
-                                                   (lane + 1) - f_before(lane + 1) <= limL));
+            const int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_hi <= limF && (lane + 1) - f_hi <= limL));
             if (B < 4) return false;
-            const int32_t nF = f_before(B), nL = B - nF;
+            const int32_t nF = __shfl_sync(FULL_MASK, f_hi, B - 1), nL = B - nF;
             const int32_t hmax = nF > 0 ? __shfl_sync(FULL_MASK, hs, nF - 1) : -1;
             if (lane < nF) s_H[lane] = hs;
             int32_t consumed = 0;
@@ -1990,8 +2004,7 @@ fast_run_kernel(FastArgs A) {
             __syncwarp();
             // commit: lane i makes decision c + i
             if (lane < B) {
-                const int32_t f0 = f_before(lane);
-                myj = f_before(lane + 1) > f0 ? s_H[f0] : s_E[lane - f0];
+                myj = f_hi > f_lo ? s_H[f_lo] : s_E[lane - f_lo];
                 atomicOr(s_done + (myj >> 5), 1u << (myj & 31));
                 atomicOr(R.skip + (myj >> 5), 1u << (myj & 31));
             }
