@@ -2097,6 +2097,7 @@ struct BulkArgs {
     const int32_t* tok; const int64_t* off;
     const int32_t* pend_in; int32_t* pend_out; unsigned int* n_out;   // walk: prompts to walk -> prompts not fully stored yet
     int32_t* pend_next; unsigned int* n_next;                          // apply: prompts that have to try again next round
+    unsigned int* n_walk;                                              // walk: work counter
     int32_t* claim;                    // per node: lowest prompt index that wants to cut its edge
     int32_t* pm; int32_t* pnode; int32_t* poff;   // per prompt: where its walk ended
 };
@@ -2104,8 +2105,11 @@ struct BulkArgs {
 __global__ void __launch_bounds__(256)
 bulk_walk_kernel(TreeDev T, BulkArgs A, unsigned n_pending) {
     const int lane = threadIdx.x & 31;
-    const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
-    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
+    for (;;) {                                              // prompts are handed out by a counter: their lengths differ widely
+        unsigned p = 0;
+        if (lane == 0) p = atomicAdd(A.n_walk, 1u);
+        p = __shfl_sync(FULL_MASK, p, 0);
+        if (p >= n_pending) return;
         const int32_t i = __ldg(A.pend_in + p);
         const int64_t lo = __ldg(A.off + i);
         const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
@@ -2420,7 +2424,7 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
             (st = dalloc(&t->bulk_pnode, n)) || (st = dalloc(&t->bulk_poff, n))) return st;
         t->bulk_cap = n;
     }
-    if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 2))) return st;      // walk's and apply's list lengths
+    if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 3))) return st;      // walk's and apply's list lengths, walk's work counter
     int32_t *pend_a = t->bulk_pend_a, *pend_b = t->bulk_pend_b, *pm = t->bulk_pm, *pnode = t->bulk_pnode, *poff = t->bulk_poff;
     unsigned int* n_out = t->bulk_n_out;
     // claim words start idle (an earlier call that ran out of capacity may have left some set)
@@ -2433,11 +2437,11 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         if (++rounds > 1000000) { st = RT_ERR_LIMIT; break; }
         BulkArgs a;
         a.tok = d_tokens; a.off = d_offsets; a.pend_in = pend_a; a.pend_out = pend_b; a.n_out = n_out;
-        a.pend_next = pend_a; a.n_next = n_out + 1;          // the walk has consumed pend_a by the time apply refills it
+        a.pend_next = pend_a; a.n_next = n_out + 1; a.n_walk = n_out + 2;          // the walk has consumed pend_a by the time apply refills it
         a.claim = t->claim; a.pm = pm; a.pnode = pnode; a.poff = poff;
         long long blocks = ((long long)count + 7) / 8;
         if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
-        e = cudaMemsetAsync(n_out, 0, 2 * sizeof(unsigned), s);
+        e = cudaMemsetAsync(n_out, 0, 3 * sizeof(unsigned), s);
         if (e != cudaSuccess) break;
         bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
         bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
