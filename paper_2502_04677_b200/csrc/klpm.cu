@@ -1269,6 +1269,7 @@ struct FastArgs {
     const long long* lk;          // list mode: every slot's key, largest first, stored as ~key with the top bit flipped
     const int32_t* ls;            //            and the slot it belongs to
     unsigned long long* counter;  // work counter of the initial walk
+    int32_t* pm; int32_t* pnode; int32_t* poff;   // per query (nullable): where its walk ended, for the insertion after the loop
     TreeState* st;
 };
 
@@ -1351,8 +1352,12 @@ fast_walk_kernel(TreeDev T, FastArgs A, long long np2) {
         const int32_t* q = A.tok + s.soff;
         int32_t node, off;
         int64_t pos;
-        const int32_t m = walk_chain<true>(T, q, len, false, &node, &off, &pos);
+        const int32_t m = walk_chain<true>(T, q, len, A.pm != nullptr, &node, &off, &pos);
         if (lane == 0) {
+            if (A.pm) {       // the insertion after the loop starts from this walk: the tree does not change in between
+                const bool full = node == 0 || off == __ldg(T.span_len + node);
+                A.pm[s.ord] = m; A.pnode[s.ord] = node; A.poff[s.ord] = full ? -1 : off;
+            }
             const int32_t ntok = m < len ? __ldg(q + m) : 0;
             st_dyn_state(A.dyn + r, pos, m, ntok);
             A.key[r] = fast_key(m, len, s.rank, A.score_mode);
@@ -2125,6 +2130,20 @@ bulk_walk_kernel(TreeDev T, BulkArgs A, unsigned n_pending) {
     }
 }
 
+// First round when the prompts have been walked already (by the scheduling loop's set-up, on the tree as it still is):
+// what bulk_walk_kernel does after its walk.
+__global__ void bulk_prewalked_kernel(BulkArgs A, unsigned n_pending) {
+    const unsigned p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n_pending) return;
+    const int32_t i = A.pend_in[p];
+    const int32_t len = (int32_t)(__ldg(A.off + i + 1) - __ldg(A.off + i));
+    const int32_t m = A.pm[i], off = A.poff[i];
+    if (!(m == len && off < 0)) {
+        if (off >= 0) atomicMin(&A.claim[A.pnode[i]], i);
+        A.pend_out[atomicAdd(A.n_out, 1u)] = i;
+    }
+}
+
 __global__ void __launch_bounds__(256)
 bulk_apply_kernel(TreeDev T, BulkArgs A) {
     const unsigned n_pending = *A.n_out;
@@ -2414,7 +2433,7 @@ TopkScratch* g_topk_scratch[64] = {nullptr};
 StaticSelectScratch* g_select_static_addr[64] = {nullptr};   // device address of g_select_static, per device
 
 // Many prompts at once into a tree without a budget (see the bulk kernels).  Waits for the stream once per round.
-rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s) {
+rt_status ensure_bulk_scratch(rt_tree* t, int32_t n) {
     rt_status st = RT_OK;
     if (n > t->bulk_cap) {                     // per-prompt scratch, kept for later calls
         cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
@@ -2425,6 +2444,13 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         t->bulk_cap = n;
     }
     if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 3))) return st;      // walk's and apply's list lengths, walk's work counter
+    return RT_OK;
+}
+
+// `prewalked`: bulk_pm / bulk_pnode / bulk_poff already hold every prompt's walk on the tree as it is now.
+rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s, bool prewalked = false) {
+    rt_status st = ensure_bulk_scratch(t, n);
+    if (st) return st;
     int32_t *pend_a = t->bulk_pend_a, *pend_b = t->bulk_pend_b, *pm = t->bulk_pm, *pnode = t->bulk_pnode, *poff = t->bulk_poff;
     unsigned int* n_out = t->bulk_n_out;
     // claim words start idle (an earlier call that ran out of capacity may have left some set)
@@ -2443,7 +2469,8 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
         e = cudaMemsetAsync(n_out, 0, 3 * sizeof(unsigned), s);
         if (e != cudaSuccess) break;
-        bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
+        if (prewalked && rounds == 1) bulk_prewalked_kernel<<<(count + 255) / 256, 256, 0, s>>>(a, count);
+        else bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
         bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
         e = cudaGetLastError();
         if (e != cudaSuccess) break;
@@ -2852,12 +2879,15 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         memset(&f, 0, sizeof(f));
         st = ensure_fast_scratch(tree, n);
         if (st) return st;
+        st = ensure_bulk_scratch(tree, n);
+        if (st) return st;
         f.tok = d_q_tokens; f.n = n; f.policy = params->policy; f.k = params->k; f.score_mode = score_mode;
         f.c_num = params->c_num; f.c_den = params->c_den; f.start_tick = params->start_tick;
         f.order = d_order; f.uncached = d_uncached; f.ttft = d_ttft; f.completion = d_completion;
         f.dyn = tree->fast_dyn; f.stat = tree->fast_stat; f.key = tree->fast_key_arr; f.mem = tree->fast_mem;
         f.pinv = d_tie_priority ? tree->run_pinv : nullptr;
         f.gh = tree->fast_gh; f.gidx = tree->fast_gidx; f.done = tree->fast_done; f.counter = tree->fast_counter;
+        f.pm = tree->bulk_pm; f.pnode = tree->bulk_pnode; f.poff = tree->bulk_poff;
         f.vbase = tree->dev.max_pool + 16;
         f.st = tree->dev.st;
         // every query is matched once against the tree as it stands
@@ -2909,7 +2939,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         tree->run_path = 2;
         // The processed prompts enter the tree together (the logical clock advances by n).  The loop itself needs
         // no room in the tree; if the tree cannot hold the queue the insertion says so through the status word.
-        return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s);
+        return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s, true);
     }
     RunBcast bc0;
     memset(&bc0, 0, sizeof(bc0));
