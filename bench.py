@@ -290,7 +290,9 @@ def run_ours(args):
         np2 <<= 1
     lg = np2.bit_length() - 1
     run_path = K.klpm_run_path(tree)
-    sort_launches = lg * (lg + 1) // 2
+    # one sort: the stages up to a tile of 2,048 pairs in one launch, then per larger stage its global steps and one tile launch
+    big = max(0, lg - 11)
+    sort_launches = 1 + big * (big + 1) // 2 + big
     if run_path == K.RUN_PATH_GROUPED:
         # match; slot keys, arrival sort, slot arrays; slot records, walk of every query, group sort, groups,
         # key list and its sort (queues up to 262,144), the loop; bulk insertion of the processed prompts: claim

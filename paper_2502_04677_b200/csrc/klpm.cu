@@ -1264,7 +1264,7 @@ struct FastArgs {
     int32_t lb_shift;             // log2 of the number of slots per tournament leaf block
     int32_t nb;                   // number of leaf blocks
     int32_t done_in_smem;
-    int32_t run_ahead;            // the list mode of the loop can be used (32-slot leaf blocks, all bitmaps in shared memory)
+    int32_t list_mode;            // the list mode of the loop can be used (32-slot leaf blocks, all bitmaps in shared memory)
     unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts
     const long long* lk;          // list mode: every slot's key, largest first, stored as ~key with the top bit flipped
     const int32_t* ls;            //            and the slot it belongs to
@@ -1678,11 +1678,11 @@ fast_run_kernel(FastArgs A) {
     int32_t* sr = reinterpret_cast<int32_t*>(sh + KLPM_FAST_SORT_CAP);
     unsigned int* s_done = reinterpret_cast<unsigned int*>(sr + KLPM_FAST_SORT_CAP);
     R.done = A.done_in_smem ? s_done : nullptr;
-    R.skip = A.run_ahead ? s_done + nwords : nullptr;
-    R.gb = A.run_ahead ? s_done + 2 * nwords : nullptr;
+    R.skip = A.list_mode ? s_done + nwords : nullptr;
+    R.gb = A.list_mode ? s_done + 2 * nwords : nullptr;
     for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
     if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
-    if (A.run_ahead) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
+    if (A.list_mode) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
     __syncthreads();
 
     if (warp != 0) {
@@ -1786,10 +1786,10 @@ fast_run_kernel(FastArgs A) {
     };
 
     // everybody is waiting as the loop starts: no arrival will ever have to be admitted
-    if (A.run_ahead && __ldg(&A.stat[n - 1].t) <= now) { admitted = n; next_t = INF; }
+    if (A.list_mode && __ldg(&A.stat[n - 1].t) <= now) { admitted = n; next_t = INF; }
 
     // ================================================================ arrivals pending: one careful step per decision
-    while (c < n && !failed && !(A.run_ahead && admitted == n)) {
+    while (c < n && !failed && !(A.list_mode && admitted == n)) {
         // ---- time and arrivals: idle until somebody has arrived, then admit everybody who has
         if (head == admitted && next_t > now) now = next_t;
         if (next_t <= now) {
@@ -2297,6 +2297,46 @@ __global__ void bitonic_step_kernel(long long* key, int32_t* idx, long long np2,
         bool gt = ki > kl || (ki == kl && ii > il);
         bool up = (i & k) == 0;
         if (gt == up) { key[i] = kl; key[l] = ki; idx[i] = il; idx[l] = ii; }
+    }
+}
+
+// The steps of the same sort whose partner distance fits a tile of 2,048 pairs, done in shared memory: all stages
+// k_lo .. k_hi when those are at most the tile (the start of the sort), otherwise the tail (distances below the
+// tile) of the one stage k_lo = k_hi.
+#define KLPM_SORT_TILE 2048
+__global__ void __launch_bounds__(512)
+bitonic_tile_kernel(long long* key, int32_t* idx, long long np2, long long k_lo, long long k_hi) {
+    __shared__ long long sk[KLPM_SORT_TILE];
+    __shared__ int32_t si[KLPM_SORT_TILE];
+    const int T = np2 < KLPM_SORT_TILE ? (int)np2 : KLPM_SORT_TILE;
+    const long long base = (long long)blockIdx.x * T;
+    for (int u = threadIdx.x; u < T; u += blockDim.x) { sk[u] = key[base + u]; si[u] = idx[base + u]; }
+    __syncthreads();
+    for (long long k = k_lo; k <= k_hi; k <<= 1) {
+        const long long jmax = (k >> 1) < (long long)(T >> 1) ? (k >> 1) : (long long)(T >> 1);
+        for (int j = (int)jmax; j > 0; j >>= 1) {
+            for (int u = threadIdx.x; u < (T >> 1); u += blockDim.x) {
+                const int i = ((u & ~(j - 1)) << 1) | (u & (j - 1)), l = i | j;      // the u-th pair at distance j
+                const long long ki = sk[i], kl = sk[l];
+                const int32_t ii = si[i], il = si[l];
+                const bool gt = ki > kl || (ki == kl && ii > il);
+                const bool up = ((base + i) & k) == 0;
+                if (gt == up) { sk[i] = kl; sk[l] = ki; si[i] = il; si[l] = ii; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int u = threadIdx.x; u < T; u += blockDim.x) { key[base + u] = sk[u]; idx[base + u] = si[u]; }
+}
+
+// (key, idx) pairs ascending by key, then idx; np2 a power of two
+void sort_pairs(long long* key, int32_t* idx, long long np2, cudaStream_t s) {
+    const long long T = np2 < KLPM_SORT_TILE ? np2 : KLPM_SORT_TILE;
+    const unsigned tiles = (unsigned)(np2 / T), blocks = (unsigned)((np2 + 255) / 256);
+    if (T >= 2) bitonic_tile_kernel<<<tiles, 512, 0, s>>>(key, idx, np2, 2, T);
+    for (long long k = T << 1; k <= np2; k <<= 1) {
+        for (long long j = k >> 1; j >= T; j >>= 1) bitonic_step_kernel<<<blocks, 256, 0, s>>>(key, idx, np2, k, j);
+        bitonic_tile_kernel<<<tiles, 512, 0, s>>>(key, idx, np2, k, k);
     }
 }
 
@@ -2861,15 +2901,11 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     {
         unsigned blocks = (unsigned)((np2 + 255) / 256);
         rank_init_kernel<<<blocks, 256, 0, s>>>(d_arrival, n, np2, tree->run_key, tree->run_ord);
-        for (long long k = 2; k <= np2; k <<= 1)
-            for (long long j = k >> 1; j > 0; j >>= 1)
-                bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_key, tree->run_ord, np2, k, j);
+        sort_pairs(tree->run_key, tree->run_ord, np2, s);
         slot_arrays_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, d_q_offsets, n, tree->run_soff, tree->run_slen);
         if (d_tie_priority) {        // rank of every slot by (priority, slot)
             prio_init_kernel<<<blocks, 256, 0, s>>>(d_tie_priority, tree->run_ord, n, np2, tree->run_pkey, tree->run_pinv);
-            for (long long k = 2; k <= np2; k <<= 1)
-                for (long long j = k >> 1; j > 0; j >>= 1)
-                    bitonic_step_kernel<<<blocks, 256, 0, s>>>(tree->run_pkey, tree->run_pinv, np2, k, j);
+            sort_pairs(tree->run_pkey, tree->run_pinv, np2, s);
             prio_rank_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_pinv, n, tree->run_prank);
         }
         CK(cudaGetLastError());
@@ -2915,22 +2951,18 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
         // list mode needs two more bitmaps in shared memory and 32-slot leaf blocks
-        f.run_ahead = (f.done_in_smem && lbs == 5 && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
-        if (f.run_ahead) smem += (size_t)nwords * 8;
+        f.list_mode = (f.done_in_smem && lbs == 5 && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
+        if (f.list_mode) smem += (size_t)nwords * 8;
         f.gbits = tree->fast_done + (np2 / 32 + 32);
         const unsigned nblk = (unsigned)((n + 255) / 256), pblk = (unsigned)((np2 + 255) / 256);
         CK(cudaMemsetAsync(f.done, 0, (size_t)(2 * (np2 / 32 + 32)) * sizeof(unsigned int), s));
         // groups: queries whose match ends at the same position and continues with the same token
-        for (long long k = 2; k <= np2; k <<= 1)
-            for (long long j = k >> 1; j > 0; j >>= 1)
-                bitonic_step_kernel<<<pblk, 256, 0, s>>>(f.gh, f.gidx, np2, k, j);
+        sort_pairs(f.gh, f.gidx, np2, s);
         fast_group_kernel<<<nblk, 256, 0, s>>>(f);
-        if (f.run_ahead) {           // all keys, largest first
+        if (f.list_mode) {           // all keys, largest first
             f.lk = tree->fast_lk; f.ls = tree->fast_ls;
             fast_list_kernel<<<pblk, 256, 0, s>>>(f.key, n, np2, tree->fast_lk, tree->fast_ls);
-            for (long long k = 2; k <= np2; k <<= 1)
-                for (long long j = k >> 1; j > 0; j >>= 1)
-                    bitonic_step_kernel<<<pblk, 256, 0, s>>>(tree->fast_lk, tree->fast_ls, np2, k, j);
+            sort_pairs(tree->fast_lk, tree->fast_ls, np2, s);
         }
         CK(cudaGetLastError());
         CK(cudaFuncSetAttribute(fast_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

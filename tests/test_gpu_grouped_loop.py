@@ -2,7 +2,7 @@
 
 klpm_run on a tree without a budget keeps every query's match state itself: queries whose match ends at the
 same tree position and continues with the same token form a group, and processing a prompt re-matches its
-group only.  These cases aim at the group machinery: groups of 2..32 (one warp), groups up to 2,048 (sorted in
+group only.  These cases aim at the group machinery: groups of 2..32 (one warp), groups up to 4,096 (sorted in
 shared memory), larger groups (kept together), queries that have not arrived when their group changes,
 identical prompts, prompts that are prefixes of others, and the tie-priority / hit-rate variants."""
 import os
@@ -173,7 +173,7 @@ def test_both_loops_agree(K, name, scale, k):
 @pytest.mark.parametrize("max_blocks,smem_kb", [(16, 0), (4, 60), (1, 0)])
 def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb, monkeypatch):
     """Queues above 262,144 use larger tournament leaf blocks, and far larger ones keep the processed bitmap in
-    global memory; neither uses run-ahead.  Shrinking the limits makes a 3,000-query stream take those paths."""
+    global memory; neither uses list mode.  Shrinking the limits makes a 3,000-query stream take those paths."""
     monkeypatch.setenv("KLPM_FAST_MAX_BLOCKS", str(max_blocks))
     if smem_kb:
         monkeypatch.setenv("KLPM_FAST_SMEM_KB", str(smem_kb))
@@ -185,9 +185,9 @@ def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb, monkeypatch
         same(got, want)
 
 
-def test_run_ahead_bursts_all_arrived(K):
-    """Everybody waiting from the start and mostly distinct continuations: the loop runs ahead in long bursts,
-    broken by the few grouped queries (medium at 1/8: 4,096 queries, 64 prefixes)."""
+def test_list_mode_all_arrived(K):
+    """Everybody waiting from the start and mostly distinct continuations: the loop works from the presorted key
+    list in warp-wide steps, cut short by the few grouped queries (medium at 1/8: 4,096 queries, 64 prefixes)."""
     w = W.medium(scale=1 / 8)
     pt, po = w.prefill.materialize()
     qt, qo = w.queries.materialize()
