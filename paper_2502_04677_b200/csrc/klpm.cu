@@ -1926,8 +1926,9 @@ fast_run_kernel(FastArgs A) {
         // interleaved as the policy says.  The warp gathers both sets side by side and checks that they cannot
         // have influenced each other: no slot in both (a list entry inside the range of slots the oldest-first
         // picks consume), none whose group has other members, none whose key sits in the tournament, and the
-        // tournament's root below the smallest key taken from the list.  Then lane i makes decision c + i.
-        // If any check fails nothing has been changed and the decisions are made one at a time below.
+        // tournament's root below the smallest key taken from the list.  The batch is cut before the first decision
+        // that fails a check; then lane i makes decision c + i.  If fewer than four decisions are left that way,
+        // nothing has been changed and the next decisions are made one at a time below.
         const int32_t lane_div_k = lane / A.k;              // y / k for y = 0..31, looked up by shuffle
         auto try_batch = [&]() -> bool {
             // oldest-first turns among the next x decisions, for x = lane (f_lo) and x = lane + 1 (f_hi): under k-LPM
