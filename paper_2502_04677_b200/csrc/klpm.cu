@@ -1963,24 +1963,32 @@ fast_run_kernel(FastArgs A) {
             // the next nF0 unprocessed slots; limF = how many of them can be taken before one needs the careful step
             int32_t hs = -1, hmax0 = -1, limF = nF0;
             if (nF0 > 0) {
-                const int32_t w0 = head >> 5, wi = w0 + lane;
-                unsigned w = wi < nwords ? s_done[wi] : 0xffffffffu;
-                if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
-                if (wi == w0) w |= (1u << (head & 31)) - 1u;
-                const unsigned fr = ~w;
-                const int32_t cnt = __popc(fr);
-                int32_t inc = cnt;
+                const int32_t w0 = head >> 5;
+                const int32_t qk = lane < nF0 ? lane : nF0 - 1;       // lane q looks for the q-th unprocessed slot
+                auto free_word = [&](int32_t wi) -> unsigned {        // unprocessed slots of bitmap word wi, from head on
+                    unsigned w = wi < nwords ? s_done[wi] : 0xffffffffu;
+                    if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
+                    if (wi == w0) w |= (1u << (head & 31)) - 1u;
+                    return ~w;
+                };
+                const unsigned f0 = free_word(w0), f1 = free_word(w0 + 1);
+                const int32_t c0 = __popc(f0);
+                if (c0 + __popc(f1) >= nF0) {                         // the usual case: they are all in the first two words
+                    hs = qk < c0 ? w0 * 32 + kth_set_bit(f0, qk + 1) : (w0 + 1) * 32 + kth_set_bit(f1, qk - c0 + 1);
+                } else {                                              // up to 32 words: running counts, then a search per lane
+                    const unsigned fr = free_word(w0 + lane);
+                    const int32_t cnt = __popc(fr);
+                    int32_t inc = cnt;
 #pragma unroll
-                for (int dlt = 1; dlt < 32; dlt <<= 1) { const int32_t o = __shfl_up_sync(FULL_MASK, inc, dlt); if (lane >= dlt) inc += o; }
-                if (__shfl_sync(FULL_MASK, inc, 31) < nF0) return false;
-                // lane q finds the q-th of them: the first word whose running count exceeds q, then the bit inside it
-                const int32_t qk = lane < nF0 ? lane : nF0 - 1;
-                int L = 0;
+                    for (int dlt = 1; dlt < 32; dlt <<= 1) { const int32_t o = __shfl_up_sync(FULL_MASK, inc, dlt); if (lane >= dlt) inc += o; }
+                    if (__shfl_sync(FULL_MASK, inc, 31) < nF0) return false;
+                    int L = 0;
 #pragma unroll
-                for (int step = 16; step > 0; step >>= 1) if (__shfl_sync(FULL_MASK, inc, L + step - 1) <= qk) L += step;
-                const unsigned frL = __shfl_sync(FULL_MASK, fr, L);
-                const int32_t preL = __shfl_sync(FULL_MASK, inc - cnt, L);
-                hs = (w0 + L) * 32 + kth_set_bit(frL, qk - preL + 1);
+                    for (int step = 16; step > 0; step >>= 1) if (__shfl_sync(FULL_MASK, inc, L + step - 1) <= qk) L += step;
+                    const unsigned frL = __shfl_sync(FULL_MASK, fr, L);
+                    const int32_t preL = __shfl_sync(FULL_MASK, inc - cnt, L);
+                    hs = (w0 + L) * 32 + kth_set_bit(frL, qk - preL + 1);
+                }
                 hmax0 = __shfl_sync(FULL_MASK, hs, nF0 - 1);
                 // its key sits in the tournament, or its group has other members
                 const unsigned badH = __ballot_sync(FULL_MASK, lane < nF0 && ((((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u)));
