@@ -1706,7 +1706,15 @@ fast_run_kernel(FastArgs A) {
 
     // first unprocessed slot at or after `head` (which is processed)
     auto advance_head = [&]() {
-        if (A.done_in_smem && head + 1 < n && !((s_done[(head + 1) >> 5] >> ((head + 1) & 31)) & 1u)) { ++head; return; }   // the usual case
+        if (A.done_in_smem && head + 1 < n) {               // the usual cases: the next slot, or one of the next 32 to 63
+            const int32_t h1 = head + 1, wi = h1 >> 5;
+            const unsigned f0 = ~s_done[wi] & ~((1u << (h1 & 31)) - 1u);
+            if (f0) { head = wi * 32 + __ffs(f0) - 1; if (head > n) head = n; return; }
+            if (wi + 1 < nwords) {
+                const unsigned f1 = ~s_done[wi + 1];
+                if (f1) { head = (wi + 1) * 32 + __ffs(f1) - 1; if (head > n) head = n; return; }
+            }
+        }
         int32_t w0 = head >> 5;
         for (;;) {
             const int32_t wi = w0 + lane;
