@@ -157,6 +157,25 @@ def test_list_mode_with_priorities_all_waiting(K, score_mode):
         same(got, want)
 
 
+@pytest.mark.parametrize("n", [1, 31, 33, 100, 1000, 5001])
+def test_list_mode_many_turn_patterns(K, n):
+    """Everybody waiting, a tree that already holds the shared prefixes, mostly distinct continuations with a few
+    identical prompts and a few shared continuations: warp-wide steps of every size and turn pattern (k below,
+    at and above 32, k = 1, pure policies), queue lengths around the 32-lane boundaries."""
+    rng = np.random.RandomState(100 + n)
+    prefixes = [rng.randint(0, 1000, size=ln).tolist() for ln in (3, 17, 40, 40, 90)]
+    prompts = []
+    for _ in range(n):
+        p = prefixes[rng.randint(5)] + rng.randint(0, 300, size=rng.randint(0, 12)).tolist()
+        prompts.append(prompts[rng.randint(len(prompts))] if prompts and rng.rand() < 0.03 else p)
+    prefill = [p + [1001] for p in prefixes]
+    arr = [0] * n
+    for policy, k in ((0, 1), (1, 1), (2, 1), (2, 2), (2, 3), (2, 5), (2, 31), (2, 32), (2, 33), (2, 1000)):
+        got = run_gpu(K, prefill, prompts, arr, policy, k, c_num=1, c_den=2)
+        want = run_oracle(prefill, prompts, arr, policy, k, c_num=1, c_den=2)
+        same(got, want)
+
+
 @pytest.mark.parametrize("name,scale,k", [("medium", 1 / 16, 4), ("adversarial", 1 / 256, 4), ("tiny", 1, 2)])
 def test_both_loops_agree(K, name, scale, k):
     """The grouped loop and the one-by-one loop (forced by KLPM_RUN_LEGACY=1) give identical schedules."""
