@@ -1074,6 +1074,13 @@ run_kernel(TreeDev T, RunArgs A) {
         if (threadIdx.x == 0) run_bound(A, s_bc, &s_bound[0], &s_bound[1]);
         __syncthreads();
         const long long head = s_bc.head, adm_new = s_bound[0];
+        // The queries that arrive next will be walked from the root by a single warp while everybody waits: bring
+        // their tokens into L2 now (slots are in arrival order, so these are known; a hint only).
+        for (long long r = adm_new; r < adm_new + 2 && r < A.n; ++r) {
+            const int32_t* q = A.tok + __ldg(A.soff + r);
+            const int32_t qlen = __ldg(A.slen + r);
+            for (int32_t i = threadIdx.x * 32; i < qlen; i += blockDim.x * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(q + i));
+        }
         unsigned long long b = 0;
         if (G == 1) {
             unsigned long long best = warp_max64(run_scan(T, A, s_bc, adm_new, 0, 1));
