@@ -1255,6 +1255,8 @@ struct alignas(32) FStat {    // constant during the loop; the first 16 bytes ar
     int32_t pad;
 };
 
+struct FastPost { int32_t c0; int32_t pad; long long now0; };   // first decision made in list mode; the time it was made at
+
 struct FastArgs {
     const int32_t* tok;
     int32_t n;
@@ -1277,6 +1279,8 @@ struct FastArgs {
     const int32_t* ls;            //            and the slot it belongs to
     unsigned long long* counter;  // work counter of the initial walk
     int32_t* pm; int32_t* pnode; int32_t* poff;   // per query (nullable): where its walk ended, for the insertion after the loop
+    const int64_t* arrival;       // per query: arrival (for the charge pass after the loop)
+    struct FastPost* post;        // where list mode began, for the charge pass after the loop
     TreeState* st;
 };
 
@@ -1703,7 +1707,7 @@ fast_run_kernel(FastArgs A) {
 
     // ---------------------------------------------------------------- the sequencer (warp 0)
     const long long INF = 0x7fffffffffffffffLL;
-    long long now = A.start_tick, vnext = A.vbase;
+    long long now = A.start_tick;
     int32_t head = 0, admitted = 0;
     long long next_t = __ldg(&A.stat[0].t);
     unsigned long long root = 0;
@@ -1748,19 +1752,23 @@ fast_run_kernel(FastArgs A) {
     };
     // Charge pick `slot` (Definition 2), write its outputs, and let the queries tied with it match into its new
     // leaf.  The caller has taken the slot out of the tournament or the list and marked it processed.
-    auto careful = [&](int32_t slot) {
+    auto careful = [&](int32_t slot, bool charge) {
         const FDyn d = ld_dyn(A.dyn + slot);
         const FStat s = ld_stat(A.stat + slot);
         const int32_t m = d.m, len = s.len, unc = len - m;
-        const long long begin = now > s.t ? now : s.t;
-        const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
-        now = Rj;
-        if (lane == 0) {
-            A.order[c] = s.ord; A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
-            if (A.completion) A.completion[s.ord] = Rj;
+        if (charge) {
+            const long long begin = now > s.t ? now : s.t;
+            const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
+            now = Rj;
+            if (lane == 0) {
+                A.order[c] = s.ord; A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
+                if (A.completion) A.completion[s.ord] = Rj;
+            }
+        } else if (lane == 0) {
+            A.order[c] = slot;                              // list mode: the charge pass after the loop does the rest
         }
-        const long long vleaf = vnext;
-        vnext += unc;
+        // the new leaf's positions: unique per decision, above every real pool index
+        const long long vleaf = A.vbase + ((long long)c << 32);
         ++c;
         if (unc > 0 && d.gcount > 1) {
             FastPick P;
@@ -1862,7 +1870,7 @@ fast_run_kernel(FastArgs A) {
         }
         root = tour_set(R, b, warp_max64r(bm), lane);
         mark_done(slot);
-        careful(slot);
+        careful(slot, true);
         if (slot == head) advance_head();
         __syncwarp();
     }
@@ -1891,51 +1899,11 @@ fast_run_kernel(FastArgs A) {
             ++cur;
             if ((cur & 31) == 0) { wk = nk; ws = ns; window(cur + 32, &nk, &ns); }
         };
-        // Picks whose group has no other member are charged 32 at a time.  Nobody waits for an arrival any more, so
-        // completion times are a running sum of the picks' costs (Definition 2 with R_prev >= t_j).  The p-th pick
-        // of a batch is remembered by lane p; when the batch is full every lane reads its own pick's state, the
-        // warp takes a prefix sum of the costs and writes the outputs -- one memory latency per 32 picks.
-        // The state is requested when a batch closes and used when the next one closes (or when exact times are needed),
-        // so its latency hides behind the picks in between.
-        int32_t p = 0, myj = 0;
-        int4 ps = make_int4(0, 0, 0, 0);                    // the closed batch: this lane's pick's arrival, length, query index
-        int32_t pm = 0, pend_p = 0, pend_c0 = 0;            // its match length; picks in the closed batch; its first decision
-        auto finish = [&]() {                               // charge the closed batch
-            if (!pend_p) return;
-            const bool v = lane < pend_p;
-            const int32_t len = ps.z, ord = ps.w, unc = len - pm;
-            const long long tj = (long long)(((unsigned long long)(unsigned)ps.y << 32) | (unsigned)ps.x);
-            long long x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
-            long long y = unc;
-            if (A.c_num == 0) {                             // cost = c_den tokens' worth each: one running sum serves both
-#pragma unroll
-                for (int dlt = 1; dlt < 32; dlt <<= 1) { const long long yo = __shfl_up_sync(FULL_MASK, y, dlt); if (lane >= dlt) y += yo; }
-                x = A.c_den * y;
-            } else {
-#pragma unroll
-                for (int dlt = 1; dlt < 32; dlt <<= 1) {
-                    const long long xo = __shfl_up_sync(FULL_MASK, x, dlt), yo = __shfl_up_sync(FULL_MASK, y, dlt);
-                    if (lane >= dlt) { x += xo; y += yo; }
-                }
-            }
-            const long long Rj = now + x;
-            if (v) {
-                A.order[pend_c0 + lane] = ord; A.uncached[ord] = unc; A.ttft[ord] = Rj - tj;
-                if (A.completion) A.completion[ord] = Rj;
-            }
-            now += __shfl_sync(FULL_MASK, x, 31);
-            vnext += __shfl_sync(FULL_MASK, y, 31);
-            pend_p = 0;
-        };
-        auto retire_batch = [&]() {                         // close the open batch: lanes below p hold picks c - p + lane
-            finish();
-            const bool v = lane < p;
-            ps = make_int4(0, 0, 0, 0);
-            pm = 0;
-            if (v) { ps = __ldg(reinterpret_cast<const int4*>(A.stat + myj)); pm = __ldcg(&A.dyn[myj].m); }
-            pend_p = p; pend_c0 = c - p;
-            p = 0;
-        };
+        // From here on the time of a decision influences no decision, so the loop only records which slot each
+        // decision takes (in `order`); the charge pass after the loop turns that into query indices, uncached tokens,
+        // completion times and TTFTs (Definition 2 with R_prev >= t_j is a running sum of the costs).
+        if (lane == 0) { A.post->c0 = c; A.post->now0 = now; }
+        int32_t myj = 0;
         // Up to 32 decisions at once.  As long as nothing interferes, the coming longest-match picks are the next
         // entries of the list that still count and the coming oldest-first picks are the next unprocessed slots,
         // interleaved as the policy says.  The warp gathers both sets side by side and checks that they cannot
@@ -2038,7 +2006,8 @@ fast_run_kernel(FastArgs A) {
                 atomicOr(R.skip + (myj >> 5), 1u << (myj & 31));
             }
             __syncwarp();
-            c += B; p = B;
+            if (lane < B) A.order[c + lane] = myj;
+            c += B;
             if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + B) % A.k;
             if (consumed) {
                 const int32_t ncur = cur + consumed;
@@ -2047,13 +2016,11 @@ fast_run_kernel(FastArgs A) {
             }
             if (nF > 0) { head = hmax; advance_head(); }
             else if (head < n && ((s_done[head >> 5] >> (head & 31)) & 1u)) advance_head();
-            retire_batch();
             return true;
         };
         int32_t vb_wait = 0, vb_back = 1;                   // decisions until the next attempt; doubles while attempts fail
         while (c < n && !failed) {
             if (vb_wait <= 0) {
-                if (p) retire_batch();
                 if (try_batch()) { vb_back = 1; continue; }
                 vb_wait = vb_back;
                 vb_back = vb_back < 64 ? vb_back * 2 : 64;
@@ -2097,22 +2064,85 @@ fast_run_kernel(FastArgs A) {
             }
             if (j == head) advance_head();
             if ((R.gb[j >> 5] >> (j & 31)) & 1u) {
-                if (p) retire_batch();
-                finish();
-                careful(j);
+                careful(j, false);
             } else {
-                if (lane == p) myj = j;
-                ++p; ++c;
-                if (p == 32) retire_batch();
+                if (lane == 0) A.order[c] = j;
+                ++c;
             }
         }
-        if (p) retire_batch();
-        finish();
+    } else if (lane == 0) {
+        A.post->c0 = n;                                     // list mode never began: nothing is left to charge
+        A.post->now0 = now;
     }
     __syncwarp();
     if (lane == 0) s_job.type = FAST_JOB_EXIT;
     __syncwarp();
     named_bar(1, KLPM_FAST_THREADS);
+}
+
+// The charge pass after the loop: the decisions made in list mode, c0 .. n-1, are in `order` as slots.  Nobody waited
+// for an arrival there, so completion times are the time list mode began plus a running sum of the costs
+// (Definition 2 with R_prev >= t_j).  Three small kernels: per decision its uncached tokens and cost (and the query
+// index put in `order`), a scan of the per-block sums, and the completion times and TTFTs.
+#define KLPM_CHARGE_THREADS 256
+__global__ void __launch_bounds__(KLPM_CHARGE_THREADS)
+charge_cost_kernel(FastArgs A, long long* cost, long long* bsum) {
+    __shared__ long long s_w[KLPM_CHARGE_THREADS / 32];
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x, c = A.post->c0 + i;
+    long long x = 0;
+    if (c < A.n) {
+        const int32_t slot = A.order[c];
+        const int4 s = __ldg(reinterpret_cast<const int4*>(A.stat + slot));     // arrival, length, query index
+        const int32_t len = s.z, ord = s.w, unc = len - A.dyn[slot].m;
+        x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
+        A.order[c] = ord;
+        A.uncached[ord] = unc;
+        cost[i] = x;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_down_sync(FULL_MASK, x, d);
+    if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long sum = 0;
+        for (int w = 0; w < KLPM_CHARGE_THREADS / 32; ++w) sum += s_w[w];
+        bsum[blockIdx.x] = sum;
+    }
+}
+// bsum[b] <- time at which block b's first decision starts (at most 1,024 blocks)
+__global__ void __launch_bounds__(1024)
+charge_scan_kernel(FastArgs A, long long* bsum, int32_t nblocks) {
+    __shared__ long long s[1024];
+    const int u = threadIdx.x;
+    const long long v = u < nblocks ? bsum[u] : 0;
+    s[u] = v;
+    __syncthreads();
+    for (int d = 1; d < 1024; d <<= 1) {
+        const long long o = u >= d ? s[u - d] : 0;
+        __syncthreads();
+        s[u] += o;
+        __syncthreads();
+    }
+    if (u < nblocks) bsum[u] = A.post->now0 + s[u] - v;
+}
+__global__ void __launch_bounds__(KLPM_CHARGE_THREADS)
+charge_apply_kernel(FastArgs A, const long long* cost, const long long* bsum) {
+    __shared__ long long s_w[KLPM_CHARGE_THREADS / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x, c = A.post->c0 + i;
+    long long x = c < A.n ? cost[i] : 0;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const long long o = __shfl_up_sync(FULL_MASK, x, d); if (lane >= d) x += o; }
+    if (lane == 31) s_w[warp] = x;
+    __syncthreads();
+    long long before = bsum[blockIdx.x];
+    for (int w = 0; w < warp; ++w) before += s_w[w];
+    if (c < A.n) {
+        const int32_t ord = A.order[c];
+        const long long Rj = before + x;
+        A.ttft[ord] = Rj - A.arrival[ord];
+        if (A.completion) A.completion[ord] = Rj;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -2386,6 +2416,7 @@ struct rt_tree {
     FDyn* fast_dyn; FStat* fast_stat; unsigned long long* fast_key_arr; int32_t* fast_mem;
     long long* fast_gh; int32_t* fast_gidx; unsigned int* fast_done; unsigned long long* fast_counter;
     long long* fast_lk; int32_t* fast_ls;
+    FastPost* fast_post; long long* fast_bsum;
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -2425,7 +2456,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->run_partial); cudaFree(t->run_bc); cudaFree(t->run_sy);
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
-    cudaFree(t->fast_lk); cudaFree(t->fast_ls);
+    cudaFree(t->fast_lk); cudaFree(t->fast_ls); cudaFree(t->fast_post); cudaFree(t->fast_bsum);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
     cudaFree(t->bulk_n_out);
@@ -2484,6 +2515,8 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_counter, 1))) return s;
     if ((s = dalloc(&t->fast_lk, np2))) return s;
     if ((s = dalloc(&t->fast_ls, np2))) return s;
+    if (!t->fast_post && (s = dalloc(&t->fast_post, 1))) return s;
+    if (!t->fast_bsum && (s = dalloc(&t->fast_bsum, 1024))) return s;
     t->fast_cap = np2;
     return RT_OK;
 }
@@ -2948,6 +2981,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.pinv = d_tie_priority ? tree->run_pinv : nullptr;
         f.gh = tree->fast_gh; f.gidx = tree->fast_gidx; f.done = tree->fast_done; f.counter = tree->fast_counter;
         f.pm = tree->bulk_pm; f.pnode = tree->bulk_pnode; f.poff = tree->bulk_poff;
+        f.arrival = d_arrival; f.post = tree->fast_post;
         f.vbase = tree->dev.max_pool + 16;
         f.st = tree->dev.st;
         // every query is matched once against the tree as it stands
@@ -2991,6 +3025,12 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         CK(cudaGetLastError());
         CK(cudaFuncSetAttribute(fast_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         fast_run_kernel<<<1, KLPM_FAST_THREADS, smem, s>>>(f);
+        if (f.list_mode) {           // the decisions made in list mode are charged here (none if list mode never began)
+            const int32_t cblocks = (n + KLPM_CHARGE_THREADS - 1) / KLPM_CHARGE_THREADS;      // at most 1,024: list mode ends at 262,144 queries
+            charge_cost_kernel<<<cblocks, KLPM_CHARGE_THREADS, 0, s>>>(f, tree->fast_gh, tree->fast_bsum);
+            charge_scan_kernel<<<1, 1024, 0, s>>>(f, tree->fast_bsum, cblocks);
+            charge_apply_kernel<<<cblocks, KLPM_CHARGE_THREADS, 0, s>>>(f, tree->fast_gh, tree->fast_bsum);
+        }
         CK(cudaGetLastError());
         tree->run_path = 2;
         // The processed prompts enter the tree together (the logical clock advances by n).  The loop itself needs
