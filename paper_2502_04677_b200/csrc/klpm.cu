@@ -2200,6 +2200,10 @@ __global__ void bulk_prewalked_kernel(BulkArgs A, unsigned n_pending) {
 
 __global__ void __launch_bounds__(256)
 bulk_apply_kernel(TreeDev T, BulkArgs A) {
+    // live nodes and live tokens are statistics only: summed per CTA here, added to the tree's counters once at the end
+    __shared__ unsigned long long s_live_nodes, s_live_tokens;
+    if (threadIdx.x == 0) { s_live_nodes = 0ULL; s_live_tokens = 0ULL; }
+    __syncthreads();
     const unsigned n_pending = *A.n_out;
     const int lane = threadIdx.x & 31;
     const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -2222,7 +2226,7 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                     const long long u = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
                     if (u >= T.max_nodes) { set_status(S, RT_ERR_CAPACITY); go = false; }
                     else {
-                        atomicAdd((unsigned long long*)&S->live_nodes, 1ULL);
+                        atomicAdd(&s_live_nodes, 1ULL);
                         const int32_t par = T.parent[node], ds = T.depth_start[node], sl = T.span_len[node];
                         const int64_t so = T.span_off[node];
                         T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
@@ -2275,8 +2279,8 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
                         T.table[won].chain_end = po + unc;
                         T.end_node[po + unc - 1] = (int32_t)leaf;
                         atomicAdd(&T.nchild[end], 1);
-                        atomicAdd((unsigned long long*)&S->tokens_live, (unsigned long long)unc);
-                        atomicAdd((unsigned long long*)&S->live_nodes, 1ULL);
+                        atomicAdd(&s_live_tokens, (unsigned long long)unc);
+                        atomicAdd(&s_live_nodes, 1ULL);
                         dst = po;
                     }
                 }
@@ -2286,6 +2290,11 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
         dst = __shfl_sync(FULL_MASK, dst, 0);
         if (dst >= 0)
             for (int32_t t = lane; t < unc; t += 32) T.pool[dst + t] = __ldg(x + m + t);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (s_live_nodes) atomicAdd((unsigned long long*)&S->live_nodes, s_live_nodes);
+        if (s_live_tokens) atomicAdd((unsigned long long*)&S->tokens_live, s_live_tokens);
     }
 }
 
