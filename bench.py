@@ -297,14 +297,14 @@ def run_ours(args):
         # match; slot keys, arrival sort, slot arrays; slot records, walk of every query, group sort, groups,
         # key list and its sort (queues up to 262,144), the loop; bulk insertion of the processed prompts: claim
         # words, pending list, at least one round of two kernels, clock
-        list_launches = 1 + sort_launches if nq <= 262144 else 0
+        list_launches = 1 + sort_launches + 3 if nq <= 262144 else 0       # key list, its sort, the three charge kernels
         launches_per_step = 1 + (1 + sort_launches + 1) + (1 + 1 + sort_launches + 1 + list_launches + 1) + (1 + 1 + 2 + 1)
         loop_kernel = "fast_run_kernel"
         loop_note = ("all decisions in one CTA: once everybody has arrived, longest-match picks come from a presorted list "
                      "of keys and oldest-first picks from a bitmap cursor, up to 32 decisions per warp-wide step when they "
-                     "cannot interfere; picks whose group has other members take a careful step; bound by the instruction "
-                     "issue of one warp; the time includes the walk of every query, three sorts and the bulk insertion of "
-                     "the processed prompts")
+                     "cannot interfere; picks whose group has other members take a careful step; those decisions are "
+                     "charged by a parallel pass after the loop; bound by the instruction issue of one warp; the time "
+                     "includes the walk of every query, three sorts and the bulk insertion of the processed prompts")
     else:
         launches_per_step = 1 + 1 + sort_launches + 1 + 1      # match, slot keys, bitonic steps, slot arrays, scheduling loop
         loop_kernel = "run_kernel"
