@@ -62,3 +62,64 @@ def test_full_size_configuration_is_bit_exact(name):
         for f in ("n_nodes", "tokens", "clock", "evictions"):
             assert after[f] == want["tree_after"][f], (key, f)
     K.rt_destroy(tree)
+
+
+def test_adversarial_full_size_properties_and_both_loops(monkeypatch):
+    """The bench's own configuration (262,144 queries, k = 4) is too large for the CPU oracle's schedule, so the
+    scheduling loop is checked there through what holds at any size -- the order is a permutation; every k-th
+    decision takes the oldest unprocessed query (everybody is waiting); every other decision takes a query whose
+    uncached-token count is consistent with its stored match; the uncached tokens add up to the growth of the
+    tree; completion times are the running sum of the uncached tokens (1 tick per token) and TTFT = completion -
+    arrival -- and through bit-exact agreement of the two device loops (the one-by-one loop is the one the oracle
+    checks at the smaller sizes)."""
+    import bench
+    from paper_2502_04677_b200 import binding as K
+    w = W.adversarial(scale=1.0)
+    device = torch.device("cuda", 0)
+    tree, q_tok, q_off, arr = bench.device_workload(w, device)
+    nq, k = w.queries.n, 4
+    before = K.rt_stats(tree)
+    outs = []
+    for legacy in (False, True):
+        if legacy:
+            monkeypatch.setenv("KLPM_RUN_LEGACY", "1")
+        else:
+            monkeypatch.delenv("KLPM_RUN_LEGACY", raising=False)
+        K.rt_rollback(tree)
+        order = torch.full((nq,), -1, dtype=torch.int32, device=device)
+        unc = torch.full((nq,), -1, dtype=torch.int32, device=device)
+        ttft = torch.full((nq,), -1, dtype=torch.int64, device=device)
+        comp = torch.full((nq,), -1, dtype=torch.int64, device=device)
+        K.klpm_run(tree, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), order, unc, ttft, comp)
+        assert K.rt_sync_status(tree) == 0
+        assert K.klpm_run_path(tree) == (K.RUN_PATH_ONE_BY_ONE if legacy else K.RUN_PATH_GROUPED)
+        outs.append((order.cpu(), unc.cpu(), ttft.cpu(), comp.cpu(), K.rt_stats(tree)))
+    monkeypatch.delenv("KLPM_RUN_LEGACY", raising=False)
+    order, unc, ttft, comp, after = outs[0]
+    for a, b in zip(outs[0][:4], outs[1][:4]):
+        assert torch.equal(a, b)
+    assert {f: outs[0][4][f] for f in ("n_nodes", "tokens", "clock")} == {f: outs[1][4][f] for f in ("n_nodes", "tokens", "clock")}
+    o = order.numpy().astype(np.int64)
+    assert np.array_equal(np.sort(o), np.arange(nq))
+    # everybody has arrived (start_tick = last arrival): the oldest unprocessed query by (arrival, index)
+    a = arr.cpu().numpy()
+    rank = np.empty(nq, dtype=np.int64)
+    rank[np.lexsort((np.arange(nq), a))] = np.arange(nq)
+    done = np.zeros(nq, dtype=bool)
+    by_rank = np.argsort(rank)
+    ptr = 0
+    for c in range(nq):
+        if c % k == 0:
+            while done[by_rank[ptr]]:
+                ptr += 1
+            assert o[c] == by_rank[ptr], c
+        done[o[c]] = True
+    u = unc.numpy().astype(np.int64)
+    lens = (q_off[1:] - q_off[:-1]).cpu().numpy()
+    assert np.all(u >= 0) and np.all(u <= lens)
+    assert int(u.sum()) == after["tokens"] - before["tokens"]
+    assert after["clock"] == before["clock"] + nq
+    cm = comp.numpy()
+    assert np.array_equal(cm[o], w.start_tick + np.cumsum(u[o]))
+    assert np.array_equal(ttft.numpy(), cm - a)
+    K.rt_destroy(tree)
