@@ -1911,7 +1911,7 @@ fast_run_kernel(FastArgs A) {
         // have influenced each other: no slot in both (a list entry inside the range of slots the oldest-first
         // picks consume), none whose group has other members, none whose key sits in the tournament, and the
         // tournament's root below the smallest key taken from the list.  The batch is cut before the first decision
-        // that fails a check; then lane i makes decision c + i.  If fewer than four decisions are left that way,
+        // that fails a check; then lane i makes decision c + i.  If fewer than two decisions are left that way,
         // nothing has been changed and the next decisions are made one at a time below.
         const int32_t lane_div_k = lane / A.k;              // y / k for y = 0..31, looked up by shuffle
         auto try_batch = [&]() -> bool {
@@ -1942,7 +1942,7 @@ fast_run_kernel(FastArgs A) {
             // as many decisions as those entries allow: lane x asks whether x + 1 decisions need no more of them
             const int32_t avail = __popc(mask);
             const int32_t B0 = __popc(__ballot_sync(FULL_MASK, c + lane < n && (lane + 1) - f_hi <= avail));
-            if (B0 < 4) return false;
+            if (B0 < 2) return false;
             const int32_t nF0 = __shfl_sync(FULL_MASK, f_hi, B0 - 1), nL0 = B0 - nF0;
             // the next nF0 unprocessed slots; limF = how many of them can be taken before one needs the careful step
             int32_t hs = -1, hmax0 = -1, limF = nF0;
@@ -1990,7 +1990,7 @@ fast_run_kernel(FastArgs A) {
                 if (badE) limL = __popc(mask & ((1u << (__ffs(badE) - 1)) - 1u));
             }
             const int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_hi <= limF && (lane + 1) - f_hi <= limL));
-            if (B < 4) return false;
+            if (B < 2) return false;
             const int32_t nF = __shfl_sync(FULL_MASK, f_hi, B - 1), nL = B - nF;
             const int32_t hmax = nF > 0 ? __shfl_sync(FULL_MASK, hs, nF - 1) : -1;
             if (lane < nF) s_H[lane] = hs;
