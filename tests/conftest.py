@@ -10,6 +10,12 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
+    # the CUDA library is built in-tree; build it if it is missing or older than its source (nvcc needs no GPU)
+    try:
+        from paper_2502_04677_b200 import build
+        build.build()
+    except Exception as e:      # the tests that need the library will say so themselves
+        print("libklpm.so could not be built: %s" % e)
 
 
 def pytest_collection_modifyitems(config, items):
