@@ -186,6 +186,8 @@ def run_ours(args):
     if multi:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
+    from paper_2502_04677_b200 import build
+    build.build()                      # in-tree library: a no-op when it is up to date (each rank writes its own temporary file)
     from paper_2502_04677_b200 import binding as K
 
     name = args.workload
