@@ -1494,7 +1494,33 @@ struct FastPick {             // the prompt being processed, as its group's memb
     int32_t gstart, gcount;
 };
 struct FastJob { int32_t type; int32_t a0, a1; FastPick pick; };
-enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2, FAST_JOB_REBUILD = 3 };
+enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2, FAST_JOB_REBUILD = 3, FAST_JOB_BATCH = 4 };
+
+// What the sequencer hands to a CTA-wide batch of decisions, and what it gets back.
+struct FastBatchIO {
+    int32_t cur, head, c, cyc;        // in: list cursor, oldest unprocessed slot, decisions made, c mod k
+    unsigned long long root;          // in: largest key in the tournament
+    int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
+    int32_t B0, nF0, nL0, limF, limL; // scratch
+};
+#define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
+#define KLPM_FAST_CTA_MIN 128         // smaller batches are left to the warp-wide step (an attempt costs about 5,000 cycles)
+
+// Exclusive prefix sum of v over the CTA's 256 threads; *total receives the sum.  s_w: 8 ints of shared scratch.
+__device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* s_w, int32_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const int32_t o = __shfl_up_sync(FULL_MASK, inc, d); if (lane >= d) inc += o; }
+    __syncthreads();                   // s_w may still be read from an earlier scan
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    int32_t before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < KLPM_FAST_THREADS / 32; ++w) { const int32_t x = s_w[w]; if (w < warp) before += x; all += x; }
+    *total = all;
+    return before + inc - v;
+}
 
 // One member of the dissolving group per lane (r < 0: none).  Members tied with the processed prompt are
 // compared with its uncached tokens and get their new state and key; every live member gets the hash of the
@@ -1530,6 +1556,102 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
     }
     if (!live) return KLPM_FAST_NOGROUP;
     return d.m < s.len ? group_hash(d.pos, d.ntok) : single_hash(r);
+}
+
+// The warp-wide step of list mode (see fast_run_kernel) with the whole CTA: 1,024 list entries and 8,192 bitmap slots
+// are examined at once, the same checks cut the batch short, block-wide prefix sums replace the warp's ballots.
+// Every thread calls it.  Nothing is changed unless at least KLPM_FAST_CTA_MIN decisions can be made.
+__device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO* io, int32_t* sH, int32_t* sE, int32_t* sEpos,
+                               int32_t* s_w, int32_t nwords) {
+    const int tid = threadIdx.x;
+    const int32_t n = A.n, cur = io->cur, head = io->head, c = io->c, cyc = io->cyc;
+    const unsigned long long root = io->root;
+    auto f = [&](int32_t x) -> int32_t {                  // oldest-first turns among the next x decisions
+        if (A.policy == KLPM_POLICY_FCFS) return x;
+        if (A.policy == KLPM_POLICY_LPM) return 0;
+        const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;
+        return x > i0 ? (x - i0 - 1) / A.k + 1 : 0;
+    };
+    // the list entries cur + 4 tid .. + 3 that still count
+    long long kk[4]; int32_t es[4]; bool ok[4];
+    int32_t cnt = 0;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const long long idx = (long long)cur + tid * 4 + r;
+        ok[r] = false; kk[r] = 0; es[r] = 0;
+        if (idx < n) {
+            kk[r] = __ldg(A.lk + idx); es[r] = __ldg(A.ls + idx);
+            ok[r] = !((R.skip[es[r] >> 5] >> (es[r] & 31)) & 1u);
+        }
+        cnt += ok[r];
+    }
+    int32_t avail;
+    const int32_t base = block_excl_scan(cnt, s_w, &avail);
+    if (tid == 0) {                                       // as many decisions as those entries allow
+        int32_t lo = 0, hi = n - c < KLPM_FAST_CTA_BATCH ? n - c : KLPM_FAST_CTA_BATCH;
+        while (lo < hi) { const int32_t mid = (lo + hi + 1) >> 1; if (mid - f(mid) <= avail) lo = mid; else hi = mid - 1; }
+        io->B0 = lo; io->nF0 = f(lo); io->nL0 = lo - f(lo);
+        io->limF = io->nF0; io->limL = io->nL0;
+    }
+    __syncthreads();
+    const int32_t B0 = io->B0, nF0 = io->nF0, nL0 = io->nL0;
+    // the next nF0 unprocessed slots (each thread one bitmap word from head on), in order
+    int32_t hmax0 = -1;
+    if (nF0 > 0) {
+        const int32_t w0 = head >> 5, wi = w0 + tid;
+        unsigned w = wi < nwords ? R.done[wi] : 0xffffffffu;
+        if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
+        if (wi == w0) w |= (1u << (head & 31)) - 1u;
+        unsigned fr = ~w;
+        int32_t nfree;
+        int32_t qk = block_excl_scan(__popc(fr), s_w, &nfree);
+        while (fr && qk < nF0) { const int bit = __ffs(fr) - 1; fr &= fr - 1; sH[qk++] = wi * 32 + bit; }
+        const int32_t nFa = nfree < nF0 ? nfree : nF0;
+        if (tid == 0 && nFa < nF0) io->limF = nFa;
+        __syncthreads();
+        if (nFa > 0) hmax0 = sH[nFa - 1];
+        for (int32_t qi = tid; qi < nFa; qi += KLPM_FAST_THREADS) {       // key in the tournament, or grouped: needs the careful step
+            const int32_t hs = sH[qi];
+            if (((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u) atomicMin(&io->limF, qi);
+        }
+    }
+    // the usable entries by rank; the first one that is grouped, could also be an oldest-first pick of this batch, or
+    // lies below the tournament's root limits the batch
+    {
+        int32_t rk = base;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            if (ok[r]) {
+                if (rk < nL0) {
+                    sE[rk] = es[r]; sEpos[rk] = tid * 4 + r;
+                    const unsigned long long ek = ~((unsigned long long)kk[r] ^ 0x8000000000000000ULL);
+                    if ((((R.gb[es[r] >> 5] >> (es[r] & 31)) & 1u)) || (es[r] >= head && es[r] <= hmax0) || root > ek) atomicMin(&io->limL, rk);
+                }
+                ++rk;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int32_t limF = io->limF, limL = io->limL;
+        int32_t lo = 0, hi = B0;
+        while (lo < hi) { const int32_t mid = (lo + hi + 1) >> 1; if (f(mid) <= limF && mid - f(mid) <= limL) lo = mid; else hi = mid - 1; }
+        const int32_t B = lo >= KLPM_FAST_CTA_MIN ? lo : 0;
+        const int32_t nF = f(B), nL = B - nF;
+        io->B = B;
+        io->consumed = nL > 0 ? sEpos[nL - 1] + 1 : 0;
+        io->hmax = nF > 0 ? sH[nF - 1] : -1;
+    }
+    __syncthreads();
+    const int32_t B = io->B;
+    for (int32_t x = tid; x < B; x += KLPM_FAST_THREADS) {   // thread makes decisions c + x
+        const int32_t f0 = f(x);
+        const int32_t slot = f(x + 1) > f0 ? sH[f0] : sE[x - f0];
+        atomicOr(R.done + (slot >> 5), 1u << (slot & 31));
+        atomicOr(R.skip + (slot >> 5), 1u << (slot & 31));
+        A.order[c + x] = slot;
+    }
+    __syncthreads();
 }
 
 // Work the whole CTA shares; every thread calls it with the same job.  Ends with t2 recomputed from t1.
@@ -1677,6 +1799,8 @@ fast_run_kernel(FastArgs A) {
     __shared__ FastJob s_job;
     __shared__ int s_cnt;
     __shared__ int32_t s_H[32], s_E[32];      // a batch's oldest-first and longest-match picks, by rank
+    __shared__ FastBatchIO s_bio;             // a CTA-wide batch: what the sequencer hands over and gets back
+    __shared__ int32_t s_scan[KLPM_FAST_THREADS / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t n = A.n;
     const int32_t nb1p = (A.nb + 31) & ~31, n2 = nb1p >> 5, n2p = (n2 + 31) & ~31, n3 = n2p >> 5;
@@ -1702,6 +1826,7 @@ fast_run_kernel(FastArgs A) {
             named_bar(1, KLPM_FAST_THREADS);
             const FastJob J = s_job;
             if (J.type == FAST_JOB_EXIT) return;
+            if (J.type == FAST_JOB_BATCH) { fast_batch_job(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords); continue; }
             fast_job(A, R, J, sh, sr, &s_cnt);
         }
     }
@@ -2020,9 +2145,38 @@ fast_run_kernel(FastArgs A) {
             return true;
         };
         int32_t vb_wait = 0, vb_back = 1;                   // decisions until the next attempt; doubles while attempts fail
+        int32_t cb_wait = 0, cb_back = 8;                   // the same for the CTA-wide batch (loop iterations; 8 .. 1,024)
+        int32_t calm = 4;                                   // consecutive full warp-wide steps: the CTA-wide batch is tried in calm water only
         while (c < n && !failed) {
+            // first choice: the whole CTA makes up to 1,024 decisions (the sort scratch is free between dissolves)
+            if (cb_wait <= 0 && calm >= 4 && n - c >= KLPM_FAST_CTA_MIN) {
+                if (lane == 0) {
+                    s_bio.cur = cur; s_bio.head = head; s_bio.c = c; s_bio.cyc = cyc; s_bio.root = root; s_bio.B = 0;
+                    s_job.type = FAST_JOB_BATCH;
+                }
+                __syncwarp();
+                named_bar(1, KLPM_FAST_THREADS);
+                fast_batch_job(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords);
+                const int32_t Bc = s_bio.B;
+                if (Bc > 0) {
+                    const int32_t consumed = s_bio.consumed, hmax = s_bio.hmax;
+                    c += Bc;
+                    if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + Bc) % A.k;
+                    if (consumed) { cur += consumed; window(cur & ~31, &wk, &ws); window((cur & ~31) + 32, &nk, &ns); }
+                    if (hmax >= 0) { head = hmax; advance_head(); }
+                    else if (head < n && ((s_done[head >> 5] >> (head & 31)) & 1u)) advance_head();
+                    cb_back = 8;
+                    continue;
+                }
+                cb_wait = cb_back;
+                cb_back = cb_back < 1024 ? cb_back * 2 : 1024;
+                calm = 0;
+            }
+            --cb_wait;
             if (vb_wait <= 0) {
-                if (try_batch()) { vb_back = 1; continue; }
+                const int32_t c_was = c;
+                if (try_batch()) { vb_back = 1; calm = c - c_was == 32 ? calm + 1 : 0; continue; }
+                calm = 0;
                 vb_wait = vb_back;
                 vb_back = vb_back < 64 ? vb_back * 2 : 64;
             }
