@@ -1791,8 +1791,9 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
 // loop changes to list mode: all keys were sorted before the loop, so the longest-match pick is the next entry of
 // that list that is still unprocessed and whose key has not changed since; the tournament is cut down to the slots
 // whose key has changed (members of dissolved groups) and the pick is the larger of the two candidates.  A pick
-// from the list touches no tournament at all, up to 32 decisions are made by one warp-wide step, and the loop only
-// records which slot each decision takes: the charge pass after the loop computes their outputs.
+// from the list touches no tournament at all, up to 32 decisions are made by one warp-wide step (up to 1,024 by a
+// CTA-wide one, fast_batch_job), and the loop only records which slot each decision takes: the charge pass after the
+// loop computes their outputs.
 __global__ void __launch_bounds__(KLPM_FAST_THREADS, 1)
 fast_run_kernel(FastArgs A) {
     extern __shared__ __align__(16) unsigned char fast_smem[];
