@@ -56,6 +56,8 @@ def lib():
         L.oc_tree_insert.argtypes = [vp, vp, vp, i32, vp]
         L.oc_tree_match.restype = None
         L.oc_tree_match.argtypes = [vp, vp, vp, i32, vp, i32]
+        L.oc_tree_match_pos.restype = None
+        L.oc_tree_match_pos.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.oc_replay.restype = i32
         L.oc_replay.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, i64, i64, i32, vp, vp, vp]
         L.oc_batch_times.restype = None
@@ -124,6 +126,15 @@ class OracleTree:
         lib().oc_tree_match(self._h, _p(t), _p(o), len(o) - 1, _p(out), threads)
         return out
 
+    def match_pos(self, tokens, offsets) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """match() plus where each match ended: (match_len, term_off, term_depth) -- how many tokens of the edge
+        holding the last matched token were matched, and how many tokens lie on the path above that edge."""
+        t, o = _i32(tokens), _i64(offsets)
+        n = len(o) - 1
+        m, off, depth = (np.zeros(n, dtype=np.int32) for _ in range(3))
+        lib().oc_tree_match_pos(self._h, _p(t), _p(o), n, _p(m), _p(off), _p(depth))
+        return m, off, depth
+
     def stats(self) -> dict:
         v = [ctypes.c_int64() for _ in range(4)]
         lib().oc_tree_stats(self._h, *[ctypes.byref(x) for x in v])
@@ -136,7 +147,7 @@ def schedule(tokens, offsets, arrivals, policy: int, k: int = 1, c_num: int = 0,
              ) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
     """Run FCFS / LPM / k-LPM over the stream.  Returns order, uncached, ttft, completion.
     tie_priority (optional int64 per query): smaller wins among equal scores of a longest-match pick.
-    score_mode 1: the score is the hit rate floor(match * 2^31 / length) instead of the match length."""
+    score_mode 1: the score is the hit rate match / length (an exact rational) instead of the match length."""
     t, o, a = _i32(tokens), _i64(offsets), _i64(arrivals)
     n = len(o) - 1
     if cache_mode == CACHE_TREE and tree is None:

@@ -20,6 +20,7 @@ count are recomputed from the set whenever they are needed.
 """
 from __future__ import annotations
 
+from fractions import Fraction
 from typing import Dict, List, Optional, Sequence, Tuple
 
 FCFS, LPM, KLPM = 0, 1, 2
@@ -44,6 +45,18 @@ class StringSetCache:
 
     def match(self, x: Sequence[int]) -> int:
         return max([overlap(x, s) for s in self.nodes] + [0])
+
+    def match_pos(self, x: Sequence[int]) -> Tuple[int, int, int]:
+        """(m, off, depth): the match length, how many tokens of the edge that holds the last matched token
+        were matched, and how many tokens lie above that edge.  The edge belongs to the shortest node-end
+        string that extends x[:m]; its parent is that string's longest proper prefix in the set."""
+        x = tuple(x)
+        m = self.match(x)
+        if m == 0:
+            return 0, 0, 0
+        holder = min((s for s in self.nodes if len(s) >= m and s[:m] == x[:m]), key=len)
+        depth = len(self.parent(holder))
+        return m, m - depth, depth
 
     def parent(self, s: Tuple[int, ...]) -> Tuple[int, ...]:
         best: Tuple[int, ...] = ()
@@ -123,8 +136,8 @@ def schedule(prompts: Sequence[Sequence[int]], arrivals: Sequence[int], policy: 
         else:
             def score(i):
                 mi = match(prompts[i])
-                if score_mode == 1:
-                    return (mi << 31) // len(prompts[i]) if len(prompts[i]) else 0
+                if score_mode == 1:         # the prompt's hit rate, an exact rational (0 for an empty prompt)
+                    return Fraction(mi, len(prompts[i])) if len(prompts[i]) else Fraction(0)
                 return mi
             j = min(waiting, key=lambda i: (-score(i), tie_priority[i] if tie_priority is not None else 0, arrivals[i], i))
         x = prompts[j]

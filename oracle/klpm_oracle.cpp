@@ -19,7 +19,8 @@
 // Readings taken where the paper is silent (the same list is in the design notes):
 //   * Algorithm 1 is followed as printed: one oldest-first pick, then k-1
 //     longest-match picks; the pick counter never resets (idle periods included).
-//   * "prefix cache hit rate" is the absolute match length in tokens.
+//   * "prefix cache hit rate" is the absolute match length in tokens; the other reading
+//     (score_mode 1) is the rational m / |x|, compared exactly by cross-multiplication.
 //   * ties go to the earliest arrival, then to the lower index.
 //   * processing starts at start_tick with the given cache; the recurrence of
 //     Definition 2 is applied to the first processed query too.
@@ -31,7 +32,7 @@
 //     and is therefore never evicted; single-child nodes are not merged.
 //   * processing x with match length m puts node boundaries at depth m and |x|.
 //
-// Parity pins (tests/test_oracle_*.py): brute-force LCP against every cached
+// Parity pins (the CPU test-suite): brute-force LCP against every cached
 // prompt; the printed toy example; k=1 -> FCFS and k>n -> LPM limits; the
 // closed forms of the proof of Theorem 2; exhaustive permutation search;
 // the NP-hardness gadget worked by hand.  The LRU reading has no value in the
@@ -255,6 +256,19 @@ void oc_tree_match(void* tp, const tok_t* tok, const int64_t* off, int32_t n, in
     for (auto& th : pool) th.join();
 }
 
+// The same walk, also reporting where each match ended: term_off[i] = how many tokens of the edge that holds the
+// last matched token were matched (0 when nothing matched), term_depth[i] = tokens on the path above that edge.
+void oc_tree_match_pos(void* tp, const tok_t* tok, const int64_t* off, int32_t n, int32_t* match_len,
+                       int32_t* term_off, int32_t* term_depth) {
+    const Tree& t = *(Tree*)tp;
+    for (int32_t i = 0; i < n; ++i) {
+        Pos p = walk(t, tok + off[i], off[i + 1] - off[i]);
+        match_len[i] = p.m;
+        term_off[i] = p.off;
+        term_depth[i] = p.m - p.off;
+    }
+}
+
 // Definition 2 along a given processing order.  The cache starts as `tp` holds it (TREE) or empty (LAST_ONLY).
 int32_t oc_replay(void* tp, const int32_t* order, int32_t n_order, const tok_t* tok, const int64_t* off,
                   const int64_t* arrival, int32_t n, int64_t c_num, int64_t c_den, int64_t start_tick,
@@ -302,8 +316,8 @@ void oc_batch_times(const int32_t* order, int32_t n_order, const int64_t* arriva
 //   tie_priority (nullable): among queries with the same score the one with the smallest priority wins, before
 //     arrival and index decide.  With priorities drawn at random this is the uniform tie-breaking the paper
 //     assumes for LPM (footnote to Theorem 2); the numbers are an input, nothing is drawn here.
-//   score_mode 0: score = match length (tokens).  score_mode 1: score = hit rate of the prompt, quantised to
-//     floor(match * 2^31 / |x|) (0 for an empty prompt) -- the other reading of "prefix cache hit rate".
+//   score_mode 0: score = match length (tokens).  score_mode 1: score = hit rate of the prompt, the rational
+//     match / |x| (0 for an empty prompt), compared exactly -- the other reading of "prefix cache hit rate".
 int32_t oc_schedule_ex(void* tp, const tok_t* tok, const int64_t* off, const int64_t* arrival, int32_t n,
                        int32_t policy, int32_t k, int64_t c_num, int64_t c_den, int64_t start_tick,
                        int32_t cache_mode, int32_t tier, const int64_t* tie_priority, int32_t score_mode,
@@ -343,19 +357,21 @@ int32_t oc_schedule_ex(void* tp, const tok_t* tok, const int64_t* off, const int
             for (int32_t i = 0; i < n; ++i)
                 if (waiting[i] && (j < 0 || earlier(s, i, j))) j = i;
         } else {
-            int64_t best = -1;
+            int64_t best_num = 0, best_den = 1;     // score of j as a fraction (denominator 1 for match lengths)
             for (int32_t i = 0; i < n; ++i) {
                 if (!waiting[i]) continue;
                 int32_t mi = tier == TIER_UPDATE ? m[i] : match_now(i);
                 if (tier != TIER_UPDATE) m[i] = mi;
-                int64_t score = mi;
-                if (score_mode == 1) score = s.len(i) > 0 ? ((int64_t)mi << 31) / s.len(i) : 0;
-                bool wins = j < 0 || score > best;
-                if (!wins && score == best) {
+                int64_t num = mi, den = 1;
+                if (score_mode == 1) { if (s.len(i) > 0) den = s.len(i); else num = 0; }
+                // num/den against best_num/best_den, exactly (all four are below 2^31)
+                const int64_t lhs = num * best_den, rhs = best_num * den;
+                bool wins = j < 0 || lhs > rhs;
+                if (!wins && lhs == rhs) {
                     if (tie_priority && tie_priority[i] != tie_priority[j]) wins = tie_priority[i] < tie_priority[j];
                     else wins = earlier(s, i, j);
                 }
-                if (wins) { j = i; best = score; }
+                if (wins) { j = i; best_num = num; best_den = den; }
             }
         }
 

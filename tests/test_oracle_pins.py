@@ -79,6 +79,38 @@ def test_match_invariants():
     assert after.tolist() == [max(int(b), D.overlap(q, p)) for b, q in zip(before, queries)]
 
 
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("budget", [0, 36])
+def test_where_a_match_ends_against_the_string_set_model(seed, budget):
+    """The edge that holds the last matched token: how far into it the match goes and how deep it starts.
+    Pointer tree vs the set-of-strings model (node = shortest node-end string extending the matched part)."""
+    cached, _ = W.random_small_queue(seed + 700, 50, vocab=2, max_len=13, min_len=1)
+    queries, _ = W.random_small_queue(seed + 800, 70, vocab=2, max_len=16)
+    model = D.StringSetCache(budget)
+    tree = oracle.OracleTree(budget)
+    for p in cached:
+        model.process(p)
+        tree.insert(*csr([p]))
+    m, off, depth = tree.match_pos(*csr(queries))
+    want = [model.match_pos(q) for q in queries]
+    assert list(zip(m.tolist(), off.tolist(), depth.tolist())) == want
+    assert m.tolist() == tree.match(*csr(queries)).tolist()
+    assert any(0 < o for _, o, _ in want) and any(d > 0 for _, _, d in want)
+    if budget:
+        assert model.evictions > 0
+
+
+def test_where_a_match_ends_by_hand():
+    """Tree of "abcd" and "abxy": nodes "ab" (depth 0), "cd" and "xy" (depth 2)."""
+    tree = oracle.OracleTree()
+    tree.insert(*csr([[1, 2, 3, 4], [1, 2, 7, 8]]))
+    qs = [[1], [1, 2], [1, 2, 3], [1, 2, 7, 8, 9], [5], [], [1, 2, 9]]
+    m, off, depth = tree.match_pos(*csr(qs))
+    assert m.tolist() == [1, 2, 3, 4, 0, 0, 2]
+    assert off.tolist() == [1, 2, 1, 2, 0, 0, 2]
+    assert depth.tolist() == [0, 0, 2, 2, 0, 0, 0]
+
+
 # ---------------------------------------------------------------- the printed toy example
 
 def _read_toy():
@@ -257,6 +289,44 @@ def test_three_partition_gadget_feasible_order():
     assert max(oracle.replay(bad, t, o, arr, cache_mode=oracle.CACHE_LAST_ONLY)[1]) > T
 
 
+# ---------------------------------------------------------------- Definition 2 along a fixed order, tree cache
+
+def test_replay_with_the_tree_cache_by_hand():
+    """Budget 6, order 0,1,2,3.  111 and 222 fill the cache (R = 3, 6).  115 matches "11": the edge 111 is cut,
+    the stale lower "1" is the oldest leaf and goes (1 token), leaf "5" is charged 1 token (R = 7).  333 arrives at
+    20: 222 is evicted, processing starts at 20 (R = 23, TTFT 3)."""
+    prompts, arr = [[1, 1, 1], [2, 2, 2], [1, 1, 5], [3, 3, 3]], [0, 0, 0, 20]
+    t, o = csr(prompts)
+    tree = oracle.OracleTree(6)
+    unc, ttft, comp = oracle.replay([0, 1, 2, 3], t, o, arr, cache_mode=oracle.CACHE_TREE, tree=tree)
+    assert unc.tolist() == [3, 3, 1, 3] and comp.tolist() == [3, 6, 7, 23] and ttft.tolist() == [3, 6, 7, 3]
+    assert tree.stats() == dict(n_nodes=3, tokens=6, clock=4, evictions=2)
+    assert tree.match(*csr([[1, 1, 1], [2, 2, 2], [1, 1, 5], [3, 3, 3]])).tolist() == [2, 0, 3, 3]
+    # c_attn = 1/2, times in half ticks: cost = (2 + |x|)(|x| - m)
+    unc, ttft, comp = oracle.replay([0, 1, 2, 3], t, o, arr, 1, 2, 0, oracle.CACHE_TREE, oracle.OracleTree(6))
+    assert comp.tolist() == [15, 30, 35, 50] and ttft.tolist() == [15, 30, 35, 30]
+    # queries that are not in the order keep their zeros; a later start delays everything
+    unc, ttft, comp = oracle.replay([2, 0], t, o, arr, 0, 1, 100, oracle.CACHE_TREE, oracle.OracleTree(6))
+    assert unc.tolist() == [1, 0, 3, 0] and comp.tolist() == [104, 0, 103, 0]
+
+
+@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("budget", [0, 30])
+def test_replay_with_the_tree_cache_against_the_definition(seed, budget):
+    """Random orders (a permutation, and a partial order with a repeat-free subset) over a pre-filled cache."""
+    prompts, arr = W.random_small_queue(seed + 1000, 24, vocab=2, max_len=12, min_len=1, max_gap=5)
+    prefill, _ = W.random_small_queue(seed + 1100, 5, vocab=2, max_len=9, min_len=1)
+    rng = np.random.RandomState(seed)
+    perm = rng.permutation(len(prompts)).tolist()
+    for order in (perm, perm[:11]):
+        for c_num, c_den in ((0, 1), (1, 3)):
+            tree = oracle.OracleTree(budget)
+            tree.insert(*csr(prefill))
+            got = oracle.replay(order, *csr(prompts), arr, c_num, c_den, 2, oracle.CACHE_TREE, tree)
+            ref = D.replay(order, prompts, arr, c_num, c_den, 2, D.TREE, prefill=prefill, budget=budget)
+            assert [g.tolist() for g in got] == [list(r) for r in ref]
+
+
 # ---------------------------------------------------------------- cost model details
 
 def test_cost_model_first_query_and_c_attn():
@@ -391,6 +461,29 @@ def test_hit_rate_score_by_hand_and_on_constant_lengths():
     # all prompts of a regular arrival queue have the same length: both scores order them alike
     prompts, arr = W.regular_arrival_shuffled_queue(12, 3, 5, 2, 1, [5, 1, 9, 3, 12, 7, 2, 11, 4, 8, 6, 10])
     assert run_ex(prompts, arr, oracle.POLICY_KLPM, k=3, score_mode=1) == run_ex(prompts, arr, oracle.POLICY_KLPM, k=3)
+
+
+def test_hit_rate_is_compared_exactly():
+    """1/100000 > 1/100001 although both round to the same multiple of 2^-31: the longer prompt arrived first and
+    would win a tie, the shorter one has the higher hit rate and is processed first."""
+    cached = [[1]]
+    a = [1] + [2] * 100000            # arrives first, hit rate 1/100001
+    b = [1] + [3] * 99999             # arrives second, hit rate 1/100000
+    assert (1 << 31) // len(a) == (1 << 31) // len(b)
+    t, o = csr([a, b])
+    for tier in (oracle.TIER_REMATCH, oracle.TIER_UPDATE):
+        tree = oracle.OracleTree()
+        tree.insert(*csr(cached))
+        order = oracle.schedule(t, o, [0, 1], oracle.POLICY_LPM, 1, 0, 1, 5, oracle.CACHE_TREE, tier, tree, None, 1)[0]
+        assert order.tolist() == [1, 0]
+    assert D.schedule([a, b], [0, 1], D.LPM, start_tick=5, prefill=cached, score_mode=1)[0] == [1, 0]
+    # equal rates (2/4 and 1/2, cache "12") are a tie that the earlier arrival wins; by match length 2 beats 1
+    t, o = csr([[1, 2, 5, 6], [1, 7]])
+    for mode, want in ((1, [1, 0]), (0, [0, 1])):
+        tree = oracle.OracleTree()
+        tree.insert(*csr([[1, 2]]))
+        order = oracle.schedule(t, o, [1, 0], oracle.POLICY_LPM, 1, 0, 1, 5, oracle.CACHE_TREE, oracle.TIER_REMATCH, tree, None, mode)[0]
+        assert order.tolist() == want
 
 
 @pytest.mark.parametrize("seed", range(6))
