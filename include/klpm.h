@@ -9,6 +9,11 @@
  *   - `d_*` arguments are DEVICE pointers owned by the caller (4-byte aligned for int32 data,
  *     8-byte aligned for int64 data).  The library never frees them and does not keep them after
  *     the work enqueued by the call has completed.  A pointer documented "nullable" may be NULL.
+ *   - token buffers are read in aligned 16-byte units: the unit that holds a prompt's first token and
+ *     the unit that holds its last token are loaded whole, so up to 12 bytes before and after the
+ *     tokens a call names may be read (never written, never interpreted).  An aligned 16-byte unit
+ *     never crosses a page, so this is safe for any pointer into an allocation; prompts may start
+ *     at any 4-byte boundary.
  *   - prompts are int32 token strings in CSR form: prompt i is tokens[offsets[i] .. offsets[i+1]);
  *     offsets are int64, non-decreasing, offsets[0] may be non-zero.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is enqueued on it;
@@ -118,8 +123,10 @@ rt_status rt_rollback(rt_tree* tree, void* stream);
 rt_status rt_sync_status(rt_tree* tree, void* stream);
 
 /* A number that says which device-side check recorded the status word (0 if none did): 101/104 a child entry
- * that should exist was not found, 102 a bounded wait of the scheduling loop ran out, 103 an internal
- * prediction did not hold.  A debugging aid; synchronises like rt_stats. */
+ * that should exist was not found, 102 a bounded wait of the scheduling loop ran out, 103/105/107 an internal
+ * prediction did not hold, 106 a child lookup probed the whole table, 108 an order entry that is not a query
+ * (or a prompt with a negative length), 109 a prompt too long for the hit-rate score.  A debugging aid;
+ * synchronises like rt_stats. */
 rt_status rt_status_detail(rt_tree* tree, int32_t* detail);
 
 /* Free the tree and everything it owns.  Synchronous. */
@@ -133,7 +140,9 @@ rt_status rt_destroy(rt_tree* tree);
  *   - longest-match pick (LPM; or KLPM otherwise): the query with the largest d_match_len, ties to the
  *     smallest (arrival, index).
  * d_pick (int32[1]) receives the index, or -1 if no query is waiting.  Uses library-owned scratch that
- * is allocated on the first call on each device. */
+ * is allocated on the first call on each device and shared by every later call on it: calls that overlap
+ * on the GPU (different streams, no dependency) race on it -- issue them on one stream or order them
+ * with events.  The same holds for klpm_select_topk. */
 rt_status klpm_select(const int32_t* d_match_len, const int64_t* d_arrival, const uint8_t* d_waiting,
                       int32_t nq, int64_t pick_counter, const klpm_params* params, int32_t* d_pick,
                       void* stream);
@@ -177,7 +186,9 @@ rt_status klpm_select_noalloc(const int32_t* d_match_len, const int64_t* d_arriv
  *   R_j = max(R_prev, t_j) + (c_den + c_num |x_j|) * uncached;  TTFT_j = R_j - t_j;
  * then x_j is stored in the tree (as rt_insert does).  Outputs are indexed by query: d_uncached
  * (int32[n_queries]), d_ttft (int64[n_queries]), d_completion (nullable, int64[n_queries]); entries of
- * queries that are not in d_order are left untouched. */
+ * queries that are not in d_order are left untouched.  An entry of d_order outside [0, n_queries) stops the
+ * replay there: nothing of it is read or written, the queries before it stay processed, and the status word
+ * reports RT_ERR_INVALID. */
 rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, const int32_t* d_q_tokens,
                       const int64_t* d_q_offsets, const int64_t* d_arrival, int32_t n_queries,
                       const klpm_params* params, int32_t* d_uncached, int64_t* d_ttft,
@@ -202,16 +213,27 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
 
 /* Which loop the last klpm_run / klpm_run_ex on this tree took: 0 = none yet, 1 = one decision at a time on the
  * tree itself (trees with a budget), 2 = the grouped loop (trees without a budget; see klpm_run).  Both give the
- * same outputs.  Setting the environment variable KLPM_RUN_LEGACY=1 makes trees without a budget take loop 1 too. */
+ * same outputs.  The debug setting "run_one_by_one" makes trees without a budget take loop 1 too. */
 int32_t klpm_run_path(const rt_tree* tree);
+
+/* Settings for tests and debugging; process-wide, read when a later call is made; value < 0 restores the default.
+ *   "run_one_by_one"   1: klpm_run takes the one-decision-at-a-time loop on every tree (default 0)
+ *   "fast_max_blocks"  grouped loop: the most tournament leaf blocks it may use (default 0 = 8,192)
+ *   "fast_smem_kb"     grouped loop: the shared memory it may use, in KiB (default 0 = 224)
+ *   "wait_limit_ns"    one-by-one loop: how long a CTA waits for another before it gives up, records
+ *                      RT_ERR_LIMIT (detail 102) and lets every CTA return (default 5e9; 0 = give up at once)
+ * RT_ERR_INVALID for an unknown name. */
+rt_status klpm_debug_set(const char* name, int64_t value);
 
 /* klpm_run with two variants of the longest-match pick (the oldest-first picks are not affected):
  *   d_tie_priority (nullable, int64[n]): among waiting queries with the same score the one with the smallest
  *     priority wins; arrival and index decide only among equal priorities.  With priorities drawn uniformly at
  *     random by the caller this is the tie-breaking the paper assumes for LPM (footnote in Section 4.2).
  *   score_mode 0: the score is the match length in tokens (Algorithm 1 as klpm_run reads it).
- *   score_mode 1: the score is the prompt's hit rate, quantised to floor(match * 2^31 / length) (0 for an empty
- *     prompt) -- the other reading of "maximizes the prefix cache hit rate".
+ *   score_mode 1: the score is the prompt's hit rate match / length (0 for an empty prompt) -- the other
+ *     reading of "maximizes the prefix cache hit rate".  It is held as floor(match * 2^31 / length), which
+ *     orders prompts exactly as the rates do while no prompt is longer than 46,340 tokens (46,340^2 < 2^31);
+ *     a longer prompt makes the status word report RT_ERR_INVALID (detail 109), and ties may then be wrong.
  * klpm_run(...) is klpm_run_ex(..., NULL, 0, ...). */
 rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
                       const int64_t* d_arrival, int32_t n, const klpm_params* params,
@@ -222,10 +244,13 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
  * the last query of its bin is).  d_order (int32[n_order]) is a processing order and d_completion (int64, indexed
  * by query) its batch-size-one completion times, as klpm_run / klpm_replay produce them; d_completion_b and
  * d_ttft_b (int64, indexed by query; entries of queries not in d_order are left untouched) receive the
- * completion time of the query's bin and that minus its arrival.  batch_size >= 1; must not alias the inputs. */
+ * completion time of the query's bin and that minus its arrival.  The per-query arrays have n_queries entries;
+ * a decision whose own entry of d_order, or the last entry of its bin, lies outside [0, n_queries) is skipped
+ * (nothing is read or written for it) and counted in d_n_skipped (nullable, int32[1], set by the call).
+ * batch_size >= 1; the outputs must not alias the inputs. */
 rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_t* d_arrival,
-                           const int64_t* d_completion, int32_t batch_size, int64_t* d_ttft_b,
-                           int64_t* d_completion_b, void* stream);
+                           const int64_t* d_completion, int32_t n_queries, int32_t batch_size,
+                           int64_t* d_ttft_b, int64_t* d_completion_b, int32_t* d_n_skipped, void* stream);
 
 /* Version of the ABI (bumped when a signature changes). */
 int32_t klpm_abi_version(void);

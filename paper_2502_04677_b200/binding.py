@@ -80,14 +80,16 @@ _lib.klpm_replay.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, ctypes.POINTER
 _lib.klpm_run_ex.restype = _i32
 _lib.klpm_run_ex.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.klpm_batch_times.restype = _i32
-_lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp]
+_lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp]
+_lib.klpm_debug_set.restype = _i32
+_lib.klpm_debug_set.argtypes = [ctypes.c_char_p, _i64]
 _lib.klpm_run_path.restype = _i32
 _lib.klpm_run_path.argtypes = [_vp]
 _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times"]
+           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times", "klpm_debug_set"]
 
 
 def lib() -> ctypes.CDLL:
@@ -208,8 +210,16 @@ def rt_destroy(tree: Tree) -> None:
     tree.destroy()
 
 
+def _same_length(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor) -> int:
+    n = match_len.numel()
+    if arrival.numel() != n or waiting.numel() != n:
+        raise ValueError("match_len, arrival and waiting must have the same number of elements")
+    return n
+
+
 def klpm_select(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, pick_counter: int,
                 params: klpm_params, pick: torch.Tensor) -> None:
+    _same_length(match_len, arrival, waiting)
     _check(_lib.klpm_select(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
                             _dev(waiting, torch.uint8, "waiting"), match_len.numel(), int(pick_counter),
                             ctypes.byref(params), _dev(pick, torch.int32, "pick"), _stream()), "klpm_select")
@@ -217,17 +227,17 @@ def klpm_select(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.T
 
 def klpm_select_topk(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, out: torch.Tensor) -> None:
     """out (int32[kk]) receives the kk best longest-match candidates of this snapshot, best first."""
+    _same_length(match_len, arrival, waiting)
     _check(_lib.klpm_select_topk(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
                                  _dev(waiting, torch.uint8, "waiting"), match_len.numel(), out.numel(),
                                  _dev(out, torch.int32, "out"), _stream()), "klpm_select_topk")
 
 
 def klpm_select_noalloc(match_len: torch.Tensor, arrival: torch.Tensor, waiting: torch.Tensor, pick_counter: int,
-                        params: klpm_params, pick: torch.Tensor, nq: Optional[int] = None) -> None:
+                        params: klpm_params, pick: torch.Tensor) -> None:
     """klpm_select without any device allocation inside the library (fixed scratch; at most
-    SELECT_NOALLOC_MAX_QUERIES queries; calls must not overlap on the GPU).  `nq` defaults to the length
-    of match_len; pass it to state a queue length without building tensors of that size."""
-    n = match_len.numel() if nq is None else int(nq)
+    SELECT_NOALLOC_MAX_QUERIES queries; calls must not overlap on the GPU)."""
+    n = _same_length(match_len, arrival, waiting)
     _check(_lib.klpm_select_noalloc(_dev(match_len, torch.int32, "match_len"), _dev(arrival, torch.int64, "arrival"),
                                     _dev(waiting, torch.uint8, "waiting"), n, int(pick_counter),
                                     ctypes.byref(params), _dev(pick, torch.int32, "pick"), _stream()),
@@ -263,11 +273,19 @@ def klpm_run_path(tree: Tree) -> int:
 
 
 def klpm_batch_times(order: torch.Tensor, arrival: torch.Tensor, completion: torch.Tensor, batch_size: int,
-                     ttft_b: torch.Tensor, completion_b: torch.Tensor) -> None:
+                     ttft_b: torch.Tensor, completion_b: torch.Tensor, n_skipped: Optional[torch.Tensor] = None) -> None:
+    n = arrival.numel()
+    if completion.numel() != n or ttft_b.numel() != n or completion_b.numel() != n:
+        raise ValueError("arrival, completion, ttft_b and completion_b must have one entry per query")
     _check(_lib.klpm_batch_times(_dev(order, torch.int32, "order"), order.numel(), _dev(arrival, torch.int64, "arrival"),
-                                 _dev(completion, torch.int64, "completion"), int(batch_size),
+                                 _dev(completion, torch.int64, "completion"), n, int(batch_size),
                                  _dev(ttft_b, torch.int64, "ttft_b"), _dev(completion_b, torch.int64, "completion_b"),
-                                 _stream()), "klpm_batch_times")
+                                 _dev(n_skipped, torch.int32, "n_skipped", True), _stream()), "klpm_batch_times")
+
+
+def klpm_debug_set(name: str, value: int) -> None:
+    """Process-wide test/debug settings of the library (see include/klpm.h); value < 0 restores the default."""
+    _check(_lib.klpm_debug_set(name.encode(), int(value)), "klpm_debug_set")
 
 
 def klpm_run_ex(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arrival: torch.Tensor, params: klpm_params,

@@ -30,7 +30,7 @@
 #include "klpm.h"
 
 #define FULL_MASK 0xffffffffu
-#define KLPM_ABI_VERSION 2
+#define KLPM_ABI_VERSION 3
 
 namespace {
 
@@ -104,6 +104,12 @@ __device__ __forceinline__ void set_status(TreeState* st, int code, int detail =
     if (atomicCAS(&st->status, 0, code) == 0) st->detail = detail;
 }
 
+// A child lookup that probed every slot of the table without meeting the key or an empty slot gives up; the
+// walk then reports a shorter match, and the status word says that it is not to be trusted.
+__device__ __noinline__ void probe_limit(const TreeDev& T) {
+    if ((threadIdx.x & 31) == 0) set_status(T.st, RT_ERR_LIMIT, 106);
+}
+
 // First index in [0, n) where a and b differ, or n.  Warp-cooperative: every lane gets the result.
 // Lane l reads elements l, l+32, l+64, ... of each chunk: each load instruction of the warp is one
 // contiguous 128-byte request, whatever the 4-byte phase of the two streams.  U * 128 tokens of both
@@ -149,9 +155,10 @@ __device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t le
     unsigned long long slot = hash_key(key) & T.table_mask;
     Entry c = ld_entry<RO>(T.table + slot);
     for (;;) {
-        unsigned probes = 0;
+        unsigned long long probes = 0;
         while (c.key != key) {
-            if (c.key == 0ULL || ++probes > 4096u) return t;
+            if (c.key == 0ULL) return t;
+            if (++probes > T.table_mask) { probe_limit(T); return t; }      // no empty slot: cannot happen below load 1
             slot = (slot + 1) & T.table_mask;
             c = ld_entry<RO>(T.table + slot);
         }
@@ -306,9 +313,10 @@ __device__ __forceinline__ int32_t walk_chain(const TreeDev& T, const int32_t* _
         const unsigned long long key = make_key(cur, __ldg(q + m));
         unsigned long long slot = hash_key(key) & T.table_mask;
         Entry c = ld_entry<true>(T.table + slot);
-        unsigned probes = 0;
+        unsigned long long probes = 0;
         while (c.key != key) {
-            if (c.key == 0ULL || ++probes > 4096u) return m;
+            if (c.key == 0ULL) return m;
+            if (++probes > T.table_mask) { probe_limit(T); return m; }      // no empty slot: cannot happen below load 1
             slot = (slot + 1) & T.table_mask;
             c = ld_entry<true>(T.table + slot);
         }
@@ -563,6 +571,7 @@ match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* _
 struct SeqArgs {
     const int32_t* tok; const int64_t* off; const int64_t* arrival; const int32_t* order;
     int32_t n;                       // prompts to process
+    int32_t n_queries;               // prompts in the CSR arrays: entries of `order` must be below this
     long long c_num, c_den, start_tick;
     int32_t* new_tokens;             // rt_insert: indexed by position
     int32_t* uncached; int64_t* ttft; int64_t* completion;   // replay: indexed by query
@@ -575,7 +584,15 @@ sequential_kernel(TreeDev T, SeqArgs A) {
     long long now = A.start_tick;
     for (int32_t k = 0; k < A.n; ++k) {
         const int32_t j = A.order ? __ldg(A.order + k) : k;
+        if (j < 0 || j >= A.n_queries) {           // not a query: nothing of it is read or written (uniform over the CTA)
+            if (threadIdx.x == 0) set_status(T.st, RT_ERR_INVALID, 108);
+            return;
+        }
         const int64_t lo = __ldg(A.off + j), hi = __ldg(A.off + j + 1);
+        if (hi < lo || hi - lo > 0x7fffffffLL) {
+            if (threadIdx.x == 0) set_status(T.st, RT_ERR_INVALID, 108);
+            return;
+        }
         const int32_t len = (int32_t)(hi - lo);
         const int32_t* x = A.tok + lo;
         if (threadIdx.x < 32) {
@@ -843,6 +860,7 @@ struct RunArgs {
     unsigned long long* partial;   // per CTA best key
     RunBcast* bc;
     RunSync* sy;
+    long long wait_limit_ns;       // limit of every hand-over wait
 };
 
 #define KLPM_RUN_THREADS 512
@@ -850,20 +868,22 @@ struct RunArgs {
 #ifndef KLPM_RUN_SPT
 #define KLPM_RUN_SPT 2            // slots per scanner thread the grid is sized for
 #endif
-#define KLPM_WAIT_LIMIT_NS 30000000000ULL
+#define KLPM_WAIT_LIMIT_NS 5000000000LL      // default limit of a hand-over wait: 5 s on the device's nanosecond timer
 
-// Thread 0 of the CTA polls *p until it reaches target (bounded), then the CTA learns whether to go on.
-__device__ bool run_wait(volatile unsigned long long* p, unsigned long long target, RunBcast* bc, TreeState* st) {
+// Thread 0 of the CTA polls *p until it reaches target, then the CTA learns whether to go on.  The wait is
+// bounded: after limit_ns (checked every 4,096 polls; a limit of 0 gives up at the first poll that fails) the
+// status word gets RT_ERR_LIMIT, every CTA is told to leave, and this one returns false.
+__device__ bool run_wait(volatile unsigned long long* p, unsigned long long target, RunBcast* bc, TreeState* st, long long limit_ns) {
     __shared__ int s_go;
     if (threadIdx.x == 0) {
         int go = 1;
         unsigned long long spins = 0, t0 = 0;
         while (*p < target) {
-            if ((++spins & 4095ULL) == 0) {            // the wait is bounded in time: 30 s on the device's nanosecond timer
+            if ((++spins & 4095ULL) == 0 || limit_ns == 0) {
                 unsigned long long now;
                 asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
                 if (t0 == 0) t0 = now;
-                if (now - t0 > KLPM_WAIT_LIMIT_NS || spins > (1ULL << 40)) {
+                if (limit_ns == 0 || now - t0 > (unsigned long long)limit_ns || spins > (1ULL << 40)) {
                     set_status(st, RT_ERR_LIMIT, 102); *(volatile int32_t*)&bc->abort = 1; go = 0; break;
                 }
             }
@@ -1031,7 +1051,7 @@ run_kernel(TreeDev T, RunArgs A) {
     if (blockIdx.x != 0) {
         // ------------------------------------------------------------ scanners
         for (long long c = 0; c < A.n; ++c) {
-            if (!run_wait(&A.sy->seq, (unsigned long long)c, A.bc, gst)) return;
+            if (!run_wait(&A.sy->seq, (unsigned long long)c, A.bc, gst, A.wait_limit_ns)) return;
             if (threadIdx.x == 0) {
                 RunBcast b;
                 const long long* src = reinterpret_cast<const long long*>(A.bc);
@@ -1088,7 +1108,7 @@ run_kernel(TreeDev T, RunArgs A) {
             __syncthreads();
             if (warp == 0) b = warp_max64(lane < (int)(blockDim.x >> 5) ? s_red[lane] : 0ULL);
         } else {
-            if (!run_wait(&A.sy->arrive, (unsigned long long)(c + 1) * nscan, A.bc, gst)) { ok = false; break; }
+            if (!run_wait(&A.sy->arrive, (unsigned long long)(c + 1) * nscan, A.bc, gst, A.wait_limit_ns)) { ok = false; break; }
             if (warp == 0) {
                 for (unsigned g = lane; g < nscan; g += 32) { const unsigned long long o = __ldcg(A.partial + g); if (o > b) b = o; }
                 b = warp_max64(b);
@@ -1341,6 +1361,16 @@ __global__ void fast_stat_kernel(const int32_t* __restrict__ ord, const long lon
     FStat s;
     s.soff = lo; s.t = sorted_t[r]; s.len = (int32_t)(off[qi + 1] - lo); s.ord = qi; s.rank = prank ? prank[r] : r; s.pad = 0;
     stat[r] = s;
+}
+
+// The hit-rate score is kept as floor(m * 2^31 / |x|) in the high half of a key.  Two different rates m/|x| and
+// m'/|x'| differ by at least 1/(|x||x'|), so while every prompt is at most 46,340 tokens long (46,340^2 < 2^31)
+// different rates get different quotients, equal rates equal ones, and the order of the keys is the order of the
+// rates.  Longer prompts could tie where the rates do not: the status word says so.
+#define KLPM_HIT_RATE_MAX_LEN 46340
+__global__ void hit_rate_guard_kernel(const int64_t* __restrict__ off, int32_t n, TreeState* st) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n && off[i + 1] - off[i] > KLPM_HIT_RATE_MAX_LEN) set_status(st, RT_ERR_INVALID, 109);
 }
 
 // The one match of every query against the tree: one warp per slot, slots handed out by a counter.
@@ -2469,13 +2499,18 @@ __global__ void bulk_finish_kernel(TreeState* S, long long n, long long max_cloc
 
 // batch size B: a query is finished when the last query of its bin of the processing order is
 __global__ void batch_times_kernel(const int32_t* __restrict__ order, int32_t n, const int64_t* __restrict__ arrival,
-                                   const int64_t* __restrict__ completion, int32_t B, int64_t* ttft_b, int64_t* completion_b) {
+                                   const int64_t* __restrict__ completion, int32_t n_queries, int32_t B, int64_t* ttft_b,
+                                   int64_t* completion_b, int32_t* bad) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     int64_t last = (i / B + 1) * (int64_t)B - 1;
     if (last > n - 1) last = n - 1;
-    const int64_t R = __ldg(completion + __ldg(order + last));
-    const int32_t j = __ldg(order + i);
+    const int32_t jl = __ldg(order + last), j = __ldg(order + i);
+    if (jl < 0 || jl >= n_queries || j < 0 || j >= n_queries) {      // not a query: skipped, counted if the caller asked
+        if (bad) atomicAdd(bad, 1);
+        return;
+    }
+    const int64_t R = __ldg(completion + jl);
     completion_b[j] = R;
     ttft_b[j] = R - __ldg(arrival + j);
 }
@@ -2690,6 +2725,15 @@ bool params_ok(const klpm_params* p) {
     return p && p->policy >= KLPM_POLICY_FCFS && p->policy <= KLPM_POLICY_KLPM && p->k >= 1 && p->c_den >= 1 && p->c_num >= 0;
 }
 
+// Settings for tests and debugging (klpm_debug_set); process-wide, read when a call is made.
+struct DebugKnobs {
+    long long run_one_by_one;     // 1: trees without a budget take the one-by-one loop too
+    long long fast_max_blocks;    // grouped loop: most tournament leaf blocks (0 = the built-in 8,192)
+    long long fast_smem_kb;       // grouped loop: shared memory it may use (0 = the built-in 224 KB)
+    long long wait_limit_ns;      // one-by-one loop: limit of a hand-over wait
+};
+DebugKnobs g_knobs = {0, 0, 0, KLPM_WAIT_LIMIT_NS};
+
 SelectScratch* g_select_scratch[64] = {nullptr};
 TopkScratch* g_topk_scratch[64] = {nullptr};
 StaticSelectScratch* g_select_static_addr[64] = {nullptr};   // device address of g_select_static, per device
@@ -2836,7 +2880,7 @@ rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_off
     }
     SeqArgs a;
     memset(&a, 0, sizeof(a));
-    a.tok = d_tokens; a.off = d_offsets; a.n = n; a.new_tokens = d_new_tokens; a.c_den = 1;
+    a.tok = d_tokens; a.off = d_offsets; a.n = n; a.n_queries = n; a.new_tokens = d_new_tokens; a.c_den = 1;
     tree->last_stream = (cudaStream_t)stream;
     sequential_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>(tree->dev, a);
     CK(cudaGetLastError());
@@ -3081,7 +3125,7 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
     if (n_order == 0) return RT_OK;
     SeqArgs a;
     memset(&a, 0, sizeof(a));
-    a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.order = d_order; a.n = n_order;
+    a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.order = d_order; a.n = n_order; a.n_queries = n_queries;
     a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
     a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion;
     tree->last_stream = (cudaStream_t)stream;
@@ -3091,12 +3135,15 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
 }
 
 rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_t* d_arrival, const int64_t* d_completion,
-                           int32_t batch_size, int64_t* d_ttft_b, int64_t* d_completion_b, void* stream) {
-    if (n_order < 0 || batch_size < 1 || (n_order > 0 && (!d_order || !d_arrival || !d_completion || !d_ttft_b || !d_completion_b)))
-        return RT_ERR_INVALID;
+                           int32_t n_queries, int32_t batch_size, int64_t* d_ttft_b, int64_t* d_completion_b,
+                           int32_t* d_n_skipped, void* stream) {
+    if (n_order < 0 || n_queries < 0 || batch_size < 1 ||
+        (n_order > 0 && (!d_order || !d_arrival || !d_completion || !d_ttft_b || !d_completion_b))) return RT_ERR_INVALID;
+    if (d_n_skipped) CK(cudaMemsetAsync(d_n_skipped, 0, sizeof(int32_t), (cudaStream_t)stream));
     if (n_order == 0) return RT_OK;
     batch_times_kernel<<<(unsigned)((n_order + 255) / 256), 256, 0, (cudaStream_t)stream>>>(d_order, n_order, d_arrival, d_completion,
-                                                                                           batch_size, d_ttft_b, d_completion_b);
+                                                                                           n_queries, batch_size, d_ttft_b,
+                                                                                           d_completion_b, d_n_skipped);
     CK(cudaGetLastError());
     return RT_OK;
 }
@@ -3113,18 +3160,15 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     if (st) return st;
     long long np2 = 1;
     while (np2 < n) np2 <<= 1;
-    // A tree without a budget takes the grouped loop.  KLPM_RUN_LEGACY=1 forces the one-by-one loop.
-    bool grouped = false;
-    if (tree->cfg.budget_tokens == 0) {
-        const char* legacy = getenv("KLPM_RUN_LEGACY");
-        grouped = !(legacy && legacy[0] == '1');
-    }
+    // A tree without a budget takes the grouped loop (unless the debug setting run_one_by_one is on).
+    const bool grouped = tree->cfg.budget_tokens == 0 && !g_knobs.run_one_by_one;
     // slots = queries ordered by (arrival, index)
     {
         unsigned blocks = (unsigned)((np2 + 255) / 256);
         rank_init_kernel<<<blocks, 256, 0, s>>>(d_arrival, n, np2, tree->run_key, tree->run_ord);
         sort_pairs(tree->run_key, tree->run_ord, np2, s);
         slot_arrays_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, d_q_offsets, n, tree->run_soff, tree->run_slen);
+        if (score_mode == 1) hit_rate_guard_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(d_q_offsets, n, tree->dev.st);
         if (d_tie_priority) {        // rank of every slot by (priority, slot)
             prio_init_kernel<<<blocks, 256, 0, s>>>(d_tie_priority, tree->run_ord, n, np2, tree->run_pkey, tree->run_pinv);
             sort_pairs(tree->run_pkey, tree->run_pinv, np2, s);
@@ -3158,12 +3202,12 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         fast_walk_kernel<<<(unsigned)wblocks, 256, 0, s>>>(tree->dev, f, np2);
         CK(cudaGetLastError());
         // Leaf blocks of 32 slots while at most 8,192 of them are needed, larger ones beyond (queues above 262,144).
-        // Two environment variables shrink the limits so that small queues can exercise the large-queue layout:
-        // KLPM_FAST_MAX_BLOCKS (leaf blocks) and KLPM_FAST_SMEM_KB (shared memory the loop may use).
+        // Two debug settings shrink the limits so that small queues can exercise the large-queue layout:
+        // fast_max_blocks (leaf blocks) and fast_smem_kb (shared memory the loop may use).
         long long max_blocks = 8192;
         size_t smem_max = 224 * 1024;
-        if (const char* e = getenv("KLPM_FAST_MAX_BLOCKS")) { const long long v = atoll(e); if (v >= 1 && v < max_blocks) max_blocks = v; }
-        if (const char* e = getenv("KLPM_FAST_SMEM_KB")) { const long long v = atoll(e); if (v >= 1 && (size_t)v * 1024 < smem_max) smem_max = (size_t)v * 1024; }
+        if (g_knobs.fast_max_blocks >= 1 && g_knobs.fast_max_blocks < max_blocks) max_blocks = g_knobs.fast_max_blocks;
+        if (g_knobs.fast_smem_kb >= 1 && (size_t)g_knobs.fast_smem_kb * 1024 < smem_max) smem_max = (size_t)g_knobs.fast_smem_kb * 1024;
         int lbs = 5;
         while ((((long long)n + (1LL << lbs) - 1) >> lbs) > max_blocks) ++lbs;
         f.lb_shift = lbs;
@@ -3217,6 +3261,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     a.score_mode = score_mode;
     a.ord = tree->run_ord; a.sorted_t = tree->run_key; a.m = tree->run_m; a.hint = tree->run_hint; a.pos = tree->run_pos;
     a.partial = tree->run_partial; a.bc = tree->run_bc; a.sy = tree->run_sy;
+    a.wait_limit_ns = g_knobs.wait_limit_ns;
     const int threads = KLPM_RUN_THREADS;
     int per_sm = 0;
     CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, run_kernel, threads, 0));
@@ -3232,6 +3277,17 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
 }
 
 int32_t klpm_run_path(const rt_tree* tree) { return tree ? tree->run_path : 0; }
+
+rt_status klpm_debug_set(const char* name, int64_t value) {
+    if (!name) return RT_ERR_INVALID;
+    const DebugKnobs defaults = {0, 0, 0, KLPM_WAIT_LIMIT_NS};
+    if (!strcmp(name, "run_one_by_one")) g_knobs.run_one_by_one = value < 0 ? defaults.run_one_by_one : (value != 0);
+    else if (!strcmp(name, "fast_max_blocks")) g_knobs.fast_max_blocks = value < 0 ? defaults.fast_max_blocks : value;
+    else if (!strcmp(name, "fast_smem_kb")) g_knobs.fast_smem_kb = value < 0 ? defaults.fast_smem_kb : value;
+    else if (!strcmp(name, "wait_limit_ns")) g_knobs.wait_limit_ns = value < 0 ? defaults.wait_limit_ns : value;
+    else return RT_ERR_INVALID;
+    return RT_OK;
+}
 
 rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
                    int32_t n, const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,

@@ -64,7 +64,7 @@ def test_full_size_configuration_is_bit_exact(name):
     K.rt_destroy(tree)
 
 
-def test_adversarial_full_size_properties_and_both_loops(monkeypatch):
+def test_adversarial_full_size_properties_and_both_loops():
     """The bench's own configuration (262,144 queries, k = 4) is too large for the CPU oracle's schedule, so the
     scheduling loop is checked there through what holds at any size -- the order is a permutation; every k-th
     decision takes the oldest unprocessed query (everybody is waiting); every other decision takes a query whose
@@ -81,10 +81,7 @@ def test_adversarial_full_size_properties_and_both_loops(monkeypatch):
     before = K.rt_stats(tree)
     outs = []
     for legacy in (False, True):
-        if legacy:
-            monkeypatch.setenv("KLPM_RUN_LEGACY", "1")
-        else:
-            monkeypatch.delenv("KLPM_RUN_LEGACY", raising=False)
+        K.klpm_debug_set("run_one_by_one", 1 if legacy else 0)
         K.rt_rollback(tree)
         order = torch.full((nq,), -1, dtype=torch.int32, device=device)
         unc = torch.full((nq,), -1, dtype=torch.int32, device=device)
@@ -94,7 +91,7 @@ def test_adversarial_full_size_properties_and_both_loops(monkeypatch):
         assert K.rt_sync_status(tree) == 0
         assert K.klpm_run_path(tree) == (K.RUN_PATH_ONE_BY_ONE if legacy else K.RUN_PATH_GROUPED)
         outs.append((order.cpu(), unc.cpu(), ttft.cpu(), comp.cpu(), K.rt_stats(tree)))
-    monkeypatch.delenv("KLPM_RUN_LEGACY", raising=False)
+    K.klpm_debug_set("run_one_by_one", -1)
     order, unc, ttft, comp, after = outs[0]
     for a, b in zip(outs[0][:4], outs[1][:4]):
         assert torch.equal(a, b)

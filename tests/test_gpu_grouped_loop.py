@@ -5,8 +5,6 @@ same tree position and continues with the same token form a group, and processin
 group only.  These cases aim at the group machinery: groups of 2..32 (one warp), groups up to 4,096 (sorted in
 shared memory), larger groups (kept together), queries that have not arrived when their group changes,
 identical prompts, prompts that are prefixes of others, and the tie-priority / hit-rate variants."""
-import os
-
 import numpy as np
 import pytest
 import torch
@@ -39,16 +37,12 @@ def run_gpu(K, prefill, prompts, arr, policy, k, prio=None, score_mode=0, start=
     ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
     comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
     d_prio = None if prio is None else dev(torch.as_tensor(prio, dtype=torch.int64))
-    old = os.environ.pop("KLPM_RUN_LEGACY", None)
-    if legacy:
-        os.environ["KLPM_RUN_LEGACY"] = "1"
+    K.klpm_debug_set("run_one_by_one", 1 if legacy else 0)
     try:
         K.klpm_run_ex(tree, dev(qt), dev(qo), dev(torch.as_tensor(arr, dtype=torch.int64)),
                       K.make_params(policy, k, c_num, c_den, start), d_prio, score_mode, order, unc, ttft, comp)
     finally:
-        os.environ.pop("KLPM_RUN_LEGACY", None)
-        if old is not None:
-            os.environ["KLPM_RUN_LEGACY"] = old
+        K.klpm_debug_set("run_one_by_one", -1)
     assert K.rt_sync_status(tree) == 0
     assert K.klpm_run_path(tree) == (K.RUN_PATH_ONE_BY_ONE if legacy else K.RUN_PATH_GROUPED)
     st = K.rt_stats(tree)
@@ -178,7 +172,7 @@ def test_list_mode_many_turn_patterns(K, n):
 
 @pytest.mark.parametrize("name,scale,k", [("medium", 1 / 16, 4), ("adversarial", 1 / 256, 4), ("tiny", 1, 2)])
 def test_both_loops_agree(K, name, scale, k):
-    """The grouped loop and the one-by-one loop (forced by KLPM_RUN_LEGACY=1) give identical schedules."""
+    """The grouped loop and the one-by-one loop (forced by the debug setting run_one_by_one) give identical schedules."""
     w = W.tiny() if name == "tiny" else W.WORKLOADS[name](scale=scale)
     pt, po = w.prefill.materialize()
     qt, qo = w.queries.materialize()
@@ -190,18 +184,21 @@ def test_both_loops_agree(K, name, scale, k):
 
 
 @pytest.mark.parametrize("max_blocks,smem_kb", [(16, 0), (4, 60), (1, 0)])
-def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb, monkeypatch):
+def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb):
     """Queues above 262,144 use larger tournament leaf blocks, and far larger ones keep the processed bitmap in
     global memory; neither uses list mode.  Shrinking the limits makes a 3,000-query stream take those paths."""
-    monkeypatch.setenv("KLPM_FAST_MAX_BLOCKS", str(max_blocks))
-    if smem_kb:
-        monkeypatch.setenv("KLPM_FAST_SMEM_KB", str(smem_kb))
-    prompts, arr = shared_prefix_queue(31, 3000, [(12, 3), (9, 4)], tail=9, vocab=5, max_gap=2)
-    prefill, _ = shared_prefix_queue(32, 200, [(12, 3), (9, 4)], tail=4, vocab=5, max_gap=0)
-    for policy, k in ((2, 4), (0, 1)):
-        got = run_gpu(K, prefill, prompts, arr, policy, k)
-        want = run_oracle(prefill, prompts, arr, policy, k)
-        same(got, want)
+    K.klpm_debug_set("fast_max_blocks", max_blocks)
+    K.klpm_debug_set("fast_smem_kb", smem_kb)
+    try:
+        prompts, arr = shared_prefix_queue(31, 3000, [(12, 3), (9, 4)], tail=9, vocab=5, max_gap=2)
+        prefill, _ = shared_prefix_queue(32, 200, [(12, 3), (9, 4)], tail=4, vocab=5, max_gap=0)
+        for policy, k in ((2, 4), (0, 1)):
+            got = run_gpu(K, prefill, prompts, arr, policy, k)
+            want = run_oracle(prefill, prompts, arr, policy, k)
+            same(got, want)
+    finally:
+        K.klpm_debug_set("fast_max_blocks", -1)
+        K.klpm_debug_set("fast_smem_kb", -1)
 
 
 def test_list_mode_all_arrived(K):

@@ -56,13 +56,22 @@ def oracle_tree(tokens, offsets, budget=0):
 
 # ------------------------------------------------------------------ batched match
 
+def assert_match_equals_oracle(K, tree, ot, qt, qo):
+    """Match length and where the match ended (tokens matched of the edge holding the last matched token; the
+    depth at which that edge starts is the difference), element by element."""
+    m, node, off = gpu_match(K, tree, qt, qo)
+    want_m, want_off, want_depth = ot.match_pos(qt.numpy(), qo.numpy())
+    assert np.array_equal(m, want_m)
+    assert np.array_equal(off, want_off)
+    assert np.array_equal(m - off, want_depth)
+    assert np.array_equal(node == 0, m == 0)
+    return m
+
+
 def check_match(K, pt, po, qt, qo):
     tree = gpu_tree(K, pt, po)
-    m, node, off = gpu_match(K, tree, qt, qo)
     ot = oracle_tree(pt, po)
-    want = ot.match(qt.numpy(), qo.numpy())
-    assert np.array_equal(m, want)
-    assert np.array_equal(node == 0, m == 0) and np.all(off >= 0) and np.all(off <= m)
+    m = assert_match_equals_oracle(K, tree, ot, qt, qo)
     st, ost = K.rt_stats(tree), ot.stats()
     assert (st["n_nodes"], st["tokens"], st["clock"]) == (ost["n_nodes"], ost["tokens"], ost["clock"])
     K.rt_destroy(tree)
@@ -132,9 +141,7 @@ def test_insert_new_tokens_and_stats(K, budget):
     if budget:
         assert ost["evictions"] > 0 and st["tokens"] <= budget
     qs, _ = W.random_small_queue(10, 100, vocab=2, max_len=18)
-    m, _, _ = gpu_match(K, tree, *csr(qs))
-    qt, qo = csr(qs)
-    assert np.array_equal(m, ot.match(qt.numpy(), qo.numpy()))
+    assert_match_equals_oracle(K, tree, ot, *csr(qs))        # hop-by-hop walk on a tree with a budget too
 
 
 def test_capacity_and_budget_errors_are_reported_not_fatal(K):
@@ -216,6 +223,29 @@ def test_replay_fixed_order(K, budget):
     assert np.array_equal(ttft.cpu().numpy(), ottft)
     assert np.array_equal(comp.cpu().numpy(), ocomp)
     assert K.rt_stats(tree)["evictions"] == ot.stats()["evictions"]
+
+
+def test_replay_stops_at_an_order_entry_that_is_not_a_query(K):
+    """An order with -1 (or an index past the queue) in it: the replay processes what comes before, touches nothing
+    for the bad entry or after it, and reports RT_ERR_INVALID through the status word."""
+    prompts, arr = W.random_small_queue(23, 12, vocab=3, max_len=9, min_len=1)
+    qt, qo = csr(prompts)
+    n = len(prompts)
+    for bad in (-1, n, 1 << 30):
+        tree = K.rt_create(**caps(qt.numel(), n_prompts=n))
+        order = torch.tensor([3, 1, bad, 2], dtype=torch.int32)
+        unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+        K.klpm_replay(tree, dev(order), dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_FCFS), unc, ttft)
+        assert K.rt_sync_status(tree) == K.RT_ERR_INVALID and K.rt_status_detail(tree) == 108
+        ou, ottft, _ = oracle.replay([3, 1], qt.numpy(), qo.numpy(), arr, cache_mode=oracle.CACHE_TREE)
+        want_u = np.full(n, -1, dtype=np.int32)
+        want_t = np.full(n, -1, dtype=np.int64)
+        want_u[[3, 1]] = ou[[3, 1]]
+        want_t[[3, 1]] = ottft[[3, 1]]
+        assert np.array_equal(unc.cpu().numpy(), want_u) and np.array_equal(ttft.cpu().numpy(), want_t)
+        assert K.rt_stats(tree)["clock"] == 2
+        K.rt_destroy(tree)
 
 
 # ------------------------------------------------------------------ the whole loop
@@ -464,6 +494,19 @@ def test_batch_times(K, B):
     assert np.array_equal(tb.cpu().numpy(), ot) and np.array_equal(cb.cpu().numpy(), oc)
 
 
+def test_batch_times_skips_order_entries_that_are_not_queries(K):
+    order = torch.tensor([2, 0, -1, 1, 7, 3], dtype=torch.int32)      # 4 queries; bins of 2: (2,0) (-1,1) (7,3)
+    arr = torch.tensor([0, 1, 2, 3], dtype=torch.int64)
+    comp = torch.tensor([20, 40, 10, 60], dtype=torch.int64)
+    tb = torch.full((4,), -1, dtype=torch.int64, device="cuda")
+    cb = torch.full((4,), -1, dtype=torch.int64, device="cuda")
+    skipped = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    K.klpm_batch_times(dev(order), dev(arr), dev(comp), 2, tb, cb, skipped)
+    # bin 1 finishes with query 0 (20); bin 2 with query 1 (40), its first entry is skipped; bin 3 with query 3 (60)
+    assert cb.tolist() == [20, 40, 20, 60] and tb.tolist() == [20, 39, 18, 57]
+    assert int(skipped.item()) == 2
+
+
 # ------------------------------------------------------------------ queues large enough for the multi-CTA loop
 # (above 4,096 queries klpm_run uses a sequencer CTA plus scanner CTAs and publishes picks early)
 
@@ -622,3 +665,56 @@ def test_run_ex_multi_cta_random_ties(K, score_mode):
     want = run_oracle_ex(pt, po, qt, qo, w.arrivals, oracle.POLICY_LPM, 1, prio, score_mode, start=w.start_tick)
     assert_same_schedule(got, want)
     assert not np.array_equal(got[0], run_oracle(pt, po, qt, qo, w.arrivals, oracle.POLICY_LPM, 1, start=w.start_tick)[0])
+
+
+# ------------------------------------------------------------------ bounded waits and guarded scores
+
+def test_a_wait_that_runs_out_is_reported_and_every_cta_returns(K):
+    """The one-by-one loop's CTAs wait for one another with a limit.  With the limit set to zero the sequencer gives
+    up on its first hand-over: the call returns, the status word says RT_ERR_LIMIT (detail 102), and after a
+    rollback the tree answers matches as before.  Nothing traps or hangs: a wait that gives up returns."""
+    prompts, arr = W.random_small_queue(77, 6000, vocab=3, max_len=24, min_len=1, max_gap=0)      # everybody waiting
+    prefill, _ = W.random_small_queue(78, 50, vocab=3, max_len=20, min_len=1)
+    qt, qo = csr(prompts)
+    pt, po = csr(prefill)
+    n = len(prompts)
+    tree = gpu_tree(K, pt, po, extra_prompts=n, extra_tokens=qt.numel(), budget=200000)
+    K.rt_checkpoint(tree)
+    out = [torch.full((n,), -1, dtype=torch.int32, device="cuda"), torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+           torch.full((n,), -1, dtype=torch.int64, device="cuda")]
+    K.klpm_debug_set("wait_limit_ns", 0)
+    try:
+        K.klpm_run(tree, dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_KLPM, 3), *out)
+        assert K.rt_sync_status(tree) == K.RT_ERR_LIMIT
+        assert K.rt_status_detail(tree) == 102
+    finally:
+        K.klpm_debug_set("wait_limit_ns", -1)
+    K.rt_rollback(tree)
+    assert K.rt_sync_status(tree) == 0
+    ot = oracle_tree(pt, po, 200000)
+    assert_match_equals_oracle(K, tree, ot, qt, qo)
+    # and with the default limit the same call completes and equals the oracle
+    K.klpm_run(tree, dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_KLPM, 3), *out)
+    assert K.rt_sync_status(tree) == 0
+    want = oracle.schedule(qt.numpy(), qo.numpy(), np.asarray(arr), oracle.POLICY_KLPM, 3, 0, 1, 0, oracle.CACHE_TREE,
+                           oracle.TIER_UPDATE, ot)
+    assert np.array_equal(out[0].cpu().numpy(), want[0]) and np.array_equal(out[2].cpu().numpy(), want[2])
+    K.rt_destroy(tree)
+
+
+def test_hit_rate_score_refuses_prompts_it_cannot_order_exactly(K):
+    """The hit-rate key orders prompts exactly as the rates m/|x| do up to 46,340 tokens per prompt; one longer
+    prompt makes the status word say so (both loops)."""
+    prompts = [[1] + [2] * 46340, [1, 3, 4]]
+    qt, qo = csr(prompts)
+    for budget in (0, 1 << 20):
+        tree = K.rt_create(budget_tokens=budget, **caps(qt.numel(), n_prompts=2))
+        out = [torch.zeros(2, dtype=torch.int32, device="cuda"), torch.zeros(2, dtype=torch.int32, device="cuda"),
+               torch.zeros(2, dtype=torch.int64, device="cuda")]
+        K.klpm_run_ex(tree, dev(qt), dev(qo), dev(torch.zeros(2, dtype=torch.int64)), K.make_params(K.POLICY_LPM), None, 1, *out)
+        assert K.rt_sync_status(tree) == K.RT_ERR_INVALID and K.rt_status_detail(tree) == 109
+        K.rt_destroy(tree)
+        tree = K.rt_create(budget_tokens=budget, **caps(qt.numel(), n_prompts=2))
+        K.klpm_run_ex(tree, dev(qt), dev(qo), dev(torch.zeros(2, dtype=torch.int64)), K.make_params(K.POLICY_LPM), None, 0, *out)
+        assert K.rt_sync_status(tree) == 0
+        K.rt_destroy(tree)
