@@ -99,6 +99,22 @@ rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const i
                          int32_t nq, int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off,
                          void* stream);
 
+/* What a batched match knows about one query beyond its match length (where in the token pool the match ended,
+ * the run of pool tokens around it, the query token that follows), kept so that the scheduling loop can start from
+ * the match instead of walking every query again.  Opaque: 32 bytes per query, 16-byte aligned. */
+typedef struct { int64_t w[4]; } klpm_match_state;
+
+/* rt_match_batch that also fills d_state (nullable, klpm_match_state[nq]) for a later klpm_run_ex on the same
+ * queries.  The records are good for that one purpose while (a) the tree has not been changed by any call since
+ * (rt_insert, klpm_replay, klpm_run*, rt_rollback), (b) d_q_tokens / d_q_offsets / nq are the ones passed here
+ * and their contents have not changed, and (c) no later rt_match_batch_ex with a state buffer was made on this
+ * tree.  On a tree with a budget the records are written but klpm_run_ex does not use them (the tree changes
+ * under the loop).  Batches of 2,048 queries or more are taken in an order bucketed by first token, for which
+ * the first such call allocates scratch (synchronously); results do not depend on the order. */
+rt_status rt_match_batch_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, int32_t nq,
+                            int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off,
+                            klpm_match_state* d_state, void* stream);
+
 /* Counters of the tree (synchronises the stream the tree was last used on).  Any pointer may be NULL.
  * n_nodes: live nodes, root excluded; n_tokens: tokens held by live nodes; clock: prompts processed;
  * evictions: leaves evicted so far; pool_used: tokens appended to the pool so far. */
@@ -234,10 +250,17 @@ rt_status klpm_debug_set(const char* name, int64_t value);
  *     reading of "maximizes the prefix cache hit rate".  It is held as floor(match * 2^31 / length), which
  *     orders prompts exactly as the rates do while no prompt is longer than 46,340 tokens (46,340^2 < 2^31);
  *     a longer prompt makes the status word report RT_ERR_INVALID (detail 109), and ties may then be wrong.
- * klpm_run(...) is klpm_run_ex(..., NULL, 0, ...). */
+ *   d_match_state (nullable): the records rt_match_batch_ex wrote for exactly these queries on this tree, if no
+ *     call has changed the tree since.  The loop then starts from that match; without them it matches every
+ *     query itself first (the same kernel), so the outputs are identical.  RT_ERR_INVALID is returned, and nothing
+ *     is enqueued, if the records are not the ones the last rt_match_batch_ex on this tree wrote for these
+ *     arguments or the tree has changed since; records the caller has overwritten are caught on the device
+ *     (status RT_ERR_INVALID, detail 110).
+ * klpm_run(...) is klpm_run_ex(..., NULL, 0, NULL, ...). */
 rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
                       const int64_t* d_arrival, int32_t n, const klpm_params* params,
-                      const int64_t* d_tie_priority, int32_t score_mode, int32_t* d_order,
+                      const int64_t* d_tie_priority, int32_t score_mode,
+                      const klpm_match_state* d_match_state, int32_t* d_order,
                       int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);
 
 /* Batch size B (Section 2.1: the order is cut into consecutive bins of B queries, and a query is finished when
@@ -251,6 +274,25 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
 rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_t* d_arrival,
                            const int64_t* d_completion, int32_t n_queries, int32_t batch_size,
                            int64_t* d_ttft_b, int64_t* d_completion_b, int32_t* d_n_skipped, void* stream);
+
+/* Many independent queues at once under the cache model the paper's analysis uses: only the previously processed
+ * prompt is cached (Definition 2 as printed; Section 2.1), so the match of a waiting prompt is its overlap with the
+ * prompt processed last and nothing is kept between queues.  This is the setting of the worked example of
+ * Section 4.2 and of Theorem 2; a Monte-Carlo over the random arrival orders of Definition 3 is one call.
+ *   Queue r consists of prompts d_queue_offsets[r] .. d_queue_offsets[r+1]-1 (int32[n_queues+1], non-decreasing) of the
+ *   CSR arrays d_tokens / d_offsets; d_arrival and d_tie_priority (nullable) are indexed like the prompts.  Each queue is
+ *   scheduled on its own by params (FCFS / LPM / k-LPM, c_attn, start_tick), starting with an empty cache: wait for
+ *   the next arrival if nobody is waiting; oldest-first pick = smallest (arrival, index); longest-match pick =
+ *   largest overlap with the prompt processed last, ties to the smallest priority, then (arrival, index); charge by
+ *   Definition 2.  d_order[d_queue_offsets[r] + c] = index WITHIN queue r of the prompt processed at its decision c;
+ *   d_uncached, d_ttft, d_completion (nullable) are indexed like the prompts.
+ * A queue of more than KLPM_LAST_ONLY_MAX_QUEUE prompts is left untouched and counted in d_n_skipped (nullable,
+ * int32[1], set by the call).  One warp runs one queue; no scratch memory, no tree. */
+#define KLPM_LAST_ONLY_MAX_QUEUE 1024
+rt_status klpm_run_last_only_batch(const int32_t* d_tokens, const int64_t* d_offsets, const int64_t* d_arrival,
+                                   const int64_t* d_tie_priority, const int32_t* d_queue_offsets, int32_t n_queues,
+                                   const klpm_params* params, int32_t* d_order, int32_t* d_uncached,
+                                   int64_t* d_ttft, int64_t* d_completion, int32_t* d_n_skipped, void* stream);
 
 /* Version of the ABI (bumped when a signature changes). */
 int32_t klpm_abi_version(void);

@@ -55,6 +55,8 @@ _lib.rt_insert.restype = _i32
 _lib.rt_insert.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp]
 _lib.rt_match_batch.restype = _i32
 _lib.rt_match_batch.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
+_lib.rt_match_batch_ex.restype = _i32
+_lib.rt_match_batch_ex.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.rt_stats.restype = _i32
 _lib.rt_stats.argtypes = [_vp] + [ctypes.POINTER(_i64)] * 5
 _lib.rt_clone.restype = _i32
@@ -78,9 +80,11 @@ _lib.klpm_select_noalloc.argtypes = [_vp, _vp, _vp, _i32, _i64, ctypes.POINTER(k
 _lib.klpm_replay.restype = _i32
 _lib.klpm_replay.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp]
 _lib.klpm_run_ex.restype = _i32
-_lib.klpm_run_ex.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.klpm_run_ex.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.klpm_batch_times.restype = _i32
 _lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp]
+_lib.klpm_run_last_only_batch.restype = _i32
+_lib.klpm_run_last_only_batch.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.klpm_debug_set.restype = _i32
 _lib.klpm_debug_set.argtypes = [ctypes.c_char_p, _i64]
 _lib.klpm_run_path.restype = _i32
@@ -88,8 +92,10 @@ _lib.klpm_run_path.argtypes = [_vp]
 _lib.klpm_run.restype = _i32
 _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp]
 
-EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_stats",
-           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times", "klpm_debug_set"]
+MATCH_STATE_BYTES = 32
+
+EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_match_batch_ex", "rt_stats",
+           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times", "klpm_debug_set", "klpm_run_last_only_batch"]
 
 
 def lib() -> ctypes.CDLL:
@@ -174,6 +180,23 @@ def rt_match_batch(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, 
     _check(_lib.rt_match_batch(tree.handle, _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
                                nq, _dev(match_len, torch.int32, "match_len"), _dev(term_node, torch.int32, "term_node", True),
                                _dev(term_off, torch.int32, "term_off", True), _stream()), "rt_match_batch")
+
+
+def match_state_buffer(nq: int, device) -> torch.Tensor:
+    """Device memory for the records rt_match_batch_ex keeps for klpm_run_ex (klpm_match_state[nq], opaque)."""
+    return torch.empty((max(int(nq), 1), MATCH_STATE_BYTES // 8), dtype=torch.int64, device=device)
+
+
+def rt_match_batch_ex(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, match_len: torch.Tensor,
+                      term_node: Optional[torch.Tensor] = None, term_off: Optional[torch.Tensor] = None,
+                      state: Optional[torch.Tensor] = None) -> None:
+    nq = q_offsets.numel() - 1
+    if state is not None and state.numel() * 8 < nq * MATCH_STATE_BYTES:
+        raise ValueError("state must hold %d bytes per query" % MATCH_STATE_BYTES)
+    _check(_lib.rt_match_batch_ex(tree.handle, _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
+                                  nq, _dev(match_len, torch.int32, "match_len"), _dev(term_node, torch.int32, "term_node", True),
+                                  _dev(term_off, torch.int32, "term_off", True), _dev(state, torch.int64, "state", True),
+                                  _stream()), "rt_match_batch_ex")
 
 
 def rt_stats(tree: Tree) -> dict:
@@ -283,6 +306,29 @@ def klpm_batch_times(order: torch.Tensor, arrival: torch.Tensor, completion: tor
                                  _dev(n_skipped, torch.int32, "n_skipped", True), _stream()), "klpm_batch_times")
 
 
+LAST_ONLY_MAX_QUEUE = 1024
+
+
+def klpm_run_last_only_batch(tokens: torch.Tensor, offsets: torch.Tensor, arrival: torch.Tensor,
+                             tie_priority: Optional[torch.Tensor], queue_offsets: torch.Tensor, params: klpm_params,
+                             order: torch.Tensor, uncached: torch.Tensor, ttft: torch.Tensor,
+                             completion: Optional[torch.Tensor] = None, n_skipped: Optional[torch.Tensor] = None) -> None:
+    """Many independent queues under the last-prompt cache, one warp each (see include/klpm.h)."""
+    n_prompts = offsets.numel() - 1
+    for t, name in ((arrival, "arrival"), (order, "order"), (uncached, "uncached"), (ttft, "ttft")):
+        if t.numel() != n_prompts:
+            raise ValueError("%s must have one entry per prompt" % name)
+    _check(_lib.klpm_run_last_only_batch(_dev(tokens, torch.int32, "tokens"), _dev(offsets, torch.int64, "offsets"),
+                                         _dev(arrival, torch.int64, "arrival"),
+                                         _dev(tie_priority, torch.int64, "tie_priority", True),
+                                         _dev(queue_offsets, torch.int32, "queue_offsets"), queue_offsets.numel() - 1,
+                                         ctypes.byref(params), _dev(order, torch.int32, "order"),
+                                         _dev(uncached, torch.int32, "uncached"), _dev(ttft, torch.int64, "ttft"),
+                                         _dev(completion, torch.int64, "completion", True),
+                                         _dev(n_skipped, torch.int32, "n_skipped", True), _stream()),
+           "klpm_run_last_only_batch")
+
+
 def klpm_debug_set(name: str, value: int) -> None:
     """Process-wide test/debug settings of the library (see include/klpm.h); value < 0 restores the default."""
     _check(_lib.klpm_debug_set(name.encode(), int(value)), "klpm_debug_set")
@@ -290,11 +336,13 @@ def klpm_debug_set(name: str, value: int) -> None:
 
 def klpm_run_ex(tree: Tree, q_tokens: torch.Tensor, q_offsets: torch.Tensor, arrival: torch.Tensor, params: klpm_params,
                 tie_priority: Optional[torch.Tensor], score_mode: int, order: torch.Tensor, uncached: torch.Tensor,
-                ttft: torch.Tensor, completion: Optional[torch.Tensor] = None) -> None:
+                ttft: torch.Tensor, completion: Optional[torch.Tensor] = None,
+                match_state: Optional[torch.Tensor] = None) -> None:
     n = arrival.numel()
     _check(_lib.klpm_run_ex(tree.handle, _dev(q_tokens, torch.int32, "q_tokens"), _dev(q_offsets, torch.int64, "q_offsets"),
                             _dev(arrival, torch.int64, "arrival"), n, ctypes.byref(params),
                             _dev(tie_priority, torch.int64, "tie_priority", True), int(score_mode),
+                            _dev(match_state, torch.int64, "match_state", True),
                             _dev(order, torch.int32, "order"), _dev(uncached, torch.int32, "uncached"),
                             _dev(ttft, torch.int64, "ttft"), _dev(completion, torch.int64, "completion", True), _stream()),
            "klpm_run_ex")

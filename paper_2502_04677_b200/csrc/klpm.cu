@@ -25,6 +25,7 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <atomic>
 #include <new>
 
 #include "klpm.h"
@@ -296,13 +297,14 @@ __device__ __noinline__ int32_t node_after(const EndIndex X, int64_t pos, int64_
 }
 
 // Returns the match length; *node / *off (where the match ended) are filled when want_node is set.
-// With WANT_POS, *last_pos receives the pool index of the last matched token (-1 if nothing matched).
+// With WANT_POS, *last_pos receives the pool index of the last matched token (-1 if nothing matched) and
+// *last_end the end of the contiguous run that token lies in (what node_after needs to name the node later).
 template <bool WANT_POS = false>
 __device__ __forceinline__ int32_t walk_chain(const TreeDev& T, const int32_t* __restrict__ q, int32_t len, bool want_node,
-                              int32_t* node, int32_t* off, int64_t* last_pos = nullptr) {
+                              int32_t* node, int32_t* off, int64_t* last_pos = nullptr, int64_t* last_end = nullptr) {
     const int lane = threadIdx.x & 31;
     *node = 0; *off = 0;
-    if (WANT_POS) *last_pos = -1;
+    if (WANT_POS) { *last_pos = -1; *last_end = 0; }
     if (len <= 0) return 0;
     QWin Q;
     Q.s = (int32_t)((reinterpret_cast<uintptr_t>(q) >> 2) & 3);
@@ -326,7 +328,7 @@ __device__ __forceinline__ int32_t walk_chain(const TreeDev& T, const int32_t* _
         const int32_t x = compare_run(Q, T.pool + (c.span_off - (int64_t)m), m, m + (int32_t)run, lane);
         const int64_t pos = c.span_off + (x - m) - 1;          // x > m: the first token is the key
         m = x;
-        if (WANT_POS) *last_pos = pos;
+        if (WANT_POS) { *last_pos = pos; *last_end = c.chain_end; }
         const int32_t e = node_ending_at(end_index(T), pos, *reinterpret_cast<const volatile long long*>(&T.st->n_nodes));
         if (e < 0) {                                           // stopped inside an edge
             if (want_node) {
@@ -518,49 +520,132 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
 #endif
 // One warp per query, queries handed out by an atomic counter (persistent grid).
 // Trees without a budget: stream along contiguous pool runs.
+//
+// Queries are taken in the order of `perm` when it is given: the host buckets them by their first token first, so
+// that queries which start down the same root child -- and therefore read the same pool tokens -- are in flight
+// at the same time and all but the first of them find those tokens in L2.
+//
+// With STATE the kernel also records, per query, what the scheduling loop needs to start from this match instead
+// of walking the query again (MatchState: where the match ended, the run that position lies in, the next token).
+struct alignas(32) MatchState {
+    long long pos;        // pool index of the last matched token, -1 if nothing matched
+    long long chain_end;  // end of the contiguous pool run `pos` lies in
+    int32_t m;            // match length
+    int32_t ntok;         // the query token right after the match (0 if the whole query matched)
+    unsigned long long tag;   // which match call wrote this record
+};
+static_assert(sizeof(MatchState) == sizeof(klpm_match_state), "klpm_match_state is the ABI's view of MatchState");
+
+template <bool STATE>
 __global__ void __launch_bounds__(256, KLPM_MATCH_MIN_BLOCKS)
 match_chain_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
-                   int32_t* __restrict__ mlen, int32_t* __restrict__ tnode, int32_t* __restrict__ toff,
+                   const int32_t* __restrict__ perm, int32_t* __restrict__ mlen, int32_t* __restrict__ tnode,
+                   int32_t* __restrict__ toff, MatchState* __restrict__ state, unsigned long long tag,
                    unsigned long long* counter) {
     const int lane = threadIdx.x & 31;
     const bool want_node = tnode != nullptr || toff != nullptr;
     for (;;) {
-        unsigned long long i = 0;
-        if (lane == 0) i = atomicAdd(counter, 1ULL);
-        i = __shfl_sync(FULL_MASK, i, 0);
-        if (i >= (unsigned long long)nq) return;
+        unsigned long long c = 0;
+        if (lane == 0) c = atomicAdd(counter, 1ULL);
+        c = __shfl_sync(FULL_MASK, c, 0);
+        if (c >= (unsigned long long)nq) return;
+        const int64_t i = perm ? (int64_t)__ldg(perm + c) : (int64_t)c;
         const int64_t lo = __ldg(qoff + i);
         int64_t len = __ldg(qoff + i + 1) - lo;
         if (len < 0 || len > 0x7fffffffLL) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
         int32_t node, off;
-        const int32_t m = walk_chain(T, qtok + lo, (int32_t)len, want_node, &node, &off);
+        int64_t pos = -1, cend = 0;
+        const int32_t m = STATE ? walk_chain<true>(T, qtok + lo, (int32_t)len, want_node, &node, &off, &pos, &cend)
+                                : walk_chain<false>(T, qtok + lo, (int32_t)len, want_node, &node, &off);
         if (lane == 0) {
-            mlen[i] = m;
+            if (mlen) mlen[i] = m;
             if (tnode) tnode[i] = node;
             if (toff) toff[i] = off;
+            if (STATE) {
+                const int32_t ntok = m < (int32_t)len ? __ldg(qtok + lo + m) : 0;
+                int4* dst = reinterpret_cast<int4*>(state + i);
+                __stcg(dst, make_int4((int)(unsigned)(unsigned long long)pos, (int)(unsigned)((unsigned long long)pos >> 32),
+                                      (int)(unsigned)(unsigned long long)cend, (int)(unsigned)((unsigned long long)cend >> 32)));
+                __stcg(dst + 1, make_int4(m, ntok, (int)(unsigned)tag, (int)(unsigned)(tag >> 32)));
+            }
         }
     }
+}
+
+// The order in which the batched match takes the queries: bucketed by first token (counting sort over a hash of
+// it; the order inside a bucket is whatever the atomics give -- results do not depend on it).
+#define KLPM_ORDER_BUCKETS 65536
+__device__ __forceinline__ unsigned order_bucket(const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t i) {
+    const int64_t lo = __ldg(qoff + i);
+    if (__ldg(qoff + i + 1) <= lo) return 0u;
+    unsigned h = (unsigned)__ldg(qtok + lo) * 0x9E3779B1u;
+    return h >> 16;
+}
+__global__ void order_hist_kernel(const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
+                                  unsigned* __restrict__ hist, unsigned short* __restrict__ bucket) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nq) return;
+    const unsigned b = order_bucket(qtok, qoff, i);
+    bucket[i] = (unsigned short)b;
+    atomicAdd(hist + b, 1u);
+}
+// hist[b] <- number of queries in buckets below b (one CTA of 1,024 threads, 64 buckets each)
+__global__ void __launch_bounds__(1024) order_scan_kernel(unsigned* hist) {
+    __shared__ unsigned s_w[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int PER = KLPM_ORDER_BUCKETS / 1024;
+    unsigned v[PER], sum = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) { v[j] = hist[tid * PER + j]; sum += v[j]; }
+    unsigned inc = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const unsigned o = __shfl_up_sync(FULL_MASK, inc, d); if (lane >= d) inc += o; }
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned w = s_w[lane], wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const unsigned o = __shfl_up_sync(FULL_MASK, wi, d); if (lane >= d) wi += o; }
+        s_w[lane] = wi - w;
+    }
+    __syncthreads();
+    unsigned run = s_w[warp] + inc - sum;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) { hist[tid * PER + j] = run; run += v[j]; }
+}
+__global__ void order_scatter_kernel(const unsigned short* __restrict__ bucket, int32_t nq, unsigned* __restrict__ cursor,
+                                     int32_t* __restrict__ perm) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nq) return;
+    perm[atomicAdd(cursor + bucket[i], 1u)] = i;
 }
 
 // Trees with a budget (evicted children break the runs): hop by hop.
 __global__ void __launch_bounds__(256)
 match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
-                   int32_t* __restrict__ mlen, int32_t* __restrict__ tnode, int32_t* __restrict__ toff,
+                   const int32_t* __restrict__ perm, int32_t* __restrict__ mlen, int32_t* __restrict__ tnode,
+                   int32_t* __restrict__ toff, MatchState* __restrict__ state, unsigned long long tag,
                    unsigned long long* counter) {
     const int lane = threadIdx.x & 31;
     for (;;) {
-        unsigned long long i = 0;
-        if (lane == 0) i = atomicAdd(counter, 1ULL);
-        i = __shfl_sync(FULL_MASK, i, 0);
-        if (i >= (unsigned long long)nq) return;
+        unsigned long long c = 0;
+        if (lane == 0) c = atomicAdd(counter, 1ULL);
+        c = __shfl_sync(FULL_MASK, c, 0);
+        if (c >= (unsigned long long)nq) return;
+        const int64_t i = perm ? (int64_t)__ldg(perm + c) : (int64_t)c;
         const int64_t lo = __ldg(qoff + i), hi = __ldg(qoff + i + 1);
         int64_t len = hi - lo;
         if (len < 0 || len > 0x7fffffffLL) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
         Term t = walk<true>(T, qtok + lo, (int32_t)len);
         if (lane == 0) {
-            mlen[i] = t.m;
+            if (mlen) mlen[i] = t.m;
             if (tnode) tnode[i] = t.node;
             if (toff) toff[i] = t.off;
+            if (state) {
+                MatchState r;
+                r.pos = t.pos; r.chain_end = 0; r.m = t.m; r.ntok = t.m < (int32_t)len ? __ldg(qtok + lo + t.m) : 0; r.tag = tag;
+                state[i] = r;
+            }
         }
     }
 }
@@ -1223,7 +1308,7 @@ run_kernel(TreeDev T, RunArgs A) {
     if (threadIdx.x == 0) {
         const int st_global = *(volatile int*)&gst->status;
         TreeState out = s_st;
-        if (out.status == 0) out.status = st_global;
+        if (out.status == 0) { out.status = st_global; out.detail = *(volatile int*)&gst->detail; }
         *gst = out;
         if (!ok) *(volatile int32_t*)&A.bc->abort = 1;
         __threadfence();
@@ -1297,8 +1382,6 @@ struct FastArgs {
     unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts
     const long long* lk;          // list mode: every slot's key, largest first, stored as ~key with the top bit flipped
     const int32_t* ls;            //            and the slot it belongs to
-    unsigned long long* counter;  // work counter of the initial walk
-    int32_t* pm; int32_t* pnode; int32_t* poff;   // per query (nullable): where its walk ended, for the insertion after the loop
     const int64_t* arrival;       // per query: arrival (for the charge pass after the loop)
     struct FastPost* post;        // where list mode began, for the charge pass after the loop
     TreeState* st;
@@ -1373,39 +1456,28 @@ __global__ void hit_rate_guard_kernel(const int64_t* __restrict__ off, int32_t n
     if (i < n && off[i + 1] - off[i] > KLPM_HIT_RATE_MAX_LEN) set_status(st, RT_ERR_INVALID, 109);
 }
 
-// The one match of every query against the tree: one warp per slot, slots handed out by a counter.
-__global__ void __launch_bounds__(256)
-fast_walk_kernel(TreeDev T, FastArgs A, long long np2) {
-    const int lane = threadIdx.x & 31;
-    for (;;) {
-        unsigned long long i = 0;
-        if (lane == 0) i = atomicAdd(A.counter, 1ULL);
-        i = __shfl_sync(FULL_MASK, i, 0);
-        if (i >= (unsigned long long)np2) return;
-        const int32_t r = (int32_t)i;
-        if (r >= A.n) {                                   // padding of the sort
-            if (lane == 0) { A.gh[r] = 0x7fffffffffffffffLL; A.gidx[r] = 0x7fffffff; }
-            continue;
-        }
-        const FStat s = ld_stat(A.stat + r);
-        int32_t len = s.len;
-        if (len < 0) { if (lane == 0) set_status(T.st, RT_ERR_INVALID); len = 0; }
-        const int32_t* q = A.tok + s.soff;
-        int32_t node, off;
-        int64_t pos;
-        const int32_t m = walk_chain<true>(T, q, len, A.pm != nullptr, &node, &off, &pos);
-        if (lane == 0) {
-            if (A.pm) {       // the insertion after the loop starts from this walk: the tree does not change in between
-                const bool full = node == 0 || off == __ldg(T.span_len + node);
-                A.pm[s.ord] = m; A.pnode[s.ord] = node; A.poff[s.ord] = full ? -1 : off;
-            }
-            const int32_t ntok = m < len ? __ldg(q + m) : 0;
-            st_dyn_state(A.dyn + r, pos, m, ntok);
-            A.key[r] = fast_key(m, len, s.rank, A.score_mode);
-            A.gh[r] = (long long)(m < len ? group_hash(pos, ntok) : single_hash(r));
-            A.gidx[r] = r;
-        }
+// Every slot's starting state from the record the batched match wrote for its query (MatchState): match length,
+// position, next token; from those its key and the hash of its group.  One thread per slot (and per padding entry
+// of the sort that follows).
+__global__ void fast_state_kernel(FastArgs A, const MatchState* __restrict__ state, unsigned long long tag, long long np2) {
+    const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= np2) return;
+    if (r >= A.n) { A.gh[r] = 0x7fffffffffffffffLL; A.gidx[r] = 0x7fffffff; return; }      // padding of the sort
+    const FStat s = ld_stat(A.stat + r);
+    const int4* src = reinterpret_cast<const int4*>(state + s.ord);
+    const int4 a = __ldcg(src), b = __ldcg(src + 1);
+    const long long pos_in = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+    int32_t m = b.x, ntok = b.y;
+    long long pos = pos_in;
+    const unsigned long long got = ((unsigned long long)(unsigned)b.w << 32) | (unsigned)b.z;
+    if (got != tag || m < 0 || m > s.len) {          // not the record of that match: say so and start this slot from nothing
+        set_status(A.st, RT_ERR_INVALID, 110);
+        m = 0; pos = -1; ntok = 0;
     }
+    st_dyn_state(A.dyn + r, pos, m, ntok);
+    A.key[r] = fast_key(m, s.len, s.rank, A.score_mode);
+    A.gh[r] = (long long)(m < s.len ? group_hash(pos, ntok) : single_hash((int32_t)r));
+    A.gidx[r] = (int32_t)r;
 }
 
 // after the sort by hash: runs of equal hashes are the groups
@@ -2370,17 +2442,41 @@ bulk_walk_kernel(TreeDev T, BulkArgs A, unsigned n_pending) {
     }
 }
 
-// First round when the prompts have been walked already (by the scheduling loop's set-up, on the tree as it still is):
-// what bulk_walk_kernel does after its walk.
-__global__ void bulk_prewalked_kernel(BulkArgs A, unsigned n_pending) {
-    const unsigned p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= n_pending) return;
-    const int32_t i = A.pend_in[p];
-    const int32_t len = (int32_t)(__ldg(A.off + i + 1) - __ldg(A.off + i));
-    const int32_t m = A.pm[i], off = A.poff[i];
-    if (!(m == len && off < 0)) {
-        if (off >= 0) atomicMin(&A.claim[A.pnode[i]], i);
-        A.pend_out[atomicAdd(A.n_out, 1u)] = i;
+// First round when a batched match of the prompts against the tree as it still is has left its records (MatchState):
+// the node where each match ended is looked up from the position (end_node[] along the run), then what
+// bulk_walk_kernel does after its walk.  One warp per prompt.
+__global__ void __launch_bounds__(256)
+bulk_from_state_kernel(TreeDev T, BulkArgs A, const MatchState* __restrict__ state, unsigned long long tag, unsigned n_pending) {
+    const int lane = threadIdx.x & 31;
+    const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
+        const int32_t i = A.pend_in[p];
+        const int32_t len = (int32_t)(__ldg(A.off + i + 1) - __ldg(A.off + i));
+        const int4* src = reinterpret_cast<const int4*>(state + i);
+        const int4 a = __ldcg(src), b = __ldcg(src + 1);
+        const long long pos = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+        const long long cend = (long long)(((unsigned long long)(unsigned)a.w << 32) | (unsigned)a.z);
+        const int32_t m = b.x;
+        const unsigned long long got = ((unsigned long long)(unsigned)b.w << 32) | (unsigned)b.z;
+        if (got != tag || m < 0 || m > len || pos < -1 || pos >= T.max_pool || cend < 0 || cend > T.max_pool) {
+            if (lane == 0) set_status(T.st, RT_ERR_INVALID, 110);           // not a record of that match: the prompt is left out
+            continue;
+        }
+        int32_t node = 0, off = -1;                          // off < 0: the match ends on a node boundary (or at the root)
+        if (pos >= 0) {
+            const EndIndex X = end_index(T);
+            node = node_ending_at(X, pos, *reinterpret_cast<const volatile long long*>(&T.st->n_nodes));
+            if (node < 0) {
+                node = node_after(X, pos, cend);
+                if (node < 0) { if (lane == 0) set_status(T.st, RT_ERR_LIMIT, 111); continue; }      // cannot happen
+                off = m - __ldg(T.depth_start + node);
+            }
+        }
+        if (lane == 0 && !(m == len && off < 0)) {
+            A.pm[i] = m; A.pnode[i] = node; A.poff[i] = off;
+            if (off >= 0) atomicMin(&A.claim[node], i);
+            A.pend_out[atomicAdd(A.n_out, 1u)] = i;
+        }
     }
 }
 
@@ -2497,6 +2593,139 @@ __global__ void bulk_finish_kernel(TreeState* S, long long n, long long max_cloc
     else S->clock += n;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Many independent small queues under the last-prompt cache (Definition 2 as printed; Section 2.1: only the
+// previously processed prompt is cached).  This is the model the paper's worked example and Theorem 2 speak
+// about, and a Monte-Carlo over random arrival orders (Definition 3) is thousands of such queues: one warp runs
+// one queue from start to finish, so the schedule loop itself is what is data-parallel here.
+// Per decision the warp looks at every prompt of its queue, 32 at a time: who has arrived, who is oldest, and --
+// for a longest-match pick -- overlap(x_i, last processed prompt), computed by the whole warp for the prompts
+// whose first token agrees with it.  The processed flags live in shared memory (one bit per prompt).
+// ------------------------------------------------------------------------------------------------
+#define KLPM_LAST_ONLY_WARPS 4
+struct LastOnlyArgs {
+    const int32_t* tok; const int64_t* off; const int64_t* arrival; const int64_t* prio; const int32_t* qoff;
+    int32_t n_queues;
+    int32_t policy, k;
+    long long c_num, c_den, start_tick;
+    int32_t* order; int32_t* uncached; int64_t* ttft; int64_t* completion; int32_t* n_skipped;
+};
+
+__global__ void __launch_bounds__(32 * KLPM_LAST_ONLY_WARPS)
+last_only_batch_kernel(LastOnlyArgs A) {
+    __shared__ unsigned s_done[KLPM_LAST_ONLY_WARPS][KLPM_LAST_ONLY_MAX_QUEUE / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long r = (long long)blockIdx.x * KLPM_LAST_ONLY_WARPS + warp;
+    if (r >= A.n_queues) return;
+    const int32_t q0 = __ldg(A.qoff + r), n = __ldg(A.qoff + r + 1) - q0;
+    if (n <= 0) return;
+    if (n > KLPM_LAST_ONLY_MAX_QUEUE) {                       // too long for this entry point: left untouched, counted
+        if (lane == 0 && A.n_skipped) atomicAdd(A.n_skipped, 1);
+        return;
+    }
+    unsigned* done = s_done[warp];
+    for (int32_t w = lane; w < KLPM_LAST_ONLY_MAX_QUEUE / 32; w += 32) done[w] = 0u;
+    __syncwarp();
+    const long long INF = 0x7fffffffffffffffLL;
+    long long now = A.start_tick;
+    int32_t last = -1, last_len = 0;                          // the cached prompt (global index) and its length
+    const int32_t* last_x = nullptr;
+    for (int32_t c = 0; c < n; ++c) {
+        // ---- who is waiting; if nobody, idle until the next arrival
+        bool any = false;
+        long long tmin = INF;
+        for (int32_t base = 0; base < n; base += 32) {
+            const int32_t i = base + lane;
+            if (i < n && !((done[i >> 5] >> (i & 31)) & 1u)) {
+                const long long t = __ldg(A.arrival + q0 + i);
+                any = any || t <= now;
+                tmin = t < tmin ? t : tmin;
+            }
+        }
+        any = __any_sync(FULL_MASK, any);
+        if (!any) {
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) { const long long o = __shfl_xor_sync(FULL_MASK, tmin, d); tmin = o < tmin ? o : tmin; }
+            now = tmin;
+        }
+        const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && (c % A.k) == 0);
+        // ---- the pick: best of (score desc, priority asc, arrival asc, index asc); score = 0 on an oldest-first turn,
+        //      and the priority plays no part in it
+        int32_t b_idx = -1, b_score = 0;
+        long long b_prio = 0, b_t = 0;
+        for (int32_t base = 0; base < n; base += 32) {
+            const int32_t i = base + lane;
+            bool waiting = false;
+            long long t = 0, pr = 0;
+            int32_t len = 0;
+            const int32_t* x = nullptr;
+            if (i < n && !((done[i >> 5] >> (i & 31)) & 1u)) {
+                t = __ldg(A.arrival + q0 + i);
+                waiting = t <= now;
+            }
+            int32_t score = 0;
+            if (!fcfs_turn) {
+                bool cmp = false;
+                if (waiting) {
+                    const int64_t lo = __ldg(A.off + q0 + i);
+                    len = (int32_t)(__ldg(A.off + q0 + i + 1) - lo);
+                    x = A.tok + lo;
+                    if (A.prio) pr = __ldg(A.prio + q0 + i);
+                    cmp = last >= 0 && len > 0 && last_len > 0 && __ldg(x) == __ldg(last_x);
+                }
+                unsigned cm = __ballot_sync(FULL_MASK, cmp);
+                while (cm) {                                  // overlap(x_i, last): the whole warp compares one prompt at a time
+                    const int src = __ffs(cm) - 1; cm &= cm - 1;
+                    const int32_t* xs = (const int32_t*)__shfl_sync(FULL_MASK, (unsigned long long)x, src);
+                    const int32_t ls = __shfl_sync(FULL_MASK, len, src);
+                    const int32_t e = first_mismatch<true, 1>(xs, last_x, ls < last_len ? ls : last_len);
+                    if (lane == src) score = e;
+                }
+            }
+            if (waiting) {
+                bool wins = b_idx < 0 || score > b_score;
+                if (!wins && score == b_score) {
+                    if (pr != b_prio) wins = pr < b_prio;
+                    else wins = t < b_t || (t == b_t && i < b_idx);
+                }
+                if (wins) { b_idx = i; b_score = score; b_prio = pr; b_t = t; }
+            }
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const int32_t o_idx = __shfl_xor_sync(FULL_MASK, b_idx, d), o_score = __shfl_xor_sync(FULL_MASK, b_score, d);
+            const long long o_prio = __shfl_xor_sync(FULL_MASK, b_prio, d), o_t = __shfl_xor_sync(FULL_MASK, b_t, d);
+            bool wins = o_idx >= 0 && (b_idx < 0 || o_score > b_score);
+            if (!wins && o_idx >= 0 && b_idx >= 0 && o_score == b_score) {
+                if (o_prio != b_prio) wins = o_prio < b_prio;
+                else wins = o_t < b_t || (o_t == b_t && o_idx < b_idx);
+            }
+            if (wins) { b_idx = o_idx; b_score = o_score; b_prio = o_prio; b_t = o_t; }
+        }
+        const int32_t j = b_idx;                               // somebody is waiting, so j >= 0
+        if (j < 0) return;
+        // ---- charge by Definition 2 against the cached prompt, then x_j is the cached prompt
+        const int64_t lo = __ldg(A.off + q0 + j);
+        const int32_t len = (int32_t)(__ldg(A.off + q0 + j + 1) - lo);
+        const int32_t* x = A.tok + lo;
+        int32_t m = 0;
+        if (last >= 0) m = first_mismatch<true, 1>(x, last_x, len < last_len ? len : last_len);
+        const int32_t unc = len - m;
+        const long long tj = __ldg(A.arrival + q0 + j);
+        const long long begin = now > tj ? now : tj;
+        const long long R = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
+        if (lane == 0) {
+            A.order[q0 + c] = j;
+            A.uncached[q0 + j] = unc;
+            A.ttft[q0 + j] = R - tj;
+            if (A.completion) A.completion[q0 + j] = R;
+            done[j >> 5] |= 1u << (j & 31);
+        }
+        __syncwarp();
+        now = R; last = j; last_len = len; last_x = x;
+    }
+}
+
 // batch size B: a query is finished when the last query of its bin of the processing order is
 __global__ void batch_times_kernel(const int32_t* __restrict__ order, int32_t n, const int64_t* __restrict__ arrival,
                                    const int64_t* __restrict__ completion, int32_t n_queries, int32_t B, int64_t* ttft_b,
@@ -2605,6 +2834,15 @@ struct rt_tree {
     int device;
     cudaStream_t last_stream;
     unsigned long long* match_counter;
+    // batched match: the order in which queries are taken (bucketed by first token)
+    long long match_cap;    // queries the three arrays below hold
+    int32_t* match_perm; unsigned short* match_bucket; unsigned int* match_hist;
+    // match records (MatchState): which match call wrote the caller's, and the library's own for klpm_run without one
+    unsigned long long version;        // bumped by every call that changes the tree
+    unsigned long long ms_tag, ms_version;
+    const void *ms_state, *ms_tok, *ms_off;
+    int32_t ms_n;
+    MatchState* own_state; long long own_state_cap;
     // klpm_run scratch
     long long run_cap;      // slots allocated (power of two)
     long long* run_key; int32_t* run_ord; int32_t* run_m; int32_t* run_hint; long long* run_pos;
@@ -2650,6 +2888,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->ck_first_tok);
     cudaFree(d.span_off); cudaFree(d.last_access); cudaFree(d.dead); cudaFree(d.clock_owner);
     cudaFree(d.table); cudaFree(d.pool); cudaFree(d.end_node); cudaFree(d.st); cudaFree(t->match_counter);
+    cudaFree(t->match_perm); cudaFree(t->match_bucket); cudaFree(t->match_hist); cudaFree(t->own_state);
     cudaFree(t->run_key); cudaFree(t->run_ord); cudaFree(t->run_m); cudaFree(t->run_hint);
     cudaFree(t->run_pos); cudaFree(t->run_soff); cudaFree(t->run_slen); cudaFree(t->run_ntok);
     cudaFree(t->run_pkey); cudaFree(t->run_pinv); cudaFree(t->run_prank);
@@ -2712,7 +2951,6 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_gh, np2))) return s;
     if ((s = dalloc(&t->fast_gidx, np2))) return s;
     if ((s = dalloc(&t->fast_done, 2 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap
-    if ((s = dalloc(&t->fast_counter, 1))) return s;
     if ((s = dalloc(&t->fast_lk, np2))) return s;
     if ((s = dalloc(&t->fast_ls, np2))) return s;
     if (!t->fast_post && (s = dalloc(&t->fast_post, 1))) return s;
@@ -2753,8 +2991,10 @@ rt_status ensure_bulk_scratch(rt_tree* t, int32_t n) {
     return RT_OK;
 }
 
-// `prewalked`: bulk_pm / bulk_pnode / bulk_poff already hold every prompt's walk on the tree as it is now.
-rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s, bool prewalked = false) {
+// `state` (nullable): records of a batched match of these prompts against the tree as it is now; the first round
+// then needs no walk.
+rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s,
+                      const MatchState* state = nullptr, unsigned long long tag = 0) {
     rt_status st = ensure_bulk_scratch(t, n);
     if (st) return st;
     int32_t *pend_a = t->bulk_pend_a, *pend_b = t->bulk_pend_b, *pm = t->bulk_pm, *pnode = t->bulk_pnode, *poff = t->bulk_poff;
@@ -2775,7 +3015,7 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
         if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
         e = cudaMemsetAsync(n_out, 0, 3 * sizeof(unsigned), s);
         if (e != cudaSuccess) break;
-        if (prewalked && rounds == 1) bulk_prewalked_kernel<<<(count + 255) / 256, 256, 0, s>>>(a, count);
+        if (state && rounds == 1) bulk_from_state_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, state, tag, count);
         else bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
         bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
         e = cudaGetLastError();
@@ -2795,6 +3035,48 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
     cudaStreamSynchronize(s);
     if (e != cudaSuccess) { fprintf(stderr, "klpm: bulk insert failed: %s\n", cudaGetErrorString(e)); return RT_ERR_CUDA; }
     return st;
+}
+
+#define KLPM_ORDER_MIN 2048       // smaller batches are matched in index order (three launches saved)
+std::atomic<unsigned long long> g_match_tag{0};
+
+// The batched match: the order in which the queries are taken, then the kernel.  `state` (nullable) receives the
+// per-query records, stamped with `tag`.
+rt_status launch_match(rt_tree* t, const int32_t* d_q_tokens, const int64_t* d_q_offsets, int32_t nq, int32_t* d_match_len,
+                       int32_t* d_term_node, int32_t* d_term_off, MatchState* state, unsigned long long tag, cudaStream_t s) {
+    const int32_t* perm = nullptr;
+    if (nq >= KLPM_ORDER_MIN) {
+        if (nq > t->match_cap) {
+            cudaFree(t->match_perm); cudaFree(t->match_bucket);
+            t->match_perm = nullptr; t->match_bucket = nullptr; t->match_cap = 0;
+            rt_status st;
+            if ((st = dalloc(&t->match_perm, nq)) || (st = dalloc(&t->match_bucket, nq))) return st;
+            t->match_cap = nq;
+        }
+        if (!t->match_hist) { rt_status st = dalloc(&t->match_hist, KLPM_ORDER_BUCKETS); if (st) return st; }
+        const unsigned qb = (unsigned)((nq + 255) / 256);
+        CK(cudaMemsetAsync(t->match_hist, 0, KLPM_ORDER_BUCKETS * sizeof(unsigned int), s));
+        order_hist_kernel<<<qb, 256, 0, s>>>(d_q_tokens, d_q_offsets, nq, t->match_hist, t->match_bucket);
+        order_scan_kernel<<<1, 1024, 0, s>>>(t->match_hist);
+        order_scatter_kernel<<<qb, 256, 0, s>>>(t->match_bucket, nq, t->match_hist, t->match_perm);
+        perm = t->match_perm;
+    }
+    CK(cudaMemsetAsync(t->match_counter, 0, sizeof(unsigned long long), s));
+    const int threads = 256, warps_per_block = threads / 32;
+    long long blocks = ((long long)nq + warps_per_block - 1) / warps_per_block;
+    const long long max_blocks = (long long)t->num_sms * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (t->cfg.budget_tokens == 0) {
+        if (state) match_chain_kernel<true><<<(unsigned)blocks, threads, 0, s>>>(t->dev, d_q_tokens, d_q_offsets, nq, perm, d_match_len,
+                                                                               d_term_node, d_term_off, state, tag, t->match_counter);
+        else match_chain_kernel<false><<<(unsigned)blocks, threads, 0, s>>>(t->dev, d_q_tokens, d_q_offsets, nq, perm, d_match_len,
+                                                                            d_term_node, d_term_off, nullptr, 0ULL, t->match_counter);
+    } else {
+        match_batch_kernel<<<(unsigned)blocks, threads, 0, s>>>(t->dev, d_q_tokens, d_q_offsets, nq, perm, d_match_len,
+                                                               d_term_node, d_term_off, state, tag, t->match_counter);
+    }
+    CK(cudaGetLastError());
+    return RT_OK;
 }
 
 }  // namespace
@@ -2874,6 +3156,7 @@ rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_off
                     int32_t* d_new_tokens, void* stream) {
     if (!tree || n < 0 || (n > 0 && (!d_tokens || !d_offsets))) return RT_ERR_INVALID;
     if (n == 0) return RT_OK;
+    tree->version++;
     if (!d_new_tokens && tree->cfg.budget_tokens == 0 && n >= 64) {
         tree->last_stream = (cudaStream_t)stream;
         return bulk_insert(tree, d_tokens, d_offsets, n, (cudaStream_t)stream);
@@ -2899,25 +3182,27 @@ rt_status rt_build(const int32_t* d_tokens, const int64_t* d_offsets, int32_t n_
     return RT_OK;
 }
 
-rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, int32_t nq,
-                         int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off, void* stream) {
+rt_status rt_match_batch_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, int32_t nq,
+                            int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off, klpm_match_state* d_state,
+                            void* stream) {
     if (!tree || nq < 0 || (nq > 0 && (!d_q_tokens || !d_q_offsets || !d_match_len))) return RT_ERR_INVALID;
     if (nq == 0) return RT_OK;
     cudaStream_t s = (cudaStream_t)stream;
-    const_cast<rt_tree*>(tree)->last_stream = s;
-    CK(cudaMemsetAsync(tree->match_counter, 0, sizeof(unsigned long long), s));
-    const int threads = 256, warps_per_block = threads / 32;
-    long long blocks = ((long long)nq + warps_per_block - 1) / warps_per_block;
-    long long max_blocks = (long long)tree->num_sms * 8;
-    if (blocks > max_blocks) blocks = max_blocks;
-    if (tree->cfg.budget_tokens == 0)
-        match_chain_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
-                                                               d_term_node, d_term_off, tree->match_counter);
-    else
-        match_batch_kernel<<<(unsigned)blocks, threads, 0, s>>>(tree->dev, d_q_tokens, d_q_offsets, nq, d_match_len,
-                                                               d_term_node, d_term_off, tree->match_counter);
-    CK(cudaGetLastError());
-    return RT_OK;
+    tree->last_stream = s;
+    unsigned long long tag = 0;
+    if (d_state) {
+        tag = ++g_match_tag;
+        tree->ms_tag = tag; tree->ms_version = tree->version; tree->ms_state = d_state; tree->ms_tok = d_q_tokens;
+        tree->ms_off = d_q_offsets; tree->ms_n = nq;
+    }
+    return launch_match(tree, d_q_tokens, d_q_offsets, nq, d_match_len, d_term_node, d_term_off,
+                        reinterpret_cast<MatchState*>(d_state), tag, s);
+}
+
+rt_status rt_match_batch(const rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, int32_t nq,
+                         int32_t* d_match_len, int32_t* d_term_node, int32_t* d_term_off, void* stream) {
+    return rt_match_batch_ex(const_cast<rt_tree*>(tree), d_q_tokens, d_q_offsets, nq, d_match_len, d_term_node, d_term_off,
+                             nullptr, stream);
 }
 
 rt_status rt_stats(rt_tree* tree, int64_t* n_nodes, int64_t* n_tokens, int64_t* clock, int64_t* evictions, int64_t* pool_used) {
@@ -3001,6 +3286,7 @@ rt_status rt_checkpoint(rt_tree* tree, void* stream) {
 
 rt_status rt_rollback(rt_tree* tree, void* stream) {
     if (!tree || !tree->ck_valid) return RT_ERR_INVALID;
+    tree->version++;
     TreeDev& d = tree->dev;
     const unsigned long long cap = d.table_mask + 1;
     cudaStream_t st = (cudaStream_t)stream;
@@ -3123,6 +3409,7 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
     if (!tree || !params_ok(params) || n_order < 0 || n_queries < 0 ||
         (n_order > 0 && (!d_order || !d_q_tokens || !d_q_offsets || !d_arrival || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
     if (n_order == 0) return RT_OK;
+    tree->version++;
     SeqArgs a;
     memset(&a, 0, sizeof(a));
     a.tok = d_q_tokens; a.off = d_q_offsets; a.arrival = d_arrival; a.order = d_order; a.n = n_order; a.n_queries = n_queries;
@@ -3150,12 +3437,17 @@ rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_
 
 rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
                       int32_t n, const klpm_params* params, const int64_t* d_tie_priority, int32_t score_mode,
-                      int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream) {
+                      const klpm_match_state* d_match_state, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                      int64_t* d_completion, void* stream) {
     if (!tree || !params_ok(params) || n < 0 || score_mode < 0 || score_mode > 1 ||
         (n > 0 && (!d_q_tokens || !d_q_offsets || !d_arrival || !d_order || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
     if (n == 0) return RT_OK;
+    // records of a batched match are only good for the queries they were written for and the tree as it was then
+    if (d_match_state && (tree->ms_state != (const void*)d_match_state || tree->ms_n != n || tree->ms_tok != (const void*)d_q_tokens ||
+                          tree->ms_off != (const void*)d_q_offsets || tree->ms_version != tree->version)) return RT_ERR_INVALID;
     cudaStream_t s = (cudaStream_t)stream;
     tree->last_stream = s;
+    tree->version++;
     rt_status st = ensure_run_scratch(tree, n);
     if (st) return st;
     long long np2 = 1;
@@ -3188,18 +3480,29 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.order = d_order; f.uncached = d_uncached; f.ttft = d_ttft; f.completion = d_completion;
         f.dyn = tree->fast_dyn; f.stat = tree->fast_stat; f.key = tree->fast_key_arr; f.mem = tree->fast_mem;
         f.pinv = d_tie_priority ? tree->run_pinv : nullptr;
-        f.gh = tree->fast_gh; f.gidx = tree->fast_gidx; f.done = tree->fast_done; f.counter = tree->fast_counter;
-        f.pm = tree->bulk_pm; f.pnode = tree->bulk_pnode; f.poff = tree->bulk_poff;
+        f.gh = tree->fast_gh; f.gidx = tree->fast_gidx; f.done = tree->fast_done;
         f.arrival = d_arrival; f.post = tree->fast_post;
         f.vbase = tree->dev.max_pool + 16;
         f.st = tree->dev.st;
-        // every query is matched once against the tree as it stands
+        // Every query is matched once against the tree as it stands: by the caller's batched match if it kept the
+        // records (rt_match_batch_ex), by the same kernel here otherwise.
+        const MatchState* state = reinterpret_cast<const MatchState*>(d_match_state);
+        unsigned long long tag = tree->ms_tag;
+        if (!state) {
+            if (n > tree->own_state_cap) {
+                cudaFree(tree->own_state);
+                tree->own_state = nullptr; tree->own_state_cap = 0;
+                if ((st = dalloc(&tree->own_state, n))) return st;
+                tree->own_state_cap = n;
+            }
+            tag = ++g_match_tag;
+            st = launch_match(tree, d_q_tokens, d_q_offsets, n, nullptr, nullptr, nullptr, tree->own_state, tag, s);
+            if (st) return st;
+            state = tree->own_state;
+        }
         fast_stat_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->run_ord, tree->run_key, d_q_offsets,
                                                                      d_tie_priority ? tree->run_prank : nullptr, n, f.stat);
-        CK(cudaMemsetAsync(f.counter, 0, sizeof(unsigned long long), s));
-        long long wblocks = (np2 + 7) / 8;
-        if (wblocks > (long long)tree->num_sms * 8) wblocks = (long long)tree->num_sms * 8;
-        fast_walk_kernel<<<(unsigned)wblocks, 256, 0, s>>>(tree->dev, f, np2);
+        fast_state_kernel<<<(unsigned)((np2 + 255) / 256), 256, 0, s>>>(f, state, tag, np2);
         CK(cudaGetLastError());
         // Leaf blocks of 32 slots while at most 8,192 of them are needed, larger ones beyond (queues above 262,144).
         // Two debug settings shrink the limits so that small queues can exercise the large-queue layout:
@@ -3244,7 +3547,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         tree->run_path = 2;
         // The processed prompts enter the tree together (the logical clock advances by n).  The loop itself needs
         // no room in the tree; if the tree cannot hold the queue the insertion says so through the status word.
-        return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s, true);
+        return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s, state, tag);
     }
     RunBcast bc0;
     memset(&bc0, 0, sizeof(bc0));
@@ -3276,6 +3579,27 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     return RT_OK;
 }
 
+rt_status klpm_run_last_only_batch(const int32_t* d_tokens, const int64_t* d_offsets, const int64_t* d_arrival,
+                                   const int64_t* d_tie_priority, const int32_t* d_queue_offsets, int32_t n_queues,
+                                   const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                                   int64_t* d_completion, int32_t* d_n_skipped, void* stream) {
+    if (!params_ok(params) || n_queues < 0 ||
+        (n_queues > 0 && (!d_tokens || !d_offsets || !d_arrival || !d_queue_offsets || !d_order || !d_uncached || !d_ttft)))
+        return RT_ERR_INVALID;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (d_n_skipped) CK(cudaMemsetAsync(d_n_skipped, 0, sizeof(int32_t), s));
+    if (n_queues == 0) return RT_OK;
+    LastOnlyArgs a;
+    a.tok = d_tokens; a.off = d_offsets; a.arrival = d_arrival; a.prio = d_tie_priority; a.qoff = d_queue_offsets;
+    a.n_queues = n_queues; a.policy = params->policy; a.k = params->k;
+    a.c_num = params->c_num; a.c_den = params->c_den; a.start_tick = params->start_tick;
+    a.order = d_order; a.uncached = d_uncached; a.ttft = d_ttft; a.completion = d_completion; a.n_skipped = d_n_skipped;
+    const unsigned blocks = (unsigned)(((long long)n_queues + KLPM_LAST_ONLY_WARPS - 1) / KLPM_LAST_ONLY_WARPS);
+    last_only_batch_kernel<<<blocks, 32 * KLPM_LAST_ONLY_WARPS, 0, s>>>(a);
+    CK(cudaGetLastError());
+    return RT_OK;
+}
+
 int32_t klpm_run_path(const rt_tree* tree) { return tree ? tree->run_path : 0; }
 
 rt_status klpm_debug_set(const char* name, int64_t value) {
@@ -3292,7 +3616,7 @@ rt_status klpm_debug_set(const char* name, int64_t value) {
 rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
                    int32_t n, const klpm_params* params, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
                    int64_t* d_completion, void* stream) {
-    return klpm_run_ex(tree, d_q_tokens, d_q_offsets, d_arrival, n, params, nullptr, 0, d_order, d_uncached, d_ttft,
+    return klpm_run_ex(tree, d_q_tokens, d_q_offsets, d_arrival, n, params, nullptr, 0, nullptr, d_order, d_uncached, d_ttft,
                        d_completion, stream);
 }
 

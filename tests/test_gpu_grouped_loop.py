@@ -25,7 +25,8 @@ def dev(t):
     return t.cuda() if isinstance(t, torch.Tensor) else torch.as_tensor(t).cuda()
 
 
-def run_gpu(K, prefill, prompts, arr, policy, k, prio=None, score_mode=0, start=0, c_num=0, c_den=1, legacy=False):
+def run_gpu(K, prefill, prompts, arr, policy, k, prio=None, score_mode=0, start=0, c_num=0, c_den=1, legacy=False,
+            from_match=False):
     pt, po = W.to_csr(prefill)
     qt, qo = W.to_csr(prompts)
     n, npre = len(prompts), len(prefill)
@@ -38,9 +39,15 @@ def run_gpu(K, prefill, prompts, arr, policy, k, prio=None, score_mode=0, start=
     comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
     d_prio = None if prio is None else dev(torch.as_tensor(prio, dtype=torch.int64))
     K.klpm_debug_set("run_one_by_one", 1 if legacy else 0)
+    d_qt, d_qo = dev(qt), dev(qo)
+    state = None
+    if from_match:       # the loop starts from the records of a batched match instead of walking the queries itself
+        state = K.match_state_buffer(n, "cuda")
+        m0 = torch.zeros(n, dtype=torch.int32, device="cuda")
+        K.rt_match_batch_ex(tree, d_qt, d_qo, m0, None, None, state)
     try:
-        K.klpm_run_ex(tree, dev(qt), dev(qo), dev(torch.as_tensor(arr, dtype=torch.int64)),
-                      K.make_params(policy, k, c_num, c_den, start), d_prio, score_mode, order, unc, ttft, comp)
+        K.klpm_run_ex(tree, d_qt, d_qo, dev(torch.as_tensor(arr, dtype=torch.int64)),
+                      K.make_params(policy, k, c_num, c_den, start), d_prio, score_mode, order, unc, ttft, comp, state)
     finally:
         K.klpm_debug_set("run_one_by_one", -1)
     assert K.rt_sync_status(tree) == 0
@@ -235,4 +242,42 @@ def test_tree_too_small_for_the_queue(K):
     m = torch.zeros(n, dtype=torch.int32, device="cuda")
     K.rt_match_batch(tree, dev(qt), dev(qo), m)           # the partly filled tree still answers
     assert int(m.max()) <= 12
+    K.rt_destroy(tree)
+
+
+@pytest.mark.parametrize("n", [37, 1500, 5000])
+def test_loop_started_from_the_records_of_a_batched_match(K, n):
+    """rt_match_batch_ex keeps, per query, where its match ended; klpm_run_ex started from those records gives the
+    oracle's schedule and tree, like the call that matches the queries itself (batches below and above the size
+    from which the match takes its queries bucketed by first token)."""
+    prompts, arr = shared_prefix_queue(41, n, [(12, 3), (9, 4)], tail=9, vocab=5, max_gap=2)
+    prefill, _ = shared_prefix_queue(42, 300, [(12, 3), (9, 4)], tail=4, vocab=5, max_gap=0)
+    for policy, k in ((K.POLICY_KLPM, 3), (K.POLICY_LPM, 1)):
+        want = run_oracle(prefill, prompts, arr, policy, k)
+        same(run_gpu(K, prefill, prompts, arr, policy, k, from_match=True), want)
+        same(run_gpu(K, prefill, prompts, arr, policy, k), want)
+
+
+def test_match_records_are_refused_once_they_are_stale(K):
+    prompts, arr = shared_prefix_queue(43, 600, [(10, 3)], tail=6, vocab=4, max_gap=1)
+    qt, qo = W.to_csr(prompts)
+    n = len(prompts)
+    tree = K.rt_create(max_nodes=4 * n + 16, max_pool_tokens=2 * qt.numel() + 16 * n + 16, max_clock=2 * n + 16)
+    d_qt, d_qo, d_arr = dev(qt), dev(qo), dev(torch.as_tensor(arr, dtype=torch.int64))
+    out = [torch.zeros(n, dtype=torch.int32, device="cuda"), torch.zeros(n, dtype=torch.int32, device="cuda"),
+           torch.zeros(n, dtype=torch.int64, device="cuda")]
+    state = K.match_state_buffer(n, "cuda")
+    m = torch.zeros(n, dtype=torch.int32, device="cuda")
+    p = K.make_params(K.POLICY_KLPM, 2)
+    K.rt_match_batch_ex(tree, d_qt, d_qo, m, None, None, state)
+    K.rt_insert(tree, d_qt, d_qo[:3])                      # the tree changes: the records no longer describe it
+    with pytest.raises(K.KlpmError) as e:
+        K.klpm_run_ex(tree, d_qt, d_qo, d_arr, p, None, 0, *out, None, state)
+    assert e.value.code == K.RT_ERR_INVALID
+    K.rt_match_batch_ex(tree, d_qt, d_qo, m, None, None, state)
+    with pytest.raises(K.KlpmError):                        # another buffer than the one the match wrote
+        K.klpm_run_ex(tree, d_qt, d_qo, d_arr, p, None, 0, *out, None, K.match_state_buffer(n, "cuda"))
+    state.zero_()                                           # the caller overwrote the records: caught on the device
+    K.klpm_run_ex(tree, d_qt, d_qo, d_arr, p, None, 0, *out, None, state)
+    assert K.rt_sync_status(tree) == K.RT_ERR_INVALID and K.rt_status_detail(tree) == 110
     K.rt_destroy(tree)
