@@ -208,13 +208,17 @@ struct QWin {
     int32_t len;
 };
 
+// Query tokens are read once and never again: they are loaded with the streaming hint, so that the pool tokens --
+// which other queries of the same trunk are about to read -- are what stays in L2.
+__device__ __forceinline__ int4 ld_query4(const int4* p) { return __ldcs(p); }
+
 // tokens of depths cb + 4 lane .. + 3 (cb a multiple of 4); zeros where nothing needs to be read
 __device__ __forceinline__ int4 qwin_load(const QWin& Q, int32_t cb, int lane) {
     const int4 z = make_int4(0, 0, 0, 0);
     const int32_t p0 = cb + 4 * lane;
-    int4 v = (p0 - Q.s < Q.len) ? __ldg(reinterpret_cast<const int4*>(Q.qa + p0)) : z;
+    int4 v = (p0 - Q.s < Q.len) ? ld_query4(reinterpret_cast<const int4*>(Q.qa + p0)) : z;
     if (Q.s == 0) return v;                                            // warp-uniform
-    int4 e = (cb + 128 - Q.s < Q.len) ? __ldg(reinterpret_cast<const int4*>(Q.qa + cb + 128)) : z;
+    int4 e = (cb + 128 - Q.s < Q.len) ? ld_query4(reinterpret_cast<const int4*>(Q.qa + cb + 128)) : z;
     int4 n;
     n.x = __shfl_down_sync(FULL_MASK, v.x, 1); n.y = __shfl_down_sync(FULL_MASK, v.y, 1); n.z = __shfl_down_sync(FULL_MASK, v.z, 1);
     if (lane == 31) { n.x = e.x; n.y = e.y; n.z = e.z; }
@@ -238,31 +242,69 @@ __device__ __forceinline__ int32_t chunk_mismatch(const int4& A, const int4& P, 
 }
 
 // First depth in [lo, hi) where the query differs from pool_d[depth], or hi.  pool_d is the pool pointer
-// shifted so that pool_d[p] pairs with depth p; it is 16-byte aligned.  KLPM_MATCH_UNROLL chunks of 128
-// tokens are loaded from both sides before the first of them is examined.
-#ifndef KLPM_MATCH_UNROLL
-#define KLPM_MATCH_UNROLL 1
+// shifted so that pool_d[p] pairs with depth p; it is 16-byte aligned.
+#ifndef KLPM_PREFETCH_DIST
+#define KLPM_PREFETCH_DIST 2
 #endif
+// One 128-token chunk with every bound checked: depths below lo and at or above hi take no part.  Returns the first
+// depth where the two sides differ (hi at most), or -1.
+__device__ __forceinline__ int32_t compare_chunk_edge(const QWin& Q, const int4* __restrict__ pool4, int32_t cb, int32_t lo, int32_t hi, int lane) {
+    const int32_t p = cb + 4 * lane;
+    const int4 A = qwin_load(Q, cb, lane);
+    int4 P = A;
+    if (p + 4 > lo && p < hi) P = __ldg(pool4 + (p >> 2));
+    const int32_t r = chunk_mismatch(A, P, p, lo);
+    if (r < 0) return -1;
+    return r < hi ? r : hi;
+}
+
+// Both streams of the chunk KLPM_PREFETCH_DIST ahead are asked into L2 (no register waits for them), so that its
+// loads find them there: a warp keeps more than one chunk of memory latency in flight.
+__device__ __forceinline__ void prefetch_chunk(const QWin& Q, const int4* __restrict__ pool4, int32_t cb, int32_t hi, int lane) {
+#if KLPM_PREFETCH_DIST > 0
+    const int32_t pf = cb + 128 * KLPM_PREFETCH_DIST + 4 * lane;
+    if (pf < hi) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(pool4 + (pf >> 2)));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(Q.qa + pf));
+    }
+#endif
+}
+
 __device__ __forceinline__ int32_t compare_run(const QWin& Q, const int32_t* __restrict__ pool_d, int32_t lo, int32_t hi, int lane) {
-    constexpr int U = KLPM_MATCH_UNROLL;
     const int4* __restrict__ pool4 = reinterpret_cast<const int4*>(pool_d);
-    for (int32_t cb = lo & ~127; cb < hi; cb += 128 * U) {
-        int4 A[U], P[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int32_t p = cb + 128 * u + 4 * lane;
-            A[u] = make_int4(0, 0, 0, 0);
-            if (cb + 128 * u < hi) A[u] = qwin_load(Q, cb + 128 * u, lane);      // warp-uniform condition
-            P[u] = A[u];
-            if (p + 4 > lo && p < hi) P[u] = __ldg(pool4 + (p >> 2));
+    const int4* __restrict__ qa4 = reinterpret_cast<const int4*>(Q.qa);
+    int32_t cb = lo & ~127;
+    // the chunk that holds lo
+    prefetch_chunk(Q, pool4, cb, hi, lane);
+    int32_t r = compare_chunk_edge(Q, pool4, cb, lo, hi, lane);
+    if (r >= 0) return r;
+    cb += 128;
+    // chunks that lie wholly inside [lo, hi): nothing to mask, nothing to bound, and the exact position of a difference
+    // is only worked out once a difference has been seen
+    for (; cb + 128 <= hi; cb += 128) {
+        prefetch_chunk(Q, pool4, cb, hi, lane);
+        const int32_t i4 = (cb >> 2) + lane;
+        int4 v = ld_query4(qa4 + i4);
+        const int4 P = __ldg(pool4 + i4);
+        if (Q.s != 0) {                                                    // warp-uniform
+            const int4 e = ld_query4(qa4 + (cb >> 2) + 32);
+            int32_t nx = __shfl_down_sync(FULL_MASK, v.x, 1), ny = __shfl_down_sync(FULL_MASK, v.y, 1), nz = __shfl_down_sync(FULL_MASK, v.z, 1);
+            if (lane == 31) { nx = e.x; ny = e.y; nz = e.z; }
+            if (Q.s == 1) v = make_int4(v.y, v.z, v.w, nx);
+            else if (Q.s == 2) v = make_int4(v.z, v.w, nx, ny);
+            else v = make_int4(v.w, nx, ny, nz);
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (cb + 128 * u < hi) {
-                const int32_t r = chunk_mismatch(A[u], P[u], cb + 128 * u + 4 * lane, lo);
-                if (r >= 0) return r < hi ? r : hi;
-            }
+        const int32_t dx = v.x ^ P.x, dy = v.y ^ P.y, dz = v.z ^ P.z, dw = v.w ^ P.w;
+        const unsigned bad = __ballot_sync(FULL_MASK, (dx | dy | dz | dw) != 0);
+        if (bad) {
+            const int32_t fc = dx ? 0 : dy ? 1 : dz ? 2 : 3;
+            return __shfl_sync(FULL_MASK, cb + 4 * lane + fc, __ffs(bad) - 1);
         }
+    }
+    // the ragged end
+    if (cb < hi) {
+        r = compare_chunk_edge(Q, pool4, cb, lo, hi, lane);
+        if (r >= 0) return r;
     }
     return hi;
 }
