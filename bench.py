@@ -413,18 +413,12 @@ def k_sweep(K, tree, q_tok, q_off, arr, w, ks, device):
         main = torch.cuda.current_stream()
         a.record(main)
         if mode == "concurrent":
-            # klpm_run waits for its stream on trees without a budget, so every run gets a host thread of its own
-            def one(k, t, st, o):
-                torch.cuda.set_device(device)
-                with torch.cuda.stream(st):
-                    K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
+            # klpm_run only enqueues work: one host thread puts every run on a stream of its own
             for st in streams:
                 st.wait_stream(main)
-            threads = [threading.Thread(target=one, args=(k, t, st, o)) for k, t, st, o in zip(ks, trees, streams, outs)]
-            for th in threads:
-                th.start()
-            for th in threads:
-                th.join()
+            for k, t, st, o in zip(ks, trees, streams, outs):
+                with torch.cuda.stream(st):
+                    K.klpm_run(t, q_tok, q_off, arr, K.make_params(K.POLICY_KLPM, k, 0, 1, w.start_tick), *o)
             for st in streams:
                 main.wait_stream(st)
         else:

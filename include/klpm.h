@@ -85,7 +85,8 @@ rt_status rt_build(const int32_t* d_tokens, const int64_t* d_offsets, int32_t n_
  * stays valid; the condition is reported by rt_sync_status.
  * When d_new_tokens is NULL, the tree has no budget and n >= 64, the prompts are inserted concurrently
  * in rounds instead (same resulting set of cached prefixes and node boundaries; node numbering may
- * differ from run to run); this form waits for `stream` between rounds. */
+ * differ from run to run).  The rounds run on the device (the later ones inside one cooperative kernel
+ * whose grid-wide waits are bounded like every other wait); the call does not wait for them. */
 rt_status rt_insert(rt_tree* tree, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n,
                     int32_t* d_new_tokens, void* stream);
 
@@ -139,7 +140,7 @@ rt_status rt_rollback(rt_tree* tree, void* stream);
 rt_status rt_sync_status(rt_tree* tree, void* stream);
 
 /* A number that says which device-side check recorded the status word (0 if none did): 101/104 a child entry
- * that should exist was not found, 102 a bounded wait of the scheduling loop ran out, 103/105/107 an internal
+ * that should exist was not found, 102/112 a bounded wait of the scheduling loop / of the concurrent insertion ran out, 103/105/107 an internal
  * prediction did not hold, 106 a child lookup probed the whole table, 108 an order entry that is not a query
  * (or a prompt with a negative length), 109 a prompt too long for the hit-rate score.  A debugging aid;
  * synchronises like rt_stats. */
@@ -219,10 +220,10 @@ rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, co
  * On a tree without a budget nothing is ever evicted, so a query's match length changes only when a prompt is
  * processed whose own match ended at the same place and goes on with the same token; the loop then keeps every
  * query's match state itself and stores all processed prompts in the tree at the end, concurrently (as rt_insert
- * does for large batches) -- same outputs, same cached prefixes and node boundaries.  In that case the call waits
- * for `stream` (the concurrent insertion does between its rounds), and a tree too small for the queue still gets
- * every output (they do not depend on the tree's capacity) while the status word reports RT_ERR_CAPACITY and the
- * tree, still valid, holds only part of the queue. */
+ * does for large batches) -- same outputs, same cached prefixes and node boundaries.  A tree too small for the
+ * queue still gets every output (they do not depend on the tree's capacity) while the status word reports
+ * RT_ERR_CAPACITY and the tree, still valid, holds only part of the queue.  Like every other call, klpm_run only
+ * enqueues work (the first call for a queue of a given size also allocates scratch, which synchronises). */
 rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets,
                    const int64_t* d_arrival, int32_t n, const klpm_params* params, int32_t* d_order,
                    int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream);

@@ -147,12 +147,13 @@ struct Term {
     int32_t full;   // 1 if the match ends exactly at the end of that node's edge (or at the root)
 };
 
-// Longest prefix of q on a root path.  Warp-cooperative and warp-uniform.
+// Longest prefix of q on a root path.  Warp-cooperative and warp-uniform.  (cur0, m0): a node boundary the walk may
+// start from instead of the root -- the first m0 tokens of q are known to end exactly at the end of cur0's edge.
 template <bool RO>
-__device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t len) {
-    Term t; t.m = 0; t.node = 0; t.off = 0; t.pos = -1; t.full = 1;
-    if (len <= 0) return t;
-    unsigned long long key = make_key(0, ld32<RO>(q));
+__device__ Term walk(const TreeDev& T, const int32_t* __restrict__ q, int32_t len, int32_t cur0 = 0, int32_t m0 = 0) {
+    Term t; t.m = m0; t.node = cur0; t.off = 0; t.pos = -1; t.full = 1;
+    if (len <= m0) return t;
+    unsigned long long key = make_key(cur0, ld32<RO>(q + m0));
     unsigned long long slot = hash_key(key) & T.table_mask;
     Entry c = ld_entry<RO>(T.table + slot);
     for (;;) {
@@ -2522,6 +2523,97 @@ bulk_from_state_kernel(TreeDev T, BulkArgs A, const MatchState* __restrict__ sta
     }
 }
 
+// What the apply step does for pending prompt number p of the list (one warp): cut the edge its match ends in if it
+// holds the claim, add its leaf if it wins the child's table slot, copy the leaf's tokens, or put the prompt on the
+// list for the next round.  Tree fields are read through L2 (__ldcg): inside the kernel that runs all later rounds,
+// another SM may have written them a moment ago.
+__device__ __forceinline__ void bulk_apply_one(const TreeDev& T, const BulkArgs& A, unsigned p, int lane,
+                                               unsigned long long* s_live_nodes, unsigned long long* s_live_tokens) {
+    TreeState* S = T.st;
+    const int32_t i = __ldcg(A.pend_out + p);
+    const int64_t lo = __ldg(A.off + i);
+    const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
+    const int32_t* x = A.tok + lo;
+    const int32_t m = __ldcg(A.pm + i), node = __ldcg(A.pnode + i), off = __ldcg(A.poff + i);
+    const int32_t unc = len - m;
+    int64_t dst = -1;
+    if (lane == 0) {
+        bool go = true, retry = false;
+        int32_t end = node;
+        if (off >= 0) {                                 // the match ends inside node's edge: cut it
+            if (__ldcg(A.claim + node) != i) { go = false; retry = true; }     // another prompt cuts this edge in this round
+            else {
+                A.claim[node] = 0x7fffffff;
+                const long long u = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
+                if (u >= T.max_nodes) { set_status(S, RT_ERR_CAPACITY); go = false; }
+                else {
+                    atomicAdd(s_live_nodes, 1ULL);
+                    const int32_t par = __ldcg(T.parent + node), ds = __ldcg(T.depth_start + node), sl = __ldcg(T.span_len + node);
+                    const int64_t so = __ldcg(T.span_off + node);
+                    const int32_t t_up = __ldcg(T.pool + so), t_low = __ldcg(T.pool + so + off);
+                    T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
+                    T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
+                    T.first_tok[u] = t_up; T.first_tok[node] = t_low;
+                    long long slot = table_find(T, par, t_up);
+                    int64_t chain_end = so + sl;
+                    if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = __ldcg(&T.table[slot].chain_end); }
+                    else set_status(S, RT_ERR_LIMIT, 104);
+                    T.end_node[so + off - 1] = (int32_t)u;
+                    T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
+                    T.parent[node] = (int32_t)u;
+                    end = (int32_t)u;
+                    // (u, first token of the lower part) -> node : nobody else can want this key
+                    unsigned long long key = make_key(end, t_low);
+                    unsigned long long sl2 = hash_key(key) & T.table_mask;
+                    for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+                        if (atomicCAS(&T.table[sl2].key, 0ULL, key) == 0ULL) {
+                            T.table[sl2].child = node; T.table[sl2].span_len = sl - off; T.table[sl2].span_off = so + off;
+                            T.table[sl2].chain_end = chain_end;
+                            break;
+                        }
+                        sl2 = (sl2 + 1) & T.table_mask;
+                    }
+                }
+            }
+        }
+        if (go && unc > 0) {
+            unsigned long long key = make_key(end, __ldg(x + m));
+            unsigned long long sl2 = hash_key(key) & T.table_mask;
+            long long won = -1;
+            for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+                unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
+                if (old == 0ULL) { won = (long long)sl2; break; }
+                if (old == key) { retry = true; break; }   // another prompt added that child (in this round, or it lost to it before)
+                sl2 = (sl2 + 1) & T.table_mask;
+            }
+            if (won >= 0) {
+                const long long leaf = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
+                const long long raw = (long long)atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)(unc + 6));
+                const long long po = ((raw + 3) & ~3LL) + (m & 3);                  // span_off = depth_start (mod 4)
+                if (leaf >= T.max_nodes || raw + unc + 6 > T.max_pool) {
+                    set_status(S, RT_ERR_CAPACITY);
+                    T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0; T.table[won].chain_end = 0;
+                } else {
+                    T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
+                    T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
+                    T.first_tok[leaf] = __ldg(x + m);
+                    T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
+                    T.table[won].chain_end = po + unc;
+                    T.end_node[po + unc - 1] = (int32_t)leaf;
+                    atomicAdd(&T.nchild[end], 1);
+                    atomicAdd(s_live_tokens, (unsigned long long)unc);
+                    atomicAdd(s_live_nodes, 1ULL);
+                    dst = po;
+                }
+            }
+        }
+        if (retry) A.pend_next[atomicAdd(A.n_next, 1u)] = i;
+    }
+    dst = __shfl_sync(FULL_MASK, dst, 0);
+    if (dst >= 0)
+        for (int32_t t = lane; t < unc; t += 32) T.pool[dst + t] = __ldg(x + m + t);
+}
+
 __global__ void __launch_bounds__(256)
 bulk_apply_kernel(TreeDev T, BulkArgs A) {
     // live nodes and live tokens are statistics only: summed per CTA here, added to the tree's counters once at the end
@@ -2531,94 +2623,123 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
     const unsigned n_pending = *A.n_out;
     const int lane = threadIdx.x & 31;
     const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
-    TreeState* S = T.st;
-    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
-        const int32_t i = A.pend_out[p];
-        const int64_t lo = __ldg(A.off + i);
-        const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
-        const int32_t* x = A.tok + lo;
-        const int32_t m = A.pm[i], node = A.pnode[i], off = A.poff[i];
-        const int32_t unc = len - m;
-        int64_t dst = -1;
-        if (lane == 0) {
-            bool go = true, retry = false;
-            int32_t end = node;
-            if (off >= 0) {                                 // the match ends inside node's edge: cut it
-                if (A.claim[node] != i) { go = false; retry = true; }     // another prompt cuts this edge in this round
-                else {
-                    A.claim[node] = 0x7fffffff;
-                    const long long u = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
-                    if (u >= T.max_nodes) { set_status(S, RT_ERR_CAPACITY); go = false; }
-                    else {
-                        atomicAdd(&s_live_nodes, 1ULL);
-                        const int32_t par = T.parent[node], ds = T.depth_start[node], sl = T.span_len[node];
-                        const int64_t so = T.span_off[node];
-                        T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
-                        T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
-                        T.first_tok[u] = T.pool[so]; T.first_tok[node] = T.pool[so + off];
-                        long long slot = table_find(T, par, T.pool[so]);
-                        int64_t chain_end = so + sl;
-                        if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = T.table[slot].chain_end; }
-                        else set_status(S, RT_ERR_LIMIT, 104);
-                        T.end_node[so + off - 1] = (int32_t)u;
-                        T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
-                        T.parent[node] = (int32_t)u;
-                        end = (int32_t)u;
-                        // (u, first token of the lower part) -> node : nobody else can want this key
-                        unsigned long long key = make_key(end, T.pool[so + off]);
-                        unsigned long long sl2 = hash_key(key) & T.table_mask;
-                        for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
-                            if (atomicCAS(&T.table[sl2].key, 0ULL, key) == 0ULL) {
-                                T.table[sl2].child = node; T.table[sl2].span_len = sl - off; T.table[sl2].span_off = so + off;
-                                T.table[sl2].chain_end = chain_end;
-                                break;
-                            }
-                            sl2 = (sl2 + 1) & T.table_mask;
-                        }
+    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps)
+        bulk_apply_one(T, A, p, lane, &s_live_nodes, &s_live_tokens);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (s_live_nodes) atomicAdd((unsigned long long*)&T.st->live_nodes, s_live_nodes);
+        if (s_live_tokens) atomicAdd((unsigned long long*)&T.st->tokens_live, s_live_tokens);
+    }
+}
+
+// Every round after the first, in one cooperative kernel (no trip to the host between rounds).  A round = bring the
+// pending prompts' positions up to date, grid barrier, apply, grid barrier.  A prompt is pending because it lost a
+// cut to another prompt -- then the depth where its match ends has not moved, only the nodes around it have, and a
+// walk up from the node it knew finds the node that holds that depth now -- or because another prompt added the
+// child it wanted -- then it walks on from the node boundary it had reached, into that child (hop by hop, read
+// through L2: the tokens may have been written by another SM a moment ago).  Counters alternate between rounds so
+// that none is reset while somebody may still read it.  The barrier is bounded in time; when it gives up the status
+// word says RT_ERR_LIMIT and every CTA returns.
+struct BulkSync {
+    unsigned int count, gen, abort, go;      // the barrier; whether another round follows
+    unsigned int cnt_w[2], cnt_a[2];         // list lengths: positions brought up to date -> pend_b; retries -> pend_a
+    unsigned int n_walk;                     // work counter of the first round's walk
+    unsigned int pad[3];
+};
+
+// All threads call it.  `last` runs in one thread of the CTA that arrives last, before anybody is released.
+template <typename F>
+__device__ bool bulk_barrier(BulkSync* g, TreeState* st, long long limit_ns, F last) {
+    __shared__ int s_ok;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        const unsigned gen = *(volatile unsigned*)&g->gen;
+        if (atomicAdd(&g->count, 1u) + 1u == gridDim.x) {
+            last();
+            g->count = 0;
+            __threadfence();
+            atomicAdd(&g->gen, 1u);
+        } else {
+            unsigned long long spins = 0, t0 = 0;
+            while (*(volatile unsigned*)&g->gen == gen) {
+                if (*(volatile unsigned*)&g->abort) { ok = 0; break; }
+                if ((++spins & 1023ULL) == 0 || limit_ns == 0) {
+                    unsigned long long now;
+                    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(now));
+                    if (t0 == 0) t0 = now;
+                    if (limit_ns == 0 || now - t0 > (unsigned long long)limit_ns || spins > (1ULL << 40)) {
+                        set_status(st, RT_ERR_LIMIT, 112); atomicExch(&g->abort, 1u); ok = 0; break;
                     }
                 }
             }
-            if (go && unc > 0) {
-                unsigned long long key = make_key(end, __ldg(x + m));
-                unsigned long long sl2 = hash_key(key) & T.table_mask;
-                long long won = -1;
-                for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
-                    unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
-                    if (old == 0ULL) { won = (long long)sl2; break; }
-                    if (old == key) { retry = true; break; }   // another prompt of this round added that child
-                    sl2 = (sl2 + 1) & T.table_mask;
-                }
-                if (won >= 0) {
-                    const long long leaf = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
-                    const long long raw = (long long)atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)(unc + 6));
-                    const long long po = ((raw + 3) & ~3LL) + (m & 3);                  // span_off = depth_start (mod 4)
-                    if (leaf >= T.max_nodes || raw + unc + 6 > T.max_pool) {
-                        set_status(S, RT_ERR_CAPACITY);
-                        T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0; T.table[won].chain_end = 0;
-                    } else {
-                        T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
-                        T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
-                        T.first_tok[leaf] = __ldg(x + m);
-                        T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
-                        T.table[won].chain_end = po + unc;
-                        T.end_node[po + unc - 1] = (int32_t)leaf;
-                        atomicAdd(&T.nchild[end], 1);
-                        atomicAdd(&s_live_tokens, (unsigned long long)unc);
-                        atomicAdd(&s_live_nodes, 1ULL);
-                        dst = po;
-                    }
-                }
-            }
-            if (retry) A.pend_next[atomicAdd(A.n_next, 1u)] = i;
         }
-        dst = __shfl_sync(FULL_MASK, dst, 0);
-        if (dst >= 0)
-            for (int32_t t = lane; t < unc; t += 32) T.pool[dst + t] = __ldg(x + m + t);
+        if (*(volatile unsigned*)&g->abort) ok = 0;
+        __threadfence();
+        s_ok = ok;
+    }
+    __syncthreads();
+    const bool ok = s_ok != 0;
+    __syncthreads();
+    return ok;
+}
+
+__global__ void __launch_bounds__(256)
+bulk_rounds_kernel(TreeDev T, BulkArgs A, BulkSync* g, long long n_total, long long limit_ns) {
+    __shared__ unsigned long long s_live_nodes, s_live_tokens;
+    if (threadIdx.x == 0) { s_live_nodes = 0ULL; s_live_tokens = 0ULL; }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const unsigned nwarps = (gridDim.x * blockDim.x) >> 5, warp0 = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    TreeState* S = T.st;
+    unsigned count = __ldcg(&g->cnt_a[0]);                 // left pending by the first round (its kernels have completed)
+    for (unsigned r = 1; count > 0; ++r) {
+        const unsigned par = r & 1u;
+        BulkArgs R = A;
+        R.pend_in = A.pend_next; R.n_out = &g->cnt_w[par]; R.n_next = &g->cnt_a[par];
+        // ---- positions of the pending prompts in the tree as it is now
+        for (unsigned p = warp0; p < count; p += nwarps) {
+            const int32_t i = __ldcg(R.pend_in + p);
+            const int64_t lo = __ldg(A.off + i);
+            const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
+            int32_t m = __ldcg(A.pm + i), node = __ldcg(A.pnode + i), off = __ldcg(A.poff + i);
+            bool full = true;
+            if (off >= 0) {                                 // lost a cut: the depth m lies in `node` or in a node cut off above it
+                int32_t a = node, ds = __ldcg(T.depth_start + a);
+                while (a != 0 && m <= ds) { a = __ldcg(T.parent + a); ds = __ldcg(T.depth_start + a); }
+                node = a; off = m - ds;
+                full = a == 0 || off == __ldcg(T.span_len + a);
+            }
+            if (full) {                                     // on a node boundary: walk on into the child that may be there now
+                const Term t = walk<false>(T, A.tok + lo, len, node, m);
+                if (t.m > m) { m = t.m; node = t.node; off = t.off; full = t.full != 0; }
+            }
+            if (lane == 0 && !(m == len && full)) {
+                A.pm[i] = m; A.pnode[i] = node; A.poff[i] = full ? -1 : off;
+                if (!full) atomicMin(&A.claim[node], i);
+                R.pend_out[atomicAdd(R.n_out, 1u)] = i;
+            }
+        }
+        if (!bulk_barrier(g, S, limit_ns, [] {})) break;
+        // ---- cuts and leaves
+        const unsigned n_apply = __ldcg(R.n_out);
+        if (blockIdx.x == 0 && threadIdx.x == 0) { g->cnt_w[par ^ 1u] = 0u; g->cnt_a[par ^ 1u] = 0u; }     // the next round's
+        for (unsigned p = warp0; p < n_apply; p += nwarps) bulk_apply_one(T, R, p, lane, &s_live_nodes, &s_live_tokens);
+        if (!bulk_barrier(g, S, limit_ns, [&] {
+                const bool stop = *(volatile int*)&S->status != 0 || r > 100000000u;
+                g->go = stop ? 0u : *(volatile unsigned*)&g->cnt_a[par];
+            })) break;
+        count = __ldcg(&g->go);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         if (s_live_nodes) atomicAdd((unsigned long long*)&S->live_nodes, s_live_nodes);
         if (s_live_tokens) atomicAdd((unsigned long long*)&S->tokens_live, s_live_tokens);
+        if (blockIdx.x == 0) {                              // the logical clock advances by one per stored prompt
+            if (S->clock + n_total + 1 >= T.max_clock) set_status(S, RT_ERR_CAPACITY);
+            else S->clock += n_total;
+        }
     }
 }
 
@@ -2630,11 +2751,6 @@ __global__ void bulk_fill_kernel(int32_t* p, long long n, int32_t v) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) p[i] = v;
 }
-__global__ void bulk_finish_kernel(TreeState* S, long long n, long long max_clock) {
-    if (S->clock + n + 1 >= max_clock) set_status(S, RT_ERR_CAPACITY);
-    else S->clock += n;
-}
-
 // ------------------------------------------------------------------------------------------------
 // Many independent small queues under the last-prompt cache (Definition 2 as printed; Section 2.1: only the
 // previously processed prompt is cached).  This is the model the paper's worked example and Theorem 2 speak
@@ -2902,7 +3018,7 @@ struct rt_tree {
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
     long long bulk_cap;     // bulk insertion: prompts its per-prompt scratch holds
     int32_t *bulk_pend_a, *bulk_pend_b, *bulk_pm, *bulk_pnode, *bulk_poff;
-    unsigned int* bulk_n_out;
+    BulkSync* bulk_sync;
     // checkpoint (rt_checkpoint / rt_rollback): copies of everything a later call can modify
     bool ck_valid;
     int32_t *ck_parent, *ck_depth_start, *ck_span_len, *ck_nchild, *ck_clock_owner, *ck_first_tok;
@@ -2940,7 +3056,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->fast_lk); cudaFree(t->fast_ls); cudaFree(t->fast_post); cudaFree(t->fast_bsum);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
-    cudaFree(t->bulk_n_out);
+    cudaFree(t->bulk_sync);
     cudaFree(t->ck_parent); cudaFree(t->ck_depth_start); cudaFree(t->ck_span_len); cudaFree(t->ck_nchild);
     cudaFree(t->ck_clock_owner); cudaFree(t->ck_span_off); cudaFree(t->ck_last_access); cudaFree(t->ck_dead);
     cudaFree(t->ck_table); cudaFree(t->ck_st);
@@ -3029,54 +3145,41 @@ rt_status ensure_bulk_scratch(rt_tree* t, int32_t n) {
             (st = dalloc(&t->bulk_pnode, n)) || (st = dalloc(&t->bulk_poff, n))) return st;
         t->bulk_cap = n;
     }
-    if (!t->bulk_n_out && (st = dalloc(&t->bulk_n_out, 3))) return st;      // walk's and apply's list lengths, walk's work counter
+    if (!t->bulk_sync && (st = dalloc(&t->bulk_sync, 1))) return st;        // list lengths, work counter, grid barrier
     return RT_OK;
 }
 
 // `state` (nullable): records of a batched match of these prompts against the tree as it is now; the first round
-// then needs no walk.
+// then needs no walk.  Everything is enqueued on `s`; nothing waits for the device.
 rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s,
                       const MatchState* state = nullptr, unsigned long long tag = 0) {
     rt_status st = ensure_bulk_scratch(t, n);
     if (st) return st;
-    int32_t *pend_a = t->bulk_pend_a, *pend_b = t->bulk_pend_b, *pm = t->bulk_pm, *pnode = t->bulk_pnode, *poff = t->bulk_poff;
-    unsigned int* n_out = t->bulk_n_out;
+    BulkSync* g = t->bulk_sync;
     // claim words start idle (an earlier call that ran out of capacity may have left some set)
     bulk_fill_kernel<<<(unsigned)((t->dev.max_nodes + 255) / 256), 256, 0, s>>>(t->claim, t->dev.max_nodes, 0x7fffffff);
-    bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(pend_a, n);
-    unsigned count = (unsigned)n;
-    cudaError_t e = cudaGetLastError();
-    int rounds = 0;
-    while (e == cudaSuccess && count > 0) {
-        if (++rounds > 1000000) { st = RT_ERR_LIMIT; break; }
-        BulkArgs a;
-        a.tok = d_tokens; a.off = d_offsets; a.pend_in = pend_a; a.pend_out = pend_b; a.n_out = n_out;
-        a.pend_next = pend_a; a.n_next = n_out + 1; a.n_walk = n_out + 2;          // the walk has consumed pend_a by the time apply refills it
-        a.claim = t->claim; a.pm = pm; a.pnode = pnode; a.poff = poff;
-        long long blocks = ((long long)count + 7) / 8;
-        if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
-        e = cudaMemsetAsync(n_out, 0, 3 * sizeof(unsigned), s);
-        if (e != cudaSuccess) break;
-        if (state && rounds == 1) bulk_from_state_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, state, tag, count);
-        else bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, count);
-        bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) break;
-        e = cudaMemcpyAsync(&count, n_out + 1, sizeof(unsigned), cudaMemcpyDeviceToHost, s);
-        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-        if (e == cudaSuccess && count > 0) {
-            TreeState h;
-            e = cudaMemcpy(&h, t->dev.st, sizeof(h), cudaMemcpyDeviceToHost);
-            if (e == cudaSuccess && h.status != 0) break;      // capacity ran out: stop, the status word says why
-        }
-    }
-    if (e == cudaSuccess && st == RT_OK) {
-        bulk_finish_kernel<<<1, 1, 0, s>>>(t->dev.st, (long long)n, t->dev.max_clock);
-        e = cudaGetLastError();
-    }
-    cudaStreamSynchronize(s);
-    if (e != cudaSuccess) { fprintf(stderr, "klpm: bulk insert failed: %s\n", cudaGetErrorString(e)); return RT_ERR_CUDA; }
-    return st;
+    bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(t->bulk_pend_a, n);
+    CK(cudaMemsetAsync(g, 0, sizeof(BulkSync), s));
+    BulkArgs a;
+    a.tok = d_tokens; a.off = d_offsets; a.pend_in = t->bulk_pend_a; a.pend_out = t->bulk_pend_b; a.n_out = &g->cnt_w[0];
+    a.pend_next = t->bulk_pend_a; a.n_next = &g->cnt_a[0]; a.n_walk = &g->n_walk;      // the walk has consumed pend_a by the time apply refills it
+    a.claim = t->claim; a.pm = t->bulk_pm; a.pnode = t->bulk_pnode; a.poff = t->bulk_poff;
+    long long blocks = ((long long)n + 7) / 8;
+    if (blocks > (long long)t->num_sms * 8) blocks = (long long)t->num_sms * 8;
+    // the first round: every prompt from the root (or from its match record), then cuts and leaves
+    if (state) bulk_from_state_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, state, tag, (unsigned)n);
+    else bulk_walk_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a, (unsigned)n);
+    bulk_apply_kernel<<<(unsigned)blocks, 256, 0, s>>>(t->dev, a);
+    CK(cudaGetLastError());
+    // every later round, and the clock, in one cooperative kernel
+    int per_sm = 0;
+    CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bulk_rounds_kernel, 256, 0));
+    if (per_sm < 1) return RT_ERR_CUDA;
+    const unsigned grid = (unsigned)t->num_sms * (unsigned)(per_sm < 2 ? per_sm : 2);
+    long long n_total = n, limit = g_knobs.wait_limit_ns;
+    void* kargs[] = {(void*)&t->dev, (void*)&a, (void*)&g, (void*)&n_total, (void*)&limit};
+    CK(cudaLaunchCooperativeKernel((void*)bulk_rounds_kernel, dim3(grid), dim3(256), kargs, 0, s));
+    return RT_OK;
 }
 
 #define KLPM_ORDER_MIN 2048       // smaller batches are matched in index order (three launches saved)
