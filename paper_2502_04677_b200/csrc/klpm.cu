@@ -572,7 +572,7 @@ __device__ void insert_serial(const TreeDev& T, const int32_t* x, int32_t len, i
 // of walking the query again (MatchState: where the match ended, the run that position lies in, the next token).
 struct alignas(32) MatchState {
     long long pos;        // pool index of the last matched token, -1 if nothing matched
-    long long chain_end;  // end of the contiguous pool run `pos` lies in
+    long long chain_end;  // end of the contiguous pool run `pos` lies in (trees with a budget: the node `pos` lies in)
     int32_t m;            // match length
     int32_t ntok;         // the query token right after the match (0 if the whole query matched)
     unsigned long long tag;   // which match call wrote this record
@@ -686,7 +686,8 @@ match_batch_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* _
             if (toff) toff[i] = t.off;
             if (state) {
                 MatchState r;
-                r.pos = t.pos; r.chain_end = 0; r.m = t.m; r.ntok = t.m < (int32_t)len ? __ldg(qtok + lo + t.m) : 0; r.tag = tag;
+                // trees with a budget have no use for the run's end; the field carries the node the match ended in instead
+                r.pos = t.pos; r.chain_end = t.node; r.m = t.m; r.ntok = t.m < (int32_t)len ? __ldg(qtok + lo + t.m) : 0; r.tag = tag;
                 state[i] = r;
             }
         }
@@ -1392,7 +1393,8 @@ struct alignas(32) FDyn {     // what the loop changes, one 32-byte sector per s
     int32_t m;                // match length; -1 once processed
     int32_t ntok;             // query token right after the match (meaningful while m < length)
     int32_t gstart, gcount;   // the slot's group: run [gstart, gstart + gcount) of the member array
-    long long pad;
+    int32_t hint;             // trees with a budget: a node at or below the node the match ends in (walk up while m <= depth_start)
+    int32_t pad;
 };
 struct alignas(32) FStat {    // constant during the loop; the first 16 bytes are all that charging a pick needs
     long long t;              // arrival
@@ -1428,6 +1430,12 @@ struct FastArgs {
     const int64_t* arrival;       // per query: arrival (for the charge pass after the loop)
     struct FastPost* post;        // where list mode began, for the charge pass after the loop
     TreeState* st;
+    // trees with a budget: the loop keeps the node arrays of the tree up to date itself (LRU needs them at every decision)
+    int32_t lru;                  // 1: the tree has a budget
+    int32_t mem_cap;              // entries of the member array (groups formed by evictions are appended behind the first n)
+    TreeDev T;
+    int32_t* parked;              // per node: unprocessed slots whose hint is that node
+    int32_t* skip;                // set by the capacity check before the loop: leave everything untouched
 };
 
 #define KLPM_FAST_THREADS 256
@@ -1454,7 +1462,7 @@ __device__ __forceinline__ FDyn ld_dyn(const FDyn* p) {
     const int4 a = __ldcg(q), b = __ldcg(q + 1);
     FDyn d;
     d.pos = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
-    d.m = a.z; d.ntok = a.w; d.gstart = b.x; d.gcount = b.y; d.pad = 0;
+    d.m = a.z; d.ntok = a.w; d.gstart = b.x; d.gcount = b.y; d.hint = b.z; d.pad = 0;
     return d;
 }
 __device__ __forceinline__ void st_dyn_state(FDyn* p, long long pos, int32_t m, int32_t ntok) {
@@ -1463,6 +1471,7 @@ __device__ __forceinline__ void st_dyn_state(FDyn* p, long long pos, int32_t m, 
 __device__ __forceinline__ void st_dyn_group(FDyn* p, int32_t gstart, int32_t gcount) {
     __stcg(reinterpret_cast<int2*>(p) + 2, make_int2(gstart, gcount));
 }
+__device__ __forceinline__ void st_dyn_hint(FDyn* p, int32_t hint) { __stcg(reinterpret_cast<int32_t*>(p) + 6, hint); }
 __device__ __forceinline__ FStat ld_stat(const FStat* p) {
     const int4* q = reinterpret_cast<const int4*>(p);
     const int4 a = __ldg(q), b = __ldg(q + 1);
@@ -1510,14 +1519,19 @@ __global__ void fast_state_kernel(FastArgs A, const MatchState* __restrict__ sta
     const int4* src = reinterpret_cast<const int4*>(state + s.ord);
     const int4 a = __ldcg(src), b = __ldcg(src + 1);
     const long long pos_in = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+    const long long node_in = (long long)(((unsigned long long)(unsigned)a.w << 32) | (unsigned)a.z);
     int32_t m = b.x, ntok = b.y;
     long long pos = pos_in;
+    int32_t hint = 0;
     const unsigned long long got = ((unsigned long long)(unsigned)b.w << 32) | (unsigned)b.z;
-    if (got != tag || m < 0 || m > s.len) {          // not the record of that match: say so and start this slot from nothing
+    bool bad = got != tag || m < 0 || m > s.len;
+    if (A.lru && !bad) { bad = node_in < 0 || node_in >= A.T.max_nodes; hint = (int32_t)node_in; }
+    if (bad) {                                       // not the record of that match: say so and start this slot from nothing
         set_status(A.st, RT_ERR_INVALID, 110);
-        m = 0; pos = -1; ntok = 0;
+        m = 0; pos = -1; ntok = 0; hint = 0;
     }
     st_dyn_state(A.dyn + r, pos, m, ntok);
+    if (A.lru) { st_dyn_hint(A.dyn + r, hint); atomicAdd(A.parked + hint, 1); }
     A.key[r] = fast_key(m, s.len, s.rank, A.score_mode);
     A.gh[r] = (long long)(m < s.len ? group_hash(pos, ntok) : single_hash((int32_t)r));
     A.gidx[r] = (int32_t)r;
@@ -1637,9 +1651,17 @@ struct FastPick {             // the prompt being processed, as its group's memb
     long long vleaf;          // virtual pool index of the first token of its new leaf
     long long admitted;       // slots below this have arrived
     int32_t gstart, gcount;
+    int32_t leaf;             // trees with a budget: id of its new leaf (the tied members are parked in it from now on)
 };
 struct FastJob { int32_t type; int32_t a0, a1; FastPick pick; };
-enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2, FAST_JOB_REBUILD = 3, FAST_JOB_BATCH = 4 };
+enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2, FAST_JOB_REBUILD = 3, FAST_JOB_BATCH = 4, FAST_JOB_FALLBACK = 5 };
+
+// trees with a budget: slot r's match now ends inside node `to` (it was counted for node `from`)
+__device__ __forceinline__ void lru_move(const FastArgs& A, int32_t r, int32_t from, int32_t to) {
+    st_dyn_hint(A.dyn + r, to);
+    atomicSub(A.parked + from, 1);
+    atomicAdd(A.parked + to, 1);
+}
 
 // What the sequencer hands to a CTA-wide batch of decisions, and what it gets back.
 struct FastBatchIO {
@@ -1694,6 +1716,7 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
     if (tied) {
         d.m = P.m + e; d.pos = P.vleaf + e - 1; d.ntok = d.m < s.len ? __ldg(q + d.m) : 0;
         st_dyn_state(A.dyn + r, d.pos, d.m, d.ntok);
+        if (A.lru) lru_move(A, r, d.hint, P.leaf);
         const unsigned long long key = fast_key(d.m, s.len, s.rank, A.score_mode);
         __stcg(A.key + r, key);
         if (R.skip) atomicOr(R.skip + (r >> 5), 1u << (r & 31));          // its entry of the sorted list is stale now
@@ -1799,23 +1822,126 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO
     __syncthreads();
 }
 
+// sh[0..p2) / sr[0..p2) hold the group hash and the slot of cnt members (padded with KLPM_FAST_NOGROUP / -1 up to the
+// power of two p2): sort them by hash and write them to the member array from `gs` on, every member with the run of
+// equal hashes it is in as its group.  Every thread of the CTA calls it.
+__device__ void sort_and_group(const FastArgs& A, const FastTour& R, unsigned long long* sh, int32_t* sr, int32_t cnt, int32_t p2, int32_t gs) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    for (int32_t k = 2; k <= p2; k <<= 1)
+        for (int32_t j = k >> 1; j > 0; j >>= 1) {
+            for (int32_t i = tid; i < p2; i += nthr) {
+                const int32_t l = i ^ j;
+                if (l > i) {
+                    const unsigned long long a = sh[i], b = sh[l];
+                    if ((a > b) == ((i & k) == 0)) { sh[i] = b; sh[l] = a; const int32_t t = sr[i]; sr[i] = sr[l]; sr[l] = t; }
+                }
+            }
+            __syncthreads();
+        }
+    for (int32_t i = tid; i < cnt; i += nthr) {
+        const unsigned long long h = sh[i];
+        if (h == KLPM_FAST_NOGROUP) continue;
+        int32_t lo = 0, hi = i;
+        while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sh[mid] < h) lo = mid + 1; else hi = mid; }
+        const int32_t first = lo;
+        lo = i + 1; hi = cnt;
+        while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sh[mid] <= h) lo = mid + 1; else hi = mid; }
+        const int32_t r = sr[i];
+        __stcg(A.mem + gs + i, r);
+        st_dyn_group(A.dyn + r, gs + first, lo - first);
+        set_grouped(R, r, lo - first > 1);
+    }
+}
+
+// t1 of every leaf block that holds a slot of [a0, a1): the largest key among its arrived (< a1), unprocessed slots.
+__device__ void admit_blocks(const FastArgs& A, const FastTour& R, int32_t a0, int32_t a1) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    if (a1 <= a0) return;
+    const int32_t b0 = a0 >> A.lb_shift, b1 = (a1 - 1) >> A.lb_shift;
+    const int32_t LB = 1 << A.lb_shift;
+    for (int32_t b = b0 + warp; b <= b1; b += nwarps) {
+        unsigned long long v = 0;
+        for (int32_t u = lane; u < LB; u += 32) {
+            const long long r = ((long long)b << A.lb_shift) + u;
+            if (r < a1 && !slot_done(R, A, r)) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
+        }
+        v = warp_max64r(v);
+        if (lane == 0) R.t1[b] = v;
+    }
+}
+
 // Work the whole CTA shares; every thread calls it with the same job.  Ends with t2 recomputed from t1.
-__device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J, unsigned long long* sh, int32_t* sr, int* s_cnt) {
+__device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J, unsigned long long* sh, int32_t* sr, int* s_cnt,
+                         int32_t* s_memcur) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int tid = threadIdx.x, nthr = blockDim.x;
     if (J.type == FAST_JOB_ADMIT) {
         // slots [a0, a1) have arrived: the largest key of every leaf block they fall into
-        const int32_t b0 = J.a0 >> A.lb_shift, b1 = (J.a1 - 1) >> A.lb_shift;
-        const int32_t LB = 1 << A.lb_shift;
-        for (int32_t b = b0 + warp; b <= b1; b += nwarps) {
-            unsigned long long v = 0;
-            for (int32_t u = lane; u < LB; u += 32) {
-                const long long r = ((long long)b << A.lb_shift) + u;
-                if (r < J.a1 && !slot_done(R, A, r)) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
+        admit_blocks(A, R, J.a0, J.a1);
+    } else if (J.type == FAST_JOB_FALLBACK) {
+        // Trees with a budget: a leaf in which queries were parked has been evicted.  Every unprocessed slot whose hint
+        // is a dead node walks up to the node its match ends in now; the slots that lose matched tokens that way (the
+        // match ended inside an evicted leaf) end at the end of a live node's edge, get their new state and key, and
+        // are grouped afresh in a run appended to the member array: everybody who falls back to one position with one
+        // next token is in this batch (a query parked there before would have matched into the leaf that was there).
+        if (tid == 0) *s_cnt = 0;
+        __syncthreads();
+        for (int32_t r = tid; r < A.n; r += nthr) {
+            if (slot_done(R, A, r)) continue;
+            const int32_t* dp = reinterpret_cast<const int32_t*>(A.dyn + r);
+            const int32_t h = __ldcg(dp + 6);
+            if (!__ldcg(A.T.dead + h)) continue;
+            const int32_t m0 = __ldcg(dp + 2);
+            int32_t m = m0, a = h;
+            while (a != 0) {
+                const bool dead = __ldcg(A.T.dead + a) != 0;
+                const int32_t ds = __ldcg(A.T.depth_start + a);
+                if (dead) { if (ds < m) m = ds; }
+                else if (m > ds) break;
+                a = __ldcg(A.T.parent + a);
             }
-            v = warp_max64r(v);
-            if (lane == 0) R.t1[b] = v;
+            st_dyn_hint(A.dyn + r, a);
+            atomicAdd(A.parked + a, 1);                      // (what the dead node was counted for no longer matters)
+            if (m != m0) {
+                const FStat s = ld_stat(A.stat + r);
+                const long long pos = a == 0 ? -1 : __ldcg(A.T.span_off + a) + (long long)(m - __ldcg(A.T.depth_start + a)) - 1;
+                const int32_t ntok = __ldg(A.tok + s.soff + m);                     // m < m0 <= length
+                st_dyn_state(A.dyn + r, pos, m, ntok);
+                __stcg(A.key + r, fast_key(m, s.len, s.rank, A.score_mode));
+                const int32_t k = atomicAdd(s_cnt, 1);
+                __stcg(A.gh + k, (long long)group_hash(pos, ntok));
+                __stcg(A.gidx + k, r);
+            }
         }
+        __syncthreads();
+        const int32_t F = *s_cnt, base = *s_memcur;
+        __syncthreads();
+        if (F > 0) {
+            if ((long long)base + F > (long long)A.mem_cap) {
+                if (tid == 0) set_status(A.st, RT_ERR_CAPACITY, 113);      // no room for the new groups: the results are void
+            } else {
+                if (tid == 0) *s_memcur = base + F;
+                if (F <= KLPM_FAST_SORT_CAP) {
+                    int32_t p2 = 1;
+                    while (p2 < F) p2 <<= 1;
+                    for (int32_t i = tid; i < p2; i += nthr) {
+                        sh[i] = i < F ? (unsigned long long)__ldcg(A.gh + i) : KLPM_FAST_NOGROUP;
+                        sr[i] = i < F ? __ldcg(A.gidx + i) : -1;
+                    }
+                    __syncthreads();
+                    sort_and_group(A, R, sh, sr, F, p2, base);
+                } else {                                     // too many to sort here: one run that holds every new group
+                    for (int32_t i = tid; i < F; i += nthr) {
+                        const int32_t r = __ldcg(A.gidx + i);
+                        __stcg(A.mem + base + i, r);
+                        st_dyn_group(A.dyn + r, base, F);
+                        set_grouped(R, r, true);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        admit_blocks(A, R, 0, J.a1);                         // keys went down: every leaf block of the arrived slots afresh
     } else if (J.type == FAST_JOB_REBUILD) {
         // entering list mode (32-slot leaf blocks): the tournament keeps only the unprocessed slots whose key has changed
         for (int32_t b = warp; b < A.nb; b += nwarps) {
@@ -1864,6 +1990,7 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
                     const long long pos2 = P.vleaf + e - 1;
                     const int32_t ntok2 = m2 < s.len ? __ldg(qq + m2) : 0;
                     st_dyn_state(A.dyn + r, pos2, m2, ntok2);
+                    if (A.lru) lru_move(A, r, __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 6), P.leaf);
                     const unsigned long long key = fast_key(m2, s.len, s.rank, A.score_mode);
                     __stcg(A.key + r, key);
                     if (R.skip) atomicOr(R.skip + (r >> 5), 1u << (r & 31));
@@ -1884,30 +2011,7 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
         __syncthreads();
         if (exact) {
             // regroup exactly: sort the members by the hash of their new group inside the run
-            for (int32_t k = 2; k <= p2; k <<= 1)
-                for (int32_t j = k >> 1; j > 0; j >>= 1) {
-                    for (int32_t i = tid; i < p2; i += nthr) {
-                        const int32_t l = i ^ j;
-                        if (l > i) {
-                            const unsigned long long a = sh[i], b = sh[l];
-                            if ((a > b) == ((i & k) == 0)) { sh[i] = b; sh[l] = a; const int32_t t = sr[i]; sr[i] = sr[l]; sr[l] = t; }
-                        }
-                    }
-                    __syncthreads();
-                }
-            for (int32_t i = tid; i < gc; i += nthr) {
-                const unsigned long long h = sh[i];
-                if (h == KLPM_FAST_NOGROUP) continue;
-                int32_t lo = 0, hi = i;
-                while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sh[mid] < h) lo = mid + 1; else hi = mid; }
-                const int32_t first = lo;
-                lo = i + 1; hi = gc;
-                while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sh[mid] <= h) lo = mid + 1; else hi = mid; }
-                const int32_t r = sr[i];
-                __stcg(A.mem + gs + i, r);
-                st_dyn_group(A.dyn + r, gs + first, lo - first);
-                set_grouped(R, r, lo - first > 1);
-            }
+            sort_and_group(A, R, sh, sr, gc, p2, gs);
         } else {
             // too large to sort here: the live members stay together as one run (a superset of every group in it)
             for (int32_t i = tid; i < gc; i += nthr)
@@ -1947,6 +2051,9 @@ fast_run_kernel(FastArgs A) {
     __shared__ int32_t s_H[32], s_E[32];      // a batch's oldest-first and longest-match picks, by rank
     __shared__ FastBatchIO s_bio;             // a CTA-wide batch: what the sequencer hands over and gets back
     __shared__ int32_t s_scan[KLPM_FAST_THREADS / 32];
+    __shared__ TreeState s_st;                // trees with a budget: the tree's counters while the loop runs
+    __shared__ int32_t s_memcur;              // trees with a budget: first free entry of the member array
+    if (A.lru && *reinterpret_cast<const volatile int32_t*>(A.skip)) return;       // the capacity check said no: nothing is touched
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t n = A.n;
     const int32_t nb1p = (A.nb + 31) & ~31, n2 = nb1p >> 5, n2p = (n2 + 31) & ~31, n3 = n2p >> 5;
@@ -1963,6 +2070,7 @@ fast_run_kernel(FastArgs A) {
     R.skip = A.list_mode ? s_done + nwords : nullptr;
     R.gb = A.list_mode ? s_done + 2 * nwords : nullptr;
     for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
+    if (threadIdx.x == 0) { s_memcur = n; if (A.lru) s_st = *A.st; }
     if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
     if (A.list_mode) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
     __syncthreads();
@@ -1973,7 +2081,7 @@ fast_run_kernel(FastArgs A) {
             const FastJob J = s_job;
             if (J.type == FAST_JOB_EXIT) return;
             if (J.type == FAST_JOB_BATCH) { fast_batch_job(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords); continue; }
-            fast_job(A, R, J, sh, sr, &s_cnt);
+            fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
         }
     }
 
@@ -2042,10 +2150,96 @@ fast_run_kernel(FastArgs A) {
         // the new leaf's positions: unique per decision, above every real pool index
         const long long vleaf = A.vbase + ((long long)c << 32);
         ++c;
+        int32_t leaf = -1;
+        if (A.lru) {
+            // ---- the tree's node arrays follow the decision (what insert_serial does, minus the child table and the
+            //      tokens, which the pass after the loop writes for the nodes that are still alive then)
+            const TreeDev& T = A.T;
+            if (lane == 0) atomicSub(A.parked + d.hint, 1);
+            if (s_st.clock + 1 >= T.max_clock || s_st.n_nodes + 2 > T.max_nodes) {        // (the check before the loop rules this out)
+                if (lane == 0) set_status(A.st, RT_ERR_CAPACITY, 114);
+                failed = true; return;
+            }
+            const long long clock = s_st.clock + 1;
+            int32_t a = d.hint, ds = T.depth_start[a];
+            while (a != 0 && m <= ds) { a = T.parent[a]; ds = T.depth_start[a]; }
+            const int32_t o = a == 0 ? 0 : m - ds, sl = T.span_len[a];
+            int32_t end = a;
+            long long n_nodes = s_st.n_nodes, live_nodes = s_st.live_nodes, tokens_live = s_st.tokens_live, evictions = s_st.evictions;
+            if (a != 0 && o < sl) {                         // node boundary inside a's edge: a new node takes the upper part
+                const int32_t u = (int32_t)n_nodes++;
+                ++live_nodes;
+                if (lane == 0) {
+                    const int64_t so = T.span_off[a];
+                    T.parent[u] = T.parent[a]; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = o;
+                    T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = T.last_access[a];
+                    T.span_off[a] = so + o; T.span_len[a] = sl - o; T.depth_start[a] = ds + o; T.parent[a] = u;
+                }
+                end = u;
+            }
+            if (end != 0 && lane == 0) { T.last_access[end] = clock; T.clock_owner[clock] = end; }
+            __syncwarp();
+            // least recently used leaves go until the prompt's uncached tokens fit (the node just stamped is safe)
+            bool scan = false;
+            long long cur = s_st.lru_cursor;
+            while (tokens_live + unc > T.budget) {
+                int32_t victim = -1;
+                while (cur < clock) {                       // 32 clock values at a time
+                    const long long cc = cur + lane;
+                    const int32_t v = cc < clock ? T.clock_owner[cc] : 0;
+                    const bool ok = v > 0 && !T.dead[v] && T.last_access[v] == cc && T.nchild[v] == 0;
+                    const unsigned bal = __ballot_sync(FULL_MASK, ok);
+                    if (bal) { const int src = __ffs(bal) - 1; victim = __shfl_sync(FULL_MASK, v, src); cur += src; break; }
+                    cur += 32;
+                }
+                if (victim < 0) {
+                    if (lane == 0) set_status(A.st, RT_ERR_BUDGET);
+                    failed = true; break;
+                }
+                const int32_t P = T.parent[victim];
+                tokens_live -= T.span_len[victim];
+                --live_nodes; ++evictions;
+                if (__ldcg(A.parked + victim) > 0) scan = true;
+                if (lane == 0) {
+                    T.dead[victim] = 1;
+                    T.nchild[P]--;
+                    const long long stamp = T.last_access[victim];
+                    if (P != 0 && stamp >= T.last_access[P]) { T.last_access[P] = stamp; T.clock_owner[stamp] = P; }
+                }
+                __syncwarp();
+            }
+            if (cur > clock) cur = clock;
+            if (!failed && unc > 0) {
+                leaf = (int32_t)n_nodes++;
+                ++live_nodes;
+                tokens_live += unc;
+                if (lane == 0) {
+                    T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = vleaf; T.span_len[leaf] = unc;
+                    T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = clock; T.clock_owner[clock] = leaf;
+                    T.nchild[end]++;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                s_st.clock = clock; s_st.n_nodes = n_nodes; s_st.live_nodes = live_nodes; s_st.tokens_live = tokens_live;
+                s_st.evictions = evictions; s_st.lru_cursor = cur;
+            }
+            __syncwarp();
+            if (scan) {                                     // somebody was parked in an evicted leaf
+                if (lane == 0) { s_job.type = FAST_JOB_FALLBACK; s_job.a0 = 0; s_job.a1 = admitted; }
+                __threadfence_block();
+                __syncwarp();
+                named_bar(1, KLPM_FAST_THREADS);
+                const FastJob J = s_job;
+                fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
+                root = tour_top(R, lane);
+            }
+            if (failed) return;
+        }
         if (unc > 0 && d.gcount > 1) {
             FastPick P;
             P.slot = slot; P.m = m; P.len = len; P.ntok = d.ntok; P.x = A.tok + s.soff; P.pos = d.pos; P.vleaf = vleaf;
-            P.admitted = admitted; P.gstart = d.gstart; P.gcount = d.gcount;
+            P.admitted = admitted; P.gstart = d.gstart; P.gcount = d.gcount; P.leaf = leaf;
             // small groups are handled by this warp alone, unless several long compares are better spread over the CTA
             if (d.gcount <= 32 && !(d.gcount > 2 && unc > 512)) {
                 const int32_t r = lane < d.gcount ? __ldcg(A.mem + d.gstart + lane) : -1;
@@ -2074,7 +2268,7 @@ fast_run_kernel(FastArgs A) {
                 __syncwarp();
                 named_bar(1, KLPM_FAST_THREADS);
                 const FastJob J = s_job;
-                fast_job(A, R, J, sh, sr, &s_cnt);
+                fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
                 root = tour_top(R, lane);
             }
         }
@@ -2118,7 +2312,7 @@ fast_run_kernel(FastArgs A) {
                 __syncwarp();
                 named_bar(1, KLPM_FAST_THREADS);
                 const FastJob J = s_job;
-                fast_job(A, R, J, sh, sr, &s_cnt);
+                fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
                 root = tour_top(R, lane);
             }
             admitted = a1;
@@ -2154,7 +2348,7 @@ fast_run_kernel(FastArgs A) {
         named_bar(1, KLPM_FAST_THREADS);
         {
             const FastJob J = s_job;
-            fast_job(A, R, J, sh, sr, &s_cnt);
+            fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
         }
         root = tour_top(R, lane);
         // the sorted list, 32 entries at a time: lane l holds entry (cur & ~31) + l, the next 32 are on their way
@@ -2376,6 +2570,12 @@ fast_run_kernel(FastArgs A) {
         A.post->now0 = now;
     }
     __syncwarp();
+    if (A.lru && lane == 0) {                               // the tree's counters go back (a status recorded meanwhile stays)
+        TreeState out = s_st;
+        out.status = *reinterpret_cast<const volatile int*>(&A.st->status);
+        out.detail = *reinterpret_cast<const volatile int*>(&A.st->detail);
+        *A.st = out;
+    }
     if (lane == 0) s_job.type = FAST_JOB_EXIT;
     __syncwarp();
     named_bar(1, KLPM_FAST_THREADS);
@@ -2884,6 +3084,102 @@ last_only_batch_kernel(LastOnlyArgs A) {
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Trees with a budget: before and after the grouped loop.
+// Before: the loop is all or nothing, so room for everything it can leave behind is checked first -- two nodes and one
+// clock tick per prompt, and pool tokens for at most a budget's worth of new tokens plus three of alignment per node.
+// After: the loop has kept the node arrays (parent, depth, length, children, stamps, dead flags) exact but has given
+// the edges of new nodes virtual positions and has touched neither the token pool nor the child table.  Every node
+// that is still alive gets its pool tokens (copied from the prompt that created its edge) and the child table is
+// written afresh from the live nodes; nodes that were evicted again along the way cost nothing.
+// ------------------------------------------------------------------------------------------------
+struct LruInfo { long long n_nodes0; unsigned long long total_len; int32_t skip; int32_t pad; };
+
+__global__ void lru_sum_kernel(const int64_t* __restrict__ off, int32_t n, LruInfo* info) {
+    __shared__ unsigned long long s_w[8];
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long x = i < n ? (unsigned long long)(off[i + 1] - off[i]) : 0ULL;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_down_sync(FULL_MASK, x, d);
+    if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long t = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += s_w[w];
+        atomicAdd(&info->total_len, t);
+    }
+}
+__global__ void lru_check_kernel(TreeDev T, int32_t n, LruInfo* info) {
+    TreeState* S = T.st;
+    long long fresh = S->tokens_live + (long long)info->total_len;
+    if (fresh > T.budget) fresh = T.budget;
+    const bool ok = S->n_nodes + 2LL * n <= T.max_nodes && S->clock + (long long)n + 1 < T.max_clock &&
+                    S->pool_used + fresh + 6LL * n + 16 <= T.max_pool;
+    info->n_nodes0 = S->n_nodes;
+    info->skip = ok ? 0 : 1;
+    if (!ok) set_status(S, RT_ERR_CAPACITY, 115);
+}
+
+// One warp per node created by the loop: if it is alive and its edge has a virtual position, give it room in the pool
+// and copy its tokens from the prompt that created the edge (decision c = the position's high bits; the edge holds
+// that prompt's tokens from the node's depth on).
+__global__ void __launch_bounds__(256)
+lru_tokens_kernel(TreeDev T, const int32_t* __restrict__ order, const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff,
+                  long long vbase, const LruInfo* info) {
+    if (info->skip) return;
+    const int lane = threadIdx.x & 31;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const long long n_end = T.st->n_nodes;
+    for (long long v = info->n_nodes0 + (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5); v < n_end; v += nwarps) {
+        if (T.dead[v]) continue;
+        const long long so = T.span_off[v];
+        if (so < vbase) continue;                           // a piece of an edge that was in the tree before: its tokens are in the pool
+        const int32_t c = (int32_t)((so - vbase) >> 32), len = T.span_len[v], depth = T.depth_start[v];
+        const int32_t* x = qtok + __ldg(qoff + __ldg(order + c)) + depth;
+        long long base = 0;
+        if (lane == 0) {
+            const long long raw = (long long)atomicAdd((unsigned long long*)&T.st->pool_used, (unsigned long long)(len + 3));
+            base = raw + (((long long)depth - raw) & 3LL);  // span_off = depth_start (mod 4), as everywhere
+            if (raw + len + 3 > T.max_pool) { set_status(T.st, RT_ERR_CAPACITY, 116); base = -1; }      // (ruled out by the check before the loop)
+        }
+        base = __shfl_sync(FULL_MASK, base, 0);
+        if (base < 0) continue;
+        for (int32_t t = lane; t < len; t += 32) T.pool[base + t] = __ldg(x + t);
+        if (lane == 0) T.span_off[v] = base;
+    }
+}
+
+__global__ void table_clear_kernel(TreeDev T, const LruInfo* info) {
+    if (info->skip) return;
+    int4* p = reinterpret_cast<int4*>(T.table);
+    const unsigned long long n16 = (T.table_mask + 1) * 2;              // an entry is two 16-byte units
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (unsigned long long)gridDim.x * blockDim.x)
+        p[i] = make_int4(0, 0, 0, 0);
+}
+
+// One thread per node: every live node's first token, the mark at the end of its edge, and its entry in the (cleared)
+// child table.
+__global__ void lru_table_kernel(TreeDev T, long long vbase, const LruInfo* info) {
+    if (info->skip) return;
+    const long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (v < 1 || v >= T.st->n_nodes || T.dead[v]) return;
+    const long long so = T.span_off[v];
+    if (so >= vbase) return;                                // no room was found for it: the status word says so
+    const int32_t len = T.span_len[v], ft = T.pool[so];
+    T.first_tok[v] = ft;
+    T.end_node[so + len - 1] = (int32_t)v;
+    const unsigned long long key = make_key(T.parent[v], ft);
+    unsigned long long slot = hash_key(key) & T.table_mask;
+    for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+        if (atomicCAS(&T.table[slot].key, 0ULL, key) == 0ULL) {
+            T.table[slot].child = (int32_t)v; T.table[slot].span_len = len; T.table[slot].span_off = so; T.table[slot].chain_end = so + len;
+            return;
+        }
+        slot = (slot + 1) & T.table_mask;
+    }
+    set_status(T.st, RT_ERR_CAPACITY, 117);
+}
+
 // batch size B: a query is finished when the last query of its bin of the processing order is
 __global__ void batch_times_kernel(const int32_t* __restrict__ order, int32_t n, const int64_t* __restrict__ arrival,
                                    const int64_t* __restrict__ completion, int32_t n_queries, int32_t B, int64_t* ttft_b,
@@ -3013,6 +3309,8 @@ struct rt_tree {
     long long* fast_gh; int32_t* fast_gidx; unsigned int* fast_done; unsigned long long* fast_counter;
     long long* fast_lk; int32_t* fast_ls;
     FastPost* fast_post; long long* fast_bsum;
+    long long fast_mem_cap;  // entries of fast_mem
+    int32_t* lru_parked; LruInfo* lru_info;     // grouped loop on a tree with a budget
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -3054,6 +3352,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
     cudaFree(t->fast_lk); cudaFree(t->fast_ls); cudaFree(t->fast_post); cudaFree(t->fast_bsum);
+    cudaFree(t->lru_parked); cudaFree(t->lru_info);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
     cudaFree(t->bulk_sync);
@@ -3105,7 +3404,9 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_dyn, np2))) return s;
     if ((s = dalloc(&t->fast_stat, np2))) return s;
     if ((s = dalloc(&t->fast_key_arr, np2))) return s;
-    if ((s = dalloc(&t->fast_mem, np2))) return s;
+    // trees with a budget: groups formed by evictions are appended behind the first n entries
+    t->fast_mem_cap = t->cfg.budget_tokens > 0 ? np2 + (8 * np2 > (1LL << 20) ? 8 * np2 : (1LL << 20)) : np2;
+    if ((s = dalloc(&t->fast_mem, t->fast_mem_cap))) return s;
     if ((s = dalloc(&t->fast_gh, np2))) return s;
     if ((s = dalloc(&t->fast_gidx, np2))) return s;
     if ((s = dalloc(&t->fast_done, 2 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap
@@ -3598,7 +3899,8 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     long long np2 = 1;
     while (np2 < n) np2 <<= 1;
     // A tree without a budget takes the grouped loop (unless the debug setting run_one_by_one is on).
-    const bool grouped = tree->cfg.budget_tokens == 0 && !g_knobs.run_one_by_one;
+    const bool grouped = !g_knobs.run_one_by_one;
+    const bool lru = tree->cfg.budget_tokens > 0;
     // slots = queries ordered by (arrival, index)
     {
         unsigned blocks = (unsigned)((np2 + 255) / 256);
@@ -3620,6 +3922,17 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         if (st) return st;
         st = ensure_bulk_scratch(tree, n);
         if (st) return st;
+        if (lru) {
+            if (!tree->lru_parked && (st = dalloc(&tree->lru_parked, tree->dev.max_nodes))) return st;
+            if (!tree->lru_info && (st = dalloc(&tree->lru_info, 1))) return st;
+            f.lru = 1; f.T = tree->dev; f.parked = tree->lru_parked; f.skip = &tree->lru_info->skip;
+            f.mem_cap = (int32_t)(tree->fast_mem_cap < 0x7fffffffLL ? tree->fast_mem_cap : 0x7fffffffLL);
+            // all or nothing: is there room for whatever the loop can leave behind?
+            CK(cudaMemsetAsync(tree->lru_info, 0, sizeof(LruInfo), s));
+            CK(cudaMemsetAsync(tree->lru_parked, 0, (size_t)tree->dev.max_nodes * sizeof(int32_t), s));
+            lru_sum_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(d_q_offsets, n, tree->lru_info);
+            lru_check_kernel<<<1, 1, 0, s>>>(tree->dev, n, tree->lru_info);
+        }
         f.tok = d_q_tokens; f.n = n; f.policy = params->policy; f.k = params->k; f.score_mode = score_mode;
         f.c_num = params->c_num; f.c_den = params->c_den; f.start_tick = params->start_tick;
         f.order = d_order; f.uncached = d_uncached; f.ttft = d_ttft; f.completion = d_completion;
@@ -3666,7 +3979,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
         // list mode needs two more bitmaps in shared memory and 32-slot leaf blocks
-        f.list_mode = (f.done_in_smem && lbs == 5 && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
+        f.list_mode = (!lru && f.done_in_smem && lbs == 5 && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
         if (f.list_mode) smem += (size_t)nwords * 8;
         f.gbits = tree->fast_done + (np2 / 32 + 32);
         const unsigned nblk = (unsigned)((n + 255) / 256), pblk = (unsigned)((np2 + 255) / 256);
@@ -3690,6 +4003,15 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         }
         CK(cudaGetLastError());
         tree->run_path = 2;
+        if (lru) {
+            // the nodes that are alive after the loop get their tokens, and the child table is written afresh
+            const TreeDev& d = tree->dev;
+            lru_tokens_kernel<<<(unsigned)tree->num_sms * 8, 256, 0, s>>>(d, d_order, d_q_tokens, d_q_offsets, f.vbase, tree->lru_info);
+            table_clear_kernel<<<(unsigned)tree->num_sms * 8, 256, 0, s>>>(d, tree->lru_info);
+            lru_table_kernel<<<(unsigned)((d.max_nodes + 255) / 256), 256, 0, s>>>(d, f.vbase, tree->lru_info);
+            CK(cudaGetLastError());
+            return RT_OK;
+        }
         // The processed prompts enter the tree together (the logical clock advances by n).  The loop itself needs
         // no room in the tree; if the tree cannot hold the queue the insertion says so through the status word.
         return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s, state, tag);

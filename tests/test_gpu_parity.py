@@ -670,9 +670,9 @@ def test_run_ex_multi_cta_random_ties(K, score_mode):
 # ------------------------------------------------------------------ bounded waits and guarded scores
 
 def test_a_wait_that_runs_out_is_reported_and_every_cta_returns(K):
-    """The one-by-one loop's CTAs wait for one another with a limit.  With the limit set to zero the sequencer gives
-    up on its first hand-over: the call returns, the status word says RT_ERR_LIMIT (detail 102), and after a
-    rollback the tree answers matches as before.  Nothing traps or hangs: a wait that gives up returns."""
+    """The CTAs of the one-decision-at-a-time loop wait for one another with a limit.  With the limit set to zero the
+    sequencer gives up on its first hand-over: the call returns, the status word says RT_ERR_LIMIT (detail 102), and
+    after a rollback the tree answers matches as before.  Nothing traps or hangs: a wait that gives up returns."""
     prompts, arr = W.random_small_queue(77, 6000, vocab=3, max_len=24, min_len=1, max_gap=0)      # everybody waiting
     prefill, _ = W.random_small_queue(78, 50, vocab=3, max_len=20, min_len=1)
     qt, qo = csr(prompts)
@@ -683,10 +683,12 @@ def test_a_wait_that_runs_out_is_reported_and_every_cta_returns(K):
     out = [torch.full((n,), -1, dtype=torch.int32, device="cuda"), torch.full((n,), -1, dtype=torch.int32, device="cuda"),
            torch.full((n,), -1, dtype=torch.int64, device="cuda")]
     K.klpm_debug_set("wait_limit_ns", 0)
+    K.klpm_debug_set("run_one_by_one", 1)
     try:
         K.klpm_run(tree, dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_KLPM, 3), *out)
         assert K.rt_sync_status(tree) == K.RT_ERR_LIMIT
         assert K.rt_status_detail(tree) == 102
+        assert K.klpm_run_path(tree) == K.RUN_PATH_ONE_BY_ONE
     finally:
         K.klpm_debug_set("wait_limit_ns", -1)
     K.rt_rollback(tree)
@@ -694,11 +696,38 @@ def test_a_wait_that_runs_out_is_reported_and_every_cta_returns(K):
     ot = oracle_tree(pt, po, 200000)
     assert_match_equals_oracle(K, tree, ot, qt, qo)
     # and with the default limit the same call completes and equals the oracle
-    K.klpm_run(tree, dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_KLPM, 3), *out)
+    try:
+        K.klpm_run(tree, dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_KLPM, 3), *out)
+    finally:
+        K.klpm_debug_set("run_one_by_one", -1)
     assert K.rt_sync_status(tree) == 0
     want = oracle.schedule(qt.numpy(), qo.numpy(), np.asarray(arr), oracle.POLICY_KLPM, 3, 0, 1, 0, oracle.CACHE_TREE,
                            oracle.TIER_UPDATE, ot)
     assert np.array_equal(out[0].cpu().numpy(), want[0]) and np.array_equal(out[2].cpu().numpy(), want[2])
+    K.rt_destroy(tree)
+
+
+def test_a_grid_barrier_that_runs_out_is_reported_too(K):
+    """The concurrent insertion's later rounds run in one cooperative kernel whose CTAs meet at barriers with the same
+    limit.  Prompts that share prefixes need several rounds; with the limit at zero the first barrier gives up, the
+    status word says RT_ERR_LIMIT (detail 112), every CTA returns, and the same insertion goes through afterwards."""
+    prompts, _ = W.random_small_queue(79, 3000, vocab=2, max_len=30, min_len=1)
+    pt, po = csr(prompts)
+    tree = K.rt_create(**caps(pt.numel(), n_prompts=len(prompts)))
+    K.rt_checkpoint(tree)
+    K.klpm_debug_set("wait_limit_ns", 0)
+    try:
+        K.rt_insert(tree, dev(pt), dev(po))
+        assert K.rt_sync_status(tree) == K.RT_ERR_LIMIT and K.rt_status_detail(tree) == 112
+    finally:
+        K.klpm_debug_set("wait_limit_ns", -1)
+    K.rt_rollback(tree)
+    K.rt_insert(tree, dev(pt), dev(po))
+    assert K.rt_sync_status(tree) == 0
+    ot = oracle_tree(pt, po)
+    st, ost = K.rt_stats(tree), ot.stats()
+    assert (st["n_nodes"], st["tokens"], st["clock"]) == (ost["n_nodes"], ost["tokens"], ost["clock"])
+    assert_match_equals_oracle(K, tree, ot, pt, po)
     K.rt_destroy(tree)
 
 
