@@ -85,6 +85,8 @@ _lib.klpm_batch_times.restype = _i32
 _lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp]
 _lib.klpm_run_last_only_batch.restype = _i32
 _lib.klpm_run_last_only_batch.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.rt_debug_counters.restype = _i32
+_lib.rt_debug_counters.argtypes = [_vp, ctypes.POINTER(_i64 * 8)]
 _lib.klpm_debug_set.restype = _i32
 _lib.klpm_debug_set.argtypes = [ctypes.c_char_p, _i64]
 _lib.klpm_run_path.restype = _i32
@@ -95,7 +97,7 @@ _lib.klpm_run.argtypes = [_vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params),
 MATCH_STATE_BYTES = 32
 
 EXPORTS = ["klpm_abi_version", "rt_create", "rt_build", "rt_insert", "rt_match_batch", "rt_match_batch_ex", "rt_stats",
-           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times", "klpm_debug_set", "klpm_run_last_only_batch"]
+           "rt_sync_status", "rt_status_detail", "rt_clone", "rt_checkpoint", "rt_rollback", "rt_destroy", "klpm_select", "klpm_select_topk", "klpm_select_noalloc", "klpm_replay", "klpm_run", "klpm_run_ex", "klpm_run_path", "klpm_batch_times", "klpm_debug_set", "klpm_run_last_only_batch", "rt_debug_counters"]
 
 
 def lib() -> ctypes.CDLL:
@@ -327,6 +329,15 @@ def klpm_run_last_only_batch(tokens: torch.Tensor, offsets: torch.Tensor, arriva
                                          _dev(completion, torch.int64, "completion", True),
                                          _dev(n_skipped, torch.int32, "n_skipped", True), _stream()),
            "klpm_run_last_only_batch")
+
+
+def rt_debug_counters(tree: Tree) -> dict:
+    """What the grouped loop of the last klpm_run on this tree did (see include/klpm.h)."""
+    v = (_i64 * 8)()
+    _check(_lib.rt_debug_counters(tree.handle, ctypes.byref(v)), "rt_debug_counters")
+    names = ("careful_steps", "cta_dissolves", "fallback_scans", "fallen_back", "evictions", "cycles_tree", "cycles_scans",
+             "cycles_cta_dissolves")
+    return dict(zip(names, [int(x) for x in v]))
 
 
 def klpm_debug_set(name: str, value: int) -> None:

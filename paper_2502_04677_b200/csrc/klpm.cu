@@ -1405,7 +1405,12 @@ struct alignas(32) FStat {    // constant during the loop; the first 16 bytes ar
     int32_t pad;
 };
 
-struct FastPost { int32_t c0; int32_t pad; long long now0; };   // first decision made in list mode; the time it was made at
+struct FastPost {
+    int32_t c0; int32_t pad; long long now0;    // first decision made in list mode; the time it was made at
+    // what the loop did (rt_debug_counters): careful steps, dissolves by the whole CTA, fallback scans, slots that fell
+    // back, evictions; cycles spent in tree updates, fallback scans, dissolves
+    long long counters[8];
+};
 
 struct FastArgs {
     const int32_t* tok;
@@ -1435,6 +1440,7 @@ struct FastArgs {
     int32_t mem_cap;              // entries of the member array (groups formed by evictions are appended behind the first n)
     TreeDev T;
     int32_t* parked;              // per node: unprocessed slots whose hint is that node
+    int32_t* hintc;               // per slot: the hint once more, side by side (what the scan after an eviction reads)
     int32_t* skip;                // set by the capacity check before the loop: leave everything untouched
 };
 
@@ -1531,7 +1537,7 @@ __global__ void fast_state_kernel(FastArgs A, const MatchState* __restrict__ sta
         m = 0; pos = -1; ntok = 0; hint = 0;
     }
     st_dyn_state(A.dyn + r, pos, m, ntok);
-    if (A.lru) { st_dyn_hint(A.dyn + r, hint); atomicAdd(A.parked + hint, 1); }
+    if (A.lru) { st_dyn_hint(A.dyn + r, hint); A.hintc[r] = hint; atomicAdd(A.parked + hint, 1); }
     A.key[r] = fast_key(m, s.len, s.rank, A.score_mode);
     A.gh[r] = (long long)(m < s.len ? group_hash(pos, ntok) : single_hash((int32_t)r));
     A.gidx[r] = (int32_t)r;
@@ -1581,6 +1587,7 @@ struct FastTour {
     unsigned int* done;       // bitmap of processed slots (shared memory), or null
     unsigned int* skip;       // bitmap of slots the sorted list must pass over: processed, or key changed (shared memory), or null
     unsigned int* gb;         // bitmap of slots whose group has more than one member (shared memory), or null
+    unsigned int* dirty;      // trees with a budget: bitmap of leaf blocks to recompute after a fallback (256 words, shared memory)
     int32_t n2;               // entries of t2 in use
     int32_t n3;               // entries of t3 in use
 };
@@ -1659,6 +1666,7 @@ enum { FAST_JOB_EXIT = 0, FAST_JOB_ADMIT = 1, FAST_JOB_DISSOLVE = 2, FAST_JOB_RE
 // trees with a budget: slot r's match now ends inside node `to` (it was counted for node `from`)
 __device__ __forceinline__ void lru_move(const FastArgs& A, int32_t r, int32_t from, int32_t to) {
     st_dyn_hint(A.dyn + r, to);
+    __stcg(A.hintc + r, to);
     atomicSub(A.parked + from, 1);
     atomicAdd(A.parked + to, 1);
 }
@@ -1853,6 +1861,88 @@ __device__ void sort_and_group(const FastArgs& A, const FastTour& R, unsigned lo
     }
 }
 
+// The same for more members than the shared-memory scratch holds: A.gh[0..cnt) / A.gidx[0..cnt) hold hash and slot.  A
+// bitonic sort of the arrays in global memory -- partner distances of a tile (4,096) and more one pass over global
+// memory each, everything below inside shared memory tile by tile -- then the runs of equal hashes become the groups.
+__device__ void sort_large_and_group(const FastArgs& A, const FastTour& R, unsigned long long* sh, int32_t* sr, int32_t cnt, int32_t gs) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    constexpr int32_t TILE = KLPM_FAST_SORT_CAP;
+    int32_t p2 = TILE;
+    while (p2 < cnt) p2 <<= 1;
+    for (int32_t i = cnt + tid; i < p2; i += nthr) { __stcg(A.gh + i, (long long)KLPM_FAST_NOGROUP); __stcg(A.gidx + i, -1); }
+    __syncthreads();
+    // stages k_lo .. k_hi (or the tail of one stage) on every tile, in shared memory
+    auto tiles = [&](int32_t k_lo, int32_t k_hi) {
+        for (int32_t base = 0; base < p2; base += TILE) {
+            for (int32_t i = tid; i < TILE; i += nthr) { sh[i] = (unsigned long long)__ldcg(A.gh + base + i); sr[i] = __ldcg(A.gidx + base + i); }
+            __syncthreads();
+            for (int32_t k = k_lo; k <= k_hi; k <<= 1) {
+                const int32_t jmax = (k >> 1) < (TILE >> 1) ? (k >> 1) : (TILE >> 1);
+                for (int32_t j = jmax; j > 0; j >>= 1) {
+                    for (int32_t i = tid; i < TILE; i += nthr) {
+                        const int32_t l = i ^ j;
+                        if (l > i) {
+                            const unsigned long long a = sh[i], b = sh[l];
+                            if ((a > b) == (((base + i) & k) == 0)) { sh[i] = b; sh[l] = a; const int32_t t = sr[i]; sr[i] = sr[l]; sr[l] = t; }
+                        }
+                    }
+                    __syncthreads();
+                }
+            }
+            for (int32_t i = tid; i < TILE; i += nthr) { __stcg(A.gh + base + i, (long long)sh[i]); __stcg(A.gidx + base + i, sr[i]); }
+            __syncthreads();
+        }
+    };
+    tiles(2, TILE);
+    for (int32_t k = TILE << 1; k <= p2; k <<= 1) {
+        for (int32_t j = k >> 1; j >= TILE; j >>= 1) {
+            for (int32_t i = tid; i < p2; i += nthr) {
+                const int32_t l = i ^ j;
+                if (l > i) {
+                    const unsigned long long a = (unsigned long long)__ldcg(A.gh + i), b = (unsigned long long)__ldcg(A.gh + l);
+                    if ((a > b) == ((i & k) == 0)) {
+                        const int32_t ri = __ldcg(A.gidx + i), rl = __ldcg(A.gidx + l);
+                        __stcg(A.gh + i, (long long)b); __stcg(A.gh + l, (long long)a); __stcg(A.gidx + i, rl); __stcg(A.gidx + l, ri);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        tiles(k, k);
+    }
+    // runs of equal hashes; nearly every member is alone, which its two neighbours show
+    for (int32_t i = tid; i < cnt; i += nthr) {
+        const unsigned long long h = (unsigned long long)__ldcg(A.gh + i);
+        if (h == KLPM_FAST_NOGROUP) continue;
+        int32_t first = i, last = i + 1;
+        if (i > 0 && (unsigned long long)__ldcg(A.gh + i - 1) == h) {
+            int32_t lo = 0, hi = i;
+            while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if ((unsigned long long)__ldcg(A.gh + mid) < h) lo = mid + 1; else hi = mid; }
+            first = lo;
+        }
+        if (i + 1 < cnt && (unsigned long long)__ldcg(A.gh + i + 1) == h) {
+            int32_t lo = i + 1, hi = cnt;
+            while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if ((unsigned long long)__ldcg(A.gh + mid) <= h) lo = mid + 1; else hi = mid; }
+            last = lo;
+        }
+        const int32_t r = __ldcg(A.gidx + i);
+        __stcg(A.mem + gs + i, r);
+        st_dyn_group(A.dyn + r, gs + first, last - first);
+        set_grouped(R, r, last - first > 1);
+    }
+}
+
+// t1 of leaf block b: the largest key among its arrived (< a1), unprocessed slots.  One warp.
+__device__ __forceinline__ void admit_blocks_one(const FastArgs& A, const FastTour& R, int32_t b, int32_t lo_slot, int32_t a1, int lane) {
+    unsigned long long v = 0;
+    for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
+        const long long r = (long long)lo_slot + u;
+        if (r < a1 && !slot_done(R, A, r)) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
+    }
+    v = warp_max64r(v);
+    if (lane == 0) R.t1[b] = v;
+}
+
 // t1 of every leaf block that holds a slot of [a0, a1): the largest key among its arrived (< a1), unprocessed slots.
 __device__ void admit_blocks(const FastArgs& A, const FastTour& R, int32_t a0, int32_t a1) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -1885,32 +1975,44 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
         // are grouped afresh in a run appended to the member array: everybody who falls back to one position with one
         // next token is in this batch (a query parked there before would have matched into the leaf that was there).
         if (tid == 0) *s_cnt = 0;
+        for (int32_t i = tid; i < 256; i += nthr) R.dirty[i] = 0u;
         __syncthreads();
-        for (int32_t r = tid; r < A.n; r += nthr) {
-            if (slot_done(R, A, r)) continue;
-            const int32_t* dp = reinterpret_cast<const int32_t*>(A.dyn + r);
-            const int32_t h = __ldcg(dp + 6);
-            if (!__ldcg(A.T.dead + h)) continue;
-            const int32_t m0 = __ldcg(dp + 2);
-            int32_t m = m0, a = h;
-            while (a != 0) {
-                const bool dead = __ldcg(A.T.dead + a) != 0;
-                const int32_t ds = __ldcg(A.T.depth_start + a);
-                if (dead) { if (ds < m) m = ds; }
-                else if (m > ds) break;
-                a = __ldcg(A.T.parent + a);
-            }
-            st_dyn_hint(A.dyn + r, a);
-            atomicAdd(A.parked + a, 1);                      // (what the dead node was counted for no longer matters)
-            if (m != m0) {
-                const FStat s = ld_stat(A.stat + r);
-                const long long pos = a == 0 ? -1 : __ldcg(A.T.span_off + a) + (long long)(m - __ldcg(A.T.depth_start + a)) - 1;
-                const int32_t ntok = __ldg(A.tok + s.soff + m);                     // m < m0 <= length
-                st_dyn_state(A.dyn + r, pos, m, ntok);
-                __stcg(A.key + r, fast_key(m, s.len, s.rank, A.score_mode));
-                const int32_t k = atomicAdd(s_cnt, 1);
-                __stcg(A.gh + k, (long long)group_hash(pos, ntok));
-                __stcg(A.gidx + k, r);
+        // slots below a0 (the oldest unprocessed slot) are all processed; four hints, then four dead flags, in flight per thread
+        for (int32_t r0 = J.a0 + tid; r0 < A.n; r0 += 4 * nthr) {
+            int32_t hh[4];
+            bool dd[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { const int32_t r = r0 + u * nthr; hh[u] = r < A.n ? __ldcg(A.hintc + r) : 0; }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) dd[u] = hh[u] != 0 && __ldcg(A.T.dead + hh[u]) != 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int32_t r = r0 + u * nthr, h = hh[u];
+                if (!dd[u] || slot_done(R, A, r)) continue;
+                const int32_t* dp = reinterpret_cast<const int32_t*>(A.dyn + r);
+                const int32_t m0 = __ldcg(dp + 2);
+                int32_t m = m0, a = h;
+                while (a != 0) {
+                    const bool dead = __ldcg(A.T.dead + a) != 0;
+                    const int32_t ds = __ldcg(A.T.depth_start + a);
+                    if (dead) { if (ds < m) m = ds; }
+                    else if (m > ds) break;
+                    a = __ldcg(A.T.parent + a);
+                }
+                st_dyn_hint(A.dyn + r, a);
+                __stcg(A.hintc + r, a);
+                atomicAdd(A.parked + a, 1);                  // (what the dead node was counted for no longer matters)
+                if (m != m0) {
+                    const FStat s = ld_stat(A.stat + r);
+                    const long long pos = a == 0 ? -1 : __ldcg(A.T.span_off + a) + (long long)(m - __ldcg(A.T.depth_start + a)) - 1;
+                    const int32_t ntok = __ldg(A.tok + s.soff + m);                 // m < m0 <= length
+                    st_dyn_state(A.dyn + r, pos, m, ntok);
+                    __stcg(A.key + r, fast_key(m, s.len, s.rank, A.score_mode));
+                    if (r < J.a1) { const int32_t b = r >> A.lb_shift; atomicOr(R.dirty + (b >> 5), 1u << (b & 31)); }
+                    const int32_t k = atomicAdd(s_cnt, 1);
+                    __stcg(A.gh + k, (long long)group_hash(pos, ntok));
+                    __stcg(A.gidx + k, r);
+                }
             }
         }
         __syncthreads();
@@ -1930,18 +2032,22 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
                     }
                     __syncthreads();
                     sort_and_group(A, R, sh, sr, F, p2, base);
-                } else {                                     // too many to sort here: one run that holds every new group
-                    for (int32_t i = tid; i < F; i += nthr) {
-                        const int32_t r = __ldcg(A.gidx + i);
-                        __stcg(A.mem + base + i, r);
-                        st_dyn_group(A.dyn + r, base, F);
-                        set_grouped(R, r, true);
-                    }
+                } else {
+                    sort_large_and_group(A, R, sh, sr, F, base);
                 }
             }
         }
         __syncthreads();
-        admit_blocks(A, R, 0, J.a1);                         // keys went down: every leaf block of the arrived slots afresh
+        // keys went down: the leaf blocks that hold an arrived slot which fell back are recomputed
+        for (int32_t w = warp; w < 256; w += nwarps) {
+            unsigned bits = R.dirty[w];
+            while (bits) {
+                const int32_t b = w * 32 + __ffs(bits) - 1;
+                bits &= bits - 1;
+                const int32_t lo_slot = b << A.lb_shift;
+                admit_blocks_one(A, R, b, lo_slot, J.a1, lane);
+            }
+        }
     } else if (J.type == FAST_JOB_REBUILD) {
         // entering list mode (32-slot leaf blocks): the tournament keeps only the unprocessed slots whose key has changed
         for (int32_t b = warp; b < A.nb; b += nwarps) {
@@ -2013,20 +2119,8 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
             // regroup exactly: sort the members by the hash of their new group inside the run
             sort_and_group(A, R, sh, sr, gc, p2, gs);
         } else {
-            // too large to sort here: the live members stay together as one run (a superset of every group in it)
-            for (int32_t i = tid; i < gc; i += nthr)
-                if ((unsigned long long)__ldcg(A.gh + i) != KLPM_FAST_NOGROUP) {
-                    const int32_t p = atomicAdd(s_cnt, 1);
-                    __stcg(A.mem + gs + p, __ldcg(A.gidx + i));
-                }
-            __syncthreads();
-            const int32_t cnt = *s_cnt;
-            for (int32_t i = tid; i < gc; i += nthr)
-                if ((unsigned long long)__ldcg(A.gh + i) != KLPM_FAST_NOGROUP) {
-                    const int32_t r = __ldcg(A.gidx + i);
-                    st_dyn_group(A.dyn + r, gs, cnt);
-                    set_grouped(R, r, cnt > 1);
-                }
+            // too many for the shared-memory sort: the same regrouping with the arrays in global memory
+            sort_large_and_group(A, R, sh, sr, gc, gs);
         }
     }
     __syncthreads();
@@ -2053,6 +2147,7 @@ fast_run_kernel(FastArgs A) {
     __shared__ int32_t s_scan[KLPM_FAST_THREADS / 32];
     __shared__ TreeState s_st;                // trees with a budget: the tree's counters while the loop runs
     __shared__ int32_t s_memcur;              // trees with a budget: first free entry of the member array
+    __shared__ unsigned int s_dirty[256];
     if (A.lru && *reinterpret_cast<const volatile int32_t*>(A.skip)) return;       // the capacity check said no: nothing is touched
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t n = A.n;
@@ -2069,6 +2164,7 @@ fast_run_kernel(FastArgs A) {
     R.done = A.done_in_smem ? s_done : nullptr;
     R.skip = A.list_mode ? s_done + nwords : nullptr;
     R.gb = A.list_mode ? s_done + 2 * nwords : nullptr;
+    R.dirty = s_dirty;
     for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
     if (threadIdx.x == 0) { s_memcur = n; if (A.lru) s_st = *A.st; }
     if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
@@ -2091,6 +2187,7 @@ fast_run_kernel(FastArgs A) {
     int32_t head = 0, admitted = 0;
     long long next_t = __ldg(&A.stat[0].t);
     unsigned long long root = 0;
+    long long n_careful = 0, n_cta_dissolve = 0, n_scan = 0, n_evict = 0, cy_tree = 0, cy_scan = 0, cy_dissolve = 0;
     int32_t cyc = 0;                                        // c mod k
     int32_t c = 0;
     bool failed = false;
@@ -2151,7 +2248,9 @@ fast_run_kernel(FastArgs A) {
         const long long vleaf = A.vbase + ((long long)c << 32);
         ++c;
         int32_t leaf = -1;
+        ++n_careful;
         if (A.lru) {
+            const long long t_tree = clock64();
             // ---- the tree's node arrays follow the decision (what insert_serial does, minus the child table and the
             //      tokens, which the pass after the loop writes for the nodes that are still alive then)
             const TreeDev& T = A.T;
@@ -2198,7 +2297,7 @@ fast_run_kernel(FastArgs A) {
                 }
                 const int32_t P = T.parent[victim];
                 tokens_live -= T.span_len[victim];
-                --live_nodes; ++evictions;
+                --live_nodes; ++evictions; ++n_evict;
                 if (__ldcg(A.parked + victim) > 0) scan = true;
                 if (lane == 0) {
                     T.dead[victim] = 1;
@@ -2225,14 +2324,18 @@ fast_run_kernel(FastArgs A) {
                 s_st.evictions = evictions; s_st.lru_cursor = cur;
             }
             __syncwarp();
+            cy_tree += clock64() - t_tree;
             if (scan) {                                     // somebody was parked in an evicted leaf
-                if (lane == 0) { s_job.type = FAST_JOB_FALLBACK; s_job.a0 = 0; s_job.a1 = admitted; }
+                const long long t_scan = clock64();
+                ++n_scan;
+                if (lane == 0) { s_job.type = FAST_JOB_FALLBACK; s_job.a0 = head < slot ? head : slot; s_job.a1 = admitted; }
                 __threadfence_block();
                 __syncwarp();
                 named_bar(1, KLPM_FAST_THREADS);
                 const FastJob J = s_job;
                 fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
                 root = tour_top(R, lane);
+                cy_scan += clock64() - t_scan;
             }
             if (failed) return;
         }
@@ -2264,12 +2367,15 @@ fast_run_kernel(FastArgs A) {
                     root = tour_update(R, bb, lane);
                 }
             } else {
+                const long long t_dis = clock64();
+                ++n_cta_dissolve;
                 if (lane == 0) { s_job.type = FAST_JOB_DISSOLVE; s_job.pick = P; }
                 __syncwarp();
                 named_bar(1, KLPM_FAST_THREADS);
                 const FastJob J = s_job;
                 fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
                 root = tour_top(R, lane);
+                cy_dissolve += clock64() - t_dis;
             }
         }
     };
@@ -2570,6 +2676,11 @@ fast_run_kernel(FastArgs A) {
         A.post->now0 = now;
     }
     __syncwarp();
+    if (lane == 0) {
+        long long* cn = A.post->counters;
+        cn[0] = n_careful; cn[1] = n_cta_dissolve; cn[2] = n_scan; cn[3] = s_memcur - n; cn[4] = n_evict;
+        cn[5] = cy_tree; cn[6] = cy_scan; cn[7] = cy_dissolve;
+    }
     if (A.lru && lane == 0) {                               // the tree's counters go back (a status recorded meanwhile stays)
         TreeState out = s_st;
         out.status = *reinterpret_cast<const volatile int*>(&A.st->status);
@@ -3311,6 +3422,7 @@ struct rt_tree {
     FastPost* fast_post; long long* fast_bsum;
     long long fast_mem_cap;  // entries of fast_mem
     int32_t* lru_parked; LruInfo* lru_info;     // grouped loop on a tree with a budget
+    int32_t* lru_hintc; long long lru_hintc_cap;
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -3352,7 +3464,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
     cudaFree(t->fast_lk); cudaFree(t->fast_ls); cudaFree(t->fast_post); cudaFree(t->fast_bsum);
-    cudaFree(t->lru_parked); cudaFree(t->lru_info);
+    cudaFree(t->lru_parked); cudaFree(t->lru_info); cudaFree(t->lru_hintc);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
     cudaFree(t->bulk_sync);
@@ -3925,6 +4037,13 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         if (lru) {
             if (!tree->lru_parked && (st = dalloc(&tree->lru_parked, tree->dev.max_nodes))) return st;
             if (!tree->lru_info && (st = dalloc(&tree->lru_info, 1))) return st;
+            if (n > tree->lru_hintc_cap) {
+                cudaFree(tree->lru_hintc);
+                tree->lru_hintc = nullptr; tree->lru_hintc_cap = 0;
+                if ((st = dalloc(&tree->lru_hintc, n))) return st;
+                tree->lru_hintc_cap = n;
+            }
+            f.hintc = tree->lru_hintc;
             f.lru = 1; f.T = tree->dev; f.parked = tree->lru_parked; f.skip = &tree->lru_info->skip;
             f.mem_cap = (int32_t)(tree->fast_mem_cap < 0x7fffffffLL ? tree->fast_mem_cap : 0x7fffffffLL);
             // all or nothing: is there room for whatever the loop can leave behind?
@@ -4068,6 +4187,17 @@ rt_status klpm_run_last_only_batch(const int32_t* d_tokens, const int64_t* d_off
 }
 
 int32_t klpm_run_path(const rt_tree* tree) { return tree ? tree->run_path : 0; }
+
+rt_status rt_debug_counters(rt_tree* tree, int64_t* out8) {
+    if (!tree || !out8) return RT_ERR_INVALID;
+    memset(out8, 0, 8 * sizeof(int64_t));
+    if (!tree->fast_post) return RT_OK;
+    CK(cudaStreamSynchronize(tree->last_stream));
+    FastPost h;
+    CK(cudaMemcpy(&h, tree->fast_post, sizeof(h), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 8; ++i) out8[i] = h.counters[i];
+    return RT_OK;
+}
 
 rt_status klpm_debug_set(const char* name, int64_t value) {
     if (!name) return RT_ERR_INVALID;
