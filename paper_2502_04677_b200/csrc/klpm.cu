@@ -1441,6 +1441,7 @@ struct FastArgs {
     TreeDev T;
     int32_t* parked;              // per node: unprocessed slots whose hint is that node
     int32_t* hintc;               // per slot: the hint once more, side by side (what the scan after an eviction reads)
+    int2* leaf_run;               // per node: the member run that holds every slot whose hint is that node (y < 0: no such run is known)
     int32_t* skip;                // set by the capacity check before the loop: leave everything untouched
 };
 
@@ -2002,6 +2003,7 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
                 st_dyn_hint(A.dyn + r, a);
                 __stcg(A.hintc + r, a);
                 atomicAdd(A.parked + a, 1);                  // (what the dead node was counted for no longer matters)
+                A.leaf_run[a].y = -1;                        // slots from elsewhere are parked in a now: no one run holds them all
                 if (m != m0) {
                     const FStat s = ld_stat(A.stat + r);
                     const long long pos = a == 0 ? -1 : __ldcg(A.T.span_off + a) + (long long)(m - __ldcg(A.T.depth_start + a)) - 1;
@@ -2280,6 +2282,8 @@ fast_run_kernel(FastArgs A) {
             __syncwarp();
             // least recently used leaves go until the prompt's uncached tokens fit (the node just stamped is safe)
             bool scan = false;
+            int32_t small_v[1];                             // the evicted leaf whose parked queries this warp looks after itself
+            int n_small = 0;
             long long cur = s_st.lru_cursor;
             while (tokens_live + unc > T.budget) {
                 int32_t victim = -1;
@@ -2298,7 +2302,15 @@ fast_run_kernel(FastArgs A) {
                 const int32_t P = T.parent[victim];
                 tokens_live -= T.span_len[victim];
                 --live_nodes; ++evictions; ++n_evict;
-                if (__ldcg(A.parked + victim) > 0) scan = true;
+                if (__ldcg(A.parked + victim) > 0) {
+                    // Queries are parked in the evicted leaf.  If the leaf was made by a processed prompt, only members of
+                    // that prompt's group can be inside it, and it is the only such leaf of this decision (two evicted
+                    // leaves, one above the other, send their queries to one and the same new group), the warp handles
+                    // them itself below (at most 32 of them fall back); otherwise the whole CTA scans the unprocessed slots.
+                    const int2 lr = __ldcg(A.leaf_run + victim);
+                    if (lr.y > 0 && lr.y <= 1024 && n_small == 0) { small_v[0] = victim; n_small = 1; }
+                    else scan = true;
+                }
                 if (lane == 0) {
                     T.dead[victim] = 1;
                     T.nchild[P]--;
@@ -2316,6 +2328,7 @@ fast_run_kernel(FastArgs A) {
                     T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = vleaf; T.span_len[leaf] = unc;
                     T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = clock; T.clock_owner[clock] = leaf;
                     T.nchild[end]++;
+                    A.leaf_run[leaf] = make_int2(d.gstart, d.gcount);     // whoever gets parked in it is a member of the pick's group
                 }
             }
             __syncwarp();
@@ -2324,6 +2337,100 @@ fast_run_kernel(FastArgs A) {
                 s_st.evictions = evictions; s_st.lru_cursor = cur;
             }
             __syncwarp();
+            // ---- evicted leaves whose parked queries sit in one known member run: the warp moves them itself
+            for (int sv = 0; sv < n_small && !scan; ++sv) {
+                const int32_t v = small_v[sv];
+                const int2 lr = __ldcg(A.leaf_run + v);
+                const int32_t ds_v = T.depth_start[v];
+                // first pass: how many of the run's members fall back (more than 32: leave it to the scan)
+                int32_t n_fall = 0;
+                for (int32_t base = 0; base < lr.y; base += 32) {
+                    const int32_t r = base + lane < lr.y ? __ldcg(A.mem + lr.x + base + lane) : -1;
+                    bool hit = r >= 0 && !slot_done(R, A, r) && __ldcg(A.hintc + r) == v;
+                    if (hit) hit = __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 2) > ds_v;
+                    const unsigned same = __match_any_sync(FULL_MASK, hit ? r : -1 - lane);       // a slot can be listed twice in a run
+                    if (hit && (int)(__ffs(same) - 1) != lane) hit = false;
+                    n_fall += __popc(__ballot_sync(FULL_MASK, hit));
+                }
+                if (n_fall > 32) { scan = true; break; }
+                // second pass: every member whose hint is the dead leaf walks up; those that lose tokens are collected
+                int32_t f_slot = -1;                        // lane k holds the k-th slot that fell back
+                unsigned long long f_hash = KLPM_FAST_NOGROUP;
+                int32_t n_f = 0;
+                for (int32_t base = 0; base < lr.y; base += 32) {
+                    const int32_t r = base + lane < lr.y ? __ldcg(A.mem + lr.x + base + lane) : -1;
+                    bool hit = r >= 0 && !slot_done(R, A, r) && __ldcg(A.hintc + r) == v;
+                    const unsigned same = __match_any_sync(FULL_MASK, hit ? r : -1 - lane);
+                    if (hit && (int)(__ffs(same) - 1) != lane) hit = false;
+                    bool fell = false;
+                    unsigned long long h = KLPM_FAST_NOGROUP;
+                    if (hit) {
+                        const int32_t m0 = __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 2);
+                        int32_t mm = m0, a = v;
+                        while (a != 0) {
+                            const bool dead = T.dead[a] != 0;
+                            const int32_t dsa = T.depth_start[a];
+                            if (dead) { if (dsa < mm) mm = dsa; }
+                            else if (mm > dsa) break;
+                            a = T.parent[a];
+                        }
+                        st_dyn_hint(A.dyn + r, a);
+                        __stcg(A.hintc + r, a);
+                        atomicAdd(A.parked + a, 1);
+                        A.leaf_run[a].y = -1;
+                        if (mm != m0) {
+                            const FStat fs = ld_stat(A.stat + r);
+                            const long long pos = a == 0 ? -1 : T.span_off[a] + (long long)(mm - T.depth_start[a]) - 1;
+                            const int32_t ntok = __ldg(A.tok + fs.soff + mm);
+                            st_dyn_state(A.dyn + r, pos, mm, ntok);
+                            __stcg(A.key + r, fast_key(mm, fs.len, fs.rank, A.score_mode));
+                            h = group_hash(pos, ntok);
+                            fell = true;
+                        }
+                    }
+                    const unsigned fb = __ballot_sync(FULL_MASK, fell);
+                    const int32_t my = n_f + __popc(fb & ((1u << lane) - 1u));
+                    for (unsigned bits = fb; bits; bits &= bits - 1) {      // hand each fallen slot to the lane that keeps it
+                        const int src = __ffs(bits) - 1;
+                        const int32_t dst = __shfl_sync(FULL_MASK, my, src);
+                        const int32_t rr = __shfl_sync(FULL_MASK, r, src);
+                        const unsigned long long hh = __shfl_sync(FULL_MASK, h, src);
+                        if (lane == dst) { f_slot = rr; f_hash = hh; }
+                    }
+                    n_f += __popc(fb);
+                }
+                if (n_f > 0) {
+                    // the fallen slots are grouped afresh in a run appended to the member array (ranked by shuffles)
+                    const int32_t base = s_memcur;
+                    if ((long long)base + n_f > (long long)A.mem_cap) {
+                        if (lane == 0) set_status(A.st, RT_ERR_CAPACITY, 113);
+                        failed = true; break;
+                    }
+                    int32_t rank = 0, start = 0, cnt = 0;
+                    for (int k2i = 0; k2i < 32; ++k2i) {
+                        const unsigned long long hk = __shfl_sync(FULL_MASK, f_hash, k2i);
+                        const bool lt = hk < f_hash, eq = hk == f_hash;
+                        start += lt; cnt += eq; rank += (lt || (eq && k2i < lane));
+                    }
+                    if (f_slot >= 0) {
+                        __stcg(A.mem + base + rank, f_slot);
+                        st_dyn_group(A.dyn + f_slot, base + start, cnt);
+                        set_grouped(R, f_slot, cnt > 1);
+                    }
+                    if (lane == 0) s_memcur = base + n_f;
+                    __syncwarp();
+                    // their keys went down: the leaf blocks of the arrived ones are recomputed
+                    for (int k2i = 0; k2i < n_f; ++k2i) {
+                        const int32_t rr = __shfl_sync(FULL_MASK, f_slot, k2i);
+                        if (rr < admitted) {
+                            const int32_t bb = rr >> A.lb_shift;
+                            admit_blocks_one(A, R, bb, bb << A.lb_shift, admitted, lane);
+                            __syncwarp();
+                            root = tour_update(R, bb, lane);
+                        }
+                    }
+                }
+            }
             cy_tree += clock64() - t_tree;
             if (scan) {                                     // somebody was parked in an evicted leaf
                 const long long t_scan = clock64();
@@ -3423,6 +3530,7 @@ struct rt_tree {
     long long fast_mem_cap;  // entries of fast_mem
     int32_t* lru_parked; LruInfo* lru_info;     // grouped loop on a tree with a budget
     int32_t* lru_hintc; long long lru_hintc_cap;
+    int2* lru_leaf_run;
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -3464,7 +3572,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
     cudaFree(t->fast_lk); cudaFree(t->fast_ls); cudaFree(t->fast_post); cudaFree(t->fast_bsum);
-    cudaFree(t->lru_parked); cudaFree(t->lru_info); cudaFree(t->lru_hintc);
+    cudaFree(t->lru_parked); cudaFree(t->lru_info); cudaFree(t->lru_hintc); cudaFree(t->lru_leaf_run);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
     cudaFree(t->bulk_sync);
@@ -4044,6 +4152,9 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
                 tree->lru_hintc_cap = n;
             }
             f.hintc = tree->lru_hintc;
+            if (!tree->lru_leaf_run && (st = dalloc(&tree->lru_leaf_run, tree->dev.max_nodes))) return st;
+            f.leaf_run = tree->lru_leaf_run;
+            CK(cudaMemsetAsync(tree->lru_leaf_run, 0xff, (size_t)tree->dev.max_nodes * sizeof(int2), s));
             f.lru = 1; f.T = tree->dev; f.parked = tree->lru_parked; f.skip = &tree->lru_info->skip;
             f.mem_cap = (int32_t)(tree->fast_mem_cap < 0x7fffffffLL ? tree->fast_mem_cap : 0x7fffffffLL);
             // all or nothing: is there room for whatever the loop can leave behind?
