@@ -1442,6 +1442,7 @@ struct FastArgs {
     int32_t* parked;              // per node: unprocessed slots whose hint is that node
     int32_t* hintc;               // per slot: the hint once more, side by side (what the scan after an eviction reads)
     int2* leaf_run;               // per node: the member run that holds every slot whose hint is that node (y < 0: no such run is known)
+    long long* pk; int32_t* pi;   // set-up: (hint, slot) pairs, sorted by hint to give every node of the tree its run
     int32_t* skip;                // set by the capacity check before the loop: leave everything untouched
 };
 
@@ -1521,7 +1522,11 @@ __global__ void hit_rate_guard_kernel(const int64_t* __restrict__ off, int32_t n
 __global__ void fast_state_kernel(FastArgs A, const MatchState* __restrict__ state, unsigned long long tag, long long np2) {
     const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= np2) return;
-    if (r >= A.n) { A.gh[r] = 0x7fffffffffffffffLL; A.gidx[r] = 0x7fffffff; return; }      // padding of the sort
+    if (r >= A.n) {                                                                        // padding of the sorts
+        A.gh[r] = 0x7fffffffffffffffLL; A.gidx[r] = 0x7fffffff;
+        if (A.lru) { A.pk[r] = 0x7fffffffffffffffLL; A.pi[r] = 0x7fffffff; }
+        return;
+    }
     const FStat s = ld_stat(A.stat + r);
     const int4* src = reinterpret_cast<const int4*>(state + s.ord);
     const int4 a = __ldcg(src), b = __ldcg(src + 1);
@@ -1538,10 +1543,26 @@ __global__ void fast_state_kernel(FastArgs A, const MatchState* __restrict__ sta
         m = 0; pos = -1; ntok = 0; hint = 0;
     }
     st_dyn_state(A.dyn + r, pos, m, ntok);
-    if (A.lru) { st_dyn_hint(A.dyn + r, hint); A.hintc[r] = hint; atomicAdd(A.parked + hint, 1); }
+    if (A.lru) {
+        st_dyn_hint(A.dyn + r, hint); A.hintc[r] = hint; atomicAdd(A.parked + hint, 1);
+        A.pk[r] = hint; A.pi[r] = (int32_t)r;
+    }
     A.key[r] = fast_key(m, s.len, s.rank, A.score_mode);
     A.gh[r] = (long long)(m < s.len ? group_hash(pos, ntok) : single_hash((int32_t)r));
     A.gidx[r] = (int32_t)r;
+}
+
+// Trees with a budget, after the sort by hint: the slots whose match ends in one node, side by side, are that node's
+// run (entries n .. 2n-1 of the member array): where the loop looks when the node is evicted with queries parked in it.
+__global__ void lru_parklist_kernel(FastArgs A) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= A.n) return;
+    A.mem[A.n + i] = A.pi[i];
+    const long long node = A.pk[i];
+    if (i > 0 && A.pk[i - 1] == node) return;              // not the first of its run
+    int32_t lo = i + 1, hi = A.n;                          // first index with a larger hint
+    while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (A.pk[mid] <= node) lo = mid + 1; else hi = mid; }
+    A.leaf_run[node] = make_int2(A.n + i, lo - i);
 }
 
 // after the sort by hash: runs of equal hashes are the groups
@@ -2168,7 +2189,7 @@ fast_run_kernel(FastArgs A) {
     R.gb = A.list_mode ? s_done + 2 * nwords : nullptr;
     R.dirty = s_dirty;
     for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
-    if (threadIdx.x == 0) { s_memcur = n; if (A.lru) s_st = *A.st; }
+    if (threadIdx.x == 0) { s_memcur = A.lru ? 2 * n : n; if (A.lru) s_st = *A.st; }
     if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
     if (A.list_mode) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
     __syncthreads();
@@ -2282,7 +2303,7 @@ fast_run_kernel(FastArgs A) {
             __syncwarp();
             // least recently used leaves go until the prompt's uncached tokens fit (the node just stamped is safe)
             bool scan = false;
-            int32_t small_v[1];                             // the evicted leaf whose parked queries this warp looks after itself
+            int32_t small_v[8];                             // evicted leaves whose parked queries this warp looks after itself
             int n_small = 0;
             long long cur = s_st.lru_cursor;
             while (tokens_live + unc > T.budget) {
@@ -2303,12 +2324,11 @@ fast_run_kernel(FastArgs A) {
                 tokens_live -= T.span_len[victim];
                 --live_nodes; ++evictions; ++n_evict;
                 if (__ldcg(A.parked + victim) > 0) {
-                    // Queries are parked in the evicted leaf.  If the leaf was made by a processed prompt, only members of
-                    // that prompt's group can be inside it, and it is the only such leaf of this decision (two evicted
-                    // leaves, one above the other, send their queries to one and the same new group), the warp handles
-                    // them itself below (at most 32 of them fall back); otherwise the whole CTA scans the unprocessed slots.
+                    // Queries are parked in the evicted leaf.  If one run of the member array is known to hold every slot
+                    // whose hint is this leaf, the warp looks after them itself below (up to 8 such leaves and 32 slots
+                    // that fall back per decision); otherwise the whole CTA scans the unprocessed slots.
                     const int2 lr = __ldcg(A.leaf_run + victim);
-                    if (lr.y > 0 && lr.y <= 1024 && n_small == 0) { small_v[0] = victim; n_small = 1; }
+                    if (lr.y > 0 && lr.y <= 1024 && n_small < 8) { small_v[n_small] = victim; ++n_small; }
                     else scan = true;
                 }
                 if (lane == 0) {
@@ -2337,96 +2357,107 @@ fast_run_kernel(FastArgs A) {
                 s_st.evictions = evictions; s_st.lru_cursor = cur;
             }
             __syncwarp();
-            // ---- evicted leaves whose parked queries sit in one known member run: the warp moves them itself
-            for (int sv = 0; sv < n_small && !scan; ++sv) {
-                const int32_t v = small_v[sv];
-                const int2 lr = __ldcg(A.leaf_run + v);
-                const int32_t ds_v = T.depth_start[v];
-                // first pass: how many of the run's members fall back (more than 32: leave it to the scan)
+            // ---- evicted leaves whose parked queries sit in known member runs: the warp moves them itself.  All leaves of
+            //      this decision are taken together: two of them, one above the other, send their queries to one group.
+            if (n_small > 0 && !scan && !failed) {
+                // first pass: how many slots fall back (more than 32: leave it to the scan)
                 int32_t n_fall = 0;
-                for (int32_t base = 0; base < lr.y; base += 32) {
-                    const int32_t r = base + lane < lr.y ? __ldcg(A.mem + lr.x + base + lane) : -1;
-                    bool hit = r >= 0 && !slot_done(R, A, r) && __ldcg(A.hintc + r) == v;
-                    if (hit) hit = __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 2) > ds_v;
-                    const unsigned same = __match_any_sync(FULL_MASK, hit ? r : -1 - lane);       // a slot can be listed twice in a run
-                    if (hit && (int)(__ffs(same) - 1) != lane) hit = false;
-                    n_fall += __popc(__ballot_sync(FULL_MASK, hit));
+                for (int sv = 0; sv < n_small; ++sv) {
+                    const int32_t v = small_v[sv];
+                    const int2 lr = __ldcg(A.leaf_run + v);
+                    const int32_t ds_v = T.depth_start[v];
+                    for (int32_t base = 0; base < lr.y; base += 32) {
+                        const int32_t r = base + lane < lr.y ? __ldcg(A.mem + lr.x + base + lane) : -1;
+                        bool hit = r >= 0 && !slot_done(R, A, r) && __ldcg(A.hintc + r) == v;
+                        if (hit) hit = __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 2) > ds_v;
+                        const unsigned same = __match_any_sync(FULL_MASK, hit ? r : -1 - lane);       // a slot can be listed twice in a run
+                        if (hit && (int)(__ffs(same) - 1) != lane) hit = false;
+                        n_fall += __popc(__ballot_sync(FULL_MASK, hit));
+                    }
                 }
-                if (n_fall > 32) { scan = true; break; }
-                // second pass: every member whose hint is the dead leaf walks up; those that lose tokens are collected
+                if (n_fall > 32) scan = true;
+            }
+            if (n_small > 0 && !scan && !failed) {
+                // second pass: every member whose hint is a dead leaf walks up; those that lose tokens are collected
                 int32_t f_slot = -1;                        // lane k holds the k-th slot that fell back
                 unsigned long long f_hash = KLPM_FAST_NOGROUP;
                 int32_t n_f = 0;
-                for (int32_t base = 0; base < lr.y; base += 32) {
-                    const int32_t r = base + lane < lr.y ? __ldcg(A.mem + lr.x + base + lane) : -1;
-                    bool hit = r >= 0 && !slot_done(R, A, r) && __ldcg(A.hintc + r) == v;
-                    const unsigned same = __match_any_sync(FULL_MASK, hit ? r : -1 - lane);
-                    if (hit && (int)(__ffs(same) - 1) != lane) hit = false;
-                    bool fell = false;
-                    unsigned long long h = KLPM_FAST_NOGROUP;
-                    if (hit) {
-                        const int32_t m0 = __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 2);
-                        int32_t mm = m0, a = v;
-                        while (a != 0) {
-                            const bool dead = T.dead[a] != 0;
-                            const int32_t dsa = T.depth_start[a];
-                            if (dead) { if (dsa < mm) mm = dsa; }
-                            else if (mm > dsa) break;
-                            a = T.parent[a];
+                for (int sv = 0; sv < n_small; ++sv) {
+                    const int32_t v = small_v[sv];
+                    const int2 lr = __ldcg(A.leaf_run + v);
+                    for (int32_t base = 0; base < lr.y; base += 32) {
+                        const int32_t r = base + lane < lr.y ? __ldcg(A.mem + lr.x + base + lane) : -1;
+                        bool hit = r >= 0 && !slot_done(R, A, r) && __ldcg(A.hintc + r) == v;
+                        const unsigned same = __match_any_sync(FULL_MASK, hit ? r : -1 - lane);
+                        if (hit && (int)(__ffs(same) - 1) != lane) hit = false;
+                        bool fell = false;
+                        unsigned long long h = KLPM_FAST_NOGROUP;
+                        if (hit) {
+                            const int32_t m0 = __ldcg(reinterpret_cast<const int32_t*>(A.dyn + r) + 2);
+                            int32_t mm = m0, a = v;
+                            while (a != 0) {
+                                const bool dead = T.dead[a] != 0;
+                                const int32_t dsa = T.depth_start[a];
+                                if (dead) { if (dsa < mm) mm = dsa; }
+                                else if (mm > dsa) break;
+                                a = T.parent[a];
+                            }
+                            st_dyn_hint(A.dyn + r, a);
+                            __stcg(A.hintc + r, a);
+                            atomicAdd(A.parked + a, 1);
+                            A.leaf_run[a].y = -1;
+                            if (mm != m0) {
+                                const FStat fs = ld_stat(A.stat + r);
+                                const long long pos = a == 0 ? -1 : T.span_off[a] + (long long)(mm - T.depth_start[a]) - 1;
+                                const int32_t ntok = __ldg(A.tok + fs.soff + mm);
+                                st_dyn_state(A.dyn + r, pos, mm, ntok);
+                                __stcg(A.key + r, fast_key(mm, fs.len, fs.rank, A.score_mode));
+                                h = group_hash(pos, ntok);
+                                fell = true;
+                            }
                         }
-                        st_dyn_hint(A.dyn + r, a);
-                        __stcg(A.hintc + r, a);
-                        atomicAdd(A.parked + a, 1);
-                        A.leaf_run[a].y = -1;
-                        if (mm != m0) {
-                            const FStat fs = ld_stat(A.stat + r);
-                            const long long pos = a == 0 ? -1 : T.span_off[a] + (long long)(mm - T.depth_start[a]) - 1;
-                            const int32_t ntok = __ldg(A.tok + fs.soff + mm);
-                            st_dyn_state(A.dyn + r, pos, mm, ntok);
-                            __stcg(A.key + r, fast_key(mm, fs.len, fs.rank, A.score_mode));
-                            h = group_hash(pos, ntok);
-                            fell = true;
+                        const unsigned fb = __ballot_sync(FULL_MASK, fell);
+                        const int32_t my = n_f + __popc(fb & ((1u << lane) - 1u));
+                        for (unsigned bits = fb; bits; bits &= bits - 1) {      // hand each fallen slot to the lane that keeps it
+                            const int src = __ffs(bits) - 1;
+                            const int32_t dst = __shfl_sync(FULL_MASK, my, src);
+                            const int32_t rr = __shfl_sync(FULL_MASK, r, src);
+                            const unsigned long long hh = __shfl_sync(FULL_MASK, h, src);
+                            if (lane == dst) { f_slot = rr; f_hash = hh; }
                         }
+                        n_f += __popc(fb);
+                        __syncwarp();
                     }
-                    const unsigned fb = __ballot_sync(FULL_MASK, fell);
-                    const int32_t my = n_f + __popc(fb & ((1u << lane) - 1u));
-                    for (unsigned bits = fb; bits; bits &= bits - 1) {      // hand each fallen slot to the lane that keeps it
-                        const int src = __ffs(bits) - 1;
-                        const int32_t dst = __shfl_sync(FULL_MASK, my, src);
-                        const int32_t rr = __shfl_sync(FULL_MASK, r, src);
-                        const unsigned long long hh = __shfl_sync(FULL_MASK, h, src);
-                        if (lane == dst) { f_slot = rr; f_hash = hh; }
-                    }
-                    n_f += __popc(fb);
                 }
                 if (n_f > 0) {
                     // the fallen slots are grouped afresh in a run appended to the member array (ranked by shuffles)
                     const int32_t base = s_memcur;
                     if ((long long)base + n_f > (long long)A.mem_cap) {
                         if (lane == 0) set_status(A.st, RT_ERR_CAPACITY, 113);
-                        failed = true; break;
-                    }
-                    int32_t rank = 0, start = 0, cnt = 0;
-                    for (int k2i = 0; k2i < 32; ++k2i) {
-                        const unsigned long long hk = __shfl_sync(FULL_MASK, f_hash, k2i);
-                        const bool lt = hk < f_hash, eq = hk == f_hash;
-                        start += lt; cnt += eq; rank += (lt || (eq && k2i < lane));
-                    }
-                    if (f_slot >= 0) {
-                        __stcg(A.mem + base + rank, f_slot);
-                        st_dyn_group(A.dyn + f_slot, base + start, cnt);
-                        set_grouped(R, f_slot, cnt > 1);
-                    }
-                    if (lane == 0) s_memcur = base + n_f;
-                    __syncwarp();
-                    // their keys went down: the leaf blocks of the arrived ones are recomputed
-                    for (int k2i = 0; k2i < n_f; ++k2i) {
-                        const int32_t rr = __shfl_sync(FULL_MASK, f_slot, k2i);
-                        if (rr < admitted) {
-                            const int32_t bb = rr >> A.lb_shift;
-                            admit_blocks_one(A, R, bb, bb << A.lb_shift, admitted, lane);
-                            __syncwarp();
-                            root = tour_update(R, bb, lane);
+                        failed = true;
+                    } else {
+                        int32_t rank = 0, start = 0, cnt = 0;
+                        for (int k2i = 0; k2i < 32; ++k2i) {
+                            const unsigned long long hk = __shfl_sync(FULL_MASK, f_hash, k2i);
+                            const bool lt = hk < f_hash, eq = hk == f_hash;
+                            start += lt; cnt += eq; rank += (lt || (eq && k2i < lane));
+                        }
+                        if (f_slot >= 0) {
+                            __stcg(A.mem + base + rank, f_slot);
+                            st_dyn_group(A.dyn + f_slot, base + start, cnt);
+                            set_grouped(R, f_slot, cnt > 1);
+                        }
+                        if (lane == 0) s_memcur = base + n_f;
+                        __syncwarp();
+                        // their keys went down: the leaf blocks of the arrived ones are recomputed
+                        for (int k2i = 0; k2i < n_f; ++k2i) {
+                            const int32_t rr = __shfl_sync(FULL_MASK, f_slot, k2i);
+                            if (rr < admitted) {
+                                const int32_t bb = rr >> A.lb_shift;
+                                admit_blocks_one(A, R, bb, bb << A.lb_shift, admitted, lane);
+                                __syncwarp();
+                                root = tour_update(R, bb, lane);
+                            }
                         }
                     }
                 }
@@ -2785,7 +2816,7 @@ fast_run_kernel(FastArgs A) {
     __syncwarp();
     if (lane == 0) {
         long long* cn = A.post->counters;
-        cn[0] = n_careful; cn[1] = n_cta_dissolve; cn[2] = n_scan; cn[3] = s_memcur - n; cn[4] = n_evict;
+        cn[0] = n_careful; cn[1] = n_cta_dissolve; cn[2] = n_scan; cn[3] = s_memcur - (A.lru ? 2 * n : n); cn[4] = n_evict;
         cn[5] = cy_tree; cn[6] = cy_scan; cn[7] = cy_dissolve;
     }
     if (A.lru && lane == 0) {                               // the tree's counters go back (a status recorded meanwhile stays)
@@ -4154,6 +4185,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
             f.hintc = tree->lru_hintc;
             if (!tree->lru_leaf_run && (st = dalloc(&tree->lru_leaf_run, tree->dev.max_nodes))) return st;
             f.leaf_run = tree->lru_leaf_run;
+            f.pk = tree->fast_lk; f.pi = tree->fast_ls;      // (the key list of list mode is not used on these trees)
             CK(cudaMemsetAsync(tree->lru_leaf_run, 0xff, (size_t)tree->dev.max_nodes * sizeof(int2), s));
             f.lru = 1; f.T = tree->dev; f.parked = tree->lru_parked; f.skip = &tree->lru_info->skip;
             f.mem_cap = (int32_t)(tree->fast_mem_cap < 0x7fffffffLL ? tree->fast_mem_cap : 0x7fffffffLL);
@@ -4217,6 +4249,10 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         // groups: queries whose match ends at the same position and continues with the same token
         sort_pairs(f.gh, f.gidx, np2, s);
         fast_group_kernel<<<nblk, 256, 0, s>>>(f);
+        if (lru) {                   // per node of the tree: the slots parked in it as the loop starts
+            sort_pairs(f.pk, f.pi, np2, s);
+            lru_parklist_kernel<<<nblk, 256, 0, s>>>(f);
+        }
         if (f.list_mode) {           // all keys, largest first
             f.lk = tree->fast_lk; f.ls = tree->fast_ls;
             fast_list_kernel<<<pblk, 256, 0, s>>>(f.key, n, np2, tree->fast_lk, tree->fast_ls);
