@@ -233,11 +233,14 @@ rt_status klpm_run(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_
  * same outputs.  The debug setting "run_one_by_one" makes trees without a budget take loop 1 too. */
 int32_t klpm_run_path(const rt_tree* tree);
 
-/* What the grouped loop of the last klpm_run / klpm_run_ex on this tree did (zeros if it has not run): out8[0] decisions
- * taken one at a time, [1] groups dissolved by the whole CTA, [2] scans after an eviction of a leaf with queries parked
- * in it, [3] queries that fell back out of evicted leaves, [4] evictions, [5..7] clock cycles spent in tree updates, in
- * those scans, in dissolves by the whole CTA.  A debugging aid; synchronises like rt_stats. */
-rt_status rt_debug_counters(rt_tree* tree, int64_t* out8);
+/* What the grouped loop of the last klpm_run / klpm_run_ex on this tree did (zeros if it has not run): out16[0] decisions
+ * taken by a careful step, [1] groups dissolved by the whole CTA, [2] scans after an eviction of a leaf with queries
+ * parked in it, [3] queries that fell back out of evicted leaves, [4] evictions, [5..7] clock cycles spent in tree
+ * updates, in those scans, in dissolves by the whole CTA; once everybody had arrived: [8] CTA-wide batches tried,
+ * [9] committed, [10] decisions they made, [11] warp-wide steps committed, [12] decisions they made, [13] decisions
+ * made one at a time, [14..15] clock cycles in CTA-wide and in warp-wide attempts.  A debugging aid; synchronises
+ * like rt_stats. */
+rt_status rt_debug_counters(rt_tree* tree, int64_t* out16);
 
 /* Settings for tests and debugging; process-wide, read when a later call is made; value < 0 restores the default.
  *   "run_one_by_one"   1: klpm_run takes the one-decision-at-a-time loop on every tree (default 0)

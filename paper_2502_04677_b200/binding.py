@@ -86,7 +86,7 @@ _lib.klpm_batch_times.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp, _vp
 _lib.klpm_run_last_only_batch.restype = _i32
 _lib.klpm_run_last_only_batch.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, ctypes.POINTER(klpm_params), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.rt_debug_counters.restype = _i32
-_lib.rt_debug_counters.argtypes = [_vp, ctypes.POINTER(_i64 * 8)]
+_lib.rt_debug_counters.argtypes = [_vp, ctypes.POINTER(_i64 * 16)]
 _lib.klpm_debug_set.restype = _i32
 _lib.klpm_debug_set.argtypes = [ctypes.c_char_p, _i64]
 _lib.klpm_run_path.restype = _i32
@@ -333,10 +333,11 @@ def klpm_run_last_only_batch(tokens: torch.Tensor, offsets: torch.Tensor, arriva
 
 def rt_debug_counters(tree: Tree) -> dict:
     """What the grouped loop of the last klpm_run on this tree did (see include/klpm.h)."""
-    v = (_i64 * 8)()
+    v = (_i64 * 16)()
     _check(_lib.rt_debug_counters(tree.handle, ctypes.byref(v)), "rt_debug_counters")
     names = ("careful_steps", "cta_dissolves", "fallback_scans", "fallen_back", "evictions", "cycles_tree", "cycles_scans",
-             "cycles_cta_dissolves")
+             "cycles_cta_dissolves", "cta_batches_tried", "cta_batches", "cta_batch_decisions", "warp_steps",
+             "warp_step_decisions", "single_decisions", "cycles_cta_batches", "cycles_warp_steps")
     return dict(zip(names, [int(x) for x in v]))
 
 

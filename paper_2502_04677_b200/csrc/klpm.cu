@@ -617,12 +617,12 @@ match_chain_kernel(TreeDev T, const int32_t* __restrict__ qtok, const int64_t* _
 
 // The order in which the batched match takes the queries: bucketed by first token (counting sort over a hash of
 // it; the order inside a bucket is whatever the atomics give -- results do not depend on it).
-#define KLPM_ORDER_BUCKETS 65536
+#define KLPM_ORDER_BUCKETS 8192
 __device__ __forceinline__ unsigned order_bucket(const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t i) {
     const int64_t lo = __ldg(qoff + i);
     if (__ldg(qoff + i + 1) <= lo) return 0u;
     unsigned h = (unsigned)__ldg(qtok + lo) * 0x9E3779B1u;
-    return h >> 16;
+    return h >> 19;                                         // 13 bits: KLPM_ORDER_BUCKETS
 }
 __global__ void order_hist_kernel(const int32_t* __restrict__ qtok, const int64_t* __restrict__ qoff, int32_t nq,
                                   unsigned* __restrict__ hist, unsigned short* __restrict__ bucket) {
@@ -632,7 +632,7 @@ __global__ void order_hist_kernel(const int32_t* __restrict__ qtok, const int64_
     bucket[i] = (unsigned short)b;
     atomicAdd(hist + b, 1u);
 }
-// hist[b] <- number of queries in buckets below b (one CTA of 1,024 threads, 64 buckets each)
+// hist[b] <- number of queries in buckets below b (one CTA of 1,024 threads, 8 buckets each)
 __global__ void __launch_bounds__(1024) order_scan_kernel(unsigned* hist) {
     __shared__ unsigned s_w[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1408,8 +1408,10 @@ struct alignas(32) FStat {    // constant during the loop; the first 16 bytes ar
 struct FastPost {
     int32_t c0; int32_t pad; long long now0;    // first decision made in list mode; the time it was made at
     // what the loop did (rt_debug_counters): careful steps, dissolves by the whole CTA, fallback scans, slots that fell
-    // back, evictions; cycles spent in tree updates, fallback scans, dissolves
-    long long counters[8];
+    // back, evictions; cycles spent in tree updates, fallback scans, dissolves; list mode: CTA-wide batches tried and
+    // committed, decisions they made, warp-wide steps, decisions they made, decisions made one at a time; cycles in
+    // CTA-wide attempts and in warp-wide attempts
+    long long counters[16];
 };
 
 struct FastArgs {
@@ -1701,7 +1703,15 @@ struct FastBatchIO {
     int32_t B0, nF0, nL0, limF, limL; // scratch
 };
 #define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
-#define KLPM_FAST_CTA_MIN 128         // smaller batches are left to the warp-wide step (an attempt costs about 5,000 cycles)
+#ifndef KLPM_FAST_CTA_MIN
+#define KLPM_FAST_CTA_MIN 128         // smaller batches are left to the warp-wide step (an attempt costs about 16,000 cycles)
+#endif
+#ifndef KLPM_FAST_CB_MAX
+#define KLPM_FAST_CB_MAX 1024         // longest back-off (loop iterations) after CTA-wide attempts that failed
+#endif
+#ifndef KLPM_FAST_CALM
+#define KLPM_FAST_CALM 4              // full warp-wide steps in a row before a CTA-wide batch is tried again
+#endif
 
 // Exclusive prefix sum of v over the CTA's 256 threads; *total receives the sum.  s_w: 8 ints of shared scratch.
 __device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* s_w, int32_t* total) {
@@ -2730,19 +2740,24 @@ fast_run_kernel(FastArgs A) {
         };
         int32_t vb_wait = 0, vb_back = 1;                   // decisions until the next attempt; doubles while attempts fail
         int32_t cb_wait = 0, cb_back = 8;                   // the same for the CTA-wide batch (loop iterations; 8 .. 1,024)
-        int32_t calm = 4;                                   // consecutive full warp-wide steps: the CTA-wide batch is tried in calm water only
+        int32_t calm = KLPM_FAST_CALM;                      // consecutive full warp-wide steps: the CTA-wide batch is tried in calm water only
+        long long n_cta_try = 0, n_cta_ok = 0, dec_cta = 0, n_warp_ok = 0, dec_warp = 0, dec_one = 0, cy_cta = 0, cy_warp = 0;
         while (c < n && !failed) {
             // first choice: the whole CTA makes up to 1,024 decisions (the sort scratch is free between dissolves)
-            if (cb_wait <= 0 && calm >= 4 && n - c >= KLPM_FAST_CTA_MIN) {
+            if (cb_wait <= 0 && calm >= KLPM_FAST_CALM && n - c >= KLPM_FAST_CTA_MIN) {
                 if (lane == 0) {
                     s_bio.cur = cur; s_bio.head = head; s_bio.c = c; s_bio.cyc = cyc; s_bio.root = root; s_bio.B = 0;
                     s_job.type = FAST_JOB_BATCH;
                 }
                 __syncwarp();
+                const long long t_cta = clock64();
+                ++n_cta_try;
                 named_bar(1, KLPM_FAST_THREADS);
                 fast_batch_job(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords);
                 const int32_t Bc = s_bio.B;
+                cy_cta += clock64() - t_cta;
                 if (Bc > 0) {
+                    ++n_cta_ok; dec_cta += Bc;
                     const int32_t consumed = s_bio.consumed, hmax = s_bio.hmax;
                     c += Bc;
                     if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + Bc) % A.k;
@@ -2753,18 +2768,22 @@ fast_run_kernel(FastArgs A) {
                     continue;
                 }
                 cb_wait = cb_back;
-                cb_back = cb_back < 1024 ? cb_back * 2 : 1024;
+                cb_back = cb_back < KLPM_FAST_CB_MAX ? cb_back * 2 : KLPM_FAST_CB_MAX;
                 calm = 0;
             }
             --cb_wait;
             if (vb_wait <= 0) {
                 const int32_t c_was = c;
-                if (try_batch()) { vb_back = 1; calm = c - c_was == 32 ? calm + 1 : 0; continue; }
+                const long long t_w = clock64();
+                const bool took = try_batch();
+                cy_warp += clock64() - t_w;
+                if (took) { ++n_warp_ok; dec_warp += c - c_was; vb_back = 1; calm = c - c_was == 32 ? calm + 1 : 0; continue; }
                 calm = 0;
                 vb_wait = vb_back;
                 vb_back = vb_back < 64 ? vb_back * 2 : 64;
             }
             --vb_wait;
+            ++dec_one;
             const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
             if (++cyc == A.k) cyc = 0;
             int32_t j;
@@ -2809,9 +2828,15 @@ fast_run_kernel(FastArgs A) {
                 ++c;
             }
         }
+        if (lane == 0) {
+            long long* cn = A.post->counters;
+            cn[8] = n_cta_try; cn[9] = n_cta_ok; cn[10] = dec_cta; cn[11] = n_warp_ok; cn[12] = dec_warp; cn[13] = dec_one;
+            cn[14] = cy_cta; cn[15] = cy_warp;
+        }
     } else if (lane == 0) {
         A.post->c0 = n;                                     // list mode never began: nothing is left to charge
         A.post->now0 = now;
+        for (int i = 8; i < 16; ++i) A.post->counters[i] = 0;
     }
     __syncwarp();
     if (lane == 0) {
@@ -4335,14 +4360,14 @@ rt_status klpm_run_last_only_batch(const int32_t* d_tokens, const int64_t* d_off
 
 int32_t klpm_run_path(const rt_tree* tree) { return tree ? tree->run_path : 0; }
 
-rt_status rt_debug_counters(rt_tree* tree, int64_t* out8) {
-    if (!tree || !out8) return RT_ERR_INVALID;
-    memset(out8, 0, 8 * sizeof(int64_t));
+rt_status rt_debug_counters(rt_tree* tree, int64_t* out16) {
+    if (!tree || !out16) return RT_ERR_INVALID;
+    memset(out16, 0, 16 * sizeof(int64_t));
     if (!tree->fast_post) return RT_OK;
     CK(cudaStreamSynchronize(tree->last_stream));
     FastPost h;
     CK(cudaMemcpy(&h, tree->fast_post, sizeof(h), cudaMemcpyDeviceToHost));
-    for (int i = 0; i < 8; ++i) out8[i] = h.counters[i];
+    for (int i = 0; i < 16; ++i) out16[i] = h.counters[i];
     return RT_OK;
 }
 
