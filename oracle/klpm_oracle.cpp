@@ -16,7 +16,7 @@
 //                        eviction under a fixed token budget (Section 1, RadixAttention)
 //   policies           FCFS, LPM (Section 1) and k-LPM (Algorithm 1)
 //
-// Readings taken where the paper is silent (the same list is in the design notes):
+// Readings taken where the paper is silent:
 //   * Algorithm 1 is followed as printed: one oldest-first pick, then k-1
 //     longest-match picks; the pick counter never resets (idle periods included).
 //   * "prefix cache hit rate" is the absolute match length in tokens; the other reading
