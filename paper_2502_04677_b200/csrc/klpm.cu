@@ -2262,9 +2262,7 @@ fast_run_kernel(FastArgs A) {
     };
     // Charge pick `slot` (Definition 2), write its outputs, and let the queries tied with it match into its new
     // leaf.  The caller has taken the slot out of the tournament or the list and marked it processed.
-    auto careful = [&](int32_t slot, bool charge) {
-        const FDyn d = ld_dyn(A.dyn + slot);
-        const FStat s = ld_stat(A.stat + slot);
+    auto careful = [&](int32_t slot, bool charge, const FDyn& d, const FStat& s) {
         const int32_t m = d.m, len = s.len, unc = len - m;
         if (charge) {
             const long long begin = now > s.t ? now : s.t;
@@ -2293,17 +2291,32 @@ fast_run_kernel(FastArgs A) {
                 failed = true; return;
             }
             const long long clock = s_st.clock + 1;
-            int32_t a = d.hint, ds = T.depth_start[a];
-            while (a != 0 && m <= ds) { a = T.parent[a]; ds = T.depth_start[a]; }
-            const int32_t o = a == 0 ? 0 : m - ds, sl = T.span_len[a];
+            // Two chains of dependent loads are started side by side: the node the match ends in (hint, then up), and
+            // the least recently used leaf (the cursor's next 32 clock values, their owners' fields) -- most decisions
+            // evict, and which leaf goes does not depend on the pick, except that the node stamped below is safe.
+            const long long cur0 = s_st.lru_cursor;
+            int32_t a = d.hint;
+            int32_t ds = T.depth_start[a], sl = T.span_len[a], pa = T.parent[a];
+            const long long pre_cc = cur0 + lane;
+            const int32_t pre_v = pre_cc < clock ? T.clock_owner[pre_cc] : 0;
+            bool pre_ok = false;
+            int32_t pre_P = 0, pre_len = 0;
+            if (pre_v > 0) {
+                pre_ok = !T.dead[pre_v] && T.last_access[pre_v] == pre_cc && T.nchild[pre_v] == 0;
+                pre_P = T.parent[pre_v]; pre_len = T.span_len[pre_v];
+            }
+            while (a != 0 && m <= ds) { a = pa; ds = T.depth_start[a]; sl = T.span_len[a]; pa = T.parent[a]; }
+            const int32_t o = a == 0 ? 0 : m - ds;
             int32_t end = a;
+            bool cut = false;
             long long n_nodes = s_st.n_nodes, live_nodes = s_st.live_nodes, tokens_live = s_st.tokens_live, evictions = s_st.evictions;
             if (a != 0 && o < sl) {                         // node boundary inside a's edge: a new node takes the upper part
                 const int32_t u = (int32_t)n_nodes++;
                 ++live_nodes;
+                cut = true;
                 if (lane == 0) {
                     const int64_t so = T.span_off[a];
-                    T.parent[u] = T.parent[a]; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = o;
+                    T.parent[u] = pa; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = o;
                     T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = T.last_access[a];
                     T.span_off[a] = so + o; T.span_len[a] = sl - o; T.depth_start[a] = ds + o; T.parent[a] = u;
                 }
@@ -2315,23 +2328,38 @@ fast_run_kernel(FastArgs A) {
             bool scan = false;
             int32_t small_v[8];                             // evicted leaves whose parked queries this warp looks after itself
             int n_small = 0;
-            long long cur = s_st.lru_cursor;
+            long long cur = cur0;
+            bool first = true;
             while (tokens_live + unc > T.budget) {
-                int32_t victim = -1;
-                while (cur < clock) {                       // 32 clock values at a time
-                    const long long cc = cur + lane;
-                    const int32_t v = cc < clock ? T.clock_owner[cc] : 0;
-                    const bool ok = v > 0 && !T.dead[v] && T.last_access[v] == cc && T.nchild[v] == 0;
-                    const unsigned bal = __ballot_sync(FULL_MASK, ok);
-                    if (bal) { const int src = __ffs(bal) - 1; victim = __shfl_sync(FULL_MASK, v, src); cur += src; break; }
-                    cur += 32;
+                int32_t victim = -1, P = 0, vlen = 0;
+                if (first) {                                // the window that was loaded ahead (the node stamped above has moved on)
+                    const unsigned bal = __ballot_sync(FULL_MASK, pre_ok && pre_v != end);
+                    if (bal) {
+                        const int src = __ffs(bal) - 1;
+                        victim = __shfl_sync(FULL_MASK, pre_v, src); P = __shfl_sync(FULL_MASK, pre_P, src); vlen = __shfl_sync(FULL_MASK, pre_len, src);
+                        cur += src;
+                        if (cut && victim == a) { P = T.parent[victim]; vlen = T.span_len[victim]; }      // the lower part of the edge just cut
+                    } else {
+                        cur += 32;
+                    }
+                    first = false;
+                }
+                if (victim < 0) {
+                    while (cur < clock) {                   // 32 clock values at a time
+                        const long long cc = cur + lane;
+                        const int32_t v = cc < clock ? T.clock_owner[cc] : 0;
+                        const bool ok = v > 0 && !T.dead[v] && T.last_access[v] == cc && T.nchild[v] == 0;
+                        const unsigned bal = __ballot_sync(FULL_MASK, ok);
+                        if (bal) { const int src = __ffs(bal) - 1; victim = __shfl_sync(FULL_MASK, v, src); cur += src; break; }
+                        cur += 32;
+                    }
+                    if (victim >= 0) { P = T.parent[victim]; vlen = T.span_len[victim]; }
                 }
                 if (victim < 0) {
                     if (lane == 0) set_status(A.st, RT_ERR_BUDGET);
                     failed = true; break;
                 }
-                const int32_t P = T.parent[victim];
-                tokens_live -= T.span_len[victim];
+                tokens_live -= vlen;
                 --live_nodes; ++evictions; ++n_evict;
                 if (__ldcg(A.parked + victim) > 0) {
                     // Queries are parked in the evicted leaf.  If one run of the member array is known to hold every slot
@@ -2581,7 +2609,9 @@ fast_run_kernel(FastArgs A) {
             slot = A.pinv ? __ldg(A.pinv + rk) : (int32_t)rk;
         }
         if (slot < 0 || slot >= admitted || slot_done(R, A, slot)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 105); failed = true; break; }   // cannot happen
-        // ---- the pick leaves its leaf block
+        // ---- the pick leaves its leaf block (its two records are asked for first: they travel with the block's keys)
+        const FDyn pd = ld_dyn(A.dyn + slot);
+        const FStat ps = ld_stat(A.stat + slot);
         const int32_t b = slot >> A.lb_shift;
         unsigned long long bm = 0;
         for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
@@ -2590,7 +2620,7 @@ fast_run_kernel(FastArgs A) {
         }
         root = tour_set(R, b, warp_max64r(bm), lane);
         mark_done(slot);
-        careful(slot, true);
+        careful(slot, true, pd, ps);
         if (slot == head) advance_head();
         __syncwarp();
     }
@@ -2822,7 +2852,7 @@ fast_run_kernel(FastArgs A) {
             }
             if (j == head) advance_head();
             if ((R.gb[j >> 5] >> (j & 31)) & 1u) {
-                careful(j, false);
+                careful(j, false, ld_dyn(A.dyn + j), ld_stat(A.stat + j));
             } else {
                 if (lane == 0) A.order[c] = j;
                 ++c;
