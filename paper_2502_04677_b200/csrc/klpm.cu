@@ -1430,8 +1430,10 @@ struct FastArgs {
     int32_t lb_shift;             // log2 of the number of slots per tournament leaf block
     int32_t nb;                   // number of leaf blocks
     int32_t done_in_smem;
-    int32_t list_mode;            // the list mode of the loop can be used (32-slot leaf blocks, all bitmaps in shared memory)
-    unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts
+    int32_t list_mode;            // the list mode of the loop can be used (trees without a budget)
+    unsigned int* gbits;          // bitmap of slots whose group has more than one member, as the loop starts (and throughout, if the bitmaps stay in global memory)
+    unsigned int* gskip;          // list mode with the bitmaps in global memory: slots the sorted list must pass over
+    int32_t bits_in_smem;         // list mode: those two bitmaps are in shared memory
     const long long* lk;          // list mode: every slot's key, largest first, stored as ~key with the top bit flipped
     const int32_t* ls;            //            and the slot it belongs to
     const int64_t* arrival;       // per query: arrival (for the charge pass after the loop)
@@ -1612,9 +1614,13 @@ struct FastTour {
     unsigned int* skip;       // bitmap of slots the sorted list must pass over: processed, or key changed (shared memory), or null
     unsigned int* gb;         // bitmap of slots whose group has more than one member (shared memory), or null
     unsigned int* dirty;      // trees with a budget: bitmap of leaf blocks to recompute after a fallback (256 words, shared memory)
+    int g_done, g_bits;       // the processed bitmap / the other two bitmaps live in global memory (queues too long for shared memory)
     int32_t n2;               // entries of t2 in use
     int32_t n3;               // entries of t3 in use
 };
+// A word of one of the loop's bitmaps: shared memory, or global memory read through L2 (other warps set bits with atomics).
+__device__ __forceinline__ unsigned bm_ld(const unsigned int* p, long long i, int g) { return g ? __ldcg(p + i) : p[i]; }
+
 // Recompute the ancestors of leaf block b; returns the root.  One warp.
 __device__ __forceinline__ unsigned long long tour_update(const FastTour& R, int32_t b, int lane) {
     const int32_t i2 = b >> 5;
@@ -1656,7 +1662,7 @@ __device__ __forceinline__ void tour_mid(const FastTour& R, int warp, int nwarps
 }
 // has slot r been processed?  (the bitmap lives in shared memory when it fits)
 __device__ __forceinline__ bool slot_done(const FastTour& R, const FastArgs& A, long long r) {
-    const unsigned w = R.done ? R.done[r >> 5] : __ldcg(A.done + (r >> 5));
+    const unsigned w = bm_ld(R.done, r >> 5, R.g_done);
     return (w >> (r & 31)) & 1u;
 }
 // position of the k-th set bit of w (k >= 1, at most the number of set bits)
@@ -1693,6 +1699,19 @@ __device__ __forceinline__ void lru_move(const FastArgs& A, int32_t r, int32_t f
     __stcg(A.hintc + r, to);
     atomicSub(A.parked + from, 1);
     atomicAdd(A.parked + to, 1);
+}
+
+// List mode: the largest key among the unprocessed slots of leaf block b whose key has changed since the sort.  One warp.
+__device__ __forceinline__ unsigned long long changed_block_max(const FastArgs& A, const FastTour& R, int32_t b, int lane) {
+    unsigned long long v = 0;
+    for (int32_t u = lane; u < (1 << A.lb_shift); u += 32) {
+        const long long r = ((long long)b << A.lb_shift) + u;
+        if (r < A.n) {
+            const unsigned w = bm_ld(R.skip, r >> 5, R.g_bits) & ~bm_ld(R.done, r >> 5, R.g_done);
+            if ((w >> (r & 31)) & 1u) { const unsigned long long kk = __ldcg(A.key + r); if (kk > v) v = kk; }
+        }
+    }
+    return warp_max64r(v);
 }
 
 // What the sequencer hands to a CTA-wide batch of decisions, and what it gets back.
@@ -1769,8 +1788,11 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
 // The warp-wide step of list mode (see fast_run_kernel) with the whole CTA: 1,024 list entries and 8,192 bitmap slots
 // are examined at once, the same checks cut the batch short, block-wide prefix sums replace the warp's ballots.
 // Every thread calls it.  Nothing is changed unless at least KLPM_FAST_CTA_MIN decisions can be made.
-__device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO* io, int32_t* sH, int32_t* sE, int32_t* sEpos,
+template <bool G>
+__device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchIO* io, int32_t* sH, int32_t* sE, int32_t* sEpos,
                                int32_t* s_w, int32_t nwords) {
+    FastTour R = R0;                                        // with the bitmaps in shared memory the flags fold away
+    if (!G) { R.g_done = 0; R.g_bits = 0; }
     const int tid = threadIdx.x;
     const int32_t n = A.n, cur = io->cur, head = io->head, c = io->c, cyc = io->cyc;
     const unsigned long long root = io->root;
@@ -1789,7 +1811,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO
         ok[r] = false; kk[r] = 0; es[r] = 0;
         if (idx < n) {
             kk[r] = __ldg(A.lk + idx); es[r] = __ldg(A.ls + idx);
-            ok[r] = !((R.skip[es[r] >> 5] >> (es[r] & 31)) & 1u);
+            ok[r] = !((bm_ld(R.skip, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u);
         }
         cnt += ok[r];
     }
@@ -1807,7 +1829,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO
     int32_t hmax0 = -1;
     if (nF0 > 0) {
         const int32_t w0 = head >> 5, wi = w0 + tid;
-        unsigned w = wi < nwords ? R.done[wi] : 0xffffffffu;
+        unsigned w = wi < nwords ? bm_ld(R.done, wi, R.g_done) : 0xffffffffu;
         if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
         if (wi == w0) w |= (1u << (head & 31)) - 1u;
         unsigned fr = ~w;
@@ -1820,7 +1842,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO
         if (nFa > 0) hmax0 = sH[nFa - 1];
         for (int32_t qi = tid; qi < nFa; qi += KLPM_FAST_THREADS) {       // key in the tournament, or grouped: needs the careful step
             const int32_t hs = sH[qi];
-            if (((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u) atomicMin(&io->limF, qi);
+            if (((bm_ld(R.skip, hs >> 5, R.g_bits) | bm_ld(R.gb, hs >> 5, R.g_bits)) >> (hs & 31)) & 1u) atomicMin(&io->limF, qi);
         }
     }
     // the usable entries by rank; the first one that is grouped, could also be an oldest-first pick of this batch, or
@@ -1833,7 +1855,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R, FastBatchIO
                 if (rk < nL0) {
                     sE[rk] = es[r]; sEpos[rk] = tid * 4 + r;
                     const unsigned long long ek = ~((unsigned long long)kk[r] ^ 0x8000000000000000ULL);
-                    if ((((R.gb[es[r] >> 5] >> (es[r] & 31)) & 1u)) || (es[r] >= head && es[r] <= hmax0) || root > ek) atomicMin(&io->limL, rk);
+                    if ((((bm_ld(R.gb, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u)) || (es[r] >= head && es[r] <= hmax0) || root > ek) atomicMin(&io->limL, rk);
                 }
                 ++rk;
             }
@@ -2084,9 +2106,7 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
     } else if (J.type == FAST_JOB_REBUILD) {
         // entering list mode (32-slot leaf blocks): the tournament keeps only the unprocessed slots whose key has changed
         for (int32_t b = warp; b < A.nb; b += nwarps) {
-            const unsigned w = R.skip[b] & ~R.done[b];
-            unsigned long long v = 0;
-            if (w) v = warp_max64r(((w >> lane) & 1u) ? __ldcg(A.key + ((long long)b << 5) + lane) : 0ULL);
+            const unsigned long long v = changed_block_max(A, R, b, lane);
             if (lane == 0) R.t1[b] = v;
         }
     } else {
@@ -2170,6 +2190,9 @@ __device__ void fast_job(const FastArgs& A, const FastTour& R, const FastJob& J,
 // from the list touches no tournament at all, up to 32 decisions are made by one warp-wide step (up to 1,024 by a
 // CTA-wide one, fast_batch_job), and the loop only records which slot each decision takes: the charge pass after the
 // loop computes their outputs.
+// G: some of the loop's bitmaps live in global memory (queues too long for shared memory).  The instance without them
+// reads its bitmaps as plain shared-memory words.
+template <bool G>
 __global__ void __launch_bounds__(KLPM_FAST_THREADS, 1)
 fast_run_kernel(FastArgs A) {
     extern __shared__ __align__(16) unsigned char fast_smem[];
@@ -2193,15 +2216,21 @@ fast_run_kernel(FastArgs A) {
     R.n2 = n2; R.n3 = n3;
     unsigned long long* sh = R.t3 + 32;
     int32_t* sr = reinterpret_cast<int32_t*>(sh + KLPM_FAST_SORT_CAP);
-    unsigned int* s_done = reinterpret_cast<unsigned int*>(sr + KLPM_FAST_SORT_CAP);
-    R.done = A.done_in_smem ? s_done : nullptr;
-    R.skip = A.list_mode ? s_done + nwords : nullptr;
-    R.gb = A.list_mode ? s_done + 2 * nwords : nullptr;
+    unsigned int* s_bits = reinterpret_cast<unsigned int*>(sr + KLPM_FAST_SORT_CAP);
+    // the bitmaps: in shared memory while they fit, in global memory (cleared / filled by the host side) otherwise
+    R.g_done = A.done_in_smem ? 0 : 1;
+    R.g_bits = A.bits_in_smem ? 0 : 1;
+    R.done = A.done_in_smem ? s_bits : A.done;
+    R.skip = !A.list_mode ? nullptr : A.bits_in_smem ? s_bits + nwords : A.gskip;
+    R.gb = !A.list_mode ? nullptr : A.bits_in_smem ? s_bits + 2 * nwords : A.gbits;
     R.dirty = s_dirty;
+    unsigned int* const s_done = R.done;
+    if (!G) { R.g_done = 0; R.g_bits = 0; }
+    const int gdone = G ? R.g_done : 0, gbits = G ? R.g_bits : 0;
     for (int32_t i = threadIdx.x; i < nb1p + n2p + 32; i += blockDim.x) R.t1[i] = 0ULL;
     if (threadIdx.x == 0) { s_memcur = A.lru ? 2 * n : n; if (A.lru) s_st = *A.st; }
-    if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_done[i] = 0u;
-    if (A.list_mode) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
+    if (A.done_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) s_bits[i] = 0u;
+    if (A.list_mode && A.bits_in_smem) for (int32_t i = threadIdx.x; i < nwords; i += blockDim.x) { R.skip[i] = 0u; R.gb[i] = __ldcg(A.gbits + i); }
     __syncthreads();
 
     if (warp != 0) {
@@ -2209,7 +2238,7 @@ fast_run_kernel(FastArgs A) {
             named_bar(1, KLPM_FAST_THREADS);
             const FastJob J = s_job;
             if (J.type == FAST_JOB_EXIT) return;
-            if (J.type == FAST_JOB_BATCH) { fast_batch_job(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords); continue; }
+            if (J.type == FAST_JOB_BATCH) { fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords); continue; }
             fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
         }
     }
@@ -2227,12 +2256,12 @@ fast_run_kernel(FastArgs A) {
 
     // first unprocessed slot at or after `head` (which is processed)
     auto advance_head = [&]() {
-        if (A.done_in_smem && head + 1 < n) {               // the usual cases: the next slot, or one of the next 32 to 63
+        if (head + 1 < n) {                                 // the usual cases: the next slot, or one of the next 32 to 63
             const int32_t h1 = head + 1, wi = h1 >> 5;
-            const unsigned f0 = ~s_done[wi] & ~((1u << (h1 & 31)) - 1u);
+            const unsigned f0 = ~bm_ld(s_done, wi, gdone) & ~((1u << (h1 & 31)) - 1u);
             if (f0) { head = wi * 32 + __ffs(f0) - 1; if (head > n) head = n; return; }
             if (wi + 1 < nwords) {
-                const unsigned f1 = ~s_done[wi + 1];
+                const unsigned f1 = ~bm_ld(s_done, wi + 1, gdone);
                 if (f1) { head = (wi + 1) * 32 + __ffs(f1) - 1; if (head > n) head = n; return; }
             }
         }
@@ -2240,7 +2269,7 @@ fast_run_kernel(FastArgs A) {
         for (;;) {
             const int32_t wi = w0 + lane;
             unsigned w = 0u;                                  // past the end: "unprocessed", so the search stops
-            if (wi < nwords) w = A.done_in_smem ? s_done[wi] : __ldcg(A.done + wi);
+            if (wi < nwords) w = bm_ld(s_done, wi, gdone);
             if (wi == (head >> 5)) w |= (1u << (head & 31)) - 1u;
             const unsigned bal = __ballot_sync(FULL_MASK, w != 0xffffffffu);
             if (bal) {
@@ -2255,9 +2284,12 @@ fast_run_kernel(FastArgs A) {
     };
     // slot j is processed from now on (every lane performs the same shared-memory stores)
     auto mark_done = [&](int32_t j) {
-        if (A.done_in_smem) s_done[j >> 5] |= 1u << (j & 31);
-        else if (lane == 0) __stcg(A.done + (j >> 5), __ldcg(A.done + (j >> 5)) | (1u << (j & 31)));
-        if (R.skip) R.skip[j >> 5] |= 1u << (j & 31);
+        if (!gdone) s_done[j >> 5] |= 1u << (j & 31);
+        else if (lane == 0) __stcg(s_done + (j >> 5), __ldcg(s_done + (j >> 5)) | (1u << (j & 31)));
+        if (R.skip) {
+            if (!gbits) R.skip[j >> 5] |= 1u << (j & 31);
+            else if (lane == 0) __stcg(R.skip + (j >> 5), __ldcg(R.skip + (j >> 5)) | (1u << (j & 31)));
+        }
         __syncwarp();
     };
     // Charge pick `slot` (Definition 2), write its outputs, and let the queries tied with it match into its new
@@ -2686,7 +2718,7 @@ fast_run_kernel(FastArgs A) {
                 kk = off < 32 ? k0 : k1;
                 es = off < 32 ? s0 : s1;
                 const bool valid = (long long)cur + lane < n;
-                mask = __ballot_sync(FULL_MASK, valid && !((R.skip[es >> 5] >> (es & 31)) & 1u));
+                mask = __ballot_sync(FULL_MASK, valid && !((bm_ld(R.skip, es >> 5, gbits) >> (es & 31)) & 1u));
             }
             // as many decisions as those entries allow: lane x asks whether x + 1 decisions need no more of them
             const int32_t avail = __popc(mask);
@@ -2699,7 +2731,7 @@ fast_run_kernel(FastArgs A) {
                 const int32_t w0 = head >> 5;
                 const int32_t qk = lane < nF0 ? lane : nF0 - 1;       // lane q looks for the q-th unprocessed slot
                 auto free_word = [&](int32_t wi) -> unsigned {        // unprocessed slots of bitmap word wi, from head on
-                    unsigned w = wi < nwords ? s_done[wi] : 0xffffffffu;
+                    unsigned w = wi < nwords ? bm_ld(s_done, wi, gdone) : 0xffffffffu;
                     if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
                     if (wi == w0) w |= (1u << (head & 31)) - 1u;
                     return ~w;
@@ -2724,7 +2756,7 @@ fast_run_kernel(FastArgs A) {
                 }
                 hmax0 = __shfl_sync(FULL_MASK, hs, nF0 - 1);
                 // its key sits in the tournament, or its group has other members
-                const unsigned badH = __ballot_sync(FULL_MASK, lane < nF0 && ((((R.skip[hs >> 5] | R.gb[hs >> 5]) >> (hs & 31)) & 1u)));
+                const unsigned badH = __ballot_sync(FULL_MASK, lane < nF0 && ((((bm_ld(R.skip, hs >> 5, gbits) | bm_ld(R.gb, hs >> 5, gbits)) >> (hs & 31)) & 1u)));
                 if (badH) limF = __ffs(badH) - 1;
             }
             // limL = how many list entries can be taken before one is grouped, could also be an oldest-first pick of
@@ -2735,7 +2767,7 @@ fast_run_kernel(FastArgs A) {
             {
                 const unsigned long long ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL);
                 const unsigned badE = __ballot_sync(FULL_MASK, ok && rank < nL0 &&
-                                                    ((((R.gb[es >> 5] >> (es & 31)) & 1u)) || (es >= head && es <= hmax0) || root > ek));
+                                                    ((((bm_ld(R.gb, es >> 5, gbits) >> (es & 31)) & 1u)) || (es >= head && es <= hmax0) || root > ek));
                 if (badE) limL = __popc(mask & ((1u << (__ffs(badE) - 1)) - 1u));
             }
             const int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_hi <= limF && (lane + 1) - f_hi <= limL));
@@ -2765,7 +2797,7 @@ fast_run_kernel(FastArgs A) {
                 cur = ncur;
             }
             if (nF > 0) { head = hmax; advance_head(); }
-            else if (head < n && ((s_done[head >> 5] >> (head & 31)) & 1u)) advance_head();
+            else if (head < n && ((bm_ld(s_done, head >> 5, gdone) >> (head & 31)) & 1u)) advance_head();
             return true;
         };
         int32_t vb_wait = 0, vb_back = 1;                   // decisions until the next attempt; doubles while attempts fail
@@ -2783,7 +2815,7 @@ fast_run_kernel(FastArgs A) {
                 const long long t_cta = clock64();
                 ++n_cta_try;
                 named_bar(1, KLPM_FAST_THREADS);
-                fast_batch_job(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords);
+                fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords);
                 const int32_t Bc = s_bio.B;
                 cy_cta += clock64() - t_cta;
                 if (Bc > 0) {
@@ -2793,7 +2825,7 @@ fast_run_kernel(FastArgs A) {
                     if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + Bc) % A.k;
                     if (consumed) { cur += consumed; window(cur & ~31, &wk, &ws); window((cur & ~31) + 32, &nk, &ns); }
                     if (hmax >= 0) { head = hmax; advance_head(); }
-                    else if (head < n && ((s_done[head >> 5] >> (head & 31)) & 1u)) advance_head();
+                    else if (head < n && ((bm_ld(s_done, head >> 5, gdone) >> (head & 31)) & 1u)) advance_head();
                     cb_back = 8;
                     continue;
                 }
@@ -2820,7 +2852,7 @@ fast_run_kernel(FastArgs A) {
             bool in_tour;                                   // the pick's key is in the tournament (it changed after the sort)
             if (fcfs_turn) {
                 j = head;
-                in_tour = (R.skip[j >> 5] >> (j & 31)) & 1u;
+                in_tour = (bm_ld(R.skip, j >> 5, gbits) >> (j & 31)) & 1u;
             } else {
                 unsigned long long ek = 0;                  // next entry of the list that still counts
                 int32_t es = -1;
@@ -2828,7 +2860,7 @@ fast_run_kernel(FastArgs A) {
                     const int src = cur & 31;
                     const long long kk = __shfl_sync(FULL_MASK, wk, src);
                     es = __shfl_sync(FULL_MASK, ws, src);
-                    if (!((R.skip[es >> 5] >> (es & 31)) & 1u)) { ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL); break; }
+                    if (!((bm_ld(R.skip, es >> 5, gbits) >> (es & 31)) & 1u)) { ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL); break; }
                     es = -1;
                     advance_cur();
                 }
@@ -2842,16 +2874,21 @@ fast_run_kernel(FastArgs A) {
                     advance_cur();
                 }
             }
-            if (j < 0 || j >= n || ((s_done[j >> 5] >> (j & 31)) & 1u)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 107); failed = true; break; }   // cannot happen
+            if (j < 0 || j >= n || ((bm_ld(s_done, j >> 5, gdone) >> (j & 31)) & 1u)) { if (lane == 0) set_status(A.st, RT_ERR_LIMIT, 107); failed = true; break; }   // cannot happen
             mark_done(j);
             if (in_tour) {                                  // its leaf block's largest changed key, without it
-                const int32_t b = j >> 5;
-                const unsigned w = R.skip[b] & ~s_done[b];
-                const unsigned long long kk = ((w >> lane) & 1u) ? __ldcg(A.key + ((long long)b << 5) + lane) : 0ULL;
-                root = tour_set(R, b, warp_max64r(kk), lane);
+                const int32_t b = j >> A.lb_shift;
+                unsigned long long kk;
+                if (!G && A.lb_shift == 5) {                // 32-slot blocks, bitmaps in shared memory: one word of each
+                    const unsigned w = R.skip[b] & ~s_done[b];
+                    kk = warp_max64r(((w >> lane) & 1u) ? __ldcg(A.key + ((long long)b << 5) + lane) : 0ULL);
+                } else {
+                    kk = changed_block_max(A, R, b, lane);
+                }
+                root = tour_set(R, b, kk, lane);
             }
             if (j == head) advance_head();
-            if ((R.gb[j >> 5] >> (j & 31)) & 1u) {
+            if ((bm_ld(R.gb, j >> 5, gbits) >> (j & 31)) & 1u) {
                 careful(j, false, ld_dyn(A.dyn + j), ld_stat(A.stat + j));
             } else {
                 if (lane == 0) A.order[c] = j;
@@ -2890,19 +2927,24 @@ fast_run_kernel(FastArgs A) {
 // (Definition 2 with R_prev >= t_j).  Three small kernels: per decision its uncached tokens and cost (and the query
 // index put in `order`), a scan of the per-block sums, and the completion times and TTFTs.
 #define KLPM_CHARGE_THREADS 256
+// `ipt` consecutive decisions per thread: at most 1,024 blocks whatever the queue's length.
 __global__ void __launch_bounds__(KLPM_CHARGE_THREADS)
-charge_cost_kernel(FastArgs A, long long* cost, long long* bsum) {
+charge_cost_kernel(FastArgs A, long long* cost, long long* bsum, int32_t ipt) {
     __shared__ long long s_w[KLPM_CHARGE_THREADS / 32];
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x, c = A.post->c0 + i;
+    const long long i0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * ipt;
     long long x = 0;
-    if (c < A.n) {
-        const int32_t slot = A.order[c];
-        const int4 s = __ldg(reinterpret_cast<const int4*>(A.stat + slot));     // arrival, length, query index
-        const int32_t len = s.z, ord = s.w, unc = len - A.dyn[slot].m;
-        x = (A.c_den + A.c_num * (long long)len) * (long long)unc;
-        A.order[c] = ord;
-        A.uncached[ord] = unc;
-        cost[i] = x;
+    for (int32_t u = 0; u < ipt; ++u) {
+        const long long i = i0 + u, c = A.post->c0 + i;
+        if (c < A.n) {
+            const int32_t slot = A.order[c];
+            const int4 s = __ldg(reinterpret_cast<const int4*>(A.stat + slot));     // arrival, length, query index
+            const int32_t len = s.z, ord = s.w, unc = len - A.dyn[slot].m;
+            const long long y = (A.c_den + A.c_num * (long long)len) * (long long)unc;
+            A.order[c] = ord;
+            A.uncached[ord] = unc;
+            cost[i] = y;
+            x += y;
+        }
     }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) x += __shfl_down_sync(FULL_MASK, x, d);
@@ -2931,22 +2973,27 @@ charge_scan_kernel(FastArgs A, long long* bsum, int32_t nblocks) {
     if (u < nblocks) bsum[u] = A.post->now0 + s[u] - v;
 }
 __global__ void __launch_bounds__(KLPM_CHARGE_THREADS)
-charge_apply_kernel(FastArgs A, const long long* cost, const long long* bsum) {
+charge_apply_kernel(FastArgs A, const long long* cost, const long long* bsum, int32_t ipt) {
     __shared__ long long s_w[KLPM_CHARGE_THREADS / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x, c = A.post->c0 + i;
-    long long x = c < A.n ? cost[i] : 0;
+    const long long i0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * ipt;
+    long long mine = 0;                                     // cost of this thread's decisions
+    for (int32_t u = 0; u < ipt; ++u) { const long long c = A.post->c0 + i0 + u; if (c < A.n) mine += cost[i0 + u]; }
+    long long x = mine;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) { const long long o = __shfl_up_sync(FULL_MASK, x, d); if (lane >= d) x += o; }
     if (lane == 31) s_w[warp] = x;
     __syncthreads();
-    long long before = bsum[blockIdx.x];
-    for (int w = 0; w < warp; ++w) before += s_w[w];
-    if (c < A.n) {
-        const int32_t ord = A.order[c];
-        const long long Rj = before + x;
-        A.ttft[ord] = Rj - A.arrival[ord];
-        if (A.completion) A.completion[ord] = Rj;
+    long long run = bsum[blockIdx.x] + x - mine;            // time at which this thread's first decision starts
+    for (int w = 0; w < warp; ++w) run += s_w[w];
+    for (int32_t u = 0; u < ipt; ++u) {
+        const long long i = i0 + u, c = A.post->c0 + i;
+        if (c < A.n) {
+            const int32_t ord = A.order[c];
+            run += cost[i];
+            A.ttft[ord] = run - A.arrival[ord];
+            if (A.completion) A.completion[ord] = run;
+        }
     }
 }
 
@@ -3715,7 +3762,7 @@ rt_status ensure_fast_scratch(rt_tree* t, long long n) {
     if ((s = dalloc(&t->fast_mem, t->fast_mem_cap))) return s;
     if ((s = dalloc(&t->fast_gh, np2))) return s;
     if ((s = dalloc(&t->fast_gidx, np2))) return s;
-    if ((s = dalloc(&t->fast_done, 2 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap
+    if ((s = dalloc(&t->fast_done, 3 * (np2 / 32 + 32)))) return s;     // processed bitmap, grouped bitmap, passed-over bitmap
     if ((s = dalloc(&t->fast_lk, np2))) return s;
     if ((s = dalloc(&t->fast_ls, np2))) return s;
     if (!t->fast_post && (s = dalloc(&t->fast_post, 1))) return s;
@@ -4295,12 +4342,14 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         size_t smem = (size_t)(nb1p + n2p + 32) * 8 + (size_t)KLPM_FAST_SORT_CAP * 12;
         f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
-        // list mode needs two more bitmaps in shared memory and 32-slot leaf blocks
-        f.list_mode = (!lru && f.done_in_smem && lbs == 5 && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
-        if (f.list_mode) smem += (size_t)nwords * 8;
+        // list mode (trees without a budget) needs two more bitmaps: in shared memory while they fit, in global memory beyond
+        f.list_mode = lru ? 0 : 1;
+        f.bits_in_smem = (f.list_mode && f.done_in_smem && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
+        if (f.bits_in_smem) smem += (size_t)nwords * 8;
         f.gbits = tree->fast_done + (np2 / 32 + 32);
+        f.gskip = tree->fast_done + 2 * (np2 / 32 + 32);
         const unsigned nblk = (unsigned)((n + 255) / 256), pblk = (unsigned)((np2 + 255) / 256);
-        CK(cudaMemsetAsync(f.done, 0, (size_t)(2 * (np2 / 32 + 32)) * sizeof(unsigned int), s));
+        CK(cudaMemsetAsync(f.done, 0, (size_t)(3 * (np2 / 32 + 32)) * sizeof(unsigned int), s));
         // groups: queries whose match ends at the same position and continues with the same token
         sort_pairs(f.gh, f.gidx, np2, s);
         fast_group_kernel<<<nblk, 256, 0, s>>>(f);
@@ -4314,13 +4363,20 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
             sort_pairs(tree->fast_lk, tree->fast_ls, np2, s);
         }
         CK(cudaGetLastError());
-        CK(cudaFuncSetAttribute(fast_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        fast_run_kernel<<<1, KLPM_FAST_THREADS, smem, s>>>(f);
+        if (f.done_in_smem && (f.bits_in_smem || !f.list_mode)) {
+            CK(cudaFuncSetAttribute(fast_run_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            fast_run_kernel<false><<<1, KLPM_FAST_THREADS, smem, s>>>(f);
+        } else {
+            CK(cudaFuncSetAttribute(fast_run_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            fast_run_kernel<true><<<1, KLPM_FAST_THREADS, smem, s>>>(f);
+        }
         if (f.list_mode) {           // the decisions made in list mode are charged here (none if list mode never began)
-            const int32_t cblocks = (n + KLPM_CHARGE_THREADS - 1) / KLPM_CHARGE_THREADS;      // at most 1,024: list mode ends at 262,144 queries
-            charge_cost_kernel<<<cblocks, KLPM_CHARGE_THREADS, 0, s>>>(f, tree->fast_gh, tree->fast_bsum);
+            const int32_t ipt = (int32_t)(((long long)n + 1024LL * KLPM_CHARGE_THREADS - 1) / (1024LL * KLPM_CHARGE_THREADS));
+            const int32_t per_block = KLPM_CHARGE_THREADS * ipt;
+            const int32_t cblocks = (n + per_block - 1) / per_block;                          // at most 1,024
+            charge_cost_kernel<<<cblocks, KLPM_CHARGE_THREADS, 0, s>>>(f, tree->fast_gh, tree->fast_bsum, ipt);
             charge_scan_kernel<<<1, 1024, 0, s>>>(f, tree->fast_bsum, cblocks);
-            charge_apply_kernel<<<cblocks, KLPM_CHARGE_THREADS, 0, s>>>(f, tree->fast_gh, tree->fast_bsum);
+            charge_apply_kernel<<<cblocks, KLPM_CHARGE_THREADS, 0, s>>>(f, tree->fast_gh, tree->fast_bsum, ipt);
         }
         CK(cudaGetLastError());
         tree->run_path = 2;

@@ -190,16 +190,19 @@ def test_both_loops_agree(K, name, scale, k):
     same(a, b)
 
 
-@pytest.mark.parametrize("max_blocks,smem_kb", [(16, 0), (4, 60), (1, 0)])
-def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb):
-    """Queues above 262,144 use larger tournament leaf blocks, and far larger ones keep the processed bitmap in
-    global memory; neither uses list mode.  Shrinking the limits makes a 3,000-query stream take those paths."""
+@pytest.mark.parametrize("max_blocks,smem_kb,n,max_gap", [(16, 0, 3000, 2), (4, 60, 3000, 2), (1, 0, 3000, 2), (4, 49, 3000, 0),
+                                                         (16, 52, 20000, 0), (64, 49, 20000, 1)])
+def test_large_queue_layout_on_a_small_queue(K, max_blocks, smem_kb, n, max_gap):
+    """Queues above 262,144 use larger tournament leaf blocks and keep the two extra bitmaps of list mode -- far
+    larger ones the processed bitmap too -- in global memory.  Shrinking the limits makes small streams take those
+    paths: 64 to 4,096 slots per leaf block; every bitmap in shared memory, only the processed one, or none; with
+    everybody waiting from the start (list mode throughout) and with arrivals over time."""
     K.klpm_debug_set("fast_max_blocks", max_blocks)
     K.klpm_debug_set("fast_smem_kb", smem_kb)
     try:
-        prompts, arr = shared_prefix_queue(31, 3000, [(12, 3), (9, 4)], tail=9, vocab=5, max_gap=2)
+        prompts, arr = shared_prefix_queue(31, n, [(12, 3), (9, 4)], tail=9, vocab=5, max_gap=max_gap)
         prefill, _ = shared_prefix_queue(32, 200, [(12, 3), (9, 4)], tail=4, vocab=5, max_gap=0)
-        for policy, k in ((2, 4), (0, 1)):
+        for policy, k in ((2, 4), (0, 1), (1, 1)):
             got = run_gpu(K, prefill, prompts, arr, policy, k)
             want = run_oracle(prefill, prompts, arr, policy, k)
             same(got, want)
@@ -281,3 +284,49 @@ def test_match_records_are_refused_once_they_are_stale(K):
     K.klpm_run_ex(tree, d_qt, d_qo, d_arr, p, None, 0, *out, None, state)
     assert K.rt_sync_status(tree) == K.RT_ERR_INVALID and K.rt_status_detail(tree) == 110
     K.rt_destroy(tree)
+
+
+def test_queue_above_the_shared_memory_bitmaps(K):
+    """300,000 queries, everybody waiting: list mode with 64-slot leaf blocks and two of its bitmaps in global memory.
+    The oracle's O(n^2) schedule is out of reach at this size, so the loop is compared bit for bit with the
+    one-decision-at-a-time loop (which the oracle checks at the smaller sizes) and through what holds at any size."""
+    n = 300_000
+    rng = np.random.RandomState(5)
+    heads = rng.randint(0, 50000, size=(64, 24))
+    which = rng.randint(0, 64, size=n)
+    cut = rng.randint(1, 25, size=n)
+    tails = rng.randint(0, 50000, size=(n, 6))
+    lens = cut + rng.randint(1, 7, size=n)
+    off = np.zeros(n + 1, dtype=np.int64)
+    off[1:] = np.cumsum(lens)
+    tok = np.empty(off[-1], dtype=np.int32)
+    for i in range(n):
+        tok[off[i]:off[i] + cut[i]] = heads[which[i], :cut[i]]
+        tok[off[i] + cut[i]:off[i + 1]] = tails[i, :lens[i] - cut[i]]
+    arr = np.sort(rng.randint(0, 1000, size=n)).astype(np.int64)
+    d_tok, d_off, d_arr = torch.from_numpy(tok).cuda(), torch.from_numpy(off).cuda(), torch.from_numpy(arr).cuda()
+    outs = []
+    for legacy in (False, True):
+        tree = K.rt_create(max_nodes=2 * n + 64, max_pool_tokens=int(off[-1]) + 8 * n + 64, max_clock=n + 64)
+        order = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+        K.klpm_debug_set("run_one_by_one", 1 if legacy else 0)
+        try:
+            K.klpm_run(tree, d_tok, d_off, d_arr, K.make_params(K.POLICY_KLPM, 3, 0, 1, 1000), order, unc, ttft)
+            assert K.rt_sync_status(tree) == 0
+        finally:
+            K.klpm_debug_set("run_one_by_one", -1)
+        assert K.klpm_run_path(tree) == (K.RUN_PATH_ONE_BY_ONE if legacy else K.RUN_PATH_GROUPED)
+        if not legacy:
+            cn = K.rt_debug_counters(tree)
+            assert cn["cta_batch_decisions"] + cn["warp_step_decisions"] + cn["single_decisions"] > n // 2      # list mode ran
+        st = K.rt_stats(tree)
+        outs.append((order.cpu().numpy(), unc.cpu().numpy(), ttft.cpu().numpy(), st))
+        K.rt_destroy(tree)
+    for a, b in zip(outs[0][:3], outs[1][:3]):
+        assert np.array_equal(a, b)
+    assert {f: outs[0][3][f] for f in ("n_nodes", "tokens", "clock")} == {f: outs[1][3][f] for f in ("n_nodes", "tokens", "clock")}
+    order, unc = outs[0][0].astype(np.int64), outs[0][1].astype(np.int64)
+    assert np.array_equal(np.sort(order), np.arange(n))
+    assert int(unc.sum()) == outs[0][3]["tokens"]
