@@ -1720,6 +1720,7 @@ struct FastBatchIO {
     unsigned long long root;          // in: largest key in the tournament
     int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
     int32_t B0, nF0, nL0, limF, limL; // scratch
+    int32_t limB;                     // scratch: the batch must end before this decision (list entries that an oldest-first pick would meet)
 };
 #define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
 #ifndef KLPM_FAST_CTA_MIN
@@ -1821,12 +1822,12 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         int32_t lo = 0, hi = n - c < KLPM_FAST_CTA_BATCH ? n - c : KLPM_FAST_CTA_BATCH;
         while (lo < hi) { const int32_t mid = (lo + hi + 1) >> 1; if (mid - f(mid) <= avail) lo = mid; else hi = mid - 1; }
         io->B0 = lo; io->nF0 = f(lo); io->nL0 = lo - f(lo);
-        io->limF = io->nF0; io->limL = io->nL0;
+        io->limF = io->nF0; io->limL = io->nL0; io->limB = lo;
     }
     __syncthreads();
     const int32_t B0 = io->B0, nF0 = io->nF0, nL0 = io->nL0;
     // the next nF0 unprocessed slots (each thread one bitmap word from head on), in order
-    int32_t hmax0 = -1;
+    int32_t hmax0 = -1, nFa0 = 0;
     if (nF0 > 0) {
         const int32_t w0 = head >> 5, wi = w0 + tid;
         unsigned w = wi < nwords ? bm_ld(R.done, wi, R.g_done) : 0xffffffffu;
@@ -1840,13 +1841,16 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         if (tid == 0 && nFa < nF0) io->limF = nFa;
         __syncthreads();
         if (nFa > 0) hmax0 = sH[nFa - 1];
+        nFa0 = nFa;
         for (int32_t qi = tid; qi < nFa; qi += KLPM_FAST_THREADS) {       // key in the tournament, or grouped: needs the careful step
             const int32_t hs = sH[qi];
             if (((bm_ld(R.skip, hs >> 5, R.g_bits) | bm_ld(R.gb, hs >> 5, R.g_bits)) >> (hs & 31)) & 1u) atomicMin(&io->limF, qi);
         }
     }
-    // the usable entries by rank; the first one that is grouped, could also be an oldest-first pick of this batch, or
-    // lies below the tournament's root limits the batch
+    // The usable entries by rank.  One that is grouped or lies below the tournament's root stops the batch before its
+    // turn.  One whose slot is among the slots the oldest-first picks of a full batch would take (rank phi there) is
+    // taken by whichever side reaches it first, and the other side must not get as far as it inside this batch: the
+    // batch ends before the later of the two decisions (its own longest-match turn, the oldest-first turn of rank phi).
     {
         int32_t rk = base;
 #pragma unroll
@@ -1855,7 +1859,25 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
                 if (rk < nL0) {
                     sE[rk] = es[r]; sEpos[rk] = tid * 4 + r;
                     const unsigned long long ek = ~((unsigned long long)kk[r] ^ 0x8000000000000000ULL);
-                    if ((((bm_ld(R.gb, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u)) || (es[r] >= head && es[r] <= hmax0) || root > ek) atomicMin(&io->limL, rk);
+                    if ((((bm_ld(R.gb, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u)) || root > ek) {
+                        atomicMin(&io->limL, rk);
+                    } else if (es[r] >= head && es[r] <= hmax0) {
+                        int32_t lo = 0, hi = nFa0;                       // phi: slots of sH before this one
+                        while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sH[mid] < es[r]) lo = mid + 1; else hi = mid; }
+                        const int32_t phi = lo;
+                        // decision of the oldest-first turn of rank phi, and of the longest-match turn of rank rk
+                        int32_t xF, xL;
+                        if (A.policy == KLPM_POLICY_FCFS) { xF = phi; xL = B0; }
+                        else if (A.policy == KLPM_POLICY_LPM) { xF = B0; xL = rk; }
+                        else {
+                            const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;
+                            xF = i0 + phi * A.k;
+                            int32_t a0 = 0, a1 = B0;                     // smallest x with x + 1 - f(x + 1) > rk
+                            while (a0 < a1) { const int32_t mid = (a0 + a1) >> 1; if (mid + 1 - f(mid + 1) > rk) a1 = mid; else a0 = mid + 1; }
+                            xL = a0;
+                        }
+                        atomicMin(&io->limB, xF > xL ? xF : xL);
+                    }
                 }
                 ++rk;
             }
@@ -1866,6 +1888,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         const int32_t limF = io->limF, limL = io->limL;
         int32_t lo = 0, hi = B0;
         while (lo < hi) { const int32_t mid = (lo + hi + 1) >> 1; if (f(mid) <= limF && mid - f(mid) <= limL) lo = mid; else hi = mid - 1; }
+        if (io->limB < lo) lo = io->limB;
         const int32_t B = lo >= KLPM_FAST_CTA_MIN ? lo : 0;
         const int32_t nF = f(B), nL = B - nF;
         io->B = B;
@@ -2764,13 +2787,25 @@ fast_run_kernel(FastArgs A) {
             const bool ok = (mask >> lane) & 1u;
             const int32_t rank = __popc(mask & ((1u << lane) - 1u));
             int32_t limL = nL0;
+            int32_t soft = -1;                              // slot of the entry that stops the batch, if it is only suspected of being an oldest-first pick too
             {
                 const unsigned long long ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL);
-                const unsigned badE = __ballot_sync(FULL_MASK, ok && rank < nL0 &&
-                                                    ((((bm_ld(R.gb, es >> 5, gbits) >> (es & 31)) & 1u)) || (es >= head && es <= hmax0) || root > ek));
-                if (badE) limL = __popc(mask & ((1u << (__ffs(badE) - 1)) - 1u));
+                const bool hard = (((bm_ld(R.gb, es >> 5, gbits) >> (es & 31)) & 1u)) || root > ek;
+                const unsigned badE = __ballot_sync(FULL_MASK, ok && rank < nL0 && (hard || (es >= head && es <= hmax0)));
+                if (badE) {
+                    const int src = __ffs(badE) - 1;
+                    limL = __popc(mask & ((1u << src) - 1u));
+                    if (!__shfl_sync(FULL_MASK, (int)hard, src)) soft = __shfl_sync(FULL_MASK, es, src);
+                }
             }
-            const int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_hi <= limF && (lane + 1) - f_hi <= limL));
+            int32_t B = __popc(__ballot_sync(FULL_MASK, lane < B0 && f_hi <= limF && (lane + 1) - f_hi <= limL));
+            if (soft >= 0 && B < B0 && B < 32) {
+                // the decision after the batch (lane B's): if it is the longest-match turn that takes that entry and the
+                // oldest-first picks made until then all lie before its slot, it becomes the batch's last decision
+                const int32_t fl = __shfl_sync(FULL_MASK, f_lo, B), fh = __shfl_sync(FULL_MASK, f_hi, B);
+                const int32_t last_h = __shfl_sync(FULL_MASK, hs, fl > 0 ? fl - 1 : 0);
+                if (fh == fl && B - fl == limL && fl <= limF && (fl == 0 || last_h < soft)) { ++B; ++limL; }
+            }
             if (B < 2) return false;
             const int32_t nF = __shfl_sync(FULL_MASK, f_hi, B - 1), nL = B - nF;
             const int32_t hmax = nF > 0 ? __shfl_sync(FULL_MASK, hs, nF - 1) : -1;
@@ -2817,7 +2852,8 @@ fast_run_kernel(FastArgs A) {
                 named_bar(1, KLPM_FAST_THREADS);
                 fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords);
                 const int32_t Bc = s_bio.B;
-                cy_cta += clock64() - t_cta;
+                const long long cy_this = clock64() - t_cta;
+                cy_cta += cy_this;
                 if (Bc > 0) {
                     ++n_cta_ok; dec_cta += Bc;
                     const int32_t consumed = s_bio.consumed, hmax = s_bio.hmax;
@@ -2826,7 +2862,13 @@ fast_run_kernel(FastArgs A) {
                     if (consumed) { cur += consumed; window(cur & ~31, &wk, &ws); window((cur & ~31) + 32, &nk, &ns); }
                     if (hmax >= 0) { head = hmax; advance_head(); }
                     else if (head < n && ((bm_ld(s_done, head >> 5, gdone) >> (head & 31)) & 1u)) advance_head();
-                    cb_back = 8;
+                    // did it pay?  its cycles per decision against what the warp-wide steps have cost per decision so far
+                    const long long warp_cpd = dec_warp >= 256 ? cy_warp / dec_warp : 100;
+                    if (cy_this <= (long long)Bc * warp_cpd) { cb_back = 8; continue; }
+                    // committed, but too short to have paid for the attempt: warp-wide steps for a while, as after a failure
+                    cb_wait = cb_back;
+                    cb_back = cb_back < KLPM_FAST_CB_MAX ? cb_back * 2 : KLPM_FAST_CB_MAX;
+                    calm = 0;
                     continue;
                 }
                 cb_wait = cb_back;
