@@ -203,9 +203,13 @@ rt_status klpm_select_noalloc(const int32_t* d_match_len, const int64_t* d_arriv
  *   R_j = max(R_prev, t_j) + (c_den + c_num |x_j|) * uncached;  TTFT_j = R_j - t_j;
  * then x_j is stored in the tree (as rt_insert does).  Outputs are indexed by query: d_uncached
  * (int32[n_queries]), d_ttft (int64[n_queries]), d_completion (nullable, int64[n_queries]); entries of
- * queries that are not in d_order are left untouched.  An entry of d_order outside [0, n_queries) stops the
- * replay there: nothing of it is read or written, the queries before it stay processed, and the status word
- * reports RT_ERR_INVALID. */
+ * queries that are not in d_order are left untouched.  A query may appear in d_order once.  An entry outside
+ * [0, n_queries), or one that names a query for the second time, stops the replay there: nothing of it is read or
+ * written, the queries before it stay processed, and the status word reports RT_ERR_INVALID (detail 108).
+ * The replay runs through the same device loop as klpm_run, with the order given instead of picked: every query
+ * is matched once, a processed prompt re-matches only the queries tied with it, and the tree is written at the
+ * end (what klpm_run says about capacity holds here too).  The debug setting "run_one_by_one" selects the plain
+ * form instead: one CTA that walks, charges and stores one prompt after the other. */
 rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, const int32_t* d_q_tokens,
                       const int64_t* d_q_offsets, const int64_t* d_arrival, int32_t n_queries,
                       const klpm_params* params, int32_t* d_uncached, int64_t* d_ttft,

@@ -1448,6 +1448,10 @@ struct FastArgs {
     int2* leaf_run;               // per node: the member run that holds every slot whose hint is that node (y < 0: no such run is known)
     long long* pk; int32_t* pi;   // set-up: (hint, slot) pairs, sorted by hint to give every node of the tree its run
     int32_t* skip;                // set by the capacity check before the loop: leave everything untouched
+    // a given processing order instead of a policy (klpm_replay): decision c processes query fixed[c]; slots are the
+    // queries in index order; *n_fixed decisions are made
+    const int32_t* fixed;
+    const int32_t* n_fixed;
 };
 
 #define KLPM_FAST_THREADS 256
@@ -2324,7 +2328,8 @@ fast_run_kernel(FastArgs A) {
             const long long Rj = begin + (A.c_den + A.c_num * (long long)len) * (long long)unc;
             now = Rj;
             if (lane == 0) {
-                A.order[c] = s.ord; A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
+                if (A.order) A.order[c] = s.ord;
+                A.uncached[s.ord] = unc; A.ttft[s.ord] = Rj - s.t;
                 if (A.completion) A.completion[s.ord] = Rj;
             }
         } else if (lane == 0) {
@@ -2610,6 +2615,20 @@ fast_run_kernel(FastArgs A) {
             }
         }
     };
+
+    // ================================================================ a given order (klpm_replay): no admission, no pick
+    if (A.fixed) {
+        const int32_t nfix = *reinterpret_cast<const volatile int32_t*>(A.n_fixed);
+        while (c < nfix && !failed) {
+            const int32_t slot = __ldg(A.fixed + c);        // slots are the queries in index order here
+            const FDyn pd = ld_dyn(A.dyn + slot);
+            const FStat ps = ld_stat(A.stat + slot);
+            mark_done(slot);
+            careful(slot, true, pd, ps);                     // (head stays 0 and nobody is admitted: scans cover every slot)
+            __syncwarp();
+        }
+        c = n;                                               // nothing is left for the policy loops below
+    }
 
     // everybody is waiting as the loop starts: no arrival will ever have to be admitted
     if (A.list_mode && __ldg(&A.stat[n - 1].t) <= now) { admitted = n; next_t = INF; }
@@ -3087,6 +3106,7 @@ bulk_from_state_kernel(TreeDev T, BulkArgs A, const MatchState* __restrict__ sta
     const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
     for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
         const int32_t i = A.pend_in[p];
+        if (i < 0) continue;                                // a replay that stopped early: not processed
         const int32_t len = (int32_t)(__ldg(A.off + i + 1) - __ldg(A.off + i));
         const int4* src = reinterpret_cast<const int4*>(state + i);
         const int4 a = __ldcg(src), b = __ldcg(src + 1);
@@ -3279,7 +3299,7 @@ __device__ bool bulk_barrier(BulkSync* g, TreeState* st, long long limit_ns, F l
 }
 
 __global__ void __launch_bounds__(256)
-bulk_rounds_kernel(TreeDev T, BulkArgs A, BulkSync* g, long long n_total, long long limit_ns) {
+bulk_rounds_kernel(TreeDev T, BulkArgs A, BulkSync* g, long long n_total, const int32_t* n_total_dev, long long limit_ns) {
     __shared__ unsigned long long s_live_nodes, s_live_tokens;
     if (threadIdx.x == 0) { s_live_nodes = 0ULL; s_live_tokens = 0ULL; }
     __syncthreads();
@@ -3330,6 +3350,7 @@ bulk_rounds_kernel(TreeDev T, BulkArgs A, BulkSync* g, long long n_total, long l
         if (s_live_nodes) atomicAdd((unsigned long long*)&S->live_nodes, s_live_nodes);
         if (s_live_tokens) atomicAdd((unsigned long long*)&S->tokens_live, s_live_tokens);
         if (blockIdx.x == 0) {                              // the logical clock advances by one per stored prompt
+            if (n_total_dev) n_total = *n_total_dev;
             if (S->clock + n_total + 1 >= T.max_clock) set_status(S, RT_ERR_CAPACITY);
             else S->clock += n_total;
         }
@@ -3591,6 +3612,42 @@ __global__ void batch_times_kernel(const int32_t* __restrict__ order, int32_t n,
     ttft_b[j] = R - __ldg(arrival + j);
 }
 
+// klpm_replay through the grouped loop.  The order is checked first: the decisions that will be made are the entries
+// before the first one that is not a query or names a query for the second time (the status word says so if there is
+// one).  Slots are the queries in index order.
+struct ReplayInfo { int32_t n_valid; int32_t pad; };
+__global__ void replay_first_kernel(const int32_t* __restrict__ order, int32_t n_order, int32_t n_queries, int32_t* first_pos) {
+    const int32_t p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n_order) return;
+    const int32_t j = order[p];
+    if (j >= 0 && j < n_queries) atomicMin(first_pos + j, p);
+}
+__global__ void replay_check_kernel(const int32_t* __restrict__ order, int32_t n_order, int32_t n_queries, const int64_t* __restrict__ off,
+                                    const int32_t* __restrict__ first_pos, ReplayInfo* info, TreeState* st) {
+    const int32_t p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n_order) return;
+    const int32_t j = order[p];
+    bool bad = j < 0 || j >= n_queries;
+    if (!bad) { const int64_t len = off[j + 1] - off[j]; bad = len < 0 || len > 0x7fffffffLL || first_pos[j] < p; }
+    if (bad) { atomicMin(&info->n_valid, p); set_status(st, RT_ERR_INVALID, 108); }
+}
+__global__ void replay_slots_kernel(const int64_t* __restrict__ arrival, int32_t n, long long* sorted_t, int32_t* ord) {
+    const int32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { sorted_t[i] = arrival[i]; ord[i] = i; }
+}
+// the prompts a replay has processed, as the list the insertion after the loop works through (-1: not processed)
+__global__ void replay_list_kernel(const int32_t* __restrict__ order, int32_t n_order, const ReplayInfo* info, int32_t* pend) {
+    const int32_t p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < n_order) pend[p] = p < info->n_valid ? order[p] : -1;
+}
+__global__ void lru_sum_order_kernel(const int64_t* __restrict__ off, const int32_t* __restrict__ order, int32_t n_order,
+                                     int32_t n_queries, LruInfo* info) {
+    const int32_t p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n_order) return;
+    const int32_t j = order[p];
+    if (j >= 0 && j < n_queries) { const int64_t len = off[j + 1] - off[j]; if (len > 0) atomicAdd(&info->total_len, (unsigned long long)len); }
+}
+
 // slot order: bitonic sort of (arrival, index) pairs, padded to a power of two
 __global__ void rank_init_kernel(const int64_t* __restrict__ arrival, int32_t n, long long np2, long long* key, int32_t* idx) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -3706,6 +3763,7 @@ struct rt_tree {
     int32_t* lru_parked; LruInfo* lru_info;     // grouped loop on a tree with a budget
     int32_t* lru_hintc; long long lru_hintc_cap;
     int2* lru_leaf_run;
+    ReplayInfo* replay_info;
     int run_path;           // which loop the last klpm_run took: 0 none yet, 1 one by one, 2 grouped
     int num_sms;
     int32_t* claim;         // bulk insertion: per-node claim words (0x7fffffff when idle)
@@ -3747,7 +3805,7 @@ void free_tree(rt_tree* t) {
     cudaFree(t->fast_dyn); cudaFree(t->fast_stat); cudaFree(t->fast_key_arr); cudaFree(t->fast_mem);
     cudaFree(t->fast_gh); cudaFree(t->fast_gidx); cudaFree(t->fast_done); cudaFree(t->fast_counter);
     cudaFree(t->fast_lk); cudaFree(t->fast_ls); cudaFree(t->fast_post); cudaFree(t->fast_bsum);
-    cudaFree(t->lru_parked); cudaFree(t->lru_info); cudaFree(t->lru_hintc); cudaFree(t->lru_leaf_run);
+    cudaFree(t->lru_parked); cudaFree(t->lru_info); cudaFree(t->lru_hintc); cudaFree(t->lru_leaf_run); cudaFree(t->replay_info);
     cudaFree(t->claim);
     cudaFree(t->bulk_pend_a); cudaFree(t->bulk_pend_b); cudaFree(t->bulk_pm); cudaFree(t->bulk_pnode); cudaFree(t->bulk_poff);
     cudaFree(t->bulk_sync);
@@ -3847,14 +3905,16 @@ rt_status ensure_bulk_scratch(rt_tree* t, int32_t n) {
 
 // `state` (nullable): records of a batched match of these prompts against the tree as it is now; the first round
 // then needs no walk.  Everything is enqueued on `s`; nothing waits for the device.
+// `list_ready`: bulk_pend_a already holds the n prompts to store (entries < 0 are skipped) and *n_total_dev how many they are.
 rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offsets, int32_t n, cudaStream_t s,
-                      const MatchState* state = nullptr, unsigned long long tag = 0) {
+                      const MatchState* state = nullptr, unsigned long long tag = 0, bool list_ready = false,
+                      const int32_t* n_total_dev = nullptr) {
     rt_status st = ensure_bulk_scratch(t, n);
     if (st) return st;
     BulkSync* g = t->bulk_sync;
     // claim words start idle (an earlier call that ran out of capacity may have left some set)
     bulk_fill_kernel<<<(unsigned)((t->dev.max_nodes + 255) / 256), 256, 0, s>>>(t->claim, t->dev.max_nodes, 0x7fffffff);
-    bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(t->bulk_pend_a, n);
+    if (!list_ready) bulk_iota_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(t->bulk_pend_a, n);
     CK(cudaMemsetAsync(g, 0, sizeof(BulkSync), s));
     BulkArgs a;
     a.tok = d_tokens; a.off = d_offsets; a.pend_in = t->bulk_pend_a; a.pend_out = t->bulk_pend_b; a.n_out = &g->cnt_w[0];
@@ -3873,7 +3933,7 @@ rt_status bulk_insert(rt_tree* t, const int32_t* d_tokens, const int64_t* d_offs
     if (per_sm < 1) return RT_ERR_CUDA;
     const unsigned grid = (unsigned)t->num_sms * (unsigned)(per_sm < 2 ? per_sm : 2);
     long long n_total = n, limit = g_knobs.wait_limit_ns;
-    void* kargs[] = {(void*)&t->dev, (void*)&a, (void*)&g, (void*)&n_total, (void*)&limit};
+    void* kargs[] = {(void*)&t->dev, (void*)&a, (void*)&g, (void*)&n_total, (void*)&n_total_dev, (void*)&limit};
     CK(cudaLaunchCooperativeKernel((void*)bulk_rounds_kernel, dim3(grid), dim3(256), kargs, 0, s));
     return RT_OK;
 }
@@ -4244,12 +4304,23 @@ rt_status klpm_select_noalloc(const int32_t* d_match_len, const int64_t* d_arriv
     return RT_OK;
 }
 
+static rt_status run_impl(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
+                          int32_t n, const klpm_params* params, const int64_t* d_tie_priority, int32_t score_mode,
+                          const klpm_match_state* d_match_state, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                          int64_t* d_completion, const int32_t* d_fixed, int32_t n_fixed, void* stream);
+
 rt_status klpm_replay(rt_tree* tree, const int32_t* d_order, int32_t n_order, const int32_t* d_q_tokens,
                       const int64_t* d_q_offsets, const int64_t* d_arrival, int32_t n_queries, const klpm_params* params,
                       int32_t* d_uncached, int64_t* d_ttft, int64_t* d_completion, void* stream) {
     if (!tree || !params_ok(params) || n_order < 0 || n_queries < 0 ||
         (n_order > 0 && (!d_order || !d_q_tokens || !d_q_offsets || !d_arrival || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
     if (n_order == 0) return RT_OK;
+    // The same loop as klpm_run with the order given instead of picked (every query's match state is kept, a processed
+    // prompt re-matches its group only, the tree is written once at the end).  The debug setting run_one_by_one keeps
+    // the plain form: one CTA that walks, charges and stores one prompt after the other on the tree itself.
+    if (!g_knobs.run_one_by_one && n_queries > 0)
+        return run_impl(tree, d_q_tokens, d_q_offsets, d_arrival, n_queries, params, nullptr, 0, nullptr, nullptr, d_uncached, d_ttft,
+                        d_completion, d_order, n_order, stream);
     tree->version++;
     SeqArgs a;
     memset(&a, 0, sizeof(a));
@@ -4276,12 +4347,14 @@ rt_status klpm_batch_times(const int32_t* d_order, int32_t n_order, const int64_
     return RT_OK;
 }
 
-rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
-                      int32_t n, const klpm_params* params, const int64_t* d_tie_priority, int32_t score_mode,
-                      const klpm_match_state* d_match_state, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
-                      int64_t* d_completion, void* stream) {
+// klpm_run_ex, and klpm_replay when d_fixed (a processing order of n_fixed entries) is given: then d_order is null,
+// no decision is taken by a policy, and only the prompts of the order are charged and stored.
+static rt_status run_impl(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
+                          int32_t n, const klpm_params* params, const int64_t* d_tie_priority, int32_t score_mode,
+                          const klpm_match_state* d_match_state, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                          int64_t* d_completion, const int32_t* d_fixed, int32_t n_fixed, void* stream) {
     if (!tree || !params_ok(params) || n < 0 || score_mode < 0 || score_mode > 1 ||
-        (n > 0 && (!d_q_tokens || !d_q_offsets || !d_arrival || !d_order || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
+        (n > 0 && (!d_q_tokens || !d_q_offsets || !d_arrival || (!d_order && !d_fixed) || !d_uncached || !d_ttft))) return RT_ERR_INVALID;
     if (n == 0) return RT_OK;
     // records of a batched match are only good for the queries they were written for and the tree as it was then
     if (d_match_state && (tree->ms_state != (const void*)d_match_state || tree->ms_n != n || tree->ms_tok != (const void*)d_q_tokens ||
@@ -4296,8 +4369,11 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
     // A tree without a budget takes the grouped loop (unless the debug setting run_one_by_one is on).
     const bool grouped = !g_knobs.run_one_by_one;
     const bool lru = tree->cfg.budget_tokens > 0;
-    // slots = queries ordered by (arrival, index)
-    {
+    // slots = queries ordered by (arrival, index); for a given order, the queries in index order
+    if (d_fixed) {
+        replay_slots_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(d_arrival, n, tree->run_key, tree->run_ord);
+        CK(cudaGetLastError());
+    } else {
         unsigned blocks = (unsigned)((np2 + 255) / 256);
         rank_init_kernel<<<blocks, 256, 0, s>>>(d_arrival, n, np2, tree->run_key, tree->run_ord);
         sort_pairs(tree->run_key, tree->run_ord, np2, s);
@@ -4315,8 +4391,18 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         memset(&f, 0, sizeof(f));
         st = ensure_fast_scratch(tree, n);
         if (st) return st;
-        st = ensure_bulk_scratch(tree, n);
+        st = ensure_bulk_scratch(tree, d_fixed && n_fixed > n ? n_fixed : n);
         if (st) return st;
+        if (d_fixed) {
+            // which entries of the order will be processed: those before the first that is not a query or comes twice
+            if (!tree->replay_info && (st = dalloc(&tree->replay_info, 1))) return st;
+            const unsigned fb = (unsigned)((n_fixed + 255) / 256);
+            bulk_fill_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(tree->bulk_pm, n, 0x7fffffff);
+            bulk_fill_kernel<<<1, 1, 0, s>>>(&tree->replay_info->n_valid, 1, n_fixed);
+            replay_first_kernel<<<fb, 256, 0, s>>>(d_fixed, n_fixed, n, tree->bulk_pm);
+            replay_check_kernel<<<fb, 256, 0, s>>>(d_fixed, n_fixed, n, d_q_offsets, tree->bulk_pm, tree->replay_info, tree->dev.st);
+            f.fixed = d_fixed; f.n_fixed = &tree->replay_info->n_valid;
+        }
         if (lru) {
             if (!tree->lru_parked && (st = dalloc(&tree->lru_parked, tree->dev.max_nodes))) return st;
             if (!tree->lru_info && (st = dalloc(&tree->lru_info, 1))) return st;
@@ -4336,8 +4422,9 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
             // all or nothing: is there room for whatever the loop can leave behind?
             CK(cudaMemsetAsync(tree->lru_info, 0, sizeof(LruInfo), s));
             CK(cudaMemsetAsync(tree->lru_parked, 0, (size_t)tree->dev.max_nodes * sizeof(int32_t), s));
-            lru_sum_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(d_q_offsets, n, tree->lru_info);
-            lru_check_kernel<<<1, 1, 0, s>>>(tree->dev, n, tree->lru_info);
+            if (d_fixed) lru_sum_order_kernel<<<(unsigned)((n_fixed + 255) / 256), 256, 0, s>>>(d_q_offsets, d_fixed, n_fixed, n, tree->lru_info);
+            else lru_sum_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(d_q_offsets, n, tree->lru_info);
+            lru_check_kernel<<<1, 1, 0, s>>>(tree->dev, d_fixed ? n_fixed : n, tree->lru_info);
         }
         f.tok = d_q_tokens; f.n = n; f.policy = params->policy; f.k = params->k; f.score_mode = score_mode;
         f.c_num = params->c_num; f.c_den = params->c_den; f.start_tick = params->start_tick;
@@ -4385,7 +4472,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         f.done_in_smem = smem + (size_t)nwords * 4 <= smem_max ? 1 : 0;
         if (f.done_in_smem) smem += (size_t)nwords * 4;
         // list mode (trees without a budget) needs two more bitmaps: in shared memory while they fit, in global memory beyond
-        f.list_mode = lru ? 0 : 1;
+        f.list_mode = (lru || d_fixed) ? 0 : 1;
         f.bits_in_smem = (f.list_mode && f.done_in_smem && smem + (size_t)nwords * 8 <= smem_max) ? 1 : 0;
         if (f.bits_in_smem) smem += (size_t)nwords * 8;
         f.gbits = tree->fast_done + (np2 / 32 + 32);
@@ -4425,7 +4512,7 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         if (lru) {
             // the nodes that are alive after the loop get their tokens, and the child table is written afresh
             const TreeDev& d = tree->dev;
-            lru_tokens_kernel<<<(unsigned)tree->num_sms * 8, 256, 0, s>>>(d, d_order, d_q_tokens, d_q_offsets, f.vbase, tree->lru_info);
+            lru_tokens_kernel<<<(unsigned)tree->num_sms * 8, 256, 0, s>>>(d, d_fixed ? d_fixed : d_order, d_q_tokens, d_q_offsets, f.vbase, tree->lru_info);
             table_clear_kernel<<<(unsigned)tree->num_sms * 8, 256, 0, s>>>(d, tree->lru_info);
             lru_table_kernel<<<(unsigned)((d.max_nodes + 255) / 256), 256, 0, s>>>(d, f.vbase, tree->lru_info);
             CK(cudaGetLastError());
@@ -4433,8 +4520,13 @@ rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d
         }
         // The processed prompts enter the tree together (the logical clock advances by n).  The loop itself needs
         // no room in the tree; if the tree cannot hold the queue the insertion says so through the status word.
+        if (d_fixed) {               // only the prompts of the order, and the clock advances by as many as were processed
+            replay_list_kernel<<<(unsigned)((n_fixed + 255) / 256), 256, 0, s>>>(d_fixed, n_fixed, tree->replay_info, tree->bulk_pend_a);
+            return bulk_insert(tree, d_q_tokens, d_q_offsets, n_fixed, s, state, tag, true, &tree->replay_info->n_valid);
+        }
         return bulk_insert(tree, d_q_tokens, d_q_offsets, n, s, state, tag);
     }
+    if (d_fixed) return RT_ERR_INVALID;       // (klpm_replay takes its sequential kernel instead of this loop)
     RunBcast bc0;
     memset(&bc0, 0, sizeof(bc0));
     bc0.now = params->start_tick;
@@ -4484,6 +4576,15 @@ rt_status klpm_run_last_only_batch(const int32_t* d_tokens, const int64_t* d_off
     last_only_batch_kernel<<<blocks, 32 * KLPM_LAST_ONLY_WARPS, 0, s>>>(a);
     CK(cudaGetLastError());
     return RT_OK;
+}
+
+rt_status klpm_run_ex(rt_tree* tree, const int32_t* d_q_tokens, const int64_t* d_q_offsets, const int64_t* d_arrival,
+                      int32_t n, const klpm_params* params, const int64_t* d_tie_priority, int32_t score_mode,
+                      const klpm_match_state* d_match_state, int32_t* d_order, int32_t* d_uncached, int64_t* d_ttft,
+                      int64_t* d_completion, void* stream) {
+    if (n > 0 && !d_order) return RT_ERR_INVALID;
+    return run_impl(tree, d_q_tokens, d_q_offsets, d_arrival, n, params, d_tie_priority, score_mode, d_match_state, d_order,
+                    d_uncached, d_ttft, d_completion, nullptr, 0, stream);
 }
 
 int32_t klpm_run_path(const rt_tree* tree) { return tree ? tree->run_path : 0; }

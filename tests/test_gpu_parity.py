@@ -225,13 +225,56 @@ def test_replay_fixed_order(K, budget):
     assert K.rt_stats(tree)["evictions"] == ot.stats()["evictions"]
 
 
+@pytest.mark.parametrize("budget", [0, 4000])
+def test_replay_both_forms_on_a_longer_queue(K, budget):
+    """6,000 prompts with shared blocks, a random order of 4,500 of them, c_attn = 1/2: the replay through the device
+    loop, the plain one-prompt-after-the-other form (debug setting) and the oracle agree on every output and on the
+    tree that is left (match of every prompt afterwards)."""
+    rng = np.random.RandomState(3)
+    blocks = [rng.randint(0, 6, size=10).tolist() for _ in range(5)]
+    prompts = [blocks[rng.randint(5)] + blocks[rng.randint(5)][:rng.randint(1, 11)] + rng.randint(0, 6, size=rng.randint(0, 7)).tolist()
+               for _ in range(6000)]
+    arr = np.cumsum(rng.randint(0, 3, size=6000)).tolist()
+    qt, qo = csr(prompts)
+    order = torch.from_numpy(rng.permutation(6000)[:4500].astype(np.int32))
+    n = len(prompts)
+    got = []
+    for plain in (False, True):
+        tree = K.rt_create(budget_tokens=budget, **caps(qt.numel(), n_prompts=n))
+        unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        ttft = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+        comp = torch.full((n,), -1, dtype=torch.int64, device="cuda")
+        K.klpm_debug_set("run_one_by_one", 1 if plain else 0)
+        try:
+            K.klpm_replay(tree, dev(order), dev(qt), dev(qo), dev(torch.tensor(arr)), K.make_params(K.POLICY_FCFS, 1, 1, 2, 3), unc, ttft, comp)
+            assert K.rt_sync_status(tree) == 0
+        finally:
+            K.klpm_debug_set("run_one_by_one", -1)
+        m, _, off = gpu_match(K, tree, qt, qo)
+        got.append((unc.cpu().numpy(), ttft.cpu().numpy(), comp.cpu().numpy(), m, off, K.rt_stats(tree)))
+        K.rt_destroy(tree)
+    ot = oracle.OracleTree(budget)
+    ou, ottft, ocomp = oracle.replay(order.numpy(), qt.numpy(), qo.numpy(), arr, 1, 2, 3, oracle.CACHE_TREE, ot)
+    want_u, want_t, want_c = (np.full(n, -1, dtype=x.dtype) for x in (ou, ottft, ocomp))
+    idx = order.numpy()
+    want_u[idx], want_t[idx], want_c[idx] = ou[idx], ottft[idx], ocomp[idx]
+    om, ooff, _ = ot.match_pos(qt.numpy(), qo.numpy())
+    for g in got:
+        assert np.array_equal(g[0], want_u) and np.array_equal(g[1], want_t) and np.array_equal(g[2], want_c)
+        assert np.array_equal(g[3], om) and np.array_equal(g[4], ooff)
+        for key in ("n_nodes", "tokens", "clock", "evictions"):
+            assert g[5][key] == ot.stats()[key], key
+    if budget:
+        assert ot.stats()["evictions"] > 0
+
+
 def test_replay_stops_at_an_order_entry_that_is_not_a_query(K):
     """An order with -1 (or an index past the queue) in it: the replay processes what comes before, touches nothing
     for the bad entry or after it, and reports RT_ERR_INVALID through the status word."""
     prompts, arr = W.random_small_queue(23, 12, vocab=3, max_len=9, min_len=1)
     qt, qo = csr(prompts)
     n = len(prompts)
-    for bad in (-1, n, 1 << 30):
+    for bad in (-1, n, 1 << 30, 3):                       # not a query, or a query that was processed already
         tree = K.rt_create(**caps(qt.numel(), n_prompts=n))
         order = torch.tensor([3, 1, bad, 2], dtype=torch.int32)
         unc = torch.full((n,), -1, dtype=torch.int32, device="cuda")
