@@ -58,6 +58,8 @@ def lib():
         L.oc_tree_match.argtypes = [vp, vp, vp, i32, vp, i32]
         L.oc_tree_match_pos.restype = None
         L.oc_tree_match_pos.argtypes = [vp, vp, vp, i32, vp, vp, vp]
+        L.oc_select.restype = i32
+        L.oc_select.argtypes = [vp, vp, vp, i32, i64, i32, i32]
         L.oc_replay.restype = i32
         L.oc_replay.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, i64, i64, i32, vp, vp, vp]
         L.oc_batch_times.restype = None
@@ -163,6 +165,13 @@ def schedule(tokens, offsets, arrivals, policy: int, k: int = 1, c_num: int = 0,
     if rc:
         raise RuntimeError("oracle: schedule failed (%d)" % rc)
     return order, unc, ttft, comp
+
+
+def select(match_len, arrivals, waiting, pick_counter: int, policy: int, k: int = 1) -> int:
+    """One decision of Algorithm 1 over a snapshot of the queue: index of the pick, -1 if nobody is waiting."""
+    m, a = _i32(match_len), _i64(arrivals)
+    w = np.ascontiguousarray(np.asarray(waiting), dtype=np.uint8)
+    return int(lib().oc_select(_p(m), _p(a), _p(w), len(m), int(pick_counter), int(policy), max(1, int(k))))
 
 
 def replay(order, tokens, offsets, arrivals, c_num: int = 0, c_den: int = 1, start_tick: int = 0,

@@ -155,6 +155,16 @@ def schedule(prompts: Sequence[Sequence[int]], arrivals: Sequence[int], policy: 
     return order, unc, ttft, comp
 
 
+def select(match_len: Sequence[int], arrivals: Sequence[int], waiting: Sequence[int], pick_counter: int, policy: int, k: int = 1) -> int:
+    """One decision of Algorithm 1 over a snapshot: the rule of schedule() above, on given match lengths."""
+    idx = [i for i in range(len(match_len)) if waiting[i]]
+    if not idx:
+        return -1
+    if policy == FCFS or (policy == KLPM and pick_counter % k == 0):
+        return min(idx, key=lambda i: (arrivals[i], i))
+    return min(idx, key=lambda i: (-match_len[i], arrivals[i], i))
+
+
 def replay(order: Sequence[int], prompts, arrivals, c_num: int = 0, c_den: int = 1, start_tick: int = 0,
            cache_mode: int = TREE, prefill=(), budget: int = 0):
     """Definition 2 along a fixed order.  Returns (uncached, ttft, completion) indexed by query."""

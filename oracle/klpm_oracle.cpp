@@ -310,6 +310,23 @@ void oc_batch_times(const int32_t* order, int32_t n_order, const int64_t* arriva
     }
 }
 
+// One decision of Algorithm 1 as a function of its inputs: among the waiting queries, the oldest one (smallest arrival,
+// then index) on an oldest-first turn -- FCFS always, k-LPM when pick_counter is a multiple of k -- and otherwise the
+// one with the longest match, ties to the oldest.  Returns its index, or -1 if nobody is waiting.
+int32_t oc_select(const int32_t* match_len, const int64_t* arrival, const uint8_t* waiting, int32_t n,
+                  int64_t pick_counter, int32_t policy, int32_t k) {
+    const bool fcfs_turn = policy == POLICY_FCFS || (policy == POLICY_KLPM && pick_counter % k == 0);
+    int32_t j = -1;
+    for (int32_t i = 0; i < n; ++i) {
+        if (!waiting[i]) continue;
+        bool wins = j < 0;
+        if (!wins && !fcfs_turn && match_len[i] != match_len[j]) wins = match_len[i] > match_len[j];
+        else if (!wins) wins = arrival[i] < arrival[j];      // equal arrivals: the lower index stays
+        if (wins) j = i;
+    }
+    return j;
+}
+
 // Algorithm 1 (k-LPM) with its FCFS and LPM limits, run over the whole stream.
 // order[c] = index processed at decision c; uncached/ttft/completion are indexed by query.
 // Variants of the longest-match pick (both leave the oldest-first picks alone):

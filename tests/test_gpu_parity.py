@@ -177,14 +177,6 @@ def test_invalid_arguments(K):
 
 # ------------------------------------------------------------------ selection (one decision)
 
-def select_by_definition(m, t, waiting, c, policy, k):
-    idx = [i for i in range(len(m)) if waiting[i]]
-    if not idx:
-        return -1
-    if policy == 0 or (policy == 2 and c % k == 0):
-        return min(idx, key=lambda i: (t[i], i))
-    return min(idx, key=lambda i: (-m[i], t[i], i))
-
 
 @pytest.mark.parametrize("n", [1, 33, 1000, 70001])
 def test_select_single_decision(K, n):
@@ -195,7 +187,7 @@ def test_select_single_decision(K, n):
     pick = torch.zeros(1, dtype=torch.int32, device="cuda")
     for policy, k, c in [(0, 1, 0), (1, 1, 5), (2, 3, 0), (2, 3, 1), (2, 3, 2), (2, 3, 3), (2, 1, 7)]:
         K.klpm_select(dev(m), dev(t), dev(waiting), c, K.make_params(policy, k), pick)
-        assert int(pick.item()) == select_by_definition(m.tolist(), t.tolist(), waiting.tolist(), c, policy, k)
+        assert int(pick.item()) == oracle.select(m.numpy(), t.numpy(), waiting.numpy(), c, policy, k)
     K.klpm_select(dev(m), dev(t), dev(torch.zeros(n, dtype=torch.uint8)), 1, K.make_params(1), pick)
     assert int(pick.item()) == -1
 
@@ -513,9 +505,11 @@ def test_select_topk_snapshot(K, n, kk):
     out = torch.full((kk,), -9, dtype=torch.int32, device="cuda")
     for _ in range(2):                                   # the scratch is reused
         K.klpm_select_topk(dev(m), dev(t), dev(waiting), out)
-        idx = [i for i in range(n) if waiting[i]]
-        idx.sort(key=lambda i: (-int(m[i]), int(t[i]), i))
-        want = (idx + [-1] * kk)[:kk]
+        left, want = waiting.numpy().copy(), []           # the oracle's longest-match pick, kk times over what is left
+        for _j in range(kk):
+            want.append(oracle.select(m.numpy(), t.numpy(), left, 1, oracle.POLICY_LPM))
+            if want[-1] >= 0:
+                left[want[-1]] = 0
         assert out.tolist() == want
     # its first entry is klpm_select's longest-match pick
     pick = torch.zeros(1, dtype=torch.int32, device="cuda")

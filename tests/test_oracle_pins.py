@@ -142,6 +142,31 @@ def test_toy_example_printed_values(tier):
     assert run(prompts, arr, oracle.POLICY_FCFS, mode=oracle.CACHE_TREE)[2] == [10, 20, 25, 30]
 
 
+# ---------------------------------------------------------------- one decision as a function of a snapshot
+
+def test_select_by_hand_and_against_the_definition():
+    """Toy queue after x1 was processed: x3 shares x1's user (match 5), the others match 0.  The longest-match turn
+    takes x3, the oldest-first turn x2; among equal matches the earliest arrival wins, among equal arrivals the
+    lower index; nobody waiting gives -1."""
+    m, t, w = [10, 0, 5, 0], [0, 0, 0, 0], [0, 1, 1, 1]
+    assert oracle.select(m, t, w, 1, oracle.POLICY_KLPM, 2) == 2        # turn 1 of a 2-cycle: longest match
+    assert oracle.select(m, t, w, 2, oracle.POLICY_KLPM, 2) == 1        # turn 2: the oldest waiting
+    assert oracle.select(m, t, w, 7, oracle.POLICY_FCFS) == 1
+    assert oracle.select(m, t, w, 0, oracle.POLICY_LPM) == 2
+    assert oracle.select([3, 3, 3], [5, 2, 2], [1, 1, 1], 1, oracle.POLICY_LPM) == 1
+    assert oracle.select([3, 3], [5, 2], [0, 0], 1, oracle.POLICY_LPM) == -1
+    rng = np.random.RandomState(0)
+    for _ in range(200):
+        n = int(rng.randint(1, 40))
+        m, t, w = rng.randint(0, 4, n), rng.randint(0, 5, n), rng.randint(0, 2, n)
+        for policy, k, c in ((0, 1, 3), (1, 1, 3), (2, 3, 0), (2, 3, 1), (2, 3, 5), (2, 1, 4)):
+            assert oracle.select(m, t, w, c, policy, k) == D.select(m.tolist(), t.tolist(), w.tolist(), c, policy, k)
+    # the loop's own picks are this rule applied to the match lengths of the moment
+    prompts, arr = W.regular_arrival_shuffled_queue(4, 2, 5, 5, 0, [1, 2, 3, 4])
+    order = run(prompts, arr, oracle.POLICY_KLPM, k=2, mode=oracle.CACHE_LAST_ONLY)[0]
+    assert order[1] == oracle.select([0, 0, 5, 0], arr, [0, 1, 1, 1], 1, oracle.POLICY_KLPM, 2)
+
+
 # ---------------------------------------------------------------- limits of k-LPM
 
 @pytest.mark.parametrize("seed", range(5))
