@@ -2360,10 +2360,10 @@ fast_run_kernel(FastArgs A) {
             const long long pre_cc = cur0 + lane;
             const int32_t pre_v = pre_cc < clock ? T.clock_owner[pre_cc] : 0;
             bool pre_ok = false;
-            int32_t pre_P = 0, pre_len = 0;
+            int32_t pre_P = 0, pre_len = 0, pre_parked = 0;
             if (pre_v > 0) {
                 pre_ok = !T.dead[pre_v] && T.last_access[pre_v] == pre_cc && T.nchild[pre_v] == 0;
-                pre_P = T.parent[pre_v]; pre_len = T.span_len[pre_v];
+                pre_P = T.parent[pre_v]; pre_len = T.span_len[pre_v]; pre_parked = __ldcg(A.parked + pre_v);
             }
             while (a != 0 && m <= ds) { a = pa; ds = T.depth_start[a]; sl = T.span_len[a]; pa = T.parent[a]; }
             const int32_t o = a == 0 ? 0 : m - ds;
@@ -2389,20 +2389,25 @@ fast_run_kernel(FastArgs A) {
             int32_t small_v[8];                             // evicted leaves whose parked queries this warp looks after itself
             int n_small = 0;
             long long cur = cur0;
-            bool first = true;
+            // The leaves of the window that was loaded ahead are taken one after the other while the window's view of who
+            // is a leaf holds: it ends when an eviction turns a parent into a leaf (that parent may be the next to go).
+            bool first = true, win_ok = true;
+            unsigned win = 0;
             while (tokens_live + unc > T.budget) {
-                int32_t victim = -1, P = 0, vlen = 0;
-                if (first) {                                // the window that was loaded ahead (the node stamped above has moved on)
-                    const unsigned bal = __ballot_sync(FULL_MASK, pre_ok && pre_v != end);
-                    if (bal) {
-                        const int src = __ffs(bal) - 1;
-                        victim = __shfl_sync(FULL_MASK, pre_v, src); P = __shfl_sync(FULL_MASK, pre_P, src); vlen = __shfl_sync(FULL_MASK, pre_len, src);
-                        cur += src;
+                int32_t victim = -1, P = 0, vlen = 0, vparked = 0;
+                if (win_ok) {
+                    if (first) { win = __ballot_sync(FULL_MASK, pre_ok && pre_v != end); first = false; }      // (the node stamped above has moved on)
+                    if (win) {
+                        const int src = __ffs(win) - 1;
+                        win &= win - 1;
+                        victim = __shfl_sync(FULL_MASK, pre_v, src); P = __shfl_sync(FULL_MASK, pre_P, src);
+                        vlen = __shfl_sync(FULL_MASK, pre_len, src); vparked = __shfl_sync(FULL_MASK, pre_parked, src);
+                        cur = cur0 + src;
                         if (cut && victim == a) { P = T.parent[victim]; vlen = T.span_len[victim]; }      // the lower part of the edge just cut
                     } else {
-                        cur += 32;
+                        cur = cur0 + 32;
+                        win_ok = false;
                     }
-                    first = false;
                 }
                 if (victim < 0) {
                     while (cur < clock) {                   // 32 clock values at a time
@@ -2413,7 +2418,7 @@ fast_run_kernel(FastArgs A) {
                         if (bal) { const int src = __ffs(bal) - 1; victim = __shfl_sync(FULL_MASK, v, src); cur += src; break; }
                         cur += 32;
                     }
-                    if (victim >= 0) { P = T.parent[victim]; vlen = T.span_len[victim]; }
+                    if (victim >= 0) { P = T.parent[victim]; vlen = T.span_len[victim]; vparked = __ldcg(A.parked + victim); }
                 }
                 if (victim < 0) {
                     if (lane == 0) set_status(A.st, RT_ERR_BUDGET);
@@ -2421,7 +2426,7 @@ fast_run_kernel(FastArgs A) {
                 }
                 tokens_live -= vlen;
                 --live_nodes; ++evictions; ++n_evict;
-                if (__ldcg(A.parked + victim) > 0) {
+                if (vparked > 0) {
                     // Queries are parked in the evicted leaf.  If one run of the member array is known to hold every slot
                     // whose hint is this leaf, the warp looks after them itself below (up to 8 such leaves and 32 slots
                     // that fall back per decision); otherwise the whole CTA scans the unprocessed slots.
@@ -2429,13 +2434,17 @@ fast_run_kernel(FastArgs A) {
                     if (lr.y > 0 && lr.y <= 1024 && n_small < 8) { small_v[n_small] = victim; ++n_small; }
                     else scan = true;
                 }
+                int new_leaf = 0;
                 if (lane == 0) {
                     T.dead[victim] = 1;
-                    T.nchild[P]--;
+                    const int32_t nc = T.nchild[P] - 1;
+                    T.nchild[P] = nc;
                     const long long stamp = T.last_access[victim];
                     if (P != 0 && stamp >= T.last_access[P]) { T.last_access[P] = stamp; T.clock_owner[stamp] = P; }
+                    new_leaf = nc == 0 && P != 0;
                 }
                 __syncwarp();
+                if (win_ok && __shfl_sync(FULL_MASK, new_leaf, 0)) win_ok = false;
             }
             if (cur > clock) cur = clock;
             if (!failed && unc > 0) {
