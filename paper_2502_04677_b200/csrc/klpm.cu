@@ -1731,10 +1731,10 @@ struct FastBatchIO {
 #define KLPM_FAST_CTA_MIN 128         // smaller batches are left to the warp-wide step (an attempt costs about 16,000 cycles)
 #endif
 #ifndef KLPM_FAST_CB_MAX
-#define KLPM_FAST_CB_MAX 1024         // longest back-off (loop iterations) after CTA-wide attempts that failed
+#define KLPM_FAST_CB_MAX 32           // longest back-off (loop iterations) after CTA-wide attempts that failed
 #endif
 #ifndef KLPM_FAST_CALM
-#define KLPM_FAST_CALM 4              // full warp-wide steps in a row before a CTA-wide batch is tried again
+#define KLPM_FAST_CALM 1              // full warp-wide steps in a row before a CTA-wide batch is tried again
 #endif
 
 // Exclusive prefix sum of v over the CTA's 256 threads; *total receives the sum.  s_w: 8 ints of shared scratch.
@@ -1795,18 +1795,22 @@ __device__ __forceinline__ unsigned long long fast_member(const FastArgs& A, con
 // Every thread calls it.  Nothing is changed unless at least KLPM_FAST_CTA_MIN decisions can be made.
 template <bool G>
 __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchIO* io, int32_t* sH, int32_t* sE, int32_t* sEpos,
-                               int32_t* s_w, int32_t nwords) {
+                               int32_t* sF, int32_t* s_w, int32_t nwords) {
     FastTour R = R0;                                        // with the bitmaps in shared memory the flags fold away
     if (!G) { R.g_done = 0; R.g_bits = 0; }
     const int tid = threadIdx.x;
     const int32_t n = A.n, cur = io->cur, head = io->head, c = io->c, cyc = io->cyc;
     const unsigned long long root = io->root;
-    auto f = [&](int32_t x) -> int32_t {                  // oldest-first turns among the next x decisions
-        if (A.policy == KLPM_POLICY_FCFS) return x;
-        if (A.policy == KLPM_POLICY_LPM) return 0;
-        const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;
-        return x > i0 ? (x - i0 - 1) / A.k + 1 : 0;
-    };
+    // sF[x] = oldest-first turns among the next x decisions, x = 0 .. 1,024 (a table: the division is done once per entry)
+    for (int32_t x = tid; x <= KLPM_FAST_CTA_BATCH; x += KLPM_FAST_THREADS) {
+        int32_t v;
+        if (A.policy == KLPM_POLICY_FCFS) v = x;
+        else if (A.policy == KLPM_POLICY_LPM) v = 0;
+        else { const int32_t i0 = cyc == 0 ? 0 : A.k - cyc; v = x > i0 ? (x - i0 - 1) / A.k + 1 : 0; }
+        sF[x] = v;
+    }
+    if (tid == 0) { io->B0 = 0; io->B = 0; }
+    auto f = [&](int32_t x) -> int32_t { return sF[x]; };
     // the list entries cur + 4 tid .. + 3 that still count
     long long kk[4]; int32_t es[4]; bool ok[4];
     int32_t cnt = 0;
@@ -1821,11 +1825,18 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         cnt += ok[r];
     }
     int32_t avail;
-    const int32_t base = block_excl_scan(cnt, s_w, &avail);
-    if (tid == 0) {                                       // as many decisions as those entries allow
-        int32_t lo = 0, hi = n - c < KLPM_FAST_CTA_BATCH ? n - c : KLPM_FAST_CTA_BATCH;
-        while (lo < hi) { const int32_t mid = (lo + hi + 1) >> 1; if (mid - f(mid) <= avail) lo = mid; else hi = mid - 1; }
-        io->B0 = lo; io->nF0 = f(lo); io->nL0 = lo - f(lo);
+    const int32_t base = block_excl_scan(cnt, s_w, &avail);      // (its barriers also publish sF and the cleared io fields)
+    {   // as many decisions as those entries allow: the largest x with x - f(x) <= avail, every thread trying four values
+        const int32_t hi = n - c < KLPM_FAST_CTA_BATCH ? n - c : KLPM_FAST_CTA_BATCH;
+        int32_t best = 0;
+#pragma unroll
+        for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= hi && x - f(x) <= avail) best = x; }
+        if (best > 0) atomicMax(&io->B0, best);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const int32_t lo = io->B0;
+        io->nF0 = f(lo); io->nL0 = lo - f(lo);
         io->limF = io->nF0; io->limL = io->nL0; io->limB = lo;
     }
     __syncthreads();
@@ -1888,11 +1899,16 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         }
     }
     __syncthreads();
+    {   // the largest x that respects the three limits, every thread trying four values
+        const int32_t limF = io->limF, limL = io->limL, limB = io->limB;
+        int32_t best = 0;
+#pragma unroll
+        for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= B0 && x <= limB && f(x) <= limF && x - f(x) <= limL) best = x; }
+        if (best > 0) atomicMax(&io->B, best);
+    }
+    __syncthreads();
     if (tid == 0) {
-        const int32_t limF = io->limF, limL = io->limL;
-        int32_t lo = 0, hi = B0;
-        while (lo < hi) { const int32_t mid = (lo + hi + 1) >> 1; if (f(mid) <= limF && mid - f(mid) <= limL) lo = mid; else hi = mid - 1; }
-        if (io->limB < lo) lo = io->limB;
+        const int32_t lo = io->B;
         const int32_t B = lo >= KLPM_FAST_CTA_MIN ? lo : 0;
         const int32_t nF = f(B), nL = B - nF;
         io->B = B;
@@ -2265,7 +2281,7 @@ fast_run_kernel(FastArgs A) {
             named_bar(1, KLPM_FAST_THREADS);
             const FastJob J = s_job;
             if (J.type == FAST_JOB_EXIT) return;
-            if (J.type == FAST_JOB_BATCH) { fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords); continue; }
+            if (J.type == FAST_JOB_BATCH) { fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, reinterpret_cast<int32_t*>(sh), s_scan, nwords); continue; }
             fast_job(A, R, J, sh, sr, &s_cnt, &s_memcur);
         }
     }
@@ -2878,7 +2894,7 @@ fast_run_kernel(FastArgs A) {
                 const long long t_cta = clock64();
                 ++n_cta_try;
                 named_bar(1, KLPM_FAST_THREADS);
-                fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, s_scan, nwords);
+                fast_batch_job<G>(A, R, &s_bio, sr, sr + 1024, sr + 2048, reinterpret_cast<int32_t*>(sh), s_scan, nwords);
                 const int32_t Bc = s_bio.B;
                 const long long cy_this = clock64() - t_cta;
                 cy_cta += cy_this;
