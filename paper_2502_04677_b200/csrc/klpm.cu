@@ -1724,11 +1724,12 @@ struct FastBatchIO {
     unsigned long long root;          // in: largest key in the tournament
     int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
     int32_t B0, nF0, nL0, limF, limL; // scratch
+    int32_t wneed;                    // scratch: bitmap words from the oldest unprocessed slot on that hold the slots wanted
     int32_t limB;                     // scratch: the batch must end before this decision (list entries that an oldest-first pick would meet)
 };
 #define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
 #ifndef KLPM_FAST_CTA_MIN
-#define KLPM_FAST_CTA_MIN 128         // smaller batches are left to the warp-wide step (an attempt costs about 16,000 cycles)
+#define KLPM_FAST_CTA_MIN 32         // smaller batches are left to the warp-wide step (an attempt costs about 16,000 cycles)
 #endif
 #ifndef KLPM_FAST_CB_MAX
 #define KLPM_FAST_CB_MAX 32           // longest back-off (loop iterations) after CTA-wide attempts that failed
@@ -1801,27 +1802,35 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     const int tid = threadIdx.x;
     const int32_t n = A.n, cur = io->cur, head = io->head, c = io->c, cyc = io->cyc;
     const unsigned long long root = io->root;
-    // sF[x] = oldest-first turns among the next x decisions, x = 0 .. 1,024 (a table: the division is done once per entry)
-    for (int32_t x = tid; x <= KLPM_FAST_CTA_BATCH; x += KLPM_FAST_THREADS) {
-        int32_t v;
-        if (A.policy == KLPM_POLICY_FCFS) v = x;
-        else if (A.policy == KLPM_POLICY_LPM) v = 0;
-        else { const int32_t i0 = cyc == 0 ? 0 : A.k - cyc; v = x > i0 ? (x - i0 - 1) / A.k + 1 : 0; }
-        sF[x] = v;
+    // the list entries cur + 4 tid .. + 3 (asked for first: the table below is filled while they travel)
+    long long kk[4]; int32_t es[4]; bool ok[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const long long idx = (long long)cur + tid * 4 + r;
+        kk[r] = 0; es[r] = 0;
+        if (idx < n) { kk[r] = __ldg(A.lk + idx); es[r] = __ldg(A.ls + idx); }
+    }
+    // sF[x] = oldest-first turns among the next x decisions, x = 0 .. 1,024.  Under k-LPM the first such turn is
+    // decision (k - cyc) mod k and then every k-th, which is floor((x + s) / k) with s = (cyc + k - 1) mod k; one
+    // division per thread, the later entries follow by adding 256 = Q k + Rm.
+    {
+        const int32_t sft = cyc == 0 ? A.k - 1 : cyc - 1;
+        int32_t q = 0, rem = 0, Q = 0, Rm = 0;
+        if (A.policy == KLPM_POLICY_KLPM) { q = (tid + sft) / A.k; rem = (tid + sft) - q * A.k; Q = KLPM_FAST_THREADS / A.k; Rm = KLPM_FAST_THREADS - Q * A.k; }
+        for (int32_t x = tid; x <= KLPM_FAST_CTA_BATCH; x += KLPM_FAST_THREADS) {
+            sF[x] = A.policy == KLPM_POLICY_FCFS ? x : A.policy == KLPM_POLICY_LPM ? 0 : q;
+            q += Q; rem += Rm;
+            if (rem >= A.k) { rem -= A.k; ++q; }
+        }
     }
     if (tid == 0) { io->B0 = 0; io->B = 0; }
     auto f = [&](int32_t x) -> int32_t { return sF[x]; };
-    // the list entries cur + 4 tid .. + 3 that still count
-    long long kk[4]; int32_t es[4]; bool ok[4];
+    // those of the entries that still count
     int32_t cnt = 0;
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         const long long idx = (long long)cur + tid * 4 + r;
-        ok[r] = false; kk[r] = 0; es[r] = 0;
-        if (idx < n) {
-            kk[r] = __ldg(A.lk + idx); es[r] = __ldg(A.ls + idx);
-            ok[r] = !((bm_ld(R.skip, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u);
-        }
+        ok[r] = idx < n && !((bm_ld(R.skip, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u);
         cnt += ok[r];
     }
     int32_t avail;
@@ -1831,7 +1840,8 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         int32_t best = 0;
 #pragma unroll
         for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= hi && x - f(x) <= avail) best = x; }
-        if (best > 0) atomicMax(&io->B0, best);
+        best = __reduce_max_sync(FULL_MASK, best);
+        if ((tid & 31) == 0 && best > 0) atomicMax(&io->B0, best);
     }
     __syncthreads();
     if (tid == 0) {
@@ -1848,19 +1858,35 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         unsigned w = wi < nwords ? bm_ld(R.done, wi, R.g_done) : 0xffffffffu;
         if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
         if (wi == w0) w |= (1u << (head & 31)) - 1u;
-        unsigned fr = ~w;
+        const unsigned fr = ~w;
         int32_t nfree;
-        int32_t qk = block_excl_scan(__popc(fr), s_w, &nfree);
-        while (fr && qk < nF0) { const int bit = __ffs(fr) - 1; fr &= fr - 1; sH[qk++] = wi * 32 + bit; }
+        const int32_t qk = block_excl_scan(__popc(fr), s_w, &nfree);
+        // every word's free slots and how many lie before it; the word that holds the last slot wanted says how far to go
+        int32_t* sP = sF + KLPM_FAST_CTA_BATCH + 8;
+        unsigned* sFr = reinterpret_cast<unsigned*>(sP + KLPM_FAST_THREADS);
+        sP[tid] = qk; sFr[tid] = fr;
         const int32_t nFa = nfree < nF0 ? nfree : nF0;
+        if (nFa > 0 && qk < nFa && qk + __popc(fr) >= nFa) io->wneed = tid + 1;
         if (tid == 0 && nFa < nF0) io->limF = nFa;
+        __syncthreads();
+        // a thread per slot, eight words at a time: the slot's rank among the free ones is where it goes; one whose key
+        // sits in the tournament or that is grouped needs the careful step
+        const int32_t wneed = nFa > 0 ? io->wneed : 0;
+        const int bit = tid & 31;
+        for (int32_t wl = tid >> 5; wl < wneed; wl += KLPM_FAST_THREADS / 32) {
+            const unsigned fw = sFr[wl];
+            if ((fw >> bit) & 1u) {
+                const int32_t rank = sP[wl] + __popc(fw & ((1u << bit) - 1u));
+                if (rank < nFa) {
+                    const int32_t hs = (w0 + wl) * 32 + bit;
+                    sH[rank] = hs;
+                    if (((bm_ld(R.skip, hs >> 5, R.g_bits) | bm_ld(R.gb, hs >> 5, R.g_bits)) >> (hs & 31)) & 1u) atomicMin(&io->limF, rank);
+                }
+            }
+        }
         __syncthreads();
         if (nFa > 0) hmax0 = sH[nFa - 1];
         nFa0 = nFa;
-        for (int32_t qi = tid; qi < nFa; qi += KLPM_FAST_THREADS) {       // key in the tournament, or grouped: needs the careful step
-            const int32_t hs = sH[qi];
-            if (((bm_ld(R.skip, hs >> 5, R.g_bits) | bm_ld(R.gb, hs >> 5, R.g_bits)) >> (hs & 31)) & 1u) atomicMin(&io->limF, qi);
-        }
     }
     // The usable entries by rank.  One that is grouped or lies below the tournament's root stops the batch before its
     // turn.  One whose slot is among the slots the oldest-first picks of a full batch would take (rank phi there) is
@@ -1904,7 +1930,8 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         int32_t best = 0;
 #pragma unroll
         for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= B0 && x <= limB && f(x) <= limF && x - f(x) <= limL) best = x; }
-        if (best > 0) atomicMax(&io->B, best);
+        best = __reduce_max_sync(FULL_MASK, best);
+        if ((tid & 31) == 0 && best > 0) atomicMax(&io->B, best);
     }
     __syncthreads();
     if (tid == 0) {
@@ -2762,6 +2789,7 @@ fast_run_kernel(FastArgs A) {
         // that fails a check; then lane i makes decision c + i.  If fewer than two decisions are left that way,
         // nothing has been changed and the next decisions are made one at a time below.
         const int32_t lane_div_k = lane / A.k;              // y / k for y = 0..31, looked up by shuffle
+        bool tb_cut = false;                                // the last warp-wide step stopped before a decision it could not take
         auto try_batch = [&]() -> bool {
             // oldest-first turns among the next x decisions, for x = lane (f_lo) and x = lane + 1 (f_hi): under k-LPM
             // the first such turn is decision i0 = (k - cyc) mod k, then every k-th
@@ -2851,6 +2879,7 @@ fast_run_kernel(FastArgs A) {
                 if (fh == fl && B - fl == limL && fl <= limF && (fl == 0 || last_h < soft)) { ++B; ++limL; }
             }
             if (B < 2) return false;
+            tb_cut = B < B0;
             const int32_t nF = __shfl_sync(FULL_MASK, f_hi, B - 1), nL = B - nF;
             const int32_t hmax = nF > 0 ? __shfl_sync(FULL_MASK, hs, nF - 1) : -1;
             if (lane < nF) s_H[lane] = hs;
@@ -2883,9 +2912,12 @@ fast_run_kernel(FastArgs A) {
         int32_t cb_wait = 0, cb_back = 8;                   // the same for the CTA-wide batch (loop iterations; 8 .. 1,024)
         int32_t calm = KLPM_FAST_CALM;                      // consecutive full warp-wide steps: the CTA-wide batch is tried in calm water only
         long long n_cta_try = 0, n_cta_ok = 0, dec_cta = 0, n_warp_ok = 0, dec_warp = 0, dec_one = 0, cy_cta = 0, cy_warp = 0;
+        // a batch that was cut short stopped before a decision only the one-at-a-time path can take: that one comes
+        // next, without another attempt that would find it again
+        bool one_next = false;
         while (c < n && !failed) {
             // first choice: the whole CTA makes up to 1,024 decisions (the sort scratch is free between dissolves)
-            if (cb_wait <= 0 && calm >= KLPM_FAST_CALM && n - c >= KLPM_FAST_CTA_MIN) {
+            if (!one_next && cb_wait <= 0 && calm >= KLPM_FAST_CALM && n - c >= KLPM_FAST_CTA_MIN) {
                 if (lane == 0) {
                     s_bio.cur = cur; s_bio.head = head; s_bio.c = c; s_bio.cyc = cyc; s_bio.root = root; s_bio.B = 0;
                     s_job.type = FAST_JOB_BATCH;
@@ -2902,6 +2934,7 @@ fast_run_kernel(FastArgs A) {
                     ++n_cta_ok; dec_cta += Bc;
                     const int32_t consumed = s_bio.consumed, hmax = s_bio.hmax;
                     c += Bc;
+                    one_next = Bc < s_bio.B0;
                     if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + Bc) % A.k;
                     if (consumed) { cur += consumed; window(cur & ~31, &wk, &ws); window((cur & ~31) + 32, &nk, &ns); }
                     if (hmax >= 0) { head = hmax; advance_head(); }
@@ -2920,17 +2953,18 @@ fast_run_kernel(FastArgs A) {
                 calm = 0;
             }
             --cb_wait;
-            if (vb_wait <= 0) {
+            if (!one_next && vb_wait <= 0) {
                 const int32_t c_was = c;
                 const long long t_w = clock64();
                 const bool took = try_batch();
                 cy_warp += clock64() - t_w;
-                if (took) { ++n_warp_ok; dec_warp += c - c_was; vb_back = 1; calm = c - c_was == 32 ? calm + 1 : 0; continue; }
+                if (took) { ++n_warp_ok; dec_warp += c - c_was; vb_back = 1; calm = c - c_was == 32 ? calm + 1 : 0; one_next = tb_cut; continue; }
                 calm = 0;
                 vb_wait = vb_back;
                 vb_back = vb_back < 64 ? vb_back * 2 : 64;
             }
-            --vb_wait;
+            if (!one_next) --vb_wait;
+            one_next = false;
             ++dec_one;
             const bool fcfs_turn = A.policy == KLPM_POLICY_FCFS || (A.policy == KLPM_POLICY_KLPM && cyc == 0);
             if (++cyc == A.k) cyc = 0;
