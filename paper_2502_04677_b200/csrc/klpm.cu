@@ -3158,132 +3158,198 @@ bulk_walk_kernel(TreeDev T, BulkArgs A, unsigned n_pending) {
 
 // First round when a batched match of the prompts against the tree as it still is has left its records (MatchState):
 // the node where each match ended is looked up from the position (end_node[] along the run), then what
-// bulk_walk_kernel does after its walk.  One warp per prompt.
+// bulk_walk_kernel does after its walk.  One lane per prompt, 32 prompts of the list per warp at a time; the search
+// along a run for a match that ended inside an edge is the whole warp's, one prompt after the other; the list of
+// pending prompts grows by one addition per warp.
 __global__ void __launch_bounds__(256)
 bulk_from_state_kernel(TreeDev T, BulkArgs A, const MatchState* __restrict__ state, unsigned long long tag, unsigned n_pending) {
     const int lane = threadIdx.x & 31;
     const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
-    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps) {
-        const int32_t i = A.pend_in[p];
-        if (i < 0) continue;                                // a replay that stopped early: not processed
-        const int32_t len = (int32_t)(__ldg(A.off + i + 1) - __ldg(A.off + i));
-        const int4* src = reinterpret_cast<const int4*>(state + i);
-        const int4 a = __ldcg(src), b = __ldcg(src + 1);
-        const long long pos = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
-        const long long cend = (long long)(((unsigned long long)(unsigned)a.w << 32) | (unsigned)a.z);
-        const int32_t m = b.x;
-        const unsigned long long got = ((unsigned long long)(unsigned)b.w << 32) | (unsigned)b.z;
-        if (got != tag || m < 0 || m > len || pos < -1 || pos >= T.max_pool || cend < 0 || cend > T.max_pool) {
-            if (lane == 0) set_status(T.st, RT_ERR_INVALID, 110);           // not a record of that match: the prompt is left out
-            continue;
-        }
-        int32_t node = 0, off = -1;                          // off < 0: the match ends on a node boundary (or at the root)
-        if (pos >= 0) {
-            const EndIndex X = end_index(T);
-            node = node_ending_at(X, pos, *reinterpret_cast<const volatile long long*>(&T.st->n_nodes));
-            if (node < 0) {
-                node = node_after(X, pos, cend);
-                if (node < 0) { if (lane == 0) set_status(T.st, RT_ERR_LIMIT, 111); continue; }      // cannot happen
-                off = m - __ldg(T.depth_start + node);
+    const EndIndex X = end_index(T);
+    for (unsigned long long p0 = (unsigned long long)((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * 32ULL; p0 < n_pending;
+         p0 += (unsigned long long)nwarps * 32ULL) {
+        const unsigned long long p = p0 + lane;
+        int32_t i = -1;
+        if (p < n_pending) i = A.pend_in[p];                 // < 0: a replay that stopped early, not processed
+        bool act = i >= 0, inside = false;
+        int32_t len = 0, m = 0, node = 0, off = -1;          // off < 0: the match ends on a node boundary (or at the root)
+        long long pos = -1, cend = 0;
+        if (act) {
+            len = (int32_t)(__ldg(A.off + i + 1) - __ldg(A.off + i));
+            const int4* src = reinterpret_cast<const int4*>(state + i);
+            const int4 a = __ldcg(src), b = __ldcg(src + 1);
+            pos = (long long)(((unsigned long long)(unsigned)a.y << 32) | (unsigned)a.x);
+            cend = (long long)(((unsigned long long)(unsigned)a.w << 32) | (unsigned)a.z);
+            m = b.x;
+            const unsigned long long got = ((unsigned long long)(unsigned)b.w << 32) | (unsigned)b.z;
+            if (got != tag || m < 0 || m > len || pos < -1 || pos >= T.max_pool || cend < 0 || cend > T.max_pool) {
+                set_status(T.st, RT_ERR_INVALID, 110);      // not a record of that match: the prompt is left out
+                act = false;
+            } else if (pos >= 0) {
+                node = node_ending_at(X, pos, *reinterpret_cast<const volatile long long*>(&T.st->n_nodes));
+                inside = node < 0;
             }
         }
-        if (lane == 0 && !(m == len && off < 0)) {
+        unsigned im = __ballot_sync(FULL_MASK, inside);
+        while (im) {
+            const int src = __ffs(im) - 1; im &= im - 1;
+            const int32_t r = node_after(X, __shfl_sync(FULL_MASK, pos, src), __shfl_sync(FULL_MASK, cend, src));
+            if (lane == src) {
+                if (r < 0) { set_status(T.st, RT_ERR_LIMIT, 111); act = false; }      // cannot happen
+                else { node = r; off = m - __ldg(T.depth_start + r); }
+            }
+        }
+        const bool pend = act && !(m == len && off < 0);
+        if (pend) {
             A.pm[i] = m; A.pnode[i] = node; A.poff[i] = off;
             if (off >= 0) atomicMin(&A.claim[node], i);
-            A.pend_out[atomicAdd(A.n_out, 1u)] = i;
+        }
+        const unsigned pm = __ballot_sync(FULL_MASK, pend);
+        if (pm) {
+            const int lead = __ffs(pm) - 1;
+            unsigned base = 0;
+            if (lane == lead) base = atomicAdd(A.n_out, (unsigned)__popc(pm));
+            base = __shfl_sync(FULL_MASK, base, lead);
+            if (pend) A.pend_out[base + __popc(pm & ((1u << lane) - 1u))] = i;
         }
     }
 }
 
-// What the apply step does for pending prompt number p of the list (one warp): cut the edge its match ends in if it
-// holds the claim, add its leaf if it wins the child's table slot, copy the leaf's tokens, or put the prompt on the
-// list for the next round.  Tree fields are read through L2 (__ldcg): inside the kernel that runs all later rounds,
-// another SM may have written them a moment ago.
-__device__ __forceinline__ void bulk_apply_one(const TreeDev& T, const BulkArgs& A, unsigned p, int lane,
-                                               unsigned long long* s_live_nodes, unsigned long long* s_live_tokens) {
+// What the apply step does for 32 pending prompts of the list (one per lane, from number p0 on): cut the edge the
+// match ends in if the prompt holds the claim, add its leaf if it wins the child's table slot, or put the prompt on
+// the list for the next round; then the warp copies the new leaves' tokens, one leaf after the other.  New nodes are
+// numbered and pool space is taken with one addition per warp.  Tree fields are read through L2 (__ldcg): inside the
+// kernel that runs all later rounds, another SM may have written them a moment ago.
+__device__ __forceinline__ void bulk_apply_warp(const TreeDev& T, const BulkArgs& A, unsigned long long p0, unsigned n_apply, int lane,
+                                                unsigned long long* s_live_nodes, unsigned long long* s_live_tokens) {
     TreeState* S = T.st;
-    const int32_t i = __ldcg(A.pend_out + p);
-    const int64_t lo = __ldg(A.off + i);
-    const int32_t len = (int32_t)(__ldg(A.off + i + 1) - lo);
-    const int32_t* x = A.tok + lo;
-    const int32_t m = __ldcg(A.pm + i), node = __ldcg(A.pnode + i), off = __ldcg(A.poff + i);
-    const int32_t unc = len - m;
-    int64_t dst = -1;
-    if (lane == 0) {
-        bool go = true, retry = false;
-        int32_t end = node;
-        if (off >= 0) {                                 // the match ends inside node's edge: cut it
-            if (__ldcg(A.claim + node) != i) { go = false; retry = true; }     // another prompt cuts this edge in this round
-            else {
-                A.claim[node] = 0x7fffffff;
-                const long long u = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
-                if (u >= T.max_nodes) { set_status(S, RT_ERR_CAPACITY); go = false; }
-                else {
-                    atomicAdd(s_live_nodes, 1ULL);
-                    const int32_t par = __ldcg(T.parent + node), ds = __ldcg(T.depth_start + node), sl = __ldcg(T.span_len + node);
-                    const int64_t so = __ldcg(T.span_off + node);
-                    const int32_t t_up = __ldcg(T.pool + so), t_low = __ldcg(T.pool + so + off);
-                    T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
-                    T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
-                    T.first_tok[u] = t_up; T.first_tok[node] = t_low;
-                    long long slot = table_find(T, par, t_up);
-                    int64_t chain_end = so + sl;
-                    if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = __ldcg(&T.table[slot].chain_end); }
-                    else set_status(S, RT_ERR_LIMIT, 104);
-                    T.end_node[so + off - 1] = (int32_t)u;
-                    T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
-                    T.parent[node] = (int32_t)u;
-                    end = (int32_t)u;
-                    // (u, first token of the lower part) -> node : nobody else can want this key
-                    unsigned long long key = make_key(end, t_low);
-                    unsigned long long sl2 = hash_key(key) & T.table_mask;
-                    for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
-                        if (atomicCAS(&T.table[sl2].key, 0ULL, key) == 0ULL) {
-                            T.table[sl2].child = node; T.table[sl2].span_len = sl - off; T.table[sl2].span_off = so + off;
-                            T.table[sl2].chain_end = chain_end;
-                            break;
-                        }
-                        sl2 = (sl2 + 1) & T.table_mask;
-                    }
-                }
-            }
-        }
-        if (go && unc > 0) {
-            unsigned long long key = make_key(end, __ldg(x + m));
-            unsigned long long sl2 = hash_key(key) & T.table_mask;
-            long long won = -1;
-            for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
-                unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
-                if (old == 0ULL) { won = (long long)sl2; break; }
-                if (old == key) { retry = true; break; }   // another prompt added that child (in this round, or it lost to it before)
-                sl2 = (sl2 + 1) & T.table_mask;
-            }
-            if (won >= 0) {
-                const long long leaf = (long long)atomicAdd((unsigned long long*)&S->n_nodes, 1ULL);
-                const long long raw = (long long)atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)(unc + 6));
-                const long long po = ((raw + 3) & ~3LL) + (m & 3);                  // span_off = depth_start (mod 4)
-                if (leaf >= T.max_nodes || raw + unc + 6 > T.max_pool) {
-                    set_status(S, RT_ERR_CAPACITY);
-                    T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0; T.table[won].chain_end = 0;
-                } else {
-                    T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
-                    T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
-                    T.first_tok[leaf] = __ldg(x + m);
-                    T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
-                    T.table[won].chain_end = po + unc;
-                    T.end_node[po + unc - 1] = (int32_t)leaf;
-                    atomicAdd(&T.nchild[end], 1);
-                    atomicAdd(s_live_tokens, (unsigned long long)unc);
-                    atomicAdd(s_live_nodes, 1ULL);
-                    dst = po;
-                }
-            }
-        }
-        if (retry) A.pend_next[atomicAdd(A.n_next, 1u)] = i;
+    const unsigned lt = (1u << lane) - 1u;
+    const bool act = p0 + lane < n_apply;
+    int32_t i = 0, len = 0, m = 0, node = 0, off = -1;
+    const int32_t* x = A.tok;
+    if (act) {
+        i = __ldcg(A.pend_out + p0 + lane);
+        const int64_t lo = __ldg(A.off + i);
+        len = (int32_t)(__ldg(A.off + i + 1) - lo);
+        x = A.tok + lo;
+        m = __ldcg(A.pm + i); node = __ldcg(A.pnode + i); off = __ldcg(A.poff + i);
     }
-    dst = __shfl_sync(FULL_MASK, dst, 0);
-    if (dst >= 0)
-        for (int32_t t = lane; t < unc; t += 32) T.pool[dst + t] = __ldg(x + m + t);
+    const int32_t unc = len - m;
+    bool go = act, retry = false;
+    int32_t end = node;
+    // ---- the match ends inside node's edge: cut it, unless another prompt cuts this edge in this round
+    bool cut = act && off >= 0;
+    if (cut && __ldcg(A.claim + node) != i) { cut = false; go = false; retry = true; }
+    const unsigned cm = __ballot_sync(FULL_MASK, cut);
+    if (cm) {
+        const int lead = __ffs(cm) - 1;
+        unsigned long long base = 0;
+        if (lane == lead) base = atomicAdd((unsigned long long*)&S->n_nodes, (unsigned long long)__popc(cm));
+        base = __shfl_sync(FULL_MASK, base, lead);
+        if (cut) {
+            const long long u = (long long)base + __popc(cm & lt);
+            A.claim[node] = 0x7fffffff;
+            if (u >= T.max_nodes) { set_status(S, RT_ERR_CAPACITY); go = false; }
+            else {
+                atomicAdd(s_live_nodes, 1ULL);
+                const int32_t par = __ldcg(T.parent + node), ds = __ldcg(T.depth_start + node), sl = __ldcg(T.span_len + node);
+                const int64_t so = __ldcg(T.span_off + node);
+                const int32_t t_up = __ldcg(T.pool + so), t_low = __ldcg(T.pool + so + off);
+                T.parent[u] = par; T.depth_start[u] = ds; T.span_off[u] = so; T.span_len[u] = off;
+                T.nchild[u] = 1; T.dead[u] = 0; T.last_access[u] = 0;
+                T.first_tok[u] = t_up; T.first_tok[node] = t_low;
+                long long slot = table_find(T, par, t_up);
+                int64_t chain_end = so + sl;
+                if (slot >= 0) { T.table[slot].child = (int32_t)u; T.table[slot].span_len = off; chain_end = __ldcg(&T.table[slot].chain_end); }
+                else set_status(S, RT_ERR_LIMIT, 104);
+                T.end_node[so + off - 1] = (int32_t)u;
+                T.span_off[node] = so + off; T.span_len[node] = sl - off; T.depth_start[node] = ds + off;
+                T.parent[node] = (int32_t)u;
+                end = (int32_t)u;
+                // (u, first token of the lower part) -> node : nobody else can want this key
+                unsigned long long key = make_key(end, t_low);
+                unsigned long long sl2 = hash_key(key) & T.table_mask;
+                for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+                    if (atomicCAS(&T.table[sl2].key, 0ULL, key) == 0ULL) {
+                        T.table[sl2].child = node; T.table[sl2].span_len = sl - off; T.table[sl2].span_off = so + off;
+                        T.table[sl2].chain_end = chain_end;
+                        break;
+                    }
+                    sl2 = (sl2 + 1) & T.table_mask;
+                }
+            }
+        }
+    }
+    // ---- the leaf: whoever puts the child's key into the table adds it
+    long long won = -1;
+    if (go && unc > 0) {
+        unsigned long long key = make_key(end, __ldg(x + m));
+        unsigned long long sl2 = hash_key(key) & T.table_mask;
+        for (unsigned long long pr = 0; pr <= T.table_mask; ++pr) {
+            unsigned long long old = atomicCAS(&T.table[sl2].key, 0ULL, key);
+            if (old == 0ULL) { won = (long long)sl2; break; }
+            if (old == key) { retry = true; break; }       // another prompt added that child (in this round, or it lost to it before)
+            sl2 = (sl2 + 1) & T.table_mask;
+        }
+    }
+    int64_t dst = -1;
+    const unsigned wm = __ballot_sync(FULL_MASK, won >= 0);
+    if (wm) {
+        const long long need = won >= 0 ? (long long)unc + 6 : 0;
+        long long inc = need;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const long long o = __shfl_up_sync(FULL_MASK, inc, d); if (lane >= d) inc += o; }
+        const long long tot = __shfl_sync(FULL_MASK, inc, 31);
+        unsigned long long nb = 0, pb = 0;
+        if (lane == 0) {
+            nb = atomicAdd((unsigned long long*)&S->n_nodes, (unsigned long long)__popc(wm));
+            pb = atomicAdd((unsigned long long*)&S->pool_used, (unsigned long long)tot);
+        }
+        nb = __shfl_sync(FULL_MASK, nb, 0); pb = __shfl_sync(FULL_MASK, pb, 0);
+        if (won >= 0) {
+            const long long leaf = (long long)nb + __popc(wm & lt);
+            const long long raw = (long long)pb + inc - need;
+            const long long po = ((raw + 3) & ~3LL) + (m & 3);                  // span_off = depth_start (mod 4)
+            if (leaf >= T.max_nodes || raw + unc + 6 > T.max_pool) {
+                set_status(S, RT_ERR_CAPACITY);
+                T.table[won].child = -1; T.table[won].span_len = 0; T.table[won].span_off = 0; T.table[won].chain_end = 0;
+            } else {
+                T.parent[leaf] = end; T.depth_start[leaf] = m; T.span_off[leaf] = po; T.span_len[leaf] = unc;
+                T.nchild[leaf] = 0; T.dead[leaf] = 0; T.last_access[leaf] = 0;
+                T.first_tok[leaf] = __ldg(x + m);
+                T.table[won].child = (int32_t)leaf; T.table[won].span_len = unc; T.table[won].span_off = po;
+                T.table[won].chain_end = po + unc;
+                T.end_node[po + unc - 1] = (int32_t)leaf;
+                atomicAdd(&T.nchild[end], 1);
+                atomicAdd(s_live_tokens, (unsigned long long)unc);
+                atomicAdd(s_live_nodes, 1ULL);
+                dst = po;
+            }
+        }
+    }
+    const unsigned rm = __ballot_sync(FULL_MASK, retry);
+    if (rm) {
+        const int lead = __ffs(rm) - 1;
+        unsigned base = 0;
+        if (lane == lead) base = atomicAdd(A.n_next, (unsigned)__popc(rm));
+        base = __shfl_sync(FULL_MASK, base, lead);
+        if (retry) A.pend_next[base + __popc(rm & lt)] = i;
+    }
+    // ---- the new leaves' tokens
+    unsigned dm = __ballot_sync(FULL_MASK, dst >= 0);
+    while (dm) {
+        const int src = __ffs(dm) - 1; dm &= dm - 1;
+        const int64_t d = __shfl_sync(FULL_MASK, dst, src);
+        const int32_t* xs = reinterpret_cast<const int32_t*>(__shfl_sync(FULL_MASK, (unsigned long long)(x + m), src));
+        const int32_t cnt = __shfl_sync(FULL_MASK, unc, src);
+        for (int32_t t0 = 0; t0 < cnt; t0 += 128) {
+            int32_t v[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) { const int32_t t = t0 + r * 32 + lane; v[r] = t < cnt ? __ldg(xs + t) : 0; }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) { const int32_t t = t0 + r * 32 + lane; if (t < cnt) T.pool[d + t] = v[r]; }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -3295,8 +3361,9 @@ bulk_apply_kernel(TreeDev T, BulkArgs A) {
     const unsigned n_pending = *A.n_out;
     const int lane = threadIdx.x & 31;
     const unsigned nwarps = (gridDim.x * blockDim.x) >> 5;
-    for (unsigned p = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; p < n_pending; p += nwarps)
-        bulk_apply_one(T, A, p, lane, &s_live_nodes, &s_live_tokens);
+    for (unsigned long long p0 = (unsigned long long)((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * 32ULL; p0 < n_pending;
+         p0 += (unsigned long long)nwarps * 32ULL)
+        bulk_apply_warp(T, A, p0, n_pending, lane, &s_live_nodes, &s_live_tokens);
     __syncthreads();
     if (threadIdx.x == 0) {
         if (s_live_nodes) atomicAdd((unsigned long long*)&T.st->live_nodes, s_live_nodes);
@@ -3397,7 +3464,8 @@ bulk_rounds_kernel(TreeDev T, BulkArgs A, BulkSync* g, long long n_total, const 
         // ---- cuts and leaves
         const unsigned n_apply = __ldcg(R.n_out);
         if (blockIdx.x == 0 && threadIdx.x == 0) { g->cnt_w[par ^ 1u] = 0u; g->cnt_a[par ^ 1u] = 0u; }     // the next round's
-        for (unsigned p = warp0; p < n_apply; p += nwarps) bulk_apply_one(T, R, p, lane, &s_live_nodes, &s_live_tokens);
+        for (unsigned long long p0 = (unsigned long long)warp0 * 32ULL; p0 < n_apply; p0 += (unsigned long long)nwarps * 32ULL)
+            bulk_apply_warp(T, R, p0, n_apply, lane, &s_live_nodes, &s_live_tokens);
         if (!bulk_barrier(g, S, limit_ns, [&] {
                 const bool stop = *(volatile int*)&S->status != 0 || r > 100000000u;
                 g->go = stop ? 0u : *(volatile unsigned*)&g->cnt_a[par];
