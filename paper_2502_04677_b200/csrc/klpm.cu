@@ -1725,6 +1725,7 @@ struct FastBatchIO {
     int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
     int32_t B0, nF0, nL0, limF, limL; // scratch
     int32_t wneed;                    // scratch: bitmap words from the oldest unprocessed slot on that hold the slots wanted
+    int32_t hard;                     // out: the batch stopped before a decision that needs the one-at-a-time path
     int32_t limB;                     // scratch: the batch must end before this decision (list entries that an oldest-first pick would meet)
 };
 #define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
@@ -1939,6 +1940,9 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         const int32_t B = lo >= KLPM_FAST_CTA_MIN ? lo : 0;
         const int32_t nF = f(B), nL = B - nF;
         io->B = B;
+        // stopped by a decision only the one-at-a-time path can take (not by the end of the entries, nor by a slot both
+        // kinds of turn reach: the next batch sorts that out)
+        io->hard = B > 0 && B < io->B0 && (f(B + 1) > io->limF || B + 1 - f(B + 1) > io->limL) ? 1 : 0;
         io->consumed = nL > 0 ? sEpos[nL - 1] + 1 : 0;
         io->hmax = nF > 0 ? sH[nF - 1] : -1;
     }
@@ -2879,7 +2883,7 @@ fast_run_kernel(FastArgs A) {
                 if (fh == fl && B - fl == limL && fl <= limF && (fl == 0 || last_h < soft)) { ++B; ++limL; }
             }
             if (B < 2) return false;
-            tb_cut = B < B0;
+            tb_cut = B < B0 && soft < 0;
             const int32_t nF = __shfl_sync(FULL_MASK, f_hi, B - 1), nL = B - nF;
             const int32_t hmax = nF > 0 ? __shfl_sync(FULL_MASK, hs, nF - 1) : -1;
             if (lane < nF) s_H[lane] = hs;
@@ -2934,7 +2938,7 @@ fast_run_kernel(FastArgs A) {
                     ++n_cta_ok; dec_cta += Bc;
                     const int32_t consumed = s_bio.consumed, hmax = s_bio.hmax;
                     c += Bc;
-                    one_next = Bc < s_bio.B0;
+                    one_next = s_bio.hard != 0;
                     if (A.policy == KLPM_POLICY_KLPM) cyc = (cyc + Bc) % A.k;
                     if (consumed) { cur += consumed; window(cur & ~31, &wk, &ws); window((cur & ~31) + 32, &nk, &ns); }
                     if (hmax >= 0) { head = hmax; advance_head(); }
