@@ -1726,6 +1726,7 @@ struct FastBatchIO {
     int32_t B0, nF0, nL0, limF, limL; // scratch
     int32_t wneed;                    // scratch: bitmap words from the oldest unprocessed slot on that hold the slots wanted
     int32_t hard;                     // out: the batch stopped before a decision that needs the one-at-a-time path
+    int32_t Braw;                     // out: decisions the batch could have made (it makes none below KLPM_FAST_CTA_MIN)
     int32_t limB;                     // scratch: the batch must end before this decision (list entries that an oldest-first pick would meet)
 };
 #define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
@@ -1937,6 +1938,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     __syncthreads();
     if (tid == 0) {
         const int32_t lo = io->B;
+        io->Braw = lo;
         const int32_t B = lo >= KLPM_FAST_CTA_MIN ? lo : 0;
         const int32_t nF = f(B), nL = B - nF;
         io->B = B;
@@ -2914,6 +2916,7 @@ fast_run_kernel(FastArgs A) {
         };
         int32_t vb_wait = 0, vb_back = 1;                   // decisions until the next attempt; doubles while attempts fail
         int32_t cb_wait = 0, cb_back = 8;                   // the same for the CTA-wide batch (loop iterations; 8 .. 1,024)
+        int32_t cb_until = 0, cb_fail = 0;                  // after an attempt that made no decision: not before decision cb_until; attempts failed in a row
         int32_t calm = KLPM_FAST_CALM;                      // consecutive full warp-wide steps: the CTA-wide batch is tried in calm water only
         long long n_cta_try = 0, n_cta_ok = 0, dec_cta = 0, n_warp_ok = 0, dec_warp = 0, dec_one = 0, cy_cta = 0, cy_warp = 0;
         // a batch that was cut short stopped before a decision only the one-at-a-time path can take: that one comes
@@ -2921,7 +2924,7 @@ fast_run_kernel(FastArgs A) {
         bool one_next = false;
         while (c < n && !failed) {
             // first choice: the whole CTA makes up to 1,024 decisions (the sort scratch is free between dissolves)
-            if (!one_next && cb_wait <= 0 && calm >= KLPM_FAST_CALM && n - c >= KLPM_FAST_CTA_MIN) {
+            if (!one_next && cb_wait <= 0 && calm >= KLPM_FAST_CALM && c >= cb_until && n - c >= KLPM_FAST_CTA_MIN) {
                 if (lane == 0) {
                     s_bio.cur = cur; s_bio.head = head; s_bio.c = c; s_bio.cyc = cyc; s_bio.root = root; s_bio.B = 0;
                     s_job.type = FAST_JOB_BATCH;
@@ -2945,16 +2948,17 @@ fast_run_kernel(FastArgs A) {
                     else if (head < n && ((bm_ld(s_done, head >> 5, gdone) >> (head & 31)) & 1u)) advance_head();
                     // did it pay?  its cycles per decision against what the warp-wide steps have cost per decision so far
                     const long long warp_cpd = dec_warp >= 256 ? cy_warp / dec_warp : 100;
-                    if (cy_this <= (long long)Bc * warp_cpd) { cb_back = 8; continue; }
+                    if (cy_this <= (long long)Bc * warp_cpd) { cb_back = 8; cb_fail = 0; continue; }
                     // committed, but too short to have paid for the attempt: warp-wide steps for a while, as after a failure
                     cb_wait = cb_back;
                     cb_back = cb_back < KLPM_FAST_CB_MAX ? cb_back * 2 : KLPM_FAST_CB_MAX;
                     calm = 0;
                     continue;
                 }
-                cb_wait = cb_back;
-                cb_back = cb_back < KLPM_FAST_CB_MAX ? cb_back * 2 : KLPM_FAST_CB_MAX;
-                calm = 0;
+                // too few decisions before one that needs the one-at-a-time path: the next attempt waits until that one has
+                // been made (and longer when attempts keep failing: such decisions come in runs)
+                cb_until = c + s_bio.Braw + 1 + (cb_fail > 0 ? (8 << cb_fail) : 0);
+                if (cb_fail < 6) ++cb_fail;
             }
             --cb_wait;
             if (!one_next && vb_wait <= 0) {
