@@ -3822,11 +3822,33 @@ __global__ void bitonic_step_kernel(long long* key, int32_t* idx, long long np2,
     }
 }
 
-// The steps of the same sort whose partner distance fits a tile of 2,048 pairs, done in shared memory: all stages
+// Two steps of one stage in one pass (partner distances j and j / 2): a thread holds the four entries that differ in
+// those two bits.
+__global__ void bitonic_step2_kernel(long long* key, int32_t* idx, long long np2, long long k, long long j) {
+    const long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= (np2 >> 2)) return;
+    const long long j2 = j >> 1;
+    const long long i0 = ((u & ~(j2 - 1)) << 2) | (u & (j2 - 1));      // u's bits with the two (adjacent) bit positions left out
+    long long kk[4]; int32_t ii[4];
+    const long long pos[4] = {i0, i0 | j2, i0 | j, i0 | j | j2};
+#pragma unroll
+    for (int r = 0; r < 4; ++r) { kk[r] = key[pos[r]]; ii[r] = idx[pos[r]]; }
+    const bool up = (i0 & k) == 0;
+    auto cx = [&](int x, int y) {
+        const bool gt = kk[x] > kk[y] || (kk[x] == kk[y] && ii[x] > ii[y]);
+        if (gt == up) { const long long tk = kk[x]; kk[x] = kk[y]; kk[y] = tk; const int32_t ti = ii[x]; ii[x] = ii[y]; ii[y] = ti; }
+    };
+    cx(0, 2); cx(1, 3);
+    cx(0, 1); cx(2, 3);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) { key[pos[r]] = kk[r]; idx[pos[r]] = ii[r]; }
+}
+
+// The steps of the same sort whose partner distance fits a tile of 4,096 pairs, done in shared memory: all stages
 // k_lo .. k_hi when those are at most the tile (the start of the sort), otherwise the tail (distances below the
 // tile) of the one stage k_lo = k_hi.
-#define KLPM_SORT_TILE 2048
-__global__ void __launch_bounds__(512)
+#define KLPM_SORT_TILE 4096
+__global__ void __launch_bounds__(1024)
 bitonic_tile_kernel(long long* key, int32_t* idx, long long np2, long long k_lo, long long k_hi) {
     __shared__ long long sk[KLPM_SORT_TILE];
     __shared__ int32_t si[KLPM_SORT_TILE];
@@ -3855,10 +3877,13 @@ bitonic_tile_kernel(long long* key, int32_t* idx, long long np2, long long k_lo,
 void sort_pairs(long long* key, int32_t* idx, long long np2, cudaStream_t s) {
     const long long T = np2 < KLPM_SORT_TILE ? np2 : KLPM_SORT_TILE;
     const unsigned tiles = (unsigned)(np2 / T), blocks = (unsigned)((np2 + 255) / 256);
-    if (T >= 2) bitonic_tile_kernel<<<tiles, 512, 0, s>>>(key, idx, np2, 2, T);
+    const unsigned blocks4 = (unsigned)(((np2 >> 2) + 255) / 256);
+    if (T >= 2) bitonic_tile_kernel<<<tiles, 1024, 0, s>>>(key, idx, np2, 2, T);
     for (long long k = T << 1; k <= np2; k <<= 1) {
-        for (long long j = k >> 1; j >= T; j >>= 1) bitonic_step_kernel<<<blocks, 256, 0, s>>>(key, idx, np2, k, j);
-        bitonic_tile_kernel<<<tiles, 512, 0, s>>>(key, idx, np2, k, k);
+        long long j = k >> 1;
+        for (; (j >> 1) >= T; j >>= 2) bitonic_step2_kernel<<<blocks4, 256, 0, s>>>(key, idx, np2, k, j);
+        if (j >= T) bitonic_step_kernel<<<blocks, 256, 0, s>>>(key, idx, np2, k, j);
+        bitonic_tile_kernel<<<tiles, 1024, 0, s>>>(key, idx, np2, k, k);
     }
 }
 
