@@ -1723,8 +1723,8 @@ struct FastBatchIO {
     int32_t cur, head, c, cyc;        // in: list cursor, oldest unprocessed slot, decisions made, c mod k
     unsigned long long root;          // in: largest key in the tournament
     int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
-    int32_t B0, nF0, nL0, limF, limL; // scratch
-    int32_t wneed;                    // scratch: bitmap words from the oldest unprocessed slot on that hold the slots wanted
+    int32_t B0, Bmax, limF, limL;     // scratch
+    int32_t B0out;                    // out: decisions the entries in sight would have allowed
     int32_t hard;                     // out: the batch stopped before a decision that needs the one-at-a-time path
     int32_t Braw;                     // out: decisions the batch could have made (it makes none below KLPM_FAST_CTA_MIN)
     int32_t limB;                     // scratch: the batch must end before this decision (list entries that an oldest-first pick would meet)
@@ -1825,7 +1825,8 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
             if (rem >= A.k) { rem -= A.k; ++q; }
         }
     }
-    if (tid == 0) { io->B0 = 0; io->B = 0; }
+    // the limits start open; every thread reads them capped by what the batch can hold
+    if (tid == 0) { io->B0 = 0; io->Bmax = 0; io->limF = 0x7fffffff; io->limL = 0x7fffffff; io->limB = 0x7fffffff; }
     auto f = [&](int32_t x) -> int32_t { return sF[x]; };
     // those of the entries that still count
     int32_t cnt = 0;
@@ -1835,8 +1836,24 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         ok[r] = idx < n && !((bm_ld(R.skip, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u);
         cnt += ok[r];
     }
-    int32_t avail;
-    const int32_t base = block_excl_scan(cnt, s_w, &avail);      // (its barriers also publish sF and the cleared io fields)
+    // the unprocessed slots from `head` on, one bitmap word per thread
+    const int32_t w0 = head >> 5;
+    unsigned fr;
+    {
+        const int32_t wi = w0 + tid;
+        unsigned w = wi < nwords ? bm_ld(R.done, wi, R.g_done) : 0xffffffffu;
+        if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
+        if (wi == w0) w |= (1u << (head & 31)) - 1u;
+        fr = ~w;
+    }
+    // both prefix sums with one scan: usable entries (at most 1,024) in the low half, free slots (at most 8,192) above
+    int32_t both;
+    const int32_t base2 = block_excl_scan(cnt + (__popc(fr) << 16), s_w, &both);    // (its barriers also publish sF and the limits)
+    const int32_t base = base2 & 0xffff, qk = base2 >> 16;
+    const int32_t avail = both & 0xffff, nfree = both >> 16;
+    int32_t* sP = sF + KLPM_FAST_CTA_BATCH + 8;             // per word: free slots before it
+    unsigned* sFr = reinterpret_cast<unsigned*>(sP + KLPM_FAST_THREADS);
+    sP[tid] = qk; sFr[tid] = fr;
     {   // as many decisions as those entries allow: the largest x with x - f(x) <= avail, every thread trying four values
         const int32_t hi = n - c < KLPM_FAST_CTA_BATCH ? n - c : KLPM_FAST_CTA_BATCH;
         int32_t best = 0;
@@ -1846,36 +1863,13 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         if ((tid & 31) == 0 && best > 0) atomicMax(&io->B0, best);
     }
     __syncthreads();
-    if (tid == 0) {
-        const int32_t lo = io->B0;
-        io->nF0 = f(lo); io->nL0 = lo - f(lo);
-        io->limF = io->nF0; io->limL = io->nL0; io->limB = lo;
-    }
-    __syncthreads();
-    const int32_t B0 = io->B0, nF0 = io->nF0, nL0 = io->nL0;
-    // the next nF0 unprocessed slots (each thread one bitmap word from head on), in order
-    int32_t hmax0 = -1, nFa0 = 0;
-    if (nF0 > 0) {
-        const int32_t w0 = head >> 5, wi = w0 + tid;
-        unsigned w = wi < nwords ? bm_ld(R.done, wi, R.g_done) : 0xffffffffu;
-        if (wi == nwords - 1 && (n & 31)) w |= ~((1u << (n & 31)) - 1u);
-        if (wi == w0) w |= (1u << (head & 31)) - 1u;
-        const unsigned fr = ~w;
-        int32_t nfree;
-        const int32_t qk = block_excl_scan(__popc(fr), s_w, &nfree);
-        // every word's free slots and how many lie before it; the word that holds the last slot wanted says how far to go
-        int32_t* sP = sF + KLPM_FAST_CTA_BATCH + 8;
-        unsigned* sFr = reinterpret_cast<unsigned*>(sP + KLPM_FAST_THREADS);
-        sP[tid] = qk; sFr[tid] = fr;
-        const int32_t nFa = nfree < nF0 ? nfree : nF0;
-        if (nFa > 0 && qk < nFa && qk + __popc(fr) >= nFa) io->wneed = tid + 1;
-        if (tid == 0 && nFa < nF0) io->limF = nFa;
-        __syncthreads();
-        // a thread per slot, eight words at a time: the slot's rank among the free ones is where it goes; one whose key
-        // sits in the tournament or that is grouped needs the careful step
-        const int32_t wneed = nFa > 0 ? io->wneed : 0;
+    const int32_t B0 = io->B0, nF0 = f(B0), nL0 = B0 - nF0;
+    const int32_t nFa = nfree < nF0 ? nfree : nF0;          // oldest-first picks there are slots for
+    // the next nFa unprocessed slots in order: a thread per slot, eight words at a time; the slot's rank among the free
+    // ones is where it goes; one whose key sits in the tournament or that is grouped needs the careful step
+    {
         const int bit = tid & 31;
-        for (int32_t wl = tid >> 5; wl < wneed; wl += KLPM_FAST_THREADS / 32) {
+        for (int32_t wl = tid >> 5; wl < KLPM_FAST_THREADS && sP[wl] < nFa; wl += KLPM_FAST_THREADS / 32) {
             const unsigned fw = sFr[wl];
             if ((fw >> bit) & 1u) {
                 const int32_t rank = sP[wl] + __popc(fw & ((1u << bit) - 1u));
@@ -1886,10 +1880,9 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
                 }
             }
         }
-        __syncthreads();
-        if (nFa > 0) hmax0 = sH[nFa - 1];
-        nFa0 = nFa;
     }
+    __syncthreads();
+    const int32_t hmax0 = nFa > 0 ? sH[nFa - 1] : -1;
     // The usable entries by rank.  One that is grouped or lies below the tournament's root stops the batch before its
     // turn.  One whose slot is among the slots the oldest-first picks of a full batch would take (rank phi there) is
     // taken by whichever side reaches it first, and the other side must not get as far as it inside this batch: the
@@ -1905,7 +1898,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
                     if ((((bm_ld(R.gb, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u)) || root > ek) {
                         atomicMin(&io->limL, rk);
                     } else if (es[r] >= head && es[r] <= hmax0) {
-                        int32_t lo = 0, hi = nFa0;                       // phi: slots of sH before this one
+                        int32_t lo = 0, hi = nFa;                        // phi: slots of sH before this one
                         while (lo < hi) { const int32_t mid = (lo + hi) >> 1; if (sH[mid] < es[r]) lo = mid + 1; else hi = mid; }
                         const int32_t phi = lo;
                         // decision of the oldest-first turn of rank phi, and of the longest-match turn of rank rk
@@ -1927,29 +1920,27 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         }
     }
     __syncthreads();
+    // the limits, capped by what the batch holds
+    const int32_t limF = io->limF < nFa ? io->limF : nFa, limL = io->limL < nL0 ? io->limL : nL0, limB = io->limB < B0 ? io->limB : B0;
     {   // the largest x that respects the three limits, every thread trying four values
-        const int32_t limF = io->limF, limL = io->limL, limB = io->limB;
         int32_t best = 0;
 #pragma unroll
-        for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= B0 && x <= limB && f(x) <= limF && x - f(x) <= limL) best = x; }
+        for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= limB && f(x) <= limF && x - f(x) <= limL) best = x; }
         best = __reduce_max_sync(FULL_MASK, best);
-        if ((tid & 31) == 0 && best > 0) atomicMax(&io->B, best);
+        if ((tid & 31) == 0 && best > 0) atomicMax(&io->Bmax, best);
     }
     __syncthreads();
+    const int32_t Braw = io->Bmax;
+    const int32_t B = Braw >= KLPM_FAST_CTA_MIN ? Braw : 0;     // nothing is changed by a batch too short to pay
     if (tid == 0) {
-        const int32_t lo = io->B;
-        io->Braw = lo;
-        const int32_t B = lo >= KLPM_FAST_CTA_MIN ? lo : 0;
         const int32_t nF = f(B), nL = B - nF;
-        io->B = B;
-        // stopped by a decision only the one-at-a-time path can take (not by the end of the entries, nor by a slot both
-        // kinds of turn reach: the next batch sorts that out)
-        io->hard = B > 0 && B < io->B0 && (f(B + 1) > io->limF || B + 1 - f(B + 1) > io->limL) ? 1 : 0;
+        io->B = B; io->Braw = Braw; io->B0out = B0;
         io->consumed = nL > 0 ? sEpos[nL - 1] + 1 : 0;
         io->hmax = nF > 0 ? sH[nF - 1] : -1;
+        // stopped by a decision only the one-at-a-time path can take (not by the end of the entries, nor by a slot both
+        // kinds of turn reach: the next batch sorts that out)
+        io->hard = B > 0 && B < B0 && (f(B + 1) > limF || B + 1 - f(B + 1) > limL) ? 1 : 0;
     }
-    __syncthreads();
-    const int32_t B = io->B;
     for (int32_t x = tid; x < B; x += KLPM_FAST_THREADS) {   // thread makes decisions c + x
         const int32_t f0 = f(x);
         const int32_t slot = f(x + 1) > f0 ? sH[f0] : sE[x - f0];
