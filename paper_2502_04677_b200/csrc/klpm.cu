@@ -2975,14 +2975,21 @@ fast_run_kernel(FastArgs A) {
             } else {
                 unsigned long long ek = 0;                  // next entry of the list that still counts
                 int32_t es = -1;
-                while (cur < n) {
-                    const int src = cur & 31;
-                    const long long kk = __shfl_sync(FULL_MASK, wk, src);
-                    es = __shfl_sync(FULL_MASK, ws, src);
-                    if (!((bm_ld(R.skip, es >> 5, gbits) >> (es & 31)) & 1u)) { ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL); break; }
-                    es = -1;
-                    advance_cur();
+                while (cur < n) {                           // (a window's 32 entries are examined at once: stale entries come in runs)
+                    const int32_t wbase = cur & ~31;
+                    const bool usable = lane >= (cur & 31) && (long long)wbase + lane < n && !((bm_ld(R.skip, ws >> 5, gbits) >> (ws & 31)) & 1u);
+                    const unsigned bal = __ballot_sync(FULL_MASK, usable);
+                    if (bal) {
+                        const int src = __ffs(bal) - 1;
+                        cur = wbase + src;
+                        const long long kk = __shfl_sync(FULL_MASK, wk, src);
+                        es = __shfl_sync(FULL_MASK, ws, src);
+                        ek = ~((unsigned long long)kk ^ 0x8000000000000000ULL);
+                        break;
+                    }
+                    cur = wbase + 32; wk = nk; ws = ns; window(cur + 32, &nk, &ns);
                 }
+                if (cur > n) cur = n;
                 if (root > ek) {
                     const unsigned rk = 0xffffffffu - (unsigned)(root & 0xffffffffULL);
                     j = A.pinv ? __ldg(A.pinv + rk) : (int32_t)rk;
