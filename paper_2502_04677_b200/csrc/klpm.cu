@@ -1736,6 +1736,9 @@ struct FastBatchIO {
 #ifndef KLPM_FAST_CB_MAX
 #define KLPM_FAST_CB_MAX 32           // longest back-off (loop iterations) after CTA-wide attempts that failed
 #endif
+#ifndef KLPM_FAST_FAIL_CAP
+#define KLPM_FAST_FAIL_CAP 6          // failed CTA-wide attempts in a row that still lengthen the wait (8 << that many decisions)
+#endif
 #ifndef KLPM_FAST_CALM
 #define KLPM_FAST_CALM 1              // full warp-wide steps in a row before a CTA-wide batch is tried again
 #endif
@@ -2949,7 +2952,7 @@ fast_run_kernel(FastArgs A) {
                 // too few decisions before one that needs the one-at-a-time path: the next attempt waits until that one has
                 // been made (and longer when attempts keep failing: such decisions come in runs)
                 cb_until = c + s_bio.Braw + 1 + (cb_fail > 0 ? (8 << cb_fail) : 0);
-                if (cb_fail < 6) ++cb_fail;
+                if (cb_fail < KLPM_FAST_FAIL_CAP) ++cb_fail;
             }
             --cb_wait;
             if (!one_next && vb_wait <= 0) {
