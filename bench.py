@@ -31,14 +31,26 @@ FALLBACK_HBM_GBS = 6650.0
 DEFAULT_WORKLOAD = "adversarial"
 
 # DRAM bytes (read + write) per launch of the match kernel, from an ncu capture: keyed by (workload, scale), with the
-# SHA-256 of the kernel source the capture was taken on.  Reported only while the source is still that one.
+# SHA-256 of the match path's source the capture was taken on (everything the kernel is compiled from and its launch).
+# Reported only while that source is still the same.
 TRAFFIC = {}
+
+MATCH_SOURCE_END = "// sequential processing of prompts by one CTA: rt_insert and klpm_replay"
+MATCH_LAUNCH_BEGIN = "// The batched match: the order in which the queries are taken, then the kernel."
+MATCH_LAUNCH_END = "}  // namespace"
 
 
 def kernel_source_sha() -> str:
+    """Hash of the part of the CUDA source the batched match is built from: the file up to the first section that
+    belongs to something else (tree layout, loads, hash table, walks, the order kernels, the match kernels) and the
+    host function that launches it."""
     import hashlib
-    with open(os.path.join(ROOT, "paper_2502_04677_b200", "csrc", "klpm.cu"), "rb") as f:
-        return hashlib.sha256(f.read()).hexdigest()
+    with open(os.path.join(ROOT, "paper_2502_04677_b200", "csrc", "klpm.cu"), "r") as f:
+        text = f.read()
+    a = text.index(MATCH_SOURCE_END)
+    b = text.index(MATCH_LAUNCH_BEGIN)
+    c = text.index(MATCH_LAUNCH_END, b)
+    return hashlib.sha256((text[:a] + text[b:c]).encode()).hexdigest()
 
 
 def measured_traffic(name: str, scale: float):
@@ -351,9 +363,10 @@ def run_ours(args):
         np2 <<= 1
     lg = np2.bit_length() - 1
     run_path = K.klpm_run_path(tree)
-    # one sort: the stages up to a tile of 2,048 pairs in one launch, then per larger stage its global steps and one tile launch
-    big = max(0, lg - 11)
-    sort_launches = 1 + big * (big + 1) // 2 + big
+    # one sort: the stages up to a tile of 4,096 pairs in one launch, then per larger stage its global steps (two per
+    # launch, a single one where their number is odd) and one tile launch
+    big = max(0, lg - 12)
+    sort_launches = 1 + sum((st + 1) // 2 + 1 for st in range(1, big + 1))
     if run_path == K.RUN_PATH_GROUPED and w.budget_tokens > 0:
         # bucketing + match; slot keys, arrival sort, slot arrays; clears, capacity check (2), slot records, slot states,
         # group sort, groups, the loop; tokens of the surviving nodes, table clear, table
@@ -367,16 +380,16 @@ def run_ours(args):
                      "that are still alive are written after the loop; bound by the latency of the dependent loads of one warp")
     elif run_path == K.RUN_PATH_GROUPED:
         # match (bucketing by first token: three kernels; the match itself); slot keys, arrival sort, slot arrays; slot
-        # records, slot states from the match records, group sort, groups, key list and its sort (queues up to
-        # 262,144), the loop; bulk insertion of the processed prompts: claim words, pending list, at least one round
+        # records, slot states from the match records, group sort, groups, key list and its sort, the loop, the three
+        # charge kernels; bulk insertion of the processed prompts: claim words, pending list, at least one round
         # of two kernels, clock
-        list_launches = 1 + sort_launches + 3 if nq <= 262144 else 0       # key list, its sort, the three charge kernels
+        list_launches = 1 + sort_launches + 3                               # key list, its sort, the three charge kernels
         order_launches = 3 if nq >= 2048 else 0
         launches_per_step = (order_launches + 1) + (1 + sort_launches + 1) + (1 + 1 + sort_launches + 1 + list_launches + 1) + (1 + 1 + 2 + 1)
         loop_kernel = "fast_run_kernel"
         loop_note = ("all decisions in one CTA: once everybody has arrived, longest-match picks come from a presorted list "
-                     "of keys and oldest-first picks from a bitmap cursor, up to 32 decisions per warp-wide step when they "
-                     "cannot interfere; picks whose group has other members take a careful step; those decisions are "
+                     "of keys and oldest-first picks from a bitmap cursor, up to 1,024 decisions per CTA-wide batch (32 per "
+                     "warp-wide step) when they cannot interfere; picks whose group has other members take a careful step; those decisions are "
                      "charged by a parallel pass after the loop; bound by the instruction issue of one warp; the loop starts "
                      "from the records rt_match_batch_ex kept (no query is walked twice); the time includes three sorts "
                      "and the bulk insertion of the processed prompts")
