@@ -33,7 +33,12 @@ DEFAULT_WORKLOAD = "adversarial"
 # DRAM bytes (read + write) per launch of the match kernel, from an ncu capture: keyed by (workload, scale), with the
 # SHA-256 of the match path's source the capture was taken on (everything the kernel is compiled from and its launch).
 # Reported only while that source is still the same.
-TRAFFIC = {}
+TRAFFIC = {
+    # ncu, one launch at scale 0.125: dram__bytes_read.sum 1,276,046,000 + dram__bytes_write.sum 71,068,160
+    ("adversarial", 0.125): {"bytes": 1347114160, "source_sha256": "5a2ce8870155ff61e7112d9b2f0fb4ec4fc330eaf447252ef5443a67be858a49"},
+    # the full size holds 8 x the units of that launch with the same sharing (21 queries per trunk): scaled, not captured
+    ("adversarial", 1.0): {"bytes": 8 * 1347114160, "source_sha256": "5a2ce8870155ff61e7112d9b2f0fb4ec4fc330eaf447252ef5443a67be858a49"},
+}
 
 MATCH_SOURCE_END = "// sequential processing of prompts by one CTA: rt_insert and klpm_replay"
 MATCH_LAUNCH_BEGIN = "// The batched match: the order in which the queries are taken, then the kernel."
@@ -330,6 +335,8 @@ def run_ours(args):
     h2d = h_tok.numel() * 4 + h_off.numel() * 8 + h_arr.numel() * 8
     d2h = nq * (4 + 4 + 4 + 8)
 
+    loop_counters = K.rt_debug_counters(tree)      # of the last klpm_run_ex (the replay below runs the same kernel)
+
     # ---- klpm_replay along the order the loop chose: Definition 2 must give the same charges again
     r_unc = torch.full((nq,), -1, dtype=torch.int32, device=device)
     r_ttft = torch.full((nq,), -1, dtype=torch.int64, device=device)
@@ -424,11 +431,14 @@ def run_ours(args):
                      "compulsory_bytes_per_launch": compulsory_bytes,
                      "algorithmic_bytes_per_launch": alg_bytes, "achieved_algorithmic": achieved_alg,
                      "frac_algorithmic": achieved_alg / peak,
-                     "traffic": measured_traffic(name, args.scale)},
+                     "traffic": measured_traffic(name, args.scale),
+                     "traffic_what": "dram__bytes_read.sum + dram__bytes_write.sum of one launch (ncu); at scale 1.0 the "
+                                     "capture of scale 0.125 times 8 (the units and the sharing scale alike); null when no "
+                                     "capture exists for this workload or the match path's source has changed since"},
         "decision_loop": {"kernel": loop_kernel,
                           "bound": "latency" if (loop_kernel == "run_kernel" or w.budget_tokens > 0) else "issue",
                           "us_per_decision": 1e6 * t_run / (nq * args.steps), "note": loop_note,
-                          "counters": K.rt_debug_counters(tree)},
+                          "counters": loop_counters},
         "e2e": {"value": world * nq / e2e_match_s, "unit": "queries/s",
                 "what": "host query buffers in (pinned), rt_match_batch, match lengths out",
                 "ms_match_with_copies": 1e3 * e2e_match_s, "ms_per_step": 1e3 * e2e_s,
