@@ -1724,6 +1724,7 @@ struct FastBatchIO {
     unsigned long long root;          // in: largest key in the tournament
     int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
     int32_t B0, Bmax, limF, limL;     // scratch
+    unsigned long long col1;          // scratch: the first slot that both kinds of turn reach (decision, who is first, its two ranks)
     int32_t B0out;                    // out: decisions the entries in sight would have allowed
     int32_t hard;                     // out: the batch stopped before a decision that needs the one-at-a-time path
     int32_t Braw;                     // out: decisions the batch could have made (it makes none below KLPM_FAST_CTA_MIN)
@@ -1829,7 +1830,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         }
     }
     // the limits start open; every thread reads them capped by what the batch can hold
-    if (tid == 0) { io->B0 = 0; io->Bmax = 0; io->limF = 0x7fffffff; io->limL = 0x7fffffff; io->limB = 0x7fffffff; }
+    if (tid == 0) { io->B0 = 0; io->Bmax = 0; io->limF = 0x7fffffff; io->limL = 0x7fffffff; io->limB = 0x7fffffff; io->col1 = ~0ULL; }
     auto f = [&](int32_t x) -> int32_t { return sF[x]; };
     // those of the entries that still count
     int32_t cnt = 0;
@@ -1867,7 +1868,14 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     }
     __syncthreads();
     const int32_t B0 = io->B0, nF0 = f(B0), nL0 = B0 - nF0;
-    const int32_t nFa = nfree < nF0 ? nfree : nF0;          // oldest-first picks there are slots for
+    // One slot and one entry more than a full batch takes are looked at: where the two pick orders meet once inside the
+    // batch (a slot that is both among the oldest unprocessed and among the next list entries), the side that comes
+    // later passes over it and takes one more of its own.
+    const bool both_kinds = A.policy == KLPM_POLICY_KLPM;
+    const int32_t nFw = both_kinds && nF0 < KLPM_FAST_CTA_BATCH ? nF0 + 1 : nF0;
+    const int32_t nLw = both_kinds && nL0 < KLPM_FAST_CTA_BATCH ? nL0 + 1 : nL0;
+    const int32_t nFa = nfree < nFw ? nfree : nFw;          // oldest-first picks there are slots for
+    const int32_t nEa = avail < nLw ? avail : nLw;          // longest-match picks there are entries for
     // the next nFa unprocessed slots in order: a thread per slot, eight words at a time; the slot's rank among the free
     // ones is where it goes; one whose key sits in the tournament or that is grouped needs the careful step
     {
@@ -1887,15 +1895,18 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     __syncthreads();
     const int32_t hmax0 = nFa > 0 ? sH[nFa - 1] : -1;
     // The usable entries by rank.  One that is grouped or lies below the tournament's root stops the batch before its
-    // turn.  One whose slot is among the slots the oldest-first picks of a full batch would take (rank phi there) is
-    // taken by whichever side reaches it first, and the other side must not get as far as it inside this batch: the
-    // batch ends before the later of the two decisions (its own longest-match turn, the oldest-first turn of rank phi).
+    // turn.  One whose slot is among the slots the oldest-first picks would take (rank phi there) is taken by whichever
+    // side reaches it first.  The first such meeting (the one whose earlier decision comes first) is resolved inside
+    // the batch: the other side passes over the slot, its later picks move up by one.  The batch ends well before any
+    // further meeting: k + 1 decisions before the earlier of its two decisions as computed without the shift, which
+    // moves a decision forward by at most k -- or before the later of its two decisions where those are far enough
+    // apart for the shift not to change their order (the earlier one is an ordinary pick then).
     {
         int32_t rk = base;
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             if (ok[r]) {
-                if (rk < nL0) {
+                if (rk < nEa) {
                     sE[rk] = es[r]; sEpos[rk] = tid * 4 + r;
                     const unsigned long long ek = ~((unsigned long long)kk[r] ^ 0x8000000000000000ULL);
                     if ((((bm_ld(R.gb, es[r] >> 5, R.g_bits) >> (es[r] & 31)) & 1u)) || root > ek) {
@@ -1915,7 +1926,22 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
                             while (a0 < a1) { const int32_t mid = (a0 + a1) >> 1; if (mid + 1 - f(mid + 1) > rk) a1 = mid; else a0 = mid + 1; }
                             xL = a0;
                         }
-                        atomicMin(&io->limB, xF > xL ? xF : xL);
+                        if (!both_kinds) {
+                            atomicMin(&io->limB, xF > xL ? xF : xL);
+                        } else {
+                            const int32_t tmin = xF < xL ? xF : xL, tmax0 = xF < xL ? xL : xF, tmax = tmax0 < 4095 ? tmax0 : 4095;
+                            const unsigned long long pack = ((unsigned long long)tmin << 52) | ((unsigned long long)tmax << 40) |
+                                                            ((unsigned long long)(xL < xF ? 1 : 0) << 30) | ((unsigned long long)phi << 16) | (unsigned long long)rk;
+                            const unsigned long long old = atomicMin(&io->col1, pack);
+                            const unsigned long long later = old > pack ? old : pack;          // not the first meeting (so far)
+                            if (later != ~0ULL) {
+                                // its first decision is an ordinary pick; the batch ends before the second one -- unless the
+                                // two are so close that the shift could change their order
+                                const int32_t t0 = (int32_t)(later >> 52), t1 = (int32_t)((later >> 40) & 0xfffULL);
+                                const int32_t cut = (t1 - t0 > A.k + 2 ? t1 : t0) - A.k - 1;
+                                atomicMin(&io->limB, cut > 0 ? cut : 0);
+                            }
+                        }
                     }
                 }
                 ++rk;
@@ -1923,12 +1949,21 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         }
     }
     __syncthreads();
-    // the limits, capped by what the batch holds
-    const int32_t limF = io->limF < nFa ? io->limF : nFa, limL = io->limL < nL0 ? io->limL : nL0, limB = io->limB < B0 ? io->limB : B0;
-    {   // the largest x that respects the three limits, every thread trying four values
+    // the limits, capped by what is in sight; the first meeting of the two orders and who passes over its slot
+    const int32_t limF = io->limF < nFa ? io->limF : nFa, limL = io->limL < nEa ? io->limL : nEa, limB = io->limB < B0 ? io->limB : B0;
+    const unsigned long long col1 = io->col1;
+    const bool met = col1 != ~0ULL;
+    const int32_t skipF = met && ((col1 >> 30) & 1ULL) ? (int32_t)((col1 >> 16) & 0x3fffULL) : 0x7fffffff;     // oldest-first ranks from here on take the next slot
+    const int32_t skipL = met && !((col1 >> 30) & 1ULL) ? (int32_t)(col1 & 0xffffULL) : 0x7fffffff;            // longest-match ranks from here on take the next entry
+    auto hI = [&](int32_t t) -> int32_t { return t + (t >= skipF ? 1 : 0); };
+    auto eI = [&](int32_t u) -> int32_t { return u + (u >= skipL ? 1 : 0); };
+    {   // the largest x that respects the limits, every thread trying four values
         int32_t best = 0;
 #pragma unroll
-        for (int r = 1; r <= 4; ++r) { const int32_t x = tid * 4 + r; if (x <= limB && f(x) <= limF && x - f(x) <= limL) best = x; }
+        for (int r = 1; r <= 4; ++r) {
+            const int32_t x = tid * 4 + r, nf = f(x), nl = x - nf;
+            if (x <= limB && (nf == 0 || hI(nf - 1) < limF) && (nl == 0 || eI(nl - 1) < limL)) best = x;
+        }
         best = __reduce_max_sync(FULL_MASK, best);
         if ((tid & 31) == 0 && best > 0) atomicMax(&io->Bmax, best);
     }
@@ -1938,15 +1973,16 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     if (tid == 0) {
         const int32_t nF = f(B), nL = B - nF;
         io->B = B; io->Braw = Braw; io->B0out = B0;
-        io->consumed = nL > 0 ? sEpos[nL - 1] + 1 : 0;
-        io->hmax = nF > 0 ? sH[nF - 1] : -1;
-        // stopped by a decision only the one-at-a-time path can take (not by the end of the entries, nor by a slot both
-        // kinds of turn reach: the next batch sorts that out)
-        io->hard = B > 0 && B < B0 && (f(B + 1) > limF || B + 1 - f(B + 1) > limL) ? 1 : 0;
+        io->consumed = nL > 0 ? sEpos[eI(nL - 1)] + 1 : 0;
+        io->hmax = nF > 0 ? sH[hI(nF - 1)] : -1;
+        // stopped by a decision only the one-at-a-time path can take (not by the end of what is in sight, nor by a
+        // further slot both kinds of turn reach: the next batch sorts that out)
+        const int32_t nf1 = f(B + 1), nl1 = B + 1 - nf1;
+        io->hard = B > 0 && B < B0 && ((nf1 > 0 && hI(nf1 - 1) >= io->limF) || (nl1 > 0 && eI(nl1 - 1) >= io->limL)) ? 1 : 0;
     }
     for (int32_t x = tid; x < B; x += KLPM_FAST_THREADS) {   // thread makes decisions c + x
         const int32_t f0 = f(x);
-        const int32_t slot = f(x + 1) > f0 ? sH[f0] : sE[x - f0];
+        const int32_t slot = f(x + 1) > f0 ? sH[hI(f0)] : sE[eI(x - f0)];
         atomicOr(R.done + (slot >> 5), 1u << (slot & 31));
         atomicOr(R.skip + (slot >> 5), 1u << (slot & 31));
         A.order[c + x] = slot;
