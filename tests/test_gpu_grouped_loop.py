@@ -330,3 +330,23 @@ def test_queue_above_the_shared_memory_bitmaps(K):
     order, unc = outs[0][0].astype(np.int64), outs[0][1].astype(np.int64)
     assert np.array_equal(np.sort(order), np.arange(n))
     assert int(unc.sum()) == outs[0][3]["tokens"]
+
+
+@pytest.mark.parametrize("k", [2, 3, 4, 7, 40])
+def test_long_batches_where_the_two_pick_orders_meet(K, k):
+    """20,000 queries, everybody waiting, nobody grouped (every query ends its match with a token of its own), match
+    lengths unrelated to the arrival order: CTA-wide batches run long and the oldest-first picks keep meeting
+    list entries inside them -- once per batch (resolved inside the batch), several times (the batch ends before
+    the second), with the two decisions close together and far apart.  Compared with the oracle's schedule."""
+    n, trunks, depth = 20_000, 200, 60
+    rng = np.random.RandomState(900 + k)
+    trunk = rng.randint(0, 50000, size=(trunks, depth))
+    prefill = [trunk[r].tolist() for r in range(trunks)]
+    prompts = []
+    for i in range(n):
+        r, p = rng.randint(trunks), rng.randint(1, depth)
+        prompts.append(trunk[r, :p].tolist() + [50000 + i] + rng.randint(0, 50000, size=rng.randint(0, 3)).tolist())
+    arr = [0] * n
+    got = run_gpu(K, prefill, prompts, arr, 2, k)
+    want = run_oracle(prefill, prompts, arr, 2, k)
+    same(got, want)
