@@ -1724,7 +1724,10 @@ struct FastBatchIO {
     unsigned long long root;          // in: largest key in the tournament
     int32_t B, consumed, hmax;        // out: decisions made (0: none), list entries passed, last slot taken by an oldest-first turn
     int32_t B0, Bmax, limF, limL;     // scratch
-    unsigned long long col1;          // scratch: the first slot that both kinds of turn reach (decision, who is first, its two ranks)
+    // scratch: the slots both kinds of turn reach inside the batch (rank among the oldest-first picks, rank among the
+    // list entries), and after they are resolved the ranks each side passes over, ascending
+    int32_t ncol, nRH, nRE;
+    int32_t colPhi[32], colRk[32], remH[32], remE[32];
     int32_t B0out;                    // out: decisions the entries in sight would have allowed
     int32_t hard;                     // out: the batch stopped before a decision that needs the one-at-a-time path
     int32_t Braw;                     // out: decisions the batch could have made (it makes none below KLPM_FAST_CTA_MIN)
@@ -1830,7 +1833,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         }
     }
     // the limits start open; every thread reads them capped by what the batch can hold
-    if (tid == 0) { io->B0 = 0; io->Bmax = 0; io->limF = 0x7fffffff; io->limL = 0x7fffffff; io->limB = 0x7fffffff; io->col1 = ~0ULL; }
+    if (tid == 0) { io->B0 = 0; io->Bmax = 0; io->limF = 0x7fffffff; io->limL = 0x7fffffff; io->limB = 0x7fffffff; io->ncol = 0; io->nRH = 0; io->nRE = 0; }
     auto f = [&](int32_t x) -> int32_t { return sF[x]; };
     // those of the entries that still count
     int32_t cnt = 0;
@@ -1871,9 +1874,9 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     // One slot and one entry more than a full batch takes are looked at: where the two pick orders meet once inside the
     // batch (a slot that is both among the oldest unprocessed and among the next list entries), the side that comes
     // later passes over it and takes one more of its own.
-    const bool both_kinds = A.policy == KLPM_POLICY_KLPM;
-    const int32_t nFw = both_kinds && nF0 < KLPM_FAST_CTA_BATCH ? nF0 + 1 : nF0;
-    const int32_t nLw = both_kinds && nL0 < KLPM_FAST_CTA_BATCH ? nL0 + 1 : nL0;
+    const bool both_kinds = A.policy == KLPM_POLICY_KLPM && A.k >= 2;       // (k = 1: every turn is an oldest-first turn)
+    const int32_t nFw = both_kinds ? (nF0 + 32 < KLPM_FAST_CTA_BATCH ? nF0 + 32 : KLPM_FAST_CTA_BATCH) : nF0;
+    const int32_t nLw = both_kinds ? (nL0 + 32 < KLPM_FAST_CTA_BATCH ? nL0 + 32 : KLPM_FAST_CTA_BATCH) : nL0;
     const int32_t nFa = nfree < nFw ? nfree : nFw;          // oldest-first picks there are slots for
     const int32_t nEa = avail < nLw ? avail : nLw;          // longest-match picks there are entries for
     // the next nFa unprocessed slots in order: a thread per slot, eight words at a time; the slot's rank among the free
@@ -1921,26 +1924,18 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
                         else if (A.policy == KLPM_POLICY_LPM) { xF = B0; xL = rk; }
                         else {
                             const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;
-                            xF = i0 + phi * A.k;
+                            const long long xF64 = i0 + (long long)phi * A.k;
+                            xF = xF64 < 0x3ffffff ? (int32_t)xF64 : 0x3ffffff;
                             int32_t a0 = 0, a1 = B0;                     // smallest x with x + 1 - f(x + 1) > rk
                             while (a0 < a1) { const int32_t mid = (a0 + a1) >> 1; if (mid + 1 - f(mid + 1) > rk) a1 = mid; else a0 = mid + 1; }
                             xL = a0;
                         }
-                        if (!both_kinds) {
-                            atomicMin(&io->limB, xF > xL ? xF : xL);
-                        } else {
-                            const int32_t tmin = xF < xL ? xF : xL, tmax0 = xF < xL ? xL : xF, tmax = tmax0 < 4095 ? tmax0 : 4095;
-                            const unsigned long long pack = ((unsigned long long)tmin << 52) | ((unsigned long long)tmax << 40) |
-                                                            ((unsigned long long)(xL < xF ? 1 : 0) << 30) | ((unsigned long long)phi << 16) | (unsigned long long)rk;
-                            const unsigned long long old = atomicMin(&io->col1, pack);
-                            const unsigned long long later = old > pack ? old : pack;          // not the first meeting (so far)
-                            if (later != ~0ULL) {
-                                // its first decision is an ordinary pick; the batch ends before the second one -- unless the
-                                // two are so close that the shift could change their order
-                                const int32_t t0 = (int32_t)(later >> 52), t1 = (int32_t)((later >> 40) & 0xfffULL);
-                                const int32_t cut = (t1 - t0 > A.k + 2 ? t1 : t0) - A.k - 1;
-                                atomicMin(&io->limB, cut > 0 ? cut : 0);
-                            }
+                        // without resolving: the batch would have to end before the later of the two decisions (used
+                        // when there are more such slots than the resolution below takes)
+                        atomicMin(&io->limB, xF > xL ? xF : xL);
+                        if (both_kinds) {
+                            const int32_t ci = atomicAdd(&io->ncol, 1);
+                            if (ci < 32) { io->colPhi[ci] = phi; io->colRk[ci] = rk; }
                         }
                     }
                 }
@@ -1949,14 +1944,73 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
         }
     }
     __syncthreads();
-    // the limits, capped by what is in sight; the first meeting of the two orders and who passes over its slot
-    const int32_t limF = io->limF < nFa ? io->limF : nFa, limL = io->limL < nEa ? io->limL : nEa, limB = io->limB < B0 ? io->limB : B0;
-    const unsigned long long col1 = io->col1;
-    const bool met = col1 != ~0ULL;
-    const int32_t skipF = met && ((col1 >> 30) & 1ULL) ? (int32_t)((col1 >> 16) & 0x3fffULL) : 0x7fffffff;     // oldest-first ranks from here on take the next slot
-    const int32_t skipL = met && !((col1 >> 30) & 1ULL) ? (int32_t)(col1 & 0xffffULL) : 0x7fffffff;            // longest-match ranks from here on take the next entry
-    auto hI = [&](int32_t t) -> int32_t { return t + (t >= skipF ? 1 : 0); };
-    auto eI = [&](int32_t u) -> int32_t { return u + (u >= skipL ? 1 : 0); };
+    // Where the two orders meet, sequential processing gives the slot to whichever turn comes first, and the other side
+    // passes over it: its later picks move up by one.  Warp 0 plays the meetings through in the order of their first
+    // decision (lane i holds meeting i; the time at which a side reaches a slot is its rank minus the ranks below it
+    // that this side has passed over so far, turned into a decision number; the earliest pending decision is final,
+    // because whatever happens later moves later picks only).  Result: the ranks each side passes over, ascending.
+    const int32_t ncol = io->ncol;                          // (block-uniform)
+    const bool resolve = both_kinds && ncol > 0 && ncol <= 32;
+    if (resolve) {
+        if (tid < 32) {
+            const int lane = tid;
+            const bool mine = lane < ncol;
+            const int32_t phi = mine ? io->colPhi[lane] : 0x7fffffff, rk = mine ? io->colRk[lane] : 0x7fffffff;
+            unsigned belowPhi = 0, belowRk = 0;             // meetings with a smaller rank on either side
+            for (int j = 0; j < ncol; ++j) {
+                const int32_t pj = __shfl_sync(FULL_MASK, phi, j), rj = __shfl_sync(FULL_MASK, rk, j);
+                if (pj < phi) belowPhi |= 1u << j;
+                if (rj < rk) belowRk |= 1u << j;
+            }
+            const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;    // decisions before the first oldest-first turn
+            const long long FAR = 0x3ffffff;
+            // decision of the longest-match turn of rank u, of the oldest-first turn of rank t
+            auto l_turn = [&](int32_t u) -> long long {
+                if (u < i0) return u;
+                const int32_t u1 = u - i0, q = u1 / (A.k - 1);
+                return i0 + (long long)q * A.k + 1 + (u1 - q * (A.k - 1));
+            };
+            // no batch gets past the first slot or entry that needs the careful step, whoever passes over what
+            const int32_t capF = io->limF < nFa ? io->limF : nFa, capL = io->limL < nEa ? io->limL : nEa;
+            long long bcap = B0;
+            { const long long a1 = i0 + (long long)capF * A.k, a2 = l_turn(capL); if (a1 < bcap) bcap = a1; if (a2 < bcap) bcap = a2; }
+            long long xF = FAR, xL = FAR;
+            if (mine) { xF = i0 + (long long)phi * A.k; xL = l_turn(rk); if (xF > FAR) xF = FAR; }
+            unsigned remH = 0, remE = 0, open_ = ncol == 32 ? 0xffffffffu : ((1u << ncol) - 1u);
+            while (open_) {
+                unsigned key = 0xffffffffu;
+                const bool l_first = xL < xF;
+                if (mine && ((open_ >> lane) & 1u)) key = ((unsigned)(l_first ? xL : xF) << 5) | (unsigned)lane;
+                const unsigned win = __reduce_min_sync(FULL_MASK, key);
+                if ((long long)(win >> 5) >= bcap) break;   // beyond what the batch can reach: nothing more to settle
+                const int wl = (int)(win & 31u);
+                const bool wl_first = __shfl_sync(FULL_MASK, (int)l_first, wl) != 0;
+                open_ &= ~(1u << wl);
+                if (wl_first) {                             // a longest-match turn took that slot: later oldest-first picks come one turn earlier
+                    remH |= 1u << wl;
+                    if (((belowPhi >> wl) & 1u) && xF < FAR) xF -= A.k;
+                } else {                                    // an oldest-first turn took that entry's slot: later list picks come one turn earlier
+                    remE |= 1u << wl;
+                    if ((belowRk >> wl) & 1u) {
+                        long long y = xL - 1;
+                        if (y >= i0 && (y - i0) % A.k == 0) --y;       // (that one is an oldest-first turn)
+                        xL = y;
+                    }
+                }
+            }
+            if (mine && ((remH >> lane) & 1u)) io->remH[__popc(remH & belowPhi)] = phi;
+            if (mine && ((remE >> lane) & 1u)) io->remE[__popc(remE & belowRk)] = rk;
+            if (lane == 0) { io->nRH = __popc(remH); io->nRE = __popc(remE); }
+        }
+        __syncthreads();
+    }
+    // the limits, capped by what is in sight
+    const int32_t limF = io->limF < nFa ? io->limF : nFa, limL = io->limL < nEa ? io->limL : nEa;
+    const int32_t limB = resolve || io->limB > B0 ? B0 : io->limB;
+    const int32_t nRH = io->nRH, nRE = io->nRE;
+    // rank t among the oldest-first picks -> index of its slot in sH; rank u among the longest-match picks -> index in sE
+    auto hI = [&](int32_t t) -> int32_t { for (int32_t j = 0; j < nRH; ++j) { if (io->remH[j] <= t) ++t; else break; } return t; };
+    auto eI = [&](int32_t u) -> int32_t { for (int32_t j = 0; j < nRE; ++j) { if (io->remE[j] <= u) ++u; else break; } return u; };
     {   // the largest x that respects the limits, every thread trying four values
         int32_t best = 0;
 #pragma unroll
