@@ -1926,9 +1926,12 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
                             const int32_t i0 = cyc == 0 ? 0 : A.k - cyc;
                             const long long xF64 = i0 + (long long)phi * A.k;
                             xF = xF64 < 0x3ffffff ? (int32_t)xF64 : 0x3ffffff;
-                            int32_t a0 = 0, a1 = B0;                     // smallest x with x + 1 - f(x + 1) > rk
-                            while (a0 < a1) { const int32_t mid = (a0 + a1) >> 1; if (mid + 1 - f(mid + 1) > rk) a1 = mid; else a0 = mid + 1; }
-                            xL = a0;
+                            xL = rk;                                       // before the first oldest-first turn; after it k - 1 of every k decisions
+                            if (rk >= i0 && A.k >= 2) {
+                                const int32_t u1 = rk - i0, q = u1 / (A.k - 1);
+                                const long long xL64 = i0 + (long long)q * A.k + 1 + (u1 - q * (A.k - 1));
+                                xL = xL64 < 0x3ffffff ? (int32_t)xL64 : 0x3ffffff;
+                            }
                         }
                         // without resolving: the batch would have to end before the later of the two decisions (used
                         // when there are more such slots than the resolution below takes)
