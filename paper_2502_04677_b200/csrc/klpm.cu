@@ -1735,7 +1735,7 @@ struct FastBatchIO {
 };
 #define KLPM_FAST_CTA_BATCH 1024      // decisions per CTA-wide batch at most (4 list entries per thread)
 #ifndef KLPM_FAST_CTA_MIN
-#define KLPM_FAST_CTA_MIN 32         // smaller batches are left to the warp-wide step (an attempt costs about 16,000 cycles)
+#define KLPM_FAST_CTA_MIN 32         // smaller batches are left to the warp-wide step (an attempt costs about 10,000 cycles)
 #endif
 #ifndef KLPM_FAST_CB_MAX
 #define KLPM_FAST_CB_MAX 32           // longest back-off (loop iterations) after CTA-wide attempts that failed
