@@ -1728,7 +1728,6 @@ struct FastBatchIO {
     // list entries), and after they are resolved the ranks each side passes over, ascending
     int32_t ncol, nRH, nRE;
     int32_t colPhi[32], colRk[32], remH[32], remE[32];
-    int32_t B0out;                    // out: decisions the entries in sight would have allowed
     int32_t hard;                     // out: the batch stopped before a decision that needs the one-at-a-time path
     int32_t Braw;                     // out: decisions the batch could have made (it makes none below KLPM_FAST_CTA_MIN)
     int32_t limB;                     // scratch: the batch must end before this decision (list entries that an oldest-first pick would meet)
@@ -2029,7 +2028,7 @@ __device__ void fast_batch_job(const FastArgs& A, const FastTour& R0, FastBatchI
     const int32_t B = Braw >= KLPM_FAST_CTA_MIN ? Braw : 0;     // nothing is changed by a batch too short to pay
     if (tid == 0) {
         const int32_t nF = f(B), nL = B - nF;
-        io->B = B; io->Braw = Braw; io->B0out = B0;
+        io->B = B; io->Braw = Braw;
         io->consumed = nL > 0 ? sEpos[eI(nL - 1)] + 1 : 0;
         io->hmax = nF > 0 ? sH[hI(nF - 1)] : -1;
         // stopped by a decision only the one-at-a-time path can take (not by the end of what is in sight, nor by a
